@@ -1,0 +1,173 @@
+/*
+ * btc.h -- C interface of the B200 tensor-contraction library.
+ *
+ * One operation:   D := alpha * op(A) * op(B) + beta * op(C)
+ *
+ * A, B, C, D are dense tensors in a general strided layout (an element with indices
+ * i_0..i_{n-1} lives at base + sum_k i_k * stride_k; Glossary, "Strided layout").  Every mode
+ * carries an index label.  Labels shared by A and B only are contracted (summed); labels shared
+ * by one input and D are free and may appear in D in any order; labels shared by A, B and D are
+ * Hadamard (batch) labels (Sec. "Operations", Cases 1-2, Eq. (case1), Eq. (case2)).  A label may
+ * occur several times inside A or inside B (Case 3; such a tensor equals one with a single mode
+ * whose stride is the sum of the strides, Note 6).  op() optionally conjugates complex operands.
+ *
+ * The object model follows Sec. "Interface Components": a library handle, tensor descriptors
+ * that hold no data pointer, an operation descriptor that is validated and planned once, and an
+ * execute call that takes only data pointers, scalars and an executor (here: a CUDA stream).
+ * Every function returns an integer error code (0 = success; the other values are not part of
+ * the contract, use btc_explain_error); outputs are returned through pointers; destroy functions
+ * take the address of the handle and null it (Sec. "Error Handling").
+ *
+ * Threads: objects are immutable after creation except through btc_set_attr; executing one
+ * contraction object from several host threads is allowed when each call has its own workspace.
+ */
+#ifndef BTC_H_
+#define BTC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int btc_error_t;
+
+enum {
+    BTC_SUCCESS = 0,
+    BTC_ERR_INVALID_ARGUMENT = 1,    /* NULL where a value is required, bad rank, bad enum      */
+    BTC_ERR_INVALID_EXTENT = 2,      /* an extent < 1 (extents are positive integers)           */
+    BTC_ERR_EXTENT_MISMATCH = 3,     /* one label with two extents (test list item 26)          */
+    BTC_ERR_C_D_MISMATCH = 4,        /* C's rank, extents, strides or labels differ from D's    */
+    BTC_ERR_D_ALIASING = 5,          /* two index tuples of D address one element (item 28)     */
+    BTC_ERR_LABEL_ONLY_IN_D = 6,     /* a label of D in neither A nor B (Eq. (FreeD), Case 5)   */
+    BTC_ERR_NOT_SUPPORTED = 7,       /* mixed element types, label repeated inside D, Case 4    */
+    BTC_ERR_WORKSPACE_TOO_SMALL = 8,
+    BTC_ERR_MISALIGNED = 9,          /* a data pointer not aligned to its element size          */
+    BTC_ERR_CUDA = 10,               /* a CUDA runtime call failed                              */
+    BTC_ERR_DEVICE_TIMEOUT = 11,     /* a bounded device-side wait expired                      */
+    BTC_ERR_OUT_OF_MEMORY = 12
+};
+
+/* Element types.  Complex values are (re, im) pairs of the stated part width. */
+typedef enum {
+    BTC_F32 = 0,
+    BTC_F64 = 1,
+    BTC_C32 = 2, /* 2 x float  (8 bytes)  */
+    BTC_C64 = 3  /* 2 x double (16 bytes) */
+} btc_dtype_t;
+
+typedef struct btc_handle_s *btc_handle_t;            /* Sec. "The Library Handle"            */
+typedef struct btc_tensor_info_s *btc_tensor_info_t;  /* Sec. "Tensor Descriptors"            */
+typedef struct btc_contraction_s *btc_contraction_t;  /* Sec. "Tensor Operation Descriptors"  */
+typedef struct btc_status_s *btc_status_t;            /* Sec. "Status Objects"                */
+
+#define BTC_MAX_RANK 32
+#define BTC_MAX_LABELS 64
+
+/* Library handle (Sec. "The Library Handle").  Binds the CUDA device that is current on the
+ * calling thread; every object made from it lives on that device.  Host memory only. */
+btc_error_t btc_create_handle(btc_handle_t *out);
+btc_error_t btc_destroy_handle(btc_handle_t *handle); /* *handle becomes NULL */
+
+/* Tensor descriptor (Sec. "Tensor Descriptors"): rank, extents, strides, element type; no data.
+ *   rank      0..BTC_MAX_RANK; rank 0 is a scalar (Note 2, Note 4)
+ *   extents   host array of `rank` entries, each >= 1; may be NULL iff rank == 0
+ *   strides   host array of `rank` entries in ELEMENTS, signed, zero allowed; NULL means dense
+ *             column-major (stride_0 = 1, stride_k = prod_{l<k} extent_l; Glossary)
+ * The arrays are copied.  Errors: INVALID_ARGUMENT, INVALID_EXTENT. */
+btc_error_t btc_create_tensor_info(btc_handle_t handle, btc_dtype_t dtype, int32_t rank,
+                                   const int64_t *extents, const int64_t *strides,
+                                   btc_tensor_info_t *out);
+btc_error_t btc_destroy_tensor_info(btc_tensor_info_t *info);
+
+/* Operation descriptor (Sec. "Tensor Operation Descriptors"; the checks of Sec. "Algorithm
+ * Structure", first paragraph; label classification of Sec. "Operations").
+ *   A, B, D     tensor descriptors (copied; they may be destroyed or reused afterwards)
+ *   C           descriptor of C, or NULL when the operation never reads C (then beta must be 0
+ *               at every execute).  C must have D's rank, extents, strides and label order
+ *               (Note 5).
+ *   labelsX     host array, one int64 label per mode of X (any values); NULL iff rank 0
+ *   conjX       non-zero: op(X) = element-wise complex conjugate; ignored for real types
+ *   alpha,beta  host scalars of D's element type stored as the defaults of the operation;
+ *               NULL means alpha = 1, beta = 0
+ * All validation and planning (label classes, mode fusion, kernel and tile choice, device-side
+ * offset tables) happens here; the call may allocate device memory and copy small tables with
+ * the default stream.  Errors: INVALID_ARGUMENT, EXTENT_MISMATCH, C_D_MISMATCH, D_ALIASING,
+ * LABEL_ONLY_IN_D, NOT_SUPPORTED, OUT_OF_MEMORY, CUDA. */
+btc_error_t btc_create_contraction(btc_handle_t handle,
+                                   btc_tensor_info_t A, const int64_t *labelsA, int conjA,
+                                   btc_tensor_info_t B, const int64_t *labelsB, int conjB,
+                                   btc_tensor_info_t C, const int64_t *labelsC, int conjC,
+                                   btc_tensor_info_t D, const int64_t *labelsD,
+                                   const void *alpha, const void *beta,
+                                   btc_contraction_t *out);
+btc_error_t btc_destroy_contraction(btc_contraction_t *op);
+
+/* Bytes of device workspace btc_execute needs for this operation (0 for most plans; split-K
+ * plans keep their partial sums there).  Alignment required: 256 bytes. */
+btc_error_t btc_contraction_workspace_size(btc_contraction_t op, size_t *bytes);
+
+/* Key-value access on an operation (Sec. "Virtual Key-Value Stores").  Values are host memory. */
+enum {
+    BTC_ATTR_KERNEL = 1,      /* int32, read/write: BTC_KERNEL_* (write re-plans)              */
+    BTC_ATTR_SPLIT_K = 2,     /* int32, read/write: number of K slices (>= 1)                  */
+    BTC_ATTR_TILE = 3,        /* int32[3], read: CTA tile extents M, N, K                      */
+    BTC_ATTR_GROUPS = 4,      /* int64[4], read: batch, M, N, K sizes after classification     */
+    BTC_ATTR_GRID = 5,        /* int32[3], read: launch grid                                   */
+    BTC_ATTR_NUM_MODES = 6,   /* int32[4], read: modes per class after fusion (batch, M, N, K) */
+    BTC_ATTR_SWAPPED = 7      /* int32, read: 1 when A and B exchanged roles                   */
+};
+enum {
+    BTC_KERNEL_AUTO = 0,
+    BTC_KERNEL_GENERIC = 1,   /* one thread per element of D, any legal input                  */
+    BTC_KERNEL_TILED = 2      /* shared-memory tiled contraction kernel                        */
+};
+btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, size_t len);
+btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t len, size_t *needed);
+
+/* Execute (Sec. "Execution"): enqueue the operation on a stream and return.
+ *   cuda_stream  a cudaStream_t passed as void*; NULL is the default stream (the "default
+ *                executor" of Sec. "Executors")
+ *   alpha, beta  HOST pointers to scalars of D's element type, or NULL for the stored defaults.
+ *                beta == 0: C is not read (may be NULL); alpha == 0: A and B are not read.
+ *   A, B, C, D   DEVICE pointers to the logical element (0,...,0) of each tensor, aligned to the
+ *                element size.  C == D (same pointer) is the in-place update.  Any other overlap
+ *                of D with A, B or C is undefined.  The caller owns all buffers.
+ *   workspace    DEVICE pointer, 256-byte aligned, at least btc_contraction_workspace_size bytes
+ *                (may be NULL when that size is 0)
+ *   status       NULL, or receives a new status object describing the launch (destroy it)
+ * The call never allocates device memory and never synchronises.  Errors: INVALID_ARGUMENT,
+ * MISALIGNED, WORKSPACE_TOO_SMALL, CUDA (launch failure). */
+btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream,
+                        const void *alpha, const void *A, const void *B,
+                        const void *beta, const void *C, void *D,
+                        void *workspace, size_t workspace_bytes,
+                        btc_status_t *status);
+
+/* Convenience for callers whose buffers live in HOST memory: copies A, B (and C when beta != 0)
+ * to device buffers it allocates, executes, copies D back, frees, and synchronises the stream.
+ * Pointers address logical element (0,...,0) of host tensors laid out as the descriptors say;
+ * each tensor's whole strided span is transferred.  Errors as btc_execute plus OUT_OF_MEMORY. */
+btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream,
+                             const void *alpha, const void *A, const void *B,
+                             const void *beta, const void *C, void *D);
+
+/* Status object (Sec. "Status Objects"): metadata of one execute call. */
+enum {
+    BTC_STATUS_KERNEL = 1,    /* int32: BTC_KERNEL_* that ran                 */
+    BTC_STATUS_LAUNCHES = 2,  /* int32: kernels enqueued by the call          */
+    BTC_STATUS_GRID = 3,      /* int32[3]                                      */
+    BTC_STATUS_SPLIT_K = 4    /* int32                                         */
+};
+btc_error_t btc_status_get(btc_status_t status, int32_t key, void *value, size_t len);
+btc_error_t btc_destroy_status(btc_status_t *status);
+
+/* Text for an error code (the strerror analogue of Sec. "Error Handling").  Writes at most `len`
+ * bytes including the terminator; *needed (if not NULL) receives the full length. */
+btc_error_t btc_explain_error(btc_error_t code, char *buf, size_t len, size_t *needed);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BTC_H_ */

@@ -1,0 +1,600 @@
+// C-ABI entry points of the contraction library (declared in include/btc.h): object management,
+// tile/split-K choice and kernel launches.  No compute happens on the host.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/btc.h"
+#include "generic_kernel.cuh"
+#include "kernel_params.h"
+#include "plan.h"
+#include "tiled_f64_kernel.cuh"
+
+using namespace btc;
+
+struct btc_handle_s {
+    int device = -1;       // -1: no CUDA device (objects can be validated and planned, not run)
+    int sm_count = 148;
+};
+
+struct btc_tensor_info_s {
+    TensorDesc desc;
+};
+
+struct btc_status_s {
+    int32_t kernel = 0, launches = 0, split_k = 1;
+    int32_t grid[3] = {0, 0, 0};
+};
+
+struct btc_contraction_s {
+    btc_handle_s handle;
+    PlanRequest req;
+    Plan plan;
+    double alpha[2] = {1.0, 0.0}, beta[2] = {0.0, 0.0};
+    // device copies of the plan's tables (one allocation)
+    int64_t *d_tables = nullptr;
+    const int64_t *d_offA_m = nullptr, *d_offD_m = nullptr, *d_offB_n = nullptr, *d_offD_n = nullptr,
+                  *d_offA_k = nullptr, *d_offB_k = nullptr, *d_offA_h = nullptr, *d_offB_h = nullptr,
+                  *d_offD_h = nullptr;
+    int32_t tiles_m = 0, tiles_n = 0, raster_n_fast = 0;
+    int64_t k_per_split = 0;
+    size_t workspace_bytes = 0;
+    int32_t grid[3] = {0, 0, 0};
+};
+
+namespace {
+
+// ---- tiled kernel variants -------------------------------------------------------------------
+using F64Big = F64Tile<false, 128, 128, 2, 4, 4>;
+using F64Small = F64Tile<false, 64, 64, 2, 2, 4>;
+using C64Big = F64Tile<true, 128, 64, 2, 4, 4>;
+using C64Small = F64Tile<true, 64, 32, 2, 2, 4>;
+
+struct VariantInfo {
+    int bm, bn, bk, threads, acc;
+    size_t smem;
+};
+template <typename T> VariantInfo info_of() { return {T::BM, T::BN, T::BK, T::THREADS, T::ACC, T::SMEM_BYTES}; }
+
+bool tiled_supported(btc_dtype_t t) { return t == BTC_F64 || t == BTC_C64; }
+
+VariantInfo variant_info(btc_dtype_t t, int variant)
+{
+    if (t == BTC_F64) return variant == 0 ? info_of<F64Big>() : info_of<F64Small>();
+    return variant == 0 ? info_of<C64Big>() : info_of<C64Small>();
+}
+
+template <typename T>
+cudaError_t launch_tiled(const TiledParams &p, int64_t ctas, int64_t reduce_ctas, cudaStream_t st)
+{
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(tiled_f64_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             int(T::SMEM_BYTES));
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    tiled_f64_kernel<T><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (p.split_k > 1) {
+        tiled_f64_splitk_reduce_kernel<T><<<unsigned(reduce_ctas), T::THREADS, 0, st>>>(p);
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+void to_double2(btc_dtype_t t, const void *src, double out[2])
+{
+    switch (t) {
+    case BTC_F32: out[0] = *static_cast<const float *>(src); out[1] = 0; break;
+    case BTC_F64: out[0] = *static_cast<const double *>(src); out[1] = 0; break;
+    case BTC_C32: out[0] = static_cast<const float *>(src)[0]; out[1] = static_cast<const float *>(src)[1]; break;
+    case BTC_C64: out[0] = static_cast<const double *>(src)[0]; out[1] = static_cast<const double *>(src)[1]; break;
+    }
+}
+
+void free_tables(btc_contraction_s *op)
+{
+    if (op->d_tables) cudaFree(op->d_tables);
+    op->d_tables = nullptr;
+}
+
+// Choose tile variant, raster order and split-K for a tiled plan; upload the offset tables.
+int finish_plan(btc_contraction_s *op)
+{
+    Plan &pl = op->plan;
+    free_tables(op);
+    op->workspace_bytes = 0;
+    if (pl.kernel == BTC_KERNEL_TILED && !tiled_supported(pl.dtype)) {
+        if (op->req.force_kernel == BTC_KERNEL_TILED) return BTC_ERR_NOT_SUPPORTED;
+        pl.kernel = BTC_KERNEL_GENERIC;
+    }
+    if (pl.kernel == BTC_KERNEL_GENERIC) {
+        if (pl.batch.size() + pl.m.size() + pl.n.size() > size_t(kGenericMaxD) || pl.k.size() > size_t(kGenericMaxK))
+            return BTC_ERR_NOT_SUPPORTED;
+        const double total = double(pl.Bt) * double(pl.M) * double(pl.N);
+        const bool warp_per_elem = total < 4096.0 * 8 && pl.K >= 64;
+        const int64_t groups = pl.Bt * pl.M * pl.N;
+        const int64_t threads = warp_per_elem ? groups * 32 : groups;
+        int64_t blocks = (threads + 255) / 256;
+        const int64_t cap = int64_t(op->handle.sm_count) * 32;
+        if (blocks > cap) blocks = cap;
+        if (blocks < 1) blocks = 1;
+        op->grid[0] = int32_t(blocks); op->grid[1] = warp_per_elem ? 32 : 1; op->grid[2] = 1;
+        pl.tile = TileConfig();
+        pl.split_k = 1;
+        return BTC_SUCCESS;
+    }
+
+    const int sms = op->handle.sm_count;
+    auto tiles_for = [&](const VariantInfo &v) {
+        return ((pl.M + v.bm - 1) / v.bm) * ((pl.N + v.bn - 1) / v.bn) * pl.Bt;
+    };
+    int variant = 0;
+    if (double(tiles_for(variant_info(pl.dtype, 0))) < 0.8 * sms) variant = 1;
+    const VariantInfo v = variant_info(pl.dtype, variant);
+    pl.tile.bm = v.bm; pl.tile.bn = v.bn; pl.tile.bk = v.bk; pl.tile.threads = v.threads;
+    pl.tile.stages = 4; pl.tile.variant = variant;
+    op->tiles_m = int32_t((pl.M + v.bm - 1) / v.bm);
+    op->tiles_n = int32_t((pl.N + v.bn - 1) / v.bn);
+    op->raster_n_fast = op->tiles_n <= op->tiles_m ? 1 : 0;
+    const int64_t tiles = tiles_for(v);
+    const int64_t k_tiles = (pl.K + v.bk - 1) / v.bk;
+    int64_t split = 1;
+    if (op->req.force_split_k > 0) {
+        split = op->req.force_split_k;
+    } else if (tiles < sms) {
+        split = (2 * int64_t(sms)) / tiles;
+        const int64_t max_split = k_tiles / 2;   // at least two K tiles per slice
+        if (split > max_split) split = max_split;
+    }
+    if (split > k_tiles) split = k_tiles;
+    if (split < 1) split = 1;
+    int64_t kt_per = (k_tiles + split - 1) / split;
+    split = (k_tiles + kt_per - 1) / kt_per;     // no empty slices
+    pl.split_k = int32_t(split);
+    op->k_per_split = kt_per * v.bk;
+    if (tiles * split > 0x7fffffffLL) return BTC_ERR_NOT_SUPPORTED;
+    op->grid[0] = int32_t(tiles * split); op->grid[1] = 1; op->grid[2] = 1;
+    if (split > 1)
+        op->workspace_bytes = size_t(tiles) * size_t(split) * size_t(v.threads) * size_t(v.acc) * sizeof(double);
+
+    if (op->handle.device >= 0) {
+        const std::vector<int64_t> *tabs[9] = {&pl.offA_m, &pl.offD_m, &pl.offB_n, &pl.offD_n, &pl.offA_k,
+                                               &pl.offB_k, &pl.offA_h, &pl.offB_h, &pl.offD_h};
+        const int64_t **dst[9] = {&op->d_offA_m, &op->d_offD_m, &op->d_offB_n, &op->d_offD_n, &op->d_offA_k,
+                                  &op->d_offB_k, &op->d_offA_h, &op->d_offB_h, &op->d_offD_h};
+        size_t total = 0;
+        for (auto *t : tabs) total += (t->size() + 31) / 32 * 32;   // keep every table 256-byte aligned
+        std::vector<int64_t> host(total, 0);
+        size_t pos = 0, starts[9];
+        for (int i = 0; i < 9; ++i) {
+            starts[i] = pos;
+            std::memcpy(host.data() + pos, tabs[i]->data(), tabs[i]->size() * sizeof(int64_t));
+            pos += (tabs[i]->size() + 31) / 32 * 32;
+        }
+        if (cudaMalloc(reinterpret_cast<void **>(&op->d_tables), total * sizeof(int64_t)) != cudaSuccess) {
+            cudaGetLastError();
+            op->d_tables = nullptr;
+            return BTC_ERR_OUT_OF_MEMORY;
+        }
+        if (cudaMemcpy(op->d_tables, host.data(), total * sizeof(int64_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError();
+            return BTC_ERR_CUDA;
+        }
+        for (int i = 0; i < 9; ++i) *dst[i] = op->d_tables + starts[i];
+    }
+    return BTC_SUCCESS;
+}
+
+int replan(btc_contraction_s *op)
+{
+    op->req.sm_count = op->handle.sm_count;
+    int rc = make_plan(op->req, op->plan);
+    if (rc != BTC_SUCCESS) return rc;
+    return finish_plan(op);
+}
+
+bool is_zero(const double v[2]) { return v[0] == 0.0 && v[1] == 0.0; }
+
+template <typename R, bool CPLX>
+cudaError_t launch_generic(const GenericParams &gp, int blocks, bool warp_per_elem, cudaStream_t st)
+{
+    if (warp_per_elem) generic_contract_kernel<R, CPLX, 32><<<blocks, 256, 0, st>>>(gp);
+    else generic_contract_kernel<R, CPLX, 1><<<blocks, 256, 0, st>>>(gp);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// =================================================================================== C ABI
+extern "C" {
+
+btc_error_t btc_create_handle(btc_handle_t *out)
+{
+    if (!out) return BTC_ERR_INVALID_ARGUMENT;
+    btc_handle_s *h = new (std::nothrow) btc_handle_s;
+    if (!h) return BTC_ERR_OUT_OF_MEMORY;
+    int dev = -1;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) {
+            h->device = dev;
+            h->sm_count = sms;
+        }
+    }
+    cudaGetLastError();   // a machine without a GPU still gets a handle that can validate and plan
+    *out = h;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_destroy_handle(btc_handle_t *handle)
+{
+    if (!handle) return BTC_ERR_INVALID_ARGUMENT;
+    delete *handle;
+    *handle = nullptr;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_create_tensor_info(btc_handle_t handle, btc_dtype_t dtype, int32_t rank, const int64_t *extents,
+                                   const int64_t *strides, btc_tensor_info_t *out)
+{
+    if (!handle || !out) return BTC_ERR_INVALID_ARGUMENT;
+    if (rank < 0 || rank > BTC_MAX_RANK) return BTC_ERR_INVALID_ARGUMENT;
+    if (int(dtype) < 0 || int(dtype) > int(BTC_C64)) return BTC_ERR_INVALID_ARGUMENT;
+    if (rank > 0 && !extents) return BTC_ERR_INVALID_ARGUMENT;
+    for (int i = 0; i < rank; ++i)
+        if (extents[i] < 1) return BTC_ERR_INVALID_EXTENT;
+    btc_tensor_info_s *t = new (std::nothrow) btc_tensor_info_s;
+    if (!t) return BTC_ERR_OUT_OF_MEMORY;
+    t->desc.dtype = dtype;
+    t->desc.extent.assign(extents, extents + rank);
+    if (strides) {
+        t->desc.stride.assign(strides, strides + rank);
+    } else {
+        int64_t s = 1;
+        for (int i = 0; i < rank; ++i) {
+            t->desc.stride.push_back(s);
+            s *= extents[i];
+        }
+    }
+    *out = t;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_destroy_tensor_info(btc_tensor_info_t *info)
+{
+    if (!info) return BTC_ERR_INVALID_ARGUMENT;
+    delete *info;
+    *info = nullptr;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_create_contraction(btc_handle_t handle, btc_tensor_info_t A, const int64_t *labelsA, int conjA,
+                                   btc_tensor_info_t B, const int64_t *labelsB, int conjB, btc_tensor_info_t C,
+                                   const int64_t *labelsC, int conjC, btc_tensor_info_t D, const int64_t *labelsD,
+                                   const void *alpha, const void *beta, btc_contraction_t *out)
+{
+    if (!handle || !A || !B || !D || !out) return BTC_ERR_INVALID_ARGUMENT;
+    if ((!labelsA && !A->desc.extent.empty()) || (!labelsB && !B->desc.extent.empty()) ||
+        (!labelsD && !D->desc.extent.empty()) || (C && !labelsC && !C->desc.extent.empty()))
+        return BTC_ERR_INVALID_ARGUMENT;
+    btc_contraction_s *op = new (std::nothrow) btc_contraction_s;
+    if (!op) return BTC_ERR_OUT_OF_MEMORY;
+    op->handle = *handle;
+    op->req.A = A->desc;
+    op->req.B = B->desc;
+    op->req.D = D->desc;
+    op->req.labelsA.assign(labelsA, labelsA + A->desc.extent.size());
+    op->req.labelsB.assign(labelsB, labelsB + B->desc.extent.size());
+    op->req.labelsD.assign(labelsD, labelsD + D->desc.extent.size());
+    op->req.has_c = C != nullptr;
+    if (C) {
+        op->req.C = C->desc;
+        op->req.labelsC.assign(labelsC, labelsC + C->desc.extent.size());
+    }
+    op->req.conjA = conjA != 0;
+    op->req.conjB = conjB != 0;
+    op->req.conjC = conjC != 0;
+    if (alpha) to_double2(D->desc.dtype, alpha, op->alpha);
+    if (beta) to_double2(D->desc.dtype, beta, op->beta);
+    if (!C && !is_zero(op->beta)) {
+        delete op;
+        return BTC_ERR_INVALID_ARGUMENT;
+    }
+    const int rc = replan(op);
+    if (rc != BTC_SUCCESS) {
+        free_tables(op);
+        delete op;
+        return rc;
+    }
+    if (std::getenv("BTC_LOG")) std::fprintf(stderr, "[btc] %s\n", op->plan.describe().c_str());
+    *out = op;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_destroy_contraction(btc_contraction_t *op)
+{
+    if (!op) return BTC_ERR_INVALID_ARGUMENT;
+    if (*op) {
+        free_tables(*op);
+        delete *op;
+    }
+    *op = nullptr;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_contraction_workspace_size(btc_contraction_t op, size_t *bytes)
+{
+    if (!op || !bytes) return BTC_ERR_INVALID_ARGUMENT;
+    *bytes = op->workspace_bytes;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, size_t len)
+{
+    if (!op || !value) return BTC_ERR_INVALID_ARGUMENT;
+    if (len != sizeof(int32_t)) return BTC_ERR_INVALID_ARGUMENT;
+    int32_t v;
+    std::memcpy(&v, value, sizeof v);
+    const PlanRequest saved = op->req;
+    if (key == BTC_ATTR_KERNEL) {
+        if (v < BTC_KERNEL_AUTO || v > BTC_KERNEL_TILED) return BTC_ERR_INVALID_ARGUMENT;
+        op->req.force_kernel = v;
+    } else if (key == BTC_ATTR_SPLIT_K) {
+        if (v < 0) return BTC_ERR_INVALID_ARGUMENT;
+        op->req.force_split_k = v;
+    } else {
+        return BTC_ERR_INVALID_ARGUMENT;
+    }
+    int rc = replan(op);
+    if (rc != BTC_SUCCESS) {   // keep the object usable with its previous plan
+        op->req = saved;
+        replan(op);
+    }
+    return rc;
+}
+
+btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t len, size_t *needed)
+{
+    if (!op) return BTC_ERR_INVALID_ARGUMENT;
+    int32_t i32[4];
+    int64_t i64[4];
+    const void *src = i32;
+    size_t n = 0;
+    const Plan &pl = op->plan;
+    switch (key) {
+    case BTC_ATTR_KERNEL: i32[0] = pl.kernel; n = 4; break;
+    case BTC_ATTR_SPLIT_K: i32[0] = pl.split_k; n = 4; break;
+    case BTC_ATTR_TILE: i32[0] = pl.tile.bm; i32[1] = pl.tile.bn; i32[2] = pl.tile.bk; n = 12; break;
+    case BTC_ATTR_GROUPS: i64[0] = pl.Bt; i64[1] = pl.M; i64[2] = pl.N; i64[3] = pl.K; src = i64; n = 32; break;
+    case BTC_ATTR_GRID: i32[0] = op->grid[0]; i32[1] = op->grid[1]; i32[2] = op->grid[2]; n = 12; break;
+    case BTC_ATTR_NUM_MODES:
+        i32[0] = int32_t(pl.batch.size()); i32[1] = int32_t(pl.m.size());
+        i32[2] = int32_t(pl.n.size()); i32[3] = int32_t(pl.k.size()); n = 16; break;
+    case BTC_ATTR_SWAPPED: i32[0] = pl.swapped ? 1 : 0; n = 4; break;
+    default: return BTC_ERR_INVALID_ARGUMENT;
+    }
+    if (needed) *needed = n;
+    if (!value) return needed ? BTC_SUCCESS : BTC_ERR_INVALID_ARGUMENT;
+    if (len < n) return BTC_ERR_INVALID_ARGUMENT;
+    std::memcpy(value, src, n);
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A, const void *B,
+                        const void *beta, const void *C, void *D, void *workspace, size_t workspace_bytes,
+                        btc_status_t *status)
+{
+    if (!op || !D) return BTC_ERR_INVALID_ARGUMENT;
+    if (op->handle.device < 0) return BTC_ERR_CUDA;   // no device: nothing can run, and nothing else will
+    const Plan &pl = op->plan;
+    double al[2] = {op->alpha[0], op->alpha[1]}, be[2] = {op->beta[0], op->beta[1]};
+    if (alpha) to_double2(pl.dtype, alpha, al);
+    if (beta) to_double2(pl.dtype, beta, be);
+    const bool use_ab = !is_zero(al), use_c = !is_zero(be);
+    if (use_ab && (!A || !B)) return BTC_ERR_INVALID_ARGUMENT;
+    if (use_c && (!C || !pl.has_c_desc)) return BTC_ERR_INVALID_ARGUMENT;
+    const size_t part = dtype_is_complex(pl.dtype) ? dtype_size(pl.dtype) / 2 : dtype_size(pl.dtype);
+    auto misaligned = [&](const void *p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) != 0; };
+    // complex128 accesses are 16-byte wide; everything else needs its element alignment
+    const size_t need = pl.dtype == BTC_C64 ? 16 : (pl.dtype == BTC_C32 ? 8 : part);
+    if (misaligned(A, need) || misaligned(B, need) || misaligned(C, need) || misaligned(D, need))
+        return BTC_ERR_MISALIGNED;
+    if (op->workspace_bytes > 0) {
+        if (!workspace || workspace_bytes < op->workspace_bytes) return BTC_ERR_WORKSPACE_TOO_SMALL;
+        if (misaligned(workspace, 256)) return BTC_ERR_MISALIGNED;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const void *pA = pl.swapped ? B : A, *pB = pl.swapped ? A : B;
+    int launches = 0;
+    cudaError_t ce = cudaSuccess;
+
+    if (pl.kernel == BTC_KERNEL_GENERIC || !use_ab) {
+        GenericParams gp;
+        std::memset(&gp, 0, sizeof gp);
+        gp.A = pA; gp.B = pB; gp.C = C; gp.D = D;
+        int nd = 0;
+        for (auto *g : {&pl.batch, &pl.m, &pl.n})
+            for (auto &md : *g) {
+                gp.ext_d[nd] = md.extent; gp.sA_d[nd] = md.sA; gp.sB_d[nd] = md.sB; gp.sD_d[nd] = md.sD;
+                ++nd;
+            }
+        if (nd > kGenericMaxD || pl.k.size() > size_t(kGenericMaxK)) return BTC_ERR_NOT_SUPPORTED;
+        gp.nd = nd;
+        gp.nk = int32_t(pl.k.size());
+        for (int i = 0; i < gp.nk; ++i) {
+            gp.ext_k[i] = pl.k[size_t(i)].extent; gp.sA_k[i] = pl.k[size_t(i)].sA; gp.sB_k[i] = pl.k[size_t(i)].sB;
+        }
+        gp.total_d = pl.Bt * pl.M * pl.N;
+        gp.total_k = pl.K;
+        gp.alpha[0] = al[0]; gp.alpha[1] = al[1]; gp.beta[0] = be[0]; gp.beta[1] = be[1];
+        gp.conjA = pl.conjA; gp.conjB = pl.conjB; gp.conjC = pl.conjC;
+        gp.use_ab = use_ab; gp.use_c = use_c;
+        bool wpe = pl.kernel == BTC_KERNEL_GENERIC && op->grid[1] == 32;
+        int blocks = op->grid[0];
+        if (pl.kernel != BTC_KERNEL_GENERIC) {   // alpha == 0 on a tiled plan: D = beta * op(C)
+            int64_t b = (gp.total_d + 255) / 256, cap = int64_t(op->handle.sm_count) * 32;
+            blocks = int(b < cap ? (b < 1 ? 1 : b) : cap);
+        }
+        switch (pl.dtype) {
+        case BTC_F32: ce = launch_generic<float, false>(gp, blocks, wpe, st); break;
+        case BTC_F64: ce = launch_generic<double, false>(gp, blocks, wpe, st); break;
+        case BTC_C32: ce = launch_generic<float, true>(gp, blocks, wpe, st); break;
+        case BTC_C64: ce = launch_generic<double, true>(gp, blocks, wpe, st); break;
+        }
+        launches = 1;
+    } else {
+        TiledParams tp;
+        std::memset(&tp, 0, sizeof tp);
+        tp.A = pA; tp.B = pB; tp.C = C; tp.D = D;
+        tp.offA_m = op->d_offA_m; tp.offD_m = op->d_offD_m; tp.offB_n = op->d_offB_n; tp.offD_n = op->d_offD_n;
+        tp.offA_k = op->d_offA_k; tp.offB_k = op->d_offB_k;
+        tp.offA_h = op->d_offA_h; tp.offB_h = op->d_offB_h; tp.offD_h = op->d_offD_h;
+        tp.M = pl.M; tp.N = pl.N; tp.K = pl.K; tp.Bt = pl.Bt;
+        tp.tiles_m = op->tiles_m; tp.tiles_n = op->tiles_n; tp.raster_n_fast = op->raster_n_fast;
+        tp.split_k = pl.split_k; tp.k_per_split = op->k_per_split;
+        tp.dirA = int32_t(pl.dirA); tp.dirB = int32_t(pl.dirB);
+        // vector copies need the base pointers aligned as well
+        tp.vecA = misaligned(pA, size_t(pl.alignA)) ? 1 : pl.vecA;
+        tp.vecB = misaligned(pB, size_t(pl.alignB)) ? 1 : pl.vecB;
+        tp.conjA = pl.conjA; tp.conjB = pl.conjB; tp.conjC = pl.conjC;
+        tp.use_c = use_c;
+        tp.alpha[0] = al[0]; tp.alpha[1] = al[1]; tp.beta[0] = be[0]; tp.beta[1] = be[1];
+        tp.partials = workspace;
+        const int64_t ctas = op->grid[0];
+        const int64_t reduce_ctas = ctas / pl.split_k;
+        if (pl.dtype == BTC_F64)
+            ce = pl.tile.variant == 0 ? launch_tiled<F64Big>(tp, ctas, reduce_ctas, st)
+                                      : launch_tiled<F64Small>(tp, ctas, reduce_ctas, st);
+        else
+            ce = pl.tile.variant == 0 ? launch_tiled<C64Big>(tp, ctas, reduce_ctas, st)
+                                      : launch_tiled<C64Small>(tp, ctas, reduce_ctas, st);
+        launches = pl.split_k > 1 ? 2 : 1;
+    }
+    if (ce != cudaSuccess) return BTC_ERR_CUDA;
+    if (status) {
+        btc_status_s *s = new (std::nothrow) btc_status_s;
+        if (!s) return BTC_ERR_OUT_OF_MEMORY;
+        s->kernel = use_ab ? pl.kernel : BTC_KERNEL_GENERIC;
+        s->launches = launches;
+        s->split_k = pl.split_k;
+        s->grid[0] = op->grid[0]; s->grid[1] = op->grid[1]; s->grid[2] = op->grid[2];
+        *status = s;
+    }
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A,
+                             const void *B, const void *beta, const void *C, void *D)
+{
+    if (!op || !D) return BTC_ERR_INVALID_ARGUMENT;
+    if (op->handle.device < 0) return BTC_ERR_CUDA;
+    const Plan &pl = op->plan;
+    const size_t esz = dtype_size(pl.dtype);
+    double al[2] = {op->alpha[0], op->alpha[1]}, be[2] = {op->beta[0], op->beta[1]};
+    if (alpha) to_double2(pl.dtype, alpha, al);
+    if (beta) to_double2(pl.dtype, beta, be);
+    const bool use_ab = !is_zero(al), use_c = !is_zero(be);
+    if ((use_ab && (!A || !B)) || (use_c && !C)) return BTC_ERR_INVALID_ARGUMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    struct Buf {
+        char *dev = nullptr;
+        int64_t lo = 0, hi = 0;
+        size_t bytes() const { return size_t(hi - lo + 1); }
+    } bA, bB, bC, bD;
+    auto span_bytes = [&](Buf &b, int64_t lo, int64_t hi) { b.lo = lo * int64_t(esz); b.hi = hi * int64_t(esz) + int64_t(esz) - 1; };
+    span_bytes(bA, pl.spanA_lo, pl.spanA_hi);
+    span_bytes(bB, pl.spanB_lo, pl.spanB_hi);
+    span_bytes(bD, pl.spanD_lo, pl.spanD_hi);
+    bC = bD;
+    const bool c_is_d = use_c && C == D;
+    void *ws = nullptr;
+    btc_error_t rc = BTC_SUCCESS;
+    auto fail = [&](btc_error_t e) { if (rc == BTC_SUCCESS) rc = e; };
+    auto up = [&](Buf &b, const void *host) {
+        if (rc != BTC_SUCCESS) return;
+        // 256-byte aligned allocation; the span's first byte keeps the host pointer's offset
+        // relative to 16 bytes so that alignment-dependent choices match device-resident use
+        if (cudaMalloc(reinterpret_cast<void **>(&b.dev), b.bytes()) != cudaSuccess) { cudaGetLastError(); b.dev = nullptr; fail(BTC_ERR_OUT_OF_MEMORY); return; }
+        if (host && cudaMemcpyAsync(b.dev, static_cast<const char *>(host) + b.lo, b.bytes(), cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
+    };
+    if (use_ab) { up(bA, A); up(bB, B); }
+    up(bD, D);   // D's span travels both ways so that padding between its elements is preserved
+    if (use_c && !c_is_d) up(bC, C);
+    if (rc == BTC_SUCCESS && op->workspace_bytes > 0 &&
+        cudaMalloc(&ws, op->workspace_bytes) != cudaSuccess) { cudaGetLastError(); ws = nullptr; fail(BTC_ERR_OUT_OF_MEMORY); }
+    if (rc == BTC_SUCCESS) {
+        const void *dA = use_ab ? bA.dev - bA.lo : nullptr, *dB = use_ab ? bB.dev - bB.lo : nullptr;
+        void *dD = bD.dev - bD.lo;
+        const void *dC = use_c ? (c_is_d ? dD : static_cast<void *>(bC.dev - bC.lo)) : nullptr;
+        rc = btc_execute(op, cuda_stream, alpha, dA, dB, beta, dC, dD, ws, op->workspace_bytes, nullptr);
+    }
+    if (rc == BTC_SUCCESS &&
+        cudaMemcpyAsync(static_cast<char *>(D) + bD.lo, bD.dev, bD.bytes(), cudaMemcpyDeviceToHost, st) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
+    for (Buf *b : {&bA, &bB, &bD}) if (b->dev) cudaFree(b->dev);
+    if (use_c && !c_is_d && bC.dev) cudaFree(bC.dev);
+    if (ws) cudaFree(ws);
+    return rc;
+}
+
+btc_error_t btc_status_get(btc_status_t status, int32_t key, void *value, size_t len)
+{
+    if (!status || !value) return BTC_ERR_INVALID_ARGUMENT;
+    switch (key) {
+    case BTC_STATUS_KERNEL: if (len < 4) return BTC_ERR_INVALID_ARGUMENT; std::memcpy(value, &status->kernel, 4); break;
+    case BTC_STATUS_LAUNCHES: if (len < 4) return BTC_ERR_INVALID_ARGUMENT; std::memcpy(value, &status->launches, 4); break;
+    case BTC_STATUS_GRID: if (len < 12) return BTC_ERR_INVALID_ARGUMENT; std::memcpy(value, status->grid, 12); break;
+    case BTC_STATUS_SPLIT_K: if (len < 4) return BTC_ERR_INVALID_ARGUMENT; std::memcpy(value, &status->split_k, 4); break;
+    default: return BTC_ERR_INVALID_ARGUMENT;
+    }
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_destroy_status(btc_status_t *status)
+{
+    if (!status) return BTC_ERR_INVALID_ARGUMENT;
+    delete *status;
+    *status = nullptr;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_explain_error(btc_error_t code, char *buf, size_t len, size_t *needed)
+{
+    const char *msg = "unknown error code";
+    switch (code) {
+    case BTC_SUCCESS: msg = "success"; break;
+    case BTC_ERR_INVALID_ARGUMENT: msg = "invalid argument (NULL where a value is required, bad rank, key or enum)"; break;
+    case BTC_ERR_INVALID_EXTENT: msg = "an extent is smaller than 1"; break;
+    case BTC_ERR_EXTENT_MISMATCH: msg = "modes that share a label have different extents"; break;
+    case BTC_ERR_C_D_MISMATCH: msg = "C does not have D's rank, extents, strides and labels"; break;
+    case BTC_ERR_D_ALIASING: msg = "two index tuples of D address the same element"; break;
+    case BTC_ERR_LABEL_ONLY_IN_D: msg = "a label of D occurs in neither A nor B"; break;
+    case BTC_ERR_NOT_SUPPORTED: msg = "operation not supported (mixed element types, label repeated inside D, or size limits)"; break;
+    case BTC_ERR_WORKSPACE_TOO_SMALL: msg = "workspace missing or smaller than btc_contraction_workspace_size"; break;
+    case BTC_ERR_MISALIGNED: msg = "a data pointer is not aligned to its element size (workspace: 256 bytes)"; break;
+    case BTC_ERR_CUDA: msg = "a CUDA runtime call failed or no CUDA device is available"; break;
+    case BTC_ERR_DEVICE_TIMEOUT: msg = "a bounded device-side wait expired"; break;
+    case BTC_ERR_OUT_OF_MEMORY: msg = "out of memory"; break;
+    default: break;
+    }
+    const size_t n = std::strlen(msg) + 1;
+    if (needed) *needed = n;
+    if (buf && len > 0) {
+        const size_t c = n < len ? n : len;
+        std::memcpy(buf, msg, c);
+        buf[c - 1] = '\0';
+    }
+    return BTC_SUCCESS;
+}
+
+}  // extern "C"

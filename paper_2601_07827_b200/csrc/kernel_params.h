@@ -1,0 +1,45 @@
+// Parameter blocks shared by the host launchers and the device kernels.
+#pragma once
+
+#include <cstdint>
+
+namespace btc {
+
+constexpr int kGenericMaxD = 32;   // loop dimensions over D (batch + free), after merging
+constexpr int kGenericMaxK = 64;   // summed loop dimensions
+
+// One thread (or one warp) per element of D; used for every input the tiled kernels decline.
+struct GenericParams {
+    const void *A, *B, *C;
+    void *D;
+    int32_t nd, nk;
+    int64_t total_d, total_k;
+    int64_t ext_d[kGenericMaxD], sA_d[kGenericMaxD], sB_d[kGenericMaxD], sD_d[kGenericMaxD];
+    int64_t ext_k[kGenericMaxK], sA_k[kGenericMaxK], sB_k[kGenericMaxK];
+    double alpha[2], beta[2];
+    int32_t conjA, conjB, conjC;
+    int32_t use_ab, use_c;
+};
+
+// Tiled contraction kernels.  All offsets are in elements of the operation's dtype.
+struct TiledParams {
+    const void *A, *B, *C;
+    void *D;
+    const int64_t *offA_m, *offD_m;   // [M]
+    const int64_t *offB_n, *offD_n;   // [N]
+    const int64_t *offA_k, *offB_k;   // [K]
+    const int64_t *offA_h, *offB_h, *offD_h;   // [Bt]
+    int64_t M, N, K, Bt;
+    int32_t tiles_m, tiles_n;
+    int32_t raster_n_fast;            // 1: consecutive CTAs walk the n tiles of one m tile
+    int32_t split_k;
+    int64_t k_per_split;              // multiple of the K tile
+    int32_t dirA, dirB;               // 0: threads run along the free index, 1: along k
+    int32_t vecA, vecB;               // elements per global->shared copy
+    int32_t conjA, conjB, conjC;
+    int32_t use_c;
+    double alpha[2], beta[2];
+    void *partials;                   // split-K scratch (workspace), or nullptr
+};
+
+}  // namespace btc

@@ -1,0 +1,353 @@
+// Planner implementation; see plan.h.
+#include "plan.h"
+
+#include <algorithm>
+#include <cstdlib>
+#include <sstream>
+
+namespace btc {
+
+size_t dtype_size(btc_dtype_t t)
+{
+    switch (t) {
+    case BTC_F32: return 4;
+    case BTC_F64: return 8;
+    case BTC_C32: return 8;
+    case BTC_C64: return 16;
+    }
+    return 0;
+}
+
+bool dtype_is_complex(btc_dtype_t t) { return t == BTC_C32 || t == BTC_C64; }
+
+namespace {
+
+inline int64_t iabs(int64_t x) { return x < 0 ? -x : x; }
+
+struct LabelRow {
+    int64_t label = 0, extent = 0;
+    int64_t sA = 0, sB = 0, sD = 0;
+    bool inA = false, inB = false, inD = false;
+};
+
+int find_label(const std::vector<LabelRow> &rows, int64_t label)
+{
+    for (size_t i = 0; i < rows.size(); ++i)
+        if (rows[i].label == label) return int(i);
+    return -1;
+}
+
+// Sufficient test that no two index tuples of D address the same element: with the modes of
+// extent > 1 sorted by |stride|, every stride must exceed the span of all smaller ones.
+bool d_may_alias(const TensorDesc &D)
+{
+    std::vector<std::pair<int64_t, int64_t>> se;
+    for (size_t i = 0; i < D.extent.size(); ++i)
+        if (D.extent[i] > 1) {
+            if (D.stride[i] == 0) return true;
+            se.emplace_back(iabs(D.stride[i]), D.extent[i]);
+        }
+    std::sort(se.begin(), se.end());
+    int64_t span = 0;
+    for (auto &p : se) {
+        if (p.first < 1 + span) return true;
+        span += p.first * (p.second - 1);
+    }
+    return false;
+}
+
+// Merge loop dimensions whose strides chain in every tensor: y follows x when
+// stride_y == stride_x * extent_x for A, B and D alike.
+void fuse_modes(std::vector<Mode> &g)
+{
+    bool changed = true;
+    while (changed) {
+        changed = false;
+        for (size_t x = 0; x < g.size() && !changed; ++x)
+            for (size_t y = 0; y < g.size() && !changed; ++y) {
+                if (x == y) continue;
+                if (g[y].sA == g[x].sA * g[x].extent && g[y].sB == g[x].sB * g[x].extent &&
+                    g[y].sD == g[x].sD * g[x].extent) {
+                    g[x].extent *= g[y].extent;
+                    g.erase(g.begin() + y);
+                    changed = true;
+                }
+            }
+    }
+}
+
+int64_t product(const std::vector<Mode> &g)
+{
+    int64_t p = 1;
+    for (auto &m : g) p *= m.extent;
+    return p;
+}
+
+// offsets of all index tuples of `g`, first mode fastest
+template <typename F>
+std::vector<int64_t> build_table(const std::vector<Mode> &g, F stride_of)
+{
+    std::vector<int64_t> t(1, 0);
+    for (auto &md : g) {
+        const int64_t s = stride_of(md);
+        const size_t len = t.size();
+        t.resize(len * size_t(md.extent));
+        for (int64_t i = 1; i < md.extent; ++i)
+            for (size_t j = 0; j < len; ++j) t[size_t(i) * len + j] = t[j] + i * s;
+    }
+    return t;
+}
+
+void span_of(const TensorDesc &t, int64_t &lo, int64_t &hi)
+{
+    lo = hi = 0;
+    for (size_t i = 0; i < t.extent.size(); ++i) {
+        const int64_t d = t.stride[i] * (t.extent[i] - 1);
+        if (d < 0) lo += d; else hi += d;
+    }
+}
+
+// Split mode `idx` of `g` into an inner part of extent f (a divisor of its extent, f > 1) that
+// stays at `idx`, and an outer part appended at the end.
+void split_mode(std::vector<Mode> &g, size_t idx, int64_t f)
+{
+    Mode outer = g[idx];
+    outer.extent = g[idx].extent / f;
+    outer.sA = g[idx].sA * f;
+    outer.sB = g[idx].sB * f;
+    outer.sD = g[idx].sD * f;
+    g[idx].extent = f;
+    if (outer.extent > 1) g.push_back(outer);
+}
+
+int64_t largest_divisor_at_most(int64_t n, int64_t cap)
+{
+    for (int64_t f = std::min(n, cap); f >= 1; --f)
+        if (n % f == 0) return f;
+    return 1;
+}
+
+}  // namespace
+
+int make_plan(const PlanRequest &req, Plan &plan)
+{
+    const TensorDesc *T[3] = {&req.A, &req.B, &req.D};
+    const std::vector<int64_t> *L[3] = {&req.labelsA, &req.labelsB, &req.labelsD};
+
+    // ---- checks (Sec. "Algorithm Structure"; test list items 26-28; Eq. (FreeD)) ----
+    for (int t = 0; t < 3; ++t) {
+        if (T[t]->extent.size() > BTC_MAX_RANK) return BTC_ERR_INVALID_ARGUMENT;
+        if (T[t]->extent.size() != T[t]->stride.size() || T[t]->extent.size() != L[t]->size())
+            return BTC_ERR_INVALID_ARGUMENT;
+        for (int64_t e : T[t]->extent)
+            if (e < 1) return BTC_ERR_INVALID_EXTENT;
+    }
+    if (req.A.dtype != req.D.dtype || req.B.dtype != req.D.dtype ||
+        (req.has_c && req.C.dtype != req.D.dtype))
+        return BTC_ERR_NOT_SUPPORTED;
+    for (size_t i = 0; i < req.labelsD.size(); ++i)
+        for (size_t j = 0; j < i; ++j)
+            if (req.labelsD[i] == req.labelsD[j]) return BTC_ERR_NOT_SUPPORTED;
+
+    std::vector<LabelRow> rows;
+    for (int t = 0; t < 3; ++t)
+        for (size_t i = 0; i < L[t]->size(); ++i) {
+            int k = find_label(rows, (*L[t])[i]);
+            if (k < 0) {
+                if (rows.size() == BTC_MAX_LABELS) return BTC_ERR_INVALID_ARGUMENT;
+                LabelRow r;
+                r.label = (*L[t])[i];
+                r.extent = T[t]->extent[i];
+                rows.push_back(r);
+                k = int(rows.size()) - 1;
+            } else if (rows[k].extent != T[t]->extent[i]) {
+                return BTC_ERR_EXTENT_MISMATCH;
+            }
+            // a repeated label acts as one mode whose stride is the sum (Note 6)
+            if (t == 0) { rows[k].sA += T[t]->stride[i]; rows[k].inA = true; }
+            if (t == 1) { rows[k].sB += T[t]->stride[i]; rows[k].inB = true; }
+            if (t == 2) { rows[k].sD += T[t]->stride[i]; rows[k].inD = true; }
+        }
+    for (auto &r : rows)
+        if (r.inD && !r.inA && !r.inB) return BTC_ERR_LABEL_ONLY_IN_D;
+    if (req.has_c) {
+        if (req.C.extent.size() != req.D.extent.size() || req.labelsC.size() != req.labelsD.size())
+            return BTC_ERR_C_D_MISMATCH;
+        for (size_t i = 0; i < req.D.extent.size(); ++i)
+            if (req.C.extent[i] != req.D.extent[i] || req.C.stride[i] != req.D.stride[i] ||
+                req.labelsC[i] != req.labelsD[i])
+                return BTC_ERR_C_D_MISMATCH;
+    }
+    if (d_may_alias(req.D)) return BTC_ERR_D_ALIASING;
+
+    // ---- classify (Sec. "Operations": H, F_A, F_B, P; I_A / I_B of Case 4) ----
+    plan = Plan();
+    plan.dtype = req.D.dtype;
+    plan.conjA = req.conjA && dtype_is_complex(plan.dtype);
+    plan.conjB = req.conjB && dtype_is_complex(plan.dtype);
+    plan.conjC = req.conjC && dtype_is_complex(plan.dtype);
+    plan.has_c_desc = req.has_c;
+    for (auto &r : rows) {
+        if (r.extent == 1) continue;  // contributes no loop and no offset
+        Mode md;
+        md.extent = r.extent;
+        md.sA = r.sA; md.sB = r.sB; md.sD = r.sD;
+        if (r.inA && r.inB && r.inD) plan.batch.push_back(md);
+        else if (r.inA && r.inD) plan.m.push_back(md);
+        else if (r.inB && r.inD) plan.n.push_back(md);
+        else if (r.inA && r.inB) plan.k.push_back(md);
+        else { plan.k.push_back(md); plan.has_isolated = true; }  // summed; stride 0 elsewhere
+    }
+    span_of(req.A, plan.spanA_lo, plan.spanA_hi);
+    span_of(req.B, plan.spanB_lo, plan.spanB_hi);
+    span_of(req.D, plan.spanD_lo, plan.spanD_hi);
+
+    // ---- fuse modes that are contiguous in every tensor that carries them ----
+    fuse_modes(plan.batch);
+    fuse_modes(plan.m);
+    fuse_modes(plan.n);
+    fuse_modes(plan.k);
+
+    // ---- roles: D's smallest-stride free mode goes to the M side (commutativity) ----
+    {
+        int64_t bestM = INT64_MAX, bestN = INT64_MAX;
+        for (auto &md : plan.m) bestM = std::min(bestM, iabs(md.sD));
+        for (auto &md : plan.n) bestN = std::min(bestN, iabs(md.sD));
+        bool swap = bestN < bestM;
+        if (plan.m.empty() && !plan.n.empty()) swap = true;
+        if (swap) {
+            std::swap(plan.m, plan.n);
+            for (auto *g : {&plan.batch, &plan.m, &plan.n, &plan.k})
+                for (auto &md : *g) std::swap(md.sA, md.sB);
+            std::swap(plan.conjA, plan.conjB);
+            plan.swapped = true;
+        }
+    }
+
+    // ---- loop order: D decides the order of the free and batch modes ----
+    auto by_sD = [](const Mode &x, const Mode &y) { return iabs(x.sD) < iabs(y.sD); };
+    std::stable_sort(plan.m.begin(), plan.m.end(), by_sD);
+    std::stable_sort(plan.n.begin(), plan.n.end(), by_sD);
+    std::stable_sort(plan.batch.begin(), plan.batch.end(), by_sD);
+
+    // which direction of each input tile is closest to contiguous in memory
+    auto min_k_stride = [&](bool forA, int &where) {
+        int64_t best = INT64_MAX;
+        where = -1;
+        for (size_t i = 0; i < plan.k.size(); ++i) {
+            const int64_t s = iabs(forA ? plan.k[i].sA : plan.k[i].sB);
+            if (s < best) { best = s; where = int(i); }
+        }
+        return best;
+    };
+    int kA = -1, kB = -1;
+    const int64_t minKA = min_k_stride(true, kA), minKB = min_k_stride(false, kB);
+    const int64_t freeA = plan.m.empty() ? INT64_MAX : iabs(plan.m[0].sA);
+    const int64_t freeB = plan.n.empty() ? INT64_MAX : iabs(plan.n[0].sB);
+    plan.dirA = (freeA <= minKA) ? LoadDir::ALONG_FREE : LoadDir::ALONG_K;
+    plan.dirB = (freeB <= minKB) ? LoadDir::ALONG_FREE : LoadDir::ALONG_K;
+
+    // contracted modes: the mode an input wants to run along comes first; when A and B want
+    // different ones both are split so that a K tile holds a small box of each
+    {
+        const bool needA = plan.dirA == LoadDir::ALONG_K, needB = plan.dirB == LoadDir::ALONG_K;
+        std::vector<Mode> ordered;
+        std::vector<Mode> rest = plan.k;
+        auto take = [&](int idx) { ordered.push_back(rest[size_t(idx)]); rest.erase(rest.begin() + idx); };
+        if (needA && needB && kA != kB) {
+            const int64_t fa = largest_divisor_at_most(rest[size_t(kA)].extent, 4);
+            const int64_t fb = largest_divisor_at_most(rest[size_t(kB)].extent, 4);
+            if (fa > 1 && fb > 1) {
+                split_mode(rest, size_t(kA), fa);
+                split_mode(rest, size_t(kB), fb);
+            }
+            take(kA);
+            take(kB > kA ? kB - 1 : kB);
+        } else if (needA) {
+            take(kA);
+        } else if (needB) {
+            take(kB);
+        }
+        const bool sortA = needA || !needB;
+        std::stable_sort(rest.begin(), rest.end(), [&](const Mode &x, const Mode &y) {
+            return sortA ? iabs(x.sA) < iabs(y.sA) : iabs(x.sB) < iabs(y.sB);
+        });
+        ordered.insert(ordered.end(), rest.begin(), rest.end());
+        plan.k = ordered;
+    }
+
+    plan.Bt = product(plan.batch);
+    plan.M = product(plan.m);
+    plan.N = product(plan.n);
+    plan.K = product(plan.k);
+
+    // ---- vector width the strides allow for each input (elements per 16-byte load) ----
+    const int64_t esz = int64_t(dtype_size(plan.dtype));
+    auto vec_for = [&](bool forA, LoadDir dir) -> int32_t {
+        const std::vector<Mode> &fastg = (dir == LoadDir::ALONG_FREE) ? (forA ? plan.m : plan.n) : plan.k;
+        if (fastg.empty()) return 1;
+        auto S = [&](const Mode &md) { return forA ? md.sA : md.sB; };
+        for (int64_t v = 16 / esz; v > 1; v /= 2) {
+            bool ok = S(fastg[0]) == 1 && fastg[0].extent % v == 0;
+            auto others_ok = [&](const std::vector<Mode> &g, size_t from) {
+                for (size_t i = from; i < g.size(); ++i)
+                    if (S(g[i]) % v) return false;
+                return true;
+            };
+            const std::vector<Mode> &freeg = forA ? plan.m : plan.n;
+            ok = ok && others_ok(freeg, dir == LoadDir::ALONG_FREE ? 1 : 0);
+            ok = ok && others_ok(plan.k, dir == LoadDir::ALONG_K ? 1 : 0);
+            ok = ok && others_ok(plan.batch, 0);
+            if (ok) return int32_t(v);
+        }
+        return 1;
+    };
+    plan.vecA = vec_for(true, plan.dirA);
+    plan.vecB = vec_for(false, plan.dirB);
+    plan.alignA = plan.vecA * esz;
+    plan.alignB = plan.vecB * esz;
+    plan.vecD = (!plan.m.empty() && plan.m[0].sD == 1) ? 1 : 0;
+
+    // ---- kernel choice ----
+    const int64_t entries = 2 * (plan.M + plan.N + plan.K) + 3 * plan.Bt;
+    const bool tiled_ok = !plan.has_isolated && entries <= kMaxTableEntries;
+    plan.kernel = BTC_KERNEL_GENERIC;
+    if (req.force_kernel == BTC_KERNEL_TILED && !tiled_ok) return BTC_ERR_NOT_SUPPORTED;
+    if (req.force_kernel == BTC_KERNEL_TILED ||
+        (req.force_kernel == BTC_KERNEL_AUTO && tiled_ok &&
+         double(plan.M) * double(plan.N) * double(plan.K) * double(plan.Bt) >= 32768.0))
+        plan.kernel = BTC_KERNEL_TILED;
+
+    if (plan.kernel == BTC_KERNEL_TILED) {
+        plan.offA_m = build_table(plan.m, [](const Mode &md) { return md.sA; });
+        plan.offD_m = build_table(plan.m, [](const Mode &md) { return md.sD; });
+        plan.offB_n = build_table(plan.n, [](const Mode &md) { return md.sB; });
+        plan.offD_n = build_table(plan.n, [](const Mode &md) { return md.sD; });
+        plan.offA_k = build_table(plan.k, [](const Mode &md) { return md.sA; });
+        plan.offB_k = build_table(plan.k, [](const Mode &md) { return md.sB; });
+        plan.offA_h = build_table(plan.batch, [](const Mode &md) { return md.sA; });
+        plan.offB_h = build_table(plan.batch, [](const Mode &md) { return md.sB; });
+        plan.offD_h = build_table(plan.batch, [](const Mode &md) { return md.sD; });
+    }
+    plan.split_k = 1;
+    return BTC_SUCCESS;
+}
+
+std::string Plan::describe() const
+{
+    std::ostringstream o;
+    auto dump = [&](const char *name, const std::vector<Mode> &g) {
+        o << name << "[";
+        for (auto &md : g) o << "(" << md.extent << ":" << md.sA << "," << md.sB << "," << md.sD << ")";
+        o << "] ";
+    };
+    o << "dtype=" << int(dtype) << " swapped=" << swapped << " Bt=" << Bt << " M=" << M << " N=" << N
+      << " K=" << K << " ";
+    dump("H", batch); dump("M", m); dump("N", n); dump("K", k);
+    o << "kernel=" << kernel << " tile=" << tile.bm << "x" << tile.bn << "x" << tile.bk
+      << " splitK=" << split_k << " dirA=" << int(dirA) << " dirB=" << int(dirB) << " vecA=" << vecA
+      << " vecB=" << vecB;
+    return o.str();
+}
+
+}  // namespace btc

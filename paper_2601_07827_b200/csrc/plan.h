@@ -1,0 +1,88 @@
+// Host-side planner of the contraction library: validation, label classification, repeated-label
+// merge, mode fusion, operand role choice, loop ordering and offset tables.
+//
+// Follows Sec. "Operations" (label classes H, F_A, F_B, P; Cases 1-4), Note 6 (repeated labels
+// add their strides) and the checks listed in Sec. "Algorithm Structure".  Everything here is
+// integer work that runs once per operation object.
+#pragma once
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "../../include/btc.h"
+
+namespace btc {
+
+struct TensorDesc {
+    btc_dtype_t dtype = BTC_F64;
+    std::vector<int64_t> extent, stride;
+};
+
+// One loop dimension after merging/fusing: its extent and its element stride in each tensor
+// (0 where the tensor does not carry it).  After a role swap "A" means the operand that plays
+// the M side.
+struct Mode {
+    int64_t extent = 1;
+    int64_t sA = 0, sB = 0, sD = 0;
+};
+
+enum class LoadDir : int32_t { ALONG_FREE = 0, ALONG_K = 1 };
+
+struct TileConfig {
+    int32_t bm = 0, bn = 0, bk = 0;   // CTA tile in elements of the operation's dtype
+    int32_t threads = 0;
+    int32_t stages = 0;
+    int32_t variant = 0;              // index into the kernel table
+};
+
+struct Plan {
+    btc_dtype_t dtype = BTC_F64;
+    bool conjA = false, conjB = false, conjC = false;  // in planned roles (after swap)
+    bool swapped = false;        // true: the caller's B is the plan's A
+    bool has_c_desc = false;
+    bool has_isolated = false;   // Case 4 labels present (summed inside the generic kernel)
+
+    // loop dimensions in planned order, first entry fastest in the linearised index
+    std::vector<Mode> batch, m, n, k;
+    int64_t Bt = 1, M = 1, N = 1, K = 1;
+
+    // tile-kernel decisions
+    int32_t kernel = BTC_KERNEL_GENERIC;
+    TileConfig tile;
+    int32_t split_k = 1;
+    LoadDir dirA = LoadDir::ALONG_FREE, dirB = LoadDir::ALONG_FREE;
+    int32_t vecA = 1, vecB = 1;          // elements per global load that the strides allow
+    int32_t vecD = 1;                    // consecutive m that are consecutive in D (0/1 flag use)
+    int64_t alignA = 1, alignB = 1;      // required base-pointer alignment (bytes) for vecA / vecB
+
+    // element-offset tables (host copies; the API object uploads them)
+    std::vector<int64_t> offA_m, offD_m, offB_n, offD_n, offA_k, offB_k, offA_h, offB_h, offD_h;
+
+    // memory span of each caller-side tensor in elements relative to its base pointer
+    int64_t spanA_lo = 0, spanA_hi = 0, spanB_lo = 0, spanB_hi = 0, spanD_lo = 0, spanD_hi = 0;
+
+    std::string describe() const;
+};
+
+struct PlanRequest {
+    TensorDesc A, B, C, D;
+    bool has_c = false;
+    std::vector<int64_t> labelsA, labelsB, labelsC, labelsD;
+    bool conjA = false, conjB = false, conjC = false;
+    int32_t force_kernel = BTC_KERNEL_AUTO;
+    int32_t force_split_k = 0;   // 0 = choose
+    int32_t sm_count = 148;
+};
+
+// Validates the request and fills `plan`.  Returns a btc_error_t.
+int make_plan(const PlanRequest &req, Plan &plan);
+
+size_t dtype_size(btc_dtype_t t);
+bool dtype_is_complex(btc_dtype_t t);
+
+// Largest total number of table entries the tiled kernels accept before the planner falls back
+// to the generic kernel.
+constexpr int64_t kMaxTableEntries = int64_t(1) << 26;
+
+}  // namespace btc

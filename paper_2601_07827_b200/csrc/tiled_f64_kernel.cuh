@@ -1,0 +1,344 @@
+// Transpose-free tiled contraction kernel for fp64 and complex128 on sm_100a.
+//
+// The three linearised indices m (free labels of A), n (free labels of B) and k (contracted
+// labels) address memory through per-index offset tables, so a CTA gathers a BM x BK tile of
+// op(A) and a BK x BN tile of op(B) straight from the strided tensors into shared memory with
+// cp.async (16-byte copies where the strides allow, element copies otherwise), in whichever
+// direction is closest to contiguous for that operand, and keeps that orientation in shared
+// memory: the FP64 tensor-core fragments (mma.sync m8n8k4, one 8-byte word per lane) can be read
+// from either orientation without bank conflicts, so no transpose is ever materialised.
+//
+// Complex128 runs on the same real MMAs: an interleaved (re, im) row of A is a real row of
+// twice the length, and each complex b expands at fragment-load time into the 2x2 real block
+// [[br, sb*bi], [-sa*sb*bi, sa*br]] (sa, sb = -1 when that operand is conjugated), which gives
+// exactly 8 real flops per complex multiply-add.  An 8x8 accumulator fragment then holds
+// 8 rows x 4 complex columns with (re, im) adjacent in one lane.
+//
+// K is pipelined through STAGES shared-memory buffers.  With split-K each CTA handles one slice
+// of k and stores raw accumulators to scratch; a second kernel adds the slices in a fixed order
+// and applies alpha/beta, so results do not depend on scheduling.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "kernel_params.h"
+
+namespace btc {
+
+template <bool CPLX_, int BM_, int BN_, int WARPS_M_, int WARPS_N_, int STAGES_>
+struct F64Tile {
+    static constexpr bool CPLX = CPLX_;
+    static constexpr int BM = BM_;                    // rows of the CTA tile (elements)
+    static constexpr int BN = BN_;                    // columns of the CTA tile (elements)
+    static constexpr int BK = CPLX_ ? 8 : 16;         // k extent of one stage (elements)
+    static constexpr int W = CPLX_ ? 2 : 1;           // 8-byte words per element
+    static constexpr int WARPS_M = WARPS_M_, WARPS_N = WARPS_N_;
+    static constexpr int THREADS = 32 * WARPS_M_ * WARPS_N_;
+    static constexpr int STAGES = STAGES_;
+    static constexpr int WM = BM / WARPS_M;           // warp tile rows
+    static constexpr int WNR = BN * W / WARPS_N;      // warp tile columns in real words
+    static constexpr int FM = WM / 8, FN = WNR / 8;   // 8x8 fragments per warp
+    static constexpr int ACC = FM * FN * 2;           // doubles per thread
+    // shared-memory pitches (elements): conflict-free fragment reads need
+    //   real:    pitch = 4 (mod 16);   complex: pitch = 4 (mod 8) along the free index,
+    //                                           pitch = 2 (mod 8) along k
+    static constexpr int PITCH_FREE_A = BM + 4, PITCH_FREE_B = BN + 4;
+    static constexpr int PITCH_K = CPLX_ ? BK + 2 : BK + 4;
+    static constexpr int A_ELEMS = (BK * PITCH_FREE_A > BM * PITCH_K) ? BK * PITCH_FREE_A : BM * PITCH_K;
+    static constexpr int B_ELEMS = (BK * PITCH_FREE_B > BN * PITCH_K) ? BK * PITCH_FREE_B : BN * PITCH_K;
+    static constexpr int STAGE_WORDS = (A_ELEMS + B_ELEMS) * W;
+    static constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * 8 + size_t(2 * BM + 2 * BN) * 8;
+};
+
+__device__ __forceinline__ int64_t imin64(int64_t a, int64_t b) { return a < b ? a : b; }
+
+__device__ __forceinline__ void cp_async_bytes(void *smem_dst, const void *gsrc, int bytes, bool valid)
+{
+    const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
+    const int src = valid ? bytes : 0;   // src-size 0 zero-fills the destination
+    if (bytes == 16)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
+    else if (bytes == 8)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
+    else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void dmma_m8n8k4(double &c0, double &c1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
+}
+
+// Gather one ROWS x BK tile (rows = free index, columns = k) into shared memory.
+//   row_off   shared array: element offset of each tile row (batch offset included)
+//   koff      global table of k offsets;  [k_begin, k_end) is this CTA's valid k range
+//   dir       0: consecutive threads take consecutive rows; 1: consecutive k
+//   vec       elements per copy along that direction (1 or 16 / sizeof(element))
+//   s_row, s_k  shared-memory strides of the tile in elements
+template <int ROWS, int BK, int THREADS, int ELEM_BYTES>
+__device__ __forceinline__ void gather_tile(char *smem, const char *__restrict__ g,
+                                            const int64_t *row_off, const int64_t *__restrict__ koff,
+                                            int rows_valid, int64_t k0, int64_t k_end,
+                                            int dir, int vec, int s_row, int s_k, int tid)
+{
+    const int nfast = (dir == 0 ? ROWS : BK) / vec;
+    const int slots = ROWS * BK / vec;
+    const int bytes = vec * ELEM_BYTES;
+    for (int s = tid; s < slots; s += THREADS) {
+        const int f = (s % nfast) * vec, o = s / nfast;
+        const int r = dir == 0 ? f : o;
+        const int k = dir == 0 ? o : f;
+        const bool valid = (r < rows_valid) && (k0 + k < k_end);
+        const int64_t off = valid ? row_off[r] + __ldg(koff + k0 + k) : 0;
+        cp_async_bytes(smem + size_t(r * s_row + k * s_k) * ELEM_BYTES, g + off * ELEM_BYTES, bytes, valid);
+    }
+}
+
+// alpha * acc + beta * op(c) for one element, written through D's offsets
+template <bool CPLX>
+__device__ __forceinline__ void store_element(const TiledParams &p, int64_t off, double acc_r, double acc_i)
+{
+    double *D = static_cast<double *>(p.D);
+    const double *C = static_cast<const double *>(p.C);
+    if (CPLX) {
+        double d_r = p.alpha[0] * acc_r - p.alpha[1] * acc_i;
+        double d_i = p.alpha[0] * acc_i + p.alpha[1] * acc_r;
+        if (p.use_c) {
+            const double2 c = *reinterpret_cast<const double2 *>(C + 2 * off);
+            const double ci = p.conjC ? -c.y : c.y;
+            d_r += p.beta[0] * c.x - p.beta[1] * ci;
+            d_i += p.beta[0] * ci + p.beta[1] * c.x;
+        }
+        *reinterpret_cast<double2 *>(D + 2 * off) = make_double2(d_r, d_i);
+    } else {
+        double d = p.alpha[0] * acc_r;
+        if (p.use_c) d += p.beta[0] * C[off];
+        D[off] = d;
+    }
+}
+
+// Map accumulator (fi, fj, c) of a lane to its tile-local (row, column) in elements and write
+// every accumulator the thread holds.
+template <typename T>
+__device__ __forceinline__ void epilogue(const TiledParams &p, const double (&acc)[T::FM][T::FN][2],
+                                         const int64_t *rowD, const int64_t *colD, int rows_valid,
+                                         int cols_valid, int wm0, int wn0_words, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int fi = 0; fi < T::FM; ++fi) {
+        const int r = wm0 + fi * 8 + g;
+        if (r >= rows_valid) continue;
+        const int64_t ro = rowD[r];
+#pragma unroll
+        for (int fj = 0; fj < T::FN; ++fj) {
+            if (T::CPLX) {
+                const int c = (wn0_words + fj * 8) / 2 + t;
+                if (c < cols_valid) store_element<true>(p, ro + colD[c], acc[fi][fj][0], acc[fi][fj][1]);
+            } else {
+                const int c = wn0_words + fj * 8 + 2 * t;
+                if (c < cols_valid) store_element<false>(p, ro + colD[c], acc[fi][fj][0], 0.0);
+                if (c + 1 < cols_valid) store_element<false>(p, ro + colD[c + 1], acc[fi][fj][1], 0.0);
+            }
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(T::THREADS, 1) tiled_f64_kernel(const TiledParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    constexpr int W = T::W;
+    constexpr int EB = 8 * W;
+    double *stage_base = reinterpret_cast<double *>(smem_raw);
+    int64_t *rowA = reinterpret_cast<int64_t *>(stage_base + size_t(T::STAGES) * T::STAGE_WORDS);
+    int64_t *rowD = rowA + T::BM;
+    int64_t *colB = rowD + T::BM;
+    int64_t *colD = colB + T::BN;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // blockIdx.x enumerates (tile, k slice, batch), tile fastest
+    const int tiles = p.tiles_m * p.tiles_n;
+    const int tile = blockIdx.x % tiles;
+    const int ks = (blockIdx.x / tiles) % p.split_k;
+    const int64_t h = blockIdx.x / (tiles * p.split_k);
+    const int tile_m = p.raster_n_fast ? tile / p.tiles_n : tile % p.tiles_m;
+    const int tile_n = p.raster_n_fast ? tile % p.tiles_n : tile / p.tiles_m;
+    const int64_t m0 = int64_t(tile_m) * T::BM, n0 = int64_t(tile_n) * T::BN;
+    const int rows_valid = int(imin64(T::BM, p.M - m0));
+    const int cols_valid = int(imin64(T::BN, p.N - n0));
+    const int64_t k_begin = int64_t(ks) * p.k_per_split;
+    const int64_t k_end = imin64(p.K, k_begin + p.k_per_split);
+
+    // per-tile row/column offsets (batch offset folded in)
+    {
+        const int64_t hA = p.offA_h[h], hB = p.offB_h[h], hD = p.offD_h[h];
+        for (int i = tid; i < T::BM; i += T::THREADS) {
+            const bool v = i < rows_valid;
+            rowA[i] = v ? p.offA_m[m0 + i] + hA : 0;
+            rowD[i] = v ? p.offD_m[m0 + i] + hD : 0;
+        }
+        for (int i = tid; i < T::BN; i += T::THREADS) {
+            const bool v = i < cols_valid;
+            colB[i] = v ? p.offB_n[n0 + i] + hB : 0;
+            colD[i] = v ? p.offD_n[n0 + i] : 0;
+        }
+    }
+    __syncthreads();
+
+    // shared-memory orientation follows the load direction of each operand
+    const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
+    const int b_srow = p.dirB == 0 ? 1 : T::PITCH_K, b_sk = p.dirB == 0 ? T::PITCH_FREE_B : 1;
+
+    const int num_kt = int((k_end - k_begin + T::BK - 1) / T::BK);
+    auto load_stage = [&](int kt) {
+        double *sa = stage_base + size_t(kt % T::STAGES) * T::STAGE_WORDS;
+        double *sb = sa + T::A_ELEMS * W;
+        const int64_t k0 = k_begin + int64_t(kt) * T::BK;
+        gather_tile<T::BM, T::BK, T::THREADS, EB>(reinterpret_cast<char *>(sa), static_cast<const char *>(p.A),
+                                                  rowA, p.offA_k, rows_valid, k0, k_end, p.dirA, p.vecA,
+                                                  a_srow, a_sk, tid);
+        gather_tile<T::BN, T::BK, T::THREADS, EB>(reinterpret_cast<char *>(sb), static_cast<const char *>(p.B),
+                                                  colB, p.offB_k, cols_valid, k0, k_end, p.dirB, p.vecB,
+                                                  b_srow, b_sk, tid);
+    };
+
+    const int warp_m = warp % T::WARPS_M, warp_n = warp / T::WARPS_M;
+    const int wm0 = warp_m * T::WM;
+    const int wn0w = warp_n * T::WNR;            // first real-word column of the warp tile
+    const int g = lane >> 2, t = lane & 3;
+
+    // word offsets of this lane's fragment entries inside a stage
+    int a_thr, a_istep, a_kstep, b_thr, b_jstep, b_kstep;
+    unsigned b_sign = 0;                         // xor mask for the high word of b
+    if (!T::CPLX) {
+        a_thr = (wm0 + g) * a_srow + t * a_sk;
+        a_istep = 8 * a_srow;
+        a_kstep = 4 * a_sk;
+        b_thr = (wn0w + g) * b_srow + t * b_sk;
+        b_jstep = 8 * b_srow;
+        b_kstep = 4 * b_sk;
+    } else {
+        const int pbit = t & 1, qbit = g & 1;
+        a_thr = ((wm0 + g) * a_srow + (t >> 1) * a_sk) * 2 + pbit;
+        a_istep = 16 * a_srow;
+        a_kstep = 4 * a_sk;
+        b_thr = ((wn0w / 2 + (g >> 1)) * b_srow + (t >> 1) * b_sk) * 2 + (pbit ^ qbit);
+        b_jstep = 8 * b_srow;
+        b_kstep = 4 * b_sk;
+        // block [[br, sb*bi], [-sa*sb*bi, sa*br]]: entry (p, q) is negative when
+        //   (0,1): sb < 0;  (1,0): sa*sb > 0;  (1,1): sa < 0
+        const bool na = p.conjA != 0, nb = p.conjB != 0;
+        bool neg = false;
+        if (pbit == 0 && qbit == 1) neg = nb;
+        if (pbit == 1 && qbit == 0) neg = (na == nb);
+        if (pbit == 1 && qbit == 1) neg = na;
+        b_sign = neg ? 0x80000000u : 0u;
+    }
+
+    double acc[T::FM][T::FN][2];
+#pragma unroll
+    for (int i = 0; i < T::FM; ++i)
+#pragma unroll
+        for (int j = 0; j < T::FN; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+
+#pragma unroll
+    for (int s = 0; s < T::STAGES - 1; ++s) {
+        if (s < num_kt) load_stage(s);
+        cp_async_commit();
+    }
+
+    for (int kt = 0; kt < num_kt; ++kt) {
+        cp_async_wait<T::STAGES - 2>();
+        __syncthreads();
+        if (kt + T::STAGES - 1 < num_kt) load_stage(kt + T::STAGES - 1);
+        cp_async_commit();
+
+        const double *sa = stage_base + size_t(kt % T::STAGES) * T::STAGE_WORDS;
+        const double *sb = sa + T::A_ELEMS * W;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {         // 16 real k per stage, 4 per MMA
+            double af[T::FM], bf[T::FN];
+#pragma unroll
+            for (int i = 0; i < T::FM; ++i) af[i] = sa[a_thr + i * a_istep + kk * a_kstep];
+#pragma unroll
+            for (int j = 0; j < T::FN; ++j) {
+                double b = sb[b_thr + j * b_jstep + kk * b_kstep];
+                if (T::CPLX) {
+                    int hi = __double2hiint(b) ^ int(b_sign);
+                    b = __hiloint2double(hi, __double2loint(b));
+                }
+                bf[j] = b;
+            }
+#pragma unroll
+            for (int i = 0; i < T::FM; ++i)
+#pragma unroll
+                for (int j = 0; j < T::FN; ++j) dmma_m8n8k4(acc[i][j][0], acc[i][j][1], af[i], bf[j]);
+        }
+    }
+    cp_async_wait<0>();
+
+    if (p.split_k == 1) {
+        epilogue<T>(p, acc, rowD, colD, rows_valid, cols_valid, wm0, wn0w, lane);
+    } else {
+        // raw accumulators -> scratch, [batch][slice][tile][acc index][thread]
+        double *ws = static_cast<double *>(p.partials);
+        const size_t tile_lin = blockIdx.x;
+        double *dst = ws + tile_lin * (size_t(T::THREADS) * T::ACC) + tid;
+#pragma unroll
+        for (int i = 0; i < T::FM; ++i)
+#pragma unroll
+            for (int j = 0; j < T::FN; ++j) {
+                dst[size_t((i * T::FN + j) * 2 + 0) * T::THREADS] = acc[i][j][0];
+                dst[size_t((i * T::FN + j) * 2 + 1) * T::THREADS] = acc[i][j][1];
+            }
+    }
+}
+
+// Second pass of split-K: fixed-order sum of the slices, then alpha/beta and the strided store.
+template <typename T>
+__global__ void __launch_bounds__(T::THREADS) tiled_f64_splitk_reduce_kernel(const TiledParams p)
+{
+    __shared__ int64_t rowD[T::BM];
+    __shared__ int64_t colD[T::BN];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // blockIdx.x enumerates (tile, batch), tile fastest
+    const int tiles_i = p.tiles_m * p.tiles_n;
+    const int tile = blockIdx.x % tiles_i;
+    const int64_t h = blockIdx.x / tiles_i;
+    const int tile_m = p.raster_n_fast ? tile / p.tiles_n : tile % p.tiles_m;
+    const int tile_n = p.raster_n_fast ? tile % p.tiles_n : tile / p.tiles_m;
+    const int64_t m0 = int64_t(tile_m) * T::BM, n0 = int64_t(tile_n) * T::BN;
+    const int rows_valid = int(imin64(T::BM, p.M - m0));
+    const int cols_valid = int(imin64(T::BN, p.N - n0));
+    const int64_t hD = p.offD_h[h];
+    for (int i = tid; i < T::BM; i += T::THREADS) rowD[i] = i < rows_valid ? p.offD_m[m0 + i] + hD : 0;
+    for (int i = tid; i < T::BN; i += T::THREADS) colD[i] = i < cols_valid ? p.offD_n[n0 + i] : 0;
+    __syncthreads();
+
+    double acc[T::FM][T::FN][2];
+#pragma unroll
+    for (int i = 0; i < T::FM; ++i)
+#pragma unroll
+        for (int j = 0; j < T::FN; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+    const double *ws = static_cast<const double *>(p.partials);
+    const size_t tiles = size_t(p.tiles_m) * p.tiles_n;
+    for (int ks = 0; ks < p.split_k; ++ks) {
+        const size_t tile_lin = (size_t(h) * p.split_k + ks) * tiles + tile;
+        const double *src = ws + tile_lin * (size_t(T::THREADS) * T::ACC) + tid;
+#pragma unroll
+        for (int i = 0; i < T::FM; ++i)
+#pragma unroll
+            for (int j = 0; j < T::FN; ++j) {
+                acc[i][j][0] += src[size_t((i * T::FN + j) * 2 + 0) * T::THREADS];
+                acc[i][j][1] += src[size_t((i * T::FN + j) * 2 + 1) * T::THREADS];
+            }
+    }
+    const int warp_m = warp % T::WARPS_M, warp_n = warp / T::WARPS_M;
+    epilogue<T>(p, acc, rowD, colD, rows_valid, cols_valid, warp_m * T::WM, warp_n * T::WNR, lane);
+}
+
+}  // namespace btc

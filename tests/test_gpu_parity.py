@@ -1,0 +1,211 @@
+"""GPU parity: the CUDA path (through the C-ABI) against the CPU oracle, element by element, on
+the same seeded inputs.  Sizes span several tiles and ragged tails; the categories follow the
+paper's test list (Appendix "Testing")."""
+import dataclasses
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import helpers
+from paper_2601_07827_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+REAL_AND_COMPLEX = [torch.float32, torch.float64, torch.complex64, torch.complex128]
+
+
+@pytest.fixture(scope="module")
+def api():
+    return helpers.api()
+
+
+@pytest.fixture(scope="module")
+def handle(api):
+    return api.Handle()
+
+
+def small_workloads():
+    W = inputs.workloads()
+    out = {
+        "cfg1": W["cfg1_f64_small"],
+        "cfg2s": inputs.scaled_down(W["cfg2_f64_ccsd_ladder"], {"a": 12, "b": 12, "c": 10, "d": 10, "i": 7, "j": 6}),
+        "cfg3s": inputs.scaled_down(W["cfg3_f32_batched_permuted"], {"z": 3, "a": 20, "b": 12, "j": 24, "k": 6, "l": 8}),
+        "cfg4s": inputs.scaled_down(W["cfg4_c64_conj"], {"p": 40, "q": 24, "r": 5, "s": 12, "t": 8}),
+        "cfg5": W["cfg5_f32_tensor_network"],
+        "cfg5b": W["cfg5b_f32_tensor_network_rev"],
+    }
+    return out
+
+
+@pytest.mark.parametrize("name", list(small_workloads()))
+@pytest.mark.parametrize("kernel", ["auto", "generic", "tiled"])
+def test_workload_shapes(api, handle, name, kernel):
+    w = small_workloads()[name]
+    code = {"auto": api.KERNEL_AUTO, "generic": api.KERNEL_GENERIC, "tiled": api.KERNEL_TILED}[kernel]
+    try:
+        worst, status, _ = helpers.workload_case(handle, w, kernel=code, want_status=True)
+    except api.BtcError as e:
+        if kernel == "tiled" and e.code == api.ERR_NOT_SUPPORTED:
+            pytest.skip("no tiled kernel for this element type yet")
+        raise
+    assert worst <= 1.0, worst
+    if kernel != "auto":
+        assert status["kernel"] == code
+
+
+@pytest.mark.parametrize("split_k", [1, 2, 3, 7])
+@pytest.mark.parametrize("name", ["cfg1", "cfg4s"])
+def test_split_k_slices(api, handle, name, split_k):
+    w = small_workloads()[name]
+    worst, status, first = helpers.workload_case(handle, w, kernel=api.KERNEL_TILED, split_k=split_k, want_status=True)
+    assert worst <= 1.0 and status["split_k"] == split_k
+    assert status["launches"] == (2 if split_k > 1 else 1)
+    _, _, second = helpers.workload_case(handle, w, kernel=api.KERNEL_TILED, split_k=split_k)
+    assert torch.equal(first.view(torch.int64), second.view(torch.int64))   # run-to-run bit identical
+
+
+def _ext(labels, table):
+    return tuple(table[l] for l in labels)
+
+
+CATEGORIES = {
+    # name: (labelsA, labelsB, labelsD, extents)
+    "hadamard": ("ij", "ij", "ij", dict(i=37, j=29)),
+    "basic": ("ikl", "ljk", "ji", dict(i=70, j=45, k=9, l=11)),
+    "equal_extents": ("aibj", "jcia", "cb", dict(a=6, b=6, c=6, i=6, j=6)),
+    "outer_product": ("ij", "kl", "kijl", dict(i=13, j=5, k=9, l=7)),
+    "all_contracted": ("ijk", "kji", "", dict(i=17, j=9, k=33)),
+    "zero_mode_A": ("", "ij", "ji", dict(i=40, j=33)),
+    "one_mode": ("k", "kj", "j", dict(k=300, j=70)),
+    "hadamard_free": ("hik", "hkj", "ijh", dict(h=5, i=33, j=18, k=40)),
+    "hadamard_contracted": ("hk", "hk", "h", dict(h=77, k=130)),
+    "repeated": ("kik", "kjj", "ij", dict(i=35, j=21, k=19)),
+    "isolated": ("ikx", "kyj", "ij", dict(i=33, j=20, k=17, x=3, y=4)),
+    "gemv_like": ("ik", "k", "i", dict(i=1000, k=333)),
+    "big_ragged": ("ik", "kj", "ij", dict(i=257, j=131, k=67)),
+}
+
+
+@pytest.mark.parametrize("dtype", REAL_AND_COMPLEX)
+@pytest.mark.parametrize("cat", list(CATEGORIES))
+def test_paper_test_categories(api, handle, cat, dtype):
+    la, lb, ld, ext = CATEGORIES[cat]
+    A = helpers.random_tensor(11, _ext(la, ext), None, dtype)
+    B = helpers.random_tensor(12, _ext(lb, ext), None, dtype)
+    C = helpers.random_tensor(13, _ext(ld, ext), None, dtype)
+    D = inputs.place(None, _ext(ld, ext), None, dtype)
+    cplx = dtype.is_complex
+    alpha = complex(0.75, -1.25) if cplx else 0.75
+    beta = complex(-0.5, 0.25) if cplx else -0.5
+    worst, _, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, beta, conjA=cplx, conjC=cplx)
+    assert worst <= 1.0, worst
+
+
+@pytest.mark.parametrize("dtype", [torch.float64, torch.complex128, torch.float32])
+@pytest.mark.parametrize("kernel", ["auto", "generic"])
+def test_strides_negative_zero_padded_subtensor(api, handle, dtype, kernel):
+    code = {"auto": api.KERNEL_AUTO, "generic": api.KERNEL_GENERIC}[kernel]
+    ext = dict(i=70, j=45, k=40, l=6)
+    # A: negative stride on i, padded; B: zero stride on l (broadcast), mixed signs; D: padded + negative
+    A = helpers.random_tensor(21, _ext("ikl", ext), (-1, 75, 75 * 41), dtype)
+    B = helpers.random_tensor(22, _ext("lkj", ext), (0, -3, 130), dtype)
+    C = helpers.random_tensor(23, _ext("ji", ext), (2, -95), dtype)
+    D = inputs.place(None, _ext("ji", ext), (2, -95), dtype)
+    worst, _, _ = helpers.run_case(handle, A, "ikl", B, "lkj", C, D, "ji", 1.5, 0.5, kernel=code)
+    assert worst <= 1.0, worst
+    # sub-tensor with fewer modes than its parent: a slice of a rank-4 buffer used as a rank-2 operand
+    A2 = helpers.random_tensor(24, (70, 40), (7, 7 * 80), dtype)
+    D2 = inputs.place(None, (70, 45), (1, 72), dtype)
+    worst, _, _ = helpers.run_case(handle, A2, "ik", B, "lkj", None, D2, "ij", kernel=code)
+    assert worst <= 1.0, worst
+
+
+@pytest.mark.parametrize("dtype", [torch.complex64, torch.complex128])
+def test_conjugation_flags(api, handle, dtype):
+    ext = dict(i=40, j=36, k=50)
+    A = helpers.random_tensor(31, _ext("ki", ext), None, dtype)
+    B = helpers.random_tensor(32, _ext("kj", ext), None, dtype)
+    C = helpers.random_tensor(33, _ext("ij", ext), None, dtype)
+    D = inputs.place(None, _ext("ij", ext), None, dtype)
+    for ca, cb, cc in itertools.product([False, True], repeat=3):
+        worst, _, _ = helpers.run_case(handle, A, "ki", B, "kj", C, D, "ij", complex(0.5, -0.25), complex(1, 2),
+                                       conjA=ca, conjB=cb, conjC=cc)
+        assert worst <= 1.0, (ca, cb, cc, worst)
+
+
+@pytest.mark.parametrize("dtype", REAL_AND_COMPLEX)
+def test_small_integers_bit_exact(api, handle, dtype):
+    """Exactly representable inputs: every summation order gives the same bits."""
+    ext = dict(i=70, j=66, k=40, l=5)
+    A = helpers.random_tensor(41, _ext("ikl", ext), None, dtype, ("smallint", 8))
+    B = helpers.random_tensor(42, _ext("lkj", ext), None, dtype, ("smallint", 8))
+    C = helpers.random_tensor(43, _ext("ji", ext), None, dtype, ("smallint", 8))
+    D = inputs.place(None, _ext("ji", ext), None, dtype)
+    for kernel in (api.KERNEL_AUTO, api.KERNEL_GENERIC):
+        worst, _, _ = helpers.run_case(handle, A, "ikl", B, "lkj", C, D, "ji", 2.0, -3.0, kernel=kernel)
+        assert worst == 0.0
+
+
+def test_alpha_zero_and_beta_zero_never_read(api, handle):
+    ext = dict(i=130, j=70, k=64)
+    A = helpers.random_tensor(51, _ext("ik", ext), None, torch.float64)
+    B = helpers.random_tensor(52, _ext("kj", ext), None, torch.float64)
+    C = helpers.random_tensor(53, _ext("ij", ext), None, torch.float64)
+    D = inputs.place(None, _ext("ij", ext), None, torch.float64)
+    nanA = inputs.place(None, _ext("ik", ext), None, torch.float64)   # all NaN
+    worst, _, _ = helpers.run_case(handle, nanA, "ik", B, "kj", C, D, "ij", 0.0, 2.0)
+    assert worst == 0.0
+    nanC = inputs.place(None, _ext("ij", ext), None, torch.float64)
+    worst, _, _ = helpers.run_case(handle, A, "ik", B, "kj", nanC, D, "ij", 1.0, 0.0)
+    assert worst <= 1.0
+
+
+def test_in_place_update(api, handle):
+    w = small_workloads()["cfg2s"]
+    assert w.in_place
+    worst, _, _ = helpers.workload_case(handle, w)
+    assert worst <= 1.0
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg3s", "cfg4s"])
+def test_host_buffer_entry_point(api, handle, name):
+    worst, _, _ = helpers.workload_case(handle, small_workloads()[name], host_path=True)
+    assert worst <= 1.0
+
+
+def test_execute_argument_errors(api, handle):
+    w = small_workloads()["cfg1"]
+    A, B, C, D = (t.to("cuda") for t in inputs.make_workload_tensors(w))
+    dt = api.F64
+    tA, tB = api.TensorInfo(handle, dt, A.extents), api.TensorInfo(handle, dt, B.extents)
+    tD = api.TensorInfo(handle, dt, D.extents)
+    op = api.Contraction(handle, tA, w.labelsA, tB, w.labelsB, tD, w.labelsD, tD, w.labelsD, 1.0, 0.5)
+    ws = torch.empty(op.workspace_size(), dtype=torch.uint8, device="cuda")
+
+    def code(fn):
+        with pytest.raises(api.BtcError) as ei:
+            fn()
+        return ei.value.code
+    assert op.workspace_size() > 0
+    assert code(lambda: op.execute(0, A.data_ptr(), B.data_ptr(), C.data_ptr(), D.data_ptr())) == api.ERR_WORKSPACE_TOO_SMALL
+    assert code(lambda: op.execute(0, A.data_ptr(), B.data_ptr(), C.data_ptr(), D.data_ptr(),
+                                   workspace=ws.data_ptr(), workspace_bytes=16)) == api.ERR_WORKSPACE_TOO_SMALL
+    assert code(lambda: op.execute(0, A.data_ptr() + 4, B.data_ptr(), C.data_ptr(), D.data_ptr(),
+                                   workspace=ws.data_ptr(), workspace_bytes=ws.numel())) == api.ERR_MISALIGNED
+    assert code(lambda: op.execute(0, A.data_ptr(), B.data_ptr(), 0, D.data_ptr(),
+                                   workspace=ws.data_ptr(), workspace_bytes=ws.numel())) == api.ERR_INVALID_ARGUMENT
+    op.execute(0, A.data_ptr(), B.data_ptr(), 0, D.data_ptr(), beta=0.0, workspace=ws.data_ptr(), workspace_bytes=ws.numel())
+    torch.cuda.synchronize()
+
+
+def test_unaligned_base_pointer_falls_back_to_element_copies(api, handle):
+    """Operands whose strides allow 16-byte copies but whose base pointer is only 8-byte aligned."""
+    ext = dict(i=128, j=64, k=32)
+    A = helpers.random_tensor(61, (4200,), None, torch.float64)
+    A_view = inputs.StridedTensor(A.buffer, (128, 32), (1, 130), 1)   # starts at element 1, ld 130
+    B = helpers.random_tensor(62, _ext("kj", ext), None, torch.float64)
+    D = inputs.place(None, _ext("ij", ext), None, torch.float64)
+    worst, _, _ = helpers.run_case(handle, A_view, "ik", B, "kj", None, D, "ij", kernel=api.KERNEL_TILED)
+    assert worst <= 1.0
