@@ -310,6 +310,10 @@ def workloads() -> Dict[str, Workload]:
         alpha=1.0, beta=1.0, in_place=True, seed=2000,
         distA=("normal", 0.1), distB=("uniform", 0.01), distC=("uniform", 0.01),
         symmetryA="pair_swap")
+    # 2p: the same ladder term with c,d = 64 (0.5 GiB of V): the case profiler captures use
+    w["cfg2p_f64_ccsd_ladder_profile"] = dataclasses.replace(
+        w["cfg2_f64_ccsd_ladder"], name="cfg2p_f64_ccsd_ladder_profile",
+        extents={**_all(128, "ab"), **_all(64, "cd"), **_all(32, "ij")})
     # 3: fp32, batch label z, permuted output with a padded leading stride
     e3 = {"z": 64, "a": 96, "b": 96, "j": 96, "k": 24, "l": 24}
     w["cfg3_f32_batched_permuted"] = Workload(

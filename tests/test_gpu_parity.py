@@ -60,7 +60,8 @@ def test_workload_shapes(api, handle, name, kernel):
 def test_split_k_slices(api, handle, name, split_k):
     w = small_workloads()[name]
     worst, status, first = helpers.workload_case(handle, w, kernel=api.KERNEL_TILED, split_k=split_k, want_status=True)
-    assert worst <= 1.0 and status["split_k"] == split_k
+    # the library may lower the request so that no slice is empty
+    assert worst <= 1.0 and (split_k > 1) == (status["split_k"] > 1) and status["split_k"] <= split_k
     assert status["launches"] == (2 if split_k > 1 else 1)
     _, _, second = helpers.workload_case(handle, w, kernel=api.KERNEL_TILED, split_k=split_k)
     assert torch.equal(first.view(torch.int64), second.view(torch.int64))   # run-to-run bit identical
