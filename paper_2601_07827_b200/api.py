@@ -37,6 +37,7 @@ F32, F64, C32, C64 = 0, 1, 2, 3
 DTYPE_SIZE = {F32: 4, F64: 8, C32: 8, C64: 16}
 
 ATTR_KERNEL, ATTR_SPLIT_K, ATTR_TILE, ATTR_GROUPS, ATTR_GRID, ATTR_NUM_MODES, ATTR_SWAPPED = 1, 2, 3, 4, 5, 6, 7
+ATTR_DEVICE_ERROR = 8
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TILED = 0, 1, 2
 STATUS_KERNEL, STATUS_LAUNCHES, STATUS_GRID, STATUS_SPLIT_K = 1, 2, 3, 4
 
@@ -203,6 +204,11 @@ class Contraction:
     @property
     def swapped(self) -> bool:
         return bool(self._get(ATTR_SWAPPED, ctypes.c_int32, 1)[0])
+
+    @property
+    def device_error(self) -> int:
+        """0, or the code of a bounded device-side wait that gave up (waits for the device)."""
+        return self._get(ATTR_DEVICE_ERROR, ctypes.c_int32, 1)[0]
 
     def set_attr(self, key: int, value: int) -> None:
         v = ctypes.c_int32(value)

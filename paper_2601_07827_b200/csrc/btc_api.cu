@@ -37,6 +37,7 @@ struct btc_contraction_s {
     double alpha[2] = {1.0, 0.0}, beta[2] = {0.0, 0.0};
     // device copies of the plan's tables (one allocation)
     int64_t *d_tables = nullptr;
+    int32_t *d_error = nullptr;   // inside d_tables' allocation; non-zero after a device-side wait gave up
     const int64_t *d_offA_m = nullptr, *d_offD_m = nullptr, *d_offB_n = nullptr, *d_offD_n = nullptr,
                   *d_offA_k = nullptr, *d_offB_k = nullptr, *d_offA_h = nullptr, *d_offB_h = nullptr,
                   *d_offD_h = nullptr;
@@ -49,16 +50,17 @@ struct btc_contraction_s {
 namespace {
 
 // ---- tiled kernel variants -------------------------------------------------------------------
-using F64Big = F64Tile<false, 128, 128, 2, 4, 4>;
-using F64Small = F64Tile<false, 64, 64, 2, 2, 4>;
-using C64Big = F64Tile<true, 128, 64, 2, 4, 4>;
-using C64Small = F64Tile<true, 64, 32, 2, 2, 4>;
+using F64Big = F64Tile<false, 128, 128, 2, 4, 4, 1>;
+using F64Small = F64Tile<false, 64, 64, 2, 2, 4, 2>;
+using C64Big = F64Tile<true, 128, 64, 2, 4, 4, 1>;
+using C64Small = F64Tile<true, 64, 32, 2, 2, 4, 2>;
 
 struct VariantInfo {
     int bm, bn, bk, threads, acc;
     size_t smem;
 };
-template <typename T> VariantInfo info_of() { return {T::BM, T::BN, T::BK, T::THREADS, T::ACC, T::SMEM_BYTES}; }
+// `threads` counts the consumer threads: they own the accumulators (split-K scratch layout)
+template <typename T> VariantInfo info_of() { return {T::BM, T::BN, T::BK, T::CONSUMER_THREADS, T::ACC, T::SMEM_BYTES}; }
 
 bool tiled_supported(btc_dtype_t t) { return t == BTC_F64 || t == BTC_C64; }
 
@@ -84,7 +86,7 @@ cudaError_t launch_tiled(const TiledParams &p, int64_t ctas, int64_t reduce_ctas
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (p.split_k > 1) {
-        tiled_f64_splitk_reduce_kernel<T><<<unsigned(reduce_ctas), T::THREADS, 0, st>>>(p);
+        tiled_f64_splitk_reduce_kernel<T><<<unsigned(reduce_ctas), T::CONSUMER_THREADS, 0, st>>>(p);
         e = cudaGetLastError();
     }
     return e;
@@ -104,6 +106,7 @@ void free_tables(btc_contraction_s *op)
 {
     if (op->d_tables) cudaFree(op->d_tables);
     op->d_tables = nullptr;
+    op->d_error = nullptr;
 }
 
 // Choose tile variant, raster order and split-K for a tiled plan; upload the offset tables.
@@ -173,6 +176,8 @@ int finish_plan(btc_contraction_s *op)
                                   &op->d_offB_k, &op->d_offA_h, &op->d_offB_h, &op->d_offD_h};
         size_t total = 0;
         for (auto *t : tabs) total += (t->size() + 31) / 32 * 32;   // keep every table 256-byte aligned
+        const size_t error_at = total;
+        total += 32;                                                  // the error word, zeroed
         std::vector<int64_t> host(total, 0);
         size_t pos = 0, starts[9];
         for (int i = 0; i < 9; ++i) {
@@ -190,6 +195,7 @@ int finish_plan(btc_contraction_s *op)
             return BTC_ERR_CUDA;
         }
         for (int i = 0; i < 9; ++i) *dst[i] = op->d_tables + starts[i];
+        op->d_error = reinterpret_cast<int32_t *>(op->d_tables + error_at);
     }
     return BTC_SUCCESS;
 }
@@ -380,6 +386,16 @@ btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t 
         i32[0] = int32_t(pl.batch.size()); i32[1] = int32_t(pl.m.size());
         i32[2] = int32_t(pl.n.size()); i32[3] = int32_t(pl.k.size()); n = 16; break;
     case BTC_ATTR_SWAPPED: i32[0] = pl.swapped ? 1 : 0; n = 4; break;
+    case BTC_ATTR_DEVICE_ERROR:
+        i32[0] = 0;
+        if (op->d_error) {
+            if (cudaMemcpy(&i32[0], op->d_error, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) {
+                cudaGetLastError();
+                return BTC_ERR_CUDA;
+            }
+        }
+        n = 4;
+        break;
     default: return BTC_ERR_INVALID_ARGUMENT;
     }
     if (needed) *needed = n;
@@ -469,6 +485,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         tp.use_c = use_c;
         tp.alpha[0] = al[0]; tp.alpha[1] = al[1]; tp.beta[0] = be[0]; tp.beta[1] = be[1];
         tp.partials = workspace;
+        tp.error_word = op->d_error;
         const int64_t ctas = op->grid[0];
         const int64_t reduce_ctas = ctas / pl.split_k;
         if (pl.dtype == BTC_F64)

@@ -40,6 +40,7 @@ struct TiledParams {
     int32_t use_c;
     double alpha[2], beta[2];
     void *partials;                   // split-K scratch (workspace), or nullptr
+    int32_t *error_word;              // device word; set non-zero when a bounded wait gave up
 };
 
 }  // namespace btc

@@ -8,15 +8,22 @@
 // memory: the FP64 tensor-core fragments (mma.sync m8n8k4, one 8-byte word per lane) can be read
 // from either orientation without bank conflicts, so no transpose is ever materialised.
 //
+// The CTA is warp-specialised: one warpgroup of producer warps does all address arithmetic and
+// issues the cp.async gathers; the consumer warps only read fragments and issue MMAs.  The two
+// sides hand shared-memory stages to each other through mbarriers ("full": armed by the
+// completion of the producers' copies; "empty": one arrival per consumer warp).  Every wait is
+// bounded: when a wait runs out the kernel records an error word, raises a CTA-wide abort flag
+// so the other waits end too, drains its copies and returns.
+//
 // Complex128 runs on the same real MMAs: an interleaved (re, im) row of A is a real row of
 // twice the length, and each complex b expands at fragment-load time into the 2x2 real block
 // [[br, sb*bi], [-sa*sb*bi, sa*br]] (sa, sb = -1 when that operand is conjugated), which gives
 // exactly 8 real flops per complex multiply-add.  An 8x8 accumulator fragment then holds
 // 8 rows x 4 complex columns with (re, im) adjacent in one lane.
 //
-// K is pipelined through STAGES shared-memory buffers.  With split-K each CTA handles one slice
-// of k and stores raw accumulators to scratch; a second kernel adds the slices in a fixed order
-// and applies alpha/beta, so results do not depend on scheduling.
+// With split-K each CTA handles one slice of k and stores raw accumulators to scratch; a second
+// kernel adds the slices in a fixed order and applies alpha/beta, so results do not depend on
+// scheduling.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -25,7 +32,9 @@
 
 namespace btc {
 
-template <bool CPLX_, int BM_, int BN_, int WARPS_M_, int WARPS_N_, int STAGES_>
+constexpr int kProducerWarps = 4;   // one warpgroup
+
+template <bool CPLX_, int BM_, int BN_, int WARPS_M_, int WARPS_N_, int STAGES_, int MIN_CTAS_>
 struct F64Tile {
     static constexpr bool CPLX = CPLX_;
     static constexpr int BM = BM_;                    // rows of the CTA tile (elements)
@@ -33,12 +42,19 @@ struct F64Tile {
     static constexpr int BK = CPLX_ ? 8 : 16;         // k extent of one stage (elements)
     static constexpr int W = CPLX_ ? 2 : 1;           // 8-byte words per element
     static constexpr int WARPS_M = WARPS_M_, WARPS_N = WARPS_N_;
-    static constexpr int THREADS = 32 * WARPS_M_ * WARPS_N_;
+    static constexpr int CONSUMER_WARPS = WARPS_M_ * WARPS_N_;
+    static constexpr int CONSUMER_THREADS = 32 * CONSUMER_WARPS;
+    static constexpr int PRODUCER_THREADS = 32 * kProducerWarps;
+    static constexpr int THREADS = CONSUMER_THREADS + PRODUCER_THREADS;
+    static constexpr int MIN_CTAS = MIN_CTAS_;
+    // with 12 warps the register file gives 168 registers per thread; the consumers need more,
+    // the producers far fewer, so the warpgroups re-split the file (setmaxnreg)
+    static constexpr bool REBALANCE_REGS = (THREADS == 384);
     static constexpr int STAGES = STAGES_;
     static constexpr int WM = BM / WARPS_M;           // warp tile rows
     static constexpr int WNR = BN * W / WARPS_N;      // warp tile columns in real words
     static constexpr int FM = WM / 8, FN = WNR / 8;   // 8x8 fragments per warp
-    static constexpr int ACC = FM * FN * 2;           // doubles per thread
+    static constexpr int ACC = FM * FN * 2;           // doubles per consumer thread
     // shared-memory pitches (elements): conflict-free fragment reads need
     //   real:    pitch = 4 (mod 16);   complex: pitch = 4 (mod 8) along the free index,
     //                                           pitch = 2 (mod 8) along k
@@ -47,24 +63,64 @@ struct F64Tile {
     static constexpr int A_ELEMS = (BK * PITCH_FREE_A > BM * PITCH_K) ? BK * PITCH_FREE_A : BM * PITCH_K;
     static constexpr int B_ELEMS = (BK * PITCH_FREE_B > BN * PITCH_K) ? BK * PITCH_FREE_B : BN * PITCH_K;
     static constexpr int STAGE_WORDS = (A_ELEMS + B_ELEMS) * W;
-    static constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_WORDS * 8 + size_t(2 * BM + 2 * BN) * 8;
+    // stages | row/column offset arrays | full[STAGES], empty[STAGES] mbarriers | abort flag
+    static constexpr size_t SMEM_BYTES =
+        size_t(STAGES) * STAGE_WORDS * 8 + size_t(2 * BM + 2 * BN) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
 
 __device__ __forceinline__ int64_t imin64(int64_t a, int64_t b) { return a < b ? a : b; }
 
-__device__ __forceinline__ void cp_async_bytes(void *smem_dst, const void *gsrc, int bytes, bool valid)
+// ---- asynchronous copies and mbarriers ---------------------------------------------------------
+template <int BYTES>
+__device__ __forceinline__ void cp_async_bytes(unsigned dst, const void *gsrc, bool valid)
 {
-    const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
-    const int src = valid ? bytes : 0;   // src-size 0 zero-fills the destination
-    if (bytes == 16)
+    const int src = valid ? BYTES : 0;   // src-size 0 zero-fills the destination
+    if (BYTES == 16)
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
-    else if (bytes == 8)
+    else if (BYTES == 8)
         asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
     else
         asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, int count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// the barrier receives one arrival from this thread once all its earlier cp.async have landed
+__device__ __forceinline__ void mbar_arrive_on_copies(unsigned bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+constexpr unsigned kWaitPollLimit = 1u << 22;   // polls before a wait gives up (a poll itself blocks briefly)
+constexpr int kErrFullWait = 1, kErrEmptyWait = 2;
+
+// Bounded wait.  Returns false when it gave up or another warp raised the abort flag.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, volatile int *abort_flag,
+                                                  int *error_word, int code)
+{
+    for (unsigned n = 0; n < kWaitPollLimit; ++n) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((n & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    if (error_word) atomicCAS(error_word, 0, code);
+    return false;
+}
 
 __device__ __forceinline__ void dmma_m8n8k4(double &c0, double &c1, double a, double b)
 {
@@ -72,28 +128,49 @@ __device__ __forceinline__ void dmma_m8n8k4(double &c0, double &c1, double a, do
                  : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
 
+template <int REGS> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS)); }
+template <int REGS> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS)); }
+
 // Gather one ROWS x BK tile (rows = free index, columns = k) into shared memory.
+//   DIR       0: consecutive threads take consecutive rows; 1: consecutive k
+//   VEC       elements per copy along that direction
 //   row_off   shared array: element offset of each tile row (batch offset included)
-//   koff      global table of k offsets;  [k_begin, k_end) is this CTA's valid k range
-//   dir       0: consecutive threads take consecutive rows; 1: consecutive k
-//   vec       elements per copy along that direction (1 or 16 / sizeof(element))
+//   koff      global table of k offsets;  [.., k_end) is this CTA's valid k range
 //   s_row, s_k  shared-memory strides of the tile in elements
-template <int ROWS, int BK, int THREADS, int ELEM_BYTES>
-__device__ __forceinline__ void gather_tile(char *smem, const char *__restrict__ g,
-                                            const int64_t *row_off, const int64_t *__restrict__ koff,
-                                            int rows_valid, int64_t k0, int64_t k_end,
-                                            int dir, int vec, int s_row, int s_k, int tid)
+template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES, int DIR, int VEC>
+__device__ __forceinline__ void gather_tile(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
+                                            const int64_t *__restrict__ koff, int rows_valid, int64_t k0,
+                                            int64_t k_end, int s_row, int s_k, int tid)
 {
-    const int nfast = (dir == 0 ? ROWS : BK) / vec;
-    const int slots = ROWS * BK / vec;
-    const int bytes = vec * ELEM_BYTES;
-    for (int s = tid; s < slots; s += THREADS) {
-        const int f = (s % nfast) * vec, o = s / nfast;
-        const int r = dir == 0 ? f : o;
-        const int k = dir == 0 ? o : f;
+    constexpr int NFAST = (DIR == 0 ? ROWS : BK) / VEC;
+    constexpr int SLOTS = ROWS * BK / VEC;
+#pragma unroll 4
+    for (int s = tid; s < SLOTS; s += NTHREADS) {
+        const int f = (s % NFAST) * VEC, o = s / NFAST;
+        const int r = DIR == 0 ? f : o;
+        const int k = DIR == 0 ? o : f;
         const bool valid = (r < rows_valid) && (k0 + k < k_end);
         const int64_t off = valid ? row_off[r] + __ldg(koff + k0 + k) : 0;
-        cp_async_bytes(smem + size_t(r * s_row + k * s_k) * ELEM_BYTES, g + off * ELEM_BYTES, bytes, valid);
+        cp_async_bytes<VEC * ELEM_BYTES>(smem + unsigned(r * s_row + k * s_k) * ELEM_BYTES, g + off * ELEM_BYTES, valid);
+    }
+}
+
+template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES>
+__device__ __forceinline__ void gather_dispatch(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
+                                                const int64_t *__restrict__ koff, int rows_valid, int64_t k0,
+                                                int64_t k_end, int dir, int vec, int s_row, int s_k, int tid)
+{
+    constexpr int VMAX = 16 / ELEM_BYTES;   // 2 for fp64, 1 for complex128
+    if (dir == 0) {
+        if (VMAX > 1 && vec == VMAX)
+            gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, 0, VMAX>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
+        else
+            gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, 0, 1>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
+    } else {
+        if (VMAX > 1 && vec == VMAX)
+            gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, 1, VMAX>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
+        else
+            gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, 1, 1>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
     }
 }
 
@@ -148,7 +225,7 @@ __device__ __forceinline__ void epilogue(const TiledParams &p, const double (&ac
 }
 
 template <typename T>
-__global__ void __launch_bounds__(T::THREADS, 1) tiled_f64_kernel(const TiledParams p)
+__global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(const TiledParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     constexpr int W = T::W;
@@ -158,6 +235,10 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_f64_kernel(const TiledPar
     int64_t *rowD = rowA + T::BM;
     int64_t *colB = rowD + T::BM;
     int64_t *colD = colB + T::BN;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(colD + T::BN);      // full[STAGES], empty[STAGES]
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * T::STAGES);
+    const unsigned full0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
+    const unsigned empty0 = full0 + 8u * T::STAGES;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // blockIdx.x enumerates (tile, k slice, batch), tile fastest
@@ -172,8 +253,9 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_f64_kernel(const TiledPar
     const int cols_valid = int(imin64(T::BN, p.N - n0));
     const int64_t k_begin = int64_t(ks) * p.k_per_split;
     const int64_t k_end = imin64(p.K, k_begin + p.k_per_split);
+    const int num_kt = int((k_end - k_begin + T::BK - 1) / T::BK);
 
-    // per-tile row/column offsets (batch offset folded in)
+    // per-tile row/column offsets (batch offset folded in), barriers
     {
         const int64_t hA = p.offA_h[h], hB = p.offB_h[h], hD = p.offD_h[h];
         for (int i = tid; i < T::BM; i += T::THREADS) {
@@ -186,6 +268,13 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_f64_kernel(const TiledPar
             colB[i] = v ? p.offB_n[n0 + i] + hB : 0;
             colD[i] = v ? p.offD_n[n0 + i] : 0;
         }
+        if (tid == 0) {
+            for (int s = 0; s < T::STAGES; ++s) {
+                mbar_init(full0 + 8u * s, T::PRODUCER_THREADS);
+                mbar_init(empty0 + 8u * s, T::CONSUMER_WARPS);
+            }
+            *abort_flag = 0;
+        }
     }
     __syncthreads();
 
@@ -193,20 +282,33 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_f64_kernel(const TiledPar
     const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
     const int b_srow = p.dirB == 0 ? 1 : T::PITCH_K, b_sk = p.dirB == 0 ? T::PITCH_FREE_B : 1;
 
-    const int num_kt = int((k_end - k_begin + T::BK - 1) / T::BK);
-    auto load_stage = [&](int kt) {
-        double *sa = stage_base + size_t(kt % T::STAGES) * T::STAGE_WORDS;
-        double *sb = sa + T::A_ELEMS * W;
-        const int64_t k0 = k_begin + int64_t(kt) * T::BK;
-        gather_tile<T::BM, T::BK, T::THREADS, EB>(reinterpret_cast<char *>(sa), static_cast<const char *>(p.A),
-                                                  rowA, p.offA_k, rows_valid, k0, k_end, p.dirA, p.vecA,
-                                                  a_srow, a_sk, tid);
-        gather_tile<T::BN, T::BK, T::THREADS, EB>(reinterpret_cast<char *>(sb), static_cast<const char *>(p.B),
-                                                  colB, p.offB_k, cols_valid, k0, k_end, p.dirB, p.vecB,
-                                                  b_srow, b_sk, tid);
-    };
+    if (warp < kProducerWarps) {
+        // ------------------------------------------------------------------ producers
+        if (T::REBALANCE_REGS) reg_dec<40>();
+        const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
+        for (int kt = 0; kt < num_kt; ++kt) {
+            const int s = kt % T::STAGES, round = kt / T::STAGES;
+            if (round > 0 &&
+                !mbar_wait_bounded(empty0 + 8u * s, unsigned(round - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait))
+                break;
+            const unsigned sa = stage0 + unsigned(s) * (T::STAGE_WORDS * 8);
+            const unsigned sb = sa + T::A_ELEMS * EB;
+            const int64_t k0 = k_begin + int64_t(kt) * T::BK;
+            gather_dispatch<T::BM, T::BK, T::PRODUCER_THREADS, EB>(sa, static_cast<const char *>(p.A), rowA, p.offA_k,
+                                                                   rows_valid, k0, k_end, p.dirA, p.vecA, a_srow, a_sk, tid);
+            gather_dispatch<T::BN, T::BK, T::PRODUCER_THREADS, EB>(sb, static_cast<const char *>(p.B), colB, p.offB_k,
+                                                                   cols_valid, k0, k_end, p.dirB, p.vecB, b_srow, b_sk, tid);
+            mbar_arrive_on_copies(full0 + 8u * s);
+        }
+        cp_async_wait_all();
+        return;
+    }
 
-    const int warp_m = warp % T::WARPS_M, warp_n = warp / T::WARPS_M;
+    // ---------------------------------------------------------------------- consumers
+    if (T::REBALANCE_REGS) reg_inc<232>();
+    const int cw = warp - kProducerWarps;
+    const int ctid = tid - T::PRODUCER_THREADS;
+    const int warp_m = cw % T::WARPS_M, warp_n = cw / T::WARPS_M;
     const int wm0 = warp_m * T::WM;
     const int wn0w = warp_n * T::WNR;            // first real-word column of the warp tile
     const int g = lane >> 2, t = lane & 3;
@@ -245,19 +347,14 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_f64_kernel(const TiledPar
 #pragma unroll
         for (int j = 0; j < T::FN; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
 
-#pragma unroll
-    for (int s = 0; s < T::STAGES - 1; ++s) {
-        if (s < num_kt) load_stage(s);
-        cp_async_commit();
-    }
-
+    bool ok = true;
     for (int kt = 0; kt < num_kt; ++kt) {
-        cp_async_wait<T::STAGES - 2>();
-        __syncthreads();
-        if (kt + T::STAGES - 1 < num_kt) load_stage(kt + T::STAGES - 1);
-        cp_async_commit();
-
-        const double *sa = stage_base + size_t(kt % T::STAGES) * T::STAGE_WORDS;
+        const int s = kt % T::STAGES, round = kt / T::STAGES;
+        if (!mbar_wait_bounded(full0 + 8u * s, unsigned(round) & 1u, abort_flag, p.error_word, kErrFullWait)) {
+            ok = false;
+            break;
+        }
+        const double *sa = stage_base + size_t(s) * T::STAGE_WORDS;
         const double *sb = sa + T::A_ELEMS * W;
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {         // 16 real k per stage, 4 per MMA
@@ -278,29 +375,31 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_f64_kernel(const TiledPar
 #pragma unroll
                 for (int j = 0; j < T::FN; ++j) dmma_m8n8k4(acc[i][j][0], acc[i][j][1], af[i], bf[j]);
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8u * s);
     }
-    cp_async_wait<0>();
+    if (!ok) return;
 
     if (p.split_k == 1) {
         epilogue<T>(p, acc, rowD, colD, rows_valid, cols_valid, wm0, wn0w, lane);
     } else {
-        // raw accumulators -> scratch, [batch][slice][tile][acc index][thread]
+        // raw accumulators -> scratch, [batch][slice][tile][acc index][consumer thread]
         double *ws = static_cast<double *>(p.partials);
-        const size_t tile_lin = blockIdx.x;
-        double *dst = ws + tile_lin * (size_t(T::THREADS) * T::ACC) + tid;
+        double *dst = ws + size_t(blockIdx.x) * (size_t(T::CONSUMER_THREADS) * T::ACC) + ctid;
 #pragma unroll
         for (int i = 0; i < T::FM; ++i)
 #pragma unroll
             for (int j = 0; j < T::FN; ++j) {
-                dst[size_t((i * T::FN + j) * 2 + 0) * T::THREADS] = acc[i][j][0];
-                dst[size_t((i * T::FN + j) * 2 + 1) * T::THREADS] = acc[i][j][1];
+                dst[size_t((i * T::FN + j) * 2 + 0) * T::CONSUMER_THREADS] = acc[i][j][0];
+                dst[size_t((i * T::FN + j) * 2 + 1) * T::CONSUMER_THREADS] = acc[i][j][1];
             }
     }
 }
 
 // Second pass of split-K: fixed-order sum of the slices, then alpha/beta and the strided store.
+// Launched with T::CONSUMER_THREADS threads: thread i takes over consumer thread i's accumulators.
 template <typename T>
-__global__ void __launch_bounds__(T::THREADS) tiled_f64_splitk_reduce_kernel(const TiledParams p)
+__global__ void __launch_bounds__(T::CONSUMER_THREADS) tiled_f64_splitk_reduce_kernel(const TiledParams p)
 {
     __shared__ int64_t rowD[T::BM];
     __shared__ int64_t colD[T::BN];
@@ -315,8 +414,8 @@ __global__ void __launch_bounds__(T::THREADS) tiled_f64_splitk_reduce_kernel(con
     const int rows_valid = int(imin64(T::BM, p.M - m0));
     const int cols_valid = int(imin64(T::BN, p.N - n0));
     const int64_t hD = p.offD_h[h];
-    for (int i = tid; i < T::BM; i += T::THREADS) rowD[i] = i < rows_valid ? p.offD_m[m0 + i] + hD : 0;
-    for (int i = tid; i < T::BN; i += T::THREADS) colD[i] = i < cols_valid ? p.offD_n[n0 + i] : 0;
+    for (int i = tid; i < T::BM; i += T::CONSUMER_THREADS) rowD[i] = i < rows_valid ? p.offD_m[m0 + i] + hD : 0;
+    for (int i = tid; i < T::BN; i += T::CONSUMER_THREADS) colD[i] = i < cols_valid ? p.offD_n[n0 + i] : 0;
     __syncthreads();
 
     double acc[T::FM][T::FN][2];
@@ -328,13 +427,13 @@ __global__ void __launch_bounds__(T::THREADS) tiled_f64_splitk_reduce_kernel(con
     const size_t tiles = size_t(p.tiles_m) * p.tiles_n;
     for (int ks = 0; ks < p.split_k; ++ks) {
         const size_t tile_lin = (size_t(h) * p.split_k + ks) * tiles + tile;
-        const double *src = ws + tile_lin * (size_t(T::THREADS) * T::ACC) + tid;
+        const double *src = ws + tile_lin * (size_t(T::CONSUMER_THREADS) * T::ACC) + tid;
 #pragma unroll
         for (int i = 0; i < T::FM; ++i)
 #pragma unroll
             for (int j = 0; j < T::FN; ++j) {
-                acc[i][j][0] += src[size_t((i * T::FN + j) * 2 + 0) * T::THREADS];
-                acc[i][j][1] += src[size_t((i * T::FN + j) * 2 + 1) * T::THREADS];
+                acc[i][j][0] += src[size_t((i * T::FN + j) * 2 + 0) * T::CONSUMER_THREADS];
+                acc[i][j][1] += src[size_t((i * T::FN + j) * 2 + 1) * T::CONSUMER_THREADS];
             }
     }
     const int warp_m = warp % T::WARPS_M, warp_n = warp / T::WARPS_M;
