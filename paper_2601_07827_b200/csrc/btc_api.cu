@@ -12,6 +12,7 @@
 #include "generic_kernel.cuh"
 #include "kernel_params.h"
 #include "plan.h"
+#include "tiled_f32_kernel.cuh"
 #include "tiled_f64_kernel.cuh"
 
 using namespace btc;
@@ -55,41 +56,81 @@ using F64Small = F64Tile<false, 64, 64, 2, 2, 4, 2>;
 using C64Big = F64Tile<true, 128, 64, 2, 4, 4, 1>;
 using C64Small = F64Tile<true, 64, 32, 2, 2, 4, 2>;
 
+using F32Big = F32Tile<128, 128, 2, 4, 5, 1>;
+using F32Small = F32Tile<64, 64, 2, 2, 5, 2>;
+
 struct VariantInfo {
     int bm, bn, bk, threads, acc;
-    size_t smem;
+    size_t smem, acc_bytes;
 };
 // `threads` counts the consumer threads: they own the accumulators (split-K scratch layout)
-template <typename T> VariantInfo info_of() { return {T::BM, T::BN, T::BK, T::CONSUMER_THREADS, T::ACC, T::SMEM_BYTES}; }
+template <typename T> VariantInfo info_of(size_t acc_bytes)
+{
+    return {T::BM, T::BN, T::BK, T::CONSUMER_THREADS, T::ACC, T::SMEM_BYTES, acc_bytes};
+}
 
-bool tiled_supported(btc_dtype_t t) { return t == BTC_F64 || t == BTC_C64; }
+bool tiled_supported(btc_dtype_t t) { return t == BTC_F64 || t == BTC_C64 || t == BTC_F32; }
 
 VariantInfo variant_info(btc_dtype_t t, int variant)
 {
-    if (t == BTC_F64) return variant == 0 ? info_of<F64Big>() : info_of<F64Small>();
-    return variant == 0 ? info_of<C64Big>() : info_of<C64Small>();
+    if (t == BTC_F64) return variant == 0 ? info_of<F64Big>(8) : info_of<F64Small>(8);
+    if (t == BTC_F32) return variant == 0 ? info_of<F32Big>(4) : info_of<F32Small>(4);
+    return variant == 0 ? info_of<C64Big>(8) : info_of<C64Small>(8);
+}
+
+template <typename K>
+cudaError_t set_smem_once(K kernel, size_t bytes, bool *configured)
+{
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes));
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    return cudaSuccess;
 }
 
 template <typename T>
 cudaError_t launch_tiled(const TiledParams &p, int64_t ctas, int64_t reduce_ctas, cudaStream_t st)
 {
     static bool configured[64] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(tiled_f64_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             int(T::SMEM_BYTES));
-        if (e != cudaSuccess) return e;
-        configured[dev] = true;
-    }
+    cudaError_t e = set_smem_once(tiled_f64_kernel<T>, T::SMEM_BYTES, configured);
+    if (e != cudaSuccess) return e;
     tiled_f64_kernel<T><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
-    cudaError_t e = cudaGetLastError();
+    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (p.split_k > 1) {
         tiled_f64_splitk_reduce_kernel<T><<<unsigned(reduce_ctas), T::CONSUMER_THREADS, 0, st>>>(p);
         e = cudaGetLastError();
     }
     return e;
+}
+
+template <typename T, bool AK, bool BK_>
+cudaError_t launch_tiled_f32_o(const TiledParams &p, int64_t ctas, int64_t reduce_ctas, cudaStream_t st)
+{
+    static bool configured[64] = {};
+    cudaError_t e = set_smem_once(tiled_f32_kernel<T, AK, BK_>, T::SMEM_BYTES, configured);
+    if (e != cudaSuccess) return e;
+    tiled_f32_kernel<T, AK, BK_><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (p.split_k > 1) {
+        tiled_f32_splitk_reduce_kernel<T, AK, BK_><<<unsigned(reduce_ctas), T::CONSUMER_THREADS, 0, st>>>(p);
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+// the shared-memory orientation of each operand is a compile-time property of the fp32 kernel
+template <typename T>
+cudaError_t launch_tiled_f32(const TiledParams &p, int64_t ctas, int64_t reduce_ctas, cudaStream_t st)
+{
+    if (p.dirA) return p.dirB ? launch_tiled_f32_o<T, true, true>(p, ctas, reduce_ctas, st)
+                              : launch_tiled_f32_o<T, true, false>(p, ctas, reduce_ctas, st);
+    return p.dirB ? launch_tiled_f32_o<T, false, true>(p, ctas, reduce_ctas, st)
+                  : launch_tiled_f32_o<T, false, false>(p, ctas, reduce_ctas, st);
 }
 
 void to_double2(btc_dtype_t t, const void *src, double out[2])
@@ -144,7 +185,7 @@ int finish_plan(btc_contraction_s *op)
     if (double(tiles_for(variant_info(pl.dtype, 0))) < 0.8 * sms) variant = 1;
     const VariantInfo v = variant_info(pl.dtype, variant);
     pl.tile.bm = v.bm; pl.tile.bn = v.bn; pl.tile.bk = v.bk; pl.tile.threads = v.threads;
-    pl.tile.stages = 4; pl.tile.variant = variant;
+    pl.tile.stages = pl.dtype == BTC_F32 ? 5 : 4; pl.tile.variant = variant;
     op->tiles_m = int32_t((pl.M + v.bm - 1) / v.bm);
     op->tiles_n = int32_t((pl.N + v.bn - 1) / v.bn);
     op->raster_n_fast = op->tiles_n <= op->tiles_m ? 1 : 0;
@@ -167,7 +208,7 @@ int finish_plan(btc_contraction_s *op)
     if (tiles * split > 0x7fffffffLL) return BTC_ERR_NOT_SUPPORTED;
     op->grid[0] = int32_t(tiles * split); op->grid[1] = 1; op->grid[2] = 1;
     if (split > 1)
-        op->workspace_bytes = size_t(tiles) * size_t(split) * size_t(v.threads) * size_t(v.acc) * sizeof(double);
+        op->workspace_bytes = size_t(tiles) * size_t(split) * size_t(v.threads) * size_t(v.acc) * v.acc_bytes;
 
     if (op->handle.device >= 0) {
         const std::vector<int64_t> *tabs[9] = {&pl.offA_m, &pl.offD_m, &pl.offB_n, &pl.offD_n, &pl.offA_k,
@@ -488,7 +529,12 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         tp.error_word = op->d_error;
         const int64_t ctas = op->grid[0];
         const int64_t reduce_ctas = ctas / pl.split_k;
-        if (pl.dtype == BTC_F64)
+        // 16-byte stores of D (and loads of C) need those base pointers aligned too
+        tp.vecD = (pl.vecD == 4 && !misaligned(D, 16) && !(use_c && misaligned(C, 16))) ? 4 : 1;
+        if (pl.dtype == BTC_F32)
+            ce = pl.tile.variant == 0 ? launch_tiled_f32<F32Big>(tp, ctas, reduce_ctas, st)
+                                      : launch_tiled_f32<F32Small>(tp, ctas, reduce_ctas, st);
+        else if (pl.dtype == BTC_F64)
             ce = pl.tile.variant == 0 ? launch_tiled<F64Big>(tp, ctas, reduce_ctas, st)
                                       : launch_tiled<F64Small>(tp, ctas, reduce_ctas, st);
         else

@@ -36,6 +36,7 @@ struct TiledParams {
     int64_t k_per_split;              // multiple of the K tile
     int32_t dirA, dirB;               // 0: threads run along the free index, 1: along k
     int32_t vecA, vecB;               // elements per global->shared copy
+    int32_t vecD;                     // 4: four consecutive m are 16 consecutive, aligned bytes of D (fp32)
     int32_t conjA, conjB, conjC;
     int32_t use_c;
     double alpha[2], beta[2];

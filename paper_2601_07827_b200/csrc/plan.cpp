@@ -306,7 +306,15 @@ int make_plan(const PlanRequest &req, Plan &plan)
     plan.vecB = vec_for(false, plan.dirB);
     plan.alignA = plan.vecA * esz;
     plan.alignB = plan.vecB * esz;
-    plan.vecD = (!plan.m.empty() && plan.m[0].sD == 1) ? 1 : 0;
+    // consecutive m that are consecutive in D: lets the fp32 epilogue store 16 bytes at a time
+    plan.vecD = 1;
+    if (esz == 4 && !plan.m.empty() && plan.m[0].sD == 1 && plan.m[0].extent % 4 == 0) {
+        bool ok = true;
+        for (size_t i = 1; i < plan.m.size(); ++i) ok = ok && plan.m[i].sD % 4 == 0;
+        for (auto &md : plan.n) ok = ok && md.sD % 4 == 0;
+        for (auto &md : plan.batch) ok = ok && md.sD % 4 == 0;
+        if (ok) plan.vecD = 4;
+    }
 
     // ---- kernel choice ----
     const int64_t entries = 2 * (plan.M + plan.N + plan.K) + 3 * plan.Bt;

@@ -53,7 +53,7 @@ struct Plan {
     int32_t split_k = 1;
     LoadDir dirA = LoadDir::ALONG_FREE, dirB = LoadDir::ALONG_FREE;
     int32_t vecA = 1, vecB = 1;          // elements per global load that the strides allow
-    int32_t vecD = 1;                    // consecutive m that are consecutive in D (0/1 flag use)
+    int32_t vecD = 1;                    // 4: groups of four consecutive m are 16 aligned bytes of D
     int64_t alignA = 1, alignB = 1;      // required base-pointer alignment (bytes) for vecA / vecB
 
     // element-offset tables (host copies; the API object uploads them)

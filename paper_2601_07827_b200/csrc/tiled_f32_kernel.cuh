@@ -1,0 +1,252 @@
+// Transpose-free tiled contraction kernel for fp32 on the FP32 FMA pipe (sm_100a).
+//
+// Same structure as the fp64 kernel: a producer warpgroup gathers strided BM x BK / BK x BN
+// tiles of A and B with cp.async into whichever shared-memory orientation matches the operand's
+// contiguous direction, consumer warps do the arithmetic, mbarriers hand stages over.  The
+// consumers keep a TM x TN register tile per thread.  An operand stored with the free index
+// contiguous is read one k at a time as 16-byte vectors over 4 consecutive rows; an operand
+// stored with k contiguous is read 4 k at a time, one 16-byte vector per row, with the rows of a
+// thread interleaved (row = lane row + 8 i) so that the vector loads of a quarter warp fall into
+// distinct banks.  Both orientations therefore cost the same number of shared-memory loads per
+// FMA, and neither needs a transposed copy of the operand.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "kernel_params.h"
+#include "tile_common.cuh"
+
+namespace btc {
+
+template <int BM_, int BN_, int WARPS_M_, int WARPS_N_, int STAGES_, int MIN_CTAS_>
+struct F32Tile {
+    static constexpr int BM = BM_, BN = BN_, BK = 16;
+    static constexpr int WARPS_M = WARPS_M_, WARPS_N = WARPS_N_;
+    static constexpr int CONSUMER_WARPS = WARPS_M_ * WARPS_N_;
+    static constexpr int CONSUMER_THREADS = 32 * CONSUMER_WARPS;
+    static constexpr int PRODUCER_THREADS = 32 * kProducerWarps;
+    static constexpr int THREADS = CONSUMER_THREADS + PRODUCER_THREADS;
+    static constexpr int MIN_CTAS = MIN_CTAS_;
+    static constexpr bool REBALANCE_REGS = (THREADS == 384);
+    static constexpr int STAGES = STAGES_;
+    static constexpr int WM = BM / WARPS_M, WN = BN / WARPS_N;
+    static constexpr int TM = WM / 8, TN = WN / 4;    // a warp is 8 (rows) x 4 (columns) threads
+    static constexpr int ACC = TM * TN;
+    static_assert(TM % 4 == 0 && TN % 4 == 0, "register tile must be made of 4-vectors");
+    // pitches in floats: multiples of 4 (16-byte vectors); the k-contiguous pitch 20 puts the
+    // 8 (or 4) rows a quarter warp reads into distinct banks
+    static constexpr int PITCH_FREE_A = BM + 4, PITCH_FREE_B = BN + 4, PITCH_K = BK + 4;
+    static constexpr int A_ELEMS = (BK * PITCH_FREE_A > BM * PITCH_K) ? BK * PITCH_FREE_A : BM * PITCH_K;
+    static constexpr int B_ELEMS = (BK * PITCH_FREE_B > BN * PITCH_K) ? BK * PITCH_FREE_B : BN * PITCH_K;
+    static constexpr int STAGE_FLOATS = A_ELEMS + B_ELEMS;
+    static constexpr size_t SMEM_BYTES =
+        size_t(STAGES) * STAGE_FLOATS * 4 + size_t(2 * BM + 2 * BN) * 8 + size_t(2 * STAGES) * 8 + 16;
+};
+
+// tile-local row of register-tile entry i (and column of entry j) for the two orientations
+template <bool KMAJ> __device__ __forceinline__ int f32_row_of(int ty, int i)
+{
+    return KMAJ ? ty + 8 * i : (i >> 2) * 32 + ty * 4 + (i & 3);
+}
+template <bool KMAJ> __device__ __forceinline__ int f32_col_of(int tx, int j)
+{
+    return KMAJ ? tx + 4 * j : (j >> 2) * 16 + tx * 4 + (j & 3);
+}
+
+template <typename T, bool A_KMAJ>
+__device__ __forceinline__ void f32_epilogue(const TiledParams &p, const float (&acc)[T::TM][T::TN],
+                                             const int64_t *rowD, const int64_t *colD, int rows_valid,
+                                             int cols_valid, int wm0, int wn0, int ty, int tx, bool b_kmaj)
+{
+    float *D = static_cast<float *>(p.D);
+    const float *C = static_cast<const float *>(p.C);
+    const float alpha = float(p.alpha[0]), beta = float(p.beta[0]);
+#pragma unroll
+    for (int j = 0; j < T::TN; ++j) {
+        const int c = wn0 + (b_kmaj ? f32_col_of<true>(tx, j) : f32_col_of<false>(tx, j));
+        if (c >= cols_valid) continue;
+        const int64_t co = colD[c];
+        if (!A_KMAJ && p.vecD == 4) {
+            // 4 consecutive rows of this thread are 4 consecutive, 16-byte aligned floats of D
+#pragma unroll
+            for (int i4 = 0; i4 < T::TM / 4; ++i4) {
+                const int r = wm0 + f32_row_of<false>(ty, i4 * 4);
+                if (r >= rows_valid) continue;     // rows_valid is a multiple of 4 here
+                const int64_t off = rowD[r] + co;
+                float4 v = make_float4(alpha * acc[i4 * 4][j], alpha * acc[i4 * 4 + 1][j],
+                                       alpha * acc[i4 * 4 + 2][j], alpha * acc[i4 * 4 + 3][j]);
+                if (p.use_c) {
+                    const float4 cv = *reinterpret_cast<const float4 *>(C + off);
+                    v.x += beta * cv.x; v.y += beta * cv.y; v.z += beta * cv.z; v.w += beta * cv.w;
+                }
+                *reinterpret_cast<float4 *>(D + off) = v;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < T::TM; ++i) {
+                const int r = wm0 + f32_row_of<A_KMAJ>(ty, i);
+                if (r >= rows_valid) continue;
+                const int64_t off = rowD[r] + co;
+                float v = alpha * acc[i][j];
+                if (p.use_c) v += beta * C[off];
+                D[off] = v;
+            }
+        }
+    }
+}
+
+template <typename T, bool A_KMAJ, bool B_KMAJ>
+__global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f32_kernel(const TiledParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *stage_base = reinterpret_cast<float *>(smem_raw);
+    int64_t *rowA = reinterpret_cast<int64_t *>(stage_base + size_t(T::STAGES) * T::STAGE_FLOATS);
+    int64_t *rowD = rowA + T::BM;
+    int64_t *colB = rowD + T::BM;
+    int64_t *colD = colB + T::BN;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(colD + T::BN);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * T::STAGES);
+    const unsigned full0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
+    const unsigned empty0 = full0 + 8u * T::STAGES;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
+    tile_setup<T::BM, T::BN, T::STAGES, T::THREADS, T::PRODUCER_THREADS, T::CONSUMER_WARPS>(
+        p, tc, rowA, rowD, colB, colD, full0, empty0, abort_flag, tid);
+
+    constexpr int a_srow = A_KMAJ ? T::PITCH_K : 1, a_sk = A_KMAJ ? 1 : T::PITCH_FREE_A;
+    constexpr int b_srow = B_KMAJ ? T::PITCH_K : 1, b_sk = B_KMAJ ? 1 : T::PITCH_FREE_B;
+
+    if (warp < kProducerWarps) {
+        if (T::REBALANCE_REGS) reg_dec<40>();
+        const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
+        producer_loop<T::BM, T::BN, T::BK, 4, T::STAGES, T::STAGE_FLOATS * 4, T::A_ELEMS * 4, T::PRODUCER_THREADS>(
+            p, tc, stage0, rowA, colB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
+        return;
+    }
+
+    if (T::REBALANCE_REGS) reg_inc<232>();
+    const int cw = warp - kProducerWarps;
+    const int ctid = tid - T::PRODUCER_THREADS;
+    const int wm0 = (cw % T::WARPS_M) * T::WM, wn0 = (cw / T::WARPS_M) * T::WN;
+    const int ty = lane >> 2, tx = lane & 3;
+
+    float acc[T::TM][T::TN];
+#pragma unroll
+    for (int i = 0; i < T::TM; ++i)
+#pragma unroll
+        for (int j = 0; j < T::TN; ++j) acc[i][j] = 0.f;
+
+    bool ok = true;
+    for (int kt = 0; kt < tc.num_kt; ++kt) {
+        const int s = kt % T::STAGES, round = kt / T::STAGES;
+        if (!mbar_wait_bounded(full0 + 8u * s, unsigned(round) & 1u, abort_flag, p.error_word, kErrFullWait)) {
+            ok = false;
+            break;
+        }
+        const float *sa = stage_base + size_t(s) * T::STAGE_FLOATS;
+        const float *sb = sa + T::A_ELEMS;
+#pragma unroll
+        for (int k4 = 0; k4 < T::BK; k4 += 4) {
+            float4 a4[A_KMAJ ? T::TM : 1], b4[B_KMAJ ? T::TN : 1];
+            if (A_KMAJ) {
+#pragma unroll
+                for (int i = 0; i < T::TM; ++i)
+                    a4[i] = *reinterpret_cast<const float4 *>(sa + (wm0 + ty + 8 * i) * T::PITCH_K + k4);
+            }
+            if (B_KMAJ) {
+#pragma unroll
+                for (int j = 0; j < T::TN; ++j)
+                    b4[j] = *reinterpret_cast<const float4 *>(sb + (wn0 + tx + 4 * j) * T::PITCH_K + k4);
+            }
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                float a[T::TM], b[T::TN];
+                if (A_KMAJ) {
+#pragma unroll
+                    for (int i = 0; i < T::TM; ++i)
+                        a[i] = kk == 0 ? a4[i].x : kk == 1 ? a4[i].y : kk == 2 ? a4[i].z : a4[i].w;
+                } else {
+#pragma unroll
+                    for (int i4 = 0; i4 < T::TM / 4; ++i4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(
+                            sa + (k4 + kk) * T::PITCH_FREE_A + wm0 + i4 * 32 + ty * 4);
+                        a[i4 * 4] = v.x; a[i4 * 4 + 1] = v.y; a[i4 * 4 + 2] = v.z; a[i4 * 4 + 3] = v.w;
+                    }
+                }
+                if (B_KMAJ) {
+#pragma unroll
+                    for (int j = 0; j < T::TN; ++j)
+                        b[j] = kk == 0 ? b4[j].x : kk == 1 ? b4[j].y : kk == 2 ? b4[j].z : b4[j].w;
+                } else {
+#pragma unroll
+                    for (int j4 = 0; j4 < T::TN / 4; ++j4) {
+                        const float4 v = *reinterpret_cast<const float4 *>(
+                            sb + (k4 + kk) * T::PITCH_FREE_B + wn0 + j4 * 16 + tx * 4);
+                        b[j4 * 4] = v.x; b[j4 * 4 + 1] = v.y; b[j4 * 4 + 2] = v.z; b[j4 * 4 + 3] = v.w;
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < T::TM; ++i)
+#pragma unroll
+                    for (int j = 0; j < T::TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8u * s);
+    }
+    if (!ok) return;
+
+    if (p.split_k == 1) {
+        f32_epilogue<T, A_KMAJ>(p, acc, rowD, colD, tc.rows_valid, tc.cols_valid, wm0, wn0, ty, tx, B_KMAJ);
+    } else {
+        // raw accumulators -> scratch, [batch][slice][tile][acc index][consumer thread]
+        float *dst = static_cast<float *>(p.partials) + size_t(blockIdx.x) * (size_t(T::CONSUMER_THREADS) * T::ACC) + ctid;
+#pragma unroll
+        for (int i = 0; i < T::TM; ++i)
+#pragma unroll
+            for (int j = 0; j < T::TN; ++j) dst[size_t(i * T::TN + j) * T::CONSUMER_THREADS] = acc[i][j];
+    }
+}
+
+// Second pass of split-K (fixed-order sum of the slices, alpha/beta, strided store); thread i
+// takes over consumer thread i's accumulators.
+template <typename T, bool A_KMAJ, bool B_KMAJ>
+__global__ void __launch_bounds__(T::CONSUMER_THREADS) tiled_f32_splitk_reduce_kernel(const TiledParams p)
+{
+    __shared__ int64_t rowD[T::BM];
+    __shared__ int64_t colD[T::BN];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tiles_i = p.tiles_m * p.tiles_n;
+    const int tile = blockIdx.x % tiles_i;
+    const int64_t h = blockIdx.x / tiles_i;
+    const int tile_m = p.raster_n_fast ? tile / p.tiles_n : tile % p.tiles_m;
+    const int tile_n = p.raster_n_fast ? tile % p.tiles_n : tile / p.tiles_m;
+    const int64_t m0 = int64_t(tile_m) * T::BM, n0 = int64_t(tile_n) * T::BN;
+    const int rows_valid = int(imin64(T::BM, p.M - m0));
+    const int cols_valid = int(imin64(T::BN, p.N - n0));
+    const int64_t hD = p.offD_h[h];
+    for (int i = tid; i < T::BM; i += T::CONSUMER_THREADS) rowD[i] = i < rows_valid ? p.offD_m[m0 + i] + hD : 0;
+    for (int i = tid; i < T::BN; i += T::CONSUMER_THREADS) colD[i] = i < cols_valid ? p.offD_n[n0 + i] : 0;
+    __syncthreads();
+
+    float acc[T::TM][T::TN];
+#pragma unroll
+    for (int i = 0; i < T::TM; ++i)
+#pragma unroll
+        for (int j = 0; j < T::TN; ++j) acc[i][j] = 0.f;
+    const float *ws = static_cast<const float *>(p.partials);
+    const size_t tiles = size_t(tiles_i);
+    for (int ks = 0; ks < p.split_k; ++ks) {
+        const size_t tile_lin = (size_t(h) * p.split_k + ks) * tiles + tile;
+        const float *src = ws + tile_lin * (size_t(T::CONSUMER_THREADS) * T::ACC) + tid;
+#pragma unroll
+        for (int i = 0; i < T::TM; ++i)
+#pragma unroll
+            for (int j = 0; j < T::TN; ++j) acc[i][j] += src[size_t(i * T::TN + j) * T::CONSUMER_THREADS];
+    }
+    const int wm0 = (warp % T::WARPS_M) * T::WM, wn0 = (warp / T::WARPS_M) * T::WN;
+    f32_epilogue<T, A_KMAJ>(p, acc, rowD, colD, rows_valid, cols_valid, wm0, wn0, lane >> 2, lane & 3, B_KMAJ);
+}
+
+}  // namespace btc

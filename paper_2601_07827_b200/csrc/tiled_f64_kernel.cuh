@@ -29,10 +29,9 @@
 #include <cuda_runtime.h>
 
 #include "kernel_params.h"
+#include "tile_common.cuh"
 
 namespace btc {
-
-constexpr int kProducerWarps = 4;   // one warpgroup
 
 template <bool CPLX_, int BM_, int BN_, int WARPS_M_, int WARPS_N_, int STAGES_, int MIN_CTAS_>
 struct F64Tile {
@@ -68,110 +67,10 @@ struct F64Tile {
         size_t(STAGES) * STAGE_WORDS * 8 + size_t(2 * BM + 2 * BN) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
 
-__device__ __forceinline__ int64_t imin64(int64_t a, int64_t b) { return a < b ? a : b; }
-
-// ---- asynchronous copies and mbarriers ---------------------------------------------------------
-template <int BYTES>
-__device__ __forceinline__ void cp_async_bytes(unsigned dst, const void *gsrc, bool valid)
-{
-    const int src = valid ? BYTES : 0;   // src-size 0 zero-fills the destination
-    if (BYTES == 16)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
-    else if (BYTES == 8)
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
-    else
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(gsrc), "r"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-
-__device__ __forceinline__ void mbar_init(unsigned bar, int count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// the barrier receives one arrival from this thread once all its earlier cp.async have landed
-__device__ __forceinline__ void mbar_arrive_on_copies(unsigned bar)
-{
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                 "selp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-
-constexpr unsigned kWaitPollLimit = 1u << 22;   // polls before a wait gives up (a poll itself blocks briefly)
-constexpr int kErrFullWait = 1, kErrEmptyWait = 2;
-
-// Bounded wait.  Returns false when it gave up or another warp raised the abort flag.
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, volatile int *abort_flag,
-                                                  int *error_word, int code)
-{
-    for (unsigned n = 0; n < kWaitPollLimit; ++n) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((n & 255u) == 255u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    if (error_word) atomicCAS(error_word, 0, code);
-    return false;
-}
-
 __device__ __forceinline__ void dmma_m8n8k4(double &c0, double &c1, double a, double b)
 {
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
                  : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
-}
-
-template <int REGS> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS)); }
-template <int REGS> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS)); }
-
-// Gather one ROWS x BK tile (rows = free index, columns = k) into shared memory.
-//   DIR       0: consecutive threads take consecutive rows; 1: consecutive k
-//   VEC       elements per copy along that direction
-//   row_off   shared array: element offset of each tile row (batch offset included)
-//   koff      global table of k offsets;  [.., k_end) is this CTA's valid k range
-//   s_row, s_k  shared-memory strides of the tile in elements
-template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES, int DIR, int VEC>
-__device__ __forceinline__ void gather_tile(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
-                                            const int64_t *__restrict__ koff, int rows_valid, int64_t k0,
-                                            int64_t k_end, int s_row, int s_k, int tid)
-{
-    constexpr int NFAST = (DIR == 0 ? ROWS : BK) / VEC;
-    constexpr int SLOTS = ROWS * BK / VEC;
-#pragma unroll 4
-    for (int s = tid; s < SLOTS; s += NTHREADS) {
-        const int f = (s % NFAST) * VEC, o = s / NFAST;
-        const int r = DIR == 0 ? f : o;
-        const int k = DIR == 0 ? o : f;
-        const bool valid = (r < rows_valid) && (k0 + k < k_end);
-        const int64_t off = valid ? row_off[r] + __ldg(koff + k0 + k) : 0;
-        cp_async_bytes<VEC * ELEM_BYTES>(smem + unsigned(r * s_row + k * s_k) * ELEM_BYTES, g + off * ELEM_BYTES, valid);
-    }
-}
-
-template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES>
-__device__ __forceinline__ void gather_dispatch(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
-                                                const int64_t *__restrict__ koff, int rows_valid, int64_t k0,
-                                                int64_t k_end, int dir, int vec, int s_row, int s_k, int tid)
-{
-    constexpr int VMAX = 16 / ELEM_BYTES;   // 2 for fp64, 1 for complex128
-    if (dir == 0) {
-        if (VMAX > 1 && vec == VMAX)
-            gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, 0, VMAX>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
-        else
-            gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, 0, 1>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
-    } else {
-        if (VMAX > 1 && vec == VMAX)
-            gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, 1, VMAX>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
-        else
-            gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, 1, 1>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
-    }
 }
 
 // alpha * acc + beta * op(c) for one element, written through D's offsets
@@ -241,42 +140,10 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     const unsigned empty0 = full0 + 8u * T::STAGES;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // blockIdx.x enumerates (tile, k slice, batch), tile fastest
-    const int tiles = p.tiles_m * p.tiles_n;
-    const int tile = blockIdx.x % tiles;
-    const int ks = (blockIdx.x / tiles) % p.split_k;
-    const int64_t h = blockIdx.x / (tiles * p.split_k);
-    const int tile_m = p.raster_n_fast ? tile / p.tiles_n : tile % p.tiles_m;
-    const int tile_n = p.raster_n_fast ? tile % p.tiles_n : tile / p.tiles_m;
-    const int64_t m0 = int64_t(tile_m) * T::BM, n0 = int64_t(tile_n) * T::BN;
-    const int rows_valid = int(imin64(T::BM, p.M - m0));
-    const int cols_valid = int(imin64(T::BN, p.N - n0));
-    const int64_t k_begin = int64_t(ks) * p.k_per_split;
-    const int64_t k_end = imin64(p.K, k_begin + p.k_per_split);
-    const int num_kt = int((k_end - k_begin + T::BK - 1) / T::BK);
-
-    // per-tile row/column offsets (batch offset folded in), barriers
-    {
-        const int64_t hA = p.offA_h[h], hB = p.offB_h[h], hD = p.offD_h[h];
-        for (int i = tid; i < T::BM; i += T::THREADS) {
-            const bool v = i < rows_valid;
-            rowA[i] = v ? p.offA_m[m0 + i] + hA : 0;
-            rowD[i] = v ? p.offD_m[m0 + i] + hD : 0;
-        }
-        for (int i = tid; i < T::BN; i += T::THREADS) {
-            const bool v = i < cols_valid;
-            colB[i] = v ? p.offB_n[n0 + i] + hB : 0;
-            colD[i] = v ? p.offD_n[n0 + i] : 0;
-        }
-        if (tid == 0) {
-            for (int s = 0; s < T::STAGES; ++s) {
-                mbar_init(full0 + 8u * s, T::PRODUCER_THREADS);
-                mbar_init(empty0 + 8u * s, T::CONSUMER_WARPS);
-            }
-            *abort_flag = 0;
-        }
-    }
-    __syncthreads();
+    const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
+    const int rows_valid = tc.rows_valid, cols_valid = tc.cols_valid, num_kt = tc.num_kt;
+    tile_setup<T::BM, T::BN, T::STAGES, T::THREADS, T::PRODUCER_THREADS, T::CONSUMER_WARPS>(
+        p, tc, rowA, rowD, colB, colD, full0, empty0, abort_flag, tid);
 
     // shared-memory orientation follows the load direction of each operand
     const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
@@ -286,21 +153,8 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
         // ------------------------------------------------------------------ producers
         if (T::REBALANCE_REGS) reg_dec<40>();
         const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
-        for (int kt = 0; kt < num_kt; ++kt) {
-            const int s = kt % T::STAGES, round = kt / T::STAGES;
-            if (round > 0 &&
-                !mbar_wait_bounded(empty0 + 8u * s, unsigned(round - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait))
-                break;
-            const unsigned sa = stage0 + unsigned(s) * (T::STAGE_WORDS * 8);
-            const unsigned sb = sa + T::A_ELEMS * EB;
-            const int64_t k0 = k_begin + int64_t(kt) * T::BK;
-            gather_dispatch<T::BM, T::BK, T::PRODUCER_THREADS, EB>(sa, static_cast<const char *>(p.A), rowA, p.offA_k,
-                                                                   rows_valid, k0, k_end, p.dirA, p.vecA, a_srow, a_sk, tid);
-            gather_dispatch<T::BN, T::BK, T::PRODUCER_THREADS, EB>(sb, static_cast<const char *>(p.B), colB, p.offB_k,
-                                                                   cols_valid, k0, k_end, p.dirB, p.vecB, b_srow, b_sk, tid);
-            mbar_arrive_on_copies(full0 + 8u * s);
-        }
-        cp_async_wait_all();
+        producer_loop<T::BM, T::BN, T::BK, EB, T::STAGES, T::STAGE_WORDS * 8, T::A_ELEMS * EB, T::PRODUCER_THREADS>(
+            p, tc, stage0, rowA, colB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
         return;
     }
 
