@@ -46,7 +46,8 @@ enum {
     BTC_ERR_MISALIGNED = 9,          /* a data pointer not aligned to its element size          */
     BTC_ERR_CUDA = 10,               /* a CUDA runtime call failed                              */
     BTC_ERR_DEVICE_TIMEOUT = 11,     /* a bounded device-side wait expired                      */
-    BTC_ERR_OUT_OF_MEMORY = 12
+    BTC_ERR_OUT_OF_MEMORY = 12,
+    BTC_ERR_SCRATCH_LIMIT = 13       /* needs more than the built-in scratch array holds        */
 };
 
 /* Element types.  Complex values are (re, im) pairs of the stated part width. */
@@ -155,6 +156,32 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream,
 btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream,
                              const void *alpha, const void *A, const void *B,
                              const void *beta, const void *C, void *D);
+
+/* Execute without allocating anything (the paper has no counterpart; this is a convenience of
+ * this library).  Same operation and argument meaning as btc_execute with DEVICE pointers, but
+ * the scratch that split-K plans need comes from an 8 MiB array that is part of the library's
+ * device image instead of a caller workspace, and no status object is created: the call makes
+ * no cudaMalloc / cudaFree, no host allocation and uses no allocating library routine.
+ *
+ * Who needs it: code that runs where device memory cannot be requested at that point -- a
+ * plug-in inside a host application that handed all device memory to its own pool, a real-time
+ * loop that may not pay for (or synchronise on) an allocation, a caller that only owns its
+ * inputs and outputs -- and that has no workspace of its own to pass to btc_execute.
+ *
+ * Limits and rules:
+ *   - operations whose btc_contraction_workspace_size exceeds 8 MiB (8 * 2^20 bytes) are refused
+ *     with BTC_ERR_SCRATCH_LIMIT before anything is enqueued; use btc_execute for those;
+ *   - the device that was current when the operation's handle was created must be current;
+ *   - the first call on each device looks up the array's device address (set-up, once per
+ *     device); make that first call before starting any stream capture;
+ *   - all calls on one device share the one array, and it keeps whatever the last call left in
+ *     it.  Nothing in it needs clearing (every partial sum is written before it is read), but
+ *     two calls that may run on the GPU at the same time (different streams, different host
+ *     threads) race on it: serialise them, e.g. by using one stream.
+ * Errors: as btc_execute, plus SCRATCH_LIMIT. */
+btc_error_t btc_execute_static_scratch(btc_contraction_t op, void *cuda_stream,
+                                       const void *alpha, const void *A, const void *B,
+                                       const void *beta, const void *C, void *D);
 
 /* Status object (Sec. "Status Objects"): metadata of one execute call. */
 enum {

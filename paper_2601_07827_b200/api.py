@@ -32,6 +32,7 @@ ERR_MISALIGNED = 9
 ERR_CUDA = 10
 ERR_DEVICE_TIMEOUT = 11
 ERR_OUT_OF_MEMORY = 12
+ERR_SCRATCH_LIMIT = 13
 
 F32, F64, C32, C64 = 0, 1, 2, 3
 DTYPE_SIZE = {F32: 4, F64: 8, C32: 8, C64: 16}
@@ -44,7 +45,8 @@ STATUS_KERNEL, STATUS_LAUNCHES, STATUS_GRID, STATUS_SPLIT_K = 1, 2, 3, 4
 EXPORTED = [
     "btc_create_handle", "btc_destroy_handle", "btc_create_tensor_info", "btc_destroy_tensor_info",
     "btc_create_contraction", "btc_destroy_contraction", "btc_contraction_workspace_size",
-    "btc_set_attr", "btc_get_attr", "btc_execute", "btc_execute_host", "btc_status_get",
+    "btc_set_attr", "btc_get_attr", "btc_execute", "btc_execute_host", "btc_execute_static_scratch",
+    "btc_status_get",
     "btc_destroy_status", "btc_explain_error",
 ]
 
@@ -63,6 +65,7 @@ _lib.btc_set_attr.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t]
 _lib.btc_get_attr.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
 _lib.btc_execute.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, ctypes.POINTER(_vp)]
 _lib.btc_execute_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.btc_execute_static_scratch.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.btc_status_get.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t]
 _lib.btc_destroy_status.argtypes = [ctypes.POINTER(_vp)]
 _lib.btc_explain_error.argtypes = [ctypes.c_int, ctypes.c_char_p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
@@ -237,6 +240,15 @@ class Contraction:
         """Host pointers as integers; copies in, runs, copies D back, synchronises."""
         _check(_lib.btc_execute_host(self._op, stream or None, _scalar(self.dtype, alpha), A or None, B or None,
                                      _scalar(self.dtype, beta), C or None, D or None), "btc_execute_host")
+
+    def execute_static_scratch(self, stream: int, A: int, B: int, C: Optional[int], D: int, alpha=None, beta=None):
+        """Like execute() with device pointers, for callers that can neither allocate device
+        memory nor bring a workspace: split-K scratch comes from the library's built-in 8 MiB
+        device array.  Calls that could overlap on the GPU must be serialised by the caller;
+        operations that need more scratch raise ERR_SCRATCH_LIMIT."""
+        _check(_lib.btc_execute_static_scratch(self._op, stream or None, _scalar(self.dtype, alpha), A or None,
+                                               B or None, _scalar(self.dtype, beta), C or None, D or None),
+               "btc_execute_static_scratch")
 
     def close(self):
         if self._op:

@@ -610,6 +610,38 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
     return rc;
 }
 
+// ---- execute without any allocation -------------------------------------------------------------
+// Scratch for split-K partial sums that belongs to the library image itself: every GPU that loads
+// the library holds these bytes until the process exits.
+#define BTC_STATIC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char btc_static_scratch[BTC_STATIC_SCRATCH_BYTES];
+
+btc_error_t btc_execute_static_scratch(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A,
+                                       const void *B, const void *beta, const void *C, void *D)
+{
+    // Device address of the array, looked up once per device.  In host code the array's name is
+    // only a stand-in for the symbol, never an address a kernel could use.
+    static void *scratch_of_device[64] = {};
+    if (!op || !D) return BTC_ERR_INVALID_ARGUMENT;
+    if (op->handle.device < 0) return BTC_ERR_CUDA;
+    if (op->workspace_bytes > size_t(BTC_STATIC_SCRATCH_BYTES)) return BTC_ERR_SCRATCH_LIMIT;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return BTC_ERR_CUDA; }
+    // the symbol's address differs per device: the operation's device must be the current one
+    if (dev != op->handle.device || dev < 0 || dev >= 64) return BTC_ERR_INVALID_ARGUMENT;
+    void *scratch = scratch_of_device[dev];
+    if (!scratch) {
+        if (cudaGetSymbolAddress(&scratch, btc_static_scratch) != cudaSuccess || !scratch) {
+            cudaGetLastError();
+            return BTC_ERR_CUDA;
+        }
+        scratch_of_device[dev] = scratch;   // racing first calls store the same value
+    }
+    // Every consumer thread of every CTA overwrites all of its partial sums before the reduction
+    // kernel reads them, so nothing in the array has to start at zero.
+    return btc_execute(op, cuda_stream, alpha, A, B, beta, C, D, scratch, size_t(BTC_STATIC_SCRATCH_BYTES), nullptr);
+}
+
 btc_error_t btc_status_get(btc_status_t status, int32_t key, void *value, size_t len)
 {
     if (!status || !value) return BTC_ERR_INVALID_ARGUMENT;
@@ -648,6 +680,7 @@ btc_error_t btc_explain_error(btc_error_t code, char *buf, size_t len, size_t *n
     case BTC_ERR_CUDA: msg = "a CUDA runtime call failed or no CUDA device is available"; break;
     case BTC_ERR_DEVICE_TIMEOUT: msg = "a bounded device-side wait expired"; break;
     case BTC_ERR_OUT_OF_MEMORY: msg = "out of memory"; break;
+    case BTC_ERR_SCRATCH_LIMIT: msg = "the operation needs more scratch than the library's built-in 8 MiB array; use btc_execute with a caller-provided workspace"; break;
     default: break;
     }
     const size_t n = std::strlen(msg) + 1;

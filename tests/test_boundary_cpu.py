@@ -33,7 +33,7 @@ def test_every_declared_symbol_is_exported(api):
 
 
 def test_error_text(api):
-    for code in range(0, 13):
+    for code in range(0, 14):
         assert len(api.explain_error(code)) > 3
     assert "success" in api.explain_error(0)
     assert "unknown" in api.explain_error(999)
