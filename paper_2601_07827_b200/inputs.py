@@ -320,6 +320,10 @@ def workloads() -> Dict[str, Workload]:
         "cfg3_f32_batched_permuted", "f32", "akzl", "lbkjz", "jbza", e3,
         alpha=1.0, beta=0.0, seed=3000, distA=("normal", 1.0), distB=("normal", 1.0),
         stridesD=(1, 104, 104 * 96, 104 * 96 * 64))
+    # 3p: workload 3 with 16 batch entries (0.4 GB on the device): the case profiler captures use
+    w["cfg3p_f32_batched_permuted_profile"] = dataclasses.replace(
+        w["cfg3_f32_batched_permuted"], name="cfg3p_f32_batched_permuted_profile", extents={**e3, "z": 16},
+        stridesD=(1, 104, 104 * 96, 104 * 96 * 16))
     # 4: complex128 with conj(A) and complex alpha
     e4 = {"p": 256, "q": 256, "r": 64, "s": 48, "t": 48}
     w["cfg4_c64_conj"] = Workload(
