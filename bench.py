@@ -69,6 +69,7 @@ def parse():
     ap.add_argument("--workload", default=WORKLOAD)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--variant", type=int, default=-1, help="force a tile variant (tuning runs)")
     return ap.parse_args()
 
 
@@ -219,6 +220,8 @@ def main():
     op = api.Contraction(handle, tA, w.labelsA, tB, w.labelsB, tC, w.labelsD, tD, w.labelsD, w.alpha, w.beta,
                          w.conjA, w.conjB, w.conjC)
     plan_ms = 1e3 * (time.perf_counter() - t0)
+    if args.variant >= 0:
+        op.set_attr(api.ATTR_VARIANT, args.variant)
     ws_bytes = op.workspace_size()
     ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
@@ -299,7 +302,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": w.name, "groups_batch_M_N_K": list(w.groups()), "kernel": op.kernel,
-                       "tile": list(op.tile), "split_k": op.split_k, "grid": list(op.grid),
+                       "tile": list(op.tile), "variant": op.variant, "split_k": op.split_k, "grid": list(op.grid),
                        "l2": l2_note, "plan_ms": plan_ms,
                        "parallelism": "independent replicas" if world > 1 else "single GPU"},
             "clocks": clocks,

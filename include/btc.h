@@ -118,6 +118,8 @@ enum {
     BTC_ATTR_GRID = 5,        /* int32[3], read: launch grid                                   */
     BTC_ATTR_NUM_MODES = 6,   /* int32[4], read: modes per class after fusion (batch, M, N, K) */
     BTC_ATTR_SWAPPED = 7,     /* int32, read: 1 when A and B exchanged roles                   */
+    BTC_ATTR_VARIANT = 9,     /* int32, read/write: index of the tile variant of the tiled
+                                 kernel for this element type (-1 on write = choose)          */
     BTC_ATTR_DEVICE_ERROR = 8 /* int32, read: 0, or which bounded device-side wait gave up in an
                                  earlier execute of this operation (its D is then incomplete);
                                  reading waits for the device                                  */

@@ -39,6 +39,7 @@ DTYPE_SIZE = {F32: 4, F64: 8, C32: 8, C64: 16}
 
 ATTR_KERNEL, ATTR_SPLIT_K, ATTR_TILE, ATTR_GROUPS, ATTR_GRID, ATTR_NUM_MODES, ATTR_SWAPPED = 1, 2, 3, 4, 5, 6, 7
 ATTR_DEVICE_ERROR = 8
+ATTR_VARIANT = 9
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TILED = 0, 1, 2
 STATUS_KERNEL, STATUS_LAUNCHES, STATUS_GRID, STATUS_SPLIT_K = 1, 2, 3, 4
 
@@ -207,6 +208,10 @@ class Contraction:
     @property
     def swapped(self) -> bool:
         return bool(self._get(ATTR_SWAPPED, ctypes.c_int32, 1)[0])
+
+    @property
+    def variant(self) -> int:
+        return self._get(ATTR_VARIANT, ctypes.c_int32, 1)[0]
 
     @property
     def device_error(self) -> int:

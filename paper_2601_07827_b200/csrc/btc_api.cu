@@ -14,6 +14,7 @@
 #include "plan.h"
 #include "tiled_f32_kernel.cuh"
 #include "tiled_f64_kernel.cuh"
+#include "tiled_tf32x3_kernel.cuh"
 
 using namespace btc;
 
@@ -56,8 +57,17 @@ using F64Small = F64Tile<false, 64, 64, 2, 2, 4, 2>;
 using C64Big = F64Tile<true, 128, 64, 2, 4, 4, 1>;
 using C64Small = F64Tile<true, 64, 32, 2, 2, 4, 2>;
 
-using F32Big = F32Tile<128, 128, 2, 4, 5, 1>;
-using F32Small = F32Tile<64, 64, 2, 2, 5, 2>;
+using F32Big = F32Tile<128, 128, 16, 2, 4, 5, 1, false>;
+using F32Small = F32Tile<64, 64, 16, 2, 2, 5, 2, false>;
+using F32Wide = F32Tile<256, 96, 16, 4, 2, 5, 1, false>;       // N = 96 fills the tile exactly
+using F32BigP = F32Tile<128, 128, 16, 2, 4, 5, 1, true>;
+using F32WideP = F32Tile<256, 96, 16, 4, 2, 5, 1, true>;
+using F32Big32 = F32Tile<128, 128, 32, 2, 4, 3, 1, false>;
+using F32Tc = TF32Tile<false, 128, 128, 2, 4, 4, 1>;             // 3xTF32 on the tensor cores
+using F32TcSmall = TF32Tile<false, 64, 64, 2, 2, 4, 2>;
+using C32Tc = TF32Tile<true, 128, 64, 2, 4, 4, 1>;
+using C32TcSmall = TF32Tile<true, 64, 32, 2, 2, 4, 2>;
+constexpr int kNumF32Variants = 8;
 
 struct VariantInfo {
     int bm, bn, bk, threads, acc;
@@ -69,12 +79,24 @@ template <typename T> VariantInfo info_of(size_t acc_bytes)
     return {T::BM, T::BN, T::BK, T::CONSUMER_THREADS, T::ACC, T::SMEM_BYTES, acc_bytes};
 }
 
-bool tiled_supported(btc_dtype_t t) { return t == BTC_F64 || t == BTC_C64 || t == BTC_F32; }
+bool tiled_supported(btc_dtype_t) { return true; }
 
 VariantInfo variant_info(btc_dtype_t t, int variant)
 {
     if (t == BTC_F64) return variant == 0 ? info_of<F64Big>(8) : info_of<F64Small>(8);
-    if (t == BTC_F32) return variant == 0 ? info_of<F32Big>(4) : info_of<F32Small>(4);
+    if (t == BTC_F32) {
+        switch (variant) {
+        case 0: return info_of<F32Big>(4);
+        case 1: return info_of<F32Small>(4);
+        case 2: return info_of<F32Wide>(4);
+        case 3: return info_of<F32BigP>(4);
+        case 4: return info_of<F32WideP>(4);
+        case 5: return info_of<F32Big32>(4);
+        case 6: return info_of<F32Tc>(4);
+        default: return info_of<F32TcSmall>(4);
+        }
+    }
+    if (t == BTC_C32) return variant == 0 ? info_of<C32Tc>(4) : info_of<C32TcSmall>(4);
     return variant == 0 ? info_of<C64Big>(8) : info_of<C64Small>(8);
 }
 
@@ -102,6 +124,22 @@ cudaError_t launch_tiled(const TiledParams &p, int64_t ctas, int64_t reduce_ctas
     if (e != cudaSuccess) return e;
     if (p.split_k > 1) {
         tiled_f64_splitk_reduce_kernel<T><<<unsigned(reduce_ctas), T::CONSUMER_THREADS, 0, st>>>(p);
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+template <typename T>
+cudaError_t launch_tiled_tf32(const TiledParams &p, int64_t ctas, int64_t reduce_ctas, cudaStream_t st)
+{
+    static bool configured[64] = {};
+    cudaError_t e = set_smem_once(tiled_tf32x3_kernel<T>, T::SMEM_BYTES, configured);
+    if (e != cudaSuccess) return e;
+    tiled_tf32x3_kernel<T><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (p.split_k > 1) {
+        tiled_tf32x3_splitk_reduce_kernel<T><<<unsigned(reduce_ctas), T::CONSUMER_THREADS, 0, st>>>(p);
         e = cudaGetLastError();
     }
     return e;
@@ -181,11 +219,19 @@ int finish_plan(btc_contraction_s *op)
     auto tiles_for = [&](const VariantInfo &v) {
         return ((pl.M + v.bm - 1) / v.bm) * ((pl.N + v.bn - 1) / v.bn) * pl.Bt;
     };
-    int variant = 0;
-    if (double(tiles_for(variant_info(pl.dtype, 0))) < 0.8 * sms) variant = 1;
+    // fp32 defaults to the 3xTF32 tensor-core variants (6: big tile, 7: small tile); the FFMA
+    // variants 0-5 compute in strict fp32 and are selected with BTC_ATTR_VARIANT
+    const int big = pl.dtype == BTC_F32 ? 6 : 0, small = pl.dtype == BTC_F32 ? 7 : 1;
+    int variant = big;
+    if (double(tiles_for(variant_info(pl.dtype, big))) < 0.8 * sms) variant = small;
+    if (op->req.force_variant >= 0) {
+        const int count = pl.dtype == BTC_F32 ? kNumF32Variants : 2;
+        if (op->req.force_variant >= count) return BTC_ERR_INVALID_ARGUMENT;
+        variant = op->req.force_variant;
+    }
     const VariantInfo v = variant_info(pl.dtype, variant);
     pl.tile.bm = v.bm; pl.tile.bn = v.bn; pl.tile.bk = v.bk; pl.tile.threads = v.threads;
-    pl.tile.stages = pl.dtype == BTC_F32 ? 5 : 4; pl.tile.variant = variant;
+    pl.tile.stages = 0; pl.tile.variant = variant;
     op->tiles_m = int32_t((pl.M + v.bm - 1) / v.bm);
     op->tiles_n = int32_t((pl.N + v.bn - 1) / v.bn);
     op->raster_n_fast = op->tiles_n <= op->tiles_m ? 1 : 0;
@@ -395,6 +441,8 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
     if (key == BTC_ATTR_KERNEL) {
         if (v < BTC_KERNEL_AUTO || v > BTC_KERNEL_TILED) return BTC_ERR_INVALID_ARGUMENT;
         op->req.force_kernel = v;
+    } else if (key == BTC_ATTR_VARIANT) {
+        op->req.force_variant = v;
     } else if (key == BTC_ATTR_SPLIT_K) {
         if (v < 0) return BTC_ERR_INVALID_ARGUMENT;
         op->req.force_split_k = v;
@@ -427,6 +475,7 @@ btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t 
         i32[0] = int32_t(pl.batch.size()); i32[1] = int32_t(pl.m.size());
         i32[2] = int32_t(pl.n.size()); i32[3] = int32_t(pl.k.size()); n = 16; break;
     case BTC_ATTR_SWAPPED: i32[0] = pl.swapped ? 1 : 0; n = 4; break;
+    case BTC_ATTR_VARIANT: i32[0] = pl.tile.variant; n = 4; break;
     case BTC_ATTR_DEVICE_ERROR:
         i32[0] = 0;
         if (op->d_error) {
@@ -531,10 +580,21 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         const int64_t reduce_ctas = ctas / pl.split_k;
         // 16-byte stores of D (and loads of C) need those base pointers aligned too
         tp.vecD = (pl.vecD == 4 && !misaligned(D, 16) && !(use_c && misaligned(C, 16))) ? 4 : 1;
-        if (pl.dtype == BTC_F32)
-            ce = pl.tile.variant == 0 ? launch_tiled_f32<F32Big>(tp, ctas, reduce_ctas, st)
-                                      : launch_tiled_f32<F32Small>(tp, ctas, reduce_ctas, st);
-        else if (pl.dtype == BTC_F64)
+        if (pl.dtype == BTC_F32) {
+            switch (pl.tile.variant) {
+            case 0: ce = launch_tiled_f32<F32Big>(tp, ctas, reduce_ctas, st); break;
+            case 1: ce = launch_tiled_f32<F32Small>(tp, ctas, reduce_ctas, st); break;
+            case 2: ce = launch_tiled_f32<F32Wide>(tp, ctas, reduce_ctas, st); break;
+            case 3: ce = launch_tiled_f32<F32BigP>(tp, ctas, reduce_ctas, st); break;
+            case 4: ce = launch_tiled_f32<F32WideP>(tp, ctas, reduce_ctas, st); break;
+            case 5: ce = launch_tiled_f32<F32Big32>(tp, ctas, reduce_ctas, st); break;
+            case 6: ce = launch_tiled_tf32<F32Tc>(tp, ctas, reduce_ctas, st); break;
+            default: ce = launch_tiled_tf32<F32TcSmall>(tp, ctas, reduce_ctas, st); break;
+            }
+        } else if (pl.dtype == BTC_C32) {
+            ce = pl.tile.variant == 0 ? launch_tiled_tf32<C32Tc>(tp, ctas, reduce_ctas, st)
+                                      : launch_tiled_tf32<C32TcSmall>(tp, ctas, reduce_ctas, st);
+        } else if (pl.dtype == BTC_F64)
             ce = pl.tile.variant == 0 ? launch_tiled<F64Big>(tp, ctas, reduce_ctas, st)
                                       : launch_tiled<F64Small>(tp, ctas, reduce_ctas, st);
         else

@@ -18,9 +18,10 @@
 
 namespace btc {
 
-template <int BM_, int BN_, int WARPS_M_, int WARPS_N_, int STAGES_, int MIN_CTAS_>
+template <int BM_, int BN_, int BK_, int WARPS_M_, int WARPS_N_, int STAGES_, int MIN_CTAS_, bool PREFETCH_>
 struct F32Tile {
-    static constexpr int BM = BM_, BN = BN_, BK = 16;
+    static constexpr int BM = BM_, BN = BN_, BK = BK_;
+    static constexpr bool PREFETCH = PREFETCH_;
     static constexpr int WARPS_M = WARPS_M_, WARPS_N = WARPS_N_;
     static constexpr int CONSUMER_WARPS = WARPS_M_ * WARPS_N_;
     static constexpr int CONSUMER_THREADS = 32 * CONSUMER_WARPS;
@@ -146,51 +147,57 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f32_kernel(cons
         }
         const float *sa = stage_base + size_t(s) * T::STAGE_FLOATS;
         const float *sb = sa + T::A_ELEMS;
-#pragma unroll
-        for (int k4 = 0; k4 < T::BK; k4 += 4) {
-            float4 a4[A_KMAJ ? T::TM : 1], b4[B_KMAJ ? T::TN : 1];
+        // fragments of 4 consecutive k live in registers; with PREFETCH the next group's loads
+        // are issued before the current group's FMAs
+        float fa[T::PREFETCH ? 2 : 1][T::TM][4], fb[T::PREFETCH ? 2 : 1][T::TN][4];
+        auto load_group = [&](int buf, int k4) {
             if (A_KMAJ) {
 #pragma unroll
-                for (int i = 0; i < T::TM; ++i)
-                    a4[i] = *reinterpret_cast<const float4 *>(sa + (wm0 + ty + 8 * i) * T::PITCH_K + k4);
-            }
-            if (B_KMAJ) {
+                for (int i = 0; i < T::TM; ++i) {
+                    const float4 v = *reinterpret_cast<const float4 *>(sa + (wm0 + ty + 8 * i) * T::PITCH_K + k4);
+                    fa[buf][i][0] = v.x; fa[buf][i][1] = v.y; fa[buf][i][2] = v.z; fa[buf][i][3] = v.w;
+                }
+            } else {
 #pragma unroll
-                for (int j = 0; j < T::TN; ++j)
-                    b4[j] = *reinterpret_cast<const float4 *>(sb + (wn0 + tx + 4 * j) * T::PITCH_K + k4);
-            }
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
-                float a[T::TM], b[T::TN];
-                if (A_KMAJ) {
-#pragma unroll
-                    for (int i = 0; i < T::TM; ++i)
-                        a[i] = kk == 0 ? a4[i].x : kk == 1 ? a4[i].y : kk == 2 ? a4[i].z : a4[i].w;
-                } else {
+                for (int kk = 0; kk < 4; ++kk)
 #pragma unroll
                     for (int i4 = 0; i4 < T::TM / 4; ++i4) {
                         const float4 v = *reinterpret_cast<const float4 *>(
                             sa + (k4 + kk) * T::PITCH_FREE_A + wm0 + i4 * 32 + ty * 4);
-                        a[i4 * 4] = v.x; a[i4 * 4 + 1] = v.y; a[i4 * 4 + 2] = v.z; a[i4 * 4 + 3] = v.w;
+                        fa[buf][i4 * 4][kk] = v.x; fa[buf][i4 * 4 + 1][kk] = v.y;
+                        fa[buf][i4 * 4 + 2][kk] = v.z; fa[buf][i4 * 4 + 3][kk] = v.w;
                     }
-                }
-                if (B_KMAJ) {
+            }
+            if (B_KMAJ) {
 #pragma unroll
-                    for (int j = 0; j < T::TN; ++j)
-                        b[j] = kk == 0 ? b4[j].x : kk == 1 ? b4[j].y : kk == 2 ? b4[j].z : b4[j].w;
-                } else {
+                for (int j = 0; j < T::TN; ++j) {
+                    const float4 v = *reinterpret_cast<const float4 *>(sb + (wn0 + tx + 4 * j) * T::PITCH_K + k4);
+                    fb[buf][j][0] = v.x; fb[buf][j][1] = v.y; fb[buf][j][2] = v.z; fb[buf][j][3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
 #pragma unroll
                     for (int j4 = 0; j4 < T::TN / 4; ++j4) {
                         const float4 v = *reinterpret_cast<const float4 *>(
                             sb + (k4 + kk) * T::PITCH_FREE_B + wn0 + j4 * 16 + tx * 4);
-                        b[j4 * 4] = v.x; b[j4 * 4 + 1] = v.y; b[j4 * 4 + 2] = v.z; b[j4 * 4 + 3] = v.w;
+                        fb[buf][j4 * 4][kk] = v.x; fb[buf][j4 * 4 + 1][kk] = v.y;
+                        fb[buf][j4 * 4 + 2][kk] = v.z; fb[buf][j4 * 4 + 3][kk] = v.w;
                     }
-                }
+            }
+        };
+        if (T::PREFETCH) load_group(0, 0);
+#pragma unroll
+        for (int g = 0; g < T::BK / 4; ++g) {
+            const int cur = T::PREFETCH ? (g & 1) : 0;
+            if (!T::PREFETCH) load_group(0, g * 4);
+            else if (g + 1 < T::BK / 4) load_group(cur ^ 1, (g + 1) * 4);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
 #pragma unroll
                 for (int i = 0; i < T::TM; ++i)
 #pragma unroll
-                    for (int j = 0; j < T::TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-            }
+                    for (int j = 0; j < T::TN; ++j) acc[i][j] = fmaf(fa[cur][i][kk], fb[cur][j][kk], acc[i][j]);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * s);
