@@ -2,6 +2,7 @@
 // tile/split-K choice and kernel launches.  No compute happens on the host.
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -67,7 +68,9 @@ using F32Tc = TF32Tile<false, 128, 128, 2, 4, 4, 1>;             // 3xTF32 on th
 using F32TcSmall = TF32Tile<false, 64, 64, 2, 2, 4, 2>;
 using C32Tc = TF32Tile<true, 128, 64, 2, 4, 4, 1>;
 using C32TcSmall = TF32Tile<true, 64, 32, 2, 2, 4, 2>;
-constexpr int kNumF32Variants = 8;
+using F32TcWide = TF32Tile<false, 256, 96, 4, 2, 4, 1>;          // N = 96 fills the tile exactly
+using F32TcMid = TF32Tile<false, 128, 96, 2, 4, 4, 1>;
+constexpr int kNumF32Variants = 10;
 
 struct VariantInfo {
     int bm, bn, bk, threads, acc;
@@ -93,7 +96,9 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
         case 4: return info_of<F32WideP>(4);
         case 5: return info_of<F32Big32>(4);
         case 6: return info_of<F32Tc>(4);
-        default: return info_of<F32TcSmall>(4);
+        case 7: return info_of<F32TcSmall>(4);
+        case 8: return info_of<F32TcWide>(4);
+        default: return info_of<F32TcMid>(4);
         }
     }
     if (t == BTC_C32) return variant == 0 ? info_of<C32Tc>(4) : info_of<C32TcSmall>(4);
@@ -219,11 +224,30 @@ int finish_plan(btc_contraction_s *op)
     auto tiles_for = [&](const VariantInfo &v) {
         return ((pl.M + v.bm - 1) / v.bm) * ((pl.N + v.bn - 1) / v.bn) * pl.Bt;
     };
-    // fp32 defaults to the 3xTF32 tensor-core variants (6: big tile, 7: small tile); the FFMA
-    // variants 0-5 compute in strict fp32 and are selected with BTC_ATTR_VARIANT
-    const int big = pl.dtype == BTC_F32 ? 6 : 0, small = pl.dtype == BTC_F32 ? 7 : 1;
-    int variant = big;
-    if (double(tiles_for(variant_info(pl.dtype, big))) < 0.8 * sms) variant = small;
+    // Candidate tile variants of the element type (fp32: the 3xTF32 tensor-core variants; the
+    // strict-fp32 FFMA variants 0-5 are selected with BTC_ATTR_VARIANT only).  Score = fraction of
+    // the padded tiles that is real work x fraction of the last wave that is filled x a mild
+    // preference for larger tiles (more flops per byte moved through shared memory).
+    int variant = 0;
+    {
+        struct Cand { int id; double weight; };
+        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}};
+        const Cand other[] = {{0, 1.0}, {1, 0.75}};
+        const Cand *cands = pl.dtype == BTC_F32 ? f32c : other;
+        const int ncand = pl.dtype == BTC_F32 ? 4 : 2;
+        double best = -1.0;
+        for (int c = 0; c < ncand; ++c) {
+            const VariantInfo vi = variant_info(pl.dtype, cands[c].id);
+            const double tiles = double(tiles_for(vi));
+            const double ctas_per_sm = vi.bm * vi.bn <= 64 * 64 ? 2.0 : 1.0;
+            const double slots = sms * ctas_per_sm;
+            const double util = double(pl.M) * double(pl.N) * double(pl.Bt) / (tiles * vi.bm * vi.bn);
+            const double waves = std::ceil(tiles / slots);
+            const double wave_eff = tiles / (waves * slots);
+            const double score = util * wave_eff * cands[c].weight;
+            if (score > best) { best = score; variant = cands[c].id; }
+        }
+    }
     if (op->req.force_variant >= 0) {
         const int count = pl.dtype == BTC_F32 ? kNumF32Variants : 2;
         if (op->req.force_variant >= count) return BTC_ERR_INVALID_ARGUMENT;
@@ -589,7 +613,9 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
             case 4: ce = launch_tiled_f32<F32WideP>(tp, ctas, reduce_ctas, st); break;
             case 5: ce = launch_tiled_f32<F32Big32>(tp, ctas, reduce_ctas, st); break;
             case 6: ce = launch_tiled_tf32<F32Tc>(tp, ctas, reduce_ctas, st); break;
-            default: ce = launch_tiled_tf32<F32TcSmall>(tp, ctas, reduce_ctas, st); break;
+            case 7: ce = launch_tiled_tf32<F32TcSmall>(tp, ctas, reduce_ctas, st); break;
+            case 8: ce = launch_tiled_tf32<F32TcWide>(tp, ctas, reduce_ctas, st); break;
+            default: ce = launch_tiled_tf32<F32TcMid>(tp, ctas, reduce_ctas, st); break;
             }
         } else if (pl.dtype == BTC_C32) {
             ce = pl.tile.variant == 0 ? launch_tiled_tf32<C32Tc>(tp, ctas, reduce_ctas, st)
