@@ -185,6 +185,58 @@ def run_reference(args, w):
     print(json.dumps(out))
 
 
+def max_over_ranks(ms: float, device="cpu") -> float:
+    """Largest per-rank time; a no-op outside torch.distributed (single process)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: float, world: int, ms: float) -> float:
+    """Independent replicas (weak scaling): all ranks' units over the slowest rank's time."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
+def small_problem_latency(step, stream, torch):
+    """For workloads with microseconds of work: median single-call latency, back-to-back plain
+    launches, and replay of a CUDA graph holding 100 calls (all in microseconds per call)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    with torch.cuda.stream(side):
+        run = lambda: step(side)
+        for _ in range(5):
+            run()
+        side.synchronize()
+        single = []
+        for _ in range(200):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(side); run(); b.record(side); side.synchronize()
+            single.append(a.elapsed_time(b) * 1e3)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        for _ in range(1000):
+            run()
+        e1.record(side); side.synchronize()
+        plain = e0.elapsed_time(e1)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(100):
+                run()
+        g.replay(); side.synchronize()
+        e0.record(side)
+        for _ in range(10):
+            g.replay()
+        e1.record(side); side.synchronize()
+        graph = e0.elapsed_time(e1)
+    stream.wait_stream(side)
+    return {"single_call_us_median": statistics.median(single), "back_to_back_us": plain,
+            "graph_replay_us": graph, "calls": {"single": 200, "back_to_back": 1000, "graph": 1000}}
+
+
 def main():
     args = parse()
     from paper_2601_07827_b200 import inputs
@@ -227,8 +279,8 @@ def main():
     stream = torch.cuda.current_stream()
     pC = C.data_ptr() if C is not None else 0
 
-    def step(status=False):
-        return op.execute(stream.cuda_stream, A.data_ptr(), B.data_ptr(), pC, D.data_ptr(),
+    def step(status=False, on=None):
+        return op.execute((on or stream).cuda_stream, A.data_ptr(), B.data_ptr(), pC, D.data_ptr(),
                           workspace=ws.data_ptr(), workspace_bytes=ws_bytes, want_status=status)
 
     def barrier():
@@ -254,15 +306,12 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     total_ms = ev[0].elapsed_time(ev[-1])
     kernel_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, "cuda")
     ms_per_step = total_ms / args.steps
     flops = w.flops()
     l2_note = ("inputs exceed L2" if w.algorithmic_bytes() > 126e6 else
                "operands fit in L2 and stay there between steps (L2-resident figure)")
-    value = world * flops / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_rate(flops, world, ms_per_step) / 1e9
 
     # ---- end to end: host buffers (pinned), copies inside the timed region
     hA = inputs.StridedTensor(A.buffer.cpu().pin_memory(), A.extents, A.strides, A.origin)
@@ -290,10 +339,7 @@ def main():
         e1.record(stream)
         barrier()
         e2e_ms = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0)) / args.e2e_steps
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_value = world * flops / (float(t.item()) * 1e-3) / 1e9
+        e2e_value = whole_job_rate(flops, world, max_over_ranks(e2e_ms, "cuda")) / 1e9
 
     if rank == 0:
         kernel_avg_ms = statistics.mean(kernel_ms)
@@ -310,6 +356,14 @@ def main():
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline_for(w, kernel_avg_ms),
         }
+        if ms_per_step < 0.2 and world == 1:
+            # microseconds of work per call: the per-step figure above includes the host's call
+            # overhead, so the device-side figures are reported beside it
+            lat = small_problem_latency(lambda s_: step(on=s_), stream, torch)
+            out["latency"] = lat
+            per_call_ms = lat["graph_replay_us"] * 1e-3
+            out["roofline"] = roofline_for(w, per_call_ms)
+            out["roofline"]["timing"] = "per call inside a replayed CUDA graph of 100 calls"
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"] = cpu_baseline(w)
         print(json.dumps(out))

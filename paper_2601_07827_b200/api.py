@@ -279,7 +279,7 @@ def dtype_code(torch_dtype) -> int:
 
 def contract(handle: Handle, A, labelsA, B, labelsB, C, D, labelsD, alpha=1.0, beta=0.0,
              conjA=False, conjB=False, conjC=False, stream: int = 0, kernel: int = KERNEL_AUTO,
-             split_k: int = 0, want_status: bool = False):
+             split_k: int = 0, want_status: bool = False, variant: int = -1):
     """One-shot helper for tensors described by objects with .dtype, .extents, .strides and
     .data_ptr() (device memory): builds the descriptors and the operation, allocates the
     workspace with torch, executes on `stream`.  Returns (Contraction, status-or-None)."""
@@ -294,6 +294,8 @@ def contract(handle: Handle, A, labelsA, B, labelsB, C, D, labelsD, alpha=1.0, b
         op.set_attr(ATTR_KERNEL, kernel)
     if split_k:
         op.set_attr(ATTR_SPLIT_K, split_k)
+    if variant >= 0:
+        op.set_attr(ATTR_VARIANT, variant)
     ws_bytes = op.workspace_size()
     ws = torch.empty(max(ws_bytes, 1), dtype=torch.uint8, device="cuda") if ws_bytes else None
     st = op.execute(stream, A.data_ptr(), B.data_ptr(), C.data_ptr() if C is not None else 0, D.data_ptr(),

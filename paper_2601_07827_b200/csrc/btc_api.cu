@@ -55,6 +55,9 @@ namespace {
 // ---- tiled kernel variants -------------------------------------------------------------------
 using F64Big = F64Tile<false, 128, 128, 2, 4, 4, 1>;
 using F64Small = F64Tile<false, 64, 64, 2, 2, 4, 2>;
+using F64Big16 = F64Tile<false, 128, 128, 2, 4, 4, 1, true>;   // m16n8k16 MMAs
+using F64Big3 = F64Tile<false, 128, 128, 2, 4, 3, 1>;           // 3 stages
+using F64BigT = F64Tile<false, 128, 128, 4, 2, 4, 1>;           // warp tile 32 x 64
 using C64Big = F64Tile<true, 128, 64, 2, 4, 4, 1>;
 using C64Small = F64Tile<true, 64, 32, 2, 2, 4, 2>;
 
@@ -86,7 +89,15 @@ bool tiled_supported(btc_dtype_t) { return true; }
 
 VariantInfo variant_info(btc_dtype_t t, int variant)
 {
-    if (t == BTC_F64) return variant == 0 ? info_of<F64Big>(8) : info_of<F64Small>(8);
+    if (t == BTC_F64) {
+        switch (variant) {
+        case 0: return info_of<F64Big>(8);
+        case 1: return info_of<F64Small>(8);
+        case 2: return info_of<F64Big16>(8);
+        case 3: return info_of<F64Big3>(8);
+        default: return info_of<F64BigT>(8);
+        }
+    }
     if (t == BTC_F32) {
         switch (variant) {
         case 0: return info_of<F32Big>(4);
@@ -232,8 +243,9 @@ int finish_plan(btc_contraction_s *op)
     {
         struct Cand { int id; double weight; };
         const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}};
+        const Cand f64c[] = {{2, 1.0}, {1, 0.75}};       // big tile: the m16n8k16 variant
         const Cand other[] = {{0, 1.0}, {1, 0.75}};
-        const Cand *cands = pl.dtype == BTC_F32 ? f32c : other;
+        const Cand *cands = pl.dtype == BTC_F32 ? f32c : (pl.dtype == BTC_F64 ? f64c : other);
         const int ncand = pl.dtype == BTC_F32 ? 4 : 2;
         double best = -1.0;
         for (int c = 0; c < ncand; ++c) {
@@ -249,7 +261,7 @@ int finish_plan(btc_contraction_s *op)
         }
     }
     if (op->req.force_variant >= 0) {
-        const int count = pl.dtype == BTC_F32 ? kNumF32Variants : 2;
+        const int count = pl.dtype == BTC_F32 ? kNumF32Variants : (pl.dtype == BTC_F64 ? 5 : 2);
         if (op->req.force_variant >= count) return BTC_ERR_INVALID_ARGUMENT;
         variant = op->req.force_variant;
     }
@@ -621,8 +633,13 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
             ce = pl.tile.variant == 0 ? launch_tiled_tf32<C32Tc>(tp, ctas, reduce_ctas, st)
                                       : launch_tiled_tf32<C32TcSmall>(tp, ctas, reduce_ctas, st);
         } else if (pl.dtype == BTC_F64)
-            ce = pl.tile.variant == 0 ? launch_tiled<F64Big>(tp, ctas, reduce_ctas, st)
-                                      : launch_tiled<F64Small>(tp, ctas, reduce_ctas, st);
+            switch (pl.tile.variant) {
+            case 0: ce = launch_tiled<F64Big>(tp, ctas, reduce_ctas, st); break;
+            case 1: ce = launch_tiled<F64Small>(tp, ctas, reduce_ctas, st); break;
+            case 2: ce = launch_tiled<F64Big16>(tp, ctas, reduce_ctas, st); break;
+            case 3: ce = launch_tiled<F64Big3>(tp, ctas, reduce_ctas, st); break;
+            default: ce = launch_tiled<F64BigT>(tp, ctas, reduce_ctas, st); break;
+            }
         else
             ce = pl.tile.variant == 0 ? launch_tiled<C64Big>(tp, ctas, reduce_ctas, st)
                                       : launch_tiled<C64Small>(tp, ctas, reduce_ctas, st);

@@ -33,9 +33,10 @@
 
 namespace btc {
 
-template <bool CPLX_, int BM_, int BN_, int WARPS_M_, int WARPS_N_, int STAGES_, int MIN_CTAS_>
+template <bool CPLX_, int BM_, int BN_, int WARPS_M_, int WARPS_N_, int STAGES_, int MIN_CTAS_, bool MMA16_ = false>
 struct F64Tile {
     static constexpr bool CPLX = CPLX_;
+    static constexpr bool MMA16 = MMA16_;             // one m16n8k16 MMA per stage instead of m8n8k4 steps
     static constexpr int BM = BM_;                    // rows of the CTA tile (elements)
     static constexpr int BN = BN_;                    // columns of the CTA tile (elements)
     static constexpr int BK = CPLX_ ? 8 : 16;         // k extent of one stage (elements)
@@ -66,6 +67,17 @@ struct F64Tile {
     static constexpr size_t SMEM_BYTES =
         size_t(STAGES) * STAGE_WORDS * 8 + size_t(2 * BM + 2 * BN) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
+
+// m16n8k16: A rows g / g+8 (even / odd register), k = t + 4 (i / 2); B k = t + 4 j, column g;
+// C rows g (c0, c1) and g + 8 (c2, c3), columns 2t, 2t + 1
+__device__ __forceinline__ void dmma_m16n8k16(double (&c)[4], const double (&a)[8], const double (&b)[4])
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f64.f64.f64.f64 {%0,%1,%2,%3}, {%4,%5,%6,%7,%8,%9,%10,%11}, "
+                 "{%12,%13,%14,%15}, {%0,%1,%2,%3};"
+                 : "+d"(c[0]), "+d"(c[1]), "+d"(c[2]), "+d"(c[3])
+                 : "d"(a[0]), "d"(a[1]), "d"(a[2]), "d"(a[3]), "d"(a[4]), "d"(a[5]), "d"(a[6]), "d"(a[7]),
+                   "d"(b[0]), "d"(b[1]), "d"(b[2]), "d"(b[3]));
+}
 
 __device__ __forceinline__ void dmma_m8n8k4(double &c0, double &c1, double a, double b)
 {
@@ -210,6 +222,38 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
         }
         const double *sa = stage_base + size_t(s) * T::STAGE_WORDS;
         const double *sb = sa + T::A_ELEMS * W;
+        if (T::MMA16) {
+            // acc[2 i2][j] / acc[2 i2 + 1][j] are the row halves g / g + 8 of a 16-row fragment
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {       // limits live fragment registers
+                double a16[T::FM / 4][8], b16[T::FN][4];
+#pragma unroll
+                for (int j = 0; j < T::FN; ++j)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        double b = sb[b_thr + j * b_jstep + q * b_kstep];
+                        if (T::CPLX) {
+                            int hi = __double2hiint(b) ^ int(b_sign);
+                            b = __hiloint2double(hi, __double2loint(b));
+                        }
+                        b16[j][q] = b;
+                    }
+#pragma unroll
+                for (int i2 = 0; i2 < T::FM / 4; ++i2)
+#pragma unroll
+                    for (int r = 0; r < 8; ++r)
+                        a16[i2][r] = sa[a_thr + ((half * (T::FM / 4) + i2) * 2 + (r & 1)) * a_istep + (r >> 1) * a_kstep];
+#pragma unroll
+                for (int i2 = 0; i2 < T::FM / 4; ++i2)
+#pragma unroll
+                    for (int j = 0; j < T::FN; ++j) {
+                        const int i = (half * (T::FM / 4) + i2) * 2;
+                        double c[4] = {acc[i][j][0], acc[i][j][1], acc[i + 1][j][0], acc[i + 1][j][1]};
+                        dmma_m16n8k16(c, a16[i2], b16[j]);
+                        acc[i][j][0] = c[0]; acc[i][j][1] = c[1]; acc[i + 1][j][0] = c[2]; acc[i + 1][j][1] = c[3];
+                    }
+            }
+        } else
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {         // 16 real k per stage, 4 per MMA
             double af[T::FM], bf[T::FN];

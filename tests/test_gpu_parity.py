@@ -210,3 +210,25 @@ def test_unaligned_base_pointer_falls_back_to_element_copies(api, handle):
     D = inputs.place(None, _ext("ij", ext), None, torch.float64)
     worst, _, _ = helpers.run_case(handle, A_view, "ik", B, "kj", None, D, "ij", kernel=api.KERNEL_TILED)
     assert worst <= 1.0
+
+
+@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(10)]
+                         + [(torch.complex128, v) for v in range(2)] + [(torch.complex64, v) for v in range(2)])
+def test_every_tile_variant(api, handle, dtype, variant):
+    """Each tile variant of the tiled kernels, forced through the attribute, on a ragged multi-tile case
+    with one operand contiguous along its free index and the other along k."""
+    ext = dict(i=300, j=200, k=150)
+    A = helpers.random_tensor(71, _ext("ik", ext), None, dtype)
+    B = helpers.random_tensor(72, _ext("kj", ext), None, dtype)
+    C = helpers.random_tensor(73, _ext("ij", ext), None, dtype)
+    D = inputs.place(None, _ext("ij", ext), None, dtype)
+    worst, status, _ = helpers.run_case(handle, A, "ik", B, "kj", C, D, "ij", 1.25, -0.5, kernel=api.KERNEL_TILED,
+                                        variant=variant, want_status=True)
+    assert worst <= 1.0 and status["kernel"] == api.KERNEL_TILED
+    # both operands contiguous along k / both along the free index
+    A2 = helpers.random_tensor(74, _ext("ki", ext), None, dtype)
+    B2 = helpers.random_tensor(75, _ext("jk", ext), None, dtype)
+    worst, _, _ = helpers.run_case(handle, A2, "ki", B, "kj", None, D, "ij", kernel=api.KERNEL_TILED, variant=variant)
+    assert worst <= 1.0
+    worst, _, _ = helpers.run_case(handle, A, "ik", B2, "jk", None, D, "ij", kernel=api.KERNEL_TILED, variant=variant)
+    assert worst <= 1.0
