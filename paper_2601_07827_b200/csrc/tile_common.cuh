@@ -10,6 +10,8 @@
 namespace btc {
 
 constexpr int kProducerWarps = 4;   // one warpgroup
+// k-offset entries per operand that a CTA keeps in shared memory (its whole k slice when it fits)
+constexpr int kKoffCap = 1024;
 
 __device__ __forceinline__ int64_t imin64(int64_t a, int64_t b) { return a < b ? a : b; }
 
@@ -72,11 +74,12 @@ template <int REGS> __device__ __forceinline__ void reg_dec() { asm volatile("se
 //   DIR       0: consecutive threads take consecutive rows; 1: consecutive k
 //   VEC       elements per copy along that direction
 //   row_off   shared array: element offset of each tile row (batch offset included)
-//   koff      global table of k offsets;  [.., k_end) is this CTA's valid k range
+//   koff      table of k offsets indexed by absolute k (global memory, or the CTA's shared copy
+//             biased by the slice start);  [.., k_end) is this CTA's valid k range
 //   s_row, s_k  shared-memory strides of the tile in elements
 template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES, int DIR, int VEC>
 __device__ __forceinline__ void gather_tile(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
-                                            const int64_t *__restrict__ koff, int rows_valid, int64_t k0,
+                                            const int64_t *koff, int rows_valid, int64_t k0,
                                             int64_t k_end, int s_row, int s_k, int tid)
 {
     constexpr int NFAST = (DIR == 0 ? ROWS : BK) / VEC;
@@ -87,14 +90,14 @@ __device__ __forceinline__ void gather_tile(unsigned smem, const char *__restric
         const int r = DIR == 0 ? f : o;
         const int k = DIR == 0 ? o : f;
         const bool valid = (r < rows_valid) && (k0 + k < k_end);
-        const int64_t off = valid ? row_off[r] + __ldg(koff + k0 + k) : 0;
+        const int64_t off = valid ? row_off[r] + koff[k0 + k] : 0;
         cp_async_bytes<VEC * ELEM_BYTES>(smem + unsigned(r * s_row + k * s_k) * ELEM_BYTES, g + off * ELEM_BYTES, valid);
     }
 }
 
 template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES, int DIR>
 __device__ __forceinline__ void gather_dispatch_vec(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
-                                                    const int64_t *__restrict__ koff, int rows_valid, int64_t k0,
+                                                    const int64_t *koff, int rows_valid, int64_t k0,
                                                     int64_t k_end, int vec, int s_row, int s_k, int tid)
 {
     constexpr int VMAX = 16 / ELEM_BYTES;   // 4 for fp32, 2 for fp64 and complex64, 1 for complex128
@@ -108,7 +111,7 @@ __device__ __forceinline__ void gather_dispatch_vec(unsigned smem, const char *_
 
 template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES>
 __device__ __forceinline__ void gather_dispatch(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
-                                                const int64_t *__restrict__ koff, int rows_valid, int64_t k0,
+                                                const int64_t *koff, int rows_valid, int64_t k0,
                                                 int64_t k_end, int dir, int vec, int s_row, int s_k, int tid)
 {
     if (dir == 0)
@@ -150,9 +153,17 @@ __device__ __forceinline__ TileCoords tile_coords(const Params &p)
 // CTA-wide barrier.
 template <int BM, int BN, int STAGES, int NTHREADS, int PRODUCERS, int CONSUMER_WARPS, typename Params>
 __device__ __forceinline__ void tile_setup(const Params &p, const TileCoords &c, int64_t *rowA, int64_t *rowD,
-                                           int64_t *colB, int64_t *colD, unsigned full0, unsigned empty0,
-                                           volatile int *abort_flag, int tid)
+                                           int64_t *colB, int64_t *colD, int64_t *koffA, int64_t *koffB,
+                                           unsigned full0, unsigned empty0, volatile int *abort_flag, int tid)
 {
+    // the k offsets of this CTA's slice, when they fit: the producers then never wait on a
+    // table load between a stage's release and its copies
+    if (c.k_end - c.k_begin <= kKoffCap) {
+        for (int i = tid; i < int(c.k_end - c.k_begin); i += NTHREADS) {
+            koffA[i] = p.offA_k[c.k_begin + i];
+            koffB[i] = p.offB_k[c.k_begin + i];
+        }
+    }
     const int64_t hA = p.offA_h[c.h], hB = p.offB_h[c.h], hD = p.offD_h[c.h];
     for (int i = tid; i < BM; i += NTHREADS) {
         const bool v = i < c.rows_valid;
@@ -178,10 +189,14 @@ __device__ __forceinline__ void tile_setup(const Params &p, const TileCoords &c,
 // A and B tiles into it, and let the stage's "full" barrier fire when the copies have landed.
 template <int BM, int BN, int BK, int EB, int STAGES, int STAGE_BYTES, int A_BYTES, int PRODUCERS, typename Params>
 __device__ __forceinline__ void producer_loop(const Params &p, const TileCoords &c, unsigned stage0,
-                                              const int64_t *rowA, const int64_t *colB, unsigned full0,
-                                              unsigned empty0, volatile int *abort_flag, int a_srow, int a_sk,
-                                              int b_srow, int b_sk, int tid)
+                                              const int64_t *rowA, const int64_t *colB, const int64_t *koffA,
+                                              const int64_t *koffB, unsigned full0, unsigned empty0,
+                                              volatile int *abort_flag, int a_srow, int a_sk, int b_srow, int b_sk,
+                                              int tid)
 {
+    const bool staged = c.k_end - c.k_begin <= kKoffCap;
+    const int64_t *ka = staged ? koffA - c.k_begin : p.offA_k;
+    const int64_t *kb = staged ? koffB - c.k_begin : p.offB_k;
     for (int kt = 0; kt < c.num_kt; ++kt) {
         const int s = kt % STAGES, round = kt / STAGES;
         if (round > 0 &&
@@ -190,9 +205,9 @@ __device__ __forceinline__ void producer_loop(const Params &p, const TileCoords 
         const unsigned sa = stage0 + unsigned(s) * STAGE_BYTES;
         const unsigned sb = sa + A_BYTES;
         const int64_t k0 = c.k_begin + int64_t(kt) * BK;
-        gather_dispatch<BM, BK, PRODUCERS, EB>(sa, static_cast<const char *>(p.A), rowA, p.offA_k, c.rows_valid, k0,
+        gather_dispatch<BM, BK, PRODUCERS, EB>(sa, static_cast<const char *>(p.A), rowA, ka, c.rows_valid, k0,
                                                c.k_end, p.dirA, p.vecA, a_srow, a_sk, tid);
-        gather_dispatch<BN, BK, PRODUCERS, EB>(sb, static_cast<const char *>(p.B), colB, p.offB_k, c.cols_valid, k0,
+        gather_dispatch<BN, BK, PRODUCERS, EB>(sb, static_cast<const char *>(p.B), colB, kb, c.cols_valid, k0,
                                                c.k_end, p.dirB, p.vecB, b_srow, b_sk, tid);
         mbar_arrive_on_copies(full0 + 8u * s);
     }

@@ -41,7 +41,7 @@ struct F32Tile {
     static constexpr int B_ELEMS = (BK * PITCH_FREE_B > BN * PITCH_K) ? BK * PITCH_FREE_B : BN * PITCH_K;
     static constexpr int STAGE_FLOATS = A_ELEMS + B_ELEMS;
     static constexpr size_t SMEM_BYTES =
-        size_t(STAGES) * STAGE_FLOATS * 4 + size_t(2 * BM + 2 * BN) * 8 + size_t(2 * STAGES) * 8 + 16;
+        size_t(STAGES) * STAGE_FLOATS * 4 + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
 
 // tile-local row of register-tile entry i (and column of entry j) for the two orientations
@@ -105,7 +105,9 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f32_kernel(cons
     int64_t *rowD = rowA + T::BM;
     int64_t *colB = rowD + T::BM;
     int64_t *colD = colB + T::BN;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(colD + T::BN);
+    int64_t *koffA = colD + T::BN;
+    int64_t *koffB = koffA + kKoffCap;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(koffB + kKoffCap);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * T::STAGES);
     const unsigned full0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
     const unsigned empty0 = full0 + 8u * T::STAGES;
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f32_kernel(cons
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
     tile_setup<T::BM, T::BN, T::STAGES, T::THREADS, T::PRODUCER_THREADS, T::CONSUMER_WARPS>(
-        p, tc, rowA, rowD, colB, colD, full0, empty0, abort_flag, tid);
+        p, tc, rowA, rowD, colB, colD, koffA, koffB, full0, empty0, abort_flag, tid);
 
     constexpr int a_srow = A_KMAJ ? T::PITCH_K : 1, a_sk = A_KMAJ ? 1 : T::PITCH_FREE_A;
     constexpr int b_srow = B_KMAJ ? T::PITCH_K : 1, b_sk = B_KMAJ ? 1 : T::PITCH_FREE_B;
@@ -122,7 +124,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f32_kernel(cons
         if (T::REBALANCE_REGS) reg_dec<40>();
         const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
         producer_loop<T::BM, T::BN, T::BK, 4, T::STAGES, T::STAGE_FLOATS * 4, T::A_ELEMS * 4, T::PRODUCER_THREADS>(
-            p, tc, stage0, rowA, colB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
+            p, tc, stage0, rowA, colB, koffA, koffB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
         return;
     }
 

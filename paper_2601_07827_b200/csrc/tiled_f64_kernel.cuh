@@ -65,7 +65,7 @@ struct F64Tile {
     static constexpr int STAGE_WORDS = (A_ELEMS + B_ELEMS) * W;
     // stages | row/column offset arrays | full[STAGES], empty[STAGES] mbarriers | abort flag
     static constexpr size_t SMEM_BYTES =
-        size_t(STAGES) * STAGE_WORDS * 8 + size_t(2 * BM + 2 * BN) * 8 + size_t(2 * STAGES) * 8 + 16;
+        size_t(STAGES) * STAGE_WORDS * 8 + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
 
 // m16n8k16: A rows g / g+8 (even / odd register), k = t + 4 (i / 2); B k = t + 4 j, column g;
@@ -146,7 +146,9 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     int64_t *rowD = rowA + T::BM;
     int64_t *colB = rowD + T::BM;
     int64_t *colD = colB + T::BN;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(colD + T::BN);      // full[STAGES], empty[STAGES]
+    int64_t *koffA = colD + T::BN;
+    int64_t *koffB = koffA + kKoffCap;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(koffB + kKoffCap);      // full[STAGES], empty[STAGES]
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * T::STAGES);
     const unsigned full0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
     const unsigned empty0 = full0 + 8u * T::STAGES;
@@ -155,7 +157,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
     const int rows_valid = tc.rows_valid, cols_valid = tc.cols_valid, num_kt = tc.num_kt;
     tile_setup<T::BM, T::BN, T::STAGES, T::THREADS, T::PRODUCER_THREADS, T::CONSUMER_WARPS>(
-        p, tc, rowA, rowD, colB, colD, full0, empty0, abort_flag, tid);
+        p, tc, rowA, rowD, colB, colD, koffA, koffB, full0, empty0, abort_flag, tid);
 
     // shared-memory orientation follows the load direction of each operand
     const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
@@ -166,7 +168,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
         if (T::REBALANCE_REGS) reg_dec<40>();
         const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
         producer_loop<T::BM, T::BN, T::BK, EB, T::STAGES, T::STAGE_WORDS * 8, T::A_ELEMS * EB, T::PRODUCER_THREADS>(
-            p, tc, stage0, rowA, colB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
+            p, tc, stage0, rowA, colB, koffA, koffB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
         return;
     }
 

@@ -47,7 +47,7 @@ struct TF32Tile {
     static constexpr int B_ELEMS = (BK * PITCH_FREE_B > BN * PITCH_K) ? BK * PITCH_FREE_B : BN * PITCH_K;
     static constexpr int STAGE_WORDS = (A_ELEMS + B_ELEMS) * W;
     static constexpr size_t SMEM_BYTES =
-        size_t(STAGES) * STAGE_WORDS * 4 + size_t(2 * BM + 2 * BN) * 8 + size_t(2 * STAGES) * 8 + 16;
+        size_t(STAGES) * STAGE_WORDS * 4 + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
 
 __device__ __forceinline__ void mma_tf32_m16n8k8(float (&c)[4], const unsigned (&a)[4], const unsigned (&b)[2])
@@ -128,7 +128,9 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
     int64_t *rowD = rowA + T::BM;
     int64_t *colB = rowD + T::BM;
     int64_t *colD = colB + T::BN;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(colD + T::BN);
+    int64_t *koffA = colD + T::BN;
+    int64_t *koffB = koffA + kKoffCap;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(koffB + kKoffCap);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * T::STAGES);
     const unsigned full0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
     const unsigned empty0 = full0 + 8u * T::STAGES;
@@ -136,7 +138,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
     tile_setup<T::BM, T::BN, T::STAGES, T::THREADS, T::PRODUCER_THREADS, T::CONSUMER_WARPS>(
-        p, tc, rowA, rowD, colB, colD, full0, empty0, abort_flag, tid);
+        p, tc, rowA, rowD, colB, colD, koffA, koffB, full0, empty0, abort_flag, tid);
 
     const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
     const int b_srow = p.dirB == 0 ? 1 : T::PITCH_K, b_sk = p.dirB == 0 ? T::PITCH_FREE_B : 1;
@@ -145,7 +147,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
         if (T::REBALANCE_REGS) reg_dec<40>();
         const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
         producer_loop<T::BM, T::BN, T::BK, EB, T::STAGES, T::STAGE_WORDS * 4, T::A_ELEMS * EB, T::PRODUCER_THREADS>(
-            p, tc, stage0, rowA, colB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
+            p, tc, stage0, rowA, colB, koffA, koffB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
         return;
     }
 
