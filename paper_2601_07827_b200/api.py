@@ -11,7 +11,7 @@ import os
 from typing import Optional, Sequence
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbtc.so")
+LIB_PATH = os.environ.get("BTC_LIB_PATH") or os.path.join(_HERE, "libbtc.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

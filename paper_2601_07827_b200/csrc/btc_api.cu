@@ -19,6 +19,10 @@
 
 using namespace btc;
 
+#ifdef BTC_STAMPS
+static __device__ long long btc_stamp_buffer[512 * 8];   // debug builds only
+#endif
+
 struct btc_handle_s {
     int device = -1;       // -1: no CUDA device (objects can be validated and planned, not run)
     int sm_count = 148;
@@ -139,7 +143,7 @@ cudaError_t launch_tiled(const TiledParams &p, int64_t ctas, int64_t reduce_ctas
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (p.split_k > 1) {
-        tiled_f64_splitk_reduce_kernel<T><<<unsigned(reduce_ctas), T::CONSUMER_THREADS, 0, st>>>(p);
+        splitk_reduce_kernel<double, T::W><<<unsigned(reduce_ctas), 256, 0, st>>>(p);
         e = cudaGetLastError();
     }
     return e;
@@ -155,7 +159,7 @@ cudaError_t launch_tiled_tf32(const TiledParams &p, int64_t ctas, int64_t reduce
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (p.split_k > 1) {
-        tiled_tf32x3_splitk_reduce_kernel<T><<<unsigned(reduce_ctas), T::CONSUMER_THREADS, 0, st>>>(p);
+        splitk_reduce_kernel<float, T::W><<<unsigned(reduce_ctas), 256, 0, st>>>(p);
         e = cudaGetLastError();
     }
     return e;
@@ -171,7 +175,7 @@ cudaError_t launch_tiled_f32_o(const TiledParams &p, int64_t ctas, int64_t reduc
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (p.split_k > 1) {
-        tiled_f32_splitk_reduce_kernel<T, AK, BK_><<<unsigned(reduce_ctas), T::CONSUMER_THREADS, 0, st>>>(p);
+        splitk_reduce_kernel<float, 1><<<unsigned(reduce_ctas), 256, 0, st>>>(p);
         e = cudaGetLastError();
     }
     return e;
@@ -602,6 +606,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         tp.offA_h = op->d_offA_h; tp.offB_h = op->d_offB_h; tp.offD_h = op->d_offD_h;
         tp.M = pl.M; tp.N = pl.N; tp.K = pl.K; tp.Bt = pl.Bt;
         tp.tiles_m = op->tiles_m; tp.tiles_n = op->tiles_n; tp.raster_n_fast = op->raster_n_fast;
+        tp.bm = pl.tile.bm; tp.bn = pl.tile.bn;
         tp.split_k = pl.split_k; tp.k_per_split = op->k_per_split;
         tp.dirA = int32_t(pl.dirA); tp.dirB = int32_t(pl.dirB);
         // vector copies need the base pointers aligned as well
@@ -612,8 +617,11 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         tp.alpha[0] = al[0]; tp.alpha[1] = al[1]; tp.beta[0] = be[0]; tp.beta[1] = be[1];
         tp.partials = workspace;
         tp.error_word = op->d_error;
+#ifdef BTC_STAMPS
+        { void *sp = nullptr; cudaGetSymbolAddress(&sp, btc_stamp_buffer); tp.stamps = static_cast<long long *>(sp); }
+#endif
         const int64_t ctas = op->grid[0];
-        const int64_t reduce_ctas = ctas / pl.split_k;
+        const int64_t reduce_ctas = (ctas / pl.split_k) * ((int64_t(pl.tile.bm) * pl.tile.bn + 1023) / 1024);
         // 16-byte stores of D (and loads of C) need those base pointers aligned too
         tp.vecD = (pl.vecD == 4 && !misaligned(D, 16) && !(use_c && misaligned(C, 16))) ? 4 : 1;
         if (pl.dtype == BTC_F32) {
@@ -712,6 +720,13 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
     if (ws) cudaFree(ws);
     return rc;
 }
+
+#ifdef BTC_STAMPS
+btc_error_t btc_debug_read_stamps(long long *dst)
+{
+    return cudaMemcpyFromSymbol(dst, btc_stamp_buffer, sizeof(long long) * 512 * 8) == cudaSuccess ? BTC_SUCCESS : BTC_ERR_CUDA;
+}
+#endif
 
 // ---- execute without any allocation -------------------------------------------------------------
 // Scratch for split-K partial sums that belongs to the library image itself: every GPU that loads

@@ -31,17 +31,21 @@ struct TiledParams {
     const int64_t *offA_h, *offB_h, *offD_h;   // [Bt]
     int64_t M, N, K, Bt;
     int32_t tiles_m, tiles_n;
+    int32_t bm, bn;                   // CTA tile extents in elements
     int32_t raster_n_fast;            // 1: consecutive CTAs walk the n tiles of one m tile
     int32_t split_k;
     int64_t k_per_split;              // multiple of the K tile
     int32_t dirA, dirB;               // 0: threads run along the free index, 1: along k
     int32_t vecA, vecB;               // elements per global->shared copy
-    int32_t vecD;                     // 4: four consecutive m are 16 consecutive, aligned bytes of D (fp32)
+    int32_t vecD;                     // v > 1: groups of v consecutive m are v consecutive, 16-byte aligned elements of D
     int32_t conjA, conjB, conjC;
     int32_t use_c;
     double alpha[2], beta[2];
     void *partials;                   // split-K scratch (workspace), or nullptr
     int32_t *error_word;              // device word; set non-zero when a bounded wait gave up
+#ifdef BTC_STAMPS
+    long long *stamps;                // debug build only: per-CTA phase time stamps (8 per CTA)
+#endif
 };
 
 }  // namespace btc

@@ -10,6 +10,13 @@
 namespace btc {
 
 constexpr int kProducerWarps = 4;   // one warpgroup
+
+// Debug builds (-DBTC_STAMPS) record the SM clock at a few points of each CTA's life.
+#ifdef BTC_STAMPS
+#define BTC_STAMP(p, slot) do { if ((p).stamps && blockIdx.x < 512) (p).stamps[blockIdx.x * 8 + (slot)] = clock64(); } while (0)
+#else
+#define BTC_STAMP(p, slot) do { } while (0)
+#endif
 // k-offset entries per operand that a CTA keeps in shared memory (its whole k slice when it fits)
 constexpr int kKoffCap = 1024;
 
@@ -84,14 +91,33 @@ __device__ __forceinline__ void gather_tile(unsigned smem, const char *__restric
 {
     constexpr int NFAST = (DIR == 0 ? ROWS : BK) / VEC;
     constexpr int SLOTS = ROWS * BK / VEC;
-#pragma unroll 4
-    for (int s = tid; s < SLOTS; s += NTHREADS) {
-        const int f = (s % NFAST) * VEC, o = s / NFAST;
-        const int r = DIR == 0 ? f : o;
-        const int k = DIR == 0 ? o : f;
-        const bool valid = (r < rows_valid) && (k0 + k < k_end);
-        const int64_t off = valid ? row_off[r] + koff[k0 + k] : 0;
-        cp_async_bytes<VEC * ELEM_BYTES>(smem + unsigned(r * s_row + k * s_k) * ELEM_BYTES, g + off * ELEM_BYTES, valid);
+    constexpr int PER = (SLOTS + NTHREADS - 1) / NTHREADS;     // copies per thread
+    constexpr int BATCH = PER < 4 ? PER : 4;
+    // offsets of a batch are looked up first and its copies issued together: a copy is an
+    // ordered memory operation, so interleaving would serialise every table look-up behind it
+#pragma unroll 1
+    for (int base = 0; base < PER; base += BATCH) {
+        int64_t off[BATCH];
+        bool valid[BATCH];
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) {
+            const int s = tid + (base + j) * NTHREADS;
+            const int f = (s % NFAST) * VEC, o = s / NFAST;
+            const int r = DIR == 0 ? f : o;
+            const int k = DIR == 0 ? o : f;
+            valid[j] = s < SLOTS && (r < rows_valid) && (k0 + k < k_end);
+            off[j] = valid[j] ? row_off[r] + koff[k0 + k] : 0;
+        }
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) {
+            const int s = tid + (base + j) * NTHREADS;
+            if (s < SLOTS) {
+                const int f = (s % NFAST) * VEC, o = s / NFAST;
+                const int r = DIR == 0 ? f : o;
+                const int k = DIR == 0 ? o : f;
+                cp_async_bytes<VEC * ELEM_BYTES>(smem + unsigned(r * s_row + k * s_k) * ELEM_BYTES, g + off[j] * ELEM_BYTES, valid[j]);
+            }
+        }
     }
 }
 

@@ -13,6 +13,7 @@
 
 #include <cuda_runtime.h>
 
+#include "epilogue_common.cuh"
 #include "kernel_params.h"
 #include "tile_common.cuh"
 
@@ -40,8 +41,10 @@ struct F32Tile {
     static constexpr int A_ELEMS = (BK * PITCH_FREE_A > BM * PITCH_K) ? BK * PITCH_FREE_A : BM * PITCH_K;
     static constexpr int B_ELEMS = (BK * PITCH_FREE_B > BN * PITCH_K) ? BK * PITCH_FREE_B : BN * PITCH_K;
     static constexpr int STAGE_FLOATS = A_ELEMS + B_ELEMS;
+    static constexpr size_t IMAGE_BYTES = size_t(BN) * (BM + 4) * 4;        // epilogue image of the tile
+    static constexpr size_t STAGES_BYTES = size_t(STAGES) * STAGE_FLOATS * 4;
     static constexpr size_t SMEM_BYTES =
-        size_t(STAGES) * STAGE_FLOATS * 4 + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
+        (STAGES_BYTES > IMAGE_BYTES ? STAGES_BYTES : IMAGE_BYTES) + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
 
 // tile-local row of register-tile entry i (and column of entry j) for the two orientations
@@ -54,54 +57,12 @@ template <bool KMAJ> __device__ __forceinline__ int f32_col_of(int tx, int j)
     return KMAJ ? tx + 4 * j : (j >> 2) * 16 + tx * 4 + (j & 3);
 }
 
-template <typename T, bool A_KMAJ>
-__device__ __forceinline__ void f32_epilogue(const TiledParams &p, const float (&acc)[T::TM][T::TN],
-                                             const int64_t *rowD, const int64_t *colD, int rows_valid,
-                                             int cols_valid, int wm0, int wn0, int ty, int tx, bool b_kmaj)
-{
-    float *D = static_cast<float *>(p.D);
-    const float *C = static_cast<const float *>(p.C);
-    const float alpha = float(p.alpha[0]), beta = float(p.beta[0]);
-#pragma unroll
-    for (int j = 0; j < T::TN; ++j) {
-        const int c = wn0 + (b_kmaj ? f32_col_of<true>(tx, j) : f32_col_of<false>(tx, j));
-        if (c >= cols_valid) continue;
-        const int64_t co = colD[c];
-        if (!A_KMAJ && p.vecD == 4) {
-            // 4 consecutive rows of this thread are 4 consecutive, 16-byte aligned floats of D
-#pragma unroll
-            for (int i4 = 0; i4 < T::TM / 4; ++i4) {
-                const int r = wm0 + f32_row_of<false>(ty, i4 * 4);
-                if (r >= rows_valid) continue;     // rows_valid is a multiple of 4 here
-                const int64_t off = rowD[r] + co;
-                float4 v = make_float4(alpha * acc[i4 * 4][j], alpha * acc[i4 * 4 + 1][j],
-                                       alpha * acc[i4 * 4 + 2][j], alpha * acc[i4 * 4 + 3][j]);
-                if (p.use_c) {
-                    const float4 cv = *reinterpret_cast<const float4 *>(C + off);
-                    v.x += beta * cv.x; v.y += beta * cv.y; v.z += beta * cv.z; v.w += beta * cv.w;
-                }
-                *reinterpret_cast<float4 *>(D + off) = v;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < T::TM; ++i) {
-                const int r = wm0 + f32_row_of<A_KMAJ>(ty, i);
-                if (r >= rows_valid) continue;
-                const int64_t off = rowD[r] + co;
-                float v = alpha * acc[i][j];
-                if (p.use_c) v += beta * C[off];
-                D[off] = v;
-            }
-        }
-    }
-}
-
 template <typename T, bool A_KMAJ, bool B_KMAJ>
 __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f32_kernel(const TiledParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *stage_base = reinterpret_cast<float *>(smem_raw);
-    int64_t *rowA = reinterpret_cast<int64_t *>(stage_base + size_t(T::STAGES) * T::STAGE_FLOATS);
+    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + (T::STAGES_BYTES > T::IMAGE_BYTES ? T::STAGES_BYTES : T::IMAGE_BYTES));
     int64_t *rowD = rowA + T::BM;
     int64_t *colB = rowD + T::BM;
     int64_t *colD = colB + T::BN;
@@ -204,58 +165,21 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f32_kernel(cons
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * s);
     }
-    if (!ok) return;
+    (void)ok;   // a wait that gave up has raised the CTA's abort flag
 
-    if (p.split_k == 1) {
-        f32_epilogue<T, A_KMAJ>(p, acc, rowD, colD, tc.rows_valid, tc.cols_valid, wm0, wn0, ty, tx, B_KMAJ);
-    } else {
-        // raw accumulators -> scratch, [batch][slice][tile][acc index][consumer thread]
-        float *dst = static_cast<float *>(p.partials) + size_t(blockIdx.x) * (size_t(T::CONSUMER_THREADS) * T::ACC) + ctid;
+    // Epilogue: register tile -> image of the CTA tile in the idle stage buffers -> rolled walk.
+    consumer_barrier<T::CONSUMER_THREADS>();
+    if (*abort_flag) return;
+    float *image = stage_base;
+    constexpr int P = ImagePitch<T::BM>::value;
 #pragma unroll
-        for (int i = 0; i < T::TM; ++i)
+    for (int j = 0; j < T::TN; ++j) {
+        const int c = wn0 + f32_col_of<B_KMAJ>(tx, j);
 #pragma unroll
-            for (int j = 0; j < T::TN; ++j) dst[size_t(i * T::TN + j) * T::CONSUMER_THREADS] = acc[i][j];
+        for (int i = 0; i < T::TM; ++i) image[c * P + wm0 + f32_row_of<A_KMAJ>(ty, i)] = acc[i][j];
     }
-}
-
-// Second pass of split-K (fixed-order sum of the slices, alpha/beta, strided store); thread i
-// takes over consumer thread i's accumulators.
-template <typename T, bool A_KMAJ, bool B_KMAJ>
-__global__ void __launch_bounds__(T::CONSUMER_THREADS) tiled_f32_splitk_reduce_kernel(const TiledParams p)
-{
-    __shared__ int64_t rowD[T::BM];
-    __shared__ int64_t colD[T::BN];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int tiles_i = p.tiles_m * p.tiles_n;
-    const int tile = blockIdx.x % tiles_i;
-    const int64_t h = blockIdx.x / tiles_i;
-    const int tile_m = p.raster_n_fast ? tile / p.tiles_n : tile % p.tiles_m;
-    const int tile_n = p.raster_n_fast ? tile % p.tiles_n : tile / p.tiles_m;
-    const int64_t m0 = int64_t(tile_m) * T::BM, n0 = int64_t(tile_n) * T::BN;
-    const int rows_valid = int(imin64(T::BM, p.M - m0));
-    const int cols_valid = int(imin64(T::BN, p.N - n0));
-    const int64_t hD = p.offD_h[h];
-    for (int i = tid; i < T::BM; i += T::CONSUMER_THREADS) rowD[i] = i < rows_valid ? p.offD_m[m0 + i] + hD : 0;
-    for (int i = tid; i < T::BN; i += T::CONSUMER_THREADS) colD[i] = i < cols_valid ? p.offD_n[n0 + i] : 0;
-    __syncthreads();
-
-    float acc[T::TM][T::TN];
-#pragma unroll
-    for (int i = 0; i < T::TM; ++i)
-#pragma unroll
-        for (int j = 0; j < T::TN; ++j) acc[i][j] = 0.f;
-    const float *ws = static_cast<const float *>(p.partials);
-    const size_t tiles = size_t(tiles_i);
-    for (int ks = 0; ks < p.split_k; ++ks) {
-        const size_t tile_lin = (size_t(h) * p.split_k + ks) * tiles + tile;
-        const float *src = ws + tile_lin * (size_t(T::CONSUMER_THREADS) * T::ACC) + tid;
-#pragma unroll
-        for (int i = 0; i < T::TM; ++i)
-#pragma unroll
-            for (int j = 0; j < T::TN; ++j) acc[i][j] += src[size_t(i * T::TN + j) * T::CONSUMER_THREADS];
-    }
-    const int wm0 = (warp % T::WARPS_M) * T::WM, wn0 = (warp / T::WARPS_M) * T::WN;
-    f32_epilogue<T, A_KMAJ>(p, acc, rowD, colD, rows_valid, cols_valid, wm0, wn0, lane >> 2, lane & 3, B_KMAJ);
+    consumer_barrier<T::CONSUMER_THREADS>();
+    store_tile_image<float, 1, T::BM, T::BN, T::CONSUMER_THREADS>(p, tc, image, rowD, colD, ctid);
 }
 
 }  // namespace btc

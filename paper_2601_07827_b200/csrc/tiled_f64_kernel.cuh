@@ -28,6 +28,7 @@
 
 #include <cuda_runtime.h>
 
+#include "epilogue_common.cuh"
 #include "kernel_params.h"
 #include "tile_common.cuh"
 
@@ -64,8 +65,10 @@ struct F64Tile {
     static constexpr int B_ELEMS = (BK * PITCH_FREE_B > BN * PITCH_K) ? BK * PITCH_FREE_B : BN * PITCH_K;
     static constexpr int STAGE_WORDS = (A_ELEMS + B_ELEMS) * W;
     // stages | row/column offset arrays | full[STAGES], empty[STAGES] mbarriers | abort flag
+    static constexpr size_t IMAGE_BYTES = size_t(BN) * (BM + 4) * W * 8;    // epilogue image of the tile
+    static constexpr size_t STAGES_BYTES = size_t(STAGES) * STAGE_WORDS * 8;
     static constexpr size_t SMEM_BYTES =
-        size_t(STAGES) * STAGE_WORDS * 8 + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
+        (STAGES_BYTES > IMAGE_BYTES ? STAGES_BYTES : IMAGE_BYTES) + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
 
 // m16n8k16: A rows g / g+8 (even / odd register), k = t + 4 (i / 2); B k = t + 4 j, column g;
@@ -85,56 +88,6 @@ __device__ __forceinline__ void dmma_m8n8k4(double &c0, double &c1, double a, do
                  : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
 
-// alpha * acc + beta * op(c) for one element, written through D's offsets
-template <bool CPLX>
-__device__ __forceinline__ void store_element(const TiledParams &p, int64_t off, double acc_r, double acc_i)
-{
-    double *D = static_cast<double *>(p.D);
-    const double *C = static_cast<const double *>(p.C);
-    if (CPLX) {
-        double d_r = p.alpha[0] * acc_r - p.alpha[1] * acc_i;
-        double d_i = p.alpha[0] * acc_i + p.alpha[1] * acc_r;
-        if (p.use_c) {
-            const double2 c = *reinterpret_cast<const double2 *>(C + 2 * off);
-            const double ci = p.conjC ? -c.y : c.y;
-            d_r += p.beta[0] * c.x - p.beta[1] * ci;
-            d_i += p.beta[0] * ci + p.beta[1] * c.x;
-        }
-        *reinterpret_cast<double2 *>(D + 2 * off) = make_double2(d_r, d_i);
-    } else {
-        double d = p.alpha[0] * acc_r;
-        if (p.use_c) d += p.beta[0] * C[off];
-        D[off] = d;
-    }
-}
-
-// Map accumulator (fi, fj, c) of a lane to its tile-local (row, column) in elements and write
-// every accumulator the thread holds.
-template <typename T>
-__device__ __forceinline__ void epilogue(const TiledParams &p, const double (&acc)[T::FM][T::FN][2],
-                                         const int64_t *rowD, const int64_t *colD, int rows_valid,
-                                         int cols_valid, int wm0, int wn0_words, int lane)
-{
-    const int g = lane >> 2, t = lane & 3;
-#pragma unroll
-    for (int fi = 0; fi < T::FM; ++fi) {
-        const int r = wm0 + fi * 8 + g;
-        if (r >= rows_valid) continue;
-        const int64_t ro = rowD[r];
-#pragma unroll
-        for (int fj = 0; fj < T::FN; ++fj) {
-            if (T::CPLX) {
-                const int c = (wn0_words + fj * 8) / 2 + t;
-                if (c < cols_valid) store_element<true>(p, ro + colD[c], acc[fi][fj][0], acc[fi][fj][1]);
-            } else {
-                const int c = wn0_words + fj * 8 + 2 * t;
-                if (c < cols_valid) store_element<false>(p, ro + colD[c], acc[fi][fj][0], 0.0);
-                if (c + 1 < cols_valid) store_element<false>(p, ro + colD[c + 1], acc[fi][fj][1], 0.0);
-            }
-        }
-    }
-}
-
 template <typename T>
 __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(const TiledParams p)
 {
@@ -142,7 +95,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     constexpr int W = T::W;
     constexpr int EB = 8 * W;
     double *stage_base = reinterpret_cast<double *>(smem_raw);
-    int64_t *rowA = reinterpret_cast<int64_t *>(stage_base + size_t(T::STAGES) * T::STAGE_WORDS);
+    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + (T::STAGES_BYTES > T::IMAGE_BYTES ? T::STAGES_BYTES : T::IMAGE_BYTES));
     int64_t *rowD = rowA + T::BM;
     int64_t *colB = rowD + T::BM;
     int64_t *colD = colB + T::BN;
@@ -154,8 +107,10 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     const unsigned empty0 = full0 + 8u * T::STAGES;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) BTC_STAMP(p, 0);
     const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
     const int rows_valid = tc.rows_valid, cols_valid = tc.cols_valid, num_kt = tc.num_kt;
+    (void)rows_valid; (void)cols_valid;
     tile_setup<T::BM, T::BN, T::STAGES, T::THREADS, T::PRODUCER_THREADS, T::CONSUMER_WARPS>(
         p, tc, rowA, rowD, colB, colD, koffA, koffB, full0, empty0, abort_flag, tid);
 
@@ -163,12 +118,14 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
     const int b_srow = p.dirB == 0 ? 1 : T::PITCH_K, b_sk = p.dirB == 0 ? T::PITCH_FREE_B : 1;
 
+    if (tid == 0) BTC_STAMP(p, 1);                      // set-up done
     if (warp < kProducerWarps) {
         // ------------------------------------------------------------------ producers
         if (T::REBALANCE_REGS) reg_dec<40>();
         const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
         producer_loop<T::BM, T::BN, T::BK, EB, T::STAGES, T::STAGE_WORDS * 8, T::A_ELEMS * EB, T::PRODUCER_THREADS>(
             p, tc, stage0, rowA, colB, koffA, koffB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
+        if (tid == 0) BTC_STAMP(p, 2);                  // producers done issuing
         return;
     }
 
@@ -215,6 +172,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
 #pragma unroll
         for (int j = 0; j < T::FN; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
 
+    if (ctid == 0) BTC_STAMP(p, 3);                     // consumers ready
     bool ok = true;
     for (int kt = 0; kt < num_kt; ++kt) {
         const int s = kt % T::STAGES, round = kt / T::STAGES;
@@ -222,6 +180,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
             ok = false;
             break;
         }
+        if (kt == 0 && ctid == 0) BTC_STAMP(p, 4);      // first stage has landed
         const double *sa = stage_base + size_t(s) * T::STAGE_WORDS;
         const double *sb = sa + T::A_ELEMS * W;
         if (T::MMA16) {
@@ -278,66 +237,34 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * s);
     }
-    if (!ok) return;
+    (void)ok;   // a wait that gave up has raised the CTA's abort flag
+    if (ctid == 0) BTC_STAMP(p, 5);                     // main loop done
 
-    if (p.split_k == 1) {
-        epilogue<T>(p, acc, rowD, colD, rows_valid, cols_valid, wm0, wn0w, lane);
-    } else {
-        // raw accumulators -> scratch, [batch][slice][tile][acc index][consumer thread]
-        double *ws = static_cast<double *>(p.partials);
-        double *dst = ws + size_t(blockIdx.x) * (size_t(T::CONSUMER_THREADS) * T::ACC) + ctid;
+    // Epilogue: park the fragments as an image of the tile (rows contiguous) in the now idle
+    // stage buffers, then all consumer threads walk it (see epilogue_common.cuh).
+    consumer_barrier<T::CONSUMER_THREADS>();        // every consumer warp is done reading the stages
+    if (*abort_flag) return;
+    double *image = stage_base;
+    constexpr int P = ImagePitch<T::BM>::value;
 #pragma unroll
-        for (int i = 0; i < T::FM; ++i)
+    for (int fi = 0; fi < T::FM; ++fi) {
+        const int r = wm0 + fi * 8 + g;
 #pragma unroll
-            for (int j = 0; j < T::FN; ++j) {
-                dst[size_t((i * T::FN + j) * 2 + 0) * T::CONSUMER_THREADS] = acc[i][j][0];
-                dst[size_t((i * T::FN + j) * 2 + 1) * T::CONSUMER_THREADS] = acc[i][j][1];
+        for (int fj = 0; fj < T::FN; ++fj) {
+            if (T::CPLX) {
+                const int c = (wn0w + fj * 8) / 2 + t;
+                *reinterpret_cast<double2 *>(image + size_t(c * P + r) * 2) = make_double2(acc[fi][fj][0], acc[fi][fj][1]);
+            } else {
+                const int c = wn0w + fj * 8 + 2 * t;
+                image[c * P + r] = acc[fi][fj][0];
+                image[(c + 1) * P + r] = acc[fi][fj][1];
             }
+        }
     }
-}
-
-// Second pass of split-K: fixed-order sum of the slices, then alpha/beta and the strided store.
-// Launched with T::CONSUMER_THREADS threads: thread i takes over consumer thread i's accumulators.
-template <typename T>
-__global__ void __launch_bounds__(T::CONSUMER_THREADS) tiled_f64_splitk_reduce_kernel(const TiledParams p)
-{
-    __shared__ int64_t rowD[T::BM];
-    __shared__ int64_t colD[T::BN];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // blockIdx.x enumerates (tile, batch), tile fastest
-    const int tiles_i = p.tiles_m * p.tiles_n;
-    const int tile = blockIdx.x % tiles_i;
-    const int64_t h = blockIdx.x / tiles_i;
-    const int tile_m = p.raster_n_fast ? tile / p.tiles_n : tile % p.tiles_m;
-    const int tile_n = p.raster_n_fast ? tile % p.tiles_n : tile / p.tiles_m;
-    const int64_t m0 = int64_t(tile_m) * T::BM, n0 = int64_t(tile_n) * T::BN;
-    const int rows_valid = int(imin64(T::BM, p.M - m0));
-    const int cols_valid = int(imin64(T::BN, p.N - n0));
-    const int64_t hD = p.offD_h[h];
-    for (int i = tid; i < T::BM; i += T::CONSUMER_THREADS) rowD[i] = i < rows_valid ? p.offD_m[m0 + i] + hD : 0;
-    for (int i = tid; i < T::BN; i += T::CONSUMER_THREADS) colD[i] = i < cols_valid ? p.offD_n[n0 + i] : 0;
-    __syncthreads();
-
-    double acc[T::FM][T::FN][2];
-#pragma unroll
-    for (int i = 0; i < T::FM; ++i)
-#pragma unroll
-        for (int j = 0; j < T::FN; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
-    const double *ws = static_cast<const double *>(p.partials);
-    const size_t tiles = size_t(p.tiles_m) * p.tiles_n;
-    for (int ks = 0; ks < p.split_k; ++ks) {
-        const size_t tile_lin = (size_t(h) * p.split_k + ks) * tiles + tile;
-        const double *src = ws + tile_lin * (size_t(T::CONSUMER_THREADS) * T::ACC) + tid;
-#pragma unroll
-        for (int i = 0; i < T::FM; ++i)
-#pragma unroll
-            for (int j = 0; j < T::FN; ++j) {
-                acc[i][j][0] += src[size_t((i * T::FN + j) * 2 + 0) * T::CONSUMER_THREADS];
-                acc[i][j][1] += src[size_t((i * T::FN + j) * 2 + 1) * T::CONSUMER_THREADS];
-            }
-    }
-    const int warp_m = warp % T::WARPS_M, warp_n = warp / T::WARPS_M;
-    epilogue<T>(p, acc, rowD, colD, rows_valid, cols_valid, warp_m * T::WM, warp_n * T::WNR, lane);
+    consumer_barrier<T::CONSUMER_THREADS>();
+    if (ctid == 0) BTC_STAMP(p, 6);                     // image parked
+    store_tile_image<double, W, T::BM, T::BN, T::CONSUMER_THREADS>(p, tc, image, rowD, colD, ctid);
+    if (ctid == 0) BTC_STAMP(p, 7);                     // stores issued
 }
 
 }  // namespace btc

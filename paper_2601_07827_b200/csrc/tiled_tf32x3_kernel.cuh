@@ -15,6 +15,7 @@
 
 #include <cuda_runtime.h>
 
+#include "epilogue_common.cuh"
 #include "kernel_params.h"
 #include "tile_common.cuh"
 
@@ -46,8 +47,10 @@ struct TF32Tile {
     static constexpr int A_ELEMS = (BK * PITCH_FREE_A > BM * PITCH_K) ? BK * PITCH_FREE_A : BM * PITCH_K;
     static constexpr int B_ELEMS = (BK * PITCH_FREE_B > BN * PITCH_K) ? BK * PITCH_FREE_B : BN * PITCH_K;
     static constexpr int STAGE_WORDS = (A_ELEMS + B_ELEMS) * W;
+    static constexpr size_t IMAGE_BYTES = size_t(BN) * (BM + 4) * W * 4;    // epilogue image of the tile
+    static constexpr size_t STAGES_BYTES = size_t(STAGES) * STAGE_WORDS * 4;
     static constexpr size_t SMEM_BYTES =
-        size_t(STAGES) * STAGE_WORDS * 4 + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
+        (STAGES_BYTES > IMAGE_BYTES ? STAGES_BYTES : IMAGE_BYTES) + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(2 * STAGES) * 8 + 16;
 };
 
 __device__ __forceinline__ void mma_tf32_m16n8k8(float (&c)[4], const unsigned (&a)[4], const unsigned (&b)[2])
@@ -66,65 +69,13 @@ __device__ __forceinline__ void split_tf32(float x, unsigned &hi, unsigned &lo)
 }
 
 template <typename T>
-__device__ __forceinline__ void tf32_store(const TiledParams &p, int64_t off, float acc_r, float acc_i)
-{
-    float *D = static_cast<float *>(p.D);
-    const float *C = static_cast<const float *>(p.C);
-    if (T::CPLX) {
-        const float ar = float(p.alpha[0]), ai = float(p.alpha[1]);
-        float d_r = ar * acc_r - ai * acc_i, d_i = ar * acc_i + ai * acc_r;
-        if (p.use_c) {
-            const float2 c = *reinterpret_cast<const float2 *>(C + 2 * off);
-            const float ci = p.conjC ? -c.y : c.y;
-            const float br = float(p.beta[0]), bi = float(p.beta[1]);
-            d_r += br * c.x - bi * ci;
-            d_i += br * ci + bi * c.x;
-        }
-        *reinterpret_cast<float2 *>(D + 2 * off) = make_float2(d_r, d_i);
-    } else {
-        float d = float(p.alpha[0]) * acc_r;
-        if (p.use_c) d += float(p.beta[0]) * C[off];
-        D[off] = d;
-    }
-}
-
-// accumulator fragment (fi, fj): c0,c1 -> row g, columns 2t, 2t+1; c2,c3 -> row g+8, same columns
-template <typename T>
-__device__ __forceinline__ void tf32_epilogue(const TiledParams &p, const float (&acc)[T::FM][T::FN][4],
-                                              const int64_t *rowD, const int64_t *colD, int rows_valid,
-                                              int cols_valid, int wm0, int wn0_words, int lane)
-{
-    const int g = lane >> 2, t = lane & 3;
-#pragma unroll
-    for (int fi = 0; fi < T::FM; ++fi)
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int r = wm0 + fi * 16 + half * 8 + g;
-            if (r >= rows_valid) continue;
-            const int64_t ro = rowD[r];
-#pragma unroll
-            for (int fj = 0; fj < T::FN; ++fj) {
-                const float v0 = acc[fi][fj][half * 2], v1 = acc[fi][fj][half * 2 + 1];
-                if (T::CPLX) {
-                    const int c = (wn0_words + fj * 8) / 2 + t;
-                    if (c < cols_valid) tf32_store<T>(p, ro + colD[c], v0, v1);
-                } else {
-                    const int c = wn0_words + fj * 8 + 2 * t;
-                    if (c < cols_valid) tf32_store<T>(p, ro + colD[c], v0, 0.f);
-                    if (c + 1 < cols_valid) tf32_store<T>(p, ro + colD[c + 1], v1, 0.f);
-                }
-            }
-        }
-}
-
-template <typename T>
 __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(const TiledParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     constexpr int W = T::W;
     constexpr int EB = 4 * W;
     float *stage_base = reinterpret_cast<float *>(smem_raw);
-    int64_t *rowA = reinterpret_cast<int64_t *>(stage_base + size_t(T::STAGES) * T::STAGE_WORDS);
+    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + (T::STAGES_BYTES > T::IMAGE_BYTES ? T::STAGES_BYTES : T::IMAGE_BYTES));
     int64_t *rowD = rowA + T::BM;
     int64_t *colB = rowD + T::BM;
     int64_t *colD = colB + T::BN;
@@ -136,6 +87,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
     const unsigned empty0 = full0 + 8u * T::STAGES;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) BTC_STAMP(p, 0);
     const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
     tile_setup<T::BM, T::BN, T::STAGES, T::THREADS, T::PRODUCER_THREADS, T::CONSUMER_WARPS>(
         p, tc, rowA, rowD, colB, colD, koffA, koffB, full0, empty0, abort_flag, tid);
@@ -143,11 +95,13 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
     const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
     const int b_srow = p.dirB == 0 ? 1 : T::PITCH_K, b_sk = p.dirB == 0 ? T::PITCH_FREE_B : 1;
 
+    if (tid == 0) BTC_STAMP(p, 1);                      // set-up done
     if (warp < kProducerWarps) {
         if (T::REBALANCE_REGS) reg_dec<40>();
         const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
         producer_loop<T::BM, T::BN, T::BK, EB, T::STAGES, T::STAGE_WORDS * 4, T::A_ELEMS * EB, T::PRODUCER_THREADS>(
             p, tc, stage0, rowA, colB, koffA, koffB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
+        if (tid == 0) BTC_STAMP(p, 2);                  // producers done issuing
         return;
     }
 
@@ -192,6 +146,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[i][j][c] = 0.f;
 
+    if (ctid == 0) BTC_STAMP(p, 3);                     // consumers ready
     bool ok = true;
     for (int kt = 0; kt < tc.num_kt; ++kt) {
         const int s = kt % T::STAGES, round = kt / T::STAGES;
@@ -199,6 +154,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
             ok = false;
             break;
         }
+        if (kt == 0 && ctid == 0) BTC_STAMP(p, 4);      // first stage has landed
         const float *sa = stage_base + size_t(s) * T::STAGE_WORDS;
         const float *sb = sa + T::A_ELEMS * W;
 #pragma unroll
@@ -235,63 +191,37 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
         __syncwarp();
         if (lane == 0) mbar_arrive(empty0 + 8u * s);
     }
-    if (!ok) return;
+    (void)ok;   // a wait that gave up has raised the CTA's abort flag
+    if (ctid == 0) BTC_STAMP(p, 5);                     // main loop done
 
-    if (p.split_k == 1) {
-        tf32_epilogue<T>(p, acc, rowD, colD, tc.rows_valid, tc.cols_valid, wm0, wn0w, lane);
-    } else {
-        float *dst = static_cast<float *>(p.partials) + size_t(blockIdx.x) * (size_t(T::CONSUMER_THREADS) * T::ACC) + ctid;
+    // Epilogue: fragments -> image of the tile in the idle stage buffers -> rolled walk.
+    // Fragment (fi, fj): c0, c1 -> row g, columns 2t, 2t+1; c2, c3 -> row g+8, same columns.
+    consumer_barrier<T::CONSUMER_THREADS>();
+    if (*abort_flag) return;
+    float *image = stage_base;
+    constexpr int P = ImagePitch<T::BM>::value;
 #pragma unroll
-        for (int i = 0; i < T::FM; ++i)
+    for (int fi = 0; fi < T::FM; ++fi)
 #pragma unroll
-            for (int j = 0; j < T::FN; ++j)
+        for (int half = 0; half < 2; ++half) {
+            const int r = wm0 + fi * 16 + half * 8 + g;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    dst[size_t((i * T::FN + j) * 4 + c) * T::CONSUMER_THREADS] = acc[i][j][c];
-    }
-}
-
-// Second pass of split-K (fixed-order sum of the slices, alpha/beta, strided store).
-template <typename T>
-__global__ void __launch_bounds__(T::CONSUMER_THREADS) tiled_tf32x3_splitk_reduce_kernel(const TiledParams p)
-{
-    __shared__ int64_t rowD[T::BM];
-    __shared__ int64_t colD[T::BN];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int tiles_i = p.tiles_m * p.tiles_n;
-    const int tile = blockIdx.x % tiles_i;
-    const int64_t h = blockIdx.x / tiles_i;
-    const int tile_m = p.raster_n_fast ? tile / p.tiles_n : tile % p.tiles_m;
-    const int tile_n = p.raster_n_fast ? tile % p.tiles_n : tile / p.tiles_m;
-    const int64_t m0 = int64_t(tile_m) * T::BM, n0 = int64_t(tile_n) * T::BN;
-    const int rows_valid = int(imin64(T::BM, p.M - m0));
-    const int cols_valid = int(imin64(T::BN, p.N - n0));
-    const int64_t hD = p.offD_h[h];
-    for (int i = tid; i < T::BM; i += T::CONSUMER_THREADS) rowD[i] = i < rows_valid ? p.offD_m[m0 + i] + hD : 0;
-    for (int i = tid; i < T::BN; i += T::CONSUMER_THREADS) colD[i] = i < cols_valid ? p.offD_n[n0 + i] : 0;
-    __syncthreads();
-
-    float acc[T::FM][T::FN][4];
-#pragma unroll
-    for (int i = 0; i < T::FM; ++i)
-#pragma unroll
-        for (int j = 0; j < T::FN; ++j)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) acc[i][j][c] = 0.f;
-    const float *ws = static_cast<const float *>(p.partials);
-    for (int ks = 0; ks < p.split_k; ++ks) {
-        const size_t tile_lin = (size_t(h) * p.split_k + ks) * size_t(tiles_i) + tile;
-        const float *src = ws + tile_lin * (size_t(T::CONSUMER_THREADS) * T::ACC) + tid;
-#pragma unroll
-        for (int i = 0; i < T::FM; ++i)
-#pragma unroll
-            for (int j = 0; j < T::FN; ++j)
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    acc[i][j][c] += src[size_t((i * T::FN + j) * 4 + c) * T::CONSUMER_THREADS];
-    }
-    const int wm0 = (warp % T::WARPS_M) * T::WM, wn0w = (warp / T::WARPS_M) * T::WNR;
-    tf32_epilogue<T>(p, acc, rowD, colD, rows_valid, cols_valid, wm0, wn0w, lane);
+            for (int fj = 0; fj < T::FN; ++fj) {
+                const float v0 = acc[fi][fj][half * 2], v1 = acc[fi][fj][half * 2 + 1];
+                if (T::CPLX) {
+                    const int c = (wn0w + fj * 8) / 2 + t;
+                    *reinterpret_cast<float2 *>(image + size_t(c * P + r) * 2) = make_float2(v0, v1);
+                } else {
+                    const int c = wn0w + fj * 8 + 2 * t;
+                    image[c * P + r] = v0;
+                    image[(c + 1) * P + r] = v1;
+                }
+            }
+        }
+    consumer_barrier<T::CONSUMER_THREADS>();
+    if (ctid == 0) BTC_STAMP(p, 6);                     // image parked
+    store_tile_image<float, W, T::BM, T::BN, T::CONSUMER_THREADS>(p, tc, image, rowD, colD, ctid);
+    if (ctid == 0) BTC_STAMP(p, 7);                     // stores issued
 }
 
 }  // namespace btc
