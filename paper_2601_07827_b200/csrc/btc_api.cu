@@ -58,12 +58,12 @@ namespace {
 
 // ---- tiled kernel variants -------------------------------------------------------------------
 using F64Big = F64Tile<false, 128, 128, 2, 4, 4, 1>;
-using F64Small = F64Tile<false, 64, 64, 2, 2, 4, 2>;
+using F64Small = F64Tile<false, 64, 64, 2, 4, 4, 2>;             // 8 consumer warps: two per scheduler
 using F64Big16 = F64Tile<false, 128, 128, 2, 4, 4, 1, true>;   // m16n8k16 MMAs
 using F64Big3 = F64Tile<false, 128, 128, 2, 4, 3, 1>;           // 3 stages
 using F64BigT = F64Tile<false, 128, 128, 4, 2, 4, 1>;           // warp tile 32 x 64
 using C64Big = F64Tile<true, 128, 64, 2, 4, 4, 1>;
-using C64Small = F64Tile<true, 64, 32, 2, 2, 4, 2>;
+using C64Small = F64Tile<true, 64, 32, 2, 4, 4, 2>;
 
 using F32Big = F32Tile<128, 128, 16, 2, 4, 5, 1, false>;
 using F32Small = F32Tile<64, 64, 16, 2, 2, 5, 2, false>;
@@ -72,9 +72,9 @@ using F32BigP = F32Tile<128, 128, 16, 2, 4, 5, 1, true>;
 using F32WideP = F32Tile<256, 96, 16, 4, 2, 5, 1, true>;
 using F32Big32 = F32Tile<128, 128, 32, 2, 4, 3, 1, false>;
 using F32Tc = TF32Tile<false, 128, 128, 2, 4, 4, 1>;             // 3xTF32 on the tensor cores
-using F32TcSmall = TF32Tile<false, 64, 64, 2, 2, 4, 2>;
+using F32TcSmall = TF32Tile<false, 64, 64, 2, 4, 4, 2>;
 using C32Tc = TF32Tile<true, 128, 64, 2, 4, 4, 1>;
-using C32TcSmall = TF32Tile<true, 64, 32, 2, 2, 4, 2>;
+using C32TcSmall = TF32Tile<true, 64, 32, 2, 4, 4, 2>;
 using F32TcWide = TF32Tile<false, 256, 96, 4, 2, 4, 1>;          // N = 96 fills the tile exactly
 using F32TcMid = TF32Tile<false, 128, 96, 2, 4, 4, 1>;
 constexpr int kNumF32Variants = 10;

@@ -29,7 +29,7 @@ struct F32Tile {
     static constexpr int PRODUCER_THREADS = 32 * kProducerWarps;
     static constexpr int THREADS = CONSUMER_THREADS + PRODUCER_THREADS;
     static constexpr int MIN_CTAS = MIN_CTAS_;
-    static constexpr bool REBALANCE_REGS = (THREADS == 384);
+    static constexpr bool REBALANCE_REGS = (THREADS == 384 && MIN_CTAS_ == 1);
     static constexpr int STAGES = STAGES_;
     static constexpr int WM = BM / WARPS_M, WN = BN / WARPS_N;
     static constexpr int TM = WM / 8, TN = WN / 4;    // a warp is 8 (rows) x 4 (columns) threads

@@ -50,7 +50,7 @@ struct F64Tile {
     static constexpr int MIN_CTAS = MIN_CTAS_;
     // with 12 warps the register file gives 168 registers per thread; the consumers need more,
     // the producers far fewer, so the warpgroups re-split the file (setmaxnreg)
-    static constexpr bool REBALANCE_REGS = (THREADS == 384);
+    static constexpr bool REBALANCE_REGS = (THREADS == 384 && MIN_CTAS_ == 1);
     static constexpr int STAGES = STAGES_;
     static constexpr int WM = BM / WARPS_M;           // warp tile rows
     static constexpr int WNR = BN * W / WARPS_N;      // warp tile columns in real words

@@ -33,7 +33,7 @@ struct TF32Tile {
     static constexpr int PRODUCER_THREADS = 32 * kProducerWarps;
     static constexpr int THREADS = CONSUMER_THREADS + PRODUCER_THREADS;
     static constexpr int MIN_CTAS = MIN_CTAS_;
-    static constexpr bool REBALANCE_REGS = (THREADS == 384);
+    static constexpr bool REBALANCE_REGS = (THREADS == 384 && MIN_CTAS_ == 1);
     static constexpr int STAGES = STAGES_;
     static constexpr int WM = BM / WARPS_M;           // warp tile rows
     static constexpr int WNR = BN * W / WARPS_N;      // warp tile columns in real words
