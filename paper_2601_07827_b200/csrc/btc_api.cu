@@ -16,6 +16,7 @@
 #include "tiled_f32_kernel.cuh"
 #include "tiled_f64_kernel.cuh"
 #include "tiled_tf32x3_kernel.cuh"
+#include "tiled_umma_tf32x3_kernel.cuh"
 
 using namespace btc;
 
@@ -77,7 +78,11 @@ using C32Tc = TF32Tile<true, 128, 64, 2, 4, 4, 1>;
 using C32TcSmall = TF32Tile<true, 64, 32, 2, 4, 4, 2>;
 using F32TcWide = TF32Tile<false, 256, 96, 4, 2, 4, 1>;          // N = 96 fills the tile exactly
 using F32TcMid = TF32Tile<false, 128, 96, 2, 4, 4, 1>;
-constexpr int kNumF32Variants = 10;
+using F32Umma96 = UmmaTile<96, 3>;                               // tcgen05 + tensor memory, 3xTF32
+using F32Umma128 = UmmaTile<128, 3>;
+using F32Umma256 = UmmaTile<256, 2>;
+constexpr int kNumF32Variants = 13;
+constexpr int kFirstUmmaVariant = 10;
 
 struct VariantInfo {
     int bm, bn, bk, threads, acc;
@@ -113,7 +118,10 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
         case 6: return info_of<F32Tc>(4);
         case 7: return info_of<F32TcSmall>(4);
         case 8: return info_of<F32TcWide>(4);
-        default: return info_of<F32TcMid>(4);
+        case 9: return info_of<F32TcMid>(4);
+        case 10: return {128, 96, 32, 256, 0, F32Umma96::SMEM_BYTES, 4};
+        case 11: return {128, 128, 32, 256, 0, F32Umma128::SMEM_BYTES, 4};
+        default: return {128, 256, 32, 256, 0, F32Umma256::SMEM_BYTES, 4};
         }
     }
     if (t == BTC_C32) return variant == 0 ? info_of<C32Tc>(4) : info_of<C32TcSmall>(4);
@@ -163,6 +171,16 @@ cudaError_t launch_tiled_tf32(const TiledParams &p, int64_t ctas, int64_t reduce
         e = cudaGetLastError();
     }
     return e;
+}
+
+template <typename T>
+cudaError_t launch_umma(const TiledParams &p, int64_t ctas, cudaStream_t st)
+{
+    static bool configured[64] = {};
+    cudaError_t e = set_smem_once(tiled_umma_tf32x3_kernel<T>, T::SMEM_BYTES, configured);
+    if (e != cudaSuccess) return e;
+    tiled_umma_tf32x3_kernel<T><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
+    return cudaGetLastError();
 }
 
 template <typename T, bool AK, bool BK_>
@@ -278,7 +296,10 @@ int finish_plan(btc_contraction_s *op)
     const int64_t tiles = tiles_for(v);
     const int64_t k_tiles = (pl.K + v.bk - 1) / v.bk;
     int64_t split = 1;
-    if (op->req.force_split_k > 0) {
+    const bool umma = pl.dtype == BTC_F32 && variant >= kFirstUmmaVariant;   // these keep all of K in one CTA
+    if (umma) {
+        split = 1;
+    } else if (op->req.force_split_k > 0) {
         split = op->req.force_split_k;
     } else if (tiles < sms) {
         split = (2 * int64_t(sms)) / tiles;
@@ -635,7 +656,10 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
             case 6: ce = launch_tiled_tf32<F32Tc>(tp, ctas, reduce_ctas, st); break;
             case 7: ce = launch_tiled_tf32<F32TcSmall>(tp, ctas, reduce_ctas, st); break;
             case 8: ce = launch_tiled_tf32<F32TcWide>(tp, ctas, reduce_ctas, st); break;
-            default: ce = launch_tiled_tf32<F32TcMid>(tp, ctas, reduce_ctas, st); break;
+            case 9: ce = launch_tiled_tf32<F32TcMid>(tp, ctas, reduce_ctas, st); break;
+            case 10: ce = launch_umma<F32Umma96>(tp, ctas, st); break;
+            case 11: ce = launch_umma<F32Umma128>(tp, ctas, st); break;
+            default: ce = launch_umma<F32Umma256>(tp, ctas, st); break;
             }
         } else if (pl.dtype == BTC_C32) {
             ce = pl.tile.variant == 0 ? launch_tiled_tf32<C32Tc>(tp, ctas, reduce_ctas, st)
