@@ -230,6 +230,37 @@ int make_plan(const PlanRequest &req, Plan &plan)
     std::stable_sort(plan.n.begin(), plan.n.end(), by_sD);
     std::stable_sort(plan.batch.begin(), plan.batch.end(), by_sD);
 
+    // When D's fastest free mode x is far apart in the input (rows of a tile would each start in
+    // a different DRAM page) and the input has a closer free mode y, block the two: a tile's rows
+    // become x_in (one 32-byte sector of D) times y_in (neighbouring rows of the input), so both
+    // the input reads and the D writes move whole sectors.  Splitting a mode is only a
+    // re-indexing: the outer parts follow as modes of their own.
+    const int64_t esz0 = int64_t(dtype_size(plan.dtype));
+    auto block_free_modes = [&](std::vector<Mode> &g, bool forA) {
+        if (g.size() < 2) return;
+        auto S = [&](const Mode &md) { return iabs(forA ? md.sA : md.sB); };
+        size_t y = 1;
+        for (size_t i = 2; i < g.size(); ++i)
+            if (S(g[i]) < S(g[y])) y = i;
+        if (S(g[0]) < 1024 || S(g[y]) * 8 > S(g[0])) return;      // x is close enough, or y no better
+        const int64_t x_in = largest_divisor_at_most(g[0].extent, std::max<int64_t>(1, 32 / esz0));
+        const int64_t y_in = largest_divisor_at_most(g[y].extent, std::max<int64_t>(1, 128 / x_in));
+        if (y_in < 2) return;
+        Mode xi = g[0], xo = g[0], yi = g[y], yo = g[y];
+        xi.extent = x_in; xo.extent = g[0].extent / x_in;
+        xo.sA *= x_in; xo.sB *= x_in; xo.sD *= x_in;
+        yi.extent = y_in; yo.extent = g[y].extent / y_in;
+        yo.sA *= y_in; yo.sB *= y_in; yo.sD *= y_in;
+        std::vector<Mode> out = {xi, yi};
+        if (xo.extent > 1) out.push_back(xo);
+        if (yo.extent > 1) out.push_back(yo);
+        for (size_t i = 1; i < g.size(); ++i)
+            if (i != y) out.push_back(g[i]);
+        g = out;
+    };
+    block_free_modes(plan.m, true);
+    block_free_modes(plan.n, false);
+
     // which direction of each input tile is closest to contiguous in memory
     auto min_k_stride = [&](bool forA, int &where) {
         int64_t best = INT64_MAX;

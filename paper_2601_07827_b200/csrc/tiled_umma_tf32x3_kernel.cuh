@@ -5,8 +5,9 @@
 //   converters  gather the strided A / B tiles through the offset tables with 16-byte global loads
 //               into registers (the next stage's loads are in flight while the current stage is
 //               converted), split every value into its TF32 head and tail, and store both as
-//               separate operand tiles in the shared-memory layout the tensor core reads without
-//               swizzling: 8 x 16-byte "core matrices".  An operand whose contiguous direction is
+//               separate operand tiles in the swizzled shared-memory layouts the tensor core
+//               reads (a warp's load covers whole 128-byte lines of global memory and its stores
+//               are free of bank conflicts).  An operand whose contiguous direction is
 //               k is stored K-major, one whose contiguous direction is the free index MN-major;
 //               the instruction descriptor carries that choice, so no transpose is ever made.
 //   MMA warp    one elected lane waits for a stage ("full" mbarrier, 256 arrivals), issues the
@@ -26,9 +27,10 @@
 
 namespace btc {
 
-template <int BN_, int STAGES_>
+template <int BN_, int STAGES_, int PREFETCH_ = 2>
 struct UmmaTile {
     static constexpr int BM = 128, BN = BN_, BK = 32;
+    static constexpr int PREFETCH = PREFETCH_;                       // stages of global loads in flight per thread
     static constexpr int STAGES = STAGES_;
     static constexpr int CONVERTER_WARPS = 8, CONVERTER_THREADS = 256;
     static constexpr int THREADS = CONVERTER_THREADS + 32;          // + the MMA warp
@@ -87,7 +89,7 @@ __device__ __forceinline__ bool elect_one()
 }
 
 // Shared-memory matrix descriptor: start address, leading and stride byte offsets (all in 16-byte
-// units), descriptor version 1, layout type (0: no swizzle, 1: 128-byte swizzle on 32-byte units).
+// units), descriptor version 1, layout type (1: 128-byte swizzle on 32-byte units, 2: 128-byte swizzle on 16-byte units).
 __device__ __forceinline__ uint64_t umma_smem_desc(unsigned saddr, unsigned lbo_bytes, unsigned sbo_bytes, unsigned layout)
 {
     return uint64_t((saddr >> 4) & 0x3fffu) | (uint64_t((lbo_bytes >> 4) & 0x3fffu) << 16) |
@@ -100,15 +102,21 @@ __host__ __device__ constexpr unsigned umma_instr_desc(int n, bool a_mn_major, b
            (unsigned(n >> 3) << 17) | (unsigned(128 >> 4) << 24);
 }
 
-// Byte position of a 16-byte piece inside one operand tile of R rows x 32 k.
-//   k-contiguous operand, K-major, no swizzle: piece = 4 consecutive k of one row at
-//        ((k/4) * R + row) * 16          [core matrix = 8 rows x 16 bytes; SBO 128, LBO 16 R]
+// Byte position of a 16-byte piece inside one operand tile of R rows x 32 k.  Both layouts are
+// 128-byte swizzles, and tiles are 1024-byte aligned so that the XOR on address bits equals the
+// XOR on tile offsets.
+//   k-contiguous operand, K-major, 128-byte swizzle on 16-byte units: a row is its 32 k = 128
+//        bytes, 8 rows form a 1024-byte atom (SBO 1024), and the 16-byte chunk index of a row is
+//        XORed with (row mod 8); piece = 4 consecutive k of one row.  A k-step of 8 advances the
+//        start address by 32 bytes inside the atom.
 //   free-index-contiguous operand, MN-major.  For 32-bit elements the tensor core accepts only
-//   the 128-byte swizzle on 32-byte units here: atoms of 32 rows x 4 k (4 lines of 128 bytes,
-//   the 32-byte unit of a line XORed with the line number), row atoms 512 bytes apart (LBO),
-//   k atoms 16 R bytes apart (SBO); piece = 4 consecutive rows at one k.  Tiles are 1024-byte
-//   aligned so that the XOR on address bits equals the XOR on tile offsets.
-template <int R> __device__ __forceinline__ unsigned piece_kmajor(int row, int k) { return unsigned(((k >> 2) * R + row) * 16); }
+//        the 128-byte swizzle on 32-byte units here: atoms of 32 rows x 4 k (4 lines of 128
+//        bytes, the 32-byte unit of a line XORed with the line number), row atoms 512 bytes
+//        apart (LBO), k atoms 16 R bytes apart (SBO); piece = 4 consecutive rows at one k.
+template <int R> __device__ __forceinline__ unsigned piece_kmajor(int row, int k)
+{
+    return unsigned((row >> 3) * 1024 + (row & 7) * 128 + ((((k >> 2) ^ row) & 7) << 4));
+}
 template <int R> __device__ __forceinline__ unsigned piece_mnmajor(int row, int k)
 {
     const int line = k & 3, unit = ((row & 31) >> 3) ^ line;
@@ -117,73 +125,178 @@ template <int R> __device__ __forceinline__ unsigned piece_mnmajor(int row, int 
 
 struct F4 { float v[4]; };
 
-// Which 16-byte piece converter slot s handles; the 8 lanes of a quarter warp store to 8
-// different 16-byte bank groups.
-//   dir 1 (k contiguous):    8 rows of one k-chunk, then the 8 chunks of the stage, then row groups
-//   dir 0 (rows contiguous): 2 adjacent row pieces x 4 k of one atom line set, then 8-row groups,
-//                            then the 8 k-atoms of the stage
-template <int R> __device__ __forceinline__ void umma_slot(int s, int dir, int &row, int &k)
+// What a converter thread needs to address one operand: the tile's row offsets (shared memory),
+// the k offsets indexed by absolute k (the staged copy in shared memory, or the global table),
+// and the valid ranges.
+struct UmmaOperand {
+    const float *g;
+    const int64_t *row_off;
+    const int64_t *koff;
+    int rows_valid;
+    int64_t k_begin, k_end;
+    int dir;                     // 1: k is the contiguous direction, 0: the rows are
+};
+
+// The 16-byte pieces of an R x 32 operand tile that converter thread ctid handles: R / 32 slots,
+// slot i = 4 consecutive elements along the contiguous direction starting at (row r0 + 32 i, k kq).
+//   dir 1 (k contiguous):    r0 = ctid / 8, kq = 4 (ctid mod 8): 8 lanes read the 128 bytes of a row
+//   dir 0 (rows contiguous): r0 = 4 (ctid mod 8), kq = ctid / 8: 8 lanes read 32 rows of one k
+// Either way a warp's global load covers 4 whole 128-byte lines, the 8 lanes of a quarter warp
+// store to 8 different 16-byte bank groups, a thread's slots share their k (one k-offset look-up
+// per stage) and keep their rows (row offsets and shared-memory positions are loop invariants:
+// slot i lies i * pstep bytes behind slot 0 in both layouts).
+template <int SLOTS> struct UmmaLane {
+    const float *base[SLOTS];    // vector path: operand base + row offset of slot i (slot 0 of the tile if outside)
+    unsigned pos0, pstep;
+    unsigned rows_in;            // vector path: bit i = slot i lies inside the tile's rows
+    int r0, kq;
+};
+
+template <int R, int SLOTS, bool VEC>
+__device__ __forceinline__ void umma_lane_init(UmmaLane<SLOTS> &l, const UmmaOperand &o, int ctid)
 {
-    if (dir == 1) {
-        row = (s & 7) + 8 * (s >> 6);
-        k = ((s >> 3) & 7) * 4;
-    } else {
-        const int rest = s >> 3;
-        row = (rest % (R / 8)) * 8 + (s & 1) * 4;
-        k = (rest / (R / 8)) * 4 + ((s >> 1) & 3);
+    l.r0 = o.dir == 1 ? ctid >> 3 : (ctid & 7) * 4;
+    l.kq = o.dir == 1 ? (ctid & 7) * 4 : ctid >> 3;
+    l.pos0 = o.dir == 1 ? piece_kmajor<R>(l.r0, l.kq) : piece_mnmajor<R>(l.r0, l.kq);
+    l.pstep = o.dir == 1 ? 4096u : 512u;
+    l.rows_in = 0;
+#pragma unroll
+    for (int i = 0; i < SLOTS; ++i) {
+        const bool in = l.r0 + 32 * i < o.rows_valid;
+        l.rows_in |= unsigned(in) << i;
+        l.base[i] = VEC ? o.g + o.row_off[in ? l.r0 + 32 * i : 0] : o.g;
     }
 }
 
-// One converter thread's pieces of an R x 32 operand tile: the global loads ...
-template <int R, int SLOTS>
-__device__ __forceinline__ void umma_gather(F4 (&reg)[SLOTS], const float *__restrict__ g, const int64_t *row_off,
-                                            const int64_t *koff, int rows_valid, int64_t k0, int64_t k_end, int dir,
-                                            int vec, int ctid)
+// The global loads of one stage ...  They carry no predicate and sit under no branch: a piece
+// outside the tile reads a valid element of the tile instead and is zeroed when it is converted.
+// A conditional load would end in a select that waits for the data, one memory round trip per
+// piece; this way the loads of a stage are issued back to back.  VEC: every piece is 16
+// contiguous, aligned bytes that are in range together; otherwise its 4 elements are loaded one
+// by one through the tables.
+template <int SLOTS, bool VEC>
+__device__ __forceinline__ void umma_gather(F4 (&reg)[SLOTS], const UmmaLane<SLOTS> &l, const UmmaOperand &o, int64_t k0)
 {
+    if (VEC) {
+        const int64_t kofs = o.koff[k0 + l.kq < o.k_end ? k0 + l.kq : o.k_begin];
 #pragma unroll
-    for (int i = 0; i < SLOTS; ++i) {
-        int row, k;
-        umma_slot<R>(ctid + i * 256, dir, row, k);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) reg[i].v[e] = 0.f;
-        if (row < rows_valid && k0 + k < k_end) {
-            if (vec == 4) {      // the 4 elements are 16 contiguous, aligned bytes and all in range
-                const float4 x = *reinterpret_cast<const float4 *>(g + row_off[row] + koff[k0 + k]);
-                reg[i].v[0] = x.x; reg[i].v[1] = x.y; reg[i].v[2] = x.z; reg[i].v[3] = x.w;
-            } else if (dir == 1) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (k0 + k + e < k_end) reg[i].v[e] = g[row_off[row] + koff[k0 + k + e]];
-            } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (row + e < rows_valid) reg[i].v[e] = g[row_off[row + e] + koff[k0 + k]];
-            }
+        for (int i = 0; i < SLOTS; ++i) {
+            const float4 x = *reinterpret_cast<const float4 *>(l.base[i] + kofs);
+            reg[i].v[0] = x.x, reg[i].v[1] = x.y, reg[i].v[2] = x.z, reg[i].v[3] = x.w;
         }
+    } else {
+#pragma unroll
+        for (int i = 0; i < SLOTS; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int re = l.r0 + 32 * i + (o.dir == 1 ? 0 : e);
+                const int64_t ke = k0 + l.kq + (o.dir == 1 ? e : 0);
+                const bool in = re < o.rows_valid && ke < o.k_end;
+                reg[i].v[e] = o.g[o.row_off[in ? re : 0] + o.koff[in ? ke : o.k_begin]];
+            }
     }
 }
 
-// ... and the split into TF32 head and tail with the stores into the hi / lo operand tiles
-template <int R, int SLOTS>
-__device__ __forceinline__ void umma_convert(const F4 (&reg)[SLOTS], unsigned hi_tile, unsigned lo_tile, int dir, int ctid)
+// ... and the split into TF32 head and tail with the stores into the hi / lo operand tiles.
+// `full`: the whole R x 32 stage lies inside the tensor, nothing has to be zeroed.
+template <int SLOTS>
+__device__ __forceinline__ void umma_convert(const F4 (&reg)[SLOTS], const UmmaLane<SLOTS> &l, const UmmaOperand &o,
+                                             int64_t k0, unsigned hi_tile, unsigned lo_tile, bool full)
 {
 #pragma unroll
     for (int i = 0; i < SLOTS; ++i) {
-        int row, k;
-        umma_slot<R>(ctid + i * 256, dir, row, k);
-        const unsigned pos = dir == 1 ? piece_kmajor<R>(row, k) : piece_mnmajor<R>(row, k);
         unsigned hi[4], lo[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            hi[e] = __float_as_uint(reg[i].v[e]) & 0xffffe000u;
-            lo[e] = __float_as_uint(reg[i].v[e] - __uint_as_float(hi[e])) & 0xffffe000u;
+            float x = reg[i].v[e];
+            if (!full) {
+                const int re = l.r0 + 32 * i + (o.dir == 1 ? 0 : e);
+                const int64_t ke = k0 + l.kq + (o.dir == 1 ? e : 0);
+                if (re >= o.rows_valid || ke >= o.k_end) x = 0.f;
+            }
+            hi[e] = __float_as_uint(x) & 0xffffe000u;
+            lo[e] = __float_as_uint(x - __uint_as_float(hi[e])) & 0xffffe000u;
         }
+        const unsigned pos = l.pos0 + unsigned(i) * l.pstep;
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(hi_tile + pos), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(lo_tile + pos), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
     }
 }
 
 constexpr int kErrAccumWait = 3;
+
+// Debug builds (-DBTC_STAMPS) add up the SM clock cycles one thread spends in each phase.
+#ifdef BTC_STAMPS
+#define BTC_PHASE_BEGIN() long long phase_t0 = clock64()
+#define BTC_PHASE_END(acc) do { const long long phase_t1 = clock64(); (acc) += phase_t1 - phase_t0; phase_t0 = phase_t1; } while (0)
+#define BTC_PHASE_STORE(p, who, slot, acc) do { if ((who) && (p).stamps && blockIdx.x < 512) (p).stamps[blockIdx.x * 8 + (slot)] = (acc); } while (0)
+#else
+#define BTC_PHASE_BEGIN() do { } while (0)
+#define BTC_PHASE_END(acc) do { } while (0)
+#define BTC_PHASE_STORE(p, who, slot, acc) do { } while (0)
+#endif
+
+// The converter warps' main loop.  A register ring keeps the loads of the next PF stages in
+// flight while a stage is converted; ring positions are compile-time register indices.
+template <typename T, bool VEC>
+__device__ __forceinline__ bool umma_converter_loop(const TiledParams &p, const TileCoords &tc, const UmmaOperand &opA,
+                                                    const UmmaOperand &opB, unsigned smem0, unsigned full0, unsigned empty0,
+                                                    volatile int *abort_flag, int tid)
+{
+    constexpr int PF = T::PREFETCH, NB = PF + 1;
+    F4 ra[NB][T::SLOTS_A], rb[NB][T::SLOTS_B];
+    UmmaLane<T::SLOTS_A> la;
+    UmmaLane<T::SLOTS_B> lb;
+    umma_lane_init<T::BM, T::SLOTS_A, VEC>(la, opA, tid);
+    umma_lane_init<T::BN, T::SLOTS_B, VEC>(lb, opB, tid);
+    const bool rows_full = opA.rows_valid == T::BM && opB.rows_valid == T::BN;
+#pragma unroll
+    for (int q = 0; q < PF; ++q)
+        if (q < tc.num_kt) {
+            const int64_t kq = tc.k_begin + int64_t(q) * T::BK;
+            umma_gather<T::SLOTS_A, VEC>(ra[q], la, opA, kq);
+            umma_gather<T::SLOTS_B, VEC>(rb[q], lb, opB, kq);
+        }
+    bool ok = true;
+    long long t_gather = 0, t_wait = 0, t_convert = 0, t_signal = 0;
+    (void)t_gather; (void)t_wait; (void)t_convert; (void)t_signal;
+    BTC_PHASE_BEGIN();
+#pragma unroll 1
+    for (int kt0 = 0; ok && kt0 < tc.num_kt; kt0 += NB) {
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            const int kt = kt0 + b;
+            if (kt >= tc.num_kt) break;
+            const int64_t k0 = tc.k_begin + int64_t(kt) * T::BK;
+            if (kt + PF < tc.num_kt) {
+                const int64_t k1 = k0 + int64_t(PF) * T::BK;
+                umma_gather<T::SLOTS_A, VEC>(ra[(b + PF) % NB], la, opA, k1);
+                umma_gather<T::SLOTS_B, VEC>(rb[(b + PF) % NB], lb, opB, k1);
+            }
+            BTC_PHASE_END(t_gather);
+            const int s = kt % T::STAGES, round = kt / T::STAGES;
+            if (round > 0 &&
+                !mbar_wait_bounded(empty0 + 8u * s, unsigned(round - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait)) {
+                ok = false;
+                break;
+            }
+            BTC_PHASE_END(t_wait);
+            const unsigned st = smem0 + unsigned(s) * T::STAGE_BYTES;
+            const bool full = rows_full && k0 + T::BK <= tc.k_end;
+            umma_convert<T::SLOTS_A>(ra[b], la, opA, k0, st, st + T::A_BYTES, full);
+            umma_convert<T::SLOTS_B>(rb[b], lb, opB, k0, st + 2 * T::A_BYTES, st + 2 * T::A_BYTES + T::B_BYTES, full);
+            BTC_PHASE_END(t_convert);
+            proxy_fence_async();                 // the tensor core reads these stores through the async proxy
+            mbar_arrive(full0 + 8u * s);
+            BTC_PHASE_END(t_signal);
+        }
+    }
+    BTC_PHASE_STORE(p, tid == 0, 0, t_gather);
+    BTC_PHASE_STORE(p, tid == 0, 1, t_wait);
+    BTC_PHASE_STORE(p, tid == 0, 2, t_convert);
+    BTC_PHASE_STORE(p, tid == 0, 3, t_signal);
+    return ok;
+}
 
 template <typename T>
 __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const TiledParams p)
@@ -247,42 +360,16 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     tc_fence_after();
     const unsigned tmem_acc = *tmem_slot;
     const bool staged = tc.k_end - tc.k_begin <= kKoffCap;
-    const int64_t *ka = staged ? koffA - tc.k_begin : p.offA_k;
-    const int64_t *kb = staged ? koffB - tc.k_begin : p.offB_k;
 
     if (warp < T::CONVERTER_WARPS) {
         // ------------------------------------------------------------- converters
-        const float *gA = static_cast<const float *>(p.A), *gB = static_cast<const float *>(p.B);
-        F4 ra[2][T::SLOTS_A], rb[2][T::SLOTS_B];
-        if (tc.num_kt > 0) {
-            umma_gather<T::BM, T::SLOTS_A>(ra[0], gA, rowA, ka, tc.rows_valid, tc.k_begin, tc.k_end, p.dirA, p.vecA, tid);
-            umma_gather<T::BN, T::SLOTS_B>(rb[0], gB, colB, kb, tc.cols_valid, tc.k_begin, tc.k_end, p.dirB, p.vecB, tid);
-        }
-        bool ok = true;
-#pragma unroll 1
-        for (int kt2 = 0; ok && kt2 < tc.num_kt; kt2 += 2) {
-#pragma unroll
-            for (int par = 0; par < 2; ++par) {      // register buffers alternate with compile-time indices
-                const int kt = kt2 + par;
-                if (kt >= tc.num_kt) break;
-                if (kt + 1 < tc.num_kt) {            // next stage's loads fly while this one is converted
-                    const int64_t k1 = tc.k_begin + int64_t(kt + 1) * T::BK;
-                    umma_gather<T::BM, T::SLOTS_A>(ra[par ^ 1], gA, rowA, ka, tc.rows_valid, k1, tc.k_end, p.dirA, p.vecA, tid);
-                    umma_gather<T::BN, T::SLOTS_B>(rb[par ^ 1], gB, colB, kb, tc.cols_valid, k1, tc.k_end, p.dirB, p.vecB, tid);
-                }
-                const int s = kt % T::STAGES, round = kt / T::STAGES;
-                if (round > 0 &&
-                    !mbar_wait_bounded(empty0 + 8u * s, unsigned(round - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait)) {
-                    ok = false;
-                    break;
-                }
-                const unsigned st = smem0 + unsigned(s) * T::STAGE_BYTES;
-                umma_convert<T::BM, T::SLOTS_A>(ra[par], st, st + T::A_BYTES, p.dirA, tid);
-                umma_convert<T::BN, T::SLOTS_B>(rb[par], st + 2 * T::A_BYTES, st + 2 * T::A_BYTES + T::B_BYTES, p.dirB, tid);
-                proxy_fence_async();                 // the tensor core reads these stores through the async proxy
-                mbar_arrive(full0 + 8u * s);
-            }
-        }
+        const UmmaOperand opA = {static_cast<const float *>(p.A), rowA, staged ? koffA - tc.k_begin : p.offA_k,
+                                 tc.rows_valid, tc.k_begin, tc.k_end, p.dirA};
+        const UmmaOperand opB = {static_cast<const float *>(p.B), colB, staged ? koffB - tc.k_begin : p.offB_k,
+                                 tc.cols_valid, tc.k_begin, tc.k_end, p.dirB};
+        const bool ok = (p.vecA == 4 && p.vecB == 4)
+                            ? umma_converter_loop<T, true>(p, tc, opA, opB, smem0, full0, empty0, abort_flag, tid)
+                            : umma_converter_loop<T, false>(p, tc, opA, opB, smem0, full0, empty0, abort_flag, tid);
 
         // ------------------------------------------------------------- epilogue
         if (ok && mbar_wait_bounded(accum_bar, 0u, abort_flag, p.error_word, kErrAccumWait)) {
@@ -322,11 +409,14 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         const bool a_mn = p.dirA == 0, b_mn = p.dirB == 0;
         const unsigned idesc = a_mn ? (b_mn ? IDESC_MM : IDESC_MK) : (b_mn ? IDESC_KM : IDESC_KK);
         // per operand: layout type, leading / stride byte offsets, start advance of one k-step (8 k)
-        const unsigned a_lay = a_mn ? 1u : 0u, a_lbo = a_mn ? 512u : 16u * T::BM, a_sbo = a_mn ? 16u * T::BM : 128u;
-        const unsigned b_lay = b_mn ? 1u : 0u, b_lbo = b_mn ? 512u : 16u * T::BN, b_sbo = b_mn ? 16u * T::BN : 128u;
-        const unsigned a_step = 32u * T::BM, b_step = 32u * T::BN;   // two k-chunks, or two k-atoms
+        const unsigned a_lay = a_mn ? 1u : 2u, a_lbo = a_mn ? 512u : 16u, a_sbo = a_mn ? 16u * T::BM : 1024u;
+        const unsigned b_lay = b_mn ? 1u : 2u, b_lbo = b_mn ? 512u : 16u, b_sbo = b_mn ? 16u * T::BN : 1024u;
+        const unsigned a_step = a_mn ? 32u * T::BM : 32u, b_step = b_mn ? 32u * T::BN : 32u;   // two k-atoms, or 8 k of a row
         const bool leader = elect_one();
         bool ok = true;
+        long long t_full = 0, t_issue = 0;
+        (void)t_full; (void)t_issue;
+        BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int kt = 0; ok && kt < tc.num_kt; ++kt) {
             const int s = kt % T::STAGES, round = kt / T::STAGES;
@@ -334,6 +424,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 ok = false;
                 break;
             }
+            BTC_PHASE_END(t_full);
             tc_fence_after();
             if (leader) {
                 const unsigned st = smem0 + unsigned(s) * T::STAGE_BYTES;
@@ -352,7 +443,10 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 if (kt + 1 == tc.num_kt) umma_commit(accum_bar);
             }
             __syncwarp();
+            BTC_PHASE_END(t_issue);
         }
+        BTC_PHASE_STORE(p, lane == 0, 4, t_full);
+        BTC_PHASE_STORE(p, lane == 0, 5, t_issue);
         tc_fence_before();
     }
 

@@ -122,7 +122,7 @@ def test_planner_groups_fusion_and_roles(api, handle):
     expect = {
         "cfg1_f64_small": ((1, 256, 256, 256), (0, 2, 2, 2), False),
         "cfg2_f64_ccsd_ladder": ((1, 16384, 1024, 16384), (0, 1, 1, 1), False),   # a plain GEMM after fusion
-        "cfg3_f32_batched_permuted": ((64, 9216, 96, 576), (1, 2, 1, 2), True),   # j is in B: roles swap
+        "cfg3_f32_batched_permuted": ((64, 9216, 96, 576), (1, 4, 1, 2), True),   # j is in B: roles swap; j and b are blocked
         "cfg4_c64_conj": ((1, 256, 16384, 2304), (0, 1, 2, 4), False),            # s and t are split
         "cfg5_f32_tensor_network": ((1, 1024, 1024, 64), (0, 5, 5, 3), False),
         "cfg5b_f32_tensor_network_rev": ((1, 1024, 1024, 64), (0, 5, 5, 3), True),
