@@ -78,9 +78,9 @@ using C32Tc = TF32Tile<true, 128, 64, 2, 4, 4, 1>;
 using C32TcSmall = TF32Tile<true, 64, 32, 2, 4, 4, 2>;
 using F32TcWide = TF32Tile<false, 256, 96, 4, 2, 4, 1>;          // N = 96 fills the tile exactly
 using F32TcMid = TF32Tile<false, 128, 96, 2, 4, 4, 1>;
-using F32Umma96 = UmmaTile<96, 3>;                               // tcgen05 + tensor memory, 3xTF32
-using F32Umma128 = UmmaTile<128, 3>;
-using F32Umma256 = UmmaTile<256, 2, 1>;
+using F32Umma96 = UmmaTile<96, 4, 2>;                              // tcgen05 + tensor memory, 3xTF32
+using F32Umma128 = UmmaTile<128, 4, 2>;
+using F32Umma256 = UmmaTile<256, 3, 1>;
 constexpr int kNumF32Variants = 13;
 constexpr int kFirstUmmaVariant = 10;
 

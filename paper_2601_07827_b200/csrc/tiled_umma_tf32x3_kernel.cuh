@@ -1,18 +1,23 @@
 // fp32 contraction on the 5th-generation tensor cores (tcgen05.mma kind::tf32, accumulators in
 // tensor memory), 3xTF32:  a*b = a_lo*b_hi + a_hi*b_lo + a_hi*b_hi  with x = x_hi + x_lo.
 //
-// CTA = 8 converter warps + 1 MMA warp, one CTA per SM, tile 128 x BN x 32 per stage.
-//   converters  gather the strided A / B tiles through the offset tables with 16-byte global loads
-//               into registers (the next stage's loads are in flight while the current stage is
-//               converted), split every value into its TF32 head and tail, and store both as
-//               separate operand tiles in the swizzled shared-memory layouts the tensor core
-//               reads (a warp's load covers whole 128-byte lines of global memory and its stores
-//               are free of bank conflicts).  An operand whose contiguous direction is
-//               k is stored K-major, one whose contiguous direction is the free index MN-major;
-//               the instruction descriptor carries that choice, so no transpose is ever made.
-//   MMA warp    one elected lane waits for a stage ("full" mbarrier, 256 arrivals), issues the
-//               4 k-steps x 3 MMAs of the stage and commits them to the stage's "empty" mbarrier;
-//               after the last stage it commits to the accumulator barrier.
+// CTA = 8 converter warps + 4 producer warps + 1 MMA warp, one CTA per SM, tile 128 x BN x 32
+// per stage.  Shared memory holds a deep ring of "raw" stages and a short ring of "tail" stages.
+//   producers   gather the strided A / B tiles through the offset tables with asynchronous
+//               16-byte copies (zero-filled outside the tensor) straight into the swizzled
+//               operand layouts the tensor core reads.  Asynchronous copies keep far more bytes
+//               in flight per SM than loads into registers can, which is what bounds this kernel.
+//               An operand whose contiguous direction is k is stored K-major, one whose
+//               contiguous direction is the free index MN-major; the instruction descriptor
+//               carries that choice, so no transpose is ever made.
+//   converters  The tensor core reads only the upper 19 bits of a 32-bit operand element, so the
+//               raw fp32 stage already is the head operand x_hi.  The converters read it, form
+//               the tail x - x_hi (exact in fp32) and store it at the same position of a tail
+//               stage: a position-independent, conflict-free pass over the stage.
+//   MMA warp    one elected lane waits for a tail stage ("tail full", 256 arrivals; it implies
+//               the raw stage), issues the 4 k-steps x 3 MMAs and commits them to the "raw empty"
+//               and "tail empty" mbarriers; after the last stage it commits to the accumulator
+//               barrier.
 //   epilogue    the converter warps read the accumulator from tensor memory (each warp its own
 //               32-lane quarter, one row of the tile per lane, so a warp's store of one column
 //               is 32 consecutive rows of D) and apply alpha / beta through D's offset tables.
@@ -27,23 +32,25 @@
 
 namespace btc {
 
-template <int BN_, int STAGES_, int PREFETCH_ = 2>
+template <int BN_, int RAW_STAGES_, int TAIL_STAGES_>
 struct UmmaTile {
     static constexpr int BM = 128, BN = BN_, BK = 32;
-    static constexpr int PREFETCH = PREFETCH_;                       // stages of global loads in flight per thread
-    static constexpr int STAGES = STAGES_;
+    static constexpr int RAW_STAGES = RAW_STAGES_, TAIL_STAGES = TAIL_STAGES_;
     static constexpr int CONVERTER_WARPS = 8, CONVERTER_THREADS = 256;
-    static constexpr int THREADS = CONVERTER_THREADS + 32;          // + the MMA warp
+    static constexpr int PRODUCER_WARPS = 4, PRODUCER_THREADS = 128;
+    static constexpr int MMA_WARP = CONVERTER_WARPS + PRODUCER_WARPS;
+    static constexpr int THREADS = CONVERTER_THREADS + PRODUCER_THREADS + 32;
     static constexpr int A_BYTES = BM * BK * 4, B_BYTES = BN * BK * 4;
-    static constexpr int STAGE_BYTES = 2 * A_BYTES + 2 * B_BYTES;   // hi and lo tile of each operand
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;           // same size for raw and tail stages
     static constexpr int TMEM_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
-    static constexpr int SLOTS_A = BM * BK / 4 / CONVERTER_THREADS; // 16-byte pieces per thread
-    static constexpr int SLOTS_B = BN * BK / 4 / CONVERTER_THREADS;
-    static_assert((BN * BK / 4) % CONVERTER_THREADS == 0, "B tile must divide among the converters");
+    static constexpr int PIECES = STAGE_BYTES / 16 / CONVERTER_THREADS;   // 16-byte pieces per converter thread
+    static constexpr int NUM_BARS = 2 * RAW_STAGES + 2 * TAIL_STAGES + 1;
+    static_assert(STAGE_BYTES % (16 * CONVERTER_THREADS) == 0, "a stage must divide among the converters");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "BN must suit UMMA N and the epilogue split");
-    // stages | row/col offsets | k offsets | full[S], empty[S], accum mbarriers | tmem ptr, abort
-    static constexpr size_t SMEM_BYTES = size_t(STAGES) * STAGE_BYTES + size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 +
-                                         size_t(2 * STAGES + 1) * 8 + 16 + 1024;   // + slack to align the tiles
+    // stages | row/col offsets | k offsets | mbarriers | tmem ptr, abort
+    static constexpr size_t SMEM_BYTES = size_t(RAW_STAGES + TAIL_STAGES) * STAGE_BYTES +
+                                         size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(NUM_BARS) * 8 + 16 +
+                                         1024;   // + slack to align the tiles
 };
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------------------
@@ -123,9 +130,8 @@ template <int R> __device__ __forceinline__ unsigned piece_mnmajor(int row, int 
     return unsigned(((k >> 2) * (R / 32) + (row >> 5)) * 512 + line * 128 + unit * 32 + (row & 7) * 4);
 }
 
-struct F4 { float v[4]; };
 
-// What a converter thread needs to address one operand: the tile's row offsets (shared memory),
+// What a producer thread needs to address one operand: the tile's row offsets (shared memory),
 // the k offsets indexed by absolute k (the staged copy in shared memory, or the global table),
 // and the valid ranges.
 struct UmmaOperand {
@@ -135,95 +141,87 @@ struct UmmaOperand {
     int rows_valid;
     int64_t k_begin, k_end;
     int dir;                     // 1: k is the contiguous direction, 0: the rows are
+    int vec;                     // 4: every 16-byte piece is contiguous, aligned and in range as a whole
 };
 
-// The 16-byte pieces of an R x 32 operand tile that converter thread ctid handles: R / 32 slots,
-// slot i = 4 consecutive elements along the contiguous direction starting at (row r0 + 32 i, k kq).
-//   dir 1 (k contiguous):    r0 = ctid / 8, kq = 4 (ctid mod 8): 8 lanes read the 128 bytes of a row
-//   dir 0 (rows contiguous): r0 = 4 (ctid mod 8), kq = ctid / 8: 8 lanes read 32 rows of one k
-// Either way a warp's global load covers 4 whole 128-byte lines, the 8 lanes of a quarter warp
-// store to 8 different 16-byte bank groups, a thread's slots share their k (one k-offset look-up
-// per stage) and keep their rows (row offsets and shared-memory positions are loop invariants:
-// slot i lies i * pstep bytes behind slot 0 in both layouts).
-template <int SLOTS> struct UmmaLane {
-    const float *base[SLOTS];    // vector path: operand base + row offset of slot i (slot 0 of the tile if outside)
-    unsigned pos0, pstep;
-    unsigned rows_in;            // vector path: bit i = slot i lies inside the tile's rows
+// The 16-byte pieces of an R x 32 operand tile that producer thread pt (0..127) copies: R / 16
+// slots, each 4 consecutive elements along the contiguous direction.
+//   dir 1 (k contiguous):    rows r0 + 16 i at k kq,  r0 = pt / 8, kq = 4 (pt mod 8):
+//                            8 lanes copy the 128 bytes of one row
+//   dir 0 (rows contiguous): rows r0 + 32 j at k kq + 16 h,  r0 = 4 (pt mod 8), kq = pt / 8,
+//                            slot i = j + (R / 32) h: 8 lanes copy 32 rows of one k
+// Either way a warp's copy covers 4 whole 128-byte lines of global memory, a thread keeps its
+// rows for the whole k loop (row offsets and shared-memory positions are loop invariants) and
+// needs at most two k-offset look-ups per stage.
+template <int R> struct UmmaProducerLane {
+    static constexpr int SLOTS = R / 16;
+    int64_t rowoff[SLOTS];       // element offset of slot i's first row (0 if outside the tile)
+    unsigned rows_in;            // bit i = slot i's first row lies inside the tile
+    unsigned pos0;               // byte position of slot 0 in the operand tile
     int r0, kq;
 };
 
-template <int R, int SLOTS, bool VEC>
-__device__ __forceinline__ void umma_lane_init(UmmaLane<SLOTS> &l, const UmmaOperand &o, int ctid)
+template <int R> __device__ __forceinline__ int umma_slot_row(int dir, int r0, int i) { return dir == 1 ? r0 + 16 * i : r0 + 32 * (i % (R / 32)); }
+template <int R> __device__ __forceinline__ int umma_slot_half(int dir, int i) { return dir == 1 ? 0 : i / (R / 32); }
+template <int R> __device__ __forceinline__ unsigned umma_slot_pos(int dir, int i)
 {
-    l.r0 = o.dir == 1 ? ctid >> 3 : (ctid & 7) * 4;
-    l.kq = o.dir == 1 ? (ctid & 7) * 4 : ctid >> 3;
+    return dir == 1 ? 2048u * unsigned(i) : 512u * unsigned(i % (R / 32)) + unsigned(R * 64) * unsigned(i / (R / 32));
+}
+
+template <int R>
+__device__ __forceinline__ void umma_producer_init(UmmaProducerLane<R> &l, const UmmaOperand &o, int pt)
+{
+    l.r0 = o.dir == 1 ? pt >> 3 : (pt & 7) * 4;
+    l.kq = o.dir == 1 ? (pt & 7) * 4 : pt >> 3;
     l.pos0 = o.dir == 1 ? piece_kmajor<R>(l.r0, l.kq) : piece_mnmajor<R>(l.r0, l.kq);
-    l.pstep = o.dir == 1 ? 4096u : 512u;
     l.rows_in = 0;
 #pragma unroll
-    for (int i = 0; i < SLOTS; ++i) {
-        const bool in = l.r0 + 32 * i < o.rows_valid;
+    for (int i = 0; i < UmmaProducerLane<R>::SLOTS; ++i) {
+        const int row = umma_slot_row<R>(o.dir, l.r0, i);
+        const bool in = row < o.rows_valid;
         l.rows_in |= unsigned(in) << i;
-        l.base[i] = VEC ? o.g + o.row_off[in ? l.r0 + 32 * i : 0] : o.g;
+        l.rowoff[i] = o.row_off[in ? row : 0];
     }
 }
 
-// The global loads of one stage ...  They carry no predicate and sit under no branch: a piece
-// outside the tile reads a valid element of the tile instead and is zeroed when it is converted.
-// A conditional load would end in a select that waits for the data, one memory round trip per
-// piece; this way the loads of a stage are issued back to back.  VEC: every piece is 16
-// contiguous, aligned bytes that are in range together; otherwise its 4 elements are loaded one
-// by one through the tables.
-template <int SLOTS, bool VEC>
-__device__ __forceinline__ void umma_gather(F4 (&reg)[SLOTS], const UmmaLane<SLOTS> &l, const UmmaOperand &o, int64_t k0)
+// The copies of one operand for one stage.  Look-ups first, copies after: a copy is an ordered
+// memory operation, so a look-up placed behind one would wait for it.
+template <int R>
+__device__ __forceinline__ void umma_produce(unsigned tile, const UmmaProducerLane<R> &l, const UmmaOperand &o, int64_t k0)
 {
-    if (VEC) {
-        const int64_t kofs = o.koff[k0 + l.kq < o.k_end ? k0 + l.kq : o.k_begin];
+    constexpr int SLOTS = UmmaProducerLane<R>::SLOTS;
+    if (o.vec == 4) {
+        const int64_t ka = k0 + l.kq, kb = ka + 16;
+        const bool in0 = ka < o.k_end, in1 = o.dir == 0 && kb < o.k_end;
+        const int64_t kofs0 = o.koff[in0 ? ka : o.k_begin], kofs1 = o.koff[in1 ? kb : o.k_begin];
 #pragma unroll
         for (int i = 0; i < SLOTS; ++i) {
-            const float4 x = *reinterpret_cast<const float4 *>(l.base[i] + kofs);
-            reg[i].v[0] = x.x, reg[i].v[1] = x.y, reg[i].v[2] = x.z, reg[i].v[3] = x.w;
+            const bool second = umma_slot_half<R>(o.dir, i) != 0;
+            const bool valid = ((l.rows_in >> i) & 1u) && (second ? in1 : in0);
+            cp_async_bytes<16>(tile + l.pos0 + umma_slot_pos<R>(o.dir, i), o.g + l.rowoff[i] + (second ? kofs1 : kofs0), valid);
         }
     } else {
-#pragma unroll
-        for (int i = 0; i < SLOTS; ++i)
+#pragma unroll 2
+        for (int i = 0; i < SLOTS; ++i) {
+            const int row = umma_slot_row<R>(o.dir, l.r0, i);
+            const int64_t k = k0 + l.kq + 16 * umma_slot_half<R>(o.dir, i);
+            int64_t off[4];
+            bool in[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int re = l.r0 + 32 * i + (o.dir == 1 ? 0 : e);
-                const int64_t ke = k0 + l.kq + (o.dir == 1 ? e : 0);
-                const bool in = re < o.rows_valid && ke < o.k_end;
-                reg[i].v[e] = o.g[o.row_off[in ? re : 0] + o.koff[in ? ke : o.k_begin]];
+                const int re = row + (o.dir == 1 ? 0 : e);
+                const int64_t ke = k + (o.dir == 1 ? e : 0);
+                in[e] = re < o.rows_valid && ke < o.k_end;
+                off[e] = in[e] ? o.row_off[re] + o.koff[ke] : 0;
             }
-    }
-}
-
-// ... and the split into TF32 head and tail with the stores into the hi / lo operand tiles.
-// `full`: the whole R x 32 stage lies inside the tensor, nothing has to be zeroed.
-template <int SLOTS>
-__device__ __forceinline__ void umma_convert(const F4 (&reg)[SLOTS], const UmmaLane<SLOTS> &l, const UmmaOperand &o,
-                                             int64_t k0, unsigned hi_tile, unsigned lo_tile, bool full)
-{
 #pragma unroll
-    for (int i = 0; i < SLOTS; ++i) {
-        unsigned hi[4], lo[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            float x = reg[i].v[e];
-            if (!full) {
-                const int re = l.r0 + 32 * i + (o.dir == 1 ? 0 : e);
-                const int64_t ke = k0 + l.kq + (o.dir == 1 ? e : 0);
-                if (re >= o.rows_valid || ke >= o.k_end) x = 0.f;
-            }
-            hi[e] = __float_as_uint(x) & 0xffffe000u;
-            lo[e] = __float_as_uint(x - __uint_as_float(hi[e])) & 0xffffe000u;
+            for (int e = 0; e < 4; ++e)
+                cp_async_bytes<4>(tile + l.pos0 + umma_slot_pos<R>(o.dir, i) + 4u * e, o.g + off[e], in[e]);
         }
-        const unsigned pos = l.pos0 + unsigned(i) * l.pstep;
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(hi_tile + pos), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(lo_tile + pos), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
     }
 }
 
-constexpr int kErrAccumWait = 3;
+constexpr int kErrAccumWait = 3, kErrTailFullWait = 4, kErrTailEmptyWait = 5;
 
 // Debug builds (-DBTC_STAMPS) add up the SM clock cycles one thread spends in each phase.
 #ifdef BTC_STAMPS
@@ -236,68 +234,6 @@ constexpr int kErrAccumWait = 3;
 #define BTC_PHASE_STORE(p, who, slot, acc) do { } while (0)
 #endif
 
-// The converter warps' main loop.  A register ring keeps the loads of the next PF stages in
-// flight while a stage is converted; ring positions are compile-time register indices.
-template <typename T, bool VEC>
-__device__ __forceinline__ bool umma_converter_loop(const TiledParams &p, const TileCoords &tc, const UmmaOperand &opA,
-                                                    const UmmaOperand &opB, unsigned smem0, unsigned full0, unsigned empty0,
-                                                    volatile int *abort_flag, int tid)
-{
-    constexpr int PF = T::PREFETCH, NB = PF + 1;
-    F4 ra[NB][T::SLOTS_A], rb[NB][T::SLOTS_B];
-    UmmaLane<T::SLOTS_A> la;
-    UmmaLane<T::SLOTS_B> lb;
-    umma_lane_init<T::BM, T::SLOTS_A, VEC>(la, opA, tid);
-    umma_lane_init<T::BN, T::SLOTS_B, VEC>(lb, opB, tid);
-    const bool rows_full = opA.rows_valid == T::BM && opB.rows_valid == T::BN;
-#pragma unroll
-    for (int q = 0; q < PF; ++q)
-        if (q < tc.num_kt) {
-            const int64_t kq = tc.k_begin + int64_t(q) * T::BK;
-            umma_gather<T::SLOTS_A, VEC>(ra[q], la, opA, kq);
-            umma_gather<T::SLOTS_B, VEC>(rb[q], lb, opB, kq);
-        }
-    bool ok = true;
-    long long t_gather = 0, t_wait = 0, t_convert = 0, t_signal = 0;
-    (void)t_gather; (void)t_wait; (void)t_convert; (void)t_signal;
-    BTC_PHASE_BEGIN();
-#pragma unroll 1
-    for (int kt0 = 0; ok && kt0 < tc.num_kt; kt0 += NB) {
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            const int kt = kt0 + b;
-            if (kt >= tc.num_kt) break;
-            const int64_t k0 = tc.k_begin + int64_t(kt) * T::BK;
-            if (kt + PF < tc.num_kt) {
-                const int64_t k1 = k0 + int64_t(PF) * T::BK;
-                umma_gather<T::SLOTS_A, VEC>(ra[(b + PF) % NB], la, opA, k1);
-                umma_gather<T::SLOTS_B, VEC>(rb[(b + PF) % NB], lb, opB, k1);
-            }
-            BTC_PHASE_END(t_gather);
-            const int s = kt % T::STAGES, round = kt / T::STAGES;
-            if (round > 0 &&
-                !mbar_wait_bounded(empty0 + 8u * s, unsigned(round - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait)) {
-                ok = false;
-                break;
-            }
-            BTC_PHASE_END(t_wait);
-            const unsigned st = smem0 + unsigned(s) * T::STAGE_BYTES;
-            const bool full = rows_full && k0 + T::BK <= tc.k_end;
-            umma_convert<T::SLOTS_A>(ra[b], la, opA, k0, st, st + T::A_BYTES, full);
-            umma_convert<T::SLOTS_B>(rb[b], lb, opB, k0, st + 2 * T::A_BYTES, st + 2 * T::A_BYTES + T::B_BYTES, full);
-            BTC_PHASE_END(t_convert);
-            proxy_fence_async();                 // the tensor core reads these stores through the async proxy
-            mbar_arrive(full0 + 8u * s);
-            BTC_PHASE_END(t_signal);
-        }
-    }
-    BTC_PHASE_STORE(p, tid == 0, 0, t_gather);
-    BTC_PHASE_STORE(p, tid == 0, 1, t_wait);
-    BTC_PHASE_STORE(p, tid == 0, 2, t_convert);
-    BTC_PHASE_STORE(p, tid == 0, 3, t_signal);
-    return ok;
-}
-
 template <typename T>
 __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const TiledParams p)
 {
@@ -305,22 +241,26 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     // operand tiles must sit on 1024-byte boundaries of the shared-memory window (swizzled layouts)
     unsigned char *smem_raw = smem_unaligned +
         ((1024u - (static_cast<unsigned>(__cvta_generic_to_shared(smem_unaligned)) & 1023u)) & 1023u);
-    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + size_t(T::STAGES) * T::STAGE_BYTES);
+    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + size_t(T::RAW_STAGES + T::TAIL_STAGES) * T::STAGE_BYTES);
     int64_t *rowD = rowA + T::BM;
     int64_t *colB = rowD + T::BM;
     int64_t *colD = colB + T::BN;
     int64_t *koffA = colD + T::BN;
     int64_t *koffB = koffA + kKoffCap;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(koffB + kKoffCap);      // full[S], empty[S], accum
-    unsigned *tmem_slot = reinterpret_cast<unsigned *>(bars + 2 * T::STAGES + 1);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(koffB + kKoffCap);
+    unsigned *tmem_slot = reinterpret_cast<unsigned *>(bars + T::NUM_BARS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    const unsigned smem0 = static_cast<unsigned>(__cvta_generic_to_shared(smem_raw));
-    const unsigned full0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
-    const unsigned empty0 = full0 + 8u * T::STAGES;
-    const unsigned accum_bar = empty0 + 8u * T::STAGES;
+    const unsigned raw0 = static_cast<unsigned>(__cvta_generic_to_shared(smem_raw));
+    const unsigned tail0 = raw0 + unsigned(T::RAW_STAGES) * T::STAGE_BYTES;
+    const unsigned raw_full0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
+    const unsigned raw_empty0 = raw_full0 + 8u * T::RAW_STAGES;
+    const unsigned tail_full0 = raw_empty0 + 8u * T::RAW_STAGES;
+    const unsigned tail_empty0 = tail_full0 + 8u * T::TAIL_STAGES;
+    const unsigned accum_bar = tail_empty0 + 8u * T::TAIL_STAGES;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
+    const bool staged = tc.k_end - tc.k_begin <= kKoffCap;
 
     // ---- set-up: offset arrays, barriers, tensor memory ----
     {
@@ -335,22 +275,25 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             colB[i] = v ? p.offB_n[tc.n0 + i] + hB : 0;
             colD[i] = v ? p.offD_n[tc.n0 + i] : 0;
         }
-        const bool staged = tc.k_end - tc.k_begin <= kKoffCap;
         if (staged)
             for (int i = tid; i < int(tc.k_end - tc.k_begin); i += T::THREADS) {
                 koffA[i] = p.offA_k[tc.k_begin + i];
                 koffB[i] = p.offB_k[tc.k_begin + i];
             }
         if (tid == 0) {
-            for (int s = 0; s < T::STAGES; ++s) {
-                mbar_init(full0 + 8u * s, T::CONVERTER_THREADS);
-                mbar_init(empty0 + 8u * s, 1);
+            for (int s = 0; s < T::RAW_STAGES; ++s) {
+                mbar_init(raw_full0 + 8u * s, T::PRODUCER_THREADS);
+                mbar_init(raw_empty0 + 8u * s, 1);
+            }
+            for (int s = 0; s < T::TAIL_STAGES; ++s) {
+                mbar_init(tail_full0 + 8u * s, T::CONVERTER_THREADS);
+                mbar_init(tail_empty0 + 8u * s, 1);
             }
             mbar_init(accum_bar, 1);
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
-        if (warp == T::CONVERTER_WARPS) {        // the MMA warp owns the tensor-memory allocation
+        if (warp == T::MMA_WARP) {               // the MMA warp owns the tensor-memory allocation
             tmem_alloc(static_cast<unsigned>(__cvta_generic_to_shared(tmem_slot)), T::TMEM_COLS);
             tmem_relinquish();
         }
@@ -359,17 +302,50 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     __syncthreads();
     tc_fence_after();
     const unsigned tmem_acc = *tmem_slot;
-    const bool staged = tc.k_end - tc.k_begin <= kKoffCap;
 
     if (warp < T::CONVERTER_WARPS) {
         // ------------------------------------------------------------- converters
-        const UmmaOperand opA = {static_cast<const float *>(p.A), rowA, staged ? koffA - tc.k_begin : p.offA_k,
-                                 tc.rows_valid, tc.k_begin, tc.k_end, p.dirA};
-        const UmmaOperand opB = {static_cast<const float *>(p.B), colB, staged ? koffB - tc.k_begin : p.offB_k,
-                                 tc.cols_valid, tc.k_begin, tc.k_end, p.dirB};
-        const bool ok = (p.vecA == 4 && p.vecB == 4)
-                            ? umma_converter_loop<T, true>(p, tc, opA, opB, smem0, full0, empty0, abort_flag, tid)
-                            : umma_converter_loop<T, false>(p, tc, opA, opB, smem0, full0, empty0, abort_flag, tid);
+        bool ok = true;
+        long long t_raw = 0, t_tail = 0, t_convert = 0, t_signal = 0;
+        (void)t_raw; (void)t_tail; (void)t_convert; (void)t_signal;
+        BTC_PHASE_BEGIN();
+#pragma unroll 1
+        for (int kt = 0; kt < tc.num_kt; ++kt) {
+            const int s = kt % T::RAW_STAGES, t = kt % T::TAIL_STAGES;
+            if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(kt / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait)) {
+                ok = false;
+                break;
+            }
+            BTC_PHASE_END(t_raw);
+            if (kt >= T::TAIL_STAGES &&
+                !mbar_wait_bounded(tail_empty0 + 8u * t, unsigned(kt / T::TAIL_STAGES - 1) & 1u, abort_flag, p.error_word, kErrTailEmptyWait)) {
+                ok = false;
+                break;
+            }
+            BTC_PHASE_END(t_tail);
+            const unsigned src = raw0 + unsigned(s) * T::STAGE_BYTES + unsigned(tid) * 16u;
+            const unsigned dst = tail0 + unsigned(t) * T::STAGE_BYTES + unsigned(tid) * 16u;
+            float x[T::PIECES][4];
+#pragma unroll
+            for (int i = 0; i < T::PIECES; ++i)
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(x[i][0]), "=f"(x[i][1]), "=f"(x[i][2]), "=f"(x[i][3]) : "r"(src + unsigned(i) * 4096u) : "memory");
+#pragma unroll
+            for (int i = 0; i < T::PIECES; ++i) {
+                float lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) lo[e] = x[i][e] - __uint_as_float(__float_as_uint(x[i][e]) & 0xffffe000u);
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + unsigned(i) * 4096u), "f"(lo[0]), "f"(lo[1]), "f"(lo[2]), "f"(lo[3]) : "memory");
+            }
+            BTC_PHASE_END(t_convert);
+            proxy_fence_async();                 // the tensor core reads both stages through the async proxy
+            mbar_arrive(tail_full0 + 8u * t);
+            BTC_PHASE_END(t_signal);
+        }
+        BTC_PHASE_STORE(p, tid == 0, 0, t_raw);
+        BTC_PHASE_STORE(p, tid == 0, 1, t_tail);
+        BTC_PHASE_STORE(p, tid == 0, 2, t_convert);
+        BTC_PHASE_STORE(p, tid == 0, 3, t_signal);
 
         // ------------------------------------------------------------- epilogue
         if (ok && mbar_wait_bounded(accum_bar, 0u, abort_flag, p.error_word, kErrAccumWait)) {
@@ -400,6 +376,30 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             }
             tc_fence_before();
         }
+    } else if (warp < T::MMA_WARP) {
+        // ------------------------------------------------------------- producers
+        const int pt = tid - T::CONVERTER_THREADS;
+        const UmmaOperand opA = {static_cast<const float *>(p.A), rowA, staged ? koffA - tc.k_begin : p.offA_k,
+                                 tc.rows_valid, tc.k_begin, tc.k_end, p.dirA, p.vecA};
+        const UmmaOperand opB = {static_cast<const float *>(p.B), colB, staged ? koffB - tc.k_begin : p.offB_k,
+                                 tc.cols_valid, tc.k_begin, tc.k_end, p.dirB, p.vecB};
+        UmmaProducerLane<T::BM> la;
+        UmmaProducerLane<T::BN> lb;
+        umma_producer_init<T::BM>(la, opA, pt);
+        umma_producer_init<T::BN>(lb, opB, pt);
+#pragma unroll 1
+        for (int kt = 0; kt < tc.num_kt; ++kt) {
+            const int s = kt % T::RAW_STAGES;
+            if (kt >= T::RAW_STAGES &&
+                !mbar_wait_bounded(raw_empty0 + 8u * s, unsigned(kt / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait))
+                break;
+            const unsigned st = raw0 + unsigned(s) * T::STAGE_BYTES;
+            const int64_t k0 = tc.k_begin + int64_t(kt) * T::BK;
+            umma_produce<T::BM>(st, la, opA, k0);
+            umma_produce<T::BN>(st + T::A_BYTES, lb, opB, k0);
+            mbar_arrive_on_copies(raw_full0 + 8u * s);
+        }
+        cp_async_wait_all();
     } else {
         // ------------------------------------------------------------- MMA warp
         constexpr unsigned IDESC_KK = umma_instr_desc(T::BN, false, false);
@@ -413,22 +413,19 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         const unsigned b_lay = b_mn ? 1u : 2u, b_lbo = b_mn ? 512u : 16u, b_sbo = b_mn ? 16u * T::BN : 1024u;
         const unsigned a_step = a_mn ? 32u * T::BM : 32u, b_step = b_mn ? 32u * T::BN : 32u;   // two k-atoms, or 8 k of a row
         const bool leader = elect_one();
-        bool ok = true;
         long long t_full = 0, t_issue = 0;
         (void)t_full; (void)t_issue;
         BTC_PHASE_BEGIN();
 #pragma unroll 1
-        for (int kt = 0; ok && kt < tc.num_kt; ++kt) {
-            const int s = kt % T::STAGES, round = kt / T::STAGES;
-            if (!mbar_wait_bounded(full0 + 8u * s, unsigned(round) & 1u, abort_flag, p.error_word, kErrFullWait)) {
-                ok = false;
+        for (int kt = 0; kt < tc.num_kt; ++kt) {
+            const int s = kt % T::RAW_STAGES, t = kt % T::TAIL_STAGES;
+            if (!mbar_wait_bounded(tail_full0 + 8u * t, unsigned(kt / T::TAIL_STAGES) & 1u, abort_flag, p.error_word, kErrTailFullWait))
                 break;
-            }
             BTC_PHASE_END(t_full);
             tc_fence_after();
             if (leader) {
-                const unsigned st = smem0 + unsigned(s) * T::STAGE_BYTES;
-                const unsigned a_hi = st, a_lo = st + T::A_BYTES, b_hi = st + 2 * T::A_BYTES, b_lo = b_hi + T::B_BYTES;
+                const unsigned a_hi = raw0 + unsigned(s) * T::STAGE_BYTES, b_hi = a_hi + T::A_BYTES;
+                const unsigned a_lo = tail0 + unsigned(t) * T::STAGE_BYTES, b_lo = a_lo + T::A_BYTES;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const uint64_t dah = umma_smem_desc(a_hi + j * a_step, a_lbo, a_sbo, a_lay);
@@ -439,7 +436,8 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     umma_tf32(tmem_acc, dah, dbl, idesc, 1u);
                     umma_tf32(tmem_acc, dah, dbh, idesc, 1u);
                 }
-                umma_commit(empty0 + 8u * s);        // fires when these MMAs have read the stage
+                umma_commit(raw_empty0 + 8u * s);    // fire when these MMAs have read the stages
+                umma_commit(tail_empty0 + 8u * t);
                 if (kt + 1 == tc.num_kt) umma_commit(accum_bar);
             }
             __syncwarp();
@@ -452,7 +450,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
 
     // ---- common tail: every role arrives here, also after an abort ----
     __syncthreads();
-    if (warp == T::CONVERTER_WARPS) {
+    if (warp == T::MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem_acc, T::TMEM_COLS);
     }
