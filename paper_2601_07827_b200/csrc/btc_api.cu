@@ -314,6 +314,7 @@ int finish_plan(btc_contraction_s *op)
     op->k_per_split = kt_per * v.bk;
     if (tiles * split > 0x7fffffffLL) return BTC_ERR_NOT_SUPPORTED;
     op->grid[0] = int32_t(tiles * split); op->grid[1] = 1; op->grid[2] = 1;
+    if (umma && op->grid[0] > sms) op->grid[0] = int32_t(sms);   // persistent CTAs walk the tile list
     if (split > 1)
         op->workspace_bytes = size_t(tiles) * size_t(split) * size_t(v.threads) * size_t(v.acc) * v.acc_bytes;
 

@@ -154,15 +154,15 @@ struct TileCoords {
     int rows_valid, cols_valid, num_kt;
 };
 
+// `work` enumerates (tile, k slice, batch), tile fastest
 template <int BM, int BN, int BK, typename Params>
-__device__ __forceinline__ TileCoords tile_coords(const Params &p)
+__device__ __forceinline__ TileCoords tile_coords_at(const Params &p, int64_t work)
 {
     TileCoords c;
-    // blockIdx.x enumerates (tile, k slice, batch), tile fastest
     const int tiles = p.tiles_m * p.tiles_n;
-    c.tile = blockIdx.x % tiles;
-    c.ks = (blockIdx.x / tiles) % p.split_k;
-    c.h = blockIdx.x / (tiles * p.split_k);
+    c.tile = int(work % tiles);
+    c.ks = int((work / tiles) % p.split_k);
+    c.h = work / (int64_t(tiles) * p.split_k);
     const int tile_m = p.raster_n_fast ? c.tile / p.tiles_n : c.tile % p.tiles_m;
     const int tile_n = p.raster_n_fast ? c.tile % p.tiles_n : c.tile / p.tiles_m;
     c.m0 = int64_t(tile_m) * BM;
@@ -173,6 +173,13 @@ __device__ __forceinline__ TileCoords tile_coords(const Params &p)
     c.k_end = imin64(p.K, c.k_begin + p.k_per_split);
     c.num_kt = int((c.k_end - c.k_begin + BK - 1) / BK);
     return c;
+}
+
+// one CTA per work item
+template <int BM, int BN, int BK, typename Params>
+__device__ __forceinline__ TileCoords tile_coords(const Params &p)
+{
+    return tile_coords_at<BM, BN, BK>(p, int64_t(blockIdx.x));
 }
 
 // Per-tile row/column offset arrays (batch offset folded in) and the stage barriers; ends with a

@@ -1,8 +1,9 @@
 // fp32 contraction on the 5th-generation tensor cores (tcgen05.mma kind::tf32, accumulators in
 // tensor memory), 3xTF32:  a*b = a_lo*b_hi + a_hi*b_lo + a_hi*b_hi  with x = x_hi + x_lo.
 //
-// CTA = 8 converter warps + 4 producer warps + 1 MMA warp, one CTA per SM, tile 128 x BN x 32
-// per stage.  Shared memory holds a deep ring of "raw" stages and a short ring of "tail" stages.
+// Persistent CTAs (one per SM) of 4 epilogue + 4 converter + 4 producer warps + 1 MMA warp walk the
+// list of 128 x BN tiles, 32 k per stage.  Shared memory holds a deep ring of "raw" stages and a
+// short ring of "tail" stages, tensor memory two accumulators.
 //   producers   gather the strided A / B tiles through the offset tables with asynchronous
 //               16-byte copies (zero-filled outside the tensor) straight into the swizzled
 //               operand layouts the tensor core reads.  Asynchronous copies keep far more bytes
@@ -14,13 +15,14 @@
 //               raw fp32 stage already is the head operand x_hi.  The converters read it, form
 //               the tail x - x_hi (exact in fp32) and store it at the same position of a tail
 //               stage: a position-independent, conflict-free pass over the stage.
-//   MMA warp    one elected lane waits for a tail stage ("tail full", 256 arrivals; it implies
-//               the raw stage), issues the 4 k-steps x 3 MMAs and commits them to the "raw empty"
-//               and "tail empty" mbarriers; after the last stage it commits to the accumulator
-//               barrier.
-//   epilogue    the converter warps read the accumulator from tensor memory (each warp its own
-//               32-lane quarter, one row of the tile per lane, so a warp's store of one column
-//               is 32 consecutive rows of D) and apply alpha / beta through D's offset tables.
+//   MMA warp    one elected lane waits for a tail stage ("tail full"; it implies the raw stage),
+//               issues the 4 k-steps x 3 MMAs and commits them to the "raw empty" and "tail
+//               empty" mbarriers; after a tile's last stage it commits to that accumulator's
+//               "full" barrier and moves on to the other accumulator.
+//   epilogue    warp w reads lanes 32 w .. 32 w + 31 of the finished accumulator (one row of the
+//               tile per lane, so a warp's store of one column is 32 consecutive rows of D),
+//               applies alpha / beta through D's offset tables and releases the accumulator,
+//               while the other roles already work on the next tile.
 // Every wait is bounded; a wait that gives up raises the CTA abort flag and the error word, all
 // roles fall through to the common tail, and the allocating warp always frees its tensor memory.
 #pragma once
@@ -36,20 +38,22 @@ template <int BN_, int RAW_STAGES_, int TAIL_STAGES_>
 struct UmmaTile {
     static constexpr int BM = 128, BN = BN_, BK = 32;
     static constexpr int RAW_STAGES = RAW_STAGES_, TAIL_STAGES = TAIL_STAGES_;
-    static constexpr int CONVERTER_WARPS = 8, CONVERTER_THREADS = 256;
+    static constexpr int EPILOGUE_WARPS = 4, EPILOGUE_THREADS = 128;  // warps 0-3: one tensor-memory lane quarter each
+    static constexpr int CONVERTER_WARPS = 4, CONVERTER_THREADS = 128;
     static constexpr int PRODUCER_WARPS = 4, PRODUCER_THREADS = 128;
-    static constexpr int MMA_WARP = CONVERTER_WARPS + PRODUCER_WARPS;
-    static constexpr int THREADS = CONVERTER_THREADS + PRODUCER_THREADS + 32;
+    static constexpr int MMA_WARP = EPILOGUE_WARPS + CONVERTER_WARPS + PRODUCER_WARPS;
+    static constexpr int THREADS = 32 * (MMA_WARP + 1);
     static constexpr int A_BYTES = BM * BK * 4, B_BYTES = BN * BK * 4;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;           // same size for raw and tail stages
-    static constexpr int TMEM_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
+    static constexpr int ACC_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;   // one accumulator
+    static constexpr int TMEM_COLS = 2 * ACC_COLS;                  // two: epilogue and main loop overlap
     static constexpr int PIECES = STAGE_BYTES / 16 / CONVERTER_THREADS;   // 16-byte pieces per converter thread
-    static constexpr int NUM_BARS = 2 * RAW_STAGES + 2 * TAIL_STAGES + 1;
+    static constexpr int NUM_BARS = 2 * RAW_STAGES + 2 * TAIL_STAGES + 8;
     static_assert(STAGE_BYTES % (16 * CONVERTER_THREADS) == 0, "a stage must divide among the converters");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "BN must suit UMMA N and the epilogue split");
     // stages | row/col offsets | k offsets | mbarriers | tmem ptr, abort
     static constexpr size_t SMEM_BYTES = size_t(RAW_STAGES + TAIL_STAGES) * STAGE_BYTES +
-                                         size_t(2 * BM + 2 * BN + 2 * kKoffCap) * 8 + size_t(NUM_BARS) * 8 + 16 +
+                                         size_t(2 * BM + 4 * BN + 2 * kKoffCap) * 8 + size_t(NUM_BARS) * 8 + 16 +
                                          1024;   // + slack to align the tiles
 };
 
@@ -221,7 +225,7 @@ __device__ __forceinline__ void umma_produce(unsigned tile, const UmmaProducerLa
     }
 }
 
-constexpr int kErrAccumWait = 3, kErrTailFullWait = 4, kErrTailEmptyWait = 5;
+constexpr int kErrAccumWait = 3, kErrTailFullWait = 4, kErrTailEmptyWait = 5, kErrGroupSync = 6;
 
 // Debug builds (-DBTC_STAMPS) add up the SM clock cycles one thread spends in each phase.
 #ifdef BTC_STAMPS
@@ -234,6 +238,17 @@ constexpr int kErrAccumWait = 3, kErrTailFullWait = 4, kErrTailEmptyWait = 5;
 #define BTC_PHASE_STORE(p, who, slot, acc) do { } while (0)
 #endif
 
+// Group-wide rendezvous on an mbarrier (every member arrives, then waits with a bound): unlike a
+// named barrier it cannot hang when a member has left after an abort.
+__device__ __forceinline__ bool umma_group_sync(unsigned bar, unsigned parity, volatile int *abort_flag, int *error_word)
+{
+    mbar_arrive(bar);
+    return mbar_wait_bounded(bar, parity, abort_flag, error_word, kErrGroupSync);
+}
+
+// Persistent: CTA b works on the items b, b + gridDim.x, ... of the (tile, batch) list; all roles
+// walk that list with the same counters.  Tensor memory holds two accumulators, so the epilogue
+// of one tile overlaps the main loop of the next; the shared-memory rings run across tiles.
 template <typename T>
 __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const TiledParams p)
 {
@@ -241,11 +256,10 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     // operand tiles must sit on 1024-byte boundaries of the shared-memory window (swizzled layouts)
     unsigned char *smem_raw = smem_unaligned +
         ((1024u - (static_cast<unsigned>(__cvta_generic_to_shared(smem_unaligned)) & 1023u)) & 1023u);
-    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + size_t(T::RAW_STAGES + T::TAIL_STAGES) * T::STAGE_BYTES);
-    int64_t *rowD = rowA + T::BM;
-    int64_t *colB = rowD + T::BM;
-    int64_t *colD = colB + T::BN;
-    int64_t *koffA = colD + T::BN;
+    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + size_t(T::RAW_STAGES + T::TAIL_STAGES) * T::STAGE_BYTES);   // [2][BM]
+    int64_t *colB = rowA + 2 * T::BM;                                    // [2][BN]
+    int64_t *colD = colB + 2 * T::BN;                                    // [2][BN]
+    int64_t *koffA = colD + 2 * T::BN;
     int64_t *koffB = koffA + kKoffCap;
     uint64_t *bars = reinterpret_cast<uint64_t *>(koffB + kKoffCap);
     unsigned *tmem_slot = reinterpret_cast<unsigned *>(bars + T::NUM_BARS);
@@ -256,29 +270,22 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     const unsigned raw_empty0 = raw_full0 + 8u * T::RAW_STAGES;
     const unsigned tail_full0 = raw_empty0 + 8u * T::RAW_STAGES;
     const unsigned tail_empty0 = tail_full0 + 8u * T::TAIL_STAGES;
-    const unsigned accum_bar = tail_empty0 + 8u * T::TAIL_STAGES;
+    const unsigned accum_full0 = tail_empty0 + 8u * T::TAIL_STAGES;      // [2]
+    const unsigned accum_empty0 = accum_full0 + 16u;                     // [2]
+    const unsigned producer_sync0 = accum_empty0 + 16u;                  // [2]
+    const unsigned epilogue_sync0 = producer_sync0 + 16u;                // [2]
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
-    const bool staged = tc.k_end - tc.k_begin <= kKoffCap;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int64_t total = int64_t(p.tiles_m) * p.tiles_n * p.Bt;         // split_k == 1 on this path
+    const int num_kt = int((p.K + T::BK - 1) / T::BK);
+    const bool staged = p.K <= kKoffCap;
 
-    // ---- set-up: offset arrays, barriers, tensor memory ----
+    // ---- set-up: k offsets, barriers, tensor memory ----
     {
-        const int64_t hA = p.offA_h[tc.h], hB = p.offB_h[tc.h], hD = p.offD_h[tc.h];
-        for (int i = tid; i < T::BM; i += T::THREADS) {
-            const bool v = i < tc.rows_valid;
-            rowA[i] = v ? p.offA_m[tc.m0 + i] + hA : 0;
-            rowD[i] = v ? p.offD_m[tc.m0 + i] + hD : 0;
-        }
-        for (int i = tid; i < T::BN; i += T::THREADS) {
-            const bool v = i < tc.cols_valid;
-            colB[i] = v ? p.offB_n[tc.n0 + i] + hB : 0;
-            colD[i] = v ? p.offD_n[tc.n0 + i] : 0;
-        }
         if (staged)
-            for (int i = tid; i < int(tc.k_end - tc.k_begin); i += T::THREADS) {
-                koffA[i] = p.offA_k[tc.k_begin + i];
-                koffB[i] = p.offB_k[tc.k_begin + i];
+            for (int i = tid; i < int(p.K); i += T::THREADS) {
+                koffA[i] = p.offA_k[i];
+                koffB[i] = p.offB_k[i];
             }
         if (tid == 0) {
             for (int s = 0; s < T::RAW_STAGES; ++s) {
@@ -289,7 +296,12 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 mbar_init(tail_full0 + 8u * s, T::CONVERTER_THREADS);
                 mbar_init(tail_empty0 + 8u * s, 1);
             }
-            mbar_init(accum_bar, 1);
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(accum_full0 + 8u * b, 1);
+                mbar_init(accum_empty0 + 8u * b, T::EPILOGUE_THREADS);
+                mbar_init(producer_sync0 + 8u * b, T::PRODUCER_THREADS);
+                mbar_init(epilogue_sync0 + 8u * b, T::EPILOGUE_THREADS);
+            }
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
@@ -301,103 +313,124 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const unsigned tmem_acc = *tmem_slot;
+    const unsigned tmem_base = *tmem_slot;
 
-    if (warp < T::CONVERTER_WARPS) {
-        // ------------------------------------------------------------- converters
-        bool ok = true;
-        long long t_raw = 0, t_tail = 0, t_convert = 0, t_signal = 0;
-        (void)t_raw; (void)t_tail; (void)t_convert; (void)t_signal;
-        BTC_PHASE_BEGIN();
-#pragma unroll 1
-        for (int kt = 0; kt < tc.num_kt; ++kt) {
-            const int s = kt % T::RAW_STAGES, t = kt % T::TAIL_STAGES;
-            if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(kt / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait)) {
-                ok = false;
-                break;
-            }
-            BTC_PHASE_END(t_raw);
-            if (kt >= T::TAIL_STAGES &&
-                !mbar_wait_bounded(tail_empty0 + 8u * t, unsigned(kt / T::TAIL_STAGES - 1) & 1u, abort_flag, p.error_word, kErrTailEmptyWait)) {
-                ok = false;
-                break;
-            }
-            BTC_PHASE_END(t_tail);
-            const unsigned src = raw0 + unsigned(s) * T::STAGE_BYTES + unsigned(tid) * 16u;
-            const unsigned dst = tail0 + unsigned(t) * T::STAGE_BYTES + unsigned(tid) * 16u;
-            float x[T::PIECES][4];
-#pragma unroll
-            for (int i = 0; i < T::PIECES; ++i)
-                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                             : "=f"(x[i][0]), "=f"(x[i][1]), "=f"(x[i][2]), "=f"(x[i][3]) : "r"(src + unsigned(i) * 4096u) : "memory");
-#pragma unroll
-            for (int i = 0; i < T::PIECES; ++i) {
-                float lo[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) lo[e] = x[i][e] - __uint_as_float(__float_as_uint(x[i][e]) & 0xffffe000u);
-                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + unsigned(i) * 4096u), "f"(lo[0]), "f"(lo[1]), "f"(lo[2]), "f"(lo[3]) : "memory");
-            }
-            BTC_PHASE_END(t_convert);
-            proxy_fence_async();                 // the tensor core reads both stages through the async proxy
-            mbar_arrive(tail_full0 + 8u * t);
-            BTC_PHASE_END(t_signal);
-        }
-        BTC_PHASE_STORE(p, tid == 0, 0, t_raw);
-        BTC_PHASE_STORE(p, tid == 0, 1, t_tail);
-        BTC_PHASE_STORE(p, tid == 0, 2, t_convert);
-        BTC_PHASE_STORE(p, tid == 0, 3, t_signal);
-
+    if (warp < T::EPILOGUE_WARPS) {
         // ------------------------------------------------------------- epilogue
-        if (ok && mbar_wait_bounded(accum_bar, 0u, abort_flag, p.error_word, kErrAccumWait)) {
-            tc_fence_after();
-            float *D = static_cast<float *>(p.D);
-            const float *C = static_cast<const float *>(p.C);
-            const float alpha = float(p.alpha[0]), beta = float(p.beta[0]);
-            const int quarter = warp & 3, half = warp >> 2;          // lanes 32 q .. 32 q + 31, column half
-            const int row = quarter * 32 + lane;
-            const bool row_ok = row < tc.rows_valid;
-            const int64_t ro = rowD[row];
+        // warp w reads tensor-memory lanes 32 w .. 32 w + 31: thread tid owns row tid of the tile
+        float *D = static_cast<float *>(p.D);
+        const float *C = static_cast<const float *>(p.C);
+        const float alpha = float(p.alpha[0]), beta = float(p.beta[0]);
+        int n = 0;
 #pragma unroll 1
-            for (int c0 = half * (T::BN / 2); c0 < (half + 1) * (T::BN / 2); c0 += 16) {
+        for (int64_t work = blockIdx.x; work < total; work += gridDim.x, ++n) {
+            const TileCoords tc = tile_coords_at<T::BM, T::BN, T::BK>(p, work);
+            const int buf = n & 1;
+            const unsigned parity = unsigned(n >> 1) & 1u;
+            int64_t *cD = colD + buf * T::BN;
+            for (int i = tid; i < T::BN; i += T::EPILOGUE_THREADS) cD[i] = i < tc.cols_valid ? p.offD_n[tc.n0 + i] : 0;
+            const bool row_ok = tid < tc.rows_valid;
+            const int64_t ro = row_ok ? p.offD_m[tc.m0 + tid] + p.offD_h[tc.h] : 0;
+            if (!umma_group_sync(epilogue_sync0 + 8u * buf, parity, abort_flag, p.error_word)) break;
+            if (!mbar_wait_bounded(accum_full0 + 8u * buf, parity, abort_flag, p.error_word, kErrAccumWait)) break;
+            tc_fence_after();
+            const unsigned tacc = tmem_base + (unsigned(warp * 32) << 16) + unsigned(buf * T::ACC_COLS);
+#pragma unroll 1
+            for (int c0 = 0; c0 < T::BN; c0 += 16) {
                 unsigned r[16];
-                tmem_load16(tmem_acc + (unsigned(quarter * 32) << 16) + unsigned(c0), r);
+                tmem_load16(tacc + unsigned(c0), r);
                 tmem_load_wait();
                 float cv[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    cv[j] = (p.use_c && row_ok && c0 + j < tc.cols_valid) ? C[ro + colD[c0 + j]] : 0.f;
+                    cv[j] = (p.use_c && row_ok && c0 + j < tc.cols_valid) ? C[ro + cD[c0 + j]] : 0.f;
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
                     if (row_ok && c0 + j < tc.cols_valid) {
                         float v = alpha * __uint_as_float(r[j]);
                         if (p.use_c) v += beta * cv[j];
-                        D[ro + colD[c0 + j]] = v;
+                        D[ro + cD[c0 + j]] = v;
                     }
             }
             tc_fence_before();
+            mbar_arrive(accum_empty0 + 8u * buf);    // this accumulator may be overwritten
+        }
+    } else if (warp < T::EPILOGUE_WARPS + T::CONVERTER_WARPS) {
+        // ------------------------------------------------------------- converters
+        const int ct = tid - T::EPILOGUE_THREADS;
+        bool ok = true;
+        int g = 0;                                   // stage counter across tiles
+#pragma unroll 1
+        for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x) {
+#pragma unroll 1
+            for (int kt = 0; kt < num_kt; ++kt, ++g) {
+                const int s = g % T::RAW_STAGES, t = g % T::TAIL_STAGES;
+                if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(g / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait) ||
+                    (g >= T::TAIL_STAGES &&
+                     !mbar_wait_bounded(tail_empty0 + 8u * t, unsigned(g / T::TAIL_STAGES - 1) & 1u, abort_flag, p.error_word, kErrTailEmptyWait))) {
+                    ok = false;
+                    break;
+                }
+                const unsigned src = raw0 + unsigned(s) * T::STAGE_BYTES + unsigned(ct) * 16u;
+                const unsigned dst = tail0 + unsigned(t) * T::STAGE_BYTES + unsigned(ct) * 16u;
+                constexpr unsigned STEP = 16u * T::CONVERTER_THREADS;
+                constexpr int CHUNK = T::PIECES % 8 == 0 ? 8 : T::PIECES % 7 == 0 ? 7 : 4;   // loads in flight per thread
+                static_assert(T::PIECES % CHUNK == 0, "pieces must divide into chunks");
+#pragma unroll
+                for (int i0 = 0; i0 < T::PIECES; i0 += CHUNK) {
+                    float x[CHUNK][4];
+#pragma unroll
+                    for (int i = 0; i < CHUNK; ++i)
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(x[i][0]), "=f"(x[i][1]), "=f"(x[i][2]), "=f"(x[i][3]) : "r"(src + unsigned(i0 + i) * STEP) : "memory");
+#pragma unroll
+                    for (int i = 0; i < CHUNK; ++i) {
+                        float lo[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) lo[e] = x[i][e] - __uint_as_float(__float_as_uint(x[i][e]) & 0xffffe000u);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + unsigned(i0 + i) * STEP), "f"(lo[0]), "f"(lo[1]), "f"(lo[2]), "f"(lo[3]) : "memory");
+                    }
+                }
+                proxy_fence_async();             // the tensor core reads both stages through the async proxy
+                mbar_arrive(tail_full0 + 8u * t);
+            }
         }
     } else if (warp < T::MMA_WARP) {
         // ------------------------------------------------------------- producers
-        const int pt = tid - T::CONVERTER_THREADS;
-        const UmmaOperand opA = {static_cast<const float *>(p.A), rowA, staged ? koffA - tc.k_begin : p.offA_k,
-                                 tc.rows_valid, tc.k_begin, tc.k_end, p.dirA, p.vecA};
-        const UmmaOperand opB = {static_cast<const float *>(p.B), colB, staged ? koffB - tc.k_begin : p.offB_k,
-                                 tc.cols_valid, tc.k_begin, tc.k_end, p.dirB, p.vecB};
-        UmmaProducerLane<T::BM> la;
-        UmmaProducerLane<T::BN> lb;
-        umma_producer_init<T::BM>(la, opA, pt);
-        umma_producer_init<T::BN>(lb, opB, pt);
+        const int pt = tid - T::EPILOGUE_THREADS - T::CONVERTER_THREADS;
+        bool ok = true;
+        int g = 0, n = 0;
 #pragma unroll 1
-        for (int kt = 0; kt < tc.num_kt; ++kt) {
-            const int s = kt % T::RAW_STAGES;
-            if (kt >= T::RAW_STAGES &&
-                !mbar_wait_bounded(raw_empty0 + 8u * s, unsigned(kt / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait))
-                break;
-            const unsigned st = raw0 + unsigned(s) * T::STAGE_BYTES;
-            const int64_t k0 = tc.k_begin + int64_t(kt) * T::BK;
-            umma_produce<T::BM>(st, la, opA, k0);
-            umma_produce<T::BN>(st + T::A_BYTES, lb, opB, k0);
-            mbar_arrive_on_copies(raw_full0 + 8u * s);
+        for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x, ++n) {
+            const TileCoords tc = tile_coords_at<T::BM, T::BN, T::BK>(p, work);
+            const int buf = n & 1;
+            int64_t *rA = rowA + buf * T::BM, *cB = colB + buf * T::BN;
+            {
+                const int64_t hA = p.offA_h[tc.h], hB = p.offB_h[tc.h];
+                for (int i = pt; i < T::BM; i += T::PRODUCER_THREADS) rA[i] = i < tc.rows_valid ? p.offA_m[tc.m0 + i] + hA : 0;
+                for (int i = pt; i < T::BN; i += T::PRODUCER_THREADS) cB[i] = i < tc.cols_valid ? p.offB_n[tc.n0 + i] + hB : 0;
+            }
+            if (!umma_group_sync(producer_sync0 + 8u * buf, unsigned(n >> 1) & 1u, abort_flag, p.error_word)) break;
+            const UmmaOperand opA = {static_cast<const float *>(p.A), rA, staged ? koffA : p.offA_k, tc.rows_valid, 0, p.K, p.dirA, p.vecA};
+            const UmmaOperand opB = {static_cast<const float *>(p.B), cB, staged ? koffB : p.offB_k, tc.cols_valid, 0, p.K, p.dirB, p.vecB};
+            UmmaProducerLane<T::BM> la;
+            UmmaProducerLane<T::BN> lb;
+            umma_producer_init<T::BM>(la, opA, pt);
+            umma_producer_init<T::BN>(lb, opB, pt);
+#pragma unroll 1
+            for (int kt = 0; kt < num_kt; ++kt, ++g) {
+                const int s = g % T::RAW_STAGES;
+                if (g >= T::RAW_STAGES &&
+                    !mbar_wait_bounded(raw_empty0 + 8u * s, unsigned(g / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait)) {
+                    ok = false;
+                    break;
+                }
+                const unsigned st = raw0 + unsigned(s) * T::STAGE_BYTES;
+                const int64_t k0 = int64_t(kt) * T::BK;
+                umma_produce<T::BM>(st, la, opA, k0);
+                umma_produce<T::BN>(st + T::A_BYTES, lb, opB, k0);
+                mbar_arrive_on_copies(raw_full0 + 8u * s);
+            }
         }
         cp_async_wait_all();
     } else {
@@ -413,38 +446,44 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         const unsigned b_lay = b_mn ? 1u : 2u, b_lbo = b_mn ? 512u : 16u, b_sbo = b_mn ? 16u * T::BN : 1024u;
         const unsigned a_step = a_mn ? 32u * T::BM : 32u, b_step = b_mn ? 32u * T::BN : 32u;   // two k-atoms, or 8 k of a row
         const bool leader = elect_one();
-        long long t_full = 0, t_issue = 0;
-        (void)t_full; (void)t_issue;
-        BTC_PHASE_BEGIN();
+        bool ok = true;
+        int g = 0, n = 0;
 #pragma unroll 1
-        for (int kt = 0; kt < tc.num_kt; ++kt) {
-            const int s = kt % T::RAW_STAGES, t = kt % T::TAIL_STAGES;
-            if (!mbar_wait_bounded(tail_full0 + 8u * t, unsigned(kt / T::TAIL_STAGES) & 1u, abort_flag, p.error_word, kErrTailFullWait))
+        for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x, ++n) {
+            const int buf = n & 1;
+            if (n >= 2 &&
+                !mbar_wait_bounded(accum_empty0 + 8u * buf, unsigned((n >> 1) - 1) & 1u, abort_flag, p.error_word, kErrAccumWait))
                 break;
-            BTC_PHASE_END(t_full);
             tc_fence_after();
-            if (leader) {
-                const unsigned a_hi = raw0 + unsigned(s) * T::STAGE_BYTES, b_hi = a_hi + T::A_BYTES;
-                const unsigned a_lo = tail0 + unsigned(t) * T::STAGE_BYTES, b_lo = a_lo + T::A_BYTES;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint64_t dah = umma_smem_desc(a_hi + j * a_step, a_lbo, a_sbo, a_lay);
-                    const uint64_t dal = umma_smem_desc(a_lo + j * a_step, a_lbo, a_sbo, a_lay);
-                    const uint64_t dbh = umma_smem_desc(b_hi + j * b_step, b_lbo, b_sbo, b_lay);
-                    const uint64_t dbl = umma_smem_desc(b_lo + j * b_step, b_lbo, b_sbo, b_lay);
-                    umma_tf32(tmem_acc, dal, dbh, idesc, (kt > 0 || j > 0) ? 1u : 0u);
-                    umma_tf32(tmem_acc, dah, dbl, idesc, 1u);
-                    umma_tf32(tmem_acc, dah, dbh, idesc, 1u);
+            const unsigned tacc = tmem_base + unsigned(buf * T::ACC_COLS);
+#pragma unroll 1
+            for (int kt = 0; kt < num_kt; ++kt, ++g) {
+                const int s = g % T::RAW_STAGES, t = g % T::TAIL_STAGES;
+                if (!mbar_wait_bounded(tail_full0 + 8u * t, unsigned(g / T::TAIL_STAGES) & 1u, abort_flag, p.error_word, kErrTailFullWait)) {
+                    ok = false;
+                    break;
                 }
-                umma_commit(raw_empty0 + 8u * s);    // fire when these MMAs have read the stages
-                umma_commit(tail_empty0 + 8u * t);
-                if (kt + 1 == tc.num_kt) umma_commit(accum_bar);
+                tc_fence_after();
+                if (leader) {
+                    const unsigned a_hi = raw0 + unsigned(s) * T::STAGE_BYTES, b_hi = a_hi + T::A_BYTES;
+                    const unsigned a_lo = tail0 + unsigned(t) * T::STAGE_BYTES, b_lo = a_lo + T::A_BYTES;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint64_t dah = umma_smem_desc(a_hi + j * a_step, a_lbo, a_sbo, a_lay);
+                        const uint64_t dal = umma_smem_desc(a_lo + j * a_step, a_lbo, a_sbo, a_lay);
+                        const uint64_t dbh = umma_smem_desc(b_hi + j * b_step, b_lbo, b_sbo, b_lay);
+                        const uint64_t dbl = umma_smem_desc(b_lo + j * b_step, b_lbo, b_sbo, b_lay);
+                        umma_tf32(tacc, dal, dbh, idesc, (kt > 0 || j > 0) ? 1u : 0u);
+                        umma_tf32(tacc, dah, dbl, idesc, 1u);
+                        umma_tf32(tacc, dah, dbh, idesc, 1u);
+                    }
+                    umma_commit(raw_empty0 + 8u * s);    // fire when these MMAs have read the stages
+                    umma_commit(tail_empty0 + 8u * t);
+                    if (kt + 1 == num_kt) umma_commit(accum_full0 + 8u * buf);
+                }
+                __syncwarp();
             }
-            __syncwarp();
-            BTC_PHASE_END(t_issue);
         }
-        BTC_PHASE_STORE(p, lane == 0, 4, t_full);
-        BTC_PHASE_STORE(p, lane == 0, 5, t_issue);
         tc_fence_before();
     }
 
@@ -452,7 +491,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     __syncthreads();
     if (warp == T::MMA_WARP) {
         tc_fence_after();
-        tmem_dealloc(tmem_acc, T::TMEM_COLS);
+        tmem_dealloc(tmem_base, T::TMEM_COLS);
     }
 }
 

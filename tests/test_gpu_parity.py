@@ -232,3 +232,20 @@ def test_every_tile_variant(api, handle, dtype, variant):
     assert worst <= 1.0
     worst, _, _ = helpers.run_case(handle, A, "ik", B2, "jk", None, D, "ij", kernel=api.KERNEL_TILED, variant=variant)
     assert worst <= 1.0
+
+
+@pytest.mark.parametrize("variant", [10, 11, 12])
+def test_persistent_tensor_memory_kernel_walks_many_tiles(api, handle, variant):
+    """The tcgen05 kernels are persistent: with more tiles than SMs every CTA takes several tiles in
+    turn, re-using both accumulators, the stage rings and the double-buffered offset arrays.  Ragged
+    extents, a batch label, beta != 0 and a strided (non-vector) operand are all in play."""
+    ext = dict(i=128 * 17 + 5, j=96 * 6 + 7, k=70, z=3)
+    A = helpers.random_tensor(81, _ext("kiz", ext), None, torch.float32)
+    B = helpers.random_tensor(82, _ext("zkj", ext), None, torch.float32)
+    C = helpers.random_tensor(83, _ext("ijz", ext), None, torch.float32)
+    D = inputs.place(None, _ext("ijz", ext), None, torch.float32)
+    worst, status, _ = helpers.run_case(handle, A, "kiz", B, "zkj", C, D, "ijz", 0.75, 1.5, kernel=api.KERNEL_TILED,
+                                        variant=variant, want_status=True)
+    assert worst <= 1.0 and status["kernel"] == api.KERNEL_TILED
+    bn = {10: 96, 11: 128, 12: 256}[variant]
+    assert status["grid"][0] < -(-ext["i"] // 128) * -(-ext["j"] // bn) * ext["z"]   # fewer CTAs than tiles
