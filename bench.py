@@ -39,7 +39,15 @@ def measured_hbm_gbs():
         return 6650.0, "fallback"
 
 
-def roofline_for(w, kernel_ms):
+def measured_tf32_tflops():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"]) * 1.1 / 2.25, "measured"
+    except (OSError, KeyError, ValueError):
+        return 1590.0 * 1.1 / 2.25, "fallback"
+
+
+def roofline_for(w, kernel_ms, variant=-1):
     """Roofline entry of the dominant kernel for this workload."""
     if w.name.startswith("cfg5"):
         peak, src = measured_hbm_gbs()
@@ -53,14 +61,33 @@ def roofline_for(w, kernel_ms):
                 "peak_source": "FP64 tensor (DMMA) pipe: 148 SMs x 64 FMA/clk x 2 x 1.965 GHz; "
                                "a register-resident DMMA loop measured 37.1 TFLOP/s on this pool",
                 "kernel": "tiled_f64_kernel", "kernel_ms": kernel_ms}
+    if variant >= 10:
+        # tcgen05 3xTF32: three TF32 MMAs per product.  TF32 dense peak = measured bf16 burst peak x
+        # the nominal TF32 : bf16 ratio (1.1 : 2.25).  Whichever of the tensor pipe and HBM needs
+        # longer for this workload is the bound.
+        hbm, src = measured_hbm_gbs()
+        tf32_peak, tsrc = measured_tf32_tflops()
+        t_hbm = w.algorithmic_bytes() / (hbm * 1e9)
+        t_tensor = 3 * w.flops() / (tf32_peak * 1e12)
+        if t_hbm >= t_tensor:
+            gbs = w.algorithmic_bytes() / (kernel_ms * 1e-3) / 1e9
+            return {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm, "traffic": None,
+                    "peak_source": f"STREAM-style copy, {src}; the tensor pipe would need {t_tensor * 1e3:.3f} ms, "
+                                   f"HBM needs {t_hbm * 1e3:.3f} ms",
+                    "useful_tflops": achieved, "kernel": "tiled_umma_tf32x3_kernel", "kernel_ms": kernel_ms}
+        return {"bound": "tensor", "achieved": 3 * achieved, "peak": tf32_peak, "unit": "TFLOP/s",
+                "frac": 3 * achieved / tf32_peak, "traffic": None,
+                "peak_source": f"TF32 dense = bf16 cuBLAS burst peak ({tsrc}) x 1.1/2.25; executed flops = 3 x useful "
+                               "(3xTF32)",
+                "useful_tflops": achieved, "kernel": "tiled_umma_tf32x3_kernel", "kernel_ms": kernel_ms}
     return {"bound": "alu", "achieved": achieved, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s",
             "frac": achieved / FP32_PEAK_TFLOPS, "traffic": None,
             "peak_source": "FP32 FMA pipe: 148 SMs x 128 FMA/clk x 2 x 1.965 GHz; "
                            "a register-resident FFMA loop measured 72.3 TFLOP/s on this pool",
-            "note": "the default fp32 kernel computes each product as three TF32 tensor-core MMAs "
+            "note": "this fp32 kernel computes each product as three TF32 tensor-core MMAs "
                     "(mma.sync m16n8k8, measured peak 277 TFLOP/s on this pool): it executes "
                     f"{3 * achieved:.1f} tensor TFLOP/s = {3 * achieved / 277.0:.2f} of that peak",
-            "kernel": "tiled_tf32x3_kernel", "kernel_ms": kernel_ms}
+            "kernel": "tiled_tf32x3_kernel" if variant >= 6 else "tiled_f32_kernel", "kernel_ms": kernel_ms}
 
 
 def parse():
@@ -357,7 +384,7 @@ def main():
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "GFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline_for(w, kernel_avg_ms),
+            "roofline": roofline_for(w, kernel_avg_ms, op.variant),
         }
         if ms_per_step < 0.2 and world == 1:
             # microseconds of work per call: the per-step figure above includes the host's call
@@ -365,7 +392,7 @@ def main():
             lat = small_problem_latency(lambda s_: step(on=s_), stream, torch)
             out["latency"] = lat
             per_call_ms = lat["graph_replay_us"] * 1e-3
-            out["roofline"] = roofline_for(w, per_call_ms)
+            out["roofline"] = roofline_for(w, per_call_ms, op.variant)
             out["roofline"]["timing"] = "per call inside a replayed CUDA graph of 100 calls"
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"] = cpu_baseline(w)

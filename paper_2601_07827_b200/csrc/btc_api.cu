@@ -257,18 +257,23 @@ int finish_plan(btc_contraction_s *op)
     auto tiles_for = [&](const VariantInfo &v) {
         return ((pl.M + v.bm - 1) / v.bm) * ((pl.N + v.bn - 1) / v.bn) * pl.Bt;
     };
-    // Candidate tile variants of the element type (fp32: the 3xTF32 tensor-core variants; the
-    // strict-fp32 FFMA variants 0-5 are selected with BTC_ATTR_VARIANT only).  Score = fraction of
+    // Candidate tile variants of the element type (fp32: the 3xTF32 tensor-core variants, mma.sync
+    // or tcgen05; the strict-fp32 FFMA variants 0-5 are selected with BTC_ATTR_VARIANT only).  Score = fraction of
     // the padded tiles that is real work x fraction of the last wave that is filled x a mild
     // preference for larger tiles (more flops per byte moved through shared memory).
     int variant = 0;
     {
         struct Cand { int id; double weight; };
-        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}};
+        // The tcgen05 variants 10-12 keep all of K in one CTA and have a longer prologue: they
+        // enter only when there is enough work to fill the SMs without split-K; their weights
+        // reflect measured throughput relative to the mma.sync variants.
+        const double flops = 2.0 * double(pl.M) * double(pl.N) * double(pl.K) * double(pl.Bt);
+        const bool umma_ok = pl.dtype == BTC_F32 && flops >= 2e9 && pl.K >= 64;
+        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {11, 1.8}, {10, 1.7}};
         const Cand f64c[] = {{2, 1.0}, {1, 0.75}};       // big tile: the m16n8k16 variant
         const Cand other[] = {{0, 1.0}, {1, 0.75}};
         const Cand *cands = pl.dtype == BTC_F32 ? f32c : (pl.dtype == BTC_F64 ? f64c : other);
-        const int ncand = pl.dtype == BTC_F32 ? 4 : 2;
+        const int ncand = pl.dtype == BTC_F32 ? (umma_ok ? 7 : 4) : 2;
         double best = -1.0;
         for (int c = 0; c < ncand; ++c) {
             const VariantInfo vi = variant_info(pl.dtype, cands[c].id);
