@@ -106,7 +106,8 @@ btc_error_t btc_create_contraction(btc_handle_t handle,
 btc_error_t btc_destroy_contraction(btc_contraction_t *op);
 
 /* Bytes of device workspace btc_execute needs for this operation (0 for most plans; split-K
- * plans keep their partial sums there).  Alignment required: 256 bytes. */
+ * plans keep their partial sums there, Case 4 plans the inputs summed over their isolated
+ * labels).  Alignment required: 256 bytes. */
 btc_error_t btc_contraction_workspace_size(btc_contraction_t op, size_t *bytes);
 
 /* Key-value access on an operation (Sec. "Virtual Key-Value Stores").  Values are host memory. */
@@ -120,9 +121,15 @@ enum {
     BTC_ATTR_SWAPPED = 7,     /* int32, read: 1 when A and B exchanged roles                   */
     BTC_ATTR_VARIANT = 9,     /* int32, read/write: index of the tile variant of the tiled
                                  kernel for this element type (-1 on write = choose)          */
-    BTC_ATTR_DEVICE_ERROR = 8 /* int32, read: 0, or which bounded device-side wait gave up in an
+    BTC_ATTR_DEVICE_ERROR = 8,/* int32, read: 0, or which bounded device-side wait gave up in an
                                  earlier execute of this operation (its D is then incomplete);
                                  reading waits for the device                                  */
+    BTC_ATTR_PRE_REDUCE = 10  /* int32.  Case 4 of Sec. "Operations": labels that occur in one input
+                                 only are summed over before the contraction.  Write 1 (default):
+                                 a separate bandwidth-bound kernel forms the summed input in the
+                                 workspace and the contraction runs on it; write 0: the isolated
+                                 labels are summed inside the generic kernel.  Read: bit 0 / bit 1
+                                 set when A / B is summed first in the current plan             */
 };
 enum {
     BTC_KERNEL_AUTO = 0,

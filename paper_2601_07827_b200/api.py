@@ -40,6 +40,7 @@ DTYPE_SIZE = {F32: 4, F64: 8, C32: 8, C64: 16}
 ATTR_KERNEL, ATTR_SPLIT_K, ATTR_TILE, ATTR_GROUPS, ATTR_GRID, ATTR_NUM_MODES, ATTR_SWAPPED = 1, 2, 3, 4, 5, 6, 7
 ATTR_DEVICE_ERROR = 8
 ATTR_VARIANT = 9
+ATTR_PRE_REDUCE = 10
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TILED = 0, 1, 2
 STATUS_KERNEL, STATUS_LAUNCHES, STATUS_GRID, STATUS_SPLIT_K = 1, 2, 3, 4
 
@@ -214,6 +215,11 @@ class Contraction:
         return self._get(ATTR_VARIANT, ctypes.c_int32, 1)[0]
 
     @property
+    def pre_reduce(self) -> int:
+        """Case 4: bit 0 / bit 1 set when A / B is summed over its isolated labels before the contraction."""
+        return self._get(ATTR_PRE_REDUCE, ctypes.c_int32, 1)[0]
+
+    @property
     def device_error(self) -> int:
         """0, or the code of a bounded device-side wait that gave up (waits for the device)."""
         return self._get(ATTR_DEVICE_ERROR, ctypes.c_int32, 1)[0]
@@ -279,7 +285,7 @@ def dtype_code(torch_dtype) -> int:
 
 def contract(handle: Handle, A, labelsA, B, labelsB, C, D, labelsD, alpha=1.0, beta=0.0,
              conjA=False, conjB=False, conjC=False, stream: int = 0, kernel: int = KERNEL_AUTO,
-             split_k: int = 0, want_status: bool = False, variant: int = -1):
+             split_k: int = 0, want_status: bool = False, variant: int = -1, pre_reduce: Optional[bool] = None):
     """One-shot helper for tensors described by objects with .dtype, .extents, .strides and
     .data_ptr() (device memory): builds the descriptors and the operation, allocates the
     workspace with torch, executes on `stream`.  Returns (Contraction, status-or-None)."""
@@ -290,6 +296,8 @@ def contract(handle: Handle, A, labelsA, B, labelsB, C, D, labelsD, alpha=1.0, b
     tD = TensorInfo(handle, dt, D.extents, D.strides)
     tC = TensorInfo(handle, dtype_code(C.dtype), C.extents, C.strides) if C is not None else None
     op = Contraction(handle, tA, labelsA, tB, labelsB, tC, labelsD, tD, labelsD, alpha, beta, conjA, conjB, conjC)
+    if pre_reduce is not None:
+        op.set_attr(ATTR_PRE_REDUCE, int(pre_reduce))
     if kernel != KERNEL_AUTO:
         op.set_attr(ATTR_KERNEL, kernel)
     if split_k:

@@ -17,6 +17,7 @@
 #include "tiled_f64_kernel.cuh"
 #include "tiled_tf32x3_kernel.cuh"
 #include "tiled_umma_tf32x3_kernel.cuh"
+#include "isolated_sum_kernel.cuh"
 
 using namespace btc;
 
@@ -53,6 +54,13 @@ struct btc_contraction_s {
     int64_t k_per_split = 0;
     size_t workspace_bytes = 0;
     int32_t grid[3] = {0, 0, 0};
+    // Case 4: inputs with isolated labels are first summed into the front of the workspace
+    // (A' at offset 0, B' behind it), split-K partial sums follow at `partials_offset`
+    bool pre_reduce = true;
+    IsolatedSum sumA, sumB;
+    size_t sumB_offset = 0, partials_offset = 0;
+    // memory spans of the caller's tensors in elements (the plan may describe A' and B' instead)
+    int64_t spanA_lo = 0, spanA_hi = 0, spanB_lo = 0, spanB_hi = 0, spanD_lo = 0, spanD_hi = 0;
 };
 
 namespace {
@@ -359,7 +367,65 @@ int replan(btc_contraction_s *op)
     op->req.sm_count = op->handle.sm_count;
     int rc = make_plan(op->req, op->plan);
     if (rc != BTC_SUCCESS) return rc;
-    return finish_plan(op);
+    const Plan &pl = op->plan;
+    op->spanA_lo = pl.spanA_lo; op->spanA_hi = pl.spanA_hi; op->spanB_lo = pl.spanB_lo; op->spanB_hi = pl.spanB_hi;
+    op->spanD_lo = pl.spanD_lo; op->spanD_hi = pl.spanD_hi;
+    op->sumA = op->sumB = IsolatedSum();
+    op->sumB_offset = op->partials_offset = 0;
+    if (pl.has_isolated && op->pre_reduce) {
+        // Case 4: plan the contraction of the summed inputs A', B' instead
+        PlanRequest inner;
+        IsolatedSum sa, sb;
+        split_isolated(op->req, inner, sa, sb);
+        Plan reduced;
+        const bool fits = sa.keep_ext.size() <= size_t(kGenericMaxD) && sa.iso_ext.size() <= size_t(kGenericMaxD) &&
+                          sb.keep_ext.size() <= size_t(kGenericMaxD) && sb.iso_ext.size() <= size_t(kGenericMaxD);
+        if (fits && make_plan(inner, reduced) == BTC_SUCCESS) {
+            op->plan = reduced;
+            op->sumA = sa;
+            op->sumB = sb;
+        }
+    }
+    rc = finish_plan(op);
+    if (rc != BTC_SUCCESS) return rc;
+    auto round256 = [](size_t b) { return (b + 255) / 256 * 256; };
+    const size_t esz = dtype_size(op->plan.dtype);
+    const size_t bytesA = op->sumA.active ? round256(size_t(op->sumA.total_keep) * esz) : 0;
+    const size_t bytesB = op->sumB.active ? round256(size_t(op->sumB.total_keep) * esz) : 0;
+    op->sumB_offset = bytesA;
+    op->partials_offset = bytesA + bytesB;
+    op->workspace_bytes += op->partials_offset;
+    return BTC_SUCCESS;
+}
+
+template <typename R, bool CPLX>
+cudaError_t launch_isolated_sum(const IsolatedSum &s, const void *src, void *dst, int sm_count, cudaStream_t st)
+{
+    IsolatedSumParams p;
+    std::memset(&p, 0, sizeof p);
+    p.src = src; p.dst = dst;
+    p.nk = int32_t(s.keep_ext.size()); p.ni = int32_t(s.iso_ext.size());
+    p.total_keep = s.total_keep; p.total_iso = s.total_iso;
+    for (int i = 0; i < p.nk; ++i) { p.ext_k[i] = s.keep_ext[size_t(i)]; p.str_k[i] = s.keep_str[size_t(i)]; }
+    for (int i = 0; i < p.ni; ++i) { p.ext_i[i] = s.iso_ext[size_t(i)]; p.str_i[i] = s.iso_str[size_t(i)]; }
+    const int lanes = s.lanes_over_iso ? 32 : 1;
+    int64_t blocks = (s.total_keep * lanes + 255) / 256;
+    const int64_t cap = int64_t(sm_count) * 32;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (lanes == 32) isolated_sum_kernel<R, CPLX, 32><<<unsigned(blocks), 256, 0, st>>>(p);
+    else isolated_sum_kernel<R, CPLX, 1><<<unsigned(blocks), 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t run_isolated_sum(btc_dtype_t dt, const IsolatedSum &s, const void *src, void *dst, int sm_count, cudaStream_t st)
+{
+    switch (dt) {
+    case BTC_F32: return launch_isolated_sum<float, false>(s, src, dst, sm_count, st);
+    case BTC_F64: return launch_isolated_sum<double, false>(s, src, dst, sm_count, st);
+    case BTC_C32: return launch_isolated_sum<float, true>(s, src, dst, sm_count, st);
+    default: return launch_isolated_sum<double, true>(s, src, dst, sm_count, st);
+    }
 }
 
 bool is_zero(const double v[2]) { return v[0] == 0.0 && v[1] == 0.0; }
@@ -505,7 +571,11 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
     int32_t v;
     std::memcpy(&v, value, sizeof v);
     const PlanRequest saved = op->req;
-    if (key == BTC_ATTR_KERNEL) {
+    const bool saved_pre_reduce = op->pre_reduce;
+    if (key == BTC_ATTR_PRE_REDUCE) {
+        if (v != 0 && v != 1) return BTC_ERR_INVALID_ARGUMENT;
+        op->pre_reduce = v != 0;
+    } else if (key == BTC_ATTR_KERNEL) {
         if (v < BTC_KERNEL_AUTO || v > BTC_KERNEL_TILED) return BTC_ERR_INVALID_ARGUMENT;
         op->req.force_kernel = v;
     } else if (key == BTC_ATTR_VARIANT) {
@@ -519,6 +589,7 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
     int rc = replan(op);
     if (rc != BTC_SUCCESS) {   // keep the object usable with its previous plan
         op->req = saved;
+        op->pre_reduce = saved_pre_reduce;
         replan(op);
     }
     return rc;
@@ -543,6 +614,7 @@ btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t 
         i32[2] = int32_t(pl.n.size()); i32[3] = int32_t(pl.k.size()); n = 16; break;
     case BTC_ATTR_SWAPPED: i32[0] = pl.swapped ? 1 : 0; n = 4; break;
     case BTC_ATTR_VARIANT: i32[0] = pl.tile.variant; n = 4; break;
+    case BTC_ATTR_PRE_REDUCE: i32[0] = (op->sumA.active ? 1 : 0) | (op->sumB.active ? 2 : 0); n = 4; break;
     case BTC_ATTR_DEVICE_ERROR:
         i32[0] = 0;
         if (op->d_error) {
@@ -586,9 +658,23 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         if (misaligned(workspace, 256)) return BTC_ERR_MISALIGNED;
     }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const void *pA = pl.swapped ? B : A, *pB = pl.swapped ? A : B;
     int launches = 0;
     cudaError_t ce = cudaSuccess;
+    // Case 4: sum the inputs over their isolated labels first; the contraction then reads A', B'
+    if (use_ab && op->sumA.active) {
+        ce = run_isolated_sum(pl.dtype, op->sumA, A, workspace, op->handle.sm_count, st);
+        if (ce != cudaSuccess) return BTC_ERR_CUDA;
+        A = workspace;
+        ++launches;
+    }
+    if (use_ab && op->sumB.active) {
+        void *dst = static_cast<char *>(workspace) + op->sumB_offset;
+        ce = run_isolated_sum(pl.dtype, op->sumB, B, dst, op->handle.sm_count, st);
+        if (ce != cudaSuccess) return BTC_ERR_CUDA;
+        B = dst;
+        ++launches;
+    }
+    const void *pA = pl.swapped ? B : A, *pB = pl.swapped ? A : B;
 
     if (pl.kernel == BTC_KERNEL_GENERIC || !use_ab) {
         GenericParams gp;
@@ -623,7 +709,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         case BTC_C32: ce = launch_generic<float, true>(gp, blocks, wpe, st); break;
         case BTC_C64: ce = launch_generic<double, true>(gp, blocks, wpe, st); break;
         }
-        launches = 1;
+        launches += 1;
     } else {
         TiledParams tp;
         std::memset(&tp, 0, sizeof tp);
@@ -642,7 +728,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         tp.conjA = pl.conjA; tp.conjB = pl.conjB; tp.conjC = pl.conjC;
         tp.use_c = use_c;
         tp.alpha[0] = al[0]; tp.alpha[1] = al[1]; tp.beta[0] = be[0]; tp.beta[1] = be[1];
-        tp.partials = workspace;
+        tp.partials = workspace ? static_cast<char *>(workspace) + op->partials_offset : nullptr;
         tp.error_word = op->d_error;
 #ifdef BTC_STAMPS
         { void *sp = nullptr; cudaGetSymbolAddress(&sp, btc_stamp_buffer); tp.stamps = static_cast<long long *>(sp); }
@@ -681,7 +767,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         else
             ce = pl.tile.variant == 0 ? launch_tiled<C64Big>(tp, ctas, reduce_ctas, st)
                                       : launch_tiled<C64Small>(tp, ctas, reduce_ctas, st);
-        launches = pl.split_k > 1 ? 2 : 1;
+        launches += pl.split_k > 1 ? 2 : 1;
     }
     if (ce != cudaSuccess) return BTC_ERR_CUDA;
     if (status) {
@@ -716,9 +802,9 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
         size_t bytes() const { return size_t(hi - lo + 1); }
     } bA, bB, bC, bD;
     auto span_bytes = [&](Buf &b, int64_t lo, int64_t hi) { b.lo = lo * int64_t(esz); b.hi = hi * int64_t(esz) + int64_t(esz) - 1; };
-    span_bytes(bA, pl.spanA_lo, pl.spanA_hi);
-    span_bytes(bB, pl.spanB_lo, pl.spanB_hi);
-    span_bytes(bD, pl.spanD_lo, pl.spanD_hi);
+    span_bytes(bA, op->spanA_lo, op->spanA_hi);
+    span_bytes(bB, op->spanB_lo, op->spanB_hi);
+    span_bytes(bD, op->spanD_lo, op->spanD_hi);
     bC = bD;
     const bool c_is_d = use_c && C == D;
     void *ws = nullptr;

@@ -21,6 +21,16 @@ struct GenericParams {
     int32_t use_ab, use_c;
 };
 
+// Sum over the isolated labels of one input (Case 4): kept and isolated loop dimensions of the
+// tensor, each with its extent and element stride, first entry fastest.
+struct IsolatedSumParams {
+    const void *src;
+    void *dst;                        // dense, kept dimensions in the order given here
+    int32_t nk, ni;
+    int64_t total_keep, total_iso;
+    int64_t ext_k[kGenericMaxD], str_k[kGenericMaxD], ext_i[kGenericMaxD], str_i[kGenericMaxD];
+};
+
 // Tiled contraction kernels.  All offsets are in elements of the operation's dtype.
 struct TiledParams {
     const void *A, *B, *C;

@@ -372,6 +372,45 @@ int make_plan(const PlanRequest &req, Plan &plan)
     return BTC_SUCCESS;
 }
 
+void split_isolated(const PlanRequest &req, PlanRequest &inner, IsolatedSum &sumA, IsolatedSum &sumB)
+{
+    inner = req;
+    auto contains = [](const std::vector<int64_t> &v, int64_t x) { return std::find(v.begin(), v.end(), x) != v.end(); };
+    auto one = [&](const TensorDesc &X, const std::vector<int64_t> &labX, const std::vector<int64_t> &labOther,
+                   TensorDesc &Xr, std::vector<int64_t> &labXr, IsolatedSum &sum) {
+        struct U { int64_t label, extent, stride; bool iso; };
+        std::vector<U> u;                                   // unique labels, strides of repeats added (Note 6)
+        for (size_t i = 0; i < labX.size(); ++i) {
+            size_t k = 0;
+            while (k < u.size() && u[k].label != labX[i]) ++k;
+            if (k == u.size()) u.push_back({labX[i], X.extent[i], 0, !contains(labOther, labX[i]) && !contains(req.labelsD, labX[i])});
+            u[k].stride += X.stride[i];
+        }
+        sum = IsolatedSum();
+        for (auto &x : u) sum.active = sum.active || (x.iso && x.extent > 1);
+        if (!sum.active) return;
+        std::stable_sort(u.begin(), u.end(), [](const U &a, const U &b) { return iabs(a.stride) < iabs(b.stride); });
+        Xr.extent.clear(); Xr.stride.clear(); labXr.clear();
+        int64_t min_keep = INT64_MAX, min_iso = INT64_MAX;
+        for (auto &x : u) {
+            if (x.iso) {
+                if (x.extent == 1) continue;
+                sum.iso_ext.push_back(x.extent); sum.iso_str.push_back(x.stride);
+                sum.total_iso *= x.extent;
+                min_iso = std::min(min_iso, iabs(x.stride));
+            } else {
+                sum.keep_ext.push_back(x.extent); sum.keep_str.push_back(x.stride);
+                Xr.extent.push_back(x.extent); Xr.stride.push_back(sum.total_keep); labXr.push_back(x.label);
+                sum.total_keep *= x.extent;
+                if (x.extent > 1) min_keep = std::min(min_keep, iabs(x.stride));
+            }
+        }
+        sum.lanes_over_iso = min_iso < min_keep && sum.total_iso >= 32;
+    };
+    one(req.A, req.labelsA, req.labelsB, inner.A, inner.labelsA, sumA);
+    one(req.B, req.labelsB, req.labelsA, inner.B, inner.labelsB, sumB);
+}
+
 std::string Plan::describe() const
 {
     std::ostringstream o;

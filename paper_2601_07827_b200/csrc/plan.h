@@ -41,7 +41,7 @@ struct Plan {
     bool conjA = false, conjB = false, conjC = false;  // in planned roles (after swap)
     bool swapped = false;        // true: the caller's B is the plan's A
     bool has_c_desc = false;
-    bool has_isolated = false;   // Case 4 labels present (summed inside the generic kernel)
+    bool has_isolated = false;   // Case 4 labels present; if planned as they are, the generic kernel sums them
 
     // loop dimensions in planned order, first entry fastest in the linearised index
     std::vector<Mode> batch, m, n, k;
@@ -78,6 +78,20 @@ struct PlanRequest {
 
 // Validates the request and fills `plan`.  Returns a btc_error_t.
 int make_plan(const PlanRequest &req, Plan &plan);
+
+// Case 4: the sum over the labels that occur in one input only, taken before the contraction.
+struct IsolatedSum {
+    bool active = false;
+    // loop dimensions of the input tensor (repeated labels merged), smallest |stride| first
+    std::vector<int64_t> keep_ext, keep_str, iso_ext, iso_str;
+    int64_t total_keep = 1, total_iso = 1;
+    bool lanes_over_iso = false;   // the isolated index is the more contiguous one: one warp per result element
+};
+
+// For a validated request: `inner` = the same contraction on A' and B', the inputs summed over
+// their isolated labels (dense, kept labels in order of increasing |stride| in the input; an
+// input without isolated labels is passed through), and how to form A' and B'.
+void split_isolated(const PlanRequest &req, PlanRequest &inner, IsolatedSum &sumA, IsolatedSum &sumB);
 
 size_t dtype_size(btc_dtype_t t);
 bool dtype_is_complex(btc_dtype_t t);

@@ -44,7 +44,7 @@ def canary_intact(before: torch.Tensor, after: torch.Tensor, touched: torch.Tens
 
 
 def run_case(handle, A, la, B, lb, C, D, ld, alpha=1.0, beta=0.0, conjA=False, conjB=False, conjC=False,
-             kernel=0, split_k=0, host_path=False, want_status=False, variant=-1):
+             kernel=0, split_k=0, host_path=False, want_status=False, variant=-1, pre_reduce=None):
     """A, B, C, D are inputs.StridedTensor on the CPU; D is not modified.  Returns
     (worst error in tolerance units, status dict or None, GPU result buffer on the CPU)."""
     _api = api()
@@ -69,7 +69,7 @@ def run_case(handle, A, la, B, lb, C, D, ld, alpha=1.0, beta=0.0, conjA=False, c
     else:
         _, status = _api.contract(handle, dA, la, dB, lb, dC, dD, ld, alpha, beta, conjA, conjB, conjC,
                                   stream=torch.cuda.current_stream().cuda_stream, kernel=kernel,
-                                  split_k=split_k, want_status=want_status, variant=variant)
+                                  split_k=split_k, want_status=want_status, variant=variant, pre_reduce=pre_reduce)
         torch.cuda.synchronize()
         result = dD.buffer.cpu()
 

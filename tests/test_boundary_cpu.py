@@ -149,10 +149,21 @@ def test_planner_kernel_choice_and_split_k(api, handle):
     assert op.kernel == api.KERNEL_GENERIC
     tiny = _op(api, handle, (2, 3), "ik", (3, 2), "kj", (2, 2), "ij")
     assert tiny.kernel == api.KERNEL_GENERIC
-    case4 = _op(api, handle, (64, 64, 5), "ikx", (64, 64), "kj", (64, 64), "ij")   # isolated label x
-    assert case4.kernel == api.KERNEL_GENERIC
+    # Case 4, isolated label x: by default A is first summed over x into the workspace and the tiled
+    # kernel contracts the result; with the pre-reduction off the generic kernel sums x itself
+    case4 = _op(api, handle, (64, 64, 5), "ikx", (64, 64), "kj", (64, 64), "ij")
+    assert case4.kernel == api.KERNEL_TILED and case4.pre_reduce == 1
+    assert case4.groups == (1, 64, 64, 64)
+    assert case4.workspace_size() >= 64 * 64 * 8
+    case4.set_attr(api.ATTR_PRE_REDUCE, 0)
+    assert case4.kernel == api.KERNEL_GENERIC and case4.pre_reduce == 0
+    assert case4.groups == (1, 64, 64, 64 * 5)
     assert _code(api, lambda: case4.set_attr(api.ATTR_KERNEL, api.KERNEL_TILED)) == api.ERR_NOT_SUPPORTED
     assert case4.kernel == api.KERNEL_GENERIC
+    case4.set_attr(api.ATTR_PRE_REDUCE, 1)
+    assert case4.kernel == api.KERNEL_TILED
+    both = _op(api, handle, (7, 64, 64), "xik", (64, 64, 3, 3), "kjyy", (64, 64), "ij")   # x in A; y twice in B
+    assert both.pre_reduce == 3 and both.groups == (1, 64, 64, 64)
 
 
 def test_execute_without_device_fails_loudly(api, handle):

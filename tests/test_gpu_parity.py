@@ -249,3 +249,41 @@ def test_persistent_tensor_memory_kernel_walks_many_tiles(api, handle, variant):
     assert worst <= 1.0 and status["kernel"] == api.KERNEL_TILED
     bn = {10: 96, 11: 128, 12: 256}[variant]
     assert status["grid"][0] < -(-ext["i"] // 128) * -(-ext["j"] // bn) * ext["z"]   # fewer CTAs than tiles
+
+
+CASE4 = {
+    # name: (labelsA, labelsB, labelsD, extents, stridesA or None)
+    "x_slowest_in_A": ("ikx", "kj", "ij", dict(i=150, j=90, k=70, x=6), None),
+    "x_fastest_in_A": ("xik", "kj", "ij", dict(i=150, j=90, k=70, x=40), None),          # one warp per element of A'
+    "both_inputs": ("ixk", "ykjz", "ij", dict(i=130, j=70, k=50, x=5, y=3, z=4), None),
+    "trace_of_repeated_isolated": ("xikx", "kj", "ij", dict(i=60, j=50, k=40, x=9), None),
+    "all_of_B_isolated": ("ik", "xy", "ik", dict(i=80, k=60, x=7, y=5), None),            # B' is a scalar
+    "padded_negative": ("ikx", "kj", "ij", dict(i=100, j=64, k=48, x=5), (-1, 104, 104 * 50)),
+    "with_batch": ("hixk", "khj", "ijh", dict(h=3, i=70, j=66, k=40, x=4), None),
+}
+
+
+@pytest.mark.parametrize("dtype", REAL_AND_COMPLEX)
+@pytest.mark.parametrize("name", list(CASE4))
+def test_case4_isolated_labels_are_summed_first(api, handle, name, dtype):
+    """Case 4: labels that occur in one input only.  The default plan sums that input over them in
+    a kernel of its own (workspace) and contracts the result with the tiled kernel; with the
+    pre-reduction switched off the generic kernel sums them inside the contraction.  Both must
+    match the oracle, which follows the definition."""
+    la, lb, ld, ext, sA = CASE4[name]
+    A = helpers.random_tensor(91, _ext(la, ext), sA, dtype)
+    B = helpers.random_tensor(92, _ext(lb, ext), None, dtype)
+    C = helpers.random_tensor(93, _ext(ld, ext), None, dtype)
+    D = inputs.place(None, _ext(ld, ext), None, dtype)
+    cplx = dtype.is_complex
+    alpha = complex(0.5, 0.25) if cplx else 0.5
+    worst, status, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, 1.0, conjA=cplx, conjB=cplx, want_status=True)
+    assert worst <= 1.0, worst
+    sums = 2 if name == "both_inputs" else 1
+    assert status["launches"] >= 1 + sums
+    worst, status, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, 1.0, conjA=cplx, conjB=cplx,
+                                        pre_reduce=False, want_status=True)
+    assert worst <= 1.0 and status["launches"] == 1 and status["kernel"] == api.KERNEL_GENERIC
+    if name == "x_slowest_in_A":
+        worst, _, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, 1.0, conjA=cplx, conjB=cplx, host_path=True)
+        assert worst <= 1.0
