@@ -413,8 +413,14 @@ cudaError_t launch_isolated_sum(const IsolatedSum &s, const void *src, void *dst
     const int64_t cap = int64_t(sm_count) * 32;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    if (lanes == 32) isolated_sum_kernel<R, CPLX, 32><<<unsigned(blocks), 256, 0, st>>>(p);
-    else isolated_sum_kernel<R, CPLX, 1><<<unsigned(blocks), 256, 0, st>>>(p);
+    const bool narrow = s.total_keep < (int64_t(1) << 31) && s.total_iso < (int64_t(1) << 31);   // indices fit 32 bits
+    if (lanes == 32) {
+        if (narrow) isolated_sum_kernel<R, CPLX, 32, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);
+        else isolated_sum_kernel<R, CPLX, 32, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);
+    } else {
+        if (narrow) isolated_sum_kernel<R, CPLX, 1, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);
+        else isolated_sum_kernel<R, CPLX, 1, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);
+    }
     return cudaGetLastError();
 }
 

@@ -14,41 +14,81 @@
 
 namespace btc {
 
-template <typename R, bool CPLX, int LANES>
+// Mixed-radix decode of a linear index into an element offset; 32-bit arithmetic when it fits
+// (64-bit division costs an order of magnitude more instructions).
+template <typename I>
+__device__ __forceinline__ int64_t decode_offset(I lin, int nd, const int64_t *ext, const int64_t *str)
+{
+    if (nd == 1) return int64_t(lin) * str[0];      // the common case after chained dimensions are merged
+    int64_t off = 0;
+    for (int d = 0; d < nd; ++d) {
+        const I e = I(ext[d]);
+        const I q = lin / e;
+        off += int64_t(lin - q * e) * str[d];
+        lin = q;
+    }
+    return off;
+}
+
+template <typename R, bool CPLX, int LANES, typename I>
 __global__ void __launch_bounds__(256) isolated_sum_kernel(const IsolatedSumParams p)
 {
     constexpr int NC = CPLX ? 2 : 1;
+    // independent loads in flight per thread: LANES = 1 unrolls the isolated index of one result
+    // element, LANES = 32 works on several result elements at a time
+    constexpr int U = LANES == 1 ? 8 : 1, E = LANES == 1 ? 1 : 4;
     const R *src = static_cast<const R *>(p.src);
     R *dst = static_cast<R *>(p.dst);
     const int lane = (LANES == 1) ? 0 : int(threadIdx.x) % LANES;
     const int64_t group = (int64_t(blockIdx.x) * blockDim.x + threadIdx.x) / LANES;
     const int64_t ngroups = (int64_t(gridDim.x) * blockDim.x) / LANES;
-    for (int64_t e = group; e < p.total_keep; e += ngroups) {
-        int64_t base = 0, lin = e;
-        for (int d = 0; d < p.nk; ++d) {
-            base += (lin % p.ext_k[d]) * p.str_k[d];
-            lin /= p.ext_k[d];
-        }
-        double acc_r = 0.0, acc_i = 0.0;
-        for (int64_t s = lane; s < p.total_iso; s += LANES) {
-            int64_t off = base, r = s;
-            for (int d = 0; d < p.ni; ++d) {
-                off += (r % p.ext_i[d]) * p.str_i[d];
-                r /= p.ext_i[d];
-            }
-            acc_r += double(src[NC * off]);
-            if (CPLX) acc_i += double(src[NC * off + (NC - 1)]);
-        }
-        if (LANES > 1) {
+    for (int64_t e0 = group; e0 < p.total_keep; e0 += ngroups * E) {
+        int64_t base[E];
+        bool live[E];
+        double acc_r[E], acc_i[E];
 #pragma unroll
-            for (int o = LANES / 2; o > 0; o >>= 1) {
-                acc_r += __shfl_xor_sync(0xffffffffu, acc_r, o);
-                if (CPLX) acc_i += __shfl_xor_sync(0xffffffffu, acc_i, o);
-            }
+        for (int j = 0; j < E; ++j) {
+            const int64_t e = e0 + j * ngroups;
+            live[j] = e < p.total_keep;
+            base[j] = live[j] ? decode_offset<I>(I(e), p.nk, p.ext_k, p.str_k) : 0;
+            acc_r[j] = acc_i[j] = 0.0;
         }
-        if (lane == 0) {
-            dst[NC * e] = R(acc_r);
-            if (CPLX) dst[NC * e + (NC - 1)] = R(acc_i);
+        for (int64_t s0 = lane; s0 < p.total_iso; s0 += int64_t(U) * LANES) {
+            R v_r[E][U], v_i[E][U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int64_t s = s0 + int64_t(u) * LANES;
+                const bool in_s = s < p.total_iso;
+                const int64_t so = in_s ? decode_offset<I>(I(s), p.ni, p.ext_i, p.str_i) : 0;
+#pragma unroll
+                for (int j = 0; j < E; ++j) {
+                    const bool in = in_s && live[j];
+                    v_r[j][u] = in ? src[NC * (base[j] + so)] : R(0);
+                    v_i[j][u] = (CPLX && in) ? src[NC * (base[j] + so) + (NC - 1)] : R(0);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < E; ++j)
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    acc_r[j] += double(v_r[j][u]);
+                    if (CPLX) acc_i[j] += double(v_i[j][u]);
+                }
+        }
+#pragma unroll
+        for (int j = 0; j < E; ++j) {
+            if (LANES > 1) {
+#pragma unroll
+                for (int o = LANES / 2; o > 0; o >>= 1) {
+                    acc_r[j] += __shfl_xor_sync(0xffffffffu, acc_r[j], o);
+                    if (CPLX) acc_i[j] += __shfl_xor_sync(0xffffffffu, acc_i[j], o);
+                }
+            }
+            const int64_t e = e0 + j * ngroups;
+            if (lane == 0 && e < p.total_keep) {
+                dst[NC * e] = R(acc_r[j]);
+                if (CPLX) dst[NC * e + (NC - 1)] = R(acc_i[j]);
+            }
         }
     }
 }

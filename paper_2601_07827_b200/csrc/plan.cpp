@@ -406,6 +406,18 @@ void split_isolated(const PlanRequest &req, PlanRequest &inner, IsolatedSum &sum
             }
         }
         sum.lanes_over_iso = min_iso < min_keep && sum.total_iso >= 32;
+        // neighbours whose strides chain act as one loop dimension (fewer divisions per element);
+        // X' keeps the same element order either way
+        auto chain = [](std::vector<int64_t> &ext, std::vector<int64_t> &str) {
+            size_t w = 0;
+            for (size_t i = 0; i < ext.size(); ++i) {
+                if (w > 0 && str[i] == str[w - 1] * ext[w - 1]) { ext[w - 1] *= ext[i]; continue; }
+                ext[w] = ext[i]; str[w] = str[i]; ++w;
+            }
+            ext.resize(w); str.resize(w);
+        };
+        chain(sum.keep_ext, sum.keep_str);
+        chain(sum.iso_ext, sum.iso_str);
     };
     one(req.A, req.labelsA, req.labelsB, inner.A, inner.labelsA, sumA);
     one(req.B, req.labelsB, req.labelsA, inner.B, inner.labelsB, sumB);

@@ -336,6 +336,16 @@ def workloads() -> Dict[str, Workload]:
     # 5b: same with D's fastest label being B's slowest (adversarial output order)
     w["cfg5b_f32_tensor_network_rev"] = dataclasses.replace(
         w["cfg5_f32_tensor_network"], name="cfg5b_f32_tensor_network_rev", labelsD="jeidhcgbfa")
+    # 6: Case 4, the ladder term with an extra label x that only A carries (summed over first):
+    #    D[a,b,i,j] = sum_cd (sum_x A[a,b,c,d,x]) T[c,d,i,j];  A is 1 GiB, the sum over x is HBM-bound
+    e6 = {**_all(64, "abcd"), **_all(32, "ij"), "x": 8}
+    w["cfg6_f64_case4_isolated"] = Workload(
+        "cfg6_f64_case4_isolated", "f64", "abcdx", "cdij", "abij", e6, alpha=1.0, beta=0.0, seed=6000,
+        distA=("normal", 0.1), distB=("uniform", 0.01))
+    # 6b: the isolated label is A's fastest one (one warp per summed element)
+    w["cfg6b_f64_case4_isolated_fast"] = dataclasses.replace(
+        w["cfg6_f64_case4_isolated"], name="cfg6b_f64_case4_isolated_fast", labelsA="xabcd",
+        extents={**e6, "x": 32, **_all(32, "ab")})
     return w
 
 

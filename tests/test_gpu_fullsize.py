@@ -20,6 +20,8 @@ CASES = {
     "cfg2_f64_ccsd_ladder": (6000, 16384),
     "cfg3_f32_batched_permuted": (40000, 96 * 96),
     "cfg4_c64_conj": (20000, 256 * 256),
+    "cfg6_f64_case4_isolated": (6000, 64 * 64),       # Case 4: A summed over its isolated label first
+    "cfg6b_f64_case4_isolated_fast": (6000, 32 * 32),
 }
 
 
