@@ -73,6 +73,7 @@ using F64Big3 = F64Tile<false, 128, 128, 2, 4, 3, 1>;           // 3 stages
 using F64BigT = F64Tile<false, 128, 128, 4, 2, 4, 1>;           // warp tile 32 x 64
 using C64Big = F64Tile<true, 128, 64, 2, 4, 4, 1>;
 using C64Small = F64Tile<true, 64, 32, 2, 4, 4, 2>;
+using C64Big16 = F64Tile<true, 128, 64, 2, 4, 4, 1, true>;     // m16n8k16 MMAs
 
 using F32Big = F32Tile<128, 128, 16, 2, 4, 5, 1, false>;
 using F32Small = F32Tile<64, 64, 16, 2, 2, 5, 2, false>;
@@ -133,7 +134,7 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
         }
     }
     if (t == BTC_C32) return variant == 0 ? info_of<C32Tc>(4) : info_of<C32TcSmall>(4);
-    return variant == 0 ? info_of<C64Big>(8) : info_of<C64Small>(8);
+    return variant == 0 ? info_of<C64Big>(8) : (variant == 1 ? info_of<C64Small>(8) : info_of<C64Big16>(8));
 }
 
 template <typename K>
@@ -279,8 +280,9 @@ int finish_plan(btc_contraction_s *op)
         const bool umma_ok = pl.dtype == BTC_F32 && flops >= 2e9 && pl.K >= 64;
         const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {11, 1.8}, {10, 1.7}};
         const Cand f64c[] = {{2, 1.0}, {1, 0.75}};       // big tile: the m16n8k16 variant
+        const Cand c64c[] = {{2, 1.0}, {1, 0.75}};       // complex128: big tile on m16n8k16 as well
         const Cand other[] = {{0, 1.0}, {1, 0.75}};
-        const Cand *cands = pl.dtype == BTC_F32 ? f32c : (pl.dtype == BTC_F64 ? f64c : other);
+        const Cand *cands = pl.dtype == BTC_F32 ? f32c : (pl.dtype == BTC_F64 ? f64c : (pl.dtype == BTC_C64 ? c64c : other));
         const int ncand = pl.dtype == BTC_F32 ? (umma_ok ? 7 : 4) : 2;
         double best = -1.0;
         for (int c = 0; c < ncand; ++c) {
@@ -296,7 +298,7 @@ int finish_plan(btc_contraction_s *op)
         }
     }
     if (op->req.force_variant >= 0) {
-        const int count = pl.dtype == BTC_F32 ? kNumF32Variants : (pl.dtype == BTC_F64 ? 5 : 2);
+        const int count = pl.dtype == BTC_F32 ? kNumF32Variants : (pl.dtype == BTC_F64 ? 5 : (pl.dtype == BTC_C64 ? 3 : 2));
         if (op->req.force_variant >= count) return BTC_ERR_INVALID_ARGUMENT;
         variant = op->req.force_variant;
     }
@@ -318,6 +320,16 @@ int finish_plan(btc_contraction_s *op)
         split = (2 * int64_t(sms)) / tiles;
         const int64_t max_split = k_tiles / 2;   // at least two K tiles per slice
         if (split > max_split) split = max_split;
+    } else {
+        // A few waves with a poorly filled last one: slicing K by 2-4 makes the CTAs shorter and the
+        // last wave fuller.  Cost model in units of one unsplit tile: waves / slices, plus the
+        // partial images' round trip through memory (about 50 elements' worth of work per slice).
+        const double slots = double(sms) * (v.bm * v.bn <= 64 * 64 ? 2.0 : 1.0);
+        double best = std::ceil(double(tiles) / slots);
+        for (int64_t sl = 2; sl <= 4 && k_tiles / sl >= 16; ++sl) {
+            const double t = std::ceil(double(tiles * sl) / slots) / double(sl) * (1.0 + 50.0 * double(sl) / double(pl.K));
+            if (t < 0.97 * best) { best = t; split = sl; }
+        }
     }
     if (split > k_tiles) split = k_tiles;
     if (split < 1) split = 1;
@@ -772,7 +784,8 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
             }
         else
             ce = pl.tile.variant == 0 ? launch_tiled<C64Big>(tp, ctas, reduce_ctas, st)
-                                      : launch_tiled<C64Small>(tp, ctas, reduce_ctas, st);
+                 : (pl.tile.variant == 1 ? launch_tiled<C64Small>(tp, ctas, reduce_ctas, st)
+                                         : launch_tiled<C64Big16>(tp, ctas, reduce_ctas, st));
         launches += pl.split_k > 1 ? 2 : 1;
     }
     if (ce != cudaSuccess) return BTC_ERR_CUDA;
