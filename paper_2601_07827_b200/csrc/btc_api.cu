@@ -87,10 +87,14 @@ using C32Tc = TF32Tile<true, 128, 64, 2, 4, 4, 1>;
 using C32TcSmall = TF32Tile<true, 64, 32, 2, 4, 4, 2>;
 using F32TcWide = TF32Tile<false, 256, 96, 4, 2, 4, 1>;          // N = 96 fills the tile exactly
 using F32TcMid = TF32Tile<false, 128, 96, 2, 4, 4, 1>;
-using F32Umma96 = UmmaTile<96, 4, 2>;                              // tcgen05 + tensor memory, 3xTF32
+using F32Umma96 = UmmaTile<96, 4, 2>;
+using F32Umma96T = UmmaTile<96, 5, 2, true>;                       // M-side operand through tensor memory
+using F32Umma128T = UmmaTile<128, 4, 2, true>;
+using F32Umma96T2 = UmmaTile<96, 5, 2, true, 2>;                   // two converter groups take the stages in turn
+using F32Umma128T2 = UmmaTile<128, 4, 2, true, 2>;                              // tcgen05 + tensor memory, 3xTF32
 using F32Umma128 = UmmaTile<128, 4, 2>;
 using F32Umma256 = UmmaTile<256, 3, 1>;
-constexpr int kNumF32Variants = 13;
+constexpr int kNumF32Variants = 17;
 constexpr int kFirstUmmaVariant = 10;
 
 struct VariantInfo {
@@ -130,7 +134,11 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
         case 9: return info_of<F32TcMid>(4);
         case 10: return {128, 96, 32, 256, 0, F32Umma96::SMEM_BYTES, 4};
         case 11: return {128, 128, 32, 256, 0, F32Umma128::SMEM_BYTES, 4};
-        default: return {128, 256, 32, 256, 0, F32Umma256::SMEM_BYTES, 4};
+        case 12: return {128, 256, 32, 256, 0, F32Umma256::SMEM_BYTES, 4};
+        case 13: return {128, 96, 32, 256, 0, F32Umma96T::SMEM_BYTES, 4};
+        case 14: return {128, 128, 32, 256, 0, F32Umma128T::SMEM_BYTES, 4};
+        case 15: return {128, 96, 32, 256, 0, F32Umma96T2::SMEM_BYTES, 4};
+        default: return {128, 128, 32, 256, 0, F32Umma128T2::SMEM_BYTES, 4};
         }
     }
     if (t == BTC_C32) return variant == 0 ? info_of<C32Tc>(4) : info_of<C32TcSmall>(4);
@@ -769,7 +777,11 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
             case 9: ce = launch_tiled_tf32<F32TcMid>(tp, ctas, reduce_ctas, st); break;
             case 10: ce = launch_umma<F32Umma96>(tp, ctas, st); break;
             case 11: ce = launch_umma<F32Umma128>(tp, ctas, st); break;
-            default: ce = launch_umma<F32Umma256>(tp, ctas, st); break;
+            case 12: ce = launch_umma<F32Umma256>(tp, ctas, st); break;
+            case 13: ce = launch_umma<F32Umma96T>(tp, ctas, st); break;
+            case 14: ce = launch_umma<F32Umma128T>(tp, ctas, st); break;
+            case 15: ce = launch_umma<F32Umma96T2>(tp, ctas, st); break;
+            default: ce = launch_umma<F32Umma128T2>(tp, ctas, st); break;
             }
         } else if (pl.dtype == BTC_C32) {
             ce = pl.tile.variant == 0 ? launch_tiled_tf32<C32Tc>(tp, ctas, reduce_ctas, st)

@@ -34,25 +34,37 @@
 
 namespace btc {
 
-template <int BN_, int RAW_STAGES_, int TAIL_STAGES_>
+template <int BN_, int RAW_STAGES_, int TAIL_STAGES_, bool A_TMEM_ = false, int CONVERTER_GROUPS_ = 1>
 struct UmmaTile {
     static constexpr int BM = 128, BN = BN_, BK = 32;
     static constexpr int RAW_STAGES = RAW_STAGES_, TAIL_STAGES = TAIL_STAGES_;
+    // A_TMEM: the M-side operand reaches the tensor core through tensor memory (the converters
+    // write its head and tail there), so the tensor core reads only the N-side operand from
+    // shared memory and a tail stage holds only that operand's tail
+    static constexpr bool A_TMEM = A_TMEM_;
     static constexpr int EPILOGUE_WARPS = 4, EPILOGUE_THREADS = 128;  // warps 0-3: one tensor-memory lane quarter each
-    static constexpr int CONVERTER_WARPS = 4, CONVERTER_THREADS = 128;
+    // converter groups of 4 warps (128 threads = the tile's 128 rows) take the stages in turn
+    static constexpr int CONVERTER_GROUPS = CONVERTER_GROUPS_;
+    static constexpr int CONVERTER_WARPS = 4 * CONVERTER_GROUPS_, CONVERTER_THREADS = 128;   // threads per group
     static constexpr int PRODUCER_WARPS = 4, PRODUCER_THREADS = 128;
     static constexpr int MMA_WARP = EPILOGUE_WARPS + CONVERTER_WARPS + PRODUCER_WARPS;
     static constexpr int THREADS = 32 * (MMA_WARP + 1);
     static constexpr int A_BYTES = BM * BK * 4, B_BYTES = BN * BK * 4;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;           // same size for raw and tail stages
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;           // a raw stage
+    static constexpr int TAIL_BYTES = A_TMEM_ ? B_BYTES : STAGE_BYTES;
+    static constexpr int TAIL_B_OFFSET = A_TMEM_ ? 0 : A_BYTES;     // where the N-side tail sits in a tail stage
     static constexpr int ACC_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;   // one accumulator
-    static constexpr int TMEM_COLS = 2 * ACC_COLS;                  // two: epilogue and main loop overlap
-    static constexpr int PIECES = STAGE_BYTES / 16 / CONVERTER_THREADS;   // 16-byte pieces per converter thread
+    static constexpr int A_COLS = A_TMEM_ ? 2 * BK : 0;             // head + tail of one stage of the M-side operand
+    static constexpr int TMEM_USED = 2 * ACC_COLS + TAIL_STAGES_ * A_COLS;
+    static constexpr int TMEM_COLS = TMEM_USED <= 32 ? 32 : TMEM_USED <= 64 ? 64 : TMEM_USED <= 128 ? 128 : TMEM_USED <= 256 ? 256 : 512;
+    static_assert(TMEM_USED <= 512, "accumulators and operand stages must fit the 512 tensor-memory columns");
+    // 16-byte pieces per converter thread in the position-independent pass (whole stage, or its N side)
+    static constexpr int PIECES = (A_TMEM_ ? B_BYTES : STAGE_BYTES) / 16 / CONVERTER_THREADS;
     static constexpr int NUM_BARS = 2 * RAW_STAGES + 2 * TAIL_STAGES + 8;
-    static_assert(STAGE_BYTES % (16 * CONVERTER_THREADS) == 0, "a stage must divide among the converters");
+    static_assert(B_BYTES % (16 * CONVERTER_THREADS) == 0, "a stage must divide among the converters");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "BN must suit UMMA N and the epilogue split");
     // stages | row/col offsets | k offsets | mbarriers | tmem ptr, abort
-    static constexpr size_t SMEM_BYTES = size_t(RAW_STAGES + TAIL_STAGES) * STAGE_BYTES +
+    static constexpr size_t SMEM_BYTES = size_t(RAW_STAGES) * STAGE_BYTES + size_t(TAIL_STAGES) * TAIL_BYTES +
                                          size_t(2 * BM + 4 * BN + 2 * kKoffCap) * 8 + size_t(NUM_BARS) * 8 + 16 +
                                          1024;   // + slack to align the tiles
 };
@@ -84,6 +96,26 @@ __device__ __forceinline__ void umma_tf32(unsigned tmem_c, uint64_t desc_a, uint
                  ::"r"(tmem_c), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
                  : "memory");
 }
+// same with the M-side operand read from tensor memory (lane = row, one column per k)
+__device__ __forceinline__ void umma_tf32_ts(unsigned tmem_c, unsigned tmem_a, uint64_t desc_b, unsigned idesc, unsigned accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+                 ::"r"(tmem_c), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+                 : "memory");
+}
+// 32 consecutive columns of this lane's tensor-memory row
+__device__ __forceinline__ void tmem_store32(unsigned taddr, const float (&v)[32])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+                 ::"r"(taddr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]),
+                   "f"(v[8]), "f"(v[9]), "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]),
+                   "f"(v[16]), "f"(v[17]), "f"(v[18]), "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]),
+                   "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_store_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_load16(unsigned taddr, unsigned (&r)[16])
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -256,7 +288,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     // operand tiles must sit on 1024-byte boundaries of the shared-memory window (swizzled layouts)
     unsigned char *smem_raw = smem_unaligned +
         ((1024u - (static_cast<unsigned>(__cvta_generic_to_shared(smem_unaligned)) & 1023u)) & 1023u);
-    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + size_t(T::RAW_STAGES + T::TAIL_STAGES) * T::STAGE_BYTES);   // [2][BM]
+    int64_t *rowA = reinterpret_cast<int64_t *>(smem_raw + size_t(T::RAW_STAGES) * T::STAGE_BYTES + size_t(T::TAIL_STAGES) * T::TAIL_BYTES);   // [2][BM]
     int64_t *colB = rowA + 2 * T::BM;                                    // [2][BN]
     int64_t *colD = colB + 2 * T::BN;                                    // [2][BN]
     int64_t *koffA = colD + 2 * T::BN;
@@ -357,13 +389,15 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         }
     } else if (warp < T::EPILOGUE_WARPS + T::CONVERTER_WARPS) {
         // ------------------------------------------------------------- converters
-        const int ct = tid - T::EPILOGUE_THREADS;
+        const int ct = (tid - T::EPILOGUE_THREADS) % T::CONVERTER_THREADS;
+        const int group = (tid - T::EPILOGUE_THREADS) / T::CONVERTER_THREADS;
         bool ok = true;
         int g = 0;                                   // stage counter across tiles
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x) {
 #pragma unroll 1
             for (int kt = 0; kt < num_kt; ++kt, ++g) {
+                if (T::CONVERTER_GROUPS > 1 && g % T::CONVERTER_GROUPS != group) continue;   // another group's stage
                 const int s = g % T::RAW_STAGES, t = g % T::TAIL_STAGES;
                 if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(g / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait) ||
                     (g >= T::TAIL_STAGES &&
@@ -371,10 +405,35 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     ok = false;
                     break;
                 }
-                const unsigned src = raw0 + unsigned(s) * T::STAGE_BYTES + unsigned(ct) * 16u;
-                const unsigned dst = tail0 + unsigned(t) * T::STAGE_BYTES + unsigned(ct) * 16u;
+                const unsigned raw_stage = raw0 + unsigned(s) * T::STAGE_BYTES;
+                if (T::A_TMEM) {
+                    // M-side operand: this thread owns row ct of the tile = lane ct of tensor memory.
+                    // It reads the row's 32 k from the raw tile (both layouts give conflict-free
+                    // reads with consecutive lanes on consecutive rows), and writes the raw values
+                    // (head: the tensor core ignores the low 13 bits) and the tails to the stage's
+                    // 32 + 32 tensor-memory columns.
+                    float x[32], lo[32];
+                    if (p.dirA == 1) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                         : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
+                                         : "r"(raw_stage + piece_kmajor<T::BM>(ct, 4 * c)) : "memory");
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x[k]) : "r"(raw_stage + piece_mnmajor<T::BM>(ct, k)) : "memory");
+                    }
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) lo[k] = x[k] - __uint_as_float(__float_as_uint(x[k]) & 0xffffe000u);
+                    const unsigned ta = tmem_base + (unsigned(ct & ~31) << 16) + unsigned(2 * T::ACC_COLS + t * T::A_COLS);
+                    tmem_store32(ta, x);
+                    tmem_store32(ta + 32u, lo);
+                }
+                const unsigned src = raw_stage + (T::A_TMEM ? T::A_BYTES : 0) + unsigned(ct) * 16u;
+                const unsigned dst = tail0 + unsigned(t) * T::TAIL_BYTES + unsigned(ct) * 16u;
                 constexpr unsigned STEP = 16u * T::CONVERTER_THREADS;
-                constexpr int CHUNK = T::PIECES % 8 == 0 ? 8 : T::PIECES % 7 == 0 ? 7 : 4;   // loads in flight per thread
+                constexpr int CHUNK = T::PIECES % 8 == 0 ? 8 : T::PIECES % 7 == 0 ? 7 : T::PIECES % 6 == 0 ? 6 : 4;   // loads in flight per thread
                 static_assert(T::PIECES % CHUNK == 0, "pieces must divide into chunks");
 #pragma unroll
                 for (int i0 = 0; i0 < T::PIECES; i0 += CHUNK) {
@@ -391,13 +450,17 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                         asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + unsigned(i0 + i) * STEP), "f"(lo[0]), "f"(lo[1]), "f"(lo[2]), "f"(lo[3]) : "memory");
                     }
                 }
+                if (T::A_TMEM) {
+                    tmem_store_wait();           // the operand columns are written ...
+                    tc_fence_before();           // ... and ordered before the arrival below
+                }
                 proxy_fence_async();             // the tensor core reads both stages through the async proxy
                 mbar_arrive(tail_full0 + 8u * t);
             }
         }
     } else if (warp < T::MMA_WARP) {
         // ------------------------------------------------------------- producers
-        const int pt = tid - T::EPILOGUE_THREADS - T::CONVERTER_THREADS;
+        const int pt = tid - T::EPILOGUE_THREADS - 32 * T::CONVERTER_WARPS;
         bool ok = true;
         int g = 0, n = 0;
 #pragma unroll 1
@@ -439,7 +502,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         constexpr unsigned IDESC_MK = umma_instr_desc(T::BN, true, false);
         constexpr unsigned IDESC_KM = umma_instr_desc(T::BN, false, true);
         constexpr unsigned IDESC_MM = umma_instr_desc(T::BN, true, true);
-        const bool a_mn = p.dirA == 0, b_mn = p.dirB == 0;
+        const bool a_mn = !T::A_TMEM && p.dirA == 0, b_mn = p.dirB == 0;   // an operand in tensor memory is K-major
         const unsigned idesc = a_mn ? (b_mn ? IDESC_MM : IDESC_MK) : (b_mn ? IDESC_KM : IDESC_KK);
         // per operand: layout type, leading / stride byte offsets, start advance of one k-step (8 k)
         const unsigned a_lay = a_mn ? 1u : 2u, a_lbo = a_mn ? 512u : 16u, a_sbo = a_mn ? 16u * T::BM : 1024u;
@@ -466,16 +529,24 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 tc_fence_after();
                 if (leader) {
                     const unsigned a_hi = raw0 + unsigned(s) * T::STAGE_BYTES, b_hi = a_hi + T::A_BYTES;
-                    const unsigned a_lo = tail0 + unsigned(t) * T::STAGE_BYTES, b_lo = a_lo + T::A_BYTES;
+                    const unsigned a_lo = tail0 + unsigned(t) * T::TAIL_BYTES, b_lo = a_lo + T::TAIL_B_OFFSET;
+                    const unsigned ta = tmem_base + unsigned(2 * T::ACC_COLS + t * T::A_COLS);   // head columns, tail 32 further
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint64_t dah = umma_smem_desc(a_hi + j * a_step, a_lbo, a_sbo, a_lay);
-                        const uint64_t dal = umma_smem_desc(a_lo + j * a_step, a_lbo, a_sbo, a_lay);
                         const uint64_t dbh = umma_smem_desc(b_hi + j * b_step, b_lbo, b_sbo, b_lay);
                         const uint64_t dbl = umma_smem_desc(b_lo + j * b_step, b_lbo, b_sbo, b_lay);
-                        umma_tf32(tacc, dal, dbh, idesc, (kt > 0 || j > 0) ? 1u : 0u);
-                        umma_tf32(tacc, dah, dbl, idesc, 1u);
-                        umma_tf32(tacc, dah, dbh, idesc, 1u);
+                        const unsigned acc_in = (kt > 0 || j > 0) ? 1u : 0u;
+                        if (T::A_TMEM) {
+                            umma_tf32_ts(tacc, ta + 32u + 8u * j, dbh, idesc, acc_in);
+                            umma_tf32_ts(tacc, ta + 8u * j, dbl, idesc, 1u);
+                            umma_tf32_ts(tacc, ta + 8u * j, dbh, idesc, 1u);
+                        } else {
+                            const uint64_t dah = umma_smem_desc(a_hi + j * a_step, a_lbo, a_sbo, a_lay);
+                            const uint64_t dal = umma_smem_desc(a_lo + j * a_step, a_lbo, a_sbo, a_lay);
+                            umma_tf32(tacc, dal, dbh, idesc, acc_in);
+                            umma_tf32(tacc, dah, dbl, idesc, 1u);
+                            umma_tf32(tacc, dah, dbh, idesc, 1u);
+                        }
                     }
                     umma_commit(raw_empty0 + 8u * s);    // fire when these MMAs have read the stages
                     umma_commit(tail_empty0 + 8u * t);

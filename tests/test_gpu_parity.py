@@ -212,7 +212,7 @@ def test_unaligned_base_pointer_falls_back_to_element_copies(api, handle):
     assert worst <= 1.0
 
 
-@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(13)]
+@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(17)]
                          + [(torch.complex128, v) for v in range(3)] + [(torch.complex64, v) for v in range(2)])
 def test_every_tile_variant(api, handle, dtype, variant):
     """Each tile variant of the tiled kernels, forced through the attribute, on a ragged multi-tile case
@@ -234,7 +234,7 @@ def test_every_tile_variant(api, handle, dtype, variant):
     assert worst <= 1.0
 
 
-@pytest.mark.parametrize("variant", [10, 11, 12])
+@pytest.mark.parametrize("variant", [10, 11, 12, 13, 14, 15, 16])
 def test_persistent_tensor_memory_kernel_walks_many_tiles(api, handle, variant):
     """The tcgen05 kernels are persistent: with more tiles than SMs every CTA takes several tiles in
     turn, re-using both accumulators, the stage rings and the double-buffered offset arrays.  Ragged
@@ -247,7 +247,7 @@ def test_persistent_tensor_memory_kernel_walks_many_tiles(api, handle, variant):
     worst, status, _ = helpers.run_case(handle, A, "kiz", B, "zkj", C, D, "ijz", 0.75, 1.5, kernel=api.KERNEL_TILED,
                                         variant=variant, want_status=True)
     assert worst <= 1.0 and status["kernel"] == api.KERNEL_TILED
-    bn = {10: 96, 11: 128, 12: 256}[variant]
+    bn = {10: 96, 11: 128, 12: 256, 13: 96, 14: 128, 15: 96, 16: 128}[variant]
     assert status["grid"][0] < -(-ext["i"] // 128) * -(-ext["j"] // bn) * ext["z"]   # fewer CTAs than tiles
 
 
