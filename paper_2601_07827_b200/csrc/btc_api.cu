@@ -281,12 +281,13 @@ int finish_plan(btc_contraction_s *op)
     int variant = 0;
     {
         struct Cand { int id; double weight; };
-        // The tcgen05 variants 10-12 keep all of K in one CTA and have a longer prologue: they
+        // The tcgen05 variants (10-16; candidates: 128x256 with both operands in shared memory,
+        // 128x128 and 128x96 with the M side through tensor memory) keep all of K in one CTA and have a longer prologue: they
         // enter only when there is enough work to fill the SMs without split-K; their weights
         // reflect measured throughput relative to the mma.sync variants.
         const double flops = 2.0 * double(pl.M) * double(pl.N) * double(pl.K) * double(pl.Bt);
         const bool umma_ok = pl.dtype == BTC_F32 && flops >= 2e9 && pl.K >= 64;
-        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {11, 1.8}, {10, 1.7}};
+        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {14, 2.3}, {13, 2.0}};
         const Cand f64c[] = {{2, 1.0}, {1, 0.75}};       // big tile: the m16n8k16 variant
         const Cand c64c[] = {{2, 1.0}, {1, 0.75}};       // complex128: big tile on m16n8k16 as well
         const Cand other[] = {{0, 1.0}, {1, 0.75}};

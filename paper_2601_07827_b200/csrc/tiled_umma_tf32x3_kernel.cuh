@@ -393,18 +393,26 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         const int group = (tid - T::EPILOGUE_THREADS) / T::CONVERTER_THREADS;
         bool ok = true;
         int g = 0;                                   // stage counter across tiles
+        long long t_raw = 0, t_tail = 0, t_work = 0;
+        (void)t_raw; (void)t_tail; (void)t_work;
+        BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x) {
 #pragma unroll 1
             for (int kt = 0; kt < num_kt; ++kt, ++g) {
                 if (T::CONVERTER_GROUPS > 1 && g % T::CONVERTER_GROUPS != group) continue;   // another group's stage
                 const int s = g % T::RAW_STAGES, t = g % T::TAIL_STAGES;
-                if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(g / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait) ||
-                    (g >= T::TAIL_STAGES &&
-                     !mbar_wait_bounded(tail_empty0 + 8u * t, unsigned(g / T::TAIL_STAGES - 1) & 1u, abort_flag, p.error_word, kErrTailEmptyWait))) {
+                if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(g / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait)) {
                     ok = false;
                     break;
                 }
+                BTC_PHASE_END(t_raw);
+                if (g >= T::TAIL_STAGES &&
+                    !mbar_wait_bounded(tail_empty0 + 8u * t, unsigned(g / T::TAIL_STAGES - 1) & 1u, abort_flag, p.error_word, kErrTailEmptyWait)) {
+                    ok = false;
+                    break;
+                }
+                BTC_PHASE_END(t_tail);
                 const unsigned raw_stage = raw0 + unsigned(s) * T::STAGE_BYTES;
                 if (T::A_TMEM) {
                     // M-side operand: this thread owns row ct of the tile = lane ct of tensor memory.
@@ -456,8 +464,12 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 }
                 proxy_fence_async();             // the tensor core reads both stages through the async proxy
                 mbar_arrive(tail_full0 + 8u * t);
+                BTC_PHASE_END(t_work);
             }
         }
+        BTC_PHASE_STORE(p, ct == 0 && group == 0, 0, t_raw);
+        BTC_PHASE_STORE(p, ct == 0 && group == 0, 1, t_tail);
+        BTC_PHASE_STORE(p, ct == 0 && group == 0, 2, t_work);
     } else if (warp < T::MMA_WARP) {
         // ------------------------------------------------------------- producers
         const int pt = tid - T::EPILOGUE_THREADS - 32 * T::CONVERTER_WARPS;
@@ -511,12 +523,16 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         const bool leader = elect_one();
         bool ok = true;
         int g = 0, n = 0;
+        long long t_acc = 0, t_full = 0, t_issue = 0;
+        (void)t_acc; (void)t_full; (void)t_issue;
+        BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x, ++n) {
             const int buf = n & 1;
             if (n >= 2 &&
                 !mbar_wait_bounded(accum_empty0 + 8u * buf, unsigned((n >> 1) - 1) & 1u, abort_flag, p.error_word, kErrAccumWait))
                 break;
+            BTC_PHASE_END(t_acc);
             tc_fence_after();
             const unsigned tacc = tmem_base + unsigned(buf * T::ACC_COLS);
 #pragma unroll 1
@@ -526,6 +542,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     ok = false;
                     break;
                 }
+                BTC_PHASE_END(t_full);
                 tc_fence_after();
                 if (leader) {
                     const unsigned a_hi = raw0 + unsigned(s) * T::STAGE_BYTES, b_hi = a_hi + T::A_BYTES;
@@ -553,8 +570,12 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     if (kt + 1 == num_kt) umma_commit(accum_full0 + 8u * buf);
                 }
                 __syncwarp();
+                BTC_PHASE_END(t_issue);
             }
         }
+        BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 4, t_full);
+        BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 5, t_issue);
+        BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 6, t_acc);
         tc_fence_before();
     }
 
