@@ -202,6 +202,17 @@ enum {
 btc_error_t btc_status_get(btc_status_t status, int32_t key, void *value, size_t len);
 btc_error_t btc_destroy_status(btc_status_t *status);
 
+/* Self-test of the device-side failure detection (no counterpart in the paper).  Every wait inside
+ * the kernels is bounded: after a fixed number of polls it gives up, records a code in the
+ * operation's device error word (BTC_ATTR_DEVICE_ERROR) and lets the kernel return.  This call
+ * launches one small kernel on `cuda_stream` whose 64 threads wait, with a limit of `polls`
+ * (1..65536) polls, on a barrier that nothing ever signals, waits for it, and reports through
+ * *error_code the code the wait recorded (non-zero) and through *threads_gave_up how many
+ * threads gave up (64).  Nothing faults or traps; the CUDA context stays usable.  Allocates and
+ * frees 8 bytes of device memory. */
+btc_error_t btc_selftest_bounded_wait(btc_handle_t handle, void *cuda_stream, int32_t polls,
+                                      int32_t *error_code, int32_t *threads_gave_up);
+
 /* Text for an error code (the strerror analogue of Sec. "Error Handling").  Writes at most `len`
  * bytes including the terminator; *needed (if not NULL) receives the full length. */
 btc_error_t btc_explain_error(btc_error_t code, char *buf, size_t len, size_t *needed);

@@ -49,7 +49,7 @@ EXPORTED = [
     "btc_create_contraction", "btc_destroy_contraction", "btc_contraction_workspace_size",
     "btc_set_attr", "btc_get_attr", "btc_execute", "btc_execute_host", "btc_execute_static_scratch",
     "btc_status_get",
-    "btc_destroy_status", "btc_explain_error",
+    "btc_destroy_status", "btc_explain_error", "btc_selftest_bounded_wait",
 ]
 
 _vp = ctypes.c_void_p
@@ -71,8 +71,18 @@ _lib.btc_execute_static_scratch.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _
 _lib.btc_status_get.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t]
 _lib.btc_destroy_status.argtypes = [ctypes.POINTER(_vp)]
 _lib.btc_explain_error.argtypes = [ctypes.c_int, ctypes.c_char_p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
+_lib.btc_selftest_bounded_wait.argtypes = [_vp, _vp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32),
+                                           ctypes.POINTER(ctypes.c_int32)]
 for _name in EXPORTED:
     getattr(_lib, _name).restype = ctypes.c_int
+
+
+def selftest_bounded_wait(handle, stream: int = 0, polls: int = 1000):
+    """Runs the device-side bounded-wait self-test; returns (error code recorded, threads that gave up)."""
+    code, count = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(_lib.btc_selftest_bounded_wait(handle._h, stream or None, polls, ctypes.byref(code), ctypes.byref(count)),
+           "btc_selftest_bounded_wait")
+    return code.value, count.value
 
 
 def explain_error(code: int) -> str:

@@ -908,6 +908,29 @@ btc_error_t btc_execute_static_scratch(btc_contraction_t op, void *cuda_stream, 
     return btc_execute(op, cuda_stream, alpha, A, B, beta, C, D, scratch, size_t(BTC_STATIC_SCRATCH_BYTES), nullptr);
 }
 
+btc_error_t btc_selftest_bounded_wait(btc_handle_t handle, void *cuda_stream, int32_t polls, int32_t *error_code,
+                                      int32_t *threads_gave_up)
+{
+    if (!handle || !error_code || !threads_gave_up || polls < 1 || polls > 65536) return BTC_ERR_INVALID_ARGUMENT;
+    if (handle->device < 0) return BTC_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int *words = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&words), 2 * sizeof(int)) != cudaSuccess) { cudaGetLastError(); return BTC_ERR_OUT_OF_MEMORY; }
+    btc_error_t rc = BTC_SUCCESS;
+    int host[2] = {0, 0};
+    if (cudaMemsetAsync(words, 0, 2 * sizeof(int), st) != cudaSuccess) rc = BTC_ERR_CUDA;
+    if (rc == BTC_SUCCESS) {
+        bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(unsigned(polls), words, words + 1);
+        if (cudaGetLastError() != cudaSuccess) rc = BTC_ERR_CUDA;
+    }
+    if (rc == BTC_SUCCESS && (cudaMemcpyAsync(host, words, sizeof host, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+                              cudaStreamSynchronize(st) != cudaSuccess)) { cudaGetLastError(); rc = BTC_ERR_CUDA; }
+    cudaFree(words);
+    *error_code = host[0];
+    *threads_gave_up = host[1];
+    return rc;
+}
+
 btc_error_t btc_status_get(btc_status_t status, int32_t key, void *value, size_t len)
 {
     if (!status || !value) return BTC_ERR_INVALID_ARGUMENT;

@@ -59,19 +59,36 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
 }
 
 constexpr unsigned kWaitPollLimit = 1u << 22;   // polls before a wait gives up (a poll itself blocks briefly)
-constexpr int kErrFullWait = 1, kErrEmptyWait = 2;
+constexpr int kErrFullWait = 1, kErrEmptyWait = 2, kErrSelfTest = 7;
 
 // Bounded wait.  Returns false when it gave up or another warp raised the abort flag.
 __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, volatile int *abort_flag,
-                                                  int *error_word, int code)
+                                                  int *error_word, int code, unsigned poll_limit = kWaitPollLimit)
 {
-    for (unsigned n = 0; n < kWaitPollLimit; ++n) {
+    for (unsigned n = 0; n < poll_limit; ++n) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((n & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1;
     if (error_word) atomicCAS(error_word, 0, code);
     return false;
+}
+
+// Self-test of the bounded wait: every thread waits on an mbarrier that nobody arrives on, with a
+// small poll limit.  The wait must give up, raise the abort flag and write the error word; the
+// kernel then returns normally, so the context stays usable.
+__global__ void bounded_wait_selftest_kernel(unsigned poll_limit, int *error_word, int *gave_up_count)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    const unsigned b = static_cast<unsigned>(__cvta_generic_to_shared(&bar));
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        abort_flag = 0;
+    }
+    __syncthreads();
+    const bool done = mbar_wait_bounded(b, 0u, &abort_flag, error_word, kErrSelfTest, poll_limit);
+    if (!done) atomicAdd(gave_up_count, 1);
 }
 
 template <int REGS> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS)); }

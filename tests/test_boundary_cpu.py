@@ -175,3 +175,4 @@ def test_execute_without_device_fails_loudly(api, handle):
     p = ctypes.addressof(buf)
     assert _code(api, lambda: op.execute(0, p, p, 0, p)) == api.ERR_CUDA
     assert _code(api, lambda: op.execute_host(0, p, p, 0, p)) == api.ERR_CUDA
+    assert _code(api, lambda: api.selftest_bounded_wait(handle)) == api.ERR_CUDA

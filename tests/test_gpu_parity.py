@@ -287,3 +287,17 @@ def test_case4_isolated_labels_are_summed_first(api, handle, name, dtype):
     if name == "x_slowest_in_A":
         worst, _, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, 1.0, conjA=cplx, conjB=cplx, host_path=True)
         assert worst <= 1.0
+
+
+def test_bounded_wait_gives_up_and_the_context_stays_usable(api, handle):
+    """Failure detection on the device: a wait on a barrier that nothing signals must run out of
+    polls, record its code and let the kernel return; afterwards the same context still computes."""
+    code, gave_up = api.selftest_bounded_wait(handle, torch.cuda.current_stream().cuda_stream, polls=500)
+    assert code == 7 and gave_up == 64
+    torch.cuda.synchronize()
+    ext = dict(i=70, j=45, k=40)
+    A = helpers.random_tensor(101, _ext("ik", ext), None, torch.float64)
+    B = helpers.random_tensor(102, _ext("kj", ext), None, torch.float64)
+    D = inputs.place(None, _ext("ij", ext), None, torch.float64)
+    worst, _, _ = helpers.run_case(handle, A, "ik", B, "kj", None, D, "ij")
+    assert worst <= 1.0
