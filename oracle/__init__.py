@@ -20,6 +20,10 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "contract_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle_contract.so")
+_SRC_EW = os.path.join(_HERE, "elementwise_oracle.c")
+_LIB_EW = os.path.join(_HERE, "liboracle_elementwise.so")
+ERR_B_C_MISMATCH = 4      # elementwise oracle: B does not have C's rank / extents / labels
+ERR_C_ALIASING = 5        # elementwise oracle: elements of C alias
 
 OK = 0
 ERR_INVALID_ARGUMENT = 1
@@ -55,16 +59,21 @@ class _Tensor(ctypes.Structure):
     ]
 
 
-def build(force: bool = False) -> str:
-    """Compile the C oracle into a shared library next to its source (gcc, OpenMP)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        tmp = _LIB + f".tmp{os.getpid()}"
+def _compile(src: str, lib: str, force: bool) -> str:
+    if force or not os.path.exists(lib) or os.path.getmtime(lib) < os.path.getmtime(src):
+        tmp = lib + f".tmp{os.getpid()}"
         subprocess.run(
-            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"],
+            ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, src, "-lm"],
             check=True,
         )
-        os.replace(tmp, _LIB)
-    return _LIB
+        os.replace(tmp, lib)
+    return lib
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracles into shared libraries next to their sources (gcc, OpenMP)."""
+    _compile(_SRC_EW, _LIB_EW, force)
+    return _compile(_SRC, _LIB, force)
 
 
 _lib = None
@@ -170,6 +179,74 @@ def contract(A: np.ndarray, labelsA, B: np.ndarray, labelsB,
         ctypes.byref(tB) if tB is not None else None,
         ctypes.byref(tC) if tC is not None else None,
         ctypes.byref(tD),
+        al.ctypes.data, be.ctypes.data, int(bool(native_acc)),
+        n_eval if want_arr is not None else 0,
+        want_arr.ctypes.data if want_arr is not None else None,
+        out_val.ctypes.data if out_val is not None else None,
+        scale.ctypes.data if scale is not None else None,
+    )
+    if rc != OK:
+        raise OracleError(rc)
+    if want_arr is not None:
+        return out_val, scale
+    return scale
+
+
+_lib_ew = None
+
+
+def _load_ew():
+    global _lib_ew
+    if _lib_ew is None:
+        build()
+        lib = ctypes.CDLL(_LIB_EW)
+        lib.ore_elementwise.restype = ctypes.c_int
+        lib.ore_elementwise.argtypes = [
+            ctypes.c_int, ctypes.POINTER(_Tensor), ctypes.POINTER(_Tensor), ctypes.POINTER(_Tensor),
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+            ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+        ]
+        _lib_ew = lib
+    return _lib_ew
+
+
+def elementwise(A: np.ndarray, labelsA, B: Optional[np.ndarray], C: np.ndarray, labelsC,
+                alpha=1.0, beta=0.0, *, conjA=False, conjB=False, native_acc=False,
+                want: Optional[Sequence[int]] = None, with_scale=True, layouts: Optional[dict] = None):
+    """Evaluate C := alpha * op(A) + beta * op(B) (Sec. "Unary and Binary Operations"): labels
+    only in A are summed over, A is broadcast along labels only in C, B carries C's labels.
+
+    Same conventions as ``contract``: without ``want`` C is overwritten in place and the flat
+    per-element error scale is returned; with ``want`` ``(values, scale)`` of those elements is
+    returned and C's memory is left alone."""
+    lib = _load_ew()
+    dt = np.dtype(C.dtype)
+    if dt not in _DTYPE_CODE:
+        raise OracleError(ERR_NOT_SUPPORTED)
+    for t in (A, B):
+        if t is not None and t.dtype != dt:
+            raise OracleError(ERR_NOT_SUPPORTED)
+    layouts = layouts or {}
+    keep: list = []
+    tA = _describe(A, labelsA, conjA, keep, *layouts.get("A", (None, None)))
+    tB = _describe(B, labelsC, conjB, keep, *layouts.get("B", (None, None)))
+    tC = _describe(C, labelsC, False, keep, *layouts.get("C", (None, None)))
+    al = np.array([alpha], dtype=dt)
+    be = np.array([beta], dtype=dt)
+    n_eval = 1
+    for e in (layouts["C"][0] if "C" in layouts else C.shape):
+        n_eval *= int(e)
+    want_arr = None
+    out_val = None
+    if want is not None:
+        want_arr = np.ascontiguousarray(np.asarray(want, dtype=np.int64)).reshape(-1)
+        n_eval = want_arr.size
+        if n_eval == 0:
+            want_arr = np.zeros(1, dtype=np.int64)
+        out_val = np.empty(max(n_eval, 1), dtype=dt)[:n_eval]
+    scale = np.empty(max(n_eval, 1), dtype=np.float64)[:n_eval] if with_scale else None
+    rc = lib.ore_elementwise(
+        _DTYPE_CODE[dt], ctypes.byref(tA), ctypes.byref(tB) if tB is not None else None, ctypes.byref(tC),
         al.ctypes.data, be.ctypes.data, int(bool(native_acc)),
         n_eval if want_arr is not None else 0,
         want_arr.ctypes.data if want_arr is not None else None,
