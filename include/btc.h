@@ -202,6 +202,43 @@ enum {
 btc_error_t btc_status_get(btc_status_t status, int32_t key, void *value, size_t len);
 btc_error_t btc_destroy_status(btc_status_t *status);
 
+/* ---- Binary and unary operations (Sec. "Unary and Binary Operations") --------------------------
+ *
+ *     C := alpha * op(A) + beta * op(B)
+ *
+ * B and C carry the same labels (labelsC; B has C's rank and extents, its strides are its own).
+ * A label in A and C is matched; a label only in A is summed over (reduction); along a label only
+ * in C the value of A is repeated (broadcast); a label repeated inside A addresses its
+ * (semi-)diagonal elements (one mode whose stride is the sum of the occurrences' strides, Note 6).
+ * Unary scaling / permutation B := alpha A is the case beta = 0 (pass B = NULL).  op conjugates
+ * complex operands when the flag is set.  All tensors share one element type.
+ *
+ * btc_create_elementwise validates (extents per label, B against C, no repeated label and no
+ * aliasing inside C) and plans once; btc_elementwise_execute takes device pointers (each the
+ * address of logical element (0,...,0)), host scalars (NULL = the values given at creation) and a
+ * CUDA stream, allocates nothing and does not synchronise.  beta == 0: B is not read; alpha == 0:
+ * A is not read.  B may be the same memory as C only with identical strides (in place).
+ * Errors: BTC_ERR_EXTENT_MISMATCH, BTC_ERR_C_D_MISMATCH (B does not match C), BTC_ERR_D_ALIASING
+ * (elements of C alias), BTC_ERR_NOT_SUPPORTED (label repeated in C, mixed types),
+ * BTC_ERR_MISALIGNED, BTC_ERR_CUDA. */
+typedef struct btc_elementwise_s *btc_elementwise_t;
+btc_error_t btc_create_elementwise(btc_handle_t handle,
+                                   btc_tensor_info_t A, const int64_t *labelsA, int conjA,
+                                   btc_tensor_info_t B, int conjB,
+                                   btc_tensor_info_t C, const int64_t *labelsC,
+                                   const void *alpha, const void *beta, btc_elementwise_t *out);
+btc_error_t btc_destroy_elementwise(btc_elementwise_t *op);
+btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, const void *alpha, const void *A,
+                                    const void *beta, const void *B, void *C);
+enum {
+    BTC_EW_ATTR_KERNEL = 1,    /* int32, read: 1 = one thread (or warp) per element of C, 2 = 32 x 32
+                                  tiles through shared memory (input and output contiguous along
+                                  different labels)                                              */
+    BTC_EW_ATTR_NUM_MODES = 2  /* int32[2], read: loop dimensions over C and summed dimensions after
+                                  merging                                                        */
+};
+btc_error_t btc_elementwise_get_attr(btc_elementwise_t op, int32_t key, void *value, size_t len, size_t *needed);
+
 /* Self-test of the device-side failure detection (no counterpart in the paper).  Every wait inside
  * the kernels is bounded: after a fixed number of polls it gives up, records a code in the
  * operation's device error word (BTC_ATTR_DEVICE_ERROR) and lets the kernel return.  This call

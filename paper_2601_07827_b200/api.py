@@ -50,6 +50,7 @@ EXPORTED = [
     "btc_set_attr", "btc_get_attr", "btc_execute", "btc_execute_host", "btc_execute_static_scratch",
     "btc_status_get",
     "btc_destroy_status", "btc_explain_error", "btc_selftest_bounded_wait",
+    "btc_create_elementwise", "btc_destroy_elementwise", "btc_elementwise_execute", "btc_elementwise_get_attr",
 ]
 
 _vp = ctypes.c_void_p
@@ -71,6 +72,11 @@ _lib.btc_execute_static_scratch.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _
 _lib.btc_status_get.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t]
 _lib.btc_destroy_status.argtypes = [ctypes.POINTER(_vp)]
 _lib.btc_explain_error.argtypes = [ctypes.c_int, ctypes.c_char_p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
+_lib.btc_create_elementwise.argtypes = [_vp, _vp, _i64p, ctypes.c_int, _vp, ctypes.c_int, _vp, _i64p, _vp, _vp,
+                                        ctypes.POINTER(_vp)]
+_lib.btc_destroy_elementwise.argtypes = [ctypes.POINTER(_vp)]
+_lib.btc_elementwise_execute.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.btc_elementwise_get_attr.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
 _lib.btc_selftest_bounded_wait.argtypes = [_vp, _vp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32),
                                            ctypes.POINTER(ctypes.c_int32)]
 for _name in EXPORTED:
@@ -291,6 +297,62 @@ def dtype_code(torch_dtype) -> int:
         import torch
         _TORCH_DTYPE = {torch.float32: F32, torch.float64: F64, torch.complex64: C32, torch.complex128: C64}
     return _TORCH_DTYPE[torch_dtype]
+
+
+EW_ATTR_KERNEL, EW_ATTR_NUM_MODES = 1, 2
+EW_KERNEL_DIRECT, EW_KERNEL_TRANSPOSING = 1, 2
+
+
+class Elementwise:
+    """C := alpha op(A) + beta op(B); B (a TensorInfo or None) carries C's labels."""
+
+    def __init__(self, handle: Handle, A: "TensorInfo", labelsA, B: Optional["TensorInfo"], C: "TensorInfo", labelsC,
+                 alpha=1.0, beta=0.0, conjA=False, conjB=False):
+        self.dtype = C.dtype
+        la, lc = _labels(labelsA), _labels(labelsC)
+        self._op = _vp()
+        _check(_lib.btc_create_elementwise(
+            handle._h, A._t, (ctypes.c_int64 * max(len(la), 1))(*la), int(conjA), B._t if B is not None else None,
+            int(conjB), C._t, (ctypes.c_int64 * max(len(lc), 1))(*lc), _scalar(self.dtype, alpha),
+            _scalar(self.dtype, beta), ctypes.byref(self._op)), "btc_create_elementwise")
+        self._keepalive = (handle, A, B, C)
+
+    def _get(self, key, n):
+        buf = (ctypes.c_int32 * n)()
+        _check(_lib.btc_elementwise_get_attr(self._op, key, buf, ctypes.sizeof(buf), None), "btc_elementwise_get_attr")
+        return list(buf)
+
+    @property
+    def kernel(self) -> int:
+        return self._get(EW_ATTR_KERNEL, 1)[0]
+
+    @property
+    def num_modes(self):
+        return tuple(self._get(EW_ATTR_NUM_MODES, 2))
+
+    def execute(self, stream: int, A: int, B: Optional[int], C: int, alpha=None, beta=None) -> None:
+        _check(_lib.btc_elementwise_execute(self._op, stream or None, _scalar(self.dtype, alpha), A or None,
+                                            _scalar(self.dtype, beta), B or None, C or None), "btc_elementwise_execute")
+
+    def close(self):
+        if self._op:
+            _lib.btc_destroy_elementwise(ctypes.byref(self._op))
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def elementwise(handle: Handle, A, labelsA, B, C, labelsC, alpha=1.0, beta=0.0, conjA=False, conjB=False, stream: int = 0):
+    """One-shot helper like ``contract`` for tensors with .dtype, .extents, .strides, .data_ptr()."""
+    tA = TensorInfo(handle, dtype_code(A.dtype), A.extents, A.strides)
+    tB = TensorInfo(handle, dtype_code(B.dtype), B.extents, B.strides) if B is not None else None
+    tC = TensorInfo(handle, dtype_code(C.dtype), C.extents, C.strides)
+    op = Elementwise(handle, tA, labelsA, tB, tC, labelsC, alpha, beta, conjA, conjB)
+    op.execute(stream, A.data_ptr(), B.data_ptr() if B is not None else 0, C.data_ptr())
+    return op
 
 
 def contract(handle: Handle, A, labelsA, B, labelsB, C, D, labelsD, alpha=1.0, beta=0.0,

@@ -18,6 +18,7 @@
 #include "tiled_tf32x3_kernel.cuh"
 #include "tiled_umma_tf32x3_kernel.cuh"
 #include "isolated_sum_kernel.cuh"
+#include "elementwise_kernels.cuh"
 
 using namespace btc;
 
@@ -61,6 +62,13 @@ struct btc_contraction_s {
     size_t sumB_offset = 0, partials_offset = 0;
     // memory spans of the caller's tensors in elements (the plan may describe A' and B' instead)
     int64_t spanA_lo = 0, spanA_hi = 0, spanB_lo = 0, spanB_hi = 0, spanD_lo = 0, spanD_hi = 0;
+};
+
+struct btc_elementwise_s {
+    btc_handle_s handle;
+    ElementwiseRequest req;
+    ElementwisePlan plan;
+    double alpha[2] = {1.0, 0.0}, beta[2] = {0.0, 0.0};
 };
 
 namespace {
@@ -906,6 +914,137 @@ btc_error_t btc_execute_static_scratch(btc_contraction_t op, void *cuda_stream, 
     // Every consumer thread of every CTA overwrites all of its partial sums before the reduction
     // kernel reads them, so nothing in the array has to start at zero.
     return btc_execute(op, cuda_stream, alpha, A, B, beta, C, D, scratch, size_t(BTC_STATIC_SCRATCH_BYTES), nullptr);
+}
+
+// ---- binary / unary operation -------------------------------------------------------------------
+btc_error_t btc_create_elementwise(btc_handle_t handle, btc_tensor_info_t A, const int64_t *labelsA, int conjA,
+                                   btc_tensor_info_t B, int conjB, btc_tensor_info_t C, const int64_t *labelsC,
+                                   const void *alpha, const void *beta, btc_elementwise_t *out)
+{
+    if (!handle || !A || !C || !out) return BTC_ERR_INVALID_ARGUMENT;
+    if ((!labelsA && !A->desc.extent.empty()) || (!labelsC && !C->desc.extent.empty())) return BTC_ERR_INVALID_ARGUMENT;
+    btc_elementwise_s *op = new (std::nothrow) btc_elementwise_s;
+    if (!op) return BTC_ERR_OUT_OF_MEMORY;
+    op->handle = *handle;
+    op->req.A = A->desc;
+    op->req.C = C->desc;
+    op->req.has_b = B != nullptr;
+    if (B) op->req.B = B->desc;
+    op->req.labelsA.assign(labelsA, labelsA + A->desc.extent.size());
+    op->req.labelsC.assign(labelsC, labelsC + C->desc.extent.size());
+    op->req.conjA = conjA != 0;
+    op->req.conjB = conjB != 0;
+    if (alpha) to_double2(C->desc.dtype, alpha, op->alpha);
+    if (beta) to_double2(C->desc.dtype, beta, op->beta);
+    int rc = (!B && !is_zero(op->beta)) ? int(BTC_ERR_INVALID_ARGUMENT) : make_elementwise_plan(op->req, op->plan);
+    if (rc == BTC_SUCCESS && (op->plan.keep.size() > size_t(kGenericMaxD) || op->plan.sum.size() > size_t(kGenericMaxD)))
+        rc = BTC_ERR_NOT_SUPPORTED;
+    if (rc != BTC_SUCCESS) {
+        delete op;
+        return btc_error_t(rc);
+    }
+    *out = op;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_destroy_elementwise(btc_elementwise_t *op)
+{
+    if (!op) return BTC_ERR_INVALID_ARGUMENT;
+    delete *op;
+    *op = nullptr;
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_elementwise_get_attr(btc_elementwise_t op, int32_t key, void *value, size_t len, size_t *needed)
+{
+    if (!op) return BTC_ERR_INVALID_ARGUMENT;
+    int32_t i32[2];
+    size_t n = 0;
+    switch (key) {
+    case BTC_EW_ATTR_KERNEL: i32[0] = int32_t(op->plan.kernel); n = 4; break;
+    case BTC_EW_ATTR_NUM_MODES: i32[0] = int32_t(op->plan.keep.size()); i32[1] = int32_t(op->plan.sum.size()); n = 8; break;
+    default: return BTC_ERR_INVALID_ARGUMENT;
+    }
+    if (needed) *needed = n;
+    if (!value) return needed ? BTC_SUCCESS : BTC_ERR_INVALID_ARGUMENT;
+    if (len < n) return BTC_ERR_INVALID_ARGUMENT;
+    std::memcpy(value, i32, n);
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, const void *alpha, const void *A,
+                                    const void *beta, const void *B, void *C)
+{
+    if (!op || !C) return BTC_ERR_INVALID_ARGUMENT;
+    if (op->handle.device < 0) return BTC_ERR_CUDA;
+    const ElementwisePlan &pl = op->plan;
+    double al[2] = {op->alpha[0], op->alpha[1]}, be[2] = {op->beta[0], op->beta[1]};
+    if (alpha) to_double2(pl.dtype, alpha, al);
+    if (beta) to_double2(pl.dtype, beta, be);
+    const bool use_a = !is_zero(al), use_b = !is_zero(be);
+    if ((use_a && !A) || (use_b && (!B || !pl.has_b))) return BTC_ERR_INVALID_ARGUMENT;
+    const size_t part = dtype_is_complex(pl.dtype) ? dtype_size(pl.dtype) / 2 : dtype_size(pl.dtype);
+    auto misaligned = [&](const void *q) { return q && (reinterpret_cast<uintptr_t>(q) % part) != 0; };
+    if (misaligned(A) || misaligned(B) || misaligned(C)) return BTC_ERR_MISALIGNED;
+    ElementwiseParams p;
+    std::memset(&p, 0, sizeof p);
+    p.A = A; p.B = B; p.C = C;
+    p.nk = int32_t(pl.keep.size()); p.ns = int32_t(pl.sum.size());
+    p.total_keep = pl.total_keep; p.total_sum = pl.total_sum;
+    for (int i = 0; i < p.nk; ++i) {
+        const Mode &m = pl.keep[size_t(i)];
+        p.ext_k[i] = m.extent; p.sA_k[i] = m.sA; p.sB_k[i] = m.sB; p.sC_k[i] = m.sD;
+    }
+    int64_t min_sum = INT64_MAX, min_keep = INT64_MAX;
+    for (int i = 0; i < p.ns; ++i) {
+        p.ext_s[i] = pl.sum[size_t(i)].extent; p.sA_s[i] = pl.sum[size_t(i)].sA;
+        min_sum = std::min<int64_t>(min_sum, std::llabs(p.sA_s[i]));
+    }
+    for (int i = 0; i < p.nk; ++i)
+        if (p.sA_k[i] != 0) min_keep = std::min<int64_t>(min_keep, std::llabs(p.sA_k[i]));
+    p.alpha[0] = al[0]; p.alpha[1] = al[1]; p.beta[0] = be[0]; p.beta[1] = be[1];
+    p.conjA = pl.conjA; p.conjB = pl.conjB;
+    p.use_a = use_a; p.use_b = use_b;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const bool narrow = pl.total_keep < (int64_t(1) << 31) && pl.total_sum < (int64_t(1) << 31);
+    const bool transposing = pl.kernel == ElementwiseKernel::TRANSPOSING && use_a;
+#define BTC_EW_LAUNCH(R, CPLX)                                                                                     \
+    do {                                                                                                           \
+        if (transposing) {                                                                                         \
+            if (narrow) elementwise_transposing_kernel<R, CPLX, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);     \
+            else elementwise_transposing_kernel<R, CPLX, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);             \
+        } else if (lanes == 32) {                                                                                  \
+            if (narrow) elementwise_direct_kernel<R, CPLX, 32, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);      \
+            else elementwise_direct_kernel<R, CPLX, 32, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);              \
+        } else {                                                                                                   \
+            if (narrow) elementwise_direct_kernel<R, CPLX, 1, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);       \
+            else elementwise_direct_kernel<R, CPLX, 1, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);               \
+        }                                                                                                          \
+    } while (0)
+    int lanes = 1;
+    int64_t blocks = 1;
+    if (transposing) {
+        p.tile_mode_a = pl.tile_mode_a;
+        p.tiles_c = int32_t((p.ext_k[0] + 31) / 32);
+        p.tiles_a = int32_t((p.ext_k[pl.tile_mode_a] + 31) / 32);
+        p.rest = pl.total_keep / (p.ext_k[0] * p.ext_k[pl.tile_mode_a]);
+        blocks = int64_t(p.tiles_c) * p.tiles_a * p.rest;
+        if (blocks > 0x7fffffffLL) return BTC_ERR_NOT_SUPPORTED;
+    } else {
+        lanes = (use_a && p.ns > 0 && min_sum < min_keep && pl.total_sum >= 32) ? 32 : 1;
+        blocks = (pl.total_keep * lanes + 255) / 256;
+        const int64_t cap = int64_t(op->handle.sm_count) * 32;
+        if (blocks > cap) blocks = cap;
+        if (blocks < 1) blocks = 1;
+    }
+    switch (pl.dtype) {
+    case BTC_F32: BTC_EW_LAUNCH(float, false); break;
+    case BTC_F64: BTC_EW_LAUNCH(double, false); break;
+    case BTC_C32: BTC_EW_LAUNCH(float, true); break;
+    default: BTC_EW_LAUNCH(double, true); break;
+    }
+#undef BTC_EW_LAUNCH
+    return cudaGetLastError() == cudaSuccess ? BTC_SUCCESS : BTC_ERR_CUDA;
 }
 
 btc_error_t btc_selftest_bounded_wait(btc_handle_t handle, void *cuda_stream, int32_t polls, int32_t *error_code,

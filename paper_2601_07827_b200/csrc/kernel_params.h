@@ -31,6 +31,23 @@ struct IsolatedSumParams {
     int64_t ext_k[kGenericMaxD], str_k[kGenericMaxD], ext_i[kGenericMaxD], str_i[kGenericMaxD];
 };
 
+// C := alpha op(A) + beta op(B): loop dimensions over C (extent, element strides in A, B, C; A's
+// stride is 0 where A is broadcast), first entry fastest, and the dimensions summed over in A.
+struct ElementwiseParams {
+    const void *A, *B;
+    void *C;
+    int32_t nk, ns;
+    int64_t total_keep, total_sum;
+    int64_t ext_k[kGenericMaxD], sA_k[kGenericMaxD], sB_k[kGenericMaxD], sC_k[kGenericMaxD];
+    int64_t ext_s[kGenericMaxD], sA_s[kGenericMaxD];
+    int32_t tile_mode_a;              // transposing kernel: the dimension A is read along (C: dimension 0)
+    int32_t tiles_c, tiles_a;         // transposing kernel: 32-element tiles along those two dimensions
+    int64_t rest;                     // transposing kernel: product of the other dimensions' extents
+    double alpha[2], beta[2];
+    int32_t conjA, conjB;
+    int32_t use_a, use_b;
+};
+
 // Tiled contraction kernels.  All offsets are in elements of the operation's dtype.
 struct TiledParams {
     const void *A, *B, *C;

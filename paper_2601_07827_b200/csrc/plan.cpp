@@ -423,6 +423,84 @@ void split_isolated(const PlanRequest &req, PlanRequest &inner, IsolatedSum &sum
     one(req.B, req.labelsB, req.labelsA, inner.B, inner.labelsB, sumB);
 }
 
+int make_elementwise_plan(const ElementwiseRequest &req, ElementwisePlan &plan)
+{
+    const TensorDesc &A = req.A, &C = req.C;
+    if (A.extent.size() != A.stride.size() || A.extent.size() != req.labelsA.size() ||
+        C.extent.size() != C.stride.size() || C.extent.size() != req.labelsC.size())
+        return BTC_ERR_INVALID_ARGUMENT;
+    if (A.dtype != C.dtype || (req.has_b && req.B.dtype != C.dtype)) return BTC_ERR_NOT_SUPPORTED;
+    for (size_t i = 0; i < C.extent.size(); ++i)
+        for (size_t j = 0; j < i; ++j)
+            if (req.labelsC[i] == req.labelsC[j]) return BTC_ERR_NOT_SUPPORTED;   // would write a diagonal of C only
+    if (req.has_b) {
+        if (req.B.extent.size() != C.extent.size()) return BTC_ERR_C_D_MISMATCH;
+        for (size_t i = 0; i < C.extent.size(); ++i)
+            if (req.B.extent[i] != C.extent[i]) return BTC_ERR_C_D_MISMATCH;
+    }
+    if (d_may_alias(C)) return BTC_ERR_D_ALIASING;
+
+    plan = ElementwisePlan();
+    plan.dtype = C.dtype;
+    plan.has_b = req.has_b;
+    plan.conjA = req.conjA && dtype_is_complex(C.dtype);
+    plan.conjB = req.conjB && dtype_is_complex(C.dtype);
+    struct Row { int64_t label; Mode m; };
+    std::vector<Row> keep, sum;
+    for (size_t i = 0; i < C.extent.size(); ++i) {
+        Mode m;
+        m.extent = C.extent[i];
+        m.sD = C.stride[i];
+        m.sB = req.has_b ? req.B.stride[i] : 0;
+        keep.push_back({req.labelsC[i], m});
+    }
+    for (size_t i = 0; i < A.extent.size(); ++i) {
+        std::vector<Row> *where = &sum;
+        size_t k = 0;
+        for (k = 0; k < keep.size(); ++k)
+            if (keep[k].label == req.labelsA[i]) { where = &keep; break; }
+        if (where == &sum) {
+            for (k = 0; k < sum.size(); ++k)
+                if (sum[k].label == req.labelsA[i]) break;
+            if (k == sum.size()) {
+                Mode m;
+                m.extent = A.extent[i];
+                sum.push_back({req.labelsA[i], m});
+            }
+        }
+        if ((*where)[k].m.extent != A.extent[i]) return BTC_ERR_EXTENT_MISMATCH;
+        (*where)[k].m.sA += A.stride[i];       // repeated labels add their strides (Note 6)
+    }
+    for (auto &r : keep) if (r.m.extent > 1) plan.keep.push_back(r.m);
+    for (auto &r : sum) if (r.m.extent > 1) plan.sum.push_back(r.m);
+    fuse_modes(plan.keep);
+    fuse_modes(plan.sum);
+    std::stable_sort(plan.keep.begin(), plan.keep.end(), [](const Mode &x, const Mode &y) { return iabs(x.sD) < iabs(y.sD); });
+    std::stable_sort(plan.sum.begin(), plan.sum.end(), [](const Mode &x, const Mode &y) { return iabs(x.sA) < iabs(y.sA); });
+    plan.total_keep = product(plan.keep);
+    plan.total_sum = product(plan.sum);
+    span_of(req.A, plan.spanA_lo, plan.spanA_hi);
+    if (req.has_b) span_of(req.B, plan.spanB_lo, plan.spanB_hi);
+    span_of(req.C, plan.spanC_lo, plan.spanC_hi);
+
+    // When A is read far more contiguously along another dimension than along the one C is
+    // written along, go through shared-memory tiles: read along A's dimension, write along C's.
+    plan.kernel = ElementwiseKernel::DIRECT;
+    if (plan.keep.size() >= 2 && plan.keep[0].extent >= 8) {
+        int best = -1;
+        for (size_t i = 1; i < plan.keep.size(); ++i)
+            if (plan.keep[i].sA != 0 && plan.keep[i].extent >= 8 &&
+                (best < 0 || iabs(plan.keep[i].sA) < iabs(plan.keep[size_t(best)].sA)))
+                best = int(i);
+        const int64_t s0 = iabs(plan.keep[0].sA);
+        if (best >= 0 && s0 != 0 && iabs(plan.keep[size_t(best)].sA) * 4 <= s0) {
+            plan.kernel = ElementwiseKernel::TRANSPOSING;
+            plan.tile_mode_a = best;
+        }
+    }
+    return BTC_SUCCESS;
+}
+
 std::string Plan::describe() const
 {
     std::ostringstream o;

@@ -93,6 +93,32 @@ struct IsolatedSum {
 // input without isolated labels is passed through), and how to form A' and B'.
 void split_isolated(const PlanRequest &req, PlanRequest &inner, IsolatedSum &sumA, IsolatedSum &sumB);
 
+// ---- binary / unary operation  C := alpha op(A) + beta op(B)  (Sec. "Unary and Binary Operations")
+struct ElementwiseRequest {
+    TensorDesc A, B, C;
+    bool has_b = false;
+    std::vector<int64_t> labelsA, labelsC;   // B carries C's labels
+    bool conjA = false, conjB = false;
+};
+
+enum class ElementwiseKernel : int32_t { DIRECT = 1, TRANSPOSING = 2 };
+
+struct ElementwisePlan {
+    btc_dtype_t dtype = BTC_F64;
+    bool conjA = false, conjB = false, has_b = false;
+    // loop dimensions over C (labels of C; sA = 0 where A is broadcast), smallest |stride in C|
+    // first, and the summed dimensions (labels only in A; only sA is used), smallest |sA| first
+    std::vector<Mode> keep, sum;
+    int64_t total_keep = 1, total_sum = 1;
+    ElementwiseKernel kernel = ElementwiseKernel::DIRECT;
+    int32_t tile_mode_a = 0;      // TRANSPOSING: index in `keep` of the dimension along which A is read
+                                  // (C is written along dimension 0)
+    int64_t spanA_lo = 0, spanA_hi = 0, spanB_lo = 0, spanB_hi = 0, spanC_lo = 0, spanC_hi = 0;
+};
+
+// Validates the request and fills `plan`.  Returns a btc_error_t.
+int make_elementwise_plan(const ElementwiseRequest &req, ElementwisePlan &plan);
+
 size_t dtype_size(btc_dtype_t t);
 bool dtype_is_complex(btc_dtype_t t);
 

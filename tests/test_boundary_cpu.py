@@ -176,3 +176,20 @@ def test_execute_without_device_fails_loudly(api, handle):
     assert _code(api, lambda: op.execute(0, p, p, 0, p)) == api.ERR_CUDA
     assert _code(api, lambda: op.execute_host(0, p, p, 0, p)) == api.ERR_CUDA
     assert _code(api, lambda: api.selftest_bounded_wait(handle)) == api.ERR_CUDA
+
+
+def test_elementwise_planning_without_a_device(api, handle):
+    """Validation, merging and kernel choice of C := alpha op(A) + beta op(B) are host work."""
+    t = lambda e, s=None: api.TensorInfo(handle, api.F32, e, s)
+    same = api.Elementwise(handle, t((64, 32, 16)), "abc", t((64, 32, 16)), t((64, 32, 16)), "abc", 1.0, 1.0)
+    assert same.kernel == api.EW_KERNEL_DIRECT and same.num_modes == (1, 0)       # everything chains into one loop
+    perm = api.Elementwise(handle, t((64, 32, 16)), "abc", None, t((16, 64, 32)), "cab")
+    assert perm.kernel == api.EW_KERNEL_TRANSPOSING and perm.num_modes == (2, 0)   # (a, b) chain in both tensors
+    red = api.Elementwise(handle, t((64, 5, 32)), "axb", None, t((64, 32)), "ab")
+    assert red.kernel == api.EW_KERNEL_DIRECT and red.num_modes == (2, 1)
+    assert _code(api, lambda: api.Elementwise(handle, t((3, 4)), "ij", None, t((4, 5)), "ji")) == api.ERR_EXTENT_MISMATCH
+    assert _code(api, lambda: api.Elementwise(handle, t((3, 4)), "ij", None, t((4, 3), (1, 2)), "ji")) == api.ERR_D_ALIASING
+    if not __import__("torch").cuda.is_available():
+        buf = (ctypes.c_float * 64 * 32 * 16)()
+        p = ctypes.addressof(buf)
+        assert _code(api, lambda: same.execute(0, p, p, p)) == api.ERR_CUDA
