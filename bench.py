@@ -270,9 +270,64 @@ def small_problem_latency(step, stream, torch):
             "graph_replay_us": graph, "calls": {"single": 200, "back_to_back": 1000, "graph": 1000}}
 
 
+def run_elementwise(args, w):
+    """`--workload ew...`: one step = one C := alpha op(A) + beta op(B) over device-resident tensors;
+    reported as GB/s of algorithmic bytes against the measured HBM bandwidth."""
+    import torch
+    from paper_2601_07827_b200 import build, inputs
+    build.build()
+    from paper_2601_07827_b200 import api
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    A, B, C = inputs.make_elementwise_tensors(w, device="cuda")
+    handle = api.Handle()
+    dt = api.dtype_code(C.dtype)
+    tA = api.TensorInfo(handle, dt, A.extents, A.strides)
+    tC = api.TensorInfo(handle, dt, C.extents, C.strides)
+    tB = api.TensorInfo(handle, dt, B.extents, B.strides) if B is not None else None
+    op = api.Elementwise(handle, tA, w.labelsA, tB, tC, w.labelsC, w.alpha, w.beta)
+    stream = torch.cuda.current_stream()
+    pB = B.data_ptr() if B is not None else 0
+
+    def step():
+        op.execute(stream.cuda_stream, A.data_ptr(), pB, C.data_ptr())
+    for _ in range(max(1, args.warmup)):
+        step()
+    sampler = ClockSampler(0)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    gbs = w.algorithmic_bytes() / (ms * 1e-3) / 1e9
+    peak, src = measured_hbm_gbs()
+    print(json.dumps({
+        "metric": "elementwise GB/s", "value": gbs, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "labels": [w.labelsA, w.labelsC], "kernel": op.kernel, "num_modes": list(op.num_modes),
+                   "l2": "tensors exceed L2"},
+        "clocks": clocks, "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
+                     "peak_source": f"STREAM-style copy, {src}",
+                     "kernel": "elementwise_transposing_kernel" if op.kernel == 2 else "elementwise_direct_kernel",
+                     "kernel_ms": ms}}))
+
+
 def main():
     args = parse()
     from paper_2601_07827_b200 import inputs
+    if args.workload in inputs.elementwise_workloads():
+        if args.impl == "reference":
+            raise SystemExit("the reference arm times the contraction oracle only")
+        run_elementwise(args, inputs.elementwise_workloads()[args.workload])
+        return
     w = inputs.workloads()[args.workload]
     if args.impl == "reference":
         run_reference(args, w)

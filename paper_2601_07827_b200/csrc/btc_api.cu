@@ -1023,10 +1023,41 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
     } while (0)
     int lanes = 1;
     int64_t blocks = 1;
+    // 16-byte vectors along dimension 0 when nothing is summed and that dimension is contiguous in
+    // every tensor in use, with all other strides and the base pointers keeping 16-byte alignment
+    const int vec = int(16 / dtype_size(pl.dtype));
+    bool vector_ok = !transposing && p.ns == 0 && p.nk >= 1 && vec > 1 && p.ext_k[0] % vec == 0 && p.sC_k[0] == 1 &&
+                     (!use_a || p.sA_k[0] == 1) && (!use_b || p.sB_k[0] == 1) &&
+                     reinterpret_cast<uintptr_t>(C) % 16 == 0 && (!use_a || reinterpret_cast<uintptr_t>(A) % 16 == 0) &&
+                     (!use_b || reinterpret_cast<uintptr_t>(B) % 16 == 0);
+    for (int i = 1; vector_ok && i < p.nk; ++i)
+        vector_ok = p.sC_k[i] % vec == 0 && (!use_a || p.sA_k[i] % vec == 0) && (!use_b || p.sB_k[i] % vec == 0);
+    if (vector_ok) {
+        blocks = (pl.total_keep / vec + 255) / 256;
+        const int64_t cap = int64_t(op->handle.sm_count) * 32;
+        if (blocks > cap) blocks = cap;
+        if (blocks < 1) blocks = 1;
+        switch (pl.dtype) {
+        case BTC_F32:
+            if (narrow) elementwise_vector_kernel<float, false, 4, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);
+            else elementwise_vector_kernel<float, false, 4, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);
+            break;
+        case BTC_F64:
+            if (narrow) elementwise_vector_kernel<double, false, 2, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);
+            else elementwise_vector_kernel<double, false, 2, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);
+            break;
+        default:   // complex64: two elements per 16 bytes (complex128 has vec == 1)
+            if (narrow) elementwise_vector_kernel<float, true, 2, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);
+            else elementwise_vector_kernel<float, true, 2, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);
+            break;
+        }
+        return cudaGetLastError() == cudaSuccess ? BTC_SUCCESS : BTC_ERR_CUDA;
+    }
     if (transposing) {
+        const int T = dtype_size(pl.dtype) == 4 ? 64 : 32;
         p.tile_mode_a = pl.tile_mode_a;
-        p.tiles_c = int32_t((p.ext_k[0] + 31) / 32);
-        p.tiles_a = int32_t((p.ext_k[pl.tile_mode_a] + 31) / 32);
+        p.tiles_c = int32_t((p.ext_k[0] + T - 1) / T);
+        p.tiles_a = int32_t((p.ext_k[pl.tile_mode_a] + T - 1) / T);
         p.rest = pl.total_keep / (p.ext_k[0] * p.ext_k[pl.tile_mode_a]);
         blocks = int64_t(p.tiles_c) * p.tiles_a * p.rest;
         if (blocks > 0x7fffffffLL) return BTC_ERR_NOT_SUPPORTED;

@@ -104,13 +104,75 @@ __global__ void __launch_bounds__(256) elementwise_direct_kernel(const Elementwi
     }
 }
 
-// blockIdx.x enumerates (tile along C's dimension 0, tile along A's dimension, rest), first fastest;
-// 32 x 8 threads, each 4 elements of the 32 x 32 tile in either phase
+// Nothing summed and dimension 0 contiguous in A, B and C alike: V consecutive elements (16 bytes)
+// per thread, one vector load per input and one vector store.
+template <typename R, bool CPLX, int V, typename I>
+__global__ void __launch_bounds__(256) elementwise_vector_kernel(const ElementwiseParams p)
+{
+    constexpr int NC = CPLX ? 2 : 1;
+    constexpr int W = V * NC;                            // words of type R per vector
+    union Pack { uint4 raw; R w[W]; };
+    static_assert(sizeof(R) * W == 16, "a vector is 16 bytes");
+    const R *A = static_cast<const R *>(p.A);
+    const R *B = static_cast<const R *>(p.B);
+    R *C = static_cast<R *>(p.C);
+    const int64_t nvec = p.total_keep / V;
+    const int64_t stride = int64_t(gridDim.x) * blockDim.x;
+    const R sgnA = (CPLX && p.conjA) ? R(-1) : R(1), sgnB = (CPLX && p.conjB) ? R(-1) : R(1);
+    for (int64_t v = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; v < nvec; v += stride) {
+        int64_t offA = 0, offB = 0, offC = 0;
+        I lin = I(v);
+        {
+            const I ext = I(p.ext_k[0] / V);
+            const I q = lin / ext;
+            const int64_t i = int64_t(lin - q * ext) * V;
+            lin = q;
+            offA = i * p.sA_k[0]; offB = i * p.sB_k[0]; offC = i;
+        }
+        for (int d = 1; d < p.nk; ++d) {
+            const I ext = I(p.ext_k[d]);
+            const I q = lin / ext;
+            const int64_t i = int64_t(lin - q * ext);
+            lin = q;
+            offA += i * p.sA_k[d];
+            offB += i * p.sB_k[d];
+            offC += i * p.sC_k[d];
+        }
+        Pack a, b, c;
+        a.raw = make_uint4(0, 0, 0, 0);
+        b.raw = make_uint4(0, 0, 0, 0);
+        if (p.use_a) a.raw = *reinterpret_cast<const uint4 *>(A + NC * offA);
+        if (p.use_b) b.raw = *reinterpret_cast<const uint4 *>(B + NC * offB);
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+            const double ar = p.use_a ? double(a.w[NC * e]) : 0.0;
+            const double ai = (CPLX && p.use_a) ? double(sgnA * a.w[NC * e + (NC - 1)]) : 0.0;
+            double c_r = p.alpha[0] * ar - p.alpha[1] * ai, c_i = p.alpha[0] * ai + p.alpha[1] * ar;
+            if (p.use_b) {
+                const double br = double(b.w[NC * e]);
+                const double bi = CPLX ? double(sgnB * b.w[NC * e + (NC - 1)]) : 0.0;
+                c_r += p.beta[0] * br - p.beta[1] * bi;
+                c_i += p.beta[0] * bi + p.beta[1] * br;
+            }
+            c.w[NC * e] = R(c_r);
+            if (CPLX) c.w[NC * e + (NC - 1)] = R(c_i);
+        }
+        *reinterpret_cast<uint4 *>(C + NC * offC) = c.raw;
+    }
+}
+
+// blockIdx.x enumerates (tile along C's dimension 0, tile along A's dimension, rest), first fastest.
+// T x T tiles (T = 64 for 4-byte elements, 32 otherwise: rows of at least 256 bytes on both sides),
+// 256 threads, each T * T / 256 elements in either phase; the tile holds values already summed and
+// rounded to the element type.
 template <typename R, bool CPLX, typename I>
 __global__ void __launch_bounds__(256) elementwise_transposing_kernel(const ElementwiseParams p)
 {
     constexpr int NC = CPLX ? 2 : 1;
-    __shared__ double tile[NC][32][33];
+    constexpr int T = (sizeof(R) * NC == 4) ? 64 : 32;
+    constexpr int ROWS = 256 / T;                        // tile rows covered by the CTA at once
+    constexpr int PER = T / ROWS;                        // rows per thread
+    __shared__ R tile[NC][T][T + 1];
     const int ma = p.tile_mode_a;
     const int64_t tile_c = blockIdx.x % p.tiles_c;
     const int64_t tile_a = (blockIdx.x / p.tiles_c) % p.tiles_a;
@@ -124,27 +186,27 @@ __global__ void __launch_bounds__(256) elementwise_transposing_kernel(const Elem
         restB += i * p.sB_k[d];
         restC += i * p.sC_k[d];
     }
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const int64_t c0 = tile_c * 32, a0 = tile_a * 32;
+    const int tx = threadIdx.x % T, ty = threadIdx.x / T;
+    const int64_t c0 = tile_c * T, a0 = tile_a * T;
     const int64_t ext_c = p.ext_k[0], ext_a = p.ext_k[ma];
     // phase 1: consecutive threads along A's dimension
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        const int64_t c = c0 + ty + 8 * r, a = a0 + tx;
+    for (int r = 0; r < PER; ++r) {
+        const int64_t c = c0 + ty + ROWS * r, a = a0 + tx;
         double acc_r = 0.0, acc_i = 0.0;
         if (c < ext_c && a < ext_a)
             elementwise_sum<R, CPLX, 1, I>(p, restA + c * p.sA_k[0] + a * p.sA_k[ma], 0, acc_r, acc_i);
-        tile[0][ty + 8 * r][tx] = acc_r;
-        if (CPLX) tile[NC - 1][ty + 8 * r][tx] = acc_i;
+        tile[0][ty + ROWS * r][tx] = R(acc_r);
+        if (CPLX) tile[NC - 1][ty + ROWS * r][tx] = R(acc_i);
     }
     __syncthreads();
     // phase 2: consecutive threads along C's dimension 0
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        const int64_t c = c0 + tx, a = a0 + ty + 8 * r;
+    for (int r = 0; r < PER; ++r) {
+        const int64_t c = c0 + tx, a = a0 + ty + ROWS * r;
         if (c < ext_c && a < ext_a)
             elementwise_finish<R, CPLX>(p, restB + c * p.sB_k[0] + a * p.sB_k[ma], restC + c * p.sC_k[0] + a * p.sC_k[ma],
-                                        tile[0][tx][ty + 8 * r], CPLX ? tile[NC - 1][tx][ty + 8 * r] : 0.0);
+                                        double(tile[0][tx][ty + ROWS * r]), CPLX ? double(tile[NC - 1][tx][ty + ROWS * r]) : 0.0);
     }
 }
 

@@ -349,6 +349,56 @@ def workloads() -> Dict[str, Workload]:
     return w
 
 
+@dataclasses.dataclass(frozen=True)
+class ElementwiseWorkload:
+    """C[labelsC] := alpha * op(A[labelsA]) + beta * op(B[labelsC]) with dense column-major tensors."""
+    name: str
+    dtype: str
+    labelsA: str
+    labelsC: str
+    extents: Dict[str, int]
+    alpha: complex = 1.0
+    beta: complex = 0.0          # != 0: B is present
+    seed: int = 0
+
+    def ext(self, labels: str) -> Tuple[int, ...]:
+        return tuple(self.extents[l] for l in labels)
+
+    def algorithmic_bytes(self) -> float:
+        """A read once, B read once when beta != 0, C written once."""
+        item = {"f32": 4, "f64": 8, "c32": 8, "c64": 16}[self.dtype]
+        size = lambda ls: math.prod(self.extents[l] for l in ls)
+        return float(item * (size(set(self.labelsA)) + size(self.labelsC) * (2 if self.beta != 0 else 1)))
+
+
+def elementwise_workloads() -> Dict[str, ElementwiseWorkload]:
+    """Bandwidth-bound cases of the binary / unary operation, each about 1-2 GB of traffic."""
+    w = {}
+    # full reversal of a rank-4 tensor: input and output contiguous along different labels
+    w["ew1_f32_permute_reverse"] = ElementwiseWorkload(
+        "ew1_f32_permute_reverse", "f32", "abcd", "dcba", {"a": 256, "b": 64, "c": 64, "d": 256}, seed=7100)
+    # the fast label stays, the others rotate (no transposition needed)
+    w["ew2_f64_permute_keep_fast"] = ElementwiseWorkload(
+        "ew2_f64_permute_keep_fast", "f64", "abcd", "acdb", {"a": 128, "b": 64, "c": 128, "d": 128}, seed=7200)
+    # C = alpha A + beta B, same layout
+    w["ew3_f64_axpby"] = ElementwiseWorkload(
+        "ew3_f64_axpby", "f64", "ab", "ab", {"a": 8192, "b": 8192}, alpha=0.75, beta=-0.5, seed=7300)
+    # reduction over a slow label with a transposition: C[j,i] = sum_x A[i,x,j]
+    w["ew4_f32_reduce_transpose"] = ElementwiseWorkload(
+        "ew4_f32_reduce_transpose", "f32", "ixj", "ji", {"i": 4096, "x": 16, "j": 4096}, seed=7400)
+    return w
+
+
+def make_elementwise_tensors(w: ElementwiseWorkload, device="cpu"):
+    """(A, B, C) as StridedTensor; B is None when beta == 0; C starts as canary NaNs."""
+    dt = DTYPES[w.dtype]
+    eA, eC = w.ext(w.labelsA), w.ext(w.labelsC)
+    A = place(logical_values(w.seed + 1, eA, dt, "uniform", 1.0, device=device), eA, None, dt, device)
+    B = place(logical_values(w.seed + 2, eC, dt, "uniform", 1.0, device=device), eC, None, dt, device) if w.beta != 0 else None
+    C = place(None, eC, None, dt, device)
+    return A, B, C
+
+
 def scaled_down(w: Workload, factors: Dict[str, int], name: Optional[str] = None) -> Workload:
     """Same structure with some extents replaced (parity cases the oracle finishes quickly).
     Explicit strides are rebuilt as column-major with the same relative padding on mode 0."""

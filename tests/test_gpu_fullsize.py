@@ -78,3 +78,29 @@ def test_full_size_sampled(name):
         after = D.buffer.view(width).reshape(D.buffer.numel(), -1)[~touched]
         assert torch.equal(before, after)
         assert not torch.isnan(torch.view_as_real(D.buffer[touched]) if D.buffer.is_complex() else D.buffer[touched]).any()
+
+
+@pytest.mark.parametrize("name", list(inputs.elementwise_workloads()))
+def test_elementwise_full_size_sampled(name):
+    """The bandwidth workloads of the binary / unary operation at the sizes bench.py times: sampled
+    elements of C (random indices plus the first slab) against the oracle's one-by-one evaluation."""
+    api = helpers.api()
+    handle = api.Handle()
+    w = inputs.elementwise_workloads()[name]
+    A, B, C = inputs.make_elementwise_tensors(w, device="cuda")
+    op = api.elementwise(handle, A, w.labelsA, B, C, w.labelsC, w.alpha, w.beta,
+                         stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    total = C.numel()
+    rng = np.random.default_rng(77)
+    want = np.unique(np.concatenate([rng.integers(0, total, size=50000), np.arange(min(65536, total))]))
+    hA = A.to("cpu")
+    hB = B.to("cpu") if B is not None else None
+    c_stub = np.zeros(1, dtype=hA.numpy().dtype)
+    vals, scale = oracle.elementwise(hA.numpy(), w.labelsA, hB.numpy() if hB is not None else None, c_stub, w.labelsC,
+                                     w.alpha, w.beta, want=want, layouts={"C": (C.extents, C.strides)})
+    # C is dense column-major with origin C.origin: the sampled linear indices are buffer positions
+    pos = torch.from_numpy(want + C.origin).to("cuda")
+    got = C.buffer[pos].cpu().numpy()
+    assert helpers.compare(got, vals, scale, C.dtype) <= 1.0
+    assert op.kernel in (api.EW_KERNEL_DIRECT, api.EW_KERNEL_TRANSPOSING)
