@@ -120,7 +120,10 @@ enum {
     BTC_ATTR_NUM_MODES = 6,   /* int32[4], read: modes per class after fusion (batch, M, N, K) */
     BTC_ATTR_SWAPPED = 7,     /* int32, read: 1 when A and B exchanged roles                   */
     BTC_ATTR_VARIANT = 9,     /* int32, read/write: index of the tile variant of the tiled
-                                 kernel for this element type (-1 on write = choose)          */
+                                 kernel for this element type (-1 on write = choose).  A variant
+                                 the operation cannot use (a bulk-tensor-copy variant whose M-side
+                                 tiles are no boxes of the operand) is replaced by its nearest
+                                 equivalent; read back what was planned                       */
     BTC_ATTR_DEVICE_ERROR = 8,/* int32, read: 0, or which bounded device-side wait gave up in an
                                  earlier execute of this operation (its D is then incomplete);
                                  reading waits for the device                                  */
@@ -197,7 +200,10 @@ enum {
     BTC_STATUS_KERNEL = 1,    /* int32: BTC_KERNEL_* that ran                 */
     BTC_STATUS_LAUNCHES = 2,  /* int32: kernels enqueued by the call          */
     BTC_STATUS_GRID = 3,      /* int32[3]                                      */
-    BTC_STATUS_SPLIT_K = 4    /* int32                                         */
+    BTC_STATUS_SPLIT_K = 4,   /* int32                                         */
+    BTC_STATUS_VARIANT = 5    /* int32: tile variant of the tiled kernel that ran (-1: generic kernel); differs
+                                 from BTC_ATTR_VARIANT when a bulk-copy variant met a base pointer that is
+                                 not 16-byte aligned and its gathering twin ran instead */
 };
 btc_error_t btc_status_get(btc_status_t status, int32_t key, void *value, size_t len);
 btc_error_t btc_destroy_status(btc_status_t *status);

@@ -42,7 +42,7 @@ ATTR_DEVICE_ERROR = 8
 ATTR_VARIANT = 9
 ATTR_PRE_REDUCE = 10
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TILED = 0, 1, 2
-STATUS_KERNEL, STATUS_LAUNCHES, STATUS_GRID, STATUS_SPLIT_K = 1, 2, 3, 4
+STATUS_KERNEL, STATUS_LAUNCHES, STATUS_GRID, STATUS_SPLIT_K, STATUS_VARIANT = 1, 2, 3, 4, 5
 
 EXPORTED = [
     "btc_create_handle", "btc_destroy_handle", "btc_create_tensor_info", "btc_destroy_tensor_info",
@@ -255,7 +255,7 @@ class Contraction:
         if want_status:
             out = {}
             for name, key, n in (("kernel", STATUS_KERNEL, 1), ("launches", STATUS_LAUNCHES, 1),
-                                 ("grid", STATUS_GRID, 3), ("split_k", STATUS_SPLIT_K, 1)):
+                                 ("grid", STATUS_GRID, 3), ("split_k", STATUS_SPLIT_K, 1), ("variant", STATUS_VARIANT, 1)):
                 buf = (ctypes.c_int32 * n)()
                 _check(_lib.btc_status_get(st, key, buf, ctypes.sizeof(buf)), "btc_status_get")
                 out[name] = list(buf) if n > 1 else buf[0]

@@ -36,7 +36,7 @@ struct btc_tensor_info_s {
 };
 
 struct btc_status_s {
-    int32_t kernel = 0, launches = 0, split_k = 1;
+    int32_t kernel = 0, launches = 0, split_k = 1, variant = -1;
     int32_t grid[3] = {0, 0, 0};
 };
 
@@ -53,6 +53,9 @@ struct btc_contraction_s {
                   *d_offD_h = nullptr;
     int32_t tiles_m = 0, tiles_n = 0, raster_n_fast = 0;
     int64_t k_per_split = 0;
+    // bulk-tensor-copy variants: the M-side operand as a tensor of boxes, its coordinate tables on the device
+    TmaOperand tmaA;
+    const int32_t *d_tma_coord_m = nullptr, *d_tma_coord_k = nullptr, *d_tma_coord_h = nullptr;
     size_t workspace_bytes = 0;
     int32_t grid[3] = {0, 0, 0};
     // Case 4: inputs with isolated labels are first summed into the front of the workspace
@@ -102,8 +105,14 @@ using F32Umma96T2 = UmmaTile<96, 5, 2, true, 2>;                   // two conver
 using F32Umma128T2 = UmmaTile<128, 4, 2, true, 2>;                              // tcgen05 + tensor memory, 3xTF32
 using F32Umma128 = UmmaTile<128, 4, 2>;
 using F32Umma256 = UmmaTile<256, 3, 1>;
-constexpr int kNumF32Variants = 17;
+// M side fetched by bulk tensor copies (one box per stage), stages of 24 or 32 k
+using F32Umma96B24 = UmmaTile<96, 7, 2, true, 1, 24, true>;
+using F32Umma96B32 = UmmaTile<96, 5, 2, true, 1, 32, true>;
+using F32Umma128B32 = UmmaTile<128, 4, 2, true, 1, 32, true>;
+using F32Umma128B24 = UmmaTile<128, 5, 2, true, 1, 24, true>;
+constexpr int kNumF32Variants = 21;
 constexpr int kFirstUmmaVariant = 10;
+constexpr int kFirstBulkVariant = 17;     // 17..20: bulk tensor copies; fall back to 13 / 14 (same tiles) at execute
 
 struct VariantInfo {
     int bm, bn, bk, threads, acc;
@@ -146,6 +155,10 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
         case 13: return {128, 96, 32, 256, 0, F32Umma96T::SMEM_BYTES, 4};
         case 14: return {128, 128, 32, 256, 0, F32Umma128T::SMEM_BYTES, 4};
         case 15: return {128, 96, 32, 256, 0, F32Umma96T2::SMEM_BYTES, 4};
+        case 17: return {128, 96, 24, 256, 0, F32Umma96B24::SMEM_BYTES, 4};
+        case 18: return {128, 96, 32, 256, 0, F32Umma96B32::SMEM_BYTES, 4};
+        case 19: return {128, 128, 32, 256, 0, F32Umma128B32::SMEM_BYTES, 4};
+        case 20: return {128, 128, 24, 256, 0, F32Umma128B24::SMEM_BYTES, 4};
         default: return {128, 128, 32, 256, 0, F32Umma128T2::SMEM_BYTES, 4};
         }
     }
@@ -199,13 +212,43 @@ cudaError_t launch_tiled_tf32(const TiledParams &p, int64_t ctas, int64_t reduce
 }
 
 template <typename T>
-cudaError_t launch_umma(const TiledParams &p, int64_t ctas, cudaStream_t st)
+cudaError_t launch_umma(const TiledParams &p, int64_t ctas, cudaStream_t st, const CUtensorMap *mapA = nullptr)
 {
     static bool configured[64] = {};
     cudaError_t e = set_smem_once(tiled_umma_tf32x3_kernel<T>, T::SMEM_BYTES, configured);
     if (e != cudaSuccess) return e;
-    tiled_umma_tf32x3_kernel<T><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
+    static const CUtensorMap none = {};
+    tiled_umma_tf32x3_kernel<T><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p, mapA ? *mapA : none);
     return cudaGetLastError();
+}
+
+// Tensor map of the M-side operand for the bulk-copy variants: fp32 elements, the planner's
+// dimensions and box, zero fill outside the tensor, 128-byte swizzle when a box row is 128 bytes
+// of k.  The encoder is a driver entry point looked up once through the runtime (no link-time
+// dependency on the driver library).  False when the driver declines the description.
+bool encode_tma_operand(const TmaOperand &t, const void *base, CUtensorMap *out)
+{
+    using Encode = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static Encode encode = [] {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            fn = nullptr;
+        }
+        return reinterpret_cast<Encode>(fn);
+    }();
+    if (!encode || !t.ok) return false;
+    cuuint64_t dim[5], stride[4];
+    cuuint32_t box[5], estr[5] = {1, 1, 1, 1, 1};
+    for (int d = 0; d < 5; ++d) { dim[d] = t.dim[d]; box[d] = t.box[d]; }
+    for (int d = 1; d < 5; ++d) stride[d - 1] = t.stride[d] * 4;
+    const bool swz = t.k_major && t.box[0] == 32;
+    return encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<void *>(base), dim, stride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <typename T, bool AK, bool BK_>
@@ -295,12 +338,17 @@ int finish_plan(btc_contraction_s *op)
         // reflect measured throughput relative to the mma.sync variants.
         const double flops = 2.0 * double(pl.M) * double(pl.N) * double(pl.K) * double(pl.Bt);
         const bool umma_ok = pl.dtype == BTC_F32 && flops >= 2e9 && pl.K >= 64;
-        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {14, 2.3}, {13, 2.0}};
+        // 17-20 fetch the M side with bulk tensor copies; they enter when that operand is a tensor of boxes
+        TmaOperand probe;
+        const bool box24 = umma_ok && make_tma_operand(pl, 128, 24, probe), box32 = umma_ok && make_tma_operand(pl, 128, 32, probe);
+        // (measured a little behind their gathering twins 13 / 14 on the batched permuted workload, hence the weights)
+        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {14, 2.3}, {13, 2.0},
+                             {box24 ? 17 : 13, 1.85}, {box32 ? 18 : 13, 1.95}, {box32 ? 19 : 14, 2.25}, {box24 ? 20 : 14, 2.1}};
         const Cand f64c[] = {{2, 1.0}, {1, 0.75}};       // big tile: the m16n8k16 variant
         const Cand c64c[] = {{2, 1.0}, {1, 0.75}};       // complex128: big tile on m16n8k16 as well
         const Cand other[] = {{0, 1.0}, {1, 0.75}};
         const Cand *cands = pl.dtype == BTC_F32 ? f32c : (pl.dtype == BTC_F64 ? f64c : (pl.dtype == BTC_C64 ? c64c : other));
-        const int ncand = pl.dtype == BTC_F32 ? (umma_ok ? 7 : 4) : 2;
+        const int ncand = pl.dtype == BTC_F32 ? (umma_ok ? 11 : 4) : 2;
         double best = -1.0;
         for (int c = 0; c < ncand; ++c) {
             const VariantInfo vi = variant_info(pl.dtype, cands[c].id);
@@ -318,6 +366,12 @@ int finish_plan(btc_contraction_s *op)
         const int count = pl.dtype == BTC_F32 ? kNumF32Variants : (pl.dtype == BTC_F64 ? 5 : (pl.dtype == BTC_C64 ? 3 : 2));
         if (op->req.force_variant >= count) return BTC_ERR_INVALID_ARGUMENT;
         variant = op->req.force_variant;
+    }
+    op->tmaA = TmaOperand();
+    if (pl.dtype == BTC_F32 && variant >= kFirstBulkVariant) {
+        // a forced bulk-copy variant whose M-side operand is no tensor of boxes: the gathering twin
+        const VariantInfo bv = variant_info(pl.dtype, variant);
+        if (!make_tma_operand(pl, bv.bm, bv.bk, op->tmaA)) variant = variant <= 18 ? 13 : 14;
     }
     const VariantInfo v = variant_info(pl.dtype, variant);
     pl.tile.bm = v.bm; pl.tile.bn = v.bn; pl.tile.bk = v.bk; pl.tile.threads = v.threads;
@@ -369,7 +423,16 @@ int finish_plan(btc_contraction_s *op)
         for (auto *t : tabs) total += (t->size() + 31) / 32 * 32;   // keep every table 256-byte aligned
         const size_t error_at = total;
         total += 32;                                                  // the error word, zeroed
+        // coordinate tables of the bulk-copy variants (int32), packed behind the error word
+        const std::vector<int32_t> *ctabs[3] = {&op->tmaA.coordM, &op->tmaA.coordK, &op->tmaA.coordH};
+        size_t cstart[3];
+        for (int i = 0; i < 3; ++i) {
+            cstart[i] = total;
+            total += (ctabs[i]->size() + 63) / 64 * 32;
+        }
         std::vector<int64_t> host(total, 0);
+        for (int i = 0; i < 3; ++i)
+            if (!ctabs[i]->empty()) std::memcpy(host.data() + cstart[i], ctabs[i]->data(), ctabs[i]->size() * sizeof(int32_t));
         size_t pos = 0, starts[9];
         for (int i = 0; i < 9; ++i) {
             starts[i] = pos;
@@ -387,6 +450,9 @@ int finish_plan(btc_contraction_s *op)
         }
         for (int i = 0; i < 9; ++i) *dst[i] = op->d_tables + starts[i];
         op->d_error = reinterpret_cast<int32_t *>(op->d_tables + error_at);
+        op->d_tma_coord_m = reinterpret_cast<const int32_t *>(op->d_tables + cstart[0]);
+        op->d_tma_coord_k = reinterpret_cast<const int32_t *>(op->d_tables + cstart[1]);
+        op->d_tma_coord_h = reinterpret_cast<const int32_t *>(op->d_tables + cstart[2]);
     }
     return BTC_SUCCESS;
 }
@@ -694,6 +760,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
     }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     int launches = 0;
+    int ran_variant = op->plan.kernel == BTC_KERNEL_TILED ? op->plan.tile.variant : -1;
     cudaError_t ce = cudaSuccess;
     // Case 4: sum the inputs over their isolated labels first; the contraction then reads A', B'
     if (use_ab && op->sumA.active) {
@@ -765,6 +832,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         tp.alpha[0] = al[0]; tp.alpha[1] = al[1]; tp.beta[0] = be[0]; tp.beta[1] = be[1];
         tp.partials = workspace ? static_cast<char *>(workspace) + op->partials_offset : nullptr;
         tp.error_word = op->d_error;
+        tp.tmaA_coord_m = op->d_tma_coord_m; tp.tmaA_coord_k = op->d_tma_coord_k; tp.tmaA_coord_h = op->d_tma_coord_h;
 #ifdef BTC_STAMPS
         { void *sp = nullptr; cudaGetSymbolAddress(&sp, btc_stamp_buffer); tp.stamps = static_cast<long long *>(sp); }
 #endif
@@ -790,7 +858,21 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
             case 13: ce = launch_umma<F32Umma96T>(tp, ctas, st); break;
             case 14: ce = launch_umma<F32Umma128T>(tp, ctas, st); break;
             case 15: ce = launch_umma<F32Umma96T2>(tp, ctas, st); break;
-            default: ce = launch_umma<F32Umma128T2>(tp, ctas, st); break;
+            case 16: ce = launch_umma<F32Umma128T2>(tp, ctas, st); break;
+            default: {
+                // bulk tensor copies need a 16-byte aligned base and a description the driver accepts;
+                // otherwise the gathering variant with the same tile runs
+                CUtensorMap mapA;
+                const int v = pl.tile.variant;
+                if (misaligned(pA, 16) || !encode_tma_operand(op->tmaA, pA, &mapA)) {
+                    ran_variant = v <= 18 ? 13 : 14;
+                    ce = v <= 18 ? launch_umma<F32Umma96T>(tp, ctas, st) : launch_umma<F32Umma128T>(tp, ctas, st);
+                }
+                else if (v == 17) ce = launch_umma<F32Umma96B24>(tp, ctas, st, &mapA);
+                else if (v == 18) ce = launch_umma<F32Umma96B32>(tp, ctas, st, &mapA);
+                else if (v == 19) ce = launch_umma<F32Umma128B32>(tp, ctas, st, &mapA);
+                else ce = launch_umma<F32Umma128B24>(tp, ctas, st, &mapA);
+            } break;
             }
         } else if (pl.dtype == BTC_C32) {
             ce = pl.tile.variant == 0 ? launch_tiled_tf32<C32Tc>(tp, ctas, reduce_ctas, st)
@@ -815,6 +897,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         if (!s) return BTC_ERR_OUT_OF_MEMORY;
         s->kernel = use_ab ? pl.kernel : BTC_KERNEL_GENERIC;
         s->launches = launches;
+        s->variant = ran_variant;
         s->split_k = pl.split_k;
         s->grid[0] = op->grid[0]; s->grid[1] = op->grid[1]; s->grid[2] = op->grid[2];
         *status = s;
@@ -1109,6 +1192,7 @@ btc_error_t btc_status_get(btc_status_t status, int32_t key, void *value, size_t
     case BTC_STATUS_LAUNCHES: if (len < 4) return BTC_ERR_INVALID_ARGUMENT; std::memcpy(value, &status->launches, 4); break;
     case BTC_STATUS_GRID: if (len < 12) return BTC_ERR_INVALID_ARGUMENT; std::memcpy(value, status->grid, 12); break;
     case BTC_STATUS_SPLIT_K: if (len < 4) return BTC_ERR_INVALID_ARGUMENT; std::memcpy(value, &status->split_k, 4); break;
+    case BTC_STATUS_VARIANT: if (len < 4) return BTC_ERR_INVALID_ARGUMENT; std::memcpy(value, &status->variant, 4); break;
     default: return BTC_ERR_INVALID_ARGUMENT;
     }
     return BTC_SUCCESS;

@@ -372,6 +372,98 @@ int make_plan(const PlanRequest &req, Plan &plan)
     return BTC_SUCCESS;
 }
 
+bool make_tma_operand(const Plan &pl, int bm, int bk, TmaOperand &out)
+{
+    out = TmaOperand();
+    if (pl.m.empty() || pl.k.empty() || dtype_size(pl.dtype) != 4) return false;
+    struct Part { int64_t extent, stride, box; int cls, idx; };       // cls 0: M, 1: K, 2: batch
+    std::vector<Part> parts;
+    int64_t rem = bm;
+    for (size_t i = 0; i < pl.m.size(); ++i) {
+        Part p{pl.m[i].extent, pl.m[i].sA, 1, 0, int(i)};
+        if (rem > 1) {
+            if (rem % p.extent == 0) { p.box = p.extent; rem /= p.extent; }
+            else if (p.extent % rem == 0) { p.box = rem; rem = 1; }
+            else if (pl.m.size() == 1 && p.extent > rem) { p.box = rem; rem = 1; }   // ragged last tile: zero-filled by the copy
+            else return false;
+        }
+        parts.push_back(p);
+    }
+    if (rem != 1) return false;
+    for (size_t i = 0; i < pl.k.size(); ++i) {
+        Part p{pl.k[i].extent, pl.k[i].sA, 1, 1, int(i)};
+        if (i == 0) {
+            if (p.extent % bk != 0 && !(pl.k.size() == 1 && p.extent > bk)) return false;
+            p.box = bk;
+        }
+        parts.push_back(p);
+    }
+    for (size_t i = 0; i < pl.batch.size(); ++i) parts.push_back(Part{pl.batch[i].extent, pl.batch[i].sA, 1, 2, int(i)});
+    for (auto &p : parts)
+        if (p.stride <= 0) return false;
+    const size_t k0 = pl.m.size();
+    if (parts[k0].stride == 1) out.k_major = true;
+    else if (parts[0].stride != 1 || parts[0].box == 1) return false;
+
+    // dimensions: the contiguous one, the other parts of the box in shared-memory order, the rest
+    struct Dim { int64_t extent, stride, box; std::vector<std::pair<size_t, int64_t>> members; };
+    std::vector<Dim> dims;
+    auto add = [&](size_t i) { dims.push_back(Dim{parts[i].extent, parts[i].stride, parts[i].box, {{i, 1}}}); };
+    if (out.k_major) add(k0);
+    for (size_t i = 0; i < pl.m.size(); ++i)
+        if (parts[i].box > 1) add(i);
+    if (!out.k_major) add(k0);
+    for (size_t i = 0; i < parts.size(); ++i)
+        if (parts[i].box == 1) add(i);
+    for (bool changed = true; changed;) {
+        changed = false;
+        for (size_t x = 0; x < dims.size() && !changed; ++x)
+            for (size_t y = 0; y < dims.size() && !changed; ++y) {
+                if (x == y || dims[y].box != 1 || dims[y].stride != dims[x].stride * dims[x].extent) continue;
+                for (auto &mb : dims[y].members) dims[x].members.push_back({mb.first, mb.second * dims[x].extent});
+                dims[x].extent *= dims[y].extent;
+                dims.erase(dims.begin() + y);
+                changed = true;
+            }
+    }
+    if (dims.size() > 5) return false;
+    out.rank = int32_t(dims.size());
+    std::vector<std::pair<int, int64_t>> where(parts.size());        // part -> (dimension, multiplier)
+    for (size_t d = 0; d < dims.size(); ++d) {
+        if (dims[d].extent >= (int64_t(1) << 31) || dims[d].box > 256) return false;
+        if (d > 0 && (dims[d].stride % 4 != 0 || dims[d].stride >= (int64_t(1) << 38))) return false;
+        out.dim[d] = uint64_t(dims[d].extent);
+        out.stride[d] = uint64_t(dims[d].stride);
+        out.box[d] = uint32_t(dims[d].box);
+        for (auto &mb : dims[d].members) where[mb.first] = {int(d), mb.second};
+    }
+    // a bulk copy starts on a 16-byte boundary: along dimension 0 the box and every coordinate
+    // step (the multipliers of the loop dimensions that share it) are multiples of four elements
+    if (out.box[0] % 4 != 0) return false;
+    for (auto &mb : dims[0].members)
+        if (mb.second != 1 && mb.second % 4 != 0) return false;
+    for (size_t d = dims.size(); d < 5; ++d) out.stride[d] = dims.size() > 1 ? out.stride[dims.size() - 1] : 4;   // extent 1: never stepped
+
+    auto coords_of = [&](int cls, const std::vector<Mode> &g, int64_t lin, int32_t *c) {
+        for (int d = 0; d < 5; ++d) c[d] = 0;
+        for (size_t i = 0; i < g.size(); ++i) {
+            const int64_t idx = lin % g[i].extent;
+            lin /= g[i].extent;
+            const size_t part = (cls == 0 ? 0 : (cls == 1 ? k0 : k0 + pl.k.size())) + i;
+            c[where[part].first] += int32_t(idx * where[part].second);
+        }
+    };
+    const int64_t tiles_m = (pl.M + bm - 1) / bm, stages = (pl.K + bk - 1) / bk;
+    out.coordM.resize(size_t(tiles_m) * 5);
+    out.coordK.resize(size_t(stages) * 5);
+    out.coordH.resize(size_t(pl.Bt) * 5);
+    for (int64_t t = 0; t < tiles_m; ++t) coords_of(0, pl.m, t * bm, &out.coordM[size_t(t) * 5]);
+    for (int64_t t = 0; t < stages; ++t) coords_of(1, pl.k, t * bk, &out.coordK[size_t(t) * 5]);
+    for (int64_t t = 0; t < pl.Bt; ++t) coords_of(2, pl.batch, t, &out.coordH[size_t(t) * 5]);
+    out.ok = true;
+    return true;
+}
+
 void split_isolated(const PlanRequest &req, PlanRequest &inner, IsolatedSum &sumA, IsolatedSum &sumB)
 {
     inner = req;

@@ -79,6 +79,26 @@ struct PlanRequest {
 // Validates the request and fills `plan`.  Returns a btc_error_t.
 int make_plan(const PlanRequest &req, Plan &plan);
 
+// The M-side operand seen as a tensor of at most five dimensions in which every (tile of `bm`
+// rows) x (stage of `bk` contracted indices) is one rectangular box, so that a single bulk tensor
+// copy (cp.async.bulk.tensor) can fetch it.  Exists when the tile's rows are whole leading M modes
+// (at most one of them partly), a stage is a whole number of entries of the first contracted
+// mode, the operand is contiguous along the first M mode or the first contracted mode, and all
+// other strides are positive multiples of 16 bytes.  Loop dimensions whose strides chain in this
+// operand share one dimension, which is how the tile index, the stage index and the batch index
+// usually collapse into a few coordinates.
+struct TmaOperand {
+    bool ok = false;
+    bool k_major = false;                 // dimension 0 is the contracted index (else the first M mode)
+    uint64_t dim[5] = {1, 1, 1, 1, 1};    // extents in elements, dimension 0 contiguous
+    uint64_t stride[5] = {1, 0, 0, 0, 0}; // element strides
+    uint32_t box[5] = {1, 1, 1, 1, 1};
+    int32_t rank = 0;                     // dimensions in use (the rest have extent 1)
+    // box origin = coordM[tile of M] + coordK[stage] + coordH[batch entry], five entries each
+    std::vector<int32_t> coordM, coordK, coordH;
+};
+bool make_tma_operand(const Plan &plan, int bm, int bk, TmaOperand &out);
+
 // Case 4: the sum over the labels that occur in one input only, taken before the contraction.
 struct IsolatedSum {
     bool active = false;

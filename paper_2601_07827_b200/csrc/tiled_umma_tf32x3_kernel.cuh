@@ -23,10 +23,16 @@
 //               tile per lane, so a warp's store of one column is 32 consecutive rows of D),
 //               applies alpha / beta through D's offset tables and releases the accumulator,
 //               while the other roles already work on the next tile.
+// A_TMA variants: when every (tile, stage) of the M-side operand is a rectangular box of a tensor
+// of at most five dimensions, one producer thread fetches it with a single bulk tensor copy
+// (cp.async.bulk.tensor, completion counted in bytes on the stage's "raw full" mbarrier) instead of
+// 128 threads issuing 16-byte copies; the box lands row by row (k contiguous) or column by column
+// (rows contiguous) and the converters move it on to tensor memory.  The N side keeps its gather.
 // Every wait is bounded; a wait that gives up raises the CTA abort flag and the error word, all
 // roles fall through to the common tail, and the allocating warp always frees its tensor memory.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "kernel_params.h"
@@ -34,10 +40,16 @@
 
 namespace btc {
 
-template <int BN_, int RAW_STAGES_, int TAIL_STAGES_, bool A_TMEM_ = false, int CONVERTER_GROUPS_ = 1>
+template <int BN_, int RAW_STAGES_, int TAIL_STAGES_, bool A_TMEM_ = false, int CONVERTER_GROUPS_ = 1, int BK_ = 32, bool A_TMA_ = false>
 struct UmmaTile {
-    static constexpr int BM = 128, BN = BN_, BK = 32;
+    static constexpr int BM = 128, BN = BN_, BK = BK_;
+    static constexpr int KSTEPS = BK_ / 8;                           // tensor-core instructions of K = 8 per stage
     static constexpr int RAW_STAGES = RAW_STAGES_, TAIL_STAGES = TAIL_STAGES_;
+    // A_TMA: the M-side tile of a stage arrives by one bulk tensor copy (needs A_TMEM: the box is
+    // not in a layout the tensor core reads, the converters take it to tensor memory)
+    static constexpr bool A_TMA = A_TMA_;
+    static_assert(BK_ == 32 || (BK_ == 24 && A_TMA_), "stages of 24 exist for the bulk-copy variants only");
+    static_assert(!A_TMA_ || A_TMEM_, "the bulk-copy variants pass the M side through tensor memory");
     // A_TMEM: the M-side operand reaches the tensor core through tensor memory (the converters
     // write its head and tail there), so the tensor core reads only the N-side operand from
     // shared memory and a tail stage holds only that operand's tail
@@ -49,8 +61,10 @@ struct UmmaTile {
     static constexpr int PRODUCER_WARPS = 4, PRODUCER_THREADS = 128;
     static constexpr int MMA_WARP = EPILOGUE_WARPS + CONVERTER_WARPS + PRODUCER_WARPS;
     static constexpr int THREADS = 32 * (MMA_WARP + 1);
-    static constexpr int A_BYTES = BM * BK * 4, B_BYTES = BN * BK * 4;
+    // a k-contiguous N-side tile keeps 128-byte rows whatever BK is (the swizzle atom)
+    static constexpr int A_BYTES = BM * BK * 4, B_BYTES = BN * 32 * 4;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;           // a raw stage
+    static_assert(A_BYTES % 1024 == 0, "operand tiles sit on 1024-byte boundaries");
     static constexpr int TAIL_BYTES = A_TMEM_ ? B_BYTES : STAGE_BYTES;
     static constexpr int TAIL_B_OFFSET = A_TMEM_ ? 0 : A_BYTES;     // where the N-side tail sits in a tail stage
     static constexpr int ACC_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;   // one accumulator
@@ -115,7 +129,26 @@ __device__ __forceinline__ void tmem_store32(unsigned taddr, const float (&v)[32
                    "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]), "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
                  : "memory");
 }
+// 8 consecutive columns of this lane's tensor-memory row
+__device__ __forceinline__ void tmem_store8(unsigned taddr, const float *v)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_store_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// one arrival on the barrier plus `bytes` that a bulk copy will report on it
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bulk tensor copy of one box (five coordinates, dimension 0 first) into shared memory; its bytes
+// are reported on `bar`.  Dimension 0's coordinate must be a multiple of four elements.
+__device__ __forceinline__ void tma_load_box(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1, int c2, int c3, int c4)
+{
+    asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+                 ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tmem_load16(unsigned taddr, unsigned (&r)[16])
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -220,26 +253,47 @@ __device__ __forceinline__ void umma_producer_init(UmmaProducerLane<R> &l, const
     }
 }
 
+// The k offsets a producer thread needs for one stage (vector path): at most two look-ups.
+struct UmmaStageOffsets {
+    int64_t kofs0, kofs1;
+    bool in0, in1;
+};
+template <int R, int BK = 32>
+__device__ __forceinline__ UmmaStageOffsets umma_lookup(const UmmaProducerLane<R> &l, const UmmaOperand &o, int64_t k0)
+{
+    UmmaStageOffsets s;
+    const int64_t ka = k0 + l.kq, kb = ka + 16;
+    s.in0 = ka < o.k_end && (BK == 32 || l.kq < BK);
+    s.in1 = o.dir == 0 && kb < o.k_end && l.kq + 16 < BK;
+    s.kofs0 = o.koff[s.in0 ? ka : o.k_begin];
+    s.kofs1 = o.koff[s.in1 ? kb : o.k_begin];
+    return s;
+}
+
 // The copies of one operand for one stage.  Look-ups first, copies after: a copy is an ordered
-// memory operation, so a look-up placed behind one would wait for it.
-template <int R>
-__device__ __forceinline__ void umma_produce(unsigned tile, const UmmaProducerLane<R> &l, const UmmaOperand &o, int64_t k0)
+// memory operation, so a look-up placed behind one would wait for it; the caller therefore looks
+// up a stage's offsets (`so`, vector path) before it issues the copies of the stage before.
+// A stage holds BK <= 32 k: slots whose k lies beyond BK are skipped (their place in the tile is
+// never read by the tensor core).
+template <int R, int BK = 32>
+__device__ __forceinline__ void umma_produce(unsigned tile, const UmmaProducerLane<R> &l, const UmmaOperand &o, int64_t k0,
+                                             const UmmaStageOffsets &so)
 {
     constexpr int SLOTS = UmmaProducerLane<R>::SLOTS;
+    if (BK < 32 && l.kq >= BK) return;
     if (o.vec == 4) {
-        const int64_t ka = k0 + l.kq, kb = ka + 16;
-        const bool in0 = ka < o.k_end, in1 = o.dir == 0 && kb < o.k_end;
-        const int64_t kofs0 = o.koff[in0 ? ka : o.k_begin], kofs1 = o.koff[in1 ? kb : o.k_begin];
 #pragma unroll
         for (int i = 0; i < SLOTS; ++i) {
             const bool second = umma_slot_half<R>(o.dir, i) != 0;
-            const bool valid = ((l.rows_in >> i) & 1u) && (second ? in1 : in0);
-            cp_async_bytes<16>(tile + l.pos0 + umma_slot_pos<R>(o.dir, i), o.g + l.rowoff[i] + (second ? kofs1 : kofs0), valid);
+            if (BK < 32 && second && l.kq + 16 >= BK) continue;
+            const bool valid = ((l.rows_in >> i) & 1u) && (second ? so.in1 : so.in0);
+            cp_async_bytes<16>(tile + l.pos0 + umma_slot_pos<R>(o.dir, i), o.g + l.rowoff[i] + (second ? so.kofs1 : so.kofs0), valid);
         }
     } else {
 #pragma unroll 2
         for (int i = 0; i < SLOTS; ++i) {
             const int row = umma_slot_row<R>(o.dir, l.r0, i);
+            if (BK < 32 && l.kq + 16 * umma_slot_half<R>(o.dir, i) >= BK) continue;
             const int64_t k = k0 + l.kq + 16 * umma_slot_half<R>(o.dir, i);
             int64_t off[4];
             bool in[4];
@@ -282,7 +336,7 @@ __device__ __forceinline__ bool umma_group_sync(unsigned bar, unsigned parity, v
 // walk that list with the same counters.  Tensor memory holds two accumulators, so the epilogue
 // of one tile overlaps the main loop of the next; the shared-memory rings run across tiles.
 template <typename T>
-__global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const TiledParams p)
+__global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const TiledParams p, const __grid_constant__ CUtensorMap tmapA)
 {
     extern __shared__ __align__(16) unsigned char smem_unaligned[];
     // operand tiles must sit on 1024-byte boundaries of the shared-memory window (swizzled layouts)
@@ -311,17 +365,21 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     const int64_t total = int64_t(p.tiles_m) * p.tiles_n * p.Bt;         // split_k == 1 on this path
     const int num_kt = int((p.K + T::BK - 1) / T::BK);
     const bool staged = p.K <= kKoffCap;
+    const bool coords_staged = 5 * num_kt <= 2 * kKoffCap;
 
     // ---- set-up: k offsets, barriers, tensor memory ----
     {
         if (staged)
             for (int i = tid; i < int(p.K); i += T::THREADS) {
-                koffA[i] = p.offA_k[i];
+                if (!T::A_TMA) koffA[i] = p.offA_k[i];
                 koffB[i] = p.offB_k[i];
             }
+        // bulk-copy variants: the stages' box coordinates take the place of the M side's k offsets
+        if (T::A_TMA && coords_staged)
+            for (int i = tid; i < 5 * num_kt; i += T::THREADS) reinterpret_cast<int32_t *>(koffA)[i] = p.tmaA_coord_k[i];
         if (tid == 0) {
             for (int s = 0; s < T::RAW_STAGES; ++s) {
-                mbar_init(raw_full0 + 8u * s, T::PRODUCER_THREADS);
+                mbar_init(raw_full0 + 8u * s, T::PRODUCER_THREADS + (T::A_TMA ? 1 : 0));   // + the bulk copy's issuer
                 mbar_init(raw_empty0 + 8u * s, 1);
             }
             for (int s = 0; s < T::TAIL_STAGES; ++s) {
@@ -334,6 +392,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 mbar_init(producer_sync0 + 8u * b, T::PRODUCER_THREADS);
                 mbar_init(epilogue_sync0 + 8u * b, T::EPILOGUE_THREADS);
             }
+
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
@@ -420,38 +479,74 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     // reads with consecutive lanes on consecutive rows), and writes the raw values
                     // (head: the tensor core ignores the low 13 bits) and the tails to the stage's
                     // 32 + 32 tensor-memory columns.
-                    float x[32], lo[32];
+                    // A bulk-copied box is plain: rows of BK k (k contiguous; 128-byte rows carry
+                    // the copy's 128-byte swizzle, which is the layout of piece_kmajor; 96-byte rows
+                    // are unswizzled and lanes 4-7 of each quarter-warp start one 16-byte chunk
+                    // later so that the quarter's eight reads hit distinct banks), or BK columns of
+                    // 128 rows (rows contiguous).
+                    float x[T::BK], lo[T::BK];
                     if (p.dirA == 1) {
+                        if (T::A_TMA && T::BK != 32) {
+                            constexpr int CH = T::BK / 4;
+                            const int rot = (ct >> 2) & 1;
+                            float y[T::BK];
 #pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                                         : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
-                                         : "r"(raw_stage + piece_kmajor<T::BM>(ct, 4 * c)) : "memory");
+                            for (int c = 0; c < CH; ++c) {
+                                const int cc = c + rot < CH ? c + rot : c + rot - CH;
+                                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                             : "=f"(y[4 * c]), "=f"(y[4 * c + 1]), "=f"(y[4 * c + 2]), "=f"(y[4 * c + 3])
+                                             : "r"(raw_stage + unsigned(ct * (T::BK * 4) + cc * 16)) : "memory");
+                            }
+#pragma unroll
+                            for (int c = 0; c < CH; ++c)       // chunk c was read into slot c - rot
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) x[4 * c + e] = rot ? y[4 * ((c + CH - 1) % CH) + e] : y[4 * c + e];
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < T::BK / 4; ++c)
+                                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                             : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
+                                             : "r"(raw_stage + piece_kmajor<T::BM>(ct, 4 * c)) : "memory");
+                        }
                     } else {
 #pragma unroll
-                        for (int k = 0; k < 32; ++k)
-                            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x[k]) : "r"(raw_stage + piece_mnmajor<T::BM>(ct, k)) : "memory");
+                        for (int k = 0; k < T::BK; ++k)
+                            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x[k])
+                                         : "r"(raw_stage + (T::A_TMA ? unsigned((k * T::BM + ct) * 4) : piece_mnmajor<T::BM>(ct, k))) : "memory");
                     }
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) lo[k] = x[k] - __uint_as_float(__float_as_uint(x[k]) & 0xffffe000u);
+                    for (int k = 0; k < T::BK; ++k) lo[k] = x[k] - __uint_as_float(__float_as_uint(x[k]) & 0xffffe000u);
                     const unsigned ta = tmem_base + (unsigned(ct & ~31) << 16) + unsigned(2 * T::ACC_COLS + t * T::A_COLS);
-                    tmem_store32(ta, x);
-                    tmem_store32(ta + 32u, lo);
+                    if constexpr (T::BK == 32) {
+                        tmem_store32(ta, x);
+                        tmem_store32(ta + 32u, lo);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < T::KSTEPS; ++j) {
+                            tmem_store8(ta + 8u * j, x + 8 * j);
+                            tmem_store8(ta + unsigned(T::BK) + 8u * j, lo + 8 * j);
+                        }
+                    }
                 }
                 const unsigned src = raw_stage + (T::A_TMEM ? T::A_BYTES : 0) + unsigned(ct) * 16u;
                 const unsigned dst = tail0 + unsigned(t) * T::TAIL_BYTES + unsigned(ct) * 16u;
                 constexpr unsigned STEP = 16u * T::CONVERTER_THREADS;
                 constexpr int CHUNK = T::PIECES % 8 == 0 ? 8 : T::PIECES % 7 == 0 ? 7 : T::PIECES % 6 == 0 ? 6 : 4;   // loads in flight per thread
                 static_assert(T::PIECES % CHUNK == 0, "pieces must divide into chunks");
+                // with fewer than 32 k per stage a rows-contiguous N-side tile fills only the front
+                // of its place (whole k atoms); a k-contiguous one is spread over all its 128-byte rows
+                const int pieces_used = (T::BK == 32 || p.dirB == 1) ? T::PIECES * T::CONVERTER_THREADS : T::BN * T::BK / 4;
 #pragma unroll
                 for (int i0 = 0; i0 < T::PIECES; i0 += CHUNK) {
                     float x[CHUNK][4];
 #pragma unroll
                     for (int i = 0; i < CHUNK; ++i)
-                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                                     : "=f"(x[i][0]), "=f"(x[i][1]), "=f"(x[i][2]), "=f"(x[i][3]) : "r"(src + unsigned(i0 + i) * STEP) : "memory");
+                        if (T::BK == 32 || (i0 + i) * T::CONVERTER_THREADS + ct < pieces_used)
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                         : "=f"(x[i][0]), "=f"(x[i][1]), "=f"(x[i][2]), "=f"(x[i][3]) : "r"(src + unsigned(i0 + i) * STEP) : "memory");
 #pragma unroll
                     for (int i = 0; i < CHUNK; ++i) {
+                        if (T::BK != 32 && (i0 + i) * T::CONVERTER_THREADS + ct >= pieces_used) continue;
                         float lo[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) lo[e] = x[i][e] - __uint_as_float(__float_as_uint(x[i][e]) & 0xffffe000u);
@@ -475,6 +570,9 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         const int pt = tid - T::EPILOGUE_THREADS - 32 * T::CONVERTER_WARPS;
         bool ok = true;
         int g = 0, n = 0;
+        long long t_setup = 0, t_empty = 0, t_copy = 0;
+        (void)t_setup; (void)t_empty; (void)t_copy;
+        BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x, ++n) {
             const TileCoords tc = tile_coords_at<T::BM, T::BN, T::BK>(p, work);
@@ -482,7 +580,8 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             int64_t *rA = rowA + buf * T::BM, *cB = colB + buf * T::BN;
             {
                 const int64_t hA = p.offA_h[tc.h], hB = p.offB_h[tc.h];
-                for (int i = pt; i < T::BM; i += T::PRODUCER_THREADS) rA[i] = i < tc.rows_valid ? p.offA_m[tc.m0 + i] + hA : 0;
+                if (!T::A_TMA)
+                    for (int i = pt; i < T::BM; i += T::PRODUCER_THREADS) rA[i] = i < tc.rows_valid ? p.offA_m[tc.m0 + i] + hA : 0;
                 for (int i = pt; i < T::BN; i += T::PRODUCER_THREADS) cB[i] = i < tc.cols_valid ? p.offB_n[tc.n0 + i] + hB : 0;
             }
             if (!umma_group_sync(producer_sync0 + 8u * buf, unsigned(n >> 1) & 1u, abort_flag, p.error_word)) break;
@@ -490,23 +589,53 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             const UmmaOperand opB = {static_cast<const float *>(p.B), cB, staged ? koffB : p.offB_k, tc.cols_valid, 0, p.K, p.dirB, p.vecB};
             UmmaProducerLane<T::BM> la;
             UmmaProducerLane<T::BN> lb;
-            umma_producer_init<T::BM>(la, opA, pt);
+            if (!T::A_TMA) umma_producer_init<T::BM>(la, opA, pt);
             umma_producer_init<T::BN>(lb, opB, pt);
+            int box0[5] = {0, 0, 0, 0, 0};           // bulk copy: the box origin of this tile at stage 0
+            if (T::A_TMA && pt == 0) {
+                const int32_t *cm = p.tmaA_coord_m + (tc.m0 / T::BM) * 5, *ch = p.tmaA_coord_h + tc.h * 5;
+#pragma unroll
+                for (int d = 0; d < 5; ++d) box0[d] = cm[d] + ch[d];
+            }
+            // offsets of the first stage; inside the loop those of the next stage are looked up
+            // before this stage's copies are issued
+            UmmaStageOffsets sa = {0, 0, false, false}, sb = sa, sa_next = sa, sb_next = sa;
+            if (!T::A_TMA && opA.vec == 4) sa_next = umma_lookup<T::BM>(la, opA, 0);
+            if (opB.vec == 4) sb_next = umma_lookup<T::BN, T::BK>(lb, opB, 0);
+            BTC_PHASE_END(t_setup);
 #pragma unroll 1
             for (int kt = 0; kt < num_kt; ++kt, ++g) {
                 const int s = g % T::RAW_STAGES;
+                sa = sa_next; sb = sb_next;
+                if (kt + 1 < num_kt) {
+                    if (!T::A_TMA && opA.vec == 4) sa_next = umma_lookup<T::BM>(la, opA, int64_t(kt + 1) * T::BK);
+                    if (opB.vec == 4) sb_next = umma_lookup<T::BN, T::BK>(lb, opB, int64_t(kt + 1) * T::BK);
+                }
                 if (g >= T::RAW_STAGES &&
                     !mbar_wait_bounded(raw_empty0 + 8u * s, unsigned(g / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait)) {
                     ok = false;
                     break;
                 }
+                BTC_PHASE_END(t_empty);
                 const unsigned st = raw0 + unsigned(s) * T::STAGE_BYTES;
                 const int64_t k0 = int64_t(kt) * T::BK;
-                umma_produce<T::BM>(st, la, opA, k0);
-                umma_produce<T::BN>(st + T::A_BYTES, lb, opB, k0);
+                if (T::A_TMA) {
+                    if (pt == 0) {
+                        const int32_t *ck = (coords_staged ? reinterpret_cast<const int32_t *>(koffA) : p.tmaA_coord_k) + kt * 5;
+                        mbar_arrive_expect_tx(raw_full0 + 8u * s, unsigned(T::A_BYTES));
+                        tma_load_box(st, &tmapA, raw_full0 + 8u * s, box0[0] + ck[0], box0[1] + ck[1], box0[2] + ck[2],
+                                     box0[3] + ck[3], box0[4] + ck[4]);
+                    }
+                } else {
+                    umma_produce<T::BM>(st, la, opA, k0, sa);
+                }
+                umma_produce<T::BN, T::BK>(st + T::A_BYTES, lb, opB, k0, sb);
                 mbar_arrive_on_copies(raw_full0 + 8u * s);
+                BTC_PHASE_END(t_copy);
             }
         }
+        BTC_PHASE_STORE(p, pt == 0, 3, t_empty);
+        BTC_PHASE_STORE(p, pt == 0, 7, t_setup);
         cp_async_wait_all();
     } else {
         // ------------------------------------------------------------- MMA warp
@@ -525,6 +654,10 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         int g = 0, n = 0;
         long long t_acc = 0, t_full = 0, t_issue = 0;
         (void)t_acc; (void)t_full; (void)t_issue;
+#ifdef BTC_STAMPS
+        long long wall_ns;                       // the main loop in wall-clock time: gives the SM clock it ran at
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(wall_ns));
+#endif
         BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x, ++n) {
@@ -547,14 +680,14 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 if (leader) {
                     const unsigned a_hi = raw0 + unsigned(s) * T::STAGE_BYTES, b_hi = a_hi + T::A_BYTES;
                     const unsigned a_lo = tail0 + unsigned(t) * T::TAIL_BYTES, b_lo = a_lo + T::TAIL_B_OFFSET;
-                    const unsigned ta = tmem_base + unsigned(2 * T::ACC_COLS + t * T::A_COLS);   // head columns, tail 32 further
+                    const unsigned ta = tmem_base + unsigned(2 * T::ACC_COLS + t * T::A_COLS);   // head columns, tail BK further
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
+                    for (int j = 0; j < T::KSTEPS; ++j) {
                         const uint64_t dbh = umma_smem_desc(b_hi + j * b_step, b_lbo, b_sbo, b_lay);
                         const uint64_t dbl = umma_smem_desc(b_lo + j * b_step, b_lbo, b_sbo, b_lay);
                         const unsigned acc_in = (kt > 0 || j > 0) ? 1u : 0u;
                         if (T::A_TMEM) {
-                            umma_tf32_ts(tacc, ta + 32u + 8u * j, dbh, idesc, acc_in);
+                            umma_tf32_ts(tacc, ta + unsigned(T::BK) + 8u * j, dbh, idesc, acc_in);
                             umma_tf32_ts(tacc, ta + 8u * j, dbl, idesc, 1u);
                             umma_tf32_ts(tacc, ta + 8u * j, dbh, idesc, 1u);
                         } else {
@@ -573,9 +706,17 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 BTC_PHASE_END(t_issue);
             }
         }
+#ifdef BTC_STAMPS
+        {
+            long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            t_full += t_acc;                     // slot 4: all waiting; slot 6: nanoseconds
+            t_acc = now - wall_ns;
+        }
+#endif
+        BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 6, t_acc);
         BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 4, t_full);
         BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 5, t_issue);
-        BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 6, t_acc);
         tc_fence_before();
     }
 

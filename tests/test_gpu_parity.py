@@ -212,7 +212,7 @@ def test_unaligned_base_pointer_falls_back_to_element_copies(api, handle):
     assert worst <= 1.0
 
 
-@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(17)]
+@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(21)]
                          + [(torch.complex128, v) for v in range(3)] + [(torch.complex64, v) for v in range(2)])
 def test_every_tile_variant(api, handle, dtype, variant):
     """Each tile variant of the tiled kernels, forced through the attribute, on a ragged multi-tile case
@@ -249,6 +249,38 @@ def test_persistent_tensor_memory_kernel_walks_many_tiles(api, handle, variant):
     assert worst <= 1.0 and status["kernel"] == api.KERNEL_TILED
     bn = {10: 96, 11: 128, 12: 256, 13: 96, 14: 128, 15: 96, 16: 128}[variant]
     assert status["grid"][0] < -(-ext["i"] // 128) * -(-ext["j"] // bn) * ext["z"]   # fewer CTAs than tiles
+
+
+BULK = {
+    # name: (labelsA, labelsB, labelsD, extents, strides of D or None); the operand that ends up on the M side
+    # is a tensor of boxes for stages of 24 and of 32 contracted indices
+    "rows_contiguous_ragged": ("ik", "kj", "ij", dict(i=128 * 3 + 44, j=200, k=150), None),
+    "k_contiguous_ragged": ("ki", "kj", "ij", dict(i=128 * 2 + 20, j=150, k=152), None),
+    "k_contiguous_two_k_modes": ("kiq", "jqk", "ij", dict(i=256, j=100, k=96, q=3), None),
+    # workload 3 scaled down: rows of a tile = 8 j x 16 b, stage = all 24 l, batch z
+    "blocked_free_modes": ("akzl", "lbkjz", "jbza", dict(z=3, a=40, b=32, j=24, k=5, l=24), (1, 28, 28 * 32, 28 * 32 * 3)),
+    "many_tiles_batch": ("kiz", "zkj", "ijz", dict(i=128 * 17 + 5, j=96 * 3 + 7, k=72, z=2), None),
+}
+
+
+@pytest.mark.parametrize("variant", [17, 18, 19, 20])
+@pytest.mark.parametrize("name", list(BULK))
+def test_bulk_tensor_copy_variants(api, handle, name, variant):
+    """The tcgen05 variants that fetch the M-side tile of every stage with one bulk tensor copy: boxes with
+    rows or k contiguous, ragged last tiles in M and in K (zero-filled by the copy), several contracted
+    modes, blocked free modes with a batch label, and more tiles than SMs.  Where a stage of that
+    variant's length is no box of the operand the planner must hand the work to the gathering twin."""
+    la, lb, ld, ext, sD = BULK[name]
+    A = helpers.random_tensor(91, _ext(la, ext), None, torch.float32)
+    B = helpers.random_tensor(92, _ext(lb, ext), None, torch.float32)
+    C = helpers.random_tensor(93, _ext(ld, ext), sD, torch.float32)
+    D = inputs.place(None, _ext(ld, ext), sD, torch.float32)
+    worst, status, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, 0.75, 1.5, kernel=api.KERNEL_TILED,
+                                        variant=variant, want_status=True)
+    assert worst <= 1.0 and status["kernel"] == api.KERNEL_TILED
+    bk = 24 if variant in (17, 20) else 32
+    boxes = not (name == "blocked_free_modes" and bk == 32)      # 24 l, then k: a stage of 32 is no box
+    assert status["variant"] == (variant if boxes else (13 if variant <= 18 else 14))
 
 
 CASE4 = {
