@@ -1094,8 +1094,15 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
 #define BTC_EW_LAUNCH(R, CPLX)                                                                                     \
     do {                                                                                                           \
         if (transposing) {                                                                                         \
-            if (narrow) elementwise_transposing_kernel<R, CPLX, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);     \
-            else elementwise_transposing_kernel<R, CPLX, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);             \
+            typedef TransposeTile<R, CPLX> TT;                                                                     \
+            static bool configured[64] = {}, configured_wide[64] = {};                                             \
+            if (narrow) {                                                                                          \
+                if (set_smem_once(elementwise_transposing_kernel<R, CPLX, uint32_t>, TT::SMEM_BYTES, configured) != cudaSuccess) return BTC_ERR_CUDA; \
+                elementwise_transposing_kernel<R, CPLX, uint32_t><<<unsigned(blocks), TT::THREADS, TT::SMEM_BYTES, st>>>(p); \
+            } else {                                                                                               \
+                if (set_smem_once(elementwise_transposing_kernel<R, CPLX, int64_t>, TT::SMEM_BYTES, configured_wide) != cudaSuccess) return BTC_ERR_CUDA; \
+                elementwise_transposing_kernel<R, CPLX, int64_t><<<unsigned(blocks), TT::THREADS, TT::SMEM_BYTES, st>>>(p); \
+            }                                                                                                      \
         } else if (lanes == 32) {                                                                                  \
             if (narrow) elementwise_direct_kernel<R, CPLX, 32, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);      \
             else elementwise_direct_kernel<R, CPLX, 32, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);              \
@@ -1137,7 +1144,7 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
         return cudaGetLastError() == cudaSuccess ? BTC_SUCCESS : BTC_ERR_CUDA;
     }
     if (transposing) {
-        const int T = dtype_size(pl.dtype) == 4 ? 64 : 32;
+        const int T = dtype_size(pl.dtype) <= 8 ? 64 : 32;
         p.tile_mode_a = pl.tile_mode_a;
         p.tiles_c = int32_t((p.ext_k[0] + T - 1) / T);
         p.tiles_a = int32_t((p.ext_k[pl.tile_mode_a] + T - 1) / T);

@@ -18,6 +18,9 @@
 
 namespace btc {
 
+// arithmetic type of alpha * a + beta * b where nothing is summed: the part type itself
+template <typename R> struct ElementwiseScalar { typedef R type; };
+
 // alpha * (acc_r, acc_i) + beta * op(b) -> C[off]
 template <typename R, bool CPLX>
 __device__ __forceinline__ void elementwise_finish(const ElementwiseParams &p, int64_t offB, int64_t offC, double acc_r, double acc_i)
@@ -59,7 +62,8 @@ __device__ __forceinline__ void elementwise_sum(const ElementwiseParams &p, int6
             for (int u = 0; u < U; ++u) {
                 const int64_t s = s0 + int64_t(u) * LANES;
                 const bool in = s < p.total_sum;
-                const int64_t off = base + (in ? decode_offset<I>(I(s), p.ns, p.ext_s, p.sA_s) : 0);
+                // one summed dimension: its index times its stride, no decoding
+                const int64_t off = base + (in ? (p.ns == 1 ? s * p.sA_s[0] : decode_offset<I>(I(s), p.ns, p.ext_s, p.sA_s)) : 0);
                 v_r[u] = in ? A[NC * off] : R(0);
                 v_i[u] = (CPLX && in) ? A[NC * off + (NC - 1)] : R(0);
             }
@@ -79,6 +83,58 @@ __global__ void __launch_bounds__(256) elementwise_direct_kernel(const Elementwi
     const int lane = (LANES == 1) ? 0 : int(threadIdx.x) % LANES;
     const int64_t group = (int64_t(blockIdx.x) * blockDim.x + threadIdx.x) / LANES;
     const int64_t ngroups = (int64_t(gridDim.x) * blockDim.x) / LANES;
+    if (LANES == 1 && p.ns == 0) {
+        // nothing summed: four elements per thread and pass, all loads issued before the first
+        // store (B may be C's memory, so the compiler would not move them by itself)
+        constexpr int NC = CPLX ? 2 : 1;
+        constexpr int U = 4;
+        const R *A = static_cast<const R *>(p.A);
+        const R *B = static_cast<const R *>(p.B);
+        R *C = static_cast<R *>(p.C);
+        for (int64_t e0 = group; e0 < p.total_keep; e0 += int64_t(U) * ngroups) {
+            int64_t offA[U], offB[U], offC[U];
+            bool in[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int64_t e = e0 + int64_t(u) * ngroups;
+                in[u] = e < p.total_keep;
+                offA[u] = offB[u] = offC[u] = 0;
+                I lin = I(in[u] ? e : 0);
+                for (int d = 0; d < p.nk; ++d) {
+                    const I ext = I(p.ext_k[d]);
+                    const I q = lin / ext;
+                    const int64_t i = int64_t(lin - q * ext);
+                    lin = q;
+                    offA[u] += i * p.sA_k[d];
+                    offB[u] += i * p.sB_k[d];
+                    offC[u] += i * p.sC_k[d];
+                }
+            }
+            R a_r[U], a_i[U], b_r[U], b_i[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                a_r[u] = (p.use_a && in[u]) ? A[NC * offA[u]] : R(0);
+                a_i[u] = (CPLX && p.use_a && in[u]) ? A[NC * offA[u] + (NC - 1)] : R(0);
+                b_r[u] = (p.use_b && in[u]) ? B[NC * offB[u]] : R(0);
+                b_i[u] = (CPLX && p.use_b && in[u]) ? B[NC * offB[u] + (NC - 1)] : R(0);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (!in[u]) continue;
+                typedef typename ElementwiseScalar<R>::type S;
+                const S al_r = S(p.alpha[0]), al_i = S(p.alpha[1]), be_r = S(p.beta[0]), be_i = S(p.beta[1]);
+                const S ar = S(a_r[u]), ai = p.conjA ? -S(a_i[u]) : S(a_i[u]);
+                const S br = S(b_r[u]), bi = p.conjB ? -S(b_i[u]) : S(b_i[u]);
+                if (CPLX) {
+                    C[NC * offC[u]] = R(al_r * ar - al_i * ai + be_r * br - be_i * bi);
+                    C[NC * offC[u] + (NC - 1)] = R(al_r * ai + al_i * ar + be_r * bi + be_i * br);
+                } else {
+                    C[NC * offC[u]] = R(al_r * ar + be_r * br);
+                }
+            }
+        }
+        return;
+    }
     for (int64_t e = group; e < p.total_keep; e += ngroups) {
         int64_t offA = 0, offB = 0, offC = 0;
         I lin = I(e);
@@ -161,18 +217,29 @@ __global__ void __launch_bounds__(256) elementwise_vector_kernel(const Elementwi
     }
 }
 
+// Tile edge and CTA size of the transposing kernel: 64 x 64 tiles for elements of up to 8 bytes (rows
+// of 256 or 512 bytes on both sides), 32 x 32 for complex128, 256 threads.  Measured on permutations of
+// 1 GB tensors: 256-byte rows reach 5.0-5.5 TB/s, 512-byte rows the copy bandwidth; 128 x 128 tiles
+// with 1024 threads for 4-byte elements were slower (3.6 TB/s: two large CTAs per SM overlap poorly).
+template <typename R, bool CPLX> struct TransposeTile {
+    static constexpr int NC = CPLX ? 2 : 1;
+    static constexpr int T = sizeof(R) * NC <= 8 ? 64 : 32;
+    static constexpr int THREADS = 256;
+    static constexpr size_t SMEM_BYTES = size_t(NC) * T * (T + 1) * sizeof(R);
+};
+
 // blockIdx.x enumerates (tile along C's dimension 0, tile along A's dimension, rest), first fastest.
-// T x T tiles (T = 64 for 4-byte elements, 32 otherwise: rows of at least 256 bytes on both sides),
-// 256 threads, each T * T / 256 elements in either phase; the tile holds values already summed and
-// rounded to the element type.
+// Each thread handles T * T / THREADS elements in either phase; the tile holds values already
+// summed and rounded to the element type.
 template <typename R, bool CPLX, typename I>
-__global__ void __launch_bounds__(256) elementwise_transposing_kernel(const ElementwiseParams p)
+__global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise_transposing_kernel(const ElementwiseParams p)
 {
     constexpr int NC = CPLX ? 2 : 1;
-    constexpr int T = (sizeof(R) * NC == 4) ? 64 : 32;
-    constexpr int ROWS = 256 / T;                        // tile rows covered by the CTA at once
+    constexpr int T = TransposeTile<R, CPLX>::T;
+    constexpr int ROWS = TransposeTile<R, CPLX>::THREADS / T;   // tile rows covered by the CTA at once
     constexpr int PER = T / ROWS;                        // rows per thread
-    __shared__ R tile[NC][T][T + 1];
+    extern __shared__ __align__(16) unsigned char tile_bytes[];
+    R (*tile)[T][T + 1] = reinterpret_cast<R (*)[T][T + 1]>(tile_bytes);
     const int ma = p.tile_mode_a;
     const int64_t tile_c = blockIdx.x % p.tiles_c;
     const int64_t tile_a = (blockIdx.x / p.tiles_c) % p.tiles_a;
@@ -189,24 +256,76 @@ __global__ void __launch_bounds__(256) elementwise_transposing_kernel(const Elem
     const int tx = threadIdx.x % T, ty = threadIdx.x / T;
     const int64_t c0 = tile_c * T, a0 = tile_a * T;
     const int64_t ext_c = p.ext_k[0], ext_a = p.ext_k[ma];
-    // phase 1: consecutive threads along A's dimension
+    // phase 1: consecutive threads along A's dimension.  Without summed dimensions (a pure
+    // permutation) all of a thread's loads are issued before the first value is used; a load
+    // inside the bounds test of its own iteration would leave one load in flight per thread.
+    if (p.ns == 0 && p.use_a) {
+        const R *A = static_cast<const R *>(p.A);
+        R v_r[PER], v_i[PER];
+        const bool a_in = a0 + tx < ext_a;
+        const R *src = A + NC * (restA + (a0 + tx) * p.sA_k[ma] + (c0 + ty) * p.sA_k[0]);
+        const int64_t step = NC * ROWS * p.sA_k[0];
+        const int rows_in = int(ext_c - c0 - ty < int64_t(T) ? ext_c - c0 - ty : int64_t(T));   // rows ty + ROWS r < rows_in exist
 #pragma unroll
-    for (int r = 0; r < PER; ++r) {
-        const int64_t c = c0 + ty + ROWS * r, a = a0 + tx;
-        double acc_r = 0.0, acc_i = 0.0;
-        if (c < ext_c && a < ext_a)
-            elementwise_sum<R, CPLX, 1, I>(p, restA + c * p.sA_k[0] + a * p.sA_k[ma], 0, acc_r, acc_i);
-        tile[0][ty + ROWS * r][tx] = R(acc_r);
-        if (CPLX) tile[NC - 1][ty + ROWS * r][tx] = R(acc_i);
+        for (int r = 0; r < PER; ++r) {
+            const bool in = a_in && ROWS * r < rows_in;
+            v_r[r] = in ? src[0] : R(0);
+            v_i[r] = (CPLX && in) ? src[NC - 1] : R(0);
+            src += step;
+        }
+#pragma unroll
+        for (int r = 0; r < PER; ++r) {
+            tile[0][ty + ROWS * r][tx] = v_r[r];
+            if (CPLX) tile[NC - 1][ty + ROWS * r][tx] = p.conjA ? -v_i[r] : v_i[r];
+        }
+    } else {
+#pragma unroll
+        for (int r = 0; r < PER; ++r) {
+            const int64_t c = c0 + ty + ROWS * r, a = a0 + tx;
+            double acc_r = 0.0, acc_i = 0.0;
+            if (c < ext_c && a < ext_a)
+                elementwise_sum<R, CPLX, 1, I>(p, restA + c * p.sA_k[0] + a * p.sA_k[ma], 0, acc_r, acc_i);
+            tile[0][ty + ROWS * r][tx] = R(acc_r);
+            if (CPLX) tile[NC - 1][ty + ROWS * r][tx] = R(acc_i);
+        }
     }
     __syncthreads();
-    // phase 2: consecutive threads along C's dimension 0
+    // phase 2: consecutive threads along C's dimension 0; B's values are loaded as a batch too
+    // (B may be the same memory as C, so the compiler cannot move its loads across the stores).
+    // alpha * t + beta * b is formed in double only for 64-bit parts: for 32-bit parts the two
+    // products and the sum in float are within a few units in the last place of |alpha t| + |beta b|.
+    {
+        typedef typename ElementwiseScalar<R>::type S;
+        const R *B = static_cast<const R *>(p.B);
+        R *C = static_cast<R *>(p.C);
+        const bool c_in = c0 + tx < ext_c;
+        const int rows_in = int(ext_a - a0 - ty < int64_t(T) ? ext_a - a0 - ty : int64_t(T));
+        const R *srcB = B + NC * (restB + (c0 + tx) * p.sB_k[0] + (a0 + ty) * p.sB_k[ma]);
+        R *dst = C + NC * (restC + (c0 + tx) * p.sC_k[0] + (a0 + ty) * p.sC_k[ma]);
+        const int64_t stepB = NC * ROWS * p.sB_k[ma], stepC = NC * ROWS * p.sC_k[ma];
+        const S al_r = S(p.alpha[0]), al_i = S(p.alpha[1]), be_r = S(p.beta[0]), be_i = S(p.beta[1]);
+        R b_r[PER], b_i[PER];
 #pragma unroll
-    for (int r = 0; r < PER; ++r) {
-        const int64_t c = c0 + tx, a = a0 + ty + ROWS * r;
-        if (c < ext_c && a < ext_a)
-            elementwise_finish<R, CPLX>(p, restB + c * p.sB_k[0] + a * p.sB_k[ma], restC + c * p.sC_k[0] + a * p.sC_k[ma],
-                                        double(tile[0][tx][ty + ROWS * r]), CPLX ? double(tile[NC - 1][tx][ty + ROWS * r]) : 0.0);
+        for (int r = 0; r < PER; ++r) {
+            const bool in = p.use_b && c_in && ROWS * r < rows_in;
+            b_r[r] = in ? srcB[0] : R(0);
+            b_i[r] = (CPLX && in) ? srcB[NC - 1] : R(0);
+            srcB += stepB;
+        }
+#pragma unroll
+        for (int r = 0; r < PER; ++r) {
+            if (c_in && ROWS * r < rows_in) {
+                const S t_r = S(tile[0][tx][ty + ROWS * r]), t_i = CPLX ? S(tile[NC - 1][tx][ty + ROWS * r]) : S(0);
+                const S br = S(b_r[r]), bi = CPLX ? (p.conjB ? -S(b_i[r]) : S(b_i[r])) : S(0);
+                if (CPLX) {
+                    dst[0] = R(al_r * t_r - al_i * t_i + be_r * br - be_i * bi);
+                    dst[NC - 1] = R(al_r * t_i + al_i * t_r + be_r * bi + be_i * br);
+                } else {
+                    dst[0] = R(al_r * t_r + be_r * br);
+                }
+            }
+            dst += stepC;
+        }
     }
 }
 
