@@ -110,9 +110,10 @@ using F32Umma96B24 = UmmaTile<96, 7, 2, true, 1, 24, true>;
 using F32Umma96B32 = UmmaTile<96, 5, 2, true, 1, 32, true>;
 using F32Umma128B32 = UmmaTile<128, 4, 2, true, 1, 32, true>;
 using F32Umma128B24 = UmmaTile<128, 5, 2, true, 1, 24, true>;
-constexpr int kNumF32Variants = 21;
+using F32Umma96B24x2 = UmmaTile<96, 3, 2, true, 1, 24, true, 2>;   // two sub-stages of 24 k per hand-off
+constexpr int kNumF32Variants = 22;
 constexpr int kFirstUmmaVariant = 10;
-constexpr int kFirstBulkVariant = 17;     // 17..20: bulk tensor copies; fall back to 13 / 14 (same tiles) at execute
+constexpr int kFirstBulkVariant = 17;     // 17..21: bulk tensor copies; fall back to 13 / 14 (same tiles) at execute
 
 struct VariantInfo {
     int bm, bn, bk, threads, acc;
@@ -159,6 +160,7 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
         case 18: return {128, 96, 32, 256, 0, F32Umma96B32::SMEM_BYTES, 4};
         case 19: return {128, 128, 32, 256, 0, F32Umma128B32::SMEM_BYTES, 4};
         case 20: return {128, 128, 24, 256, 0, F32Umma128B24::SMEM_BYTES, 4};
+        case 21: return {128, 96, 24, 256, 0, F32Umma96B24x2::SMEM_BYTES, 4};
         default: return {128, 128, 32, 256, 0, F32Umma128T2::SMEM_BYTES, 4};
         }
     }
@@ -341,14 +343,16 @@ int finish_plan(btc_contraction_s *op)
         // 17-20 fetch the M side with bulk tensor copies; they enter when that operand is a tensor of boxes
         TmaOperand probe;
         const bool box24 = umma_ok && make_tma_operand(pl, 128, 24, probe), box32 = umma_ok && make_tma_operand(pl, 128, 32, probe);
-        // (measured a little behind their gathering twins 13 / 14 on the batched permuted workload, hence the weights)
+        // (weights from the batched permuted workload: 21, two sub-stages of 24 k per hand-off, is 2 % ahead of
+        // the gathering variant 13, the single-sub-stage ones 17-20 a little behind their twins 13 / 14)
         const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {14, 2.3}, {13, 2.0},
-                             {box24 ? 17 : 13, 1.85}, {box32 ? 18 : 13, 1.95}, {box32 ? 19 : 14, 2.25}, {box24 ? 20 : 14, 2.1}};
+                             {box24 ? 17 : 13, 1.85}, {box32 ? 18 : 13, 1.95}, {box32 ? 19 : 14, 2.25}, {box24 ? 20 : 14, 2.1},
+                             {box24 ? 21 : 13, 2.04}};
         const Cand f64c[] = {{2, 1.0}, {1, 0.75}};       // big tile: the m16n8k16 variant
         const Cand c64c[] = {{2, 1.0}, {1, 0.75}};       // complex128: big tile on m16n8k16 as well
         const Cand other[] = {{0, 1.0}, {1, 0.75}};
         const Cand *cands = pl.dtype == BTC_F32 ? f32c : (pl.dtype == BTC_F64 ? f64c : (pl.dtype == BTC_C64 ? c64c : other));
-        const int ncand = pl.dtype == BTC_F32 ? (umma_ok ? 11 : 4) : 2;
+        const int ncand = pl.dtype == BTC_F32 ? (umma_ok ? 12 : 4) : 2;
         double best = -1.0;
         for (int c = 0; c < ncand; ++c) {
             const VariantInfo vi = variant_info(pl.dtype, cands[c].id);
@@ -371,7 +375,7 @@ int finish_plan(btc_contraction_s *op)
     if (pl.dtype == BTC_F32 && variant >= kFirstBulkVariant) {
         // a forced bulk-copy variant whose M-side operand is no tensor of boxes: the gathering twin
         const VariantInfo bv = variant_info(pl.dtype, variant);
-        if (!make_tma_operand(pl, bv.bm, bv.bk, op->tmaA)) variant = variant <= 18 ? 13 : 14;
+        if (!make_tma_operand(pl, bv.bm, bv.bk, op->tmaA)) variant = (variant <= 18 || variant == 21) ? 13 : 14;
     }
     const VariantInfo v = variant_info(pl.dtype, variant);
     pl.tile.bm = v.bm; pl.tile.bn = v.bn; pl.tile.bk = v.bk; pl.tile.threads = v.threads;
@@ -865,12 +869,13 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
                 CUtensorMap mapA;
                 const int v = pl.tile.variant;
                 if (misaligned(pA, 16) || !encode_tma_operand(op->tmaA, pA, &mapA)) {
-                    ran_variant = v <= 18 ? 13 : 14;
-                    ce = v <= 18 ? launch_umma<F32Umma96T>(tp, ctas, st) : launch_umma<F32Umma128T>(tp, ctas, st);
+                    ran_variant = (v <= 18 || v == 21) ? 13 : 14;
+                    ce = ran_variant == 13 ? launch_umma<F32Umma96T>(tp, ctas, st) : launch_umma<F32Umma128T>(tp, ctas, st);
                 }
                 else if (v == 17) ce = launch_umma<F32Umma96B24>(tp, ctas, st, &mapA);
                 else if (v == 18) ce = launch_umma<F32Umma96B32>(tp, ctas, st, &mapA);
                 else if (v == 19) ce = launch_umma<F32Umma128B32>(tp, ctas, st, &mapA);
+                else if (v == 21) ce = launch_umma<F32Umma96B24x2>(tp, ctas, st, &mapA);
                 else ce = launch_umma<F32Umma128B24>(tp, ctas, st, &mapA);
             } break;
             }

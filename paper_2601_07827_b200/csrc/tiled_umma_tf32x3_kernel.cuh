@@ -40,10 +40,15 @@
 
 namespace btc {
 
-template <int BN_, int RAW_STAGES_, int TAIL_STAGES_, bool A_TMEM_ = false, int CONVERTER_GROUPS_ = 1, int BK_ = 32, bool A_TMA_ = false>
+template <int BN_, int RAW_STAGES_, int TAIL_STAGES_, bool A_TMEM_ = false, int CONVERTER_GROUPS_ = 1, int BK_ = 32, bool A_TMA_ = false,
+          int SUBS_ = 1>
 struct UmmaTile {
     static constexpr int BM = 128, BN = BN_, BK = BK_;
-    static constexpr int KSTEPS = BK_ / 8;                           // tensor-core instructions of K = 8 per stage
+    static constexpr int KSTEPS = BK_ / 8;                           // tensor-core instructions of K = 8 per sub-stage
+    // A stage (the unit the roles hand to one another through mbarriers) holds SUBS sub-stages of BK
+    // k each, laid out one after the other.  A hand-off costs several hundred cycles whatever the
+    // stage holds, so two sub-stages per stage halve that cost per k.
+    static constexpr int SUBS = SUBS_;
     static constexpr int RAW_STAGES = RAW_STAGES_, TAIL_STAGES = TAIL_STAGES_;
     // A_TMA: the M-side tile of a stage arrives by one bulk tensor copy (needs A_TMEM: the box is
     // not in a layout the tensor core reads, the converters take it to tensor memory)
@@ -63,17 +68,20 @@ struct UmmaTile {
     static constexpr int THREADS = 32 * (MMA_WARP + 1);
     // a k-contiguous N-side tile keeps 128-byte rows whatever BK is (the swizzle atom)
     static constexpr int A_BYTES = BM * BK * 4, B_BYTES = BN * 32 * 4;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;           // a raw stage
+    static constexpr int SUB_BYTES = A_BYTES + B_BYTES;             // one sub-stage of a raw stage: M-side tile, N-side tile
+    static constexpr int STAGE_BYTES = SUBS_ * SUB_BYTES;           // a raw stage
     static_assert(A_BYTES % 1024 == 0, "operand tiles sit on 1024-byte boundaries");
-    static constexpr int TAIL_BYTES = A_TMEM_ ? B_BYTES : STAGE_BYTES;
+    static constexpr int TAIL_SUB_BYTES = A_TMEM_ ? B_BYTES : SUB_BYTES;
+    static constexpr int TAIL_BYTES = SUBS_ * TAIL_SUB_BYTES;
     static constexpr int TAIL_B_OFFSET = A_TMEM_ ? 0 : A_BYTES;     // where the N-side tail sits in a tail stage
     static constexpr int ACC_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;   // one accumulator
-    static constexpr int A_COLS = A_TMEM_ ? 2 * BK : 0;             // head + tail of one stage of the M-side operand
+    static constexpr int A_SUB_COLS = A_TMEM_ ? 2 * BK : 0;         // head + tail of one sub-stage of the M-side operand
+    static constexpr int A_COLS = SUBS_ * A_SUB_COLS;
     static constexpr int TMEM_USED = 2 * ACC_COLS + TAIL_STAGES_ * A_COLS;
     static constexpr int TMEM_COLS = TMEM_USED <= 32 ? 32 : TMEM_USED <= 64 ? 64 : TMEM_USED <= 128 ? 128 : TMEM_USED <= 256 ? 256 : 512;
     static_assert(TMEM_USED <= 512, "accumulators and operand stages must fit the 512 tensor-memory columns");
     // 16-byte pieces per converter thread in the position-independent pass (whole stage, or its N side)
-    static constexpr int PIECES = (A_TMEM_ ? B_BYTES : STAGE_BYTES) / 16 / CONVERTER_THREADS;
+    static constexpr int PIECES = (A_TMEM_ ? B_BYTES : SUB_BYTES) / 16 / CONVERTER_THREADS;
     static constexpr int NUM_BARS = 2 * RAW_STAGES + 2 * TAIL_STAGES + 8;
     static_assert(B_BYTES % (16 * CONVERTER_THREADS) == 0, "a stage must divide among the converters");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "BN must suit UMMA N and the epilogue split");
@@ -363,7 +371,8 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int64_t total = int64_t(p.tiles_m) * p.tiles_n * p.Bt;         // split_k == 1 on this path
-    const int num_kt = int((p.K + T::BK - 1) / T::BK);
+    const int num_kt = int((p.K + T::BK - 1) / T::BK);                   // sub-stages of a tile
+    const int num_st = (num_kt + T::SUBS - 1) / T::SUBS;                 // stages of a tile
     const bool staged = p.K <= kKoffCap;
     const bool coords_staged = 5 * num_kt <= 2 * kKoffCap;
 
@@ -458,7 +467,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x) {
 #pragma unroll 1
-            for (int kt = 0; kt < num_kt; ++kt, ++g) {
+            for (int st = 0; st < num_st; ++st, ++g) {
                 if (T::CONVERTER_GROUPS > 1 && g % T::CONVERTER_GROUPS != group) continue;   // another group's stage
                 const int s = g % T::RAW_STAGES, t = g % T::TAIL_STAGES;
                 if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(g / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait)) {
@@ -472,7 +481,10 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     break;
                 }
                 BTC_PHASE_END(t_tail);
-                const unsigned raw_stage = raw0 + unsigned(s) * T::STAGE_BYTES;
+#pragma unroll
+                for (int sub = 0; sub < T::SUBS; ++sub) {
+                if (st * T::SUBS + sub >= num_kt) break;     // a tile's last stage may hold fewer sub-stages
+                const unsigned raw_stage = raw0 + unsigned(s) * T::STAGE_BYTES + unsigned(sub) * T::SUB_BYTES;
                 if (T::A_TMEM) {
                     // M-side operand: this thread owns row ct of the tile = lane ct of tensor memory.
                     // It reads the row's 32 k from the raw tile (both layouts give conflict-free
@@ -516,7 +528,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     }
 #pragma unroll
                     for (int k = 0; k < T::BK; ++k) lo[k] = x[k] - __uint_as_float(__float_as_uint(x[k]) & 0xffffe000u);
-                    const unsigned ta = tmem_base + (unsigned(ct & ~31) << 16) + unsigned(2 * T::ACC_COLS + t * T::A_COLS);
+                    const unsigned ta = tmem_base + (unsigned(ct & ~31) << 16) + unsigned(2 * T::ACC_COLS + t * T::A_COLS + sub * T::A_SUB_COLS);
                     if constexpr (T::BK == 32) {
                         tmem_store32(ta, x);
                         tmem_store32(ta + 32u, lo);
@@ -529,7 +541,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     }
                 }
                 const unsigned src = raw_stage + (T::A_TMEM ? T::A_BYTES : 0) + unsigned(ct) * 16u;
-                const unsigned dst = tail0 + unsigned(t) * T::TAIL_BYTES + unsigned(ct) * 16u;
+                const unsigned dst = tail0 + unsigned(t) * T::TAIL_BYTES + unsigned(sub) * T::TAIL_SUB_BYTES + unsigned(ct) * 16u;
                 constexpr unsigned STEP = 16u * T::CONVERTER_THREADS;
                 constexpr int CHUNK = T::PIECES % 8 == 0 ? 8 : T::PIECES % 7 == 0 ? 7 : T::PIECES % 6 == 0 ? 6 : 4;   // loads in flight per thread
                 static_assert(T::PIECES % CHUNK == 0, "pieces must divide into chunks");
@@ -553,6 +565,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                         asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + unsigned(i0 + i) * STEP), "f"(lo[0]), "f"(lo[1]), "f"(lo[2]), "f"(lo[3]) : "memory");
                     }
                 }
+                }   // sub-stages
                 if (T::A_TMEM) {
                     tmem_store_wait();           // the operand columns are written ...
                     tc_fence_before();           // ... and ordered before the arrival below
@@ -604,12 +617,14 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             if (opB.vec == 4) sb_next = umma_lookup<T::BN, T::BK>(lb, opB, 0);
             BTC_PHASE_END(t_setup);
 #pragma unroll 1
-            for (int kt = 0; kt < num_kt; ++kt, ++g) {
+            for (int st_i = 0; st_i < num_st; ++st_i, ++g) {
                 const int s = g % T::RAW_STAGES;
-                sa = sa_next; sb = sb_next;
-                if (kt + 1 < num_kt) {
-                    if (!T::A_TMA && opA.vec == 4) sa_next = umma_lookup<T::BM>(la, opA, int64_t(kt + 1) * T::BK);
-                    if (opB.vec == 4) sb_next = umma_lookup<T::BN, T::BK>(lb, opB, int64_t(kt + 1) * T::BK);
+                if (T::SUBS == 1) {
+                    sa = sa_next; sb = sb_next;
+                    if (st_i + 1 < num_st) {
+                        if (!T::A_TMA && opA.vec == 4) sa_next = umma_lookup<T::BM>(la, opA, int64_t(st_i + 1) * T::BK);
+                        if (opB.vec == 4) sb_next = umma_lookup<T::BN, T::BK>(lb, opB, int64_t(st_i + 1) * T::BK);
+                    }
                 }
                 if (g >= T::RAW_STAGES &&
                     !mbar_wait_bounded(raw_empty0 + 8u * s, unsigned(g / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait)) {
@@ -617,19 +632,29 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     break;
                 }
                 BTC_PHASE_END(t_empty);
-                const unsigned st = raw0 + unsigned(s) * T::STAGE_BYTES;
-                const int64_t k0 = int64_t(kt) * T::BK;
-                if (T::A_TMA) {
-                    if (pt == 0) {
-                        const int32_t *ck = (coords_staged ? reinterpret_cast<const int32_t *>(koffA) : p.tmaA_coord_k) + kt * 5;
-                        mbar_arrive_expect_tx(raw_full0 + 8u * s, unsigned(T::A_BYTES));
-                        tma_load_box(st, &tmapA, raw_full0 + 8u * s, box0[0] + ck[0], box0[1] + ck[1], box0[2] + ck[2],
-                                     box0[3] + ck[3], box0[4] + ck[4]);
+                const int subs_here = num_kt - st_i * T::SUBS < T::SUBS ? num_kt - st_i * T::SUBS : T::SUBS;
+                if (T::A_TMA && pt == 0) mbar_arrive_expect_tx(raw_full0 + 8u * s, unsigned(T::A_BYTES) * unsigned(subs_here));
+#pragma unroll
+                for (int sub = 0; sub < T::SUBS; ++sub) {
+                    if (sub >= subs_here) break;
+                    const int kt = st_i * T::SUBS + sub;
+                    const unsigned st = raw0 + unsigned(s) * T::STAGE_BYTES + unsigned(sub) * T::SUB_BYTES;
+                    const int64_t k0 = int64_t(kt) * T::BK;
+                    if (T::SUBS > 1) {
+                        if (!T::A_TMA && opA.vec == 4) sa = umma_lookup<T::BM>(la, opA, k0);
+                        if (opB.vec == 4) sb = umma_lookup<T::BN, T::BK>(lb, opB, k0);
                     }
-                } else {
-                    umma_produce<T::BM>(st, la, opA, k0, sa);
+                    if (T::A_TMA) {
+                        if (pt == 0) {
+                            const int32_t *ck = (coords_staged ? reinterpret_cast<const int32_t *>(koffA) : p.tmaA_coord_k) + kt * 5;
+                            tma_load_box(st, &tmapA, raw_full0 + 8u * s, box0[0] + ck[0], box0[1] + ck[1], box0[2] + ck[2],
+                                         box0[3] + ck[3], box0[4] + ck[4]);
+                        }
+                    } else {
+                        umma_produce<T::BM>(st, la, opA, k0, sa);
+                    }
+                    umma_produce<T::BN, T::BK>(st + T::A_BYTES, lb, opB, k0, sb);
                 }
-                umma_produce<T::BN, T::BK>(st + T::A_BYTES, lb, opB, k0, sb);
                 mbar_arrive_on_copies(raw_full0 + 8u * s);
                 BTC_PHASE_END(t_copy);
             }
@@ -669,7 +694,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             tc_fence_after();
             const unsigned tacc = tmem_base + unsigned(buf * T::ACC_COLS);
 #pragma unroll 1
-            for (int kt = 0; kt < num_kt; ++kt, ++g) {
+            for (int st = 0; st < num_st; ++st, ++g) {
                 const int s = g % T::RAW_STAGES, t = g % T::TAIL_STAGES;
                 if (!mbar_wait_bounded(tail_full0 + 8u * t, unsigned(g / T::TAIL_STAGES) & 1u, abort_flag, p.error_word, kErrTailFullWait)) {
                     ok = false;
@@ -678,14 +703,17 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 BTC_PHASE_END(t_full);
                 tc_fence_after();
                 if (leader) {
-                    const unsigned a_hi = raw0 + unsigned(s) * T::STAGE_BYTES, b_hi = a_hi + T::A_BYTES;
-                    const unsigned a_lo = tail0 + unsigned(t) * T::TAIL_BYTES, b_lo = a_lo + T::TAIL_B_OFFSET;
-                    const unsigned ta = tmem_base + unsigned(2 * T::ACC_COLS + t * T::A_COLS);   // head columns, tail BK further
+#pragma unroll
+                    for (int sub = 0; sub < T::SUBS; ++sub) {
+                    if (st * T::SUBS + sub >= num_kt) break;
+                    const unsigned a_hi = raw0 + unsigned(s) * T::STAGE_BYTES + unsigned(sub) * T::SUB_BYTES, b_hi = a_hi + T::A_BYTES;
+                    const unsigned a_lo = tail0 + unsigned(t) * T::TAIL_BYTES + unsigned(sub) * T::TAIL_SUB_BYTES, b_lo = a_lo + T::TAIL_B_OFFSET;
+                    const unsigned ta = tmem_base + unsigned(2 * T::ACC_COLS + t * T::A_COLS + sub * T::A_SUB_COLS);   // head columns, tail BK further
 #pragma unroll
                     for (int j = 0; j < T::KSTEPS; ++j) {
                         const uint64_t dbh = umma_smem_desc(b_hi + j * b_step, b_lbo, b_sbo, b_lay);
                         const uint64_t dbl = umma_smem_desc(b_lo + j * b_step, b_lbo, b_sbo, b_lay);
-                        const unsigned acc_in = (kt > 0 || j > 0) ? 1u : 0u;
+                        const unsigned acc_in = (st > 0 || sub > 0 || j > 0) ? 1u : 0u;
                         if (T::A_TMEM) {
                             umma_tf32_ts(tacc, ta + unsigned(T::BK) + 8u * j, dbh, idesc, acc_in);
                             umma_tf32_ts(tacc, ta + 8u * j, dbl, idesc, 1u);
@@ -698,9 +726,10 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                             umma_tf32(tacc, dah, dbh, idesc, 1u);
                         }
                     }
+                    }   // sub-stages
                     umma_commit(raw_empty0 + 8u * s);    // fire when these MMAs have read the stages
                     umma_commit(tail_empty0 + 8u * t);
-                    if (kt + 1 == num_kt) umma_commit(accum_full0 + 8u * buf);
+                    if (st + 1 == num_st) umma_commit(accum_full0 + 8u * buf);
                 }
                 __syncwarp();
                 BTC_PHASE_END(t_issue);

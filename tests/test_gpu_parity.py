@@ -212,7 +212,7 @@ def test_unaligned_base_pointer_falls_back_to_element_copies(api, handle):
     assert worst <= 1.0
 
 
-@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(21)]
+@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(22)]
                          + [(torch.complex128, v) for v in range(3)] + [(torch.complex64, v) for v in range(2)])
 def test_every_tile_variant(api, handle, dtype, variant):
     """Each tile variant of the tiled kernels, forced through the attribute, on a ragged multi-tile case
@@ -263,7 +263,7 @@ BULK = {
 }
 
 
-@pytest.mark.parametrize("variant", [17, 18, 19, 20])
+@pytest.mark.parametrize("variant", [17, 18, 19, 20, 21])
 @pytest.mark.parametrize("name", list(BULK))
 def test_bulk_tensor_copy_variants(api, handle, name, variant):
     """The tcgen05 variants that fetch the M-side tile of every stage with one bulk tensor copy: boxes with
@@ -278,9 +278,9 @@ def test_bulk_tensor_copy_variants(api, handle, name, variant):
     worst, status, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, 0.75, 1.5, kernel=api.KERNEL_TILED,
                                         variant=variant, want_status=True)
     assert worst <= 1.0 and status["kernel"] == api.KERNEL_TILED
-    bk = 24 if variant in (17, 20) else 32
+    bk = 24 if variant in (17, 20, 21) else 32
     boxes = not (name == "blocked_free_modes" and bk == 32)      # 24 l, then k: a stage of 32 is no box
-    assert status["variant"] == (variant if boxes else (13 if variant <= 18 else 14))
+    assert status["variant"] == (variant if boxes else (13 if variant in (17, 18, 21) else 14))
 
 
 CASE4 = {
