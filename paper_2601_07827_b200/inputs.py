@@ -414,3 +414,44 @@ def scaled_down(w: Workload, factors: Dict[str, int], name: Optional[str] = None
             s *= lead if i == 0 else e
         out = dataclasses.replace(out, stridesD=tuple(strides))
     return out
+
+
+def random_contraction(seed: int, max_work: int = 1 << 21):
+    """A seeded random contraction in the spirit of a randomized benchmark set: 0-1 batch labels,
+    0-3 free labels per input, 0-3 contracted labels, extents from a mixed list, every tensor in its
+    own random memory order with padding on one mode, negative strides on some modes of A and B.
+    Returns (labelsA, labelsB, labelsD, extents, stridesA, stridesB, stridesD); no arithmetic of the
+    method happens here."""
+    import numpy as np
+    rng = np.random.default_rng(seed)
+    pool = [1, 2, 3, 4, 5, 7, 8, 12, 16, 24, 33]
+    while True:
+        counts = [int(rng.integers(0, 2)), int(rng.integers(0, 4)), int(rng.integers(0, 4)), int(rng.integers(0, 4))]
+        if counts[0] + counts[1] + counts[3] > 8 or counts[0] + counts[2] + counts[3] > 8:
+            continue
+        names = iter("abcdefghijklmnopqrstuvwxyz")
+        groups = [[next(names) for _ in range(c)] for c in counts]          # H, M, N, K
+        extents = {l: int(rng.choice(pool)) for g in groups for l in g}
+        work = math.prod(extents.values()) if extents else 1
+        if work <= max_work:
+            break
+    H, M, N, K = groups
+
+    def shuffled(ls):
+        ls = list(ls)
+        rng.shuffle(ls)
+        return "".join(ls)
+    la, lb, ld = shuffled(H + M + K), shuffled(H + N + K), shuffled(H + M + N)
+
+    def strides_for(labels, allow_negative):
+        order = list(range(len(labels)))
+        rng.shuffle(order)                                   # memory order: order[0] is the fastest mode
+        st, run = [0] * len(labels), 1
+        padded = int(rng.integers(0, len(labels))) if labels else -1
+        for pos, mode in enumerate(order):
+            st[mode] = run
+            run *= extents[labels[mode]] + (int(rng.integers(0, 4)) if pos == padded else 0)
+        if allow_negative:
+            st = [-x if rng.random() < 0.25 else x for x in st]
+        return tuple(st)
+    return la, lb, ld, extents, strides_for(la, True), strides_for(lb, True), strides_for(ld, False)

@@ -104,6 +104,26 @@ def test_paper_test_categories(api, handle, cat, dtype):
     assert worst <= 1.0, worst
 
 
+@pytest.mark.parametrize("seed", range(64))
+def test_seeded_random_contractions(api, handle, seed):
+    """Randomized set (the paper plans randomized benchmarks; these are seeded stand-ins): random numbers
+    of batch, free and contracted labels (rank 0-8), mixed extents including 1, every tensor in its own
+    memory order with padding, negative strides in A and B, all four element types in turn, whatever
+    kernel the planner picks; padding bytes of D must stay untouched."""
+    la, lb, ld, ext, sA, sB, sD = inputs.random_contraction(9000 + seed)
+    dtype = REAL_AND_COMPLEX[seed % len(REAL_AND_COMPLEX)]
+    A = helpers.random_tensor(3 * seed + 1, _ext(la, ext), sA, dtype)
+    B = helpers.random_tensor(3 * seed + 2, _ext(lb, ext), sB, dtype)
+    C = helpers.random_tensor(3 * seed + 3, _ext(ld, ext), sD, dtype)
+    D = inputs.place(None, _ext(ld, ext), sD, dtype)
+    cplx = dtype.is_complex
+    alpha = complex(1.25, -0.5) if cplx else 1.25
+    beta = (complex(0.5, 0.75) if cplx else 0.5) if seed % 3 else 0.0
+    worst, _, _ = helpers.run_case(handle, A, la, B, lb, C if seed % 3 else None, D, ld, alpha, beta,
+                                   conjA=cplx and seed % 2 == 0, conjB=cplx and seed % 4 == 1)
+    assert worst <= 1.0, (worst, la, lb, ld, ext)
+
+
 @pytest.mark.parametrize("dtype", [torch.float64, torch.complex128, torch.float32])
 @pytest.mark.parametrize("kernel", ["auto", "generic"])
 def test_strides_negative_zero_padded_subtensor(api, handle, dtype, kernel):
