@@ -64,7 +64,7 @@ def roofline_for(w, kernel_ms, variant=-1):
                 "peak_source": "FP64 tensor (DMMA) pipe: 148 SMs x 64 FMA/clk x 2 x 1.965 GHz; "
                                "a register-resident DMMA loop measured 37.1 TFLOP/s on this pool",
                 "kernel": "tiled_f64_kernel", "kernel_ms": kernel_ms}
-    if variant >= 10:
+    if 10 <= variant <= 21:
         # tcgen05 3xTF32: three TF32 MMAs per product.  TF32 dense peak = measured bf16 burst peak x
         # the nominal TF32 : bf16 ratio (1.1 : 2.25).  Whichever of the tensor pipe and HBM needs
         # longer for this workload is the bound.
@@ -90,7 +90,7 @@ def roofline_for(w, kernel_ms, variant=-1):
             "note": "this fp32 kernel computes each product as three TF32 tensor-core MMAs "
                     "(mma.sync m16n8k8, measured peak 277 TFLOP/s on this pool): it executes "
                     f"{3 * achieved:.1f} tensor TFLOP/s = {3 * achieved / 277.0:.2f} of that peak",
-            "kernel": "tiled_tf32x3_kernel" if variant >= 6 else "tiled_f32_kernel", "kernel_ms": kernel_ms}
+            "kernel": "tiled_tf32x3_kernel" if (6 <= variant <= 9 or variant == 22) else "tiled_f32_kernel", "kernel_ms": kernel_ms}
 
 
 def parse():
@@ -103,6 +103,8 @@ def parse():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--variant", type=int, default=-1, help="force a tile variant (tuning runs)")
+    ap.add_argument("--batched", type=int, default=0,
+                    help="one step = one btc_execute_batched call over this many distinct (A, B, D) buffer sets")
     return ap.parse_args()
 
 
@@ -320,6 +322,66 @@ def run_elementwise(args, w):
                      "kernel_ms": ms}}))
 
 
+def run_batched(args, w):
+    """`--batched N`: N distinct buffer sets of the workload (more than L2 together for the small
+    workloads), one pointer-array call per step: the device-side rate of a small contraction
+    without the per-call launch latency."""
+    import torch
+    from paper_2601_07827_b200 import build, inputs
+    build.build()
+    from paper_2601_07827_b200 import api
+    torch.cuda.set_device(0)
+    n = args.batched
+    A, B, C, D = inputs.make_workload_tensors(w, device="cuda")
+    rep = lambda t: torch.stack([t.buffer] * n).contiguous()
+    pA, pB, pD = rep(A), rep(B), rep(D)
+    pC = rep(C) if (C is not None and not w.in_place) else None
+    handle = api.Handle()
+    dt = api.dtype_code(D.dtype)
+    tA = api.TensorInfo(handle, dt, A.extents, A.strides)
+    tB = api.TensorInfo(handle, dt, B.extents, B.strides)
+    tD = api.TensorInfo(handle, dt, D.extents, D.strides)
+    op = api.Contraction(handle, tA, w.labelsA, tB, w.labelsB, tD if C is not None else None, w.labelsD, tD, w.labelsD,
+                         w.alpha, w.beta, w.conjA, w.conjB, w.conjC)
+    op.set_attr(api.ATTR_BATCH_HINT, n)
+    if args.variant >= 0:
+        op.set_attr(api.ATTR_VARIANT, args.variant)
+    item = D.buffer.element_size()
+    ptrs = lambda pool, t: [pool.data_ptr() + (i * t.buffer.numel() + t.origin) * item for i in range(n)]
+    lA, lB, lD = ptrs(pA, A), ptrs(pB, B), ptrs(pD, D)
+    lC = None if C is None else (lD if w.in_place else ptrs(pC, C))
+    ws_bytes = op.batched_workspace_size(n)
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    step = lambda: op.execute_batched(stream.cuda_stream, lA, lB, lC, lD, workspace=ws.data_ptr(), workspace_bytes=ws_bytes)
+    for _ in range(max(1, args.warmup)):
+        step()
+    sampler = ClockSampler(0)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    gbs = n * w.algorithmic_bytes() / (ms * 1e-3) / 1e9
+    peak, src = measured_hbm_gbs()
+    total_bytes = n * w.algorithmic_bytes()
+    print(json.dumps({
+        "metric": METRIC, "value": n * w.flops() / (ms * 1e-3) / 1e9, "unit": "GFLOP/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "batched_entries": n, "us_per_entry": 1e3 * ms / n, "kernel": op.kernel,
+                   "tile": list(op.tile), "variant": op.variant, "split_k": op.split_k,
+                   "l2": "buffer sets exceed L2" if total_bytes > 126e6 else "buffer sets fit in L2"},
+        "clocks": clocks, "gpu_launches": args.steps * (2 if op.split_k > 1 else 1),
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
+                     "peak_source": f"STREAM-style copy, {src}", "kernel_ms": ms}}))
+
+
 def main():
     args = parse()
     from paper_2601_07827_b200 import inputs
@@ -329,6 +391,9 @@ def main():
         run_elementwise(args, inputs.elementwise_workloads()[args.workload])
         return
     w = inputs.workloads()[args.workload]
+    if args.batched > 0 and args.impl != "reference":
+        run_batched(args, w)
+        return
     if args.impl == "reference":
         run_reference(args, w)
         return

@@ -127,6 +127,10 @@ enum {
     BTC_ATTR_DEVICE_ERROR = 8,/* int32, read: 0, or which bounded device-side wait gave up in an
                                  earlier execute of this operation (its D is then incomplete);
                                  reading waits for the device                                  */
+    BTC_ATTR_BATCH_HINT = 11, /* int32 >= 1, read/write (write re-plans): how many pointer-array entries
+                                 btc_execute_batched will usually be given.  Tile variant and split-K
+                                 are then chosen for that many entries in flight (no split-K when the
+                                 array alone fills the GPU); any count still works with any hint    */
     BTC_ATTR_PRE_REDUCE = 10  /* int32.  Case 4 of Sec. "Operations": labels that occur in one input
                                  only are summed over before the contraction.  Write 1 (default):
                                  a separate bandwidth-bound kernel forms the summed input in the
@@ -168,6 +172,25 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream,
 btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream,
                              const void *alpha, const void *A, const void *B,
                              const void *beta, const void *C, void *D);
+
+/* Batched execution with pointer arrays (Sec. "Tensor Descriptors": descriptors hold no data pointer
+ * so that one description serves many tensors, "in particular for batched tensor operations").
+ * Executes the operation `count` times, entry i on A[i], B[i], C[i], D[i]; alpha and beta are shared.
+ *   A, B, C, D   HOST arrays of `count` DEVICE pointers (each as in btc_execute; C may be NULL when
+ *                beta == 0).  Entries must not overlap one another's D.
+ *   workspace    DEVICE memory, 256-byte aligned, btc_contraction_batched_workspace_size(count) bytes
+ * Plans that run the tiled kernels serve the whole array with ONE launch (plus one split-K reduce):
+ * the pointer array acts as a further batch dimension whose offsets are uploaded into the workspace
+ * (a small host-to-device copy on the stream).  That path needs C[i] - C[0] == D[i] - D[0] for all i
+ * (true for in-place updates and for C, D carved alike out of two pools) and returns NOT_SUPPORTED
+ * otherwise.  Generic-kernel and Case 4 plans are executed entry by entry in stream order.
+ * Nothing is allocated on the device; the call does not synchronise.
+ * Errors: as btc_execute. */
+btc_error_t btc_contraction_batched_workspace_size(btc_contraction_t op, int64_t count, size_t *bytes);
+btc_error_t btc_execute_batched(btc_contraction_t op, void *cuda_stream, const void *alpha,
+                                const void *const *A, const void *const *B, const void *beta,
+                                const void *const *C, void *const *D, int64_t count,
+                                void *workspace, size_t workspace_bytes);
 
 /* Execute without allocating anything (the paper has no counterpart; this is a convenience of
  * this library).  Same operation and argument meaning as btc_execute with DEVICE pointers, but

@@ -41,6 +41,7 @@ ATTR_KERNEL, ATTR_SPLIT_K, ATTR_TILE, ATTR_GROUPS, ATTR_GRID, ATTR_NUM_MODES, AT
 ATTR_DEVICE_ERROR = 8
 ATTR_VARIANT = 9
 ATTR_PRE_REDUCE = 10
+ATTR_BATCH_HINT = 11
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TILED = 0, 1, 2
 STATUS_KERNEL, STATUS_LAUNCHES, STATUS_GRID, STATUS_SPLIT_K, STATUS_VARIANT = 1, 2, 3, 4, 5
 
@@ -48,6 +49,7 @@ EXPORTED = [
     "btc_create_handle", "btc_destroy_handle", "btc_create_tensor_info", "btc_destroy_tensor_info",
     "btc_create_contraction", "btc_destroy_contraction", "btc_contraction_workspace_size",
     "btc_set_attr", "btc_get_attr", "btc_execute", "btc_execute_host", "btc_execute_static_scratch",
+    "btc_execute_batched", "btc_contraction_batched_workspace_size",
     "btc_status_get",
     "btc_destroy_status", "btc_explain_error", "btc_selftest_bounded_wait",
     "btc_create_elementwise", "btc_destroy_elementwise", "btc_elementwise_execute", "btc_elementwise_get_attr",
@@ -68,6 +70,9 @@ _lib.btc_set_attr.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t]
 _lib.btc_get_attr.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
 _lib.btc_execute.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, ctypes.POINTER(_vp)]
 _lib.btc_execute_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.btc_contraction_batched_workspace_size.argtypes = [_vp, ctypes.c_int64, ctypes.POINTER(ctypes.c_size_t)]
+_lib.btc_execute_batched.argtypes = [_vp, _vp, _vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp, ctypes.POINTER(_vp),
+                                     ctypes.POINTER(_vp), ctypes.c_int64, _vp, ctypes.c_size_t]
 _lib.btc_execute_static_scratch.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.btc_status_get.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t]
 _lib.btc_destroy_status.argtypes = [ctypes.POINTER(_vp)]
@@ -262,6 +267,21 @@ class Contraction:
             _lib.btc_destroy_status(ctypes.byref(st))
             return out
         return None
+
+    def batched_workspace_size(self, count: int) -> int:
+        n = ctypes.c_size_t(0)
+        _check(_lib.btc_contraction_batched_workspace_size(self._op, count, ctypes.byref(n)),
+               "btc_contraction_batched_workspace_size")
+        return int(n.value)
+
+    def execute_batched(self, stream: int, A: Sequence[int], B: Sequence[int], C: Optional[Sequence[int]], D: Sequence[int],
+                        alpha=None, beta=None, workspace: int = 0, workspace_bytes: int = 0) -> None:
+        """Pointer arrays (device pointers as integers), one entry per execution; see btc_execute_batched."""
+        n = len(D)
+        arr = lambda ps: (_vp * n)(*[p or None for p in ps]) if ps is not None else None
+        _check(_lib.btc_execute_batched(self._op, stream or None, _scalar(self.dtype, alpha), arr(A), arr(B),
+                                        _scalar(self.dtype, beta), arr(C), arr(D), n, workspace or None, workspace_bytes),
+               "btc_execute_batched")
 
     def execute_host(self, stream: int, A: int, B: int, C: Optional[int], D: int, alpha=None, beta=None):
         """Host pointers as integers; copies in, runs, copies D back, synchronises."""

@@ -94,6 +94,7 @@ using F32WideP = F32Tile<256, 96, 16, 4, 2, 5, 1, true>;
 using F32Big32 = F32Tile<128, 128, 32, 2, 4, 3, 1, false>;
 using F32Tc = TF32Tile<false, 128, 128, 2, 4, 4, 1>;             // 3xTF32 on the tensor cores
 using F32TcSmall = TF32Tile<false, 64, 64, 2, 4, 4, 2>;
+using F32TcTiny = TF32Tile<false, 64, 64, 2, 4, 2, 3>;            // two stages, three CTAs per SM: short-K, low-intensity problems
 using C32Tc = TF32Tile<true, 128, 64, 2, 4, 4, 1>;
 using C32TcSmall = TF32Tile<true, 64, 32, 2, 4, 4, 2>;
 using F32TcWide = TF32Tile<false, 256, 96, 4, 2, 4, 1>;          // N = 96 fills the tile exactly
@@ -111,7 +112,7 @@ using F32Umma96B32 = UmmaTile<96, 5, 2, true, 1, 32, true>;
 using F32Umma128B32 = UmmaTile<128, 4, 2, true, 1, 32, true>;
 using F32Umma128B24 = UmmaTile<128, 5, 2, true, 1, 24, true>;
 using F32Umma96B24x2 = UmmaTile<96, 3, 2, true, 1, 24, true, 2>;   // two sub-stages of 24 k per hand-off
-constexpr int kNumF32Variants = 22;
+constexpr int kNumF32Variants = 23;
 constexpr int kFirstUmmaVariant = 10;
 constexpr int kFirstBulkVariant = 17;     // 17..21: bulk tensor copies; fall back to 13 / 14 (same tiles) at execute
 
@@ -161,6 +162,7 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
         case 19: return {128, 128, 32, 256, 0, F32Umma128B32::SMEM_BYTES, 4};
         case 20: return {128, 128, 24, 256, 0, F32Umma128B24::SMEM_BYTES, 4};
         case 21: return {128, 96, 24, 256, 0, F32Umma96B24x2::SMEM_BYTES, 4};
+        case 22: return info_of<F32TcTiny>(4);
         default: return {128, 128, 32, 256, 0, F32Umma128T2::SMEM_BYTES, 4};
         }
     }
@@ -327,6 +329,9 @@ int finish_plan(btc_contraction_s *op)
     auto tiles_for = [&](const VariantInfo &v) {
         return ((pl.M + v.bm - 1) / v.bm) * ((pl.N + v.bn - 1) / v.bn) * pl.Bt;
     };
+    // tiles in flight at a time when the operation runs over a pointer array (BTC_ATTR_BATCH_HINT):
+    // what tile choice and split-K are judged by; grid and workspace stay those of one entry
+    const int64_t hint = op->req.batch_hint > 1 ? op->req.batch_hint : 1;
     // Candidate tile variants of the element type (fp32: the 3xTF32 tensor-core variants, mma.sync
     // or tcgen05; the strict-fp32 FFMA variants 0-5 are selected with BTC_ATTR_VARIANT only).  Score = fraction of
     // the padded tiles that is real work x fraction of the last wave that is filled x a mild
@@ -339,7 +344,7 @@ int finish_plan(btc_contraction_s *op)
         // enter only when there is enough work to fill the SMs without split-K; their weights
         // reflect measured throughput relative to the mma.sync variants.
         const double flops = 2.0 * double(pl.M) * double(pl.N) * double(pl.K) * double(pl.Bt);
-        const bool umma_ok = pl.dtype == BTC_F32 && flops >= 2e9 && pl.K >= 64;
+        const bool umma_ok = pl.dtype == BTC_F32 && flops * double(hint) >= 2e9 && pl.K >= 64;
         // 17-20 fetch the M side with bulk tensor copies; they enter when that operand is a tensor of boxes
         TmaOperand probe;
         const bool box24 = umma_ok && make_tma_operand(pl, 128, 24, probe), box32 = umma_ok && make_tma_operand(pl, 128, 32, probe);
@@ -356,10 +361,10 @@ int finish_plan(btc_contraction_s *op)
         double best = -1.0;
         for (int c = 0; c < ncand; ++c) {
             const VariantInfo vi = variant_info(pl.dtype, cands[c].id);
-            const double tiles = double(tiles_for(vi));
+            const double tiles = double(tiles_for(vi)) * double(hint);
             const double ctas_per_sm = vi.bm * vi.bn <= 64 * 64 ? 2.0 : 1.0;
             const double slots = sms * ctas_per_sm;
-            const double util = double(pl.M) * double(pl.N) * double(pl.Bt) / (tiles * vi.bm * vi.bn);
+            const double util = double(pl.M) * double(pl.N) * double(pl.Bt) * double(hint) / (tiles * vi.bm * vi.bn);
             const double waves = std::ceil(tiles / slots);
             const double wave_eff = tiles / (waves * slots);
             const double score = util * wave_eff * cands[c].weight;
@@ -372,7 +377,7 @@ int finish_plan(btc_contraction_s *op)
         variant = op->req.force_variant;
     }
     op->tmaA = TmaOperand();
-    if (pl.dtype == BTC_F32 && variant >= kFirstBulkVariant) {
+    if (pl.dtype == BTC_F32 && variant >= kFirstBulkVariant && variant <= 21) {
         // a forced bulk-copy variant whose M-side operand is no tensor of boxes: the gathering twin
         const VariantInfo bv = variant_info(pl.dtype, variant);
         if (!make_tma_operand(pl, bv.bm, bv.bk, op->tmaA)) variant = (variant <= 18 || variant == 21) ? 13 : 14;
@@ -386,13 +391,13 @@ int finish_plan(btc_contraction_s *op)
     const int64_t tiles = tiles_for(v);
     const int64_t k_tiles = (pl.K + v.bk - 1) / v.bk;
     int64_t split = 1;
-    const bool umma = pl.dtype == BTC_F32 && variant >= kFirstUmmaVariant;   // these keep all of K in one CTA
+    const bool umma = pl.dtype == BTC_F32 && variant >= kFirstUmmaVariant && variant <= 21;   // these keep all of K in one CTA
     if (umma) {
         split = 1;
     } else if (op->req.force_split_k > 0) {
         split = op->req.force_split_k;
-    } else if (tiles < sms) {
-        split = (2 * int64_t(sms)) / tiles;
+    } else if (tiles * hint < sms) {
+        split = (2 * int64_t(sms)) / (tiles * hint);
         const int64_t max_split = k_tiles / 2;   // at least two K tiles per slice
         if (split > max_split) split = max_split;
     } else {
@@ -400,9 +405,9 @@ int finish_plan(btc_contraction_s *op)
         // last wave fuller.  Cost model in units of one unsplit tile: waves / slices, plus the
         // partial images' round trip through memory (about 50 elements' worth of work per slice).
         const double slots = double(sms) * (v.bm * v.bn <= 64 * 64 ? 2.0 : 1.0);
-        double best = std::ceil(double(tiles) / slots);
+        double best = std::ceil(double(tiles * hint) / slots);
         for (int64_t sl = 2; sl <= 4 && k_tiles / sl >= 16; ++sl) {
-            const double t = std::ceil(double(tiles * sl) / slots) / double(sl) * (1.0 + 50.0 * double(sl) / double(pl.K));
+            const double t = std::ceil(double(tiles * hint * sl) / slots) / double(sl) * (1.0 + 50.0 * double(sl) / double(pl.K));
             if (t < 0.97 * best) { best = t; split = sl; }
         }
     }
@@ -688,6 +693,9 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
     } else if (key == BTC_ATTR_SPLIT_K) {
         if (v < 0) return BTC_ERR_INVALID_ARGUMENT;
         op->req.force_split_k = v;
+    } else if (key == BTC_ATTR_BATCH_HINT) {
+        if (v < 1) return BTC_ERR_INVALID_ARGUMENT;
+        op->req.batch_hint = v;
     } else {
         return BTC_ERR_INVALID_ARGUMENT;
     }
@@ -720,6 +728,7 @@ btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t 
     case BTC_ATTR_SWAPPED: i32[0] = pl.swapped ? 1 : 0; n = 4; break;
     case BTC_ATTR_VARIANT: i32[0] = pl.tile.variant; n = 4; break;
     case BTC_ATTR_PRE_REDUCE: i32[0] = (op->sumA.active ? 1 : 0) | (op->sumB.active ? 2 : 0); n = 4; break;
+    case BTC_ATTR_BATCH_HINT: i32[0] = op->req.batch_hint; n = 4; break;
     case BTC_ATTR_DEVICE_ERROR:
         i32[0] = 0;
         if (op->d_error) {
@@ -739,9 +748,32 @@ btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t 
     return BTC_SUCCESS;
 }
 
+namespace {
+// Pointer-array batch seen by the tiled kernels: `count` times the operation's own batch entries,
+// with offset tables (elements, relative to entry 0's pointers) that live in the caller's workspace.
+struct BatchView {
+    int64_t count;
+    const int64_t *offA_h, *offB_h, *offD_h;   // [count * Bt], planned roles
+    void *partials;
+    bool aligned16_D, aligned_A, aligned_B;     // every entry's pointer keeps the vector alignment
+};
+
+btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A, const void *B,
+                         const void *beta, const void *C, void *D, void *workspace, size_t workspace_bytes,
+                         btc_status_t *status, const BatchView *bv);
+}  // namespace
+
 btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A, const void *B,
                         const void *beta, const void *C, void *D, void *workspace, size_t workspace_bytes,
                         btc_status_t *status)
+{
+    return execute_impl(op, cuda_stream, alpha, A, B, beta, C, D, workspace, workspace_bytes, status, nullptr);
+}
+
+namespace {
+btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A, const void *B,
+                         const void *beta, const void *C, void *D, void *workspace, size_t workspace_bytes,
+                         btc_status_t *status, const BatchView *bv)
 {
     if (!op || !D) return BTC_ERR_INVALID_ARGUMENT;
     if (op->handle.device < 0) return BTC_ERR_CUDA;   // no device: nothing can run, and nothing else will
@@ -758,7 +790,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
     const size_t need = pl.dtype == BTC_C64 ? 16 : (pl.dtype == BTC_C32 ? 8 : part);
     if (misaligned(A, need) || misaligned(B, need) || misaligned(C, need) || misaligned(D, need))
         return BTC_ERR_MISALIGNED;
-    if (op->workspace_bytes > 0) {
+    if (op->workspace_bytes > 0 && !bv) {        // a pointer-array batch has checked its own layout
         if (!workspace || workspace_bytes < op->workspace_bytes) return BTC_ERR_WORKSPACE_TOO_SMALL;
         if (misaligned(workspace, 256)) return BTC_ERR_MISALIGNED;
     }
@@ -829,8 +861,8 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         tp.split_k = pl.split_k; tp.k_per_split = op->k_per_split;
         tp.dirA = int32_t(pl.dirA); tp.dirB = int32_t(pl.dirB);
         // vector copies need the base pointers aligned as well
-        tp.vecA = misaligned(pA, size_t(pl.alignA)) ? 1 : pl.vecA;
-        tp.vecB = misaligned(pB, size_t(pl.alignB)) ? 1 : pl.vecB;
+        tp.vecA = (misaligned(pA, size_t(pl.alignA)) || (bv && !bv->aligned_A)) ? 1 : pl.vecA;
+        tp.vecB = (misaligned(pB, size_t(pl.alignB)) || (bv && !bv->aligned_B)) ? 1 : pl.vecB;
         tp.conjA = pl.conjA; tp.conjB = pl.conjB; tp.conjC = pl.conjC;
         tp.use_c = use_c;
         tp.alpha[0] = al[0]; tp.alpha[1] = al[1]; tp.beta[0] = be[0]; tp.beta[1] = be[1];
@@ -840,10 +872,21 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
 #ifdef BTC_STAMPS
         { void *sp = nullptr; cudaGetSymbolAddress(&sp, btc_stamp_buffer); tp.stamps = static_cast<long long *>(sp); }
 #endif
-        const int64_t ctas = op->grid[0];
-        const int64_t reduce_ctas = (ctas / pl.split_k) * ((int64_t(pl.tile.bm) * pl.tile.bn + 1023) / 1024);
+        int64_t ctas = op->grid[0];
+        int64_t reduce_ctas = (ctas / pl.split_k) * ((int64_t(pl.tile.bm) * pl.tile.bn + 1023) / 1024);
         // 16-byte stores of D (and loads of C) need those base pointers aligned too
-        tp.vecD = (pl.vecD == 4 && !misaligned(D, 16) && !(use_c && misaligned(C, 16))) ? 4 : 1;
+        tp.vecD = (pl.vecD == 4 && !misaligned(D, 16) && !(use_c && misaligned(C, 16)) && !(bv && !bv->aligned16_D)) ? 4 : 1;
+        const bool persistent = pl.dtype == BTC_F32 && pl.tile.variant >= kFirstUmmaVariant && pl.tile.variant <= 21;
+        if (bv) {
+            // the pointer array multiplies the batch entries; everything else of the plan stands
+            tp.Bt = pl.Bt * bv->count;
+            tp.offA_h = bv->offA_h; tp.offB_h = bv->offB_h; tp.offD_h = bv->offD_h;
+            tp.partials = bv->partials;
+            const int64_t work = int64_t(op->tiles_m) * op->tiles_n * pl.split_k * tp.Bt;
+            if (work > 0x7fffffffLL) return BTC_ERR_NOT_SUPPORTED;
+            ctas = persistent ? (work < op->handle.sm_count ? work : op->handle.sm_count) : work;
+            reduce_ctas = (work / pl.split_k) * ((int64_t(pl.tile.bm) * pl.tile.bn + 1023) / 1024);
+        }
         if (pl.dtype == BTC_F32) {
             switch (pl.tile.variant) {
             case 0: ce = launch_tiled_f32<F32Big>(tp, ctas, reduce_ctas, st); break;
@@ -854,6 +897,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
             case 5: ce = launch_tiled_f32<F32Big32>(tp, ctas, reduce_ctas, st); break;
             case 6: ce = launch_tiled_tf32<F32Tc>(tp, ctas, reduce_ctas, st); break;
             case 7: ce = launch_tiled_tf32<F32TcSmall>(tp, ctas, reduce_ctas, st); break;
+            case 22: ce = launch_tiled_tf32<F32TcTiny>(tp, ctas, reduce_ctas, st); break;
             case 8: ce = launch_tiled_tf32<F32TcWide>(tp, ctas, reduce_ctas, st); break;
             case 9: ce = launch_tiled_tf32<F32TcMid>(tp, ctas, reduce_ctas, st); break;
             case 10: ce = launch_umma<F32Umma96>(tp, ctas, st); break;
@@ -868,7 +912,7 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
                 // otherwise the gathering variant with the same tile runs
                 CUtensorMap mapA;
                 const int v = pl.tile.variant;
-                if (misaligned(pA, 16) || !encode_tma_operand(op->tmaA, pA, &mapA)) {
+                if (bv || misaligned(pA, 16) || !encode_tma_operand(op->tmaA, pA, &mapA)) {   // (a pointer array is no box dimension)
                     ran_variant = (v <= 18 || v == 21) ? 13 : 14;
                     ce = ran_variant == 13 ? launch_umma<F32Umma96T>(tp, ctas, st) : launch_umma<F32Umma128T>(tp, ctas, st);
                 }
@@ -908,6 +952,92 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
         *status = s;
     }
     return BTC_SUCCESS;
+}
+
+// one launch serves the whole pointer array: tiled plan, both inputs read as they are
+bool batch_in_one_launch(const btc_contraction_s *op)
+{
+    return op->plan.kernel == BTC_KERNEL_TILED && !op->sumA.active && !op->sumB.active;
+}
+size_t batch_tables_bytes(const btc_contraction_s *op, int64_t count)
+{
+    return (size_t(3) * size_t(count) * size_t(op->plan.Bt) * sizeof(int64_t) + 255) / 256 * 256;
+}
+}  // namespace
+
+btc_error_t btc_contraction_batched_workspace_size(btc_contraction_t op, int64_t count, size_t *bytes)
+{
+    if (!op || !bytes || count < 1) return BTC_ERR_INVALID_ARGUMENT;
+    if (!batch_in_one_launch(op)) { *bytes = op->workspace_bytes; return BTC_SUCCESS; }
+    *bytes = batch_tables_bytes(op, count) + (op->workspace_bytes - op->partials_offset) * size_t(count);
+    return BTC_SUCCESS;
+}
+
+btc_error_t btc_execute_batched(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *const *A,
+                                const void *const *B, const void *beta, const void *const *C, void *const *D,
+                                int64_t count, void *workspace, size_t workspace_bytes)
+{
+    if (!op || !D || count < 1) return BTC_ERR_INVALID_ARGUMENT;
+    if (op->handle.device < 0) return BTC_ERR_CUDA;
+    const Plan &pl = op->plan;
+    double al[2] = {op->alpha[0], op->alpha[1]}, be[2] = {op->beta[0], op->beta[1]};
+    if (alpha) to_double2(pl.dtype, alpha, al);
+    if (beta) to_double2(pl.dtype, beta, be);
+    const bool use_ab = !is_zero(al), use_c = !is_zero(be);
+    if ((use_ab && (!A || !B)) || (use_c && !C)) return BTC_ERR_INVALID_ARGUMENT;
+    for (int64_t i = 0; i < count; ++i)
+        if (!D[i] || (use_ab && (!A[i] || !B[i])) || (use_c && !C[i])) return BTC_ERR_INVALID_ARGUMENT;
+    size_t need = 0;
+    btc_contraction_batched_workspace_size(op, count, &need);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return BTC_ERR_WORKSPACE_TOO_SMALL;
+    if (need > 0 && reinterpret_cast<uintptr_t>(workspace) % 256) return BTC_ERR_MISALIGNED;
+
+    if (!batch_in_one_launch(op) || !use_ab) {
+        // generic-kernel and Case 4 plans: one execute per entry, in order on the stream
+        for (int64_t i = 0; i < count; ++i) {
+            const btc_error_t rc = execute_impl(op, cuda_stream, alpha, use_ab ? A[i] : nullptr, use_ab ? B[i] : nullptr, beta,
+                                                use_c ? C[i] : nullptr, D[i], workspace, workspace_bytes, nullptr, nullptr);
+            if (rc != BTC_SUCCESS) return rc;
+        }
+        return BTC_SUCCESS;
+    }
+
+    // offsets of every entry relative to entry 0, in elements, added to the operation's own batch offsets
+    const int64_t esz = int64_t(dtype_size(pl.dtype));
+    const int64_t Bt = pl.Bt;
+    std::vector<int64_t> tab(size_t(3) * size_t(count) * size_t(Bt));
+    int64_t *tA = tab.data(), *tB = tA + count * Bt, *tD = tB + count * Bt;
+    BatchView bv;
+    bv.count = count;
+    bv.aligned16_D = bv.aligned_A = bv.aligned_B = true;
+    const void *const *pA = pl.swapped ? B : A, *const *pB = pl.swapped ? A : B;
+    for (int64_t i = 0; i < count; ++i) {
+        const int64_t dA = reinterpret_cast<intptr_t>(pA[i]) - reinterpret_cast<intptr_t>(pA[0]);
+        const int64_t dB = reinterpret_cast<intptr_t>(pB[i]) - reinterpret_cast<intptr_t>(pB[0]);
+        const int64_t dD = reinterpret_cast<intptr_t>(D[i]) - reinterpret_cast<intptr_t>(D[0]);
+        if (dA % esz || dB % esz || dD % esz) return BTC_ERR_MISALIGNED;
+        // C travels with D: one offset table serves both, so C[i] - C[0] must equal D[i] - D[0]
+        if (use_c && reinterpret_cast<intptr_t>(C[i]) - reinterpret_cast<intptr_t>(C[0]) != dD) return BTC_ERR_NOT_SUPPORTED;
+        bv.aligned_A = bv.aligned_A && reinterpret_cast<uintptr_t>(pA[i]) % size_t(pl.alignA) == 0;
+        bv.aligned_B = bv.aligned_B && reinterpret_cast<uintptr_t>(pB[i]) % size_t(pl.alignB) == 0;
+        bv.aligned16_D = bv.aligned16_D && reinterpret_cast<uintptr_t>(D[i]) % 16 == 0 &&
+                         (!use_c || reinterpret_cast<uintptr_t>(C[i]) % 16 == 0);
+        for (int64_t h = 0; h < Bt; ++h) {
+            tA[i * Bt + h] = pl.offA_h[size_t(h)] + dA / esz;
+            tB[i * Bt + h] = pl.offB_h[size_t(h)] + dB / esz;
+            tD[i * Bt + h] = pl.offD_h[size_t(h)] + dD / esz;
+        }
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int64_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return BTC_ERR_CUDA;
+    }
+    const int64_t *dtab = static_cast<const int64_t *>(workspace);
+    bv.offA_h = dtab; bv.offB_h = dtab + count * Bt; bv.offD_h = dtab + 2 * count * Bt;
+    bv.partials = static_cast<char *>(workspace) + batch_tables_bytes(op, count);
+    return execute_impl(op, cuda_stream, alpha, A[0], B[0], beta, use_c ? C[0] : nullptr, D[0], workspace, workspace_bytes,
+                        nullptr, &bv);
 }
 
 btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A,

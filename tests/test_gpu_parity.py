@@ -232,7 +232,7 @@ def test_unaligned_base_pointer_falls_back_to_element_copies(api, handle):
     assert worst <= 1.0
 
 
-@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(22)]
+@pytest.mark.parametrize("dtype,variant", [(torch.float64, v) for v in range(5)] + [(torch.float32, v) for v in range(23)]
                          + [(torch.complex128, v) for v in range(3)] + [(torch.complex64, v) for v in range(2)])
 def test_every_tile_variant(api, handle, dtype, variant):
     """Each tile variant of the tiled kernels, forced through the attribute, on a ragged multi-tile case
