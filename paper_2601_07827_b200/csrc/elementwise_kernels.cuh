@@ -46,7 +46,7 @@ template <typename R, bool CPLX, int LANES, typename I>
 __device__ __forceinline__ void elementwise_sum(const ElementwiseParams &p, int64_t base, int lane, double &acc_r, double &acc_i)
 {
     constexpr int NC = CPLX ? 2 : 1;
-    constexpr int U = 4;
+    constexpr int U = LANES == 1 ? 8 : 4;   // loads in flight per thread (16 spill: 4x slower)
     const R *A = static_cast<const R *>(p.A);
     acc_r = acc_i = 0.0;
     if (!p.use_a) return;
