@@ -175,45 +175,57 @@ __global__ void __launch_bounds__(256) elementwise_vector_kernel(const Elementwi
     const int64_t nvec = p.total_keep / V;
     const int64_t stride = int64_t(gridDim.x) * blockDim.x;
     const R sgnA = (CPLX && p.conjA) ? R(-1) : R(1), sgnB = (CPLX && p.conjB) ? R(-1) : R(1);
-    for (int64_t v = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; v < nvec; v += stride) {
-        int64_t offA = 0, offB = 0, offC = 0;
-        I lin = I(v);
-        {
-            const I ext = I(p.ext_k[0] / V);
-            const I q = lin / ext;
-            const int64_t i = int64_t(lin - q * ext) * V;
-            lin = q;
-            offA = i * p.sA_k[0]; offB = i * p.sB_k[0]; offC = i;
-        }
-        for (int d = 1; d < p.nk; ++d) {
-            const I ext = I(p.ext_k[d]);
-            const I q = lin / ext;
-            const int64_t i = int64_t(lin - q * ext);
-            lin = q;
-            offA += i * p.sA_k[d];
-            offB += i * p.sB_k[d];
-            offC += i * p.sC_k[d];
-        }
-        Pack a, b, c;
-        a.raw = make_uint4(0, 0, 0, 0);
-        b.raw = make_uint4(0, 0, 0, 0);
-        if (p.use_a) a.raw = *reinterpret_cast<const uint4 *>(A + NC * offA);
-        if (p.use_b) b.raw = *reinterpret_cast<const uint4 *>(B + NC * offB);
+    typedef typename ElementwiseScalar<R>::type S;
+    const S al_r = S(p.alpha[0]), al_i = S(p.alpha[1]), be_r = S(p.beta[0]), be_i = S(p.beta[1]);
+    constexpr int U = 4;                                 // vectors in flight per thread
+    for (int64_t v0 = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; v0 < nvec; v0 += int64_t(U) * stride) {
+        int64_t offA[U], offB[U], offC[U];
+        bool in[U];
 #pragma unroll
-        for (int e = 0; e < V; ++e) {
-            const double ar = p.use_a ? double(a.w[NC * e]) : 0.0;
-            const double ai = (CPLX && p.use_a) ? double(sgnA * a.w[NC * e + (NC - 1)]) : 0.0;
-            double c_r = p.alpha[0] * ar - p.alpha[1] * ai, c_i = p.alpha[0] * ai + p.alpha[1] * ar;
-            if (p.use_b) {
-                const double br = double(b.w[NC * e]);
-                const double bi = CPLX ? double(sgnB * b.w[NC * e + (NC - 1)]) : 0.0;
-                c_r += p.beta[0] * br - p.beta[1] * bi;
-                c_i += p.beta[0] * bi + p.beta[1] * br;
+        for (int u = 0; u < U; ++u) {
+            const int64_t v = v0 + int64_t(u) * stride;
+            in[u] = v < nvec;
+            I lin = I(in[u] ? v : 0);
+            const I ext0 = I(p.ext_k[0] / V);
+            const I q0 = lin / ext0;
+            const int64_t i0 = int64_t(lin - q0 * ext0) * V;
+            lin = q0;
+            offA[u] = i0 * p.sA_k[0]; offB[u] = i0 * p.sB_k[0]; offC[u] = i0;
+            for (int d = 1; d < p.nk; ++d) {
+                const I ext = I(p.ext_k[d]);
+                const I q = lin / ext;
+                const int64_t i = int64_t(lin - q * ext);
+                lin = q;
+                offA[u] += i * p.sA_k[d];
+                offB[u] += i * p.sB_k[d];
+                offC[u] += i * p.sC_k[d];
             }
-            c.w[NC * e] = R(c_r);
-            if (CPLX) c.w[NC * e + (NC - 1)] = R(c_i);
         }
-        *reinterpret_cast<uint4 *>(C + NC * offC) = c.raw;
+        Pack a[U], b[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            a[u].raw = make_uint4(0, 0, 0, 0);
+            b[u].raw = make_uint4(0, 0, 0, 0);
+            if (p.use_a && in[u]) a[u].raw = *reinterpret_cast<const uint4 *>(A + NC * offA[u]);
+            if (p.use_b && in[u]) b[u].raw = *reinterpret_cast<const uint4 *>(B + NC * offB[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (!in[u]) continue;
+            Pack c;
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+                const S ar = S(a[u].w[NC * e]), br = S(b[u].w[NC * e]);
+                if (CPLX) {
+                    const S ai = S(sgnA * a[u].w[NC * e + (NC - 1)]), bi = S(sgnB * b[u].w[NC * e + (NC - 1)]);
+                    c.w[NC * e] = R(al_r * ar - al_i * ai + be_r * br - be_i * bi);
+                    c.w[NC * e + (NC - 1)] = R(al_r * ai + al_i * ar + be_r * bi + be_i * br);
+                } else {
+                    c.w[NC * e] = R(al_r * ar + be_r * br);
+                }
+            }
+            *reinterpret_cast<uint4 *>(C + NC * offC[u]) = c.raw;
+        }
     }
 }
 
