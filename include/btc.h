@@ -184,7 +184,9 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream,
  * (a small host-to-device copy on the stream).  That path needs C[i] - C[0] == D[i] - D[0] for all i
  * (true for in-place updates and for C, D carved alike out of two pools) and returns NOT_SUPPORTED
  * otherwise.  Generic-kernel and Case 4 plans are executed entry by entry in stream order.
- * Nothing is allocated on the device; the call does not synchronise.
+ * Nothing is allocated on the device.  The upload of the offsets is a copy from ordinary host memory,
+ * which the CUDA runtime may start only after earlier work on the stream has finished (and which
+ * cannot be part of a stream capture); apart from that the call does not wait for the device.
  * Errors: as btc_execute. */
 btc_error_t btc_contraction_batched_workspace_size(btc_contraction_t op, int64_t count, size_t *bytes);
 btc_error_t btc_execute_batched(btc_contraction_t op, void *cuda_stream, const void *alpha,
