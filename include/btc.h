@@ -127,6 +127,12 @@ enum {
     BTC_ATTR_DEVICE_ERROR = 8,/* int32, read: 0, or which bounded device-side wait gave up in an
                                  earlier execute of this operation (its D is then incomplete);
                                  reading waits for the device                                  */
+    BTC_ATTR_COMPUTE_PRECISION = 12, /* int32, read/write (write re-plans): BTC_PRECISION_* -- the "desired
+                                 computational precision" of Sec. "Tensor Operation Descriptors".  DEFAULT:
+                                 fp32 products are formed from three TF32 tensor-core products (error of a
+                                 product <= 2^-22 |a||b|, fp32 accumulation); STRICT: fp32 operations run on
+                                 the FMA pipe in IEEE fp32 (about a third of the speed).  No effect on fp64
+                                 and complex128 (always IEEE fp64); STRICT is NOT_SUPPORTED for complex64 */
     BTC_ATTR_BATCH_HINT = 11, /* int32 >= 1, read/write (write re-plans): how many pointer-array entries
                                  btc_execute_batched will usually be given.  Tile variant and split-K
                                  are then chosen for that many entries in flight (no split-K when the
@@ -138,6 +144,7 @@ enum {
                                  labels are summed inside the generic kernel.  Read: bit 0 / bit 1
                                  set when A / B is summed first in the current plan             */
 };
+enum { BTC_PRECISION_DEFAULT = 0, BTC_PRECISION_STRICT = 1 };
 enum {
     BTC_KERNEL_AUTO = 0,
     BTC_KERNEL_GENERIC = 1,   /* one thread per element of D, any legal input                  */

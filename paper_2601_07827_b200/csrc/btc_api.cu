@@ -353,11 +353,13 @@ int finish_plan(btc_contraction_s *op)
         const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {14, 2.3}, {13, 2.0},
                              {box24 ? 17 : 13, 1.85}, {box32 ? 18 : 13, 1.95}, {box32 ? 19 : 14, 2.25}, {box24 ? 20 : 14, 2.1},
                              {box24 ? 21 : 13, 2.04}};
+        const Cand f32strict[] = {{0, 1.0}, {2, 1.0}, {1, 0.75}};   // FFMA kernels: 128x128, 256x96, 64x64
         const Cand f64c[] = {{2, 1.0}, {1, 0.75}};       // big tile: the m16n8k16 variant
         const Cand c64c[] = {{2, 1.0}, {1, 0.75}};       // complex128: big tile on m16n8k16 as well
         const Cand other[] = {{0, 1.0}, {1, 0.75}};
-        const Cand *cands = pl.dtype == BTC_F32 ? f32c : (pl.dtype == BTC_F64 ? f64c : (pl.dtype == BTC_C64 ? c64c : other));
-        const int ncand = pl.dtype == BTC_F32 ? (umma_ok ? 12 : 4) : 2;
+        const bool strict = pl.dtype == BTC_F32 && op->req.strict_fp32 != 0;
+        const Cand *cands = strict ? f32strict : (pl.dtype == BTC_F32 ? f32c : (pl.dtype == BTC_F64 ? f64c : (pl.dtype == BTC_C64 ? c64c : other)));
+        const int ncand = strict ? 3 : (pl.dtype == BTC_F32 ? (umma_ok ? 12 : 4) : 2);
         double best = -1.0;
         for (int c = 0; c < ncand; ++c) {
             const VariantInfo vi = variant_info(pl.dtype, cands[c].id);
@@ -693,6 +695,10 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
     } else if (key == BTC_ATTR_SPLIT_K) {
         if (v < 0) return BTC_ERR_INVALID_ARGUMENT;
         op->req.force_split_k = v;
+    } else if (key == BTC_ATTR_COMPUTE_PRECISION) {
+        if (v != BTC_PRECISION_DEFAULT && v != BTC_PRECISION_STRICT) return BTC_ERR_INVALID_ARGUMENT;
+        if (v == BTC_PRECISION_STRICT && op->plan.dtype == BTC_C32) return BTC_ERR_NOT_SUPPORTED;
+        op->req.strict_fp32 = v == BTC_PRECISION_STRICT ? 1 : 0;
     } else if (key == BTC_ATTR_BATCH_HINT) {
         if (v < 1) return BTC_ERR_INVALID_ARGUMENT;
         op->req.batch_hint = v;
@@ -729,6 +735,7 @@ btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t 
     case BTC_ATTR_VARIANT: i32[0] = pl.tile.variant; n = 4; break;
     case BTC_ATTR_PRE_REDUCE: i32[0] = (op->sumA.active ? 1 : 0) | (op->sumB.active ? 2 : 0); n = 4; break;
     case BTC_ATTR_BATCH_HINT: i32[0] = op->req.batch_hint; n = 4; break;
+    case BTC_ATTR_COMPUTE_PRECISION: i32[0] = op->req.strict_fp32 ? BTC_PRECISION_STRICT : BTC_PRECISION_DEFAULT; n = 4; break;
     case BTC_ATTR_DEVICE_ERROR:
         i32[0] = 0;
         if (op->d_error) {

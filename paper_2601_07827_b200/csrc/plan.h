@@ -73,6 +73,7 @@ struct PlanRequest {
     int32_t force_kernel = BTC_KERNEL_AUTO;
     int32_t force_split_k = 0;   // 0 = choose
     int32_t force_variant = -1;  // -1 = choose; otherwise index of the tile variant for the dtype
+    int32_t strict_fp32 = 0;     // 1: fp32 / complex64 products and sums in IEEE fp32 (no TF32 split)
     int32_t batch_hint = 1;      // pointer-array entries the operation is expected to run with at a time
     int32_t sm_count = 148;
 };

@@ -9,6 +9,7 @@ import pytest
 import torch
 
 import helpers
+import oracle
 from paper_2601_07827_b200 import inputs
 
 pytestmark = pytest.mark.gpu
@@ -102,6 +103,34 @@ def test_paper_test_categories(api, handle, cat, dtype):
     beta = complex(-0.5, 0.25) if cplx else -0.5
     worst, _, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, beta, conjA=cplx, conjC=cplx)
     assert worst <= 1.0, worst
+
+
+def test_strict_fp32_precision_runs_the_fma_kernels(api, handle):
+    """BTC_ATTR_COMPUTE_PRECISION = STRICT: the planner must leave the TF32-split tensor-core variants (6 and up)
+    for the FFMA variants (0-5); the result meets the same tolerance, and on small integers it is bit exact
+    either way."""
+    ext = dict(i=300, j=200, k=150)
+    A = helpers.random_tensor(71, _ext("ik", ext), None, torch.float32)
+    B = helpers.random_tensor(72, _ext("kj", ext), None, torch.float32)
+    D = inputs.place(None, _ext("ij", ext), None, torch.float32)
+    dt = api.dtype_code(torch.float32)
+    tA, tB, tD = (api.TensorInfo(handle, dt, x.extents, x.strides) for x in (A, B, D))
+    op = api.Contraction(handle, tA, "ik", tB, "kj", None, "ij", tD, "ij", 1.0, 0.0)
+    assert op.variant >= 6
+    op.set_attr(api.ATTR_COMPUTE_PRECISION, api.PRECISION_STRICT)
+    assert 0 <= op.variant <= 5
+    dA, dB, dD = A.to("cuda"), B.to("cuda"), D.to("cuda")
+    need = op.workspace_size()
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+    op.execute(torch.cuda.current_stream().cuda_stream, dA.data_ptr(), dB.data_ptr(), 0, dD.data_ptr(), workspace=ws.data_ptr(),
+               workspace_bytes=need)
+    torch.cuda.synchronize()
+    want = D.clone()
+    scale = oracle.contract(A.numpy(), "ik", B.numpy(), "kj", None, "ij", want.numpy(), "ij", 1.0, 0.0)
+    pos = D.offsets()
+    assert helpers.compare(dD.buffer.cpu()[pos].numpy(), want.buffer[pos].numpy(), scale, torch.float32) <= 1.0
+    op.set_attr(api.ATTR_COMPUTE_PRECISION, api.PRECISION_DEFAULT)
+    assert op.variant >= 6
 
 
 @pytest.mark.parametrize("seed", range(64))
