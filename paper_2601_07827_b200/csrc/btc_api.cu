@@ -1287,9 +1287,11 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
     }
     if (transposing) {
         const int T = dtype_size(pl.dtype) <= 8 ? 64 : 32;
+        const int TC = dtype_size(pl.dtype) == 4 ? TransposeTile<float, false>::TC : T;
+        const int TA = dtype_size(pl.dtype) == 4 ? TransposeTile<float, false>::TA : T;
         p.tile_mode_a = pl.tile_mode_a;
-        p.tiles_c = int32_t((p.ext_k[0] + T - 1) / T);
-        p.tiles_a = int32_t((p.ext_k[pl.tile_mode_a] + T - 1) / T);
+        p.tiles_c = int32_t((p.ext_k[0] + TC - 1) / TC);
+        p.tiles_a = int32_t((p.ext_k[pl.tile_mode_a] + TA - 1) / TA);
         p.rest = pl.total_keep / (p.ext_k[0] * p.ext_k[pl.tile_mode_a]);
         blocks = int64_t(p.tiles_c) * p.tiles_a * p.rest;
         if (blocks > 0x7fffffffLL) return BTC_ERR_NOT_SUPPORTED;

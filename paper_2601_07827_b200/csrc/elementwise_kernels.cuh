@@ -229,29 +229,32 @@ __global__ void __launch_bounds__(256) elementwise_vector_kernel(const Elementwi
     }
 }
 
-// Tile edge and CTA size of the transposing kernel: 64 x 64 tiles for elements of up to 8 bytes (rows
-// of 256 or 512 bytes on both sides), 32 x 32 for complex128, 256 threads.  Measured on permutations of
-// 1 GB tensors: 256-byte rows reach 5.0-5.5 TB/s, 512-byte rows the copy bandwidth; 128 x 128 tiles
-// with 1024 threads for 4-byte elements were slower (3.6 TB/s: two large CTAs per SM overlap poorly).
+// Tile and CTA size of the transposing kernel, 256 threads: 128 (along C's dimension 0) x 64 (along A's
+// dimension) for 4-byte elements, 64 x 64 for 8-byte ones, 32 x 32 for complex128, i.e. rows of 512 bytes
+// where shared memory and registers allow.  Measured on permutations of 1 GB fp32 tensors: 64 x 64
+// (256-byte rows) 5.0-5.4 TB/s, 128 x 64 or 64 x 128 6.0-6.3 TB/s, 128 x 128 with 1024 threads 3.6 TB/s
+// (two large CTAs per SM overlap poorly).
 template <typename R, bool CPLX> struct TransposeTile {
     static constexpr int NC = CPLX ? 2 : 1;
     static constexpr int T = sizeof(R) * NC <= 8 ? 64 : 32;
+    // tile extent along C's dimension 0 (rows written) and along A's dimension (rows read)
+    static constexpr int TC = sizeof(R) * NC == 4 ? 128 : T, TA = T;
     static constexpr int THREADS = 256;
-    static constexpr size_t SMEM_BYTES = size_t(NC) * T * (T + 1) * sizeof(R);
+    static constexpr size_t SMEM_BYTES = size_t(NC) * TC * (TA + 1) * sizeof(R);
 };
 
 // blockIdx.x enumerates (tile along C's dimension 0, tile along A's dimension, rest), first fastest.
-// Each thread handles T * T / THREADS elements in either phase; the tile holds values already
+// Each thread handles TC * TA / THREADS elements in either phase; the tile holds values already
 // summed and rounded to the element type.
 template <typename R, bool CPLX, typename I>
 __global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise_transposing_kernel(const ElementwiseParams p)
 {
     constexpr int NC = CPLX ? 2 : 1;
-    constexpr int T = TransposeTile<R, CPLX>::T;
-    constexpr int ROWS = TransposeTile<R, CPLX>::THREADS / T;   // tile rows covered by the CTA at once
-    constexpr int PER = T / ROWS;                        // rows per thread
+    constexpr int TC = TransposeTile<R, CPLX>::TC, TA = TransposeTile<R, CPLX>::TA;
+    constexpr int ROWS1 = TransposeTile<R, CPLX>::THREADS / TA, PER1 = TC / ROWS1;   // phase 1: rows of TA along A's dimension
+    constexpr int ROWS2 = TransposeTile<R, CPLX>::THREADS / TC, PER2 = TA / ROWS2;   // phase 2: rows of TC along C's dimension 0
     extern __shared__ __align__(16) unsigned char tile_bytes[];
-    R (*tile)[T][T + 1] = reinterpret_cast<R (*)[T][T + 1]>(tile_bytes);
+    R (*tile)[TC][TA + 1] = reinterpret_cast<R (*)[TC][TA + 1]>(tile_bytes);
     const int ma = p.tile_mode_a;
     const int64_t tile_c = blockIdx.x % p.tiles_c;
     const int64_t tile_a = (blockIdx.x / p.tiles_c) % p.tiles_a;
@@ -265,41 +268,43 @@ __global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise
         restB += i * p.sB_k[d];
         restC += i * p.sC_k[d];
     }
-    const int tx = threadIdx.x % T, ty = threadIdx.x / T;
-    const int64_t c0 = tile_c * T, a0 = tile_a * T;
+    const int64_t c0 = tile_c * TC, a0 = tile_a * TA;
     const int64_t ext_c = p.ext_k[0], ext_a = p.ext_k[ma];
     // phase 1: consecutive threads along A's dimension.  Without summed dimensions (a pure
     // permutation) all of a thread's loads are issued before the first value is used; a load
     // inside the bounds test of its own iteration would leave one load in flight per thread.
+    {
+    const int tx = threadIdx.x % TA, ty = threadIdx.x / TA;
     if (p.ns == 0 && p.use_a) {
         const R *A = static_cast<const R *>(p.A);
-        R v_r[PER], v_i[PER];
+        R v_r[PER1], v_i[PER1];
         const bool a_in = a0 + tx < ext_a;
         const R *src = A + NC * (restA + (a0 + tx) * p.sA_k[ma] + (c0 + ty) * p.sA_k[0]);
-        const int64_t step = NC * ROWS * p.sA_k[0];
-        const int rows_in = int(ext_c - c0 - ty < int64_t(T) ? ext_c - c0 - ty : int64_t(T));   // rows ty + ROWS r < rows_in exist
+        const int64_t step = NC * ROWS1 * p.sA_k[0];
+        const int rows_in = int(ext_c - c0 - ty < int64_t(TC) ? ext_c - c0 - ty : int64_t(TC));   // rows ty + ROWS1 r < rows_in exist
 #pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            const bool in = a_in && ROWS * r < rows_in;
+        for (int r = 0; r < PER1; ++r) {
+            const bool in = a_in && ROWS1 * r < rows_in;
             v_r[r] = in ? src[0] : R(0);
             v_i[r] = (CPLX && in) ? src[NC - 1] : R(0);
             src += step;
         }
 #pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            tile[0][ty + ROWS * r][tx] = v_r[r];
-            if (CPLX) tile[NC - 1][ty + ROWS * r][tx] = p.conjA ? -v_i[r] : v_i[r];
+        for (int r = 0; r < PER1; ++r) {
+            tile[0][ty + ROWS1 * r][tx] = v_r[r];
+            if (CPLX) tile[NC - 1][ty + ROWS1 * r][tx] = p.conjA ? -v_i[r] : v_i[r];
         }
     } else {
 #pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            const int64_t c = c0 + ty + ROWS * r, a = a0 + tx;
+        for (int r = 0; r < PER1; ++r) {
+            const int64_t c = c0 + ty + ROWS1 * r, a = a0 + tx;
             double acc_r = 0.0, acc_i = 0.0;
             if (c < ext_c && a < ext_a)
                 elementwise_sum<R, CPLX, 1, I>(p, restA + c * p.sA_k[0] + a * p.sA_k[ma], 0, acc_r, acc_i);
-            tile[0][ty + ROWS * r][tx] = R(acc_r);
-            if (CPLX) tile[NC - 1][ty + ROWS * r][tx] = R(acc_i);
+            tile[0][ty + ROWS1 * r][tx] = R(acc_r);
+            if (CPLX) tile[NC - 1][ty + ROWS1 * r][tx] = R(acc_i);
         }
+    }
     }
     __syncthreads();
     // phase 2: consecutive threads along C's dimension 0; B's values are loaded as a batch too
@@ -307,27 +312,28 @@ __global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise
     // alpha * t + beta * b is formed in double only for 64-bit parts: for 32-bit parts the two
     // products and the sum in float are within a few units in the last place of |alpha t| + |beta b|.
     {
+        const int tx = threadIdx.x % TC, ty = threadIdx.x / TC;
         typedef typename ElementwiseScalar<R>::type S;
         const R *B = static_cast<const R *>(p.B);
         R *C = static_cast<R *>(p.C);
         const bool c_in = c0 + tx < ext_c;
-        const int rows_in = int(ext_a - a0 - ty < int64_t(T) ? ext_a - a0 - ty : int64_t(T));
+        const int rows_in = int(ext_a - a0 - ty < int64_t(TA) ? ext_a - a0 - ty : int64_t(TA));
         const R *srcB = B + NC * (restB + (c0 + tx) * p.sB_k[0] + (a0 + ty) * p.sB_k[ma]);
         R *dst = C + NC * (restC + (c0 + tx) * p.sC_k[0] + (a0 + ty) * p.sC_k[ma]);
-        const int64_t stepB = NC * ROWS * p.sB_k[ma], stepC = NC * ROWS * p.sC_k[ma];
+        const int64_t stepB = NC * ROWS2 * p.sB_k[ma], stepC = NC * ROWS2 * p.sC_k[ma];
         const S al_r = S(p.alpha[0]), al_i = S(p.alpha[1]), be_r = S(p.beta[0]), be_i = S(p.beta[1]);
-        R b_r[PER], b_i[PER];
+        R b_r[PER2], b_i[PER2];
 #pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            const bool in = p.use_b && c_in && ROWS * r < rows_in;
+        for (int r = 0; r < PER2; ++r) {
+            const bool in = p.use_b && c_in && ROWS2 * r < rows_in;
             b_r[r] = in ? srcB[0] : R(0);
             b_i[r] = (CPLX && in) ? srcB[NC - 1] : R(0);
             srcB += stepB;
         }
 #pragma unroll
-        for (int r = 0; r < PER; ++r) {
-            if (c_in && ROWS * r < rows_in) {
-                const S t_r = S(tile[0][tx][ty + ROWS * r]), t_i = CPLX ? S(tile[NC - 1][tx][ty + ROWS * r]) : S(0);
+        for (int r = 0; r < PER2; ++r) {
+            if (c_in && ROWS2 * r < rows_in) {
+                const S t_r = S(tile[0][tx][ty + ROWS2 * r]), t_i = CPLX ? S(tile[NC - 1][tx][ty + ROWS2 * r]) : S(0);
                 const S br = S(b_r[r]), bi = CPLX ? (p.conjB ? -S(b_i[r]) : S(b_i[r])) : S(0);
                 if (CPLX) {
                     dst[0] = R(al_r * t_r - al_i * t_i + be_r * br - be_i * bi);
