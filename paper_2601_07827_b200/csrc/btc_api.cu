@@ -2,6 +2,8 @@
 // tile/split-K choice and kernel launches.  No compute happens on the host.
 #include <cuda_runtime.h>
 
+#include <algorithm>
+#include <climits>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -12,6 +14,8 @@
 #include "../../include/btc.h"
 #include "generic_kernel.cuh"
 #include "kernel_params.h"
+#include "launchers.h"
+#include "skinny_layout.h"
 #include "plan.h"
 #include "tiled_f32_kernel.cuh"
 #include "tiled_f64_kernel.cuh"
@@ -56,6 +60,13 @@ struct btc_contraction_s {
     // bulk-tensor-copy variants: the M-side operand as a tensor of boxes, its coordinate tables on the device
     TmaOperand tmaA;
     const int32_t *d_tma_coord_m = nullptr, *d_tma_coord_k = nullptr, *d_tma_coord_h = nullptr;
+    // short-K streaming kernel: piece orders of the operand tiles; how many consecutive m are contiguous in D
+    // ([0], [1]: the plan's A as the kernel's M side / N side; [2], [3]: the plan's B likewise)
+    std::vector<uint16_t> skinny_order[4];
+    const uint16_t *d_skinny_order[4] = {nullptr, nullptr, nullptr, nullptr};
+    int64_t skinny_run_m = 1;
+    bool skinny_regular = false;
+    bool skinny_d_regular[2] = {false, false};     // D's rows (m) / columns (n) regular
     size_t workspace_bytes = 0;
     int32_t grid[3] = {0, 0, 0};
     // Case 4: inputs with isolated labels are first summed into the front of the workspace
@@ -112,9 +123,13 @@ using F32Umma96B32 = UmmaTile<96, 5, 2, true, 1, 32, true>;
 using F32Umma128B32 = UmmaTile<128, 4, 2, true, 1, 32, true>;
 using F32Umma128B24 = UmmaTile<128, 5, 2, true, 1, 24, true>;
 using F32Umma96B24x2 = UmmaTile<96, 3, 2, true, 1, 24, true, 2>;   // two sub-stages of 24 k per hand-off
-constexpr int kNumF32Variants = 23;
+constexpr int kNumF32Variants = 24;
 constexpr int kFirstUmmaVariant = 10;
 constexpr int kFirstBulkVariant = 17;     // 17..21: bulk tensor copies; fall back to 13 / 14 (same tiles) at execute
+constexpr int SKINNY_LINES = 256;         // 128-byte lines of a 32 KiB operand tile
+constexpr int kSkinnyVariant = 23;        // short-K streaming kernel (tcgen05); falls back to 6 (same tiles) at execute
+// fp32 variants whose CTAs are persistent and keep all of K (no split-K)
+inline bool f32_persistent(int variant) { return (variant >= kFirstUmmaVariant && variant <= 21) || variant == kSkinnyVariant; }
 
 struct VariantInfo {
     int bm, bn, bk, threads, acc;
@@ -163,6 +178,7 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
         case 20: return {128, 128, 24, 256, 0, F32Umma128B24::SMEM_BYTES, 4};
         case 21: return {128, 96, 24, 256, 0, F32Umma96B24x2::SMEM_BYTES, 4};
         case 22: return info_of<F32TcTiny>(4);
+        case 23: return {128, 128, 64, 256, 0, 0, 4};
         default: return {128, 128, 32, 256, 0, F32Umma128T2::SMEM_BYTES, 4};
         }
     }
@@ -373,10 +389,16 @@ int finish_plan(btc_contraction_s *op)
             if (score > best) { best = score; variant = cands[c].id; }
         }
     }
+    // fp32 with a short contracted extent (all of K in one shared-memory tile): the streaming kernel,
+    // when both operands can be fetched in 16-byte pieces and there are enough 128 x 128 tiles to
+    // occupy a good part of the machine
+    const bool skinny_fits = pl.dtype == BTC_F32 && op->req.strict_fp32 == 0 && pl.K <= kSkinnyMaxK && pl.vecA == 4 && pl.vecB == 4;
+    if (skinny_fits && ((pl.M + 127) / 128) * ((pl.N + 127) / 128) * pl.Bt * hint >= 32) variant = kSkinnyVariant;
     if (op->req.force_variant >= 0) {
         const int count = pl.dtype == BTC_F32 ? kNumF32Variants : (pl.dtype == BTC_F64 ? 5 : (pl.dtype == BTC_C64 ? 3 : 2));
         if (op->req.force_variant >= count) return BTC_ERR_INVALID_ARGUMENT;
         variant = op->req.force_variant;
+        if (pl.dtype == BTC_F32 && variant == kSkinnyVariant && !skinny_fits) variant = 6;   // the mma.sync twin (same tiles)
     }
     op->tmaA = TmaOperand();
     if (pl.dtype == BTC_F32 && variant >= kFirstBulkVariant && variant <= 21) {
@@ -393,7 +415,7 @@ int finish_plan(btc_contraction_s *op)
     const int64_t tiles = tiles_for(v);
     const int64_t k_tiles = (pl.K + v.bk - 1) / v.bk;
     int64_t split = 1;
-    const bool umma = pl.dtype == BTC_F32 && variant >= kFirstUmmaVariant && variant <= 21;   // these keep all of K in one CTA
+    const bool umma = pl.dtype == BTC_F32 && f32_persistent(variant);   // these keep all of K in one CTA
     if (umma) {
         split = 1;
     } else if (op->req.force_split_k > 0) {
@@ -425,6 +447,65 @@ int finish_plan(btc_contraction_s *op)
     if (split > 1)
         op->workspace_bytes = size_t(tiles) * size_t(split) * size_t(v.threads) * size_t(v.acc) * v.acc_bytes;
 
+    for (auto &o : op->skinny_order) o.clear();
+    if (pl.dtype == BTC_F32 && variant == kSkinnyVariant) {
+        // Piece orders.  An operand tile (128 rows x K padded to a multiple of 8) is fetched in 16-byte
+        // pieces, 32 per warp instruction.  Such a copy runs at full speed when its 32 destinations fill
+        // whole 128-byte lines of shared memory and its sources few lines of global memory, so the
+        // pieces are grouped by the shared-memory line they land in (which depends on the side of the
+        // kernel the operand plays), pieces of a line in position order, and the lines sorted by the
+        // address of their first piece in the tensor.  Every tile uses the order computed for the first:
+        // any order is correct, this one is fast whenever tiles are laid out alike.
+        const int kp = int((pl.K + 7) / 8 * 8);
+        auto operand_order = [&](const std::vector<int64_t> &row_off, const std::vector<int64_t> &k_off, int64_t rows, LoadDir dir, bool n_side) {
+            struct Piece { int64_t addr; unsigned dst; uint16_t e; };
+            std::vector<Piece> v;
+            const int d = dir == LoadDir::ALONG_FREE ? 0 : 1;
+            for (int e = 0; e < 32 * kp; ++e) {
+                int row, k;
+                const unsigned dst = n_side ? skinny_b_pos(d, unsigned(e), row, k) : skinny_a_pos(d, unsigned(e), row, k);
+                v.push_back({(row < rows && k < pl.K) ? row_off[size_t(row)] + k_off[size_t(k)] : INT64_MAX, dst, uint16_t(e)});
+            }
+            std::vector<int64_t> first(size_t(SKINNY_LINES), INT64_MAX);     // smallest address of each line
+            for (auto &x : v) first[x.dst >> 7] = std::min(first[x.dst >> 7], x.addr);
+            std::stable_sort(v.begin(), v.end(), [&](const Piece &a, const Piece &b) {
+                const unsigned la = a.dst >> 7, lb = b.dst >> 7;
+                if (la == lb) return a.dst < b.dst;
+                return first[la] != first[lb] ? first[la] < first[lb] : la < lb;
+            });
+            std::vector<uint16_t> out;
+            for (auto &x : v) out.push_back(x.e);
+            return out;
+        };
+        op->skinny_order[0] = operand_order(pl.offA_m, pl.offA_k, pl.M, pl.dirA, false);
+        op->skinny_order[1] = operand_order(pl.offA_m, pl.offA_k, pl.M, pl.dirA, true);
+        op->skinny_order[2] = operand_order(pl.offB_n, pl.offB_k, pl.N, pl.dirB, false);
+        op->skinny_order[3] = operand_order(pl.offB_n, pl.offB_k, pl.N, pl.dirB, true);
+        // regular operand: rows m0 + r of every tile lie relative to row m0 as rows r of tile 0 relative to row 0
+        auto regular = [&](const std::vector<int64_t> &row_off, const std::vector<int64_t> &k_off) {
+            const int64_t n = int64_t(row_off.size());
+            int64_t lo = 0, hi = 0;
+            for (int64_t r = 0; r < n; ++r) {
+                const int64_t rel = row_off[size_t(r)] - row_off[size_t(r - r % 128)];
+                if (rel != row_off[size_t(r % 128)] - row_off[0]) return false;
+                lo = std::min(lo, rel); hi = std::max(hi, rel);
+            }
+            int64_t klo = 0, khi = 0;
+            for (int64_t k = 0; k < int64_t(k_off.size()); ++k) { klo = std::min(klo, k_off[size_t(k)]); khi = std::max(khi, k_off[size_t(k)]); }
+            return hi + khi < (int64_t(1) << 30) && lo + klo > -(int64_t(1) << 30);
+        };
+        op->skinny_regular = regular(pl.offA_m, pl.offA_k) && regular(pl.offB_n, pl.offB_k);
+        const std::vector<int64_t> none(1, 0);
+        op->skinny_d_regular[0] = regular(pl.offD_m, none);
+        op->skinny_d_regular[1] = regular(pl.offD_n, none);
+        // consecutive m that are consecutive elements of D
+        op->skinny_run_m = 1;
+        for (auto &md : pl.m) {
+            if (md.sD != op->skinny_run_m) break;
+            op->skinny_run_m *= md.extent;
+        }
+    }
+
     if (op->handle.device >= 0) {
         const std::vector<int64_t> *tabs[9] = {&pl.offA_m, &pl.offD_m, &pl.offB_n, &pl.offD_n, &pl.offA_k,
                                                &pl.offB_k, &pl.offA_h, &pl.offB_h, &pl.offD_h};
@@ -441,9 +522,20 @@ int finish_plan(btc_contraction_s *op)
             cstart[i] = total;
             total += (ctabs[i]->size() + 63) / 64 * 32;
         }
+        // piece orders of the short-K streaming kernel, as raw bytes
+        const void *blob[4];
+        size_t blob_bytes[4], bstart[4];
+        for (int i = 0; i < 4; ++i) {
+            blob[i] = op->skinny_order[i].data();
+            blob_bytes[i] = op->skinny_order[i].size() * 2;
+            bstart[i] = total;
+            total += (blob_bytes[i] + 255) / 256 * 32;
+        }
         std::vector<int64_t> host(total, 0);
         for (int i = 0; i < 3; ++i)
             if (!ctabs[i]->empty()) std::memcpy(host.data() + cstart[i], ctabs[i]->data(), ctabs[i]->size() * sizeof(int32_t));
+        for (int i = 0; i < 4; ++i)
+            if (blob_bytes[i]) std::memcpy(host.data() + bstart[i], blob[i], blob_bytes[i]);
         size_t pos = 0, starts[9];
         for (int i = 0; i < 9; ++i) {
             starts[i] = pos;
@@ -464,6 +556,7 @@ int finish_plan(btc_contraction_s *op)
         op->d_tma_coord_m = reinterpret_cast<const int32_t *>(op->d_tables + cstart[0]);
         op->d_tma_coord_k = reinterpret_cast<const int32_t *>(op->d_tables + cstart[1]);
         op->d_tma_coord_h = reinterpret_cast<const int32_t *>(op->d_tables + cstart[2]);
+        for (int i = 0; i < 4; ++i) op->d_skinny_order[i] = reinterpret_cast<const uint16_t *>(op->d_tables + bstart[i]);
     }
     return BTC_SUCCESS;
 }
@@ -876,6 +969,8 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
         tp.partials = workspace ? static_cast<char *>(workspace) + op->partials_offset : nullptr;
         tp.error_word = op->d_error;
         tp.tmaA_coord_m = op->d_tma_coord_m; tp.tmaA_coord_k = op->d_tma_coord_k; tp.tmaA_coord_h = op->d_tma_coord_h;
+        tp.skinny_orderA = op->d_skinny_order[0]; tp.skinny_orderB = op->d_skinny_order[3];
+        tp.skinny_regular = op->skinny_regular ? 1 : 0;
 #ifdef BTC_STAMPS
         { void *sp = nullptr; cudaGetSymbolAddress(&sp, btc_stamp_buffer); tp.stamps = static_cast<long long *>(sp); }
 #endif
@@ -883,7 +978,7 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
         int64_t reduce_ctas = (ctas / pl.split_k) * ((int64_t(pl.tile.bm) * pl.tile.bn + 1023) / 1024);
         // 16-byte stores of D (and loads of C) need those base pointers aligned too
         tp.vecD = (pl.vecD == 4 && !misaligned(D, 16) && !(use_c && misaligned(C, 16)) && !(bv && !bv->aligned16_D)) ? 4 : 1;
-        const bool persistent = pl.dtype == BTC_F32 && pl.tile.variant >= kFirstUmmaVariant && pl.tile.variant <= 21;
+        const bool persistent = pl.dtype == BTC_F32 && f32_persistent(pl.tile.variant);
         if (bv) {
             // the pointer array multiplies the batch entries; everything else of the plan stands
             tp.Bt = pl.Bt * bv->count;
@@ -905,6 +1000,35 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
             case 6: ce = launch_tiled_tf32<F32Tc>(tp, ctas, reduce_ctas, st); break;
             case 7: ce = launch_tiled_tf32<F32TcSmall>(tp, ctas, reduce_ctas, st); break;
             case 22: ce = launch_tiled_tf32<F32TcTiny>(tp, ctas, reduce_ctas, st); break;
+            case 23:
+                // 16-byte pieces need 16-byte aligned operands; otherwise the mma.sync kernel with the same tiles
+                if (tp.vecA != 4 || tp.vecB != 4) {
+                    ran_variant = 6;
+                    ce = launch_tiled_tf32<F32Tc>(tp, int64_t(op->tiles_m) * op->tiles_n * tp.Bt, reduce_ctas, st);
+                } else {
+                    // Where D's contiguous runs along m are short (interleaved small modes) the kernel runs
+                    // with the roles exchanged: D's smallest-stride label on its column side, so that each
+                    // thread writes 16-byte pieces and neighbouring threads neighbouring pieces.  With long
+                    // runs a warp's 32 consecutive rows of one column are a whole line as they are.
+                    TiledParams sp = tp;
+                    if (tp.vecD == 4 && op->skinny_run_m < 32) {
+                        std::swap(sp.A, sp.B);
+                        std::swap(sp.offA_m, sp.offB_n); std::swap(sp.offD_m, sp.offD_n);
+                        std::swap(sp.offA_k, sp.offB_k); std::swap(sp.offA_h, sp.offB_h);
+                        std::swap(sp.M, sp.N); std::swap(sp.tiles_m, sp.tiles_n);
+                        std::swap(sp.dirA, sp.dirB); std::swap(sp.vecA, sp.vecB);
+                        std::swap(sp.conjA, sp.conjB);
+                        sp.skinny_orderA = op->d_skinny_order[2]; sp.skinny_orderB = op->d_skinny_order[1];
+                        sp.skinny_vec_n = 4;
+                    }
+                    // D's column offsets inside a tile, when every tile's columns are laid out alike
+                    const bool exchanged = sp.skinny_vec_n == 4;
+                    const std::vector<int64_t> &col_off = exchanged ? pl.offD_m : pl.offD_n;
+                    sp.skinny_d_regular = op->skinny_d_regular[exchanged ? 0 : 1] ? 1 : 0;
+                    for (size_t c = 0; c < 128; ++c) sp.skinny_col_rel[c] = c < col_off.size() ? int32_t(col_off[c] - col_off[0]) : 0;
+                    ce = launch_skinny_umma(sp, int(ctas), st);
+                }
+                break;
             case 8: ce = launch_tiled_tf32<F32TcWide>(tp, ctas, reduce_ctas, st); break;
             case 9: ce = launch_tiled_tf32<F32TcMid>(tp, ctas, reduce_ctas, st); break;
             case 10: ce = launch_umma<F32Umma96>(tp, ctas, st); break;
@@ -1324,7 +1448,7 @@ btc_error_t btc_selftest_bounded_wait(btc_handle_t handle, void *cuda_stream, in
     int host[2] = {0, 0};
     if (cudaMemsetAsync(words, 0, 2 * sizeof(int), st) != cudaSuccess) rc = BTC_ERR_CUDA;
     if (rc == BTC_SUCCESS) {
-        bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(unsigned(polls), words, words + 1);
+        bounded_wait_selftest_kernel<0><<<1, 64, 0, st>>>(unsigned(polls), words, words + 1);
         if (cudaGetLastError() != cudaSuccess) rc = BTC_ERR_CUDA;
     }
     if (rc == BTC_SUCCESS && (cudaMemcpyAsync(host, words, sizeof host, cudaMemcpyDeviceToHost, st) != cudaSuccess ||

@@ -73,6 +73,18 @@ struct TiledParams {
     // bulk-tensor-copy variants: box origin of the M-side operand = coord_m[tile of M] + coord_k[stage]
     // + coord_h[batch entry], five coordinates each
     const int32_t *tmaA_coord_m, *tmaA_coord_k, *tmaA_coord_h;
+    // short-K streaming kernel: the 16-byte pieces of an operand tile (128 rows x up to 64 k), each
+    // list sorted by address in its tensor (see skinny_umma_kernel.cuh); skinny_vec_n = 4: groups of
+    // four consecutive n are four consecutive, 16-byte aligned elements of D (and C)
+    const uint16_t *skinny_orderA, *skinny_orderB;
+    int32_t skinny_vec_n;
+    // 1: in both operands every tile's rows lie relative to the tile's first row as those of tile 0 do, and
+    // the offsets inside a tile fit 32 bits: tiles are addressed by their first row's offset alone
+    int32_t skinny_regular;
+    // 1: D's columns are regular in the same sense; column c of a tile then lies skinny_col_rel[c] elements
+    // after the tile's first column (read through the constant bank instead of per-lane tables)
+    int32_t skinny_d_regular;
+    int32_t skinny_col_rel[128];
 #ifdef BTC_STAMPS
     long long *stamps;                // debug build only: per-CTA phase time stamps (8 per CTA)
 #endif

@@ -76,7 +76,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity,
 
 // Self-test of the bounded wait: every thread waits on an mbarrier that nobody arrives on, with a
 // small poll limit.  The wait must give up, raise the abort flag and write the error word; the
-// kernel then returns normally, so the context stays usable.
+// kernel then returns normally, so the context stays usable.  (A template only so that the
+// header can be included by several translation units.)
+template <int UNUSED = 0>
 __global__ void bounded_wait_selftest_kernel(unsigned poll_limit, int *error_word, int *gave_up_count)
 {
     __shared__ __align__(8) uint64_t bar;

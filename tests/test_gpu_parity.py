@@ -382,3 +382,56 @@ def test_bounded_wait_gives_up_and_the_context_stays_usable(api, handle):
     D = inputs.place(None, _ext("ij", ext), None, torch.float64)
     worst, _, _ = helpers.run_case(handle, A, "ik", B, "kj", None, D, "ij")
     assert worst <= 1.0
+
+
+SHORT_K = {
+    # name: (labelsA, labelsB, labelsD, extents, strides of D or None, beta)
+    "rows_rows": ("ik", "jk", "ij", dict(i=300, j=200, k=64), None, 0.0),
+    "k_k_ragged_k": ("ki", "kj", "ij", dict(i=300, j=200, k=36), None, -0.5),
+    "rows_k": ("ik", "kj", "ij", dict(i=132, j=260, k=20), None, 1.5),
+    "k_rows_outer_product": ("ki", "jk", "ij", dict(i=256, j=128, k=4), None, 0.0),
+    "transposed_output": ("ik", "kj", "ji", dict(i=260, j=136, k=48), None, 0.5),
+    "strided_output_element_stores": ("ik", "kj", "ij", dict(i=256, j=130, k=32), (2, 520), 0.25),
+    "padded_output": ("ik", "kj", "ij", dict(i=256, j=130, k=64), (1, 260), 0.0),
+    "batch_label_many_tiles": ("kiz", "jkz", "ijz", dict(i=128 * 9 + 4, j=128 * 6 + 8, k=24, z=3), None, 2.0),
+    "interleaved_small_modes": ("axbycw", "wfygxh", "afbgch", dict(a=4, b=8, c=8, f=4, g=8, h=4, x=4, y=4, w=4), None, 0.0),
+}
+
+
+@pytest.mark.parametrize("name", list(SHORT_K))
+def test_short_k_streaming_kernel(api, handle, name):
+    """The fp32 streaming kernel for contracted extents up to 64 (tcgen05, piece-order loads and stores),
+    forced through the attribute: both memory orders of either operand, K that is no multiple of 8 (zero
+    padded), ragged last tiles, beta != 0, a batch label with more tiles than SMs, an output written in
+    16-byte pieces or element by element, and interleaved modes of extent 4 to 8."""
+    la, lb, ld, ext, sD, beta = SHORT_K[name]
+    A = helpers.random_tensor(111, _ext(la, ext), None, torch.float32)
+    B = helpers.random_tensor(112, _ext(lb, ext), None, torch.float32)
+    C = helpers.random_tensor(113, _ext(ld, ext), sD, torch.float32)
+    D = inputs.place(None, _ext(ld, ext), sD, torch.float32)
+    worst, status, _ = helpers.run_case(handle, A, la, B, lb, C if beta else None, D, ld, 0.75, beta, kernel=api.KERNEL_TILED,
+                                        variant=23, want_status=True)
+    assert worst <= 1.0, worst
+    assert status["variant"] == 23 and status["launches"] == 1
+
+
+def test_short_k_streaming_kernel_is_the_default_for_the_tensor_network_workload(api, handle):
+    for name in ("cfg5", "cfg5b"):
+        worst, status, _ = helpers.workload_case(handle, small_workloads()[name], want_status=True)
+        assert worst <= 1.0 and status["variant"] == 23, (name, worst, status)
+
+
+def test_short_k_streaming_kernel_declines_what_it_cannot_fetch_in_16_byte_pieces(api, handle):
+    """K above 64, or an operand whose strides or base pointer rule out 16-byte pieces: the mma.sync
+    kernel with the same tiles runs instead, and the result is the same."""
+    ext = dict(i=256, j=128, k=72)
+    A = helpers.random_tensor(121, _ext("ik", ext), None, torch.float32)
+    B = helpers.random_tensor(122, _ext("kj", ext), None, torch.float32)
+    D = inputs.place(None, _ext("ij", ext), None, torch.float32)
+    worst, status, _ = helpers.run_case(handle, A, "ik", B, "kj", None, D, "ij", kernel=api.KERNEL_TILED, variant=23, want_status=True)
+    assert worst <= 1.0 and status["variant"] == 6
+    buf = helpers.random_tensor(123, (256 * 32 + 8,), None, torch.float32)
+    A_off = inputs.StridedTensor(buf.buffer, (256, 32), (1, 256), 1)      # base pointer 4 bytes past a 16-byte boundary
+    B2 = helpers.random_tensor(124, (32, 128), None, torch.float32)
+    worst, status, _ = helpers.run_case(handle, A_off, "ik", B2, "kj", None, D, "ij", kernel=api.KERNEL_TILED, variant=23, want_status=True)
+    assert worst <= 1.0 and status["variant"] == 6
