@@ -260,6 +260,20 @@ int make_plan(const PlanRequest &req, Plan &plan)
     };
     block_free_modes(plan.m, true);
     block_free_modes(plan.n, false);
+    // The N-side input's stride-1 mode, when it is a free mode that D happens to place late (and no
+    // contracted mode is contiguous in that input), comes first among the N modes: the input can then
+    // be fetched in 16-byte pieces along it.  The order of the N modes only decides which columns of D
+    // share a tile; D itself is written along the M modes.
+    {
+        bool k_contiguous = false;
+        for (auto &md : plan.k) k_contiguous = k_contiguous || iabs(md.sB) == 1;
+        if (!k_contiguous)
+            for (size_t i = 1; i < plan.n.size(); ++i)
+                if (iabs(plan.n[i].sB) == 1 && plan.n[i].extent % 4 == 0) {
+                    std::rotate(plan.n.begin(), plan.n.begin() + long(i), plan.n.begin() + long(i) + 1);
+                    break;
+                }
+    }
 
     // which direction of each input tile is closest to contiguous in memory
     auto min_k_stride = [&](bool forA, int &where) {

@@ -51,6 +51,7 @@ struct SkinnyTile {
     static constexpr int ACC_COLS = 128, A_COLS = 2 * KMAX;  // tensor-memory columns: accumulator; head + tail of the M side
     static constexpr int TMEM_COLS = 512;                    // 2 accumulators + 2 M-side operand buffers
     static constexpr int NUM_BARS = 20;
+    static constexpr int SPLIT_COL = 64;                     // columns below: epilogue warps; from here on: the converter warps, between conversions
     // N-side raw[2] | N-side tail[2] | M-side raw | row / column offsets | k offsets | piece tables | barriers | slot, abort
     static constexpr size_t SMEM_BYTES = size_t(2 * B_STAGES) * B_BYTES + A_BYTES +
                                          size_t(2 * BM + B_STAGES * BN + 2 * KMAX) * 8 + size_t(2 * PIECES) * 8 +
@@ -157,6 +158,112 @@ __device__ __forceinline__ SkinnyWork skinny_work_next(const TiledParams &p, con
     return n;
 }
 
+// What one thread keeps to write its row of the accumulators to D.  Thread `row` owns row `row` of every
+// tile (tensor-memory lane `row`).  Two ways to write:
+//   vecn (groups of four consecutive columns are 16 contiguous, aligned bytes of D): one 16-byte store
+//        per group straight from the accumulator registers.  The host puts D's smallest-stride label on
+//        the column side when its contiguous runs are short, so that the few lanes whose rows are
+//        neighbours in D complete whole 128-byte lines between them.
+//   otherwise: one element per store; a warp's store of one column = 32 consecutive rows.
+// Offsets: row part from the tables (fetched when a strip starts), column part either from the constant
+// bank (regular columns: offset of the tile's first column + skinny_col_rel) or from per-lane table
+// entries handed round by shuffle (vecn: lane l holds column group l; else co[c] = column 32 c + lane).
+// Both are fetched one tile ahead of their use.
+struct SkinnyStore {
+    float *D;
+    const float *C;
+    float alpha, beta;
+    bool vecn, dreg;
+    int row, lane;
+    int64_t ro, ro_next, co_next[4];
+    bool row_ok, row_ok_next;
+
+    __device__ __forceinline__ void init(const TiledParams &p, int row_, int lane_)
+    {
+        D = static_cast<float *>(p.D);
+        C = static_cast<const float *>(p.C);
+        alpha = float(p.alpha[0]); beta = float(p.beta[0]);
+        vecn = p.skinny_vec_n == 4; dreg = p.skinny_d_regular != 0;
+        row = row_; lane = lane_;
+        ro = ro_next = 0; row_ok = row_ok_next = false;
+        co_next[0] = co_next[1] = co_next[2] = co_next[3] = 0;
+    }
+    // start fetching what tile wk needs; `strip_start`: wk is the first tile of a strip for this CTA
+    __device__ __forceinline__ void fetch(const TiledParams &p, const SkinnyWork &wk, bool strip_start)
+    {
+        if (strip_start) {
+            row_ok_next = row < wk.rows_valid;
+            ro_next = row_ok_next ? p.offD_m[wk.m0 + row] + p.offD_h[wk.h] : 0;
+        }
+        if (dreg) {
+            co_next[0] = p.offD_n[wk.n0];
+        } else if (vecn) {
+            co_next[0] = 4 * lane < wk.cols_valid ? p.offD_n[wk.n0 + 4 * lane] : 0;
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) co_next[c] = (c * 32 + lane < wk.cols_valid) ? p.offD_n[wk.n0 + c * 32 + lane] : 0;
+        }
+    }
+    // Columns [c_begin, c_end) (multiples of 32) of the accumulator at `tacc` (this warp's lane quarter)
+    // -> D.  `co` = the column offsets fetched for this tile.  Arrives on `done_bar` as soon as the
+    // columns are in registers.
+    __device__ __forceinline__ void tile(const TiledParams &p, const SkinnyWork &w, unsigned tacc, int c_begin, int c_end,
+                                         unsigned done_bar, const int64_t (&co)[4])
+    {
+#pragma unroll 1
+        for (int c0 = c_begin; c0 < c_end; c0 += 32) {       // rolled: keeps the code small
+            unsigned r[32];
+            tmem_load16(tacc + unsigned(c0), *reinterpret_cast<unsigned (*)[16]>(&r[0]));
+            tmem_load16(tacc + unsigned(c0 + 16), *reinterpret_cast<unsigned (*)[16]>(&r[16]));
+            tmem_load_wait();
+            if (c0 + 32 == c_end) {                  // this thread's share of the accumulator is in registers
+                tc_fence_before();
+                mbar_arrive(done_bar);
+            }
+            const int cols_here = w.cols_valid - c0;         // valid columns from c0 on (may be <= 0)
+            if (vecn) {
+                int64_t off[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    off[q] = ro + (dreg ? co[0] + p.skinny_col_rel[c0 + 4 * q] : __shfl_sync(0xffffffffu, co[0], (c0 >> 2) + q));
+                float4 v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    v[q] = make_float4(alpha * __uint_as_float(r[4 * q]), alpha * __uint_as_float(r[4 * q + 1]),
+                                       alpha * __uint_as_float(r[4 * q + 2]), alpha * __uint_as_float(r[4 * q + 3]));
+                if (p.use_c) {
+#pragma unroll
+                    for (int q0 = 0; q0 < 8; q0 += 4) {
+                        float4 cv[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            cv[q] = (row_ok && 4 * (q0 + q) < cols_here) ? *reinterpret_cast<const float4 *>(C + off[q0 + q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            v[q0 + q].x += beta * cv[q].x; v[q0 + q].y += beta * cv[q].y;
+                            v[q0 + q].z += beta * cv[q].z; v[q0 + q].w += beta * cv[q].w;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (row_ok && 4 * q < cols_here) *reinterpret_cast<float4 *>(D + off[q]) = v[q];
+            } else {
+                const int64_t mine = c0 == 0 ? co[0] : c0 == 32 ? co[1] : c0 == 64 ? co[2] : co[3];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int64_t off = ro + (dreg ? co[0] + p.skinny_col_rel[c0 + j] : __shfl_sync(0xffffffffu, mine, j));
+                    if (row_ok && j < cols_here) {
+                        float v = alpha * __uint_as_float(r[j]);
+                        if (p.use_c) v += beta * C[off];
+                        D[off] = v;
+                    }
+                }
+            }
+        }
+    }
+};
+
 __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(const TiledParams p)
 {
     using T = SkinnyTile;
@@ -216,7 +323,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             mbar_init(ta_full0 + 8u * s, T::GROUP_THREADS);
             mbar_init(ta_empty0 + 8u * s, 1);
             mbar_init(acc_full0 + 8u * s, 1);
-            mbar_init(acc_empty0 + 8u * s, T::GROUP_THREADS);
+            mbar_init(acc_empty0 + 8u * s, 2 * T::GROUP_THREADS);
         }
         mbar_init(loader_sync, T::GROUP_THREADS);
         mbar_init(drain, 1);
@@ -234,37 +341,11 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
     const unsigned tmem_a0 = tmem_base + 2u * T::ACC_COLS;
 
     if (warp < T::EPILOGUE_WARPS) {
-        // ------------------------------------------------------------- epilogue
-        // Thread tid owns row tid of the tile (tensor-memory lane tid).  Two ways to write D:
-        //   vecn (groups of four consecutive columns are 16 contiguous, aligned bytes of D): one 16-byte
-        //        store per group, straight from the accumulator registers; lane l keeps the offset of
-        //        column group l and hands it round by shuffle.  The host puts D's smallest-stride label
-        //        on the column side when its contiguous runs are short, so that the four lanes or so
-        //        whose rows are neighbours in D complete whole 128-byte lines between them.
-        //   otherwise: one element per store, a warp's store of one column = 32 consecutive rows.
-        float *D = static_cast<float *>(p.D);
-        const float *C = static_cast<const float *>(p.C);
-        const float alpha = float(p.alpha[0]), beta = float(p.beta[0]);
-        const bool vecn = p.skinny_vec_n == 4;
-        int64_t ro = 0;
-        bool row_ok = false;
-        // Column offsets are fetched one tile ahead.  Regular columns: co[0] = offset of the tile's first
-        // column (the rest comes from the constant bank); otherwise per-lane entries handed round by
-        // shuffle: vecn: co[0] = group `lane`; else co[c] = column 32 c + lane.
-        const bool dreg = p.skinny_d_regular != 0;
-        int64_t co_next[4] = {0, 0, 0, 0};
-        auto fetch_columns = [&](const SkinnyWork &wk, int64_t (&dst)[4]) {
-            if (dreg) {
-                dst[0] = p.offD_n[wk.n0];
-            } else if (vecn) {
-                dst[0] = 4 * lane < wk.cols_valid ? p.offD_n[wk.n0 + 4 * lane] : 0;
-            } else {
-#pragma unroll
-                for (int c = 0; c < 4; ++c) dst[c] = (c * 32 + lane < wk.cols_valid) ? p.offD_n[wk.n0 + c * 32 + lane] : 0;
-            }
-        };
+        // ------------------------------------------------------------- epilogue (first half of the columns)
+        SkinnyStore st;
+        st.init(p, tid, lane);
         SkinnyWork w = skinny_work_at(p, t0);
-        if (t0 < t1) fetch_columns(w, co_next);
+        if (t0 < t1) st.fetch(p, w, true);
         long long t_wait = 0, t_work = 0;
         (void)t_wait; (void)t_work;
         BTC_PHASE_BEGIN();
@@ -272,77 +353,17 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         for (int64_t t = t0; t < t1; ++t) {
             const int i = int(t - t0), buf = i & 1;
             const SkinnyWork wn = skinny_work_next(p, w);
-            if (t == t0 || w.nt == 0) {
-                row_ok = tid < w.rows_valid;
-                ro = row_ok ? p.offD_m[w.m0 + tid] + p.offD_h[w.h] : 0;
-            }
+            if (t == t0 || w.nt == 0) { st.ro = st.ro_next; st.row_ok = st.row_ok_next; }
             int64_t co[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) co[c] = co_next[c];
-            if (t + 1 < t1) fetch_columns(wn, co_next);
+            for (int c = 0; c < 4; ++c) co[c] = st.co_next[c];
+            if (t + 1 < t1) st.fetch(p, wn, wn.nt == 0);
             BTC_PHASE_END(t_work);
             if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue)) break;
             BTC_PHASE_END(t_wait);
             BTC_EVENT(p, tid == 0, 6, i);
             tc_fence_after();
-            const unsigned tacc = tmem_base + (unsigned(warp * 32) << 16) + unsigned(buf * T::ACC_COLS);
-#pragma unroll 1
-            for (int c0 = 0; c0 < T::BN; c0 += 32) {       // rolled: the loop body stays small enough for the instruction cache
-                unsigned r[32];
-                BTC_EPI_EVENT(p, tid == 0 && c0 == 32, 0, i);
-                tmem_load16(tacc + unsigned(c0), *reinterpret_cast<unsigned (*)[16]>(&r[0]));
-                tmem_load16(tacc + unsigned(c0 + 16), *reinterpret_cast<unsigned (*)[16]>(&r[16]));
-                BTC_EPI_EVENT(p, tid == 0 && c0 == 32, 1, i);
-                tmem_load_wait();
-                BTC_EPI_EVENT(p, tid == 0 && c0 == 32, 2, i);
-                if (c0 + 32 == T::BN) {              // the accumulator is in registers: the MMA warp may reuse it
-                    tc_fence_before();
-                    mbar_arrive(acc_empty0 + 8u * buf);
-                }
-                const int cols_here = w.cols_valid - c0;         // valid columns from c0 on (may be <= 0)
-                if (vecn) {
-                    int64_t off[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        off[q] = ro + (dreg ? co[0] + p.skinny_col_rel[c0 + 4 * q] : __shfl_sync(0xffffffffu, co[0], (c0 >> 2) + q));
-                    BTC_EPI_EVENT(p, tid == 0 && c0 == 32 && off[7] != 1, 3, i);
-                    float4 v[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        v[q] = make_float4(alpha * __uint_as_float(r[4 * q]), alpha * __uint_as_float(r[4 * q + 1]),
-                                           alpha * __uint_as_float(r[4 * q + 2]), alpha * __uint_as_float(r[4 * q + 3]));
-                    BTC_EPI_EVENT(p, tid == 0 && c0 == 32 && v[7].w != 1.2345f, 4, i);
-                    if (p.use_c) {
-#pragma unroll
-                        for (int q0 = 0; q0 < 8; q0 += 4) {
-                            float4 cv[4];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q)
-                                cv[q] = (row_ok && 4 * (q0 + q) < cols_here) ? *reinterpret_cast<const float4 *>(C + off[q0 + q]) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                v[q0 + q].x += beta * cv[q].x; v[q0 + q].y += beta * cv[q].y;
-                                v[q0 + q].z += beta * cv[q].z; v[q0 + q].w += beta * cv[q].w;
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        if (row_ok && 4 * q < cols_here) *reinterpret_cast<float4 *>(D + off[q]) = v[q];
-                    BTC_EPI_EVENT(p, tid == 0 && c0 == 32, 5, i);
-                } else {
-                    const int64_t mine = c0 == 0 ? co[0] : c0 == 32 ? co[1] : c0 == 64 ? co[2] : co[3];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int64_t off = ro + (dreg ? co[0] + p.skinny_col_rel[c0 + j] : __shfl_sync(0xffffffffu, mine, j));
-                        if (row_ok && j < cols_here) {
-                            float v = alpha * __uint_as_float(r[j]);
-                            if (p.use_c) v += beta * C[off];
-                            D[off] = v;
-                        }
-                    }
-                }
-            }
+            st.tile(p, w, tmem_base + (unsigned(warp * 32) << 16) + unsigned(buf * T::ACC_COLS), 0, T::SPLIT_COL, acc_empty0 + 8u * buf, co);
             BTC_EVENT(p, tid == 0, 7, i);
             w = wn;
         }
@@ -355,13 +376,18 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         int sidx = -1;
         long long t_wait = 0, t_work = 0;
         (void)t_wait; (void)t_work;
-        int nt = skinny_work_at(p, t0).nt;            // tile column: a new strip starts where it is 0
+        // Between conversions these warps also write the second half of the columns of the tile before
+        // (its accumulator is complete by then), which doubles the warps that keep stores in flight.
+        SkinnyStore st;
+        st.init(p, ct, lane);
+        SkinnyWork w = skinny_work_at(p, t0), wprev = w;
+        int64_t co_prev[4] = {0, 0, 0, 0};
         BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int64_t t = t0; t < t1; ++t) {
             const int i = int(t - t0), s = i & 1;
-            const bool new_strip = t == t0 || nt == 0;
-            if (++nt == p.tiles_n) nt = 0;
+            const bool new_strip = t == t0 || w.nt == 0;
+            st.fetch(p, w, new_strip);                // for this tile's store, one iteration from now
             if (new_strip) {
                 ++sidx;
                 const int ab = sidx & 1;
@@ -425,6 +451,27 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             proxy_fence_async();                      // the tensor core reads both stages through the async proxy
             mbar_arrive(b_conv0 + 8u * s);
             BTC_EVENT(p, ct == 0, 3, i);
+            if (i > 0) {
+                const int ip = i - 1, buf = ip & 1;
+                if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue)) break;
+                tc_fence_after();
+                st.tile(p, wprev, tmem_base + (unsigned(ct & ~31) << 16) + unsigned(buf * T::ACC_COLS), T::SPLIT_COL, T::BN,
+                        acc_empty0 + 8u * buf, co_prev);
+            }
+            // what was fetched at the top of this iteration belongs to this tile: keep it for the next iteration
+#pragma unroll
+            for (int c = 0; c < 4; ++c) co_prev[c] = st.co_next[c];
+            if (new_strip) { st.ro = st.ro_next; st.row_ok = st.row_ok_next; }
+            wprev = w;
+            w = skinny_work_next(p, w);
+        }
+        if (t1 > t0 && !*abort_flag) {                // the last tile's second half
+            const int ip = int(t1 - t0) - 1, buf = ip & 1;
+            if (mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue)) {
+                tc_fence_after();
+                st.tile(p, wprev, tmem_base + (unsigned(ct & ~31) << 16) + unsigned(buf * T::ACC_COLS), T::SPLIT_COL, T::BN,
+                        acc_empty0 + 8u * buf, co_prev);
+            }
         }
         BTC_PHASE_END(t_work);
         BTC_PHASE_STORE(p, ct == 0, 2, t_wait);
