@@ -5,7 +5,11 @@ A step is one execution of the fp64 coupled-cluster ladder contraction
 R[a,b,i,j] += sum_{c,d} V[a,b,c,d] T[c,d,i,j]  (a,b,c,d = 128; i,j = 32; 0.55 TFLOP per step)
 through the C-ABI library.  `value` is GFLOP/s with the operands resident in HBM; `e2e` is the
 same metric through btc_execute_host with pinned HOST buffers (copies inside the timed region).
-`--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
+The same line carries `peaks` (what this device's pipes and memory sustain, measured at the start
+of the run with the library's micro-benchmarks) and `per_config`: every other workload timed in the
+same process (small ones also as a replayed CUDA graph and over many buffer sets in one batched
+call), each with its rate and roofline fraction.  `--workload NAME` times one workload alone.
+`--impl reference` times the CPU oracle on a bounded sample of the headline workload instead.
 Prints one JSON line.
 """
 from __future__ import annotations
@@ -47,50 +51,79 @@ def measured_tf32_tflops():
         return 1590.0 * 1.1 / 2.25, "fallback"
 
 
-def roofline_for(w, kernel_ms, variant=-1):
-    """Roofline entry of the dominant kernel for this workload."""
-    if w.name.startswith("cfg5"):
-        peak, src = measured_hbm_gbs()
-        achieved = w.algorithmic_bytes() / (kernel_ms * 1e-3) / 1e9
-        return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": f"STREAM-style copy, {src}", "kernel_ms": kernel_ms}
-    achieved = w.flops() / (kernel_ms * 1e-3) / 1e12
-    if w.dtype in ("f64", "c64"):
-        # DRAM bytes of one launch from a one-pass ncu capture of this kernel on this workload
-        # (dram__bytes_read.sum + dram__bytes_write.sum = 3.28 GB + 0.124 GB)
-        traffic = 3.40e9 if (w.name == "cfg2_f64_ccsd_ladder" and variant == 2) else None
-        return {"bound": "tensor", "achieved": achieved, "peak": FP64_PEAK_TFLOPS, "unit": "TFLOP/s",
-                "frac": achieved / FP64_PEAK_TFLOPS, "traffic": traffic,
-                "peak_source": "FP64 tensor (DMMA) pipe: 148 SMs x 64 FMA/clk x 2 x 1.965 GHz; "
-                               "a register-resident DMMA loop measured 37.1 TFLOP/s on this pool",
-                "kernel": "tiled_f64_kernel", "kernel_ms": kernel_ms}
-    if 10 <= variant <= 21:
-        # tcgen05 3xTF32: three TF32 MMAs per product.  TF32 dense peak = measured bf16 burst peak x
-        # the nominal TF32 : bf16 ratio (1.1 : 2.25).  Whichever of the tensor pipe and HBM needs
-        # longer for this workload is the bound.
-        hbm, src = measured_hbm_gbs()
-        tf32_peak, tsrc = measured_tf32_tflops()
-        t_hbm = w.algorithmic_bytes() / (hbm * 1e9)
-        t_tensor = 3 * w.flops() / (tf32_peak * 1e12)
-        if t_hbm >= t_tensor:
-            gbs = w.algorithmic_bytes() / (kernel_ms * 1e-3) / 1e9
-            return {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm, "traffic": None,
-                    "peak_source": f"STREAM-style copy, {src}; the tensor pipe would need {t_tensor * 1e3:.3f} ms, "
-                                   f"HBM needs {t_hbm * 1e3:.3f} ms",
-                    "useful_tflops": achieved, "kernel": "tiled_umma_tf32x3_kernel", "kernel_ms": kernel_ms}
-        return {"bound": "tensor", "achieved": 3 * achieved, "peak": tf32_peak, "unit": "TFLOP/s",
-                "frac": 3 * achieved / tf32_peak, "traffic": None,
-                "peak_source": f"TF32 dense = bf16 cuBLAS burst peak ({tsrc}) x 1.1/2.25; executed flops = 3 x useful "
-                               "(3xTF32)",
-                "useful_tflops": achieved, "kernel": "tiled_umma_tf32x3_kernel", "kernel_ms": kernel_ms}
-    return {"bound": "alu", "achieved": achieved, "peak": FP32_PEAK_TFLOPS, "unit": "TFLOP/s",
-            "frac": achieved / FP32_PEAK_TFLOPS, "traffic": None,
-            "peak_source": "FP32 FMA pipe: 148 SMs x 128 FMA/clk x 2 x 1.965 GHz; "
-                           "a register-resident FFMA loop measured 72.3 TFLOP/s on this pool",
-            "note": "this fp32 kernel computes each product as three TF32 tensor-core MMAs "
-                    "(mma.sync m16n8k8, measured peak 277 TFLOP/s on this pool): it executes "
-                    f"{3 * achieved:.1f} tensor TFLOP/s = {3 * achieved / 277.0:.2f} of that peak",
-            "kernel": "tiled_tf32x3_kernel" if (6 <= variant <= 9 or variant == 22) else "tiled_f32_kernel", "kernel_ms": kernel_ms}
+PEAKS = {}    # filled by measure_peaks(): this device, this run
+
+
+def measure_peaks(api, handle, torch):
+    """The library's micro-benchmarks (btc_measure_peak): arithmetic pipes in TFLOP/s, memory in GB/s."""
+    st = torch.cuda.current_stream().cuda_stream
+    buf = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")      # 1 GiB: eight times the L2
+    out = {}
+    for name, which in (("fp64_fma_tflops", api.PEAK_FP64_FMA), ("fp64_mma_m16n8k16_tflops", api.PEAK_FP64_MMA_K16),
+                        ("fp64_mma_m8n8k4_tflops", api.PEAK_FP64_MMA_K4), ("fp32_fma_tflops", api.PEAK_FP32_FMA),
+                        ("tf32_mma_sync_tflops", api.PEAK_TF32_MMA_SYNC)):
+        out[name] = api.measure_peak(handle, which, st, repeats=2) / 1e12
+    for name, which in (("hbm_read_gbs", api.PEAK_HBM_READ), ("hbm_write_gbs", api.PEAK_HBM_WRITE), ("hbm_copy_gbs", api.PEAK_HBM_COPY)):
+        out[name] = api.measure_peak(handle, which, st, buf.data_ptr(), buf.numel(), repeats=5) / 1e9
+    del buf
+    torch.cuda.empty_cache()
+    out["how"] = ("btc_measure_peak: register-resident FMA / MMA loops (8 CTAs of 256 threads per SM, 4096 iterations); "
+                  "one pass of 16-byte accesses over 1 GiB (copy: read + written bytes); CUDA events")
+    PEAKS.update(out)
+    return out
+
+
+def roofline_for(w, kernel_ms, variant=-1, units=1):
+    """Roofline entry of the dominant kernel for this workload (`units` buffer sets per launch): whichever
+    of the arithmetic pipe the kernel runs on and HBM needs longer for the algorithmic work is the bound."""
+    flops, nbytes = units * w.flops(), units * w.algorithmic_bytes()
+    hbm, src = measured_hbm_gbs()
+    t_hbm = nbytes / (hbm * 1e9)
+    achieved = flops / (kernel_ms * 1e-3) / 1e12
+    gbs = nbytes / (kernel_ms * 1e-3) / 1e9
+    f32 = w.dtype in ("f32", "c32")
+    umma = f32 and (10 <= variant <= 21 or variant == 23)
+    if not f32:
+        kernel, bound, executed = "tiled_f64_kernel", "tensor", flops
+        peak, peak_measured = FP64_PEAK_TFLOPS, PEAKS.get("fp64_mma_m16n8k16_tflops")
+        source = ("FP64 tensor (DMMA) pipe: 148 SMs x 64 FMA/clk x 2 x 1.965 GHz (unit count); peak_measured = the "
+                  "register-resident m16n8k16 loop of this run")
+    elif umma:
+        # tcgen05 3xTF32: three TF32 MMAs per product; TF32 dense peak = measured bf16 burst peak x the
+        # nominal TF32 : bf16 ratio (1.1 : 2.25)
+        kernel, bound, executed = ("skinny_umma_kernel" if variant == 23 else "tiled_umma_tf32x3_kernel"), "tensor", 3 * flops
+        peak, tsrc = measured_tf32_tflops()
+        peak_measured = None
+        source = f"TF32 dense = bf16 cuBLAS burst peak ({tsrc}) x 1.1/2.25; executed flops = 3 x useful (3xTF32)"
+    else:
+        kernel = "tiled_tf32x3_kernel" if (w.dtype == "c32" or 6 <= variant <= 9 or variant == 22) else "tiled_f32_kernel"
+        bound, executed = "alu", flops
+        peak, peak_measured = FP32_PEAK_TFLOPS, PEAKS.get("fp32_fma_tflops")
+        source = ("FP32 FMA pipe: 148 SMs x 128 FMA/clk x 2 x 1.965 GHz (unit count); peak_measured = the "
+                  "register-resident FFMA loop of this run")
+    t_pipe = executed / (peak * 1e12)
+    if t_hbm >= t_pipe:
+        out = {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm, "traffic": None,
+               "peak_source": f"STREAM-style copy, {src}; HBM needs {t_hbm * 1e3:.4f} ms for the algorithmic bytes, "
+                              f"the arithmetic pipe {t_pipe * 1e3:.4f} ms",
+               "peak_measured": PEAKS.get("hbm_copy_gbs"), "useful_tflops": achieved}
+    else:
+        ach = executed / (kernel_ms * 1e-3) / 1e12
+        out = {"bound": bound, "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
+               "peak_source": source, "peak_measured": peak_measured, "useful_tflops": achieved}
+        if peak_measured:
+            out["frac_of_measured"] = ach / peak_measured
+        if bound == "alu":
+            tf32_sync = PEAKS.get("tf32_mma_sync_tflops") or 277.0
+            out["note"] = ("this kernel computes each product as three TF32 tensor-core MMAs (mma.sync m16n8k8, measured "
+                           f"{tf32_sync:.0f} TFLOP/s in this run): it executes {3 * achieved:.1f} tensor TFLOP/s = "
+                           f"{3 * achieved / tf32_sync:.2f} of that peak")
+    # DRAM bytes of one launch from a one-pass ncu capture of this kernel on this workload
+    # (dram__bytes_read.sum + dram__bytes_write.sum = 3.28 GB + 0.124 GB)
+    if w.name == "cfg2_f64_ccsd_ladder" and variant == 2 and units == 1:
+        out["traffic"] = 3.40e9
+    out["kernel"], out["kernel_ms"] = kernel, kernel_ms
+    return out
 
 
 def parse():
@@ -99,7 +132,7 @@ def parse():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=WORKLOAD)
+    ap.add_argument("--workload", default="all", help="one workload name, or 'all': the headline workload plus per_config")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--variant", type=int, default=-1, help="force a tile variant (tuning runs)")
@@ -272,18 +305,14 @@ def small_problem_latency(step, stream, torch):
             "graph_replay_us": graph, "calls": {"single": 200, "back_to_back": 1000, "graph": 1000}}
 
 
-def run_elementwise(args, w):
-    """`--workload ew...`: one step = one C := alpha op(A) + beta op(B) over device-resident tensors;
-    reported as GB/s of algorithmic bytes against the measured HBM bandwidth."""
-    import torch
-    from paper_2601_07827_b200 import build, inputs
-    build.build()
-    from paper_2601_07827_b200 import api
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device")
-    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+def ew_kernel_name(code):
+    return {1: "elementwise_direct_kernel", 2: "elementwise_transposing_kernel", 3: "elementwise_vector_kernel"}.get(code, "?")
+
+
+def measure_elementwise(args, w, torch, api, inputs, handle, sample_clocks=True):
+    """One step = one C := alpha op(A) + beta op(B) over device-resident tensors; GB/s of algorithmic
+    bytes against the measured HBM bandwidth."""
     A, B, C = inputs.make_elementwise_tensors(w, device="cuda")
-    handle = api.Handle()
     dt = api.dtype_code(C.dtype)
     tA = api.TensorInfo(handle, dt, A.extents, A.strides)
     tC = api.TensorInfo(handle, dt, C.extents, C.strides)
@@ -296,47 +325,53 @@ def run_elementwise(args, w):
         op.execute(stream.cuda_stream, A.data_ptr(), pB, C.data_ptr())
     for _ in range(max(1, args.warmup)):
         step()
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(0) if sample_clocks else None
     torch.cuda.synchronize()
-    sampler.start()
+    if sampler:
+        sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
         step()
     e1.record(stream)
     torch.cuda.synchronize()
-    clocks = sampler.stop()
+    clocks = sampler.stop() if sampler else None
     ms = e0.elapsed_time(e1) / args.steps
     gbs = w.algorithmic_bytes() / (ms * 1e-3) / 1e9
     peak, src = measured_hbm_gbs()
-    print(json.dumps({
+    kernel = op.kernel_ran
+    return {
         "metric": "elementwise GB/s", "value": gbs, "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": w.dtype, "data": "synthetic",
-        "config": {"workload": w.name, "labels": [w.labelsA, w.labelsC], "kernel": op.kernel, "num_modes": list(op.num_modes),
+        "config": {"workload": w.name, "labels": [w.labelsA, w.labelsC], "kernel": kernel, "num_modes": list(op.num_modes),
                    "l2": "tensors exceed L2"},
         "clocks": clocks, "gpu_launches": args.steps,
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
-                     "peak_source": f"STREAM-style copy, {src}",
-                     "kernel": "elementwise_transposing_kernel" if op.kernel == 2 else "elementwise_direct_kernel",
-                     "kernel_ms": ms}}))
+                     "peak_source": f"STREAM-style copy, {src}", "peak_measured": PEAKS.get("hbm_copy_gbs"),
+                     "kernel": ew_kernel_name(kernel), "kernel_ms": ms}}
 
 
-def run_batched(args, w):
-    """`--batched N`: N distinct buffer sets of the workload (more than L2 together for the small
-    workloads), one pointer-array call per step: the device-side rate of a small contraction
-    without the per-call launch latency."""
+def run_elementwise(args, w):
+    """`--workload ew...` alone."""
     import torch
     from paper_2601_07827_b200 import build, inputs
     build.build()
     from paper_2601_07827_b200 import api
-    torch.cuda.set_device(0)
-    n = args.batched
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    print(json.dumps(measure_elementwise(args, w, torch, api, inputs, api.Handle())))
+
+
+def measure_batched(args, w, n, torch, api, inputs, handle, sample_clocks=True):
+    """N distinct buffer sets of the workload (more than L2 together for the small workloads), one
+    pointer-array call per step: the device-side rate of a small contraction without the per-call
+    launch latency."""
     A, B, C, D = inputs.make_workload_tensors(w, device="cuda")
     rep = lambda t: torch.stack([t.buffer] * n).contiguous()
     pA, pB, pD = rep(A), rep(B), rep(D)
     pC = rep(C) if (C is not None and not w.in_place) else None
-    handle = api.Handle()
     dt = api.dtype_code(D.dtype)
     tA = api.TensorInfo(handle, dt, A.extents, A.strides)
     tB = api.TensorInfo(handle, dt, B.extents, B.strides)
@@ -356,21 +391,21 @@ def run_batched(args, w):
     step = lambda: op.execute_batched(stream.cuda_stream, lA, lB, lC, lD, workspace=ws.data_ptr(), workspace_bytes=ws_bytes)
     for _ in range(max(1, args.warmup)):
         step()
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(0) if sample_clocks else None
     torch.cuda.synchronize()
-    sampler.start()
+    if sampler:
+        sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
         step()
     e1.record(stream)
     torch.cuda.synchronize()
-    clocks = sampler.stop()
+    clocks = sampler.stop() if sampler else None
     ms = e0.elapsed_time(e1) / args.steps
-    gbs = n * w.algorithmic_bytes() / (ms * 1e-3) / 1e9
-    peak, src = measured_hbm_gbs()
     total_bytes = n * w.algorithmic_bytes()
-    print(json.dumps({
+    roof = roofline_for(w, ms, op.variant, units=n)
+    return {
         "metric": METRIC, "value": n * w.flops() / (ms * 1e-3) / 1e9, "unit": "GFLOP/s", "n_gpus": 1, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": w.dtype, "data": "synthetic",
@@ -378,13 +413,104 @@ def run_batched(args, w):
                    "tile": list(op.tile), "variant": op.variant, "split_k": op.split_k,
                    "l2": "buffer sets exceed L2" if total_bytes > 126e6 else "buffer sets fit in L2"},
         "clocks": clocks, "gpu_launches": args.steps * (2 if op.split_k > 1 else 1),
-        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
-                     "peak_source": f"STREAM-style copy, {src}", "kernel_ms": ms}}))
+        "roofline": roof}
+
+
+def run_batched(args, w):
+    """`--batched N` alone."""
+    import torch
+    from paper_2601_07827_b200 import build, inputs
+    build.build()
+    from paper_2601_07827_b200 import api
+    torch.cuda.set_device(0)
+    print(json.dumps(measure_batched(args, w, args.batched, torch, api, inputs, api.Handle())))
+
+
+def measure_single(args, w, torch, api, inputs, handle, latency=False):
+    """Device-side time of one execute of a contraction workload (operands resident in HBM)."""
+    A, B, C, D = inputs.make_workload_tensors(w, device="cuda")
+    dt = api.dtype_code(D.dtype)
+    tA = api.TensorInfo(handle, dt, A.extents, A.strides)
+    tB = api.TensorInfo(handle, dt, B.extents, B.strides)
+    tD = api.TensorInfo(handle, dt, D.extents, D.strides)
+    op = api.Contraction(handle, tA, w.labelsA, tB, w.labelsB, tD if C is not None else None, w.labelsD, tD, w.labelsD,
+                         w.alpha, w.beta, w.conjA, w.conjB, w.conjC)
+    ws_bytes = op.workspace_size()
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    pC = C.data_ptr() if C is not None else 0
+
+    def step(status=False, on=None):
+        return op.execute((on or stream).cuda_stream, A.data_ptr(), B.data_ptr(), pC, D.data_ptr(),
+                          workspace=ws.data_ptr(), workspace_bytes=ws_bytes, want_status=status)
+    st = step(status=True)
+    for _ in range(max(1, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    out = {"workload": w.name, "mode": "single execute, back to back", "dtype": w.dtype, "ms": ms,
+           "gflops": w.flops() / (ms * 1e-3) / 1e9, "gbs": w.algorithmic_bytes() / (ms * 1e-3) / 1e9,
+           "kernel": st["kernel"], "variant": st["variant"], "tile": list(op.tile), "split_k": op.split_k,
+           "launches": st["launches"], "groups_batch_M_N_K": list(w.groups()),
+           "l2": "inputs exceed L2" if w.algorithmic_bytes() > 126e6 else "operands fit in L2 (L2-resident figure)",
+           "roofline": roofline_for(w, ms, st["variant"])}
+    if latency:
+        lat = small_problem_latency(lambda s_: step(on=s_), stream, torch)
+        out["latency"] = lat
+        out["mode"] = "per call inside a replayed CUDA graph of 100 calls"
+        out["ms"] = lat["graph_replay_us"] * 1e-3
+        out["gflops"] = w.flops() / (out["ms"] * 1e-3) / 1e9
+        out["gbs"] = w.algorithmic_bytes() / (out["ms"] * 1e-3) / 1e9
+        out["roofline"] = roofline_for(w, out["ms"], st["variant"])
+    return out
+
+
+def per_config(args, torch, api, inputs, handle):
+    """Every workload other than the headline one, timed in this process; small ones three ways."""
+    W, E = inputs.workloads(), inputs.elementwise_workloads()
+    sub = argparse.Namespace(**vars(args))
+    sub.steps, sub.warmup, sub.variant = 20, 3, -1
+    out = []
+
+    def flat(d, mode):        # a full bench line reduced to a per_config entry
+        c = d["config"]
+        return {"workload": c["workload"], "mode": mode, "dtype": d["dtype"], "ms": d["ms_per_step"],
+                "gflops": d["value"] if d["unit"] == "GFLOP/s" else None,
+                "gbs": d["roofline"]["achieved"] if d["roofline"]["unit"] == "GB/s" else None,
+                "kernel": c.get("kernel"), "variant": c.get("variant"), "tile": c.get("tile"), "split_k": c.get("split_k"),
+                "l2": c.get("l2"), "roofline": d["roofline"]}
+    plan = [("single", "cfg1_f64_small", True), ("batched", "cfg1_f64_small", 148),
+            ("single", "cfg3_f32_batched_permuted", False), ("single", "cfg4_c64_conj", False), ("single", "cfg4c_c32_conj", False),
+            ("single", "cfg5_f32_tensor_network", True), ("batched", "cfg5_f32_tensor_network", 64),
+            ("single", "cfg5b_f32_tensor_network_rev", True), ("batched", "cfg5b_f32_tensor_network_rev", 64),
+            ("single", "cfg6_f64_case4_isolated", False)] + [("ew", name, None) for name in E]
+    for kind, name, arg in plan:
+        try:
+            if kind == "single":
+                out.append(measure_single(sub, W[name], torch, api, inputs, handle, latency=bool(arg)))
+            elif kind == "batched":
+                out.append(flat(measure_batched(sub, W[name], arg, torch, api, inputs, handle, sample_clocks=False),
+                                f"{arg} buffer sets in one batched call"))
+            else:
+                out.append(flat(measure_elementwise(sub, E[name], torch, api, inputs, handle, sample_clocks=False), "single execute"))
+        except Exception as e:      # one failing workload must not lose the line
+            out.append({"workload": name, "error": f"{type(e).__name__}: {e}"})
+        torch.cuda.empty_cache()
+    return out
 
 
 def main():
     args = parse()
     from paper_2601_07827_b200 import inputs
+    with_per_config = args.workload == "all"
+    if with_per_config:
+        args.workload = WORKLOAD
     if args.workload in inputs.elementwise_workloads():
         if args.impl == "reference":
             raise SystemExit("the reference arm times the contraction oracle only")
@@ -413,9 +539,10 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
+    handle = api.Handle()
+    peaks = measure_peaks(api, handle, torch) if rank == 0 else None
     # ---- operands: every rank holds its own replica of the workload (no exchange on this path)
     A, B, C, D = inputs.make_workload_tensors(w, device="cuda")
-    handle = api.Handle()
     dt = api.dtype_code(D.dtype)
     tA = api.TensorInfo(handle, dt, A.extents, A.strides)
     tB = api.TensorInfo(handle, dt, B.extents, B.strides)
@@ -508,6 +635,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": "GFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline_for(w, kernel_avg_ms, op.variant),
+            "peaks": peaks,
         }
         if ms_per_step < 0.2 and world == 1:
             # microseconds of work per call: the per-step figure above includes the host's call
@@ -519,6 +647,13 @@ def main():
             out["roofline"]["timing"] = "per call inside a replayed CUDA graph of 100 calls"
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"] = cpu_baseline(w)
+        if with_per_config and world == 1:
+            del A, B, C, D, hA, hB, hD, ws
+            torch.cuda.empty_cache()
+            sampler = ClockSampler(local)
+            sampler.start()
+            out["per_config"] = per_config(args, torch, api, inputs, handle)
+            out["per_config_clocks"] = sampler.stop()
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

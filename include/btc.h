@@ -41,7 +41,7 @@ enum {
     BTC_ERR_C_D_MISMATCH = 4,        /* C's rank, extents, strides or labels differ from D's    */
     BTC_ERR_D_ALIASING = 5,          /* two index tuples of D address one element (item 28)     */
     BTC_ERR_LABEL_ONLY_IN_D = 6,     /* a label of D in neither A nor B (Eq. (FreeD), Case 5)   */
-    BTC_ERR_NOT_SUPPORTED = 7,       /* mixed element types, label repeated inside D, Case 4    */
+    BTC_ERR_NOT_SUPPORTED = 7,       /* unsupported mix of element types, label repeated inside D */
     BTC_ERR_WORKSPACE_TOO_SMALL = 8,
     BTC_ERR_MISALIGNED = 9,          /* a data pointer not aligned to its element size          */
     BTC_ERR_CUDA = 10,               /* a CUDA runtime call failed                              */
@@ -269,13 +269,40 @@ btc_error_t btc_destroy_elementwise(btc_elementwise_t *op);
 btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, const void *alpha, const void *A,
                                     const void *beta, const void *B, void *C);
 enum {
-    BTC_EW_ATTR_KERNEL = 1,    /* int32, read: 1 = one thread (or warp) per element of C, 2 = 32 x 32
-                                  tiles through shared memory (input and output contiguous along
-                                  different labels)                                              */
-    BTC_EW_ATTR_NUM_MODES = 2  /* int32[2], read: loop dimensions over C and summed dimensions after
+    BTC_EW_ATTR_KERNEL = 1,    /* int32, read: the planned kernel.  1 = one thread (or warp) per element
+                                  of C, 2 = tiles through shared memory (input and output contiguous
+                                  along different labels; 128 x 64 elements of 4 bytes, 64 x 64 of 8,
+                                  32 x 32 of 16)                                                 */
+    BTC_EW_ATTR_NUM_MODES = 2, /* int32[2], read: loop dimensions over C and summed dimensions after
                                   merging                                                        */
+    BTC_EW_ATTR_LAST_KERNEL = 3 /* int32, read: the kernel the last execute launched (0 before the
+                                  first): 1, 2 as above, 3 = 16-byte vectors along C's contiguous
+                                  label, chosen at execute time when strides and pointers allow  */
 };
 btc_error_t btc_elementwise_get_attr(btc_elementwise_t op, int32_t key, void *value, size_t len, size_t *needed);
+
+/* Peak micro-benchmarks (no counterpart in the paper; the paper leaves benchmarks to future work, Sec.
+ * "Outlook").  Measures what this device sustains with a kernel that does nothing else, so that the
+ * roofline fraction of a contraction can be quoted against a figure taken on the same device in the
+ * same run.  Arithmetic kinds run register-resident loops of independent FMA / MMA chains and need no
+ * buffer (`buffer` may be NULL); memory kinds make one pass of 16-byte accesses over the caller's
+ * DEVICE buffer of `bytes` bytes (16-byte aligned, at least 1 MiB; the copy reads the first half and
+ * writes the second; use more than the L2 size for a DRAM figure).  One untimed launch, then `repeats`
+ * timed launches between two CUDA events on `cuda_stream`; the call waits for them.  *value = flop/s
+ * (two per FMA) or byte/s (copy: bytes read + bytes written).  Allocates nothing on the device.
+ * Errors: INVALID_ARGUMENT, CUDA. */
+enum {
+    BTC_PEAK_FP64_FMA = 0,      /* DFMA, 16 independent chains per thread                         */
+    BTC_PEAK_FP32_FMA = 1,      /* FFMA likewise                                                  */
+    BTC_PEAK_FP64_MMA_K16 = 2,  /* mma.sync m16n8k16 f64: the FP64 tensor pipe the fp64 kernels use */
+    BTC_PEAK_FP64_MMA_K4 = 3,   /* mma.sync m8n8k4 f64                                            */
+    BTC_PEAK_TF32_MMA_SYNC = 4, /* mma.sync m16n8k8 tf32: the warp-level tensor path              */
+    BTC_PEAK_HBM_READ = 5,
+    BTC_PEAK_HBM_WRITE = 6,
+    BTC_PEAK_HBM_COPY = 7
+};
+btc_error_t btc_measure_peak(btc_handle_t handle, int32_t which, void *cuda_stream, void *buffer, size_t bytes,
+                             int32_t repeats, double *value);
 
 /* Self-test of the device-side failure detection (no counterpart in the paper).  Every wait inside
  * the kernels is bounded: after a fixed number of polls it gives up, records a code in the

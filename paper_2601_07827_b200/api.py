@@ -53,7 +53,7 @@ EXPORTED = [
     "btc_set_attr", "btc_get_attr", "btc_execute", "btc_execute_host", "btc_execute_static_scratch",
     "btc_execute_batched", "btc_contraction_batched_workspace_size",
     "btc_status_get",
-    "btc_destroy_status", "btc_explain_error", "btc_selftest_bounded_wait",
+    "btc_destroy_status", "btc_explain_error", "btc_selftest_bounded_wait", "btc_measure_peak",
     "btc_create_elementwise", "btc_destroy_elementwise", "btc_elementwise_execute", "btc_elementwise_get_attr",
 ]
 
@@ -86,8 +86,20 @@ _lib.btc_elementwise_execute.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.btc_elementwise_get_attr.argtypes = [_vp, ctypes.c_int32, _vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
 _lib.btc_selftest_bounded_wait.argtypes = [_vp, _vp, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32),
                                            ctypes.POINTER(ctypes.c_int32)]
+_lib.btc_measure_peak.argtypes = [_vp, ctypes.c_int32, _vp, _vp, ctypes.c_size_t, ctypes.c_int32, ctypes.POINTER(ctypes.c_double)]
 for _name in EXPORTED:
     getattr(_lib, _name).restype = ctypes.c_int
+
+PEAK_FP64_FMA, PEAK_FP32_FMA, PEAK_FP64_MMA_K16, PEAK_FP64_MMA_K4, PEAK_TF32_MMA_SYNC = 0, 1, 2, 3, 4
+PEAK_HBM_READ, PEAK_HBM_WRITE, PEAK_HBM_COPY = 5, 6, 7
+
+
+def measure_peak(handle, which: int, stream: int = 0, buffer: int = 0, nbytes: int = 0, repeats: int = 3) -> float:
+    """flop/s or byte/s this device sustains on one pipe or on its memory (see btc_measure_peak)."""
+    out = ctypes.c_double(0.0)
+    _check(_lib.btc_measure_peak(handle._h, which, stream or None, buffer or None, nbytes, repeats, ctypes.byref(out)),
+           "btc_measure_peak")
+    return out.value
 
 
 def selftest_bounded_wait(handle, stream: int = 0, polls: int = 1000):
@@ -321,8 +333,8 @@ def dtype_code(torch_dtype) -> int:
     return _TORCH_DTYPE[torch_dtype]
 
 
-EW_ATTR_KERNEL, EW_ATTR_NUM_MODES = 1, 2
-EW_KERNEL_DIRECT, EW_KERNEL_TRANSPOSING = 1, 2
+EW_ATTR_KERNEL, EW_ATTR_NUM_MODES, EW_ATTR_LAST_KERNEL = 1, 2, 3
+EW_KERNEL_DIRECT, EW_KERNEL_TRANSPOSING, EW_KERNEL_VECTOR = 1, 2, 3
 
 
 class Elementwise:
@@ -347,6 +359,11 @@ class Elementwise:
     @property
     def kernel(self) -> int:
         return self._get(EW_ATTR_KERNEL, 1)[0]
+
+    @property
+    def kernel_ran(self) -> int:
+        """The kernel the last execute launched (0 before the first)."""
+        return self._get(EW_ATTR_LAST_KERNEL, 1)[0]
 
     @property
     def num_modes(self):

@@ -83,6 +83,7 @@ struct btc_elementwise_s {
     ElementwiseRequest req;
     ElementwisePlan plan;
     double alpha[2] = {1.0, 0.0}, beta[2] = {0.0, 0.0};
+    int32_t last_kernel = 0;      // what the last execute launched: 1 direct, 2 transposing, 3 vector
 };
 
 namespace {
@@ -1311,6 +1312,7 @@ btc_error_t btc_elementwise_get_attr(btc_elementwise_t op, int32_t key, void *va
     size_t n = 0;
     switch (key) {
     case BTC_EW_ATTR_KERNEL: i32[0] = int32_t(op->plan.kernel); n = 4; break;
+    case BTC_EW_ATTR_LAST_KERNEL: i32[0] = op->last_kernel; n = 4; break;
     case BTC_EW_ATTR_NUM_MODES: i32[0] = int32_t(op->plan.keep.size()); i32[1] = int32_t(op->plan.sum.size()); n = 8; break;
     default: return BTC_ERR_INVALID_ARGUMENT;
     }
@@ -1388,6 +1390,7 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
                      (!use_b || reinterpret_cast<uintptr_t>(B) % 16 == 0);
     for (int i = 1; vector_ok && i < p.nk; ++i)
         vector_ok = p.sC_k[i] % vec == 0 && (!use_a || p.sA_k[i] % vec == 0) && (!use_b || p.sB_k[i] % vec == 0);
+    op->last_kernel = vector_ok ? 3 : (transposing ? 2 : 1);
     if (vector_ok) {
         blocks = (pl.total_keep / vec + 255) / 256;
         const int64_t cap = int64_t(op->handle.sm_count) * 32;

@@ -1,13 +1,15 @@
 // C := alpha op(A) + beta op(B)  (Sec. "Unary and Binary Operations"): labels only in A are summed
 // over, A is broadcast along labels only in C, repeated labels of A act through summed strides.
-// Both kernels are bandwidth-bound passes: A (and B) read once through their strides, C written
+// All kernels are bandwidth-bound passes: A (and B) read once through their strides, C written
 // once through its own.
 //   direct       one thread (or one warp, lanes over the summed index) per element of C, C's
 //                most contiguous dimension fastest.  Right when A is contiguous along the same
 //                dimension (scaling, addition, reduction, broadcast).
 //   transposing  permutations whose input is contiguous along another dimension than the output:
-//                a CTA moves a 32 x 32 tile through shared memory, reading along A's dimension and
-//                writing along C's, so both sides see whole 128-byte lines.
+//                a CTA moves a tile (128 x 64 elements of 4 bytes, 64 x 64 of 8, 32 x 32 of 16) through
+//                shared memory, reading along A's dimension and writing along C's, so both sides
+//                move rows of 256-512 bytes.
+//   vector       nothing summed and dimension 0 contiguous in every tensor: 16-byte vectors.
 // Sums are kept in double (pairs for complex) for every element type.
 #pragma once
 

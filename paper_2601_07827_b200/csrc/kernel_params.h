@@ -41,7 +41,7 @@ struct ElementwiseParams {
     int64_t ext_k[kGenericMaxD], sA_k[kGenericMaxD], sB_k[kGenericMaxD], sC_k[kGenericMaxD];
     int64_t ext_s[kGenericMaxD], sA_s[kGenericMaxD];
     int32_t tile_mode_a;              // transposing kernel: the dimension A is read along (C: dimension 0)
-    int32_t tiles_c, tiles_a;         // transposing kernel: 32-element tiles along those two dimensions
+    int32_t tiles_c, tiles_a;         // transposing kernel: tiles along those two dimensions
     int64_t rest;                     // transposing kernel: product of the other dimensions' extents
     double alpha[2], beta[2];
     int32_t conjA, conjB;

@@ -329,6 +329,8 @@ def workloads() -> Dict[str, Workload]:
     w["cfg4_c64_conj"] = Workload(
         "cfg4_c64_conj", "c64", "spt", "tqsr", "pqr", e4,
         alpha=complex(0.5, -0.25), beta=0.0, conjA=True, seed=4000)
+    # 4c: the same contraction in complex64 (the element type the five fixed workloads leave out)
+    w["cfg4c_c32_conj"] = dataclasses.replace(w["cfg4_c64_conj"], name="cfg4c_c32_conj", dtype="c32", seed=4500)
     # 5: memory-bound tensor-network case, rank-8 inputs of extent 4, rank-10 output
     w["cfg5_f32_tensor_network"] = Workload(
         "cfg5_f32_tensor_network", "f32", "axbycwde", "wfygxhij", "afbgchdiej",
