@@ -125,10 +125,19 @@ enum {
                                  tiles are no boxes of the operand) is replaced by its nearest
                                  equivalent; read back what was planned                       */
     BTC_ATTR_DEVICE_ERROR = 8,/* int32, read: 0, or which bounded device-side wait gave up in an
-                                 earlier execute of this operation (its D is then incomplete);
-                                 reading waits for the device                                  */
-    BTC_ATTR_COMPUTE_PRECISION = 12, /* int32, read/write (write re-plans): BTC_PRECISION_* -- the "desired
-                                 computational precision" of Sec. "Tensor Operation Descriptors".  DEFAULT:
+                                 earlier execute of this operation (its D is then incomplete, and
+                                 a split-K result is not written at all); reading waits for the
+                                 device.  The word is sticky: write 0 to clear it.  btc_execute
+                                 cannot report it (it never waits for the device): callers that
+                                 need to know poll this attribute after synchronising;
+                                 btc_execute_host returns BTC_ERR_DEVICE_TIMEOUT itself           */
+    BTC_ATTR_POLL_LIMIT = 13, /* int32 >= 0, write: polls after which a device-side wait gives up
+                                 (default 4194304).  For tests of the failure path: with a limit of 0
+                                 every wait of the tiled kernels gives up at once, the kernels
+                                 return without writing D, and the error word tells; nothing faults
+                                 or hangs                                                          */
+    BTC_ATTR_COMPUTE_PRECISION = 12, /* int32, read/write (write re-plans): BTC_PRECISION_* -- the compute
+                                 precision an operation may ask for (Sec. "Tensor Operation Descriptors").  DEFAULT:
                                  fp32 products are formed from three TF32 tensor-core products (error of a
                                  product <= 2^-22 |a||b|, fp32 accumulation); STRICT: fp32 operations run on
                                  the FMA pipe in IEEE fp32 (about a third of the speed).  No effect on fp64
@@ -175,13 +184,14 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream,
 /* Convenience for callers whose buffers live in HOST memory: copies A, B (and C when beta != 0)
  * to device buffers it allocates, executes, copies D back, frees, and synchronises the stream.
  * Pointers address logical element (0,...,0) of host tensors laid out as the descriptors say;
- * each tensor's whole strided span is transferred.  Errors as btc_execute plus OUT_OF_MEMORY. */
+ * each tensor's whole strided span is transferred.  Errors as btc_execute plus OUT_OF_MEMORY, and
+ * DEVICE_TIMEOUT when a bounded device-side wait gave up (D is then incomplete). */
 btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream,
                              const void *alpha, const void *A, const void *B,
                              const void *beta, const void *C, void *D);
 
 /* Batched execution with pointer arrays (Sec. "Tensor Descriptors": descriptors hold no data pointer
- * so that one description serves many tensors, "in particular for batched tensor operations").
+ * so that one description serves many tensors, batched operations among them).
  * Executes the operation `count` times, entry i on A[i], B[i], C[i], D[i]; alpha and beta are shared.
  *   A, B, C, D   HOST arrays of `count` DEVICE pointers (each as in btc_execute; C may be NULL when
  *                beta == 0).  Entries must not overlap one another's D.
@@ -217,7 +227,11 @@ btc_error_t btc_execute_batched(btc_contraction_t op, void *cuda_stream, const v
  *     with BTC_ERR_SCRATCH_LIMIT before anything is enqueued; use btc_execute for those;
  *   - the device that was current when the operation's handle was created must be current;
  *   - the first call on each device looks up the array's device address (set-up, once per
- *     device); make that first call before starting any stream capture;
+ *     device) and keeps it for the life of the process; make that first call before starting any
+ *     stream capture, and do not reset the device (cudaDeviceReset) afterwards: the kept address
+ *     would be stale;
+ *   - after a bounded device-side wait gave up, the array may hold partial sums of an earlier call;
+ *     the split-K reduction then leaves D untouched (poll BTC_ATTR_DEVICE_ERROR to find out);
  *   - all calls on one device share the one array, and it keeps whatever the last call left in
  *     it.  Nothing in it needs clearing (every partial sum is written before it is read), but
  *     two calls that may run on the GPU at the same time (different streams, different host

@@ -8,7 +8,7 @@
  *
  * What it follows in the paper (Sec. "Unary and Binary Operations"): B and C carry the same
  * labels; the labels of A and C split into H (in both), I_A (only in A) and I_B (only in B / C).
- * "Indices in I_A imply reduction, while indices in I_B imply broadcasting", so for every
+ * Labels only in A are summed over and labels only in B / C repeat A along them, so for every
  * multi-index over C's labels
  *         C[.] = alpha * sum_{I_A} op(A)[.] + beta * op(B)[.]
  * with A independent of the I_B indices.  Unary scaling B := alpha A is the case beta = 0; a

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <climits>
 #include <cmath>
 #include <cstdio>
@@ -72,6 +73,7 @@ struct btc_contraction_s {
     // Case 4: inputs with isolated labels are first summed into the front of the workspace
     // (A' at offset 0, B' behind it), split-K partial sums follow at `partials_offset`
     bool pre_reduce = true;
+    uint32_t poll_limit = kWaitPollLimit;   // BTC_ATTR_POLL_LIMIT
     IsolatedSum sumA, sumB;
     size_t sumB_offset = 0, partials_offset = 0;
     // memory spans of the caller's tensors in elements (the plan may describe A' and B' instead)
@@ -187,15 +189,17 @@ VariantInfo variant_info(btc_dtype_t t, int variant)
     return variant == 0 ? info_of<C64Big>(8) : (variant == 1 ? info_of<C64Small>(8) : info_of<C64Big16>(8));
 }
 
+// (racing first calls on one device both set the attribute: harmless; the flags are atomics so that
+// host threads may execute concurrently)
 template <typename K>
-cudaError_t set_smem_once(K kernel, size_t bytes, bool *configured)
+cudaError_t set_smem_once(K kernel, size_t bytes, std::atomic<bool> *configured)
 {
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (dev >= 0 && dev < 64 && !configured[dev].load(std::memory_order_relaxed)) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes));
         if (e != cudaSuccess) return e;
-        configured[dev] = true;
+        configured[dev].store(true, std::memory_order_relaxed);
     }
     return cudaSuccess;
 }
@@ -203,7 +207,7 @@ cudaError_t set_smem_once(K kernel, size_t bytes, bool *configured)
 template <typename T>
 cudaError_t launch_tiled(const TiledParams &p, int64_t ctas, int64_t reduce_ctas, cudaStream_t st)
 {
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64] = {};
     cudaError_t e = set_smem_once(tiled_f64_kernel<T>, T::SMEM_BYTES, configured);
     if (e != cudaSuccess) return e;
     tiled_f64_kernel<T><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
@@ -219,7 +223,7 @@ cudaError_t launch_tiled(const TiledParams &p, int64_t ctas, int64_t reduce_ctas
 template <typename T>
 cudaError_t launch_tiled_tf32(const TiledParams &p, int64_t ctas, int64_t reduce_ctas, cudaStream_t st)
 {
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64] = {};
     cudaError_t e = set_smem_once(tiled_tf32x3_kernel<T>, T::SMEM_BYTES, configured);
     if (e != cudaSuccess) return e;
     tiled_tf32x3_kernel<T><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
@@ -235,7 +239,7 @@ cudaError_t launch_tiled_tf32(const TiledParams &p, int64_t ctas, int64_t reduce
 template <typename T>
 cudaError_t launch_umma(const TiledParams &p, int64_t ctas, cudaStream_t st, const CUtensorMap *mapA = nullptr)
 {
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64] = {};
     cudaError_t e = set_smem_once(tiled_umma_tf32x3_kernel<T>, T::SMEM_BYTES, configured);
     if (e != cudaSuccess) return e;
     static const CUtensorMap none = {};
@@ -275,7 +279,7 @@ bool encode_tma_operand(const TmaOperand &t, const void *base, CUtensorMap *out)
 template <typename T, bool AK, bool BK_>
 cudaError_t launch_tiled_f32_o(const TiledParams &p, int64_t ctas, int64_t reduce_ctas, cudaStream_t st)
 {
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64] = {};
     cudaError_t e = set_smem_once(tiled_f32_kernel<T, AK, BK_>, T::SMEM_BYTES, configured);
     if (e != cudaSuccess) return e;
     tiled_f32_kernel<T, AK, BK_><<<unsigned(ctas), T::THREADS, T::SMEM_BYTES, st>>>(p);
@@ -776,6 +780,19 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
     if (len != sizeof(int32_t)) return BTC_ERR_INVALID_ARGUMENT;
     int32_t v;
     std::memcpy(&v, value, sizeof v);
+    if (key == BTC_ATTR_POLL_LIMIT) {            // no re-planning: the next execute uses it
+        if (v < 0) return BTC_ERR_INVALID_ARGUMENT;
+        op->poll_limit = uint32_t(v);
+        return BTC_SUCCESS;
+    }
+    if (key == BTC_ATTR_DEVICE_ERROR) {          // writing 0 clears the device error word
+        if (v != 0) return BTC_ERR_INVALID_ARGUMENT;
+        if (op->d_error && cudaMemset(op->d_error, 0, sizeof(int32_t)) != cudaSuccess) {
+            cudaGetLastError();
+            return BTC_ERR_CUDA;
+        }
+        return BTC_SUCCESS;
+    }
     const PlanRequest saved = op->req;
     const bool saved_pre_reduce = op->pre_reduce;
     if (key == BTC_ATTR_PRE_REDUCE) {
@@ -969,6 +986,7 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
         tp.alpha[0] = al[0]; tp.alpha[1] = al[1]; tp.beta[0] = be[0]; tp.beta[1] = be[1];
         tp.partials = workspace ? static_cast<char *>(workspace) + op->partials_offset : nullptr;
         tp.error_word = op->d_error;
+        tp.poll_limit = op->poll_limit;
         tp.tmaA_coord_m = op->d_tma_coord_m; tp.tmaA_coord_k = op->d_tma_coord_k; tp.tmaA_coord_h = op->d_tma_coord_h;
         tp.skinny_orderA = op->d_skinny_order[0]; tp.skinny_orderB = op->d_skinny_order[3];
         tp.skinny_regular = op->skinny_regular ? 1 : 0;
@@ -1221,6 +1239,12 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
     if (rc == BTC_SUCCESS &&
         cudaMemcpyAsync(static_cast<char *>(D) + bD.lo, bD.dev, bD.bytes(), cudaMemcpyDeviceToHost, st) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
     if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
+    // a bounded device-side wait that gave up left D incomplete: say so
+    if (rc == BTC_SUCCESS && op->d_error) {
+        int32_t word = 0;
+        if (cudaMemcpy(&word, op->d_error, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
+        else if (word != 0) fail(BTC_ERR_DEVICE_TIMEOUT);
+    }
     for (Buf *b : {&bA, &bB, &bD}) if (b->dev) cudaFree(b->dev);
     if (use_c && !c_is_d && bC.dev) cudaFree(bC.dev);
     if (ws) cudaFree(ws);
@@ -1245,7 +1269,7 @@ btc_error_t btc_execute_static_scratch(btc_contraction_t op, void *cuda_stream, 
 {
     // Device address of the array, looked up once per device.  In host code the array's name is
     // only a stand-in for the symbol, never an address a kernel could use.
-    static void *scratch_of_device[64] = {};
+    static std::atomic<void *> scratch_of_device[64] = {};
     if (!op || !D) return BTC_ERR_INVALID_ARGUMENT;
     if (op->handle.device < 0) return BTC_ERR_CUDA;
     if (op->workspace_bytes > size_t(BTC_STATIC_SCRATCH_BYTES)) return BTC_ERR_SCRATCH_LIMIT;
@@ -1253,13 +1277,13 @@ btc_error_t btc_execute_static_scratch(btc_contraction_t op, void *cuda_stream, 
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return BTC_ERR_CUDA; }
     // the symbol's address differs per device: the operation's device must be the current one
     if (dev != op->handle.device || dev < 0 || dev >= 64) return BTC_ERR_INVALID_ARGUMENT;
-    void *scratch = scratch_of_device[dev];
+    void *scratch = scratch_of_device[dev].load(std::memory_order_relaxed);
     if (!scratch) {
         if (cudaGetSymbolAddress(&scratch, btc_static_scratch) != cudaSuccess || !scratch) {
             cudaGetLastError();
             return BTC_ERR_CUDA;
         }
-        scratch_of_device[dev] = scratch;   // racing first calls store the same value
+        scratch_of_device[dev].store(scratch, std::memory_order_relaxed);   // racing first calls store the same value
     }
     // Every consumer thread of every CTA overwrites all of its partial sums before the reduction
     // kernel reads them, so nothing in the array has to start at zero.
@@ -1363,7 +1387,7 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
     do {                                                                                                           \
         if (transposing) {                                                                                         \
             typedef TransposeTile<R, CPLX> TT;                                                                     \
-            static bool configured[64] = {}, configured_wide[64] = {};                                             \
+            static std::atomic<bool> configured[64] = {}, configured_wide[64] = {};                                             \
             if (narrow) {                                                                                          \
                 if (set_smem_once(elementwise_transposing_kernel<R, CPLX, uint32_t>, TT::SMEM_BYTES, configured) != cudaSuccess) return BTC_ERR_CUDA; \
                 elementwise_transposing_kernel<R, CPLX, uint32_t><<<unsigned(blocks), TT::THREADS, TT::SMEM_BYTES, st>>>(p); \

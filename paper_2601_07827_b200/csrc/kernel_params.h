@@ -70,6 +70,7 @@ struct TiledParams {
     double alpha[2], beta[2];
     void *partials;                   // split-K scratch (workspace), or nullptr
     int32_t *error_word;              // device word; set non-zero when a bounded wait gave up
+    uint32_t poll_limit;              // polls after which a device-side wait gives up
     // bulk-tensor-copy variants: box origin of the M-side operand = coord_m[tile of M] + coord_k[stage]
     // + coord_h[batch entry], five coordinates each
     const int32_t *tmaA_coord_m, *tmaA_coord_k, *tmaA_coord_h;

@@ -359,7 +359,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             for (int c = 0; c < 4; ++c) co[c] = st.co_next[c];
             if (t + 1 < t1) st.fetch(p, wn, wn.nt == 0);
             BTC_PHASE_END(t_work);
-            if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue)) break;
+            if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit)) break;
             BTC_PHASE_END(t_wait);
             BTC_EVENT(p, tid == 0, 6, i);
             tc_fence_after();
@@ -391,9 +391,9 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             if (new_strip) {
                 ++sidx;
                 const int ab = sidx & 1;
-                if (!mbar_wait_bounded(a_full, unsigned(sidx) & 1u, abort_flag, p.error_word, kErrSkinnyConvert)) break;
+                if (!mbar_wait_bounded(a_full, unsigned(sidx) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)) break;
                 if (sidx >= 2 &&
-                    !mbar_wait_bounded(ta_empty0 + 8u * ab, unsigned((sidx >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert))
+                    !mbar_wait_bounded(ta_empty0 + 8u * ab, unsigned((sidx >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit))
                     break;
                 tc_fence_after();
                 const unsigned ta = tmem_a0 + unsigned(ab * T::A_COLS) + (unsigned(ct & ~31) << 16);
@@ -423,7 +423,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
                 mbar_arrive(a_empty);                 // the raw M-side buffer may be refilled
             }
             BTC_PHASE_END(t_work);
-            if (!mbar_wait_bounded(b_full0 + 8u * s, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert)) break;
+            if (!mbar_wait_bounded(b_full0 + 8u * s, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)) break;
             BTC_PHASE_END(t_wait);
             BTC_EVENT(p, ct == 0, 2, i);
             // N side: position-independent pass; the raw stage is the head, the tail goes to the same
@@ -453,7 +453,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             BTC_EVENT(p, ct == 0, 3, i);
             if (i > 0) {
                 const int ip = i - 1, buf = ip & 1;
-                if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue)) break;
+                if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit)) break;
                 tc_fence_after();
                 st.tile(p, wprev, tmem_base + (unsigned(ct & ~31) << 16) + unsigned(buf * T::ACC_COLS), T::SPLIT_COL, T::BN,
                         acc_empty0 + 8u * buf, co_prev);
@@ -467,7 +467,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         }
         if (t1 > t0 && !*abort_flag) {                // the last tile's second half
             const int ip = int(t1 - t0) - 1, buf = ip & 1;
-            if (mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue)) {
+            if (mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit)) {
                 tc_fence_after();
                 st.tile(p, wprev, tmem_base + (unsigned(ct & ~31) << 16) + unsigned(buf * T::ACC_COLS), T::SPLIT_COL, T::BN,
                         acc_empty0 + 8u * buf, co_prev);
@@ -506,18 +506,18 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             if (!regular) {
                 if (new_strip) rA[pt] = next_row;
                 cB[pt] = next_col;
-                if (!umma_group_sync(loader_sync, unsigned(i) & 1u, abort_flag, p.error_word)) break;
+                if (!umma_group_sync(loader_sync, unsigned(i) & 1u, abort_flag, p.error_word, p.poll_limit)) break;
             }
             const SkinnyWork wn = skinny_work_next(p, w);
             if (t + 1 < t1) fetch(wn);
             if (new_strip) {
-                if (sidx > 0 && !mbar_wait_bounded(a_empty, unsigned(sidx - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad)) break;
+                if (sidx > 0 && !mbar_wait_bounded(a_empty, unsigned(sidx - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
                 if (regular) skinny_load_tile_regular(araw, A + row_base, pieceA, pieces, w.rows_valid, pt);
                 else skinny_load_tile(araw, A, rA, koffA, pieceA, pieces, w.rows_valid, pt);
                 mbar_arrive_on_copies(a_full);
             }
             BTC_PHASE_END(t_work);
-            if (i >= 2 && !mbar_wait_bounded(b_empty0 + 8u * s, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad)) break;
+            if (i >= 2 && !mbar_wait_bounded(b_empty0 + 8u * s, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
             BTC_PHASE_END(t_wait);
             BTC_EVENT(p, pt == 0, 0, i);
             if (regular) skinny_load_tile_regular(braw0 + unsigned(s) * T::B_BYTES, B + col_base, pieceB, pieces, w.cols_valid, pt);
@@ -551,12 +551,12 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             if (++nt == p.tiles_n) nt = 0;           // now the column of the next tile
             if (new_strip) {
                 ++sidx;
-                if (!mbar_wait_bounded(ta_full0 + 8u * (sidx & 1), unsigned(sidx >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma)) break;
+                if (!mbar_wait_bounded(ta_full0 + 8u * (sidx & 1), unsigned(sidx >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
             }
             BTC_PHASE_END(t_issue);
-            if (i >= 2 && !mbar_wait_bounded(acc_empty0 + 8u * buf, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma)) break;
+            if (i >= 2 && !mbar_wait_bounded(acc_empty0 + 8u * buf, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
             BTC_PHASE_END(t_acc);
-            if (!mbar_wait_bounded(b_conv0 + 8u * s, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma)) break;
+            if (!mbar_wait_bounded(b_conv0 + 8u * s, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
             BTC_PHASE_END(t_conv);
             BTC_EVENT(p, lane == 0, 4, i);
             tc_fence_after();

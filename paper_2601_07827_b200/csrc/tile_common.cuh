@@ -252,7 +252,7 @@ __device__ __forceinline__ void producer_loop(const Params &p, const TileCoords 
     for (int kt = 0; kt < c.num_kt; ++kt) {
         const int s = kt % STAGES, round = kt / STAGES;
         if (round > 0 &&
-            !mbar_wait_bounded(empty0 + 8u * s, unsigned(round - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait))
+            !mbar_wait_bounded(empty0 + 8u * s, unsigned(round - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait, p.poll_limit))
             break;
         const unsigned sa = stage0 + unsigned(s) * STAGE_BYTES;
         const unsigned sb = sa + A_BYTES;

@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
     bool ok = true;
     for (int kt = 0; kt < tc.num_kt; ++kt) {
         const int s = kt % T::STAGES, round = kt / T::STAGES;
-        if (!mbar_wait_bounded(full0 + 8u * s, unsigned(round) & 1u, abort_flag, p.error_word, kErrFullWait)) {
+        if (!mbar_wait_bounded(full0 + 8u * s, unsigned(round) & 1u, abort_flag, p.error_word, kErrFullWait, p.poll_limit)) {
             ok = false;
             break;
         }

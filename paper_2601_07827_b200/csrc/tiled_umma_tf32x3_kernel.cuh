@@ -82,7 +82,7 @@ struct UmmaTile {
     static_assert(TMEM_USED <= 512, "accumulators and operand stages must fit the 512 tensor-memory columns");
     // 16-byte pieces per converter thread in the position-independent pass (whole stage, or its N side)
     static constexpr int PIECES = (A_TMEM_ ? B_BYTES : SUB_BYTES) / 16 / CONVERTER_THREADS;
-    static constexpr int NUM_BARS = 2 * RAW_STAGES + 2 * TAIL_STAGES + 8;
+    static constexpr int NUM_BARS = 2 * RAW_STAGES + 2 * TAIL_STAGES + 9;    // ... + the drain barrier of the abort path
     static_assert(B_BYTES % (16 * CONVERTER_THREADS) == 0, "a stage must divide among the converters");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "BN must suit UMMA N and the epilogue split");
     // stages | row/col offsets | k offsets | mbarriers | tmem ptr, abort
@@ -334,10 +334,11 @@ constexpr int kErrAccumWait = 3, kErrTailFullWait = 4, kErrTailEmptyWait = 5, kE
 
 // Group-wide rendezvous on an mbarrier (every member arrives, then waits with a bound): unlike a
 // named barrier it cannot hang when a member has left after an abort.
-__device__ __forceinline__ bool umma_group_sync(unsigned bar, unsigned parity, volatile int *abort_flag, int *error_word)
+__device__ __forceinline__ bool umma_group_sync(unsigned bar, unsigned parity, volatile int *abort_flag, int *error_word,
+                                                unsigned poll_limit = kWaitPollLimit)
 {
     mbar_arrive(bar);
-    return mbar_wait_bounded(bar, parity, abort_flag, error_word, kErrGroupSync);
+    return mbar_wait_bounded(bar, parity, abort_flag, error_word, kErrGroupSync, poll_limit);
 }
 
 // Persistent: CTA b works on the items b, b + gridDim.x, ... of the (tile, batch) list; all roles
@@ -401,6 +402,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 mbar_init(producer_sync0 + 8u * b, T::PRODUCER_THREADS);
                 mbar_init(epilogue_sync0 + 8u * b, T::EPILOGUE_THREADS);
             }
+            mbar_init(epilogue_sync0 + 16u, 1);      // drain
 
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -431,8 +433,8 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             for (int i = tid; i < T::BN; i += T::EPILOGUE_THREADS) cD[i] = i < tc.cols_valid ? p.offD_n[tc.n0 + i] : 0;
             const bool row_ok = tid < tc.rows_valid;
             const int64_t ro = row_ok ? p.offD_m[tc.m0 + tid] + p.offD_h[tc.h] : 0;
-            if (!umma_group_sync(epilogue_sync0 + 8u * buf, parity, abort_flag, p.error_word)) break;
-            if (!mbar_wait_bounded(accum_full0 + 8u * buf, parity, abort_flag, p.error_word, kErrAccumWait)) break;
+            if (!umma_group_sync(epilogue_sync0 + 8u * buf, parity, abort_flag, p.error_word, p.poll_limit)) break;
+            if (!mbar_wait_bounded(accum_full0 + 8u * buf, parity, abort_flag, p.error_word, kErrAccumWait, p.poll_limit)) break;
             tc_fence_after();
             const unsigned tacc = tmem_base + (unsigned(warp * 32) << 16) + unsigned(buf * T::ACC_COLS);
 #pragma unroll 1
@@ -470,13 +472,13 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             for (int st = 0; st < num_st; ++st, ++g) {
                 if (T::CONVERTER_GROUPS > 1 && g % T::CONVERTER_GROUPS != group) continue;   // another group's stage
                 const int s = g % T::RAW_STAGES, t = g % T::TAIL_STAGES;
-                if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(g / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait)) {
+                if (!mbar_wait_bounded(raw_full0 + 8u * s, unsigned(g / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrFullWait, p.poll_limit)) {
                     ok = false;
                     break;
                 }
                 BTC_PHASE_END(t_raw);
                 if (g >= T::TAIL_STAGES &&
-                    !mbar_wait_bounded(tail_empty0 + 8u * t, unsigned(g / T::TAIL_STAGES - 1) & 1u, abort_flag, p.error_word, kErrTailEmptyWait)) {
+                    !mbar_wait_bounded(tail_empty0 + 8u * t, unsigned(g / T::TAIL_STAGES - 1) & 1u, abort_flag, p.error_word, kErrTailEmptyWait, p.poll_limit)) {
                     ok = false;
                     break;
                 }
@@ -597,7 +599,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     for (int i = pt; i < T::BM; i += T::PRODUCER_THREADS) rA[i] = i < tc.rows_valid ? p.offA_m[tc.m0 + i] + hA : 0;
                 for (int i = pt; i < T::BN; i += T::PRODUCER_THREADS) cB[i] = i < tc.cols_valid ? p.offB_n[tc.n0 + i] + hB : 0;
             }
-            if (!umma_group_sync(producer_sync0 + 8u * buf, unsigned(n >> 1) & 1u, abort_flag, p.error_word)) break;
+            if (!umma_group_sync(producer_sync0 + 8u * buf, unsigned(n >> 1) & 1u, abort_flag, p.error_word, p.poll_limit)) break;
             const UmmaOperand opA = {static_cast<const float *>(p.A), rA, staged ? koffA : p.offA_k, tc.rows_valid, 0, p.K, p.dirA, p.vecA};
             const UmmaOperand opB = {static_cast<const float *>(p.B), cB, staged ? koffB : p.offB_k, tc.cols_valid, 0, p.K, p.dirB, p.vecB};
             UmmaProducerLane<T::BM> la;
@@ -627,7 +629,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     }
                 }
                 if (g >= T::RAW_STAGES &&
-                    !mbar_wait_bounded(raw_empty0 + 8u * s, unsigned(g / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait)) {
+                    !mbar_wait_bounded(raw_empty0 + 8u * s, unsigned(g / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrEmptyWait, p.poll_limit)) {
                     ok = false;
                     break;
                 }
@@ -688,7 +690,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x, ++n) {
             const int buf = n & 1;
             if (n >= 2 &&
-                !mbar_wait_bounded(accum_empty0 + 8u * buf, unsigned((n >> 1) - 1) & 1u, abort_flag, p.error_word, kErrAccumWait))
+                !mbar_wait_bounded(accum_empty0 + 8u * buf, unsigned((n >> 1) - 1) & 1u, abort_flag, p.error_word, kErrAccumWait, p.poll_limit))
                 break;
             BTC_PHASE_END(t_acc);
             tc_fence_after();
@@ -696,7 +698,7 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
 #pragma unroll 1
             for (int st = 0; st < num_st; ++st, ++g) {
                 const int s = g % T::RAW_STAGES, t = g % T::TAIL_STAGES;
-                if (!mbar_wait_bounded(tail_full0 + 8u * t, unsigned(g / T::TAIL_STAGES) & 1u, abort_flag, p.error_word, kErrTailFullWait)) {
+                if (!mbar_wait_bounded(tail_full0 + 8u * t, unsigned(g / T::TAIL_STAGES) & 1u, abort_flag, p.error_word, kErrTailFullWait, p.poll_limit)) {
                     ok = false;
                     break;
                 }
@@ -750,8 +752,20 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
     }
 
     // ---- common tail: every role arrives here, also after an abort ----
+    // After an abort work may still be in flight that must not outlive the CTA: asynchronous copies
+    // (the producers have waited for theirs above), tensor-core instructions (drained below through a
+    // commit on a barrier of its own, with a bounded wait) and, in the bulk-copy variants, box copies
+    // whose completion barrier may never fire because some producers have left: those land within a
+    // few microseconds, so the CTA lingers that long before it gives up its shared memory.
+    if (T::A_TMA && *abort_flag && tid == T::EPILOGUE_THREADS + 32 * T::CONVERTER_WARPS) __nanosleep(20000);
     __syncthreads();
     if (warp == T::MMA_WARP) {
+        if (*abort_flag) {
+            const unsigned drain = epilogue_sync0 + 16u;
+            if (elect_one()) umma_commit(drain);
+            __syncwarp();
+            for (unsigned n = 0; n < (1u << 16) && !mbar_try_wait(drain, 0u); ++n) { }
+        }
         tc_fence_after();
         tmem_dealloc(tmem_base, T::TMEM_COLS);
     }

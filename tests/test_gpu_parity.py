@@ -435,3 +435,80 @@ def test_short_k_streaming_kernel_declines_what_it_cannot_fetch_in_16_byte_piece
     B2 = helpers.random_tensor(124, (32, 128), None, torch.float32)
     worst, status, _ = helpers.run_case(handle, A_off, "ik", B2, "kj", None, D, "ij", kernel=api.KERNEL_TILED, variant=23, want_status=True)
     assert worst <= 1.0 and status["variant"] == 6
+
+
+@pytest.mark.parametrize("limit", [0, 1])
+@pytest.mark.parametrize("dtype,variant", [(torch.float64, 2), (torch.float64, 1), (torch.complex128, 0), (torch.float32, 7),
+                                           (torch.float32, 13), (torch.float32, 21), (torch.float32, 23)])
+def test_waits_that_run_out_are_reported_and_the_operation_recovers(api, handle, dtype, variant, limit):
+    """Failure detection in the real kernels.  With a poll limit of zero every device-side wait gives up at
+    once; with a limit of one, waits on shared-memory stages may run out while their copies are still in
+    flight (that depends on timing; when none did, the result must simply be right).  Either way the kernel
+    must return (nothing traps or hangs), the operation's device error word must tell, bytes outside D's
+    elements must stay untouched, and after the limit is put back and the word cleared the same operation
+    computes the right result."""
+    ext = dict(i=128 * 3 + 8, j=128 * 2 + 4, k=64 if variant == 23 else 200)
+    A = helpers.random_tensor(131, _ext("ki", ext), None, dtype)
+    B = helpers.random_tensor(132, _ext("kj", ext), None, dtype)
+    D = inputs.place(None, _ext("ij", ext), (1, ext["i"] + 4), dtype)
+    dt = api.dtype_code(dtype)
+    tA, tB, tD = (api.TensorInfo(handle, dt, x.extents, x.strides) for x in (A, B, D))
+    op = api.Contraction(handle, tA, "ki", tB, "kj", None, "ij", tD, "ij", 1.0, 0.0)
+    op.set_attr(api.ATTR_KERNEL, api.KERNEL_TILED)
+    op.set_attr(api.ATTR_VARIANT, variant)
+    assert op.variant == variant
+    dA, dB, dD = A.to("cuda"), B.to("cuda"), D.to("cuda")
+    need = op.workspace_size()
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device="cuda")
+    run = lambda: op.execute(torch.cuda.current_stream().cuda_stream, dA.data_ptr(), dB.data_ptr(), 0, dD.data_ptr(),
+                             workspace=ws.data_ptr(), workspace_bytes=need)
+    op.set_attr(api.ATTR_POLL_LIMIT, limit)
+    run()
+    torch.cuda.synchronize()
+    word = op.device_error
+    if limit == 0:
+        assert word != 0
+        assert torch.equal(dD.buffer.cpu().view(torch.uint8), D.buffer.view(torch.uint8))   # nothing was written
+    pos = D.offsets()
+    assert helpers.canary_intact(D.buffer, dD.buffer.cpu(), pos)
+    want = D.clone()
+    scale = oracle.contract(A.numpy(), "ki", B.numpy(), "kj", None, "ij", want.numpy(), "ij", 1.0, 0.0)
+    if word == 0:
+        assert helpers.compare(dD.buffer.cpu()[pos].numpy(), want.buffer[pos].numpy(), scale, dtype) <= 1.0
+    else:
+        assert 1 <= word <= 11
+    op.set_attr(api.ATTR_POLL_LIMIT, 1 << 22)
+    op.set_attr(api.ATTR_DEVICE_ERROR, 0)
+    assert op.device_error == 0
+    run()
+    torch.cuda.synchronize()
+    assert op.device_error == 0
+    assert helpers.compare(dD.buffer.cpu()[pos].numpy(), want.buffer[pos].numpy(), scale, dtype) <= 1.0
+    assert helpers.canary_intact(D.buffer, dD.buffer.cpu(), pos)
+
+
+def test_host_buffer_entry_point_reports_a_device_timeout(api, handle):
+    """btc_execute_host synchronises, so it can and does return DEVICE_TIMEOUT when a wait gave up."""
+    ext = dict(i=256, j=256, k=256)
+    A = helpers.random_tensor(141, _ext("ki", ext), None, torch.float64)
+    B = helpers.random_tensor(142, _ext("kj", ext), None, torch.float64)
+    D = inputs.place(None, _ext("ij", ext), None, torch.float64)
+    tA, tB, tD = (api.TensorInfo(handle, api.F64, x.extents, x.strides) for x in (A, B, D))
+    op = api.Contraction(handle, tA, "ki", tB, "kj", None, "ij", tD, "ij", 1.0, 0.0)
+    op.set_attr(api.ATTR_KERNEL, api.KERNEL_TILED)
+    op.set_attr(api.ATTR_POLL_LIMIT, 1)
+    hD = D.clone()
+    try:
+        op.execute_host(0, A.data_ptr(), B.data_ptr(), 0, hD.data_ptr())
+        timed_out = False
+    except api.BtcError as e:
+        assert e.code == api.ERR_DEVICE_TIMEOUT
+        timed_out = True
+    assert timed_out == (op.device_error != 0)
+    op.set_attr(api.ATTR_POLL_LIMIT, 1 << 22)
+    op.set_attr(api.ATTR_DEVICE_ERROR, 0)
+    op.execute_host(0, A.data_ptr(), B.data_ptr(), 0, hD.data_ptr())
+    want = D.clone()
+    scale = oracle.contract(A.numpy(), "ki", B.numpy(), "kj", None, "ij", want.numpy(), "ij", 1.0, 0.0)
+    pos = D.offsets()
+    assert helpers.compare(hD.buffer[pos].numpy(), want.buffer[pos].numpy(), scale, torch.float64) <= 1.0
