@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libbtc.so")
-SOURCES = ["btc_api.cu", "plan.cpp", "skinny_umma.cu", "peaks.cu"]
+SOURCES = ["btc_api.cu", "plan.cpp", "skinny_umma.cu", "stream.cu", "peaks.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v",

@@ -399,7 +399,12 @@ int finish_plan(btc_contraction_s *op)
     // occupy a good part of the machine
     const bool skinny_fits = pl.dtype == BTC_F32 && op->req.strict_fp32 == 0 && pl.K <= kSkinnyMaxK && pl.vecA == 4 && pl.vecB == 4;
     if (skinny_fits && ((pl.M + 127) / 128) * ((pl.N + 127) / 128) * pl.Bt * hint >= 32) variant = kSkinnyVariant;
-    if (op->req.force_variant >= 0) {
+    // at most four contracted indices (outer products, Hadamard products, a scalar operand): the streaming kernel
+    const bool stream_fits = pl.K <= kStreamMaxContracted;
+    if (stream_fits) variant = kStreamVariant;
+    if (op->req.force_variant == kStreamVariant) {
+        if (!stream_fits) return BTC_ERR_NOT_SUPPORTED;
+    } else if (op->req.force_variant >= 0) {
         const int count = pl.dtype == BTC_F32 ? kNumF32Variants : (pl.dtype == BTC_F64 ? 5 : (pl.dtype == BTC_C64 ? 3 : 2));
         if (op->req.force_variant >= count) return BTC_ERR_INVALID_ARGUMENT;
         variant = op->req.force_variant;
@@ -411,7 +416,19 @@ int finish_plan(btc_contraction_s *op)
         const VariantInfo bv = variant_info(pl.dtype, variant);
         if (!make_tma_operand(pl, bv.bm, bv.bk, op->tmaA)) variant = (variant <= 18 || variant == 21) ? 13 : 14;
     }
-    const VariantInfo v = variant_info(pl.dtype, variant);
+    if (variant == kStreamVariant) {
+        // no tiles: one thread per 16 bytes of D, grid-stride
+        pl.tile = TileConfig();
+        pl.tile.variant = variant;
+        pl.split_k = 1;
+        op->tiles_m = op->tiles_n = 0;
+        const int64_t vectors = (pl.M * pl.N * pl.Bt + 3) / 4;
+        int64_t blocks = (vectors + 255) / 256;
+        const int64_t cap = int64_t(sms) * 32;
+        op->grid[0] = int32_t(blocks < 1 ? 1 : (blocks > cap ? cap : blocks)); op->grid[1] = op->grid[2] = 1;
+    }
+    const VariantInfo v = variant == kStreamVariant ? VariantInfo{1, 1, 1, 0, 0, 0, 0} : variant_info(pl.dtype, variant);
+    if (variant != kStreamVariant) {
     pl.tile.bm = v.bm; pl.tile.bn = v.bn; pl.tile.bk = v.bk; pl.tile.threads = v.threads;
     pl.tile.stages = 0; pl.tile.variant = variant;
     op->tiles_m = int32_t((pl.M + v.bm - 1) / v.bm);
@@ -451,6 +468,7 @@ int finish_plan(btc_contraction_s *op)
     if (umma && op->grid[0] > sms) op->grid[0] = int32_t(sms);   // persistent CTAs walk the tile list
     if (split > 1)
         op->workspace_bytes = size_t(tiles) * size_t(split) * size_t(v.threads) * size_t(v.acc) * v.acc_bytes;
+    }   // tiled variants
 
     for (auto &o : op->skinny_order) o.clear();
     if (pl.dtype == BTC_F32 && variant == kSkinnyVariant) {
@@ -874,6 +892,7 @@ struct BatchView {
     const int64_t *offA_h, *offB_h, *offD_h;   // [count * Bt], planned roles
     void *partials;
     bool aligned16_D, aligned_A, aligned_B;     // every entry's pointer keeps the vector alignment
+    bool aligned16_A;                           // every entry's M-side input pointer is 16-byte aligned
 };
 
 btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A, const void *B,
@@ -1008,7 +1027,12 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
             ctas = persistent ? (work < op->handle.sm_count ? work : op->handle.sm_count) : work;
             reduce_ctas = (work / pl.split_k) * ((int64_t(pl.tile.bm) * pl.tile.bn + 1023) / 1024);
         }
-        if (pl.dtype == BTC_F32) {
+        if (pl.tile.variant == kStreamVariant) {
+            // 16-byte accesses along the first M mode where the plan's strides and these pointers allow
+            const bool vec_d = pl.rows16D && !misaligned(D, 16) && !(use_c && misaligned(C, 16)) && !(bv && !bv->aligned16_D);
+            const bool vec_a = vec_d && pl.rows16A && !misaligned(pA, 16) && !(bv && !bv->aligned16_A);
+            ce = launch_stream(tp, int(pl.dtype), vec_d, vec_a, op->handle.sm_count, st);
+        } else if (pl.dtype == BTC_F32) {
             switch (pl.tile.variant) {
             case 0: ce = launch_tiled_f32<F32Big>(tp, ctas, reduce_ctas, st); break;
             case 1: ce = launch_tiled_f32<F32Small>(tp, ctas, reduce_ctas, st); break;
@@ -1159,7 +1183,7 @@ btc_error_t btc_execute_batched(btc_contraction_t op, void *cuda_stream, const v
     int64_t *tA = tab.data(), *tB = tA + count * Bt, *tD = tB + count * Bt;
     BatchView bv;
     bv.count = count;
-    bv.aligned16_D = bv.aligned_A = bv.aligned_B = true;
+    bv.aligned16_D = bv.aligned_A = bv.aligned_B = bv.aligned16_A = true;
     const void *const *pA = pl.swapped ? B : A, *const *pB = pl.swapped ? A : B;
     for (int64_t i = 0; i < count; ++i) {
         const int64_t dA = reinterpret_cast<intptr_t>(pA[i]) - reinterpret_cast<intptr_t>(pA[0]);
@@ -1170,6 +1194,7 @@ btc_error_t btc_execute_batched(btc_contraction_t op, void *cuda_stream, const v
         if (use_c && reinterpret_cast<intptr_t>(C[i]) - reinterpret_cast<intptr_t>(C[0]) != dD) return BTC_ERR_NOT_SUPPORTED;
         bv.aligned_A = bv.aligned_A && reinterpret_cast<uintptr_t>(pA[i]) % size_t(pl.alignA) == 0;
         bv.aligned_B = bv.aligned_B && reinterpret_cast<uintptr_t>(pB[i]) % size_t(pl.alignB) == 0;
+        bv.aligned16_A = bv.aligned16_A && reinterpret_cast<uintptr_t>(pA[i]) % 16 == 0;
         bv.aligned16_D = bv.aligned16_D && reinterpret_cast<uintptr_t>(D[i]) % 16 == 0 &&
                          (!use_c || reinterpret_cast<uintptr_t>(C[i]) % 16 == 0);
         for (int64_t h = 0; h < Bt; ++h) {

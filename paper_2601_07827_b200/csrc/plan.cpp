@@ -361,14 +361,30 @@ int make_plan(const PlanRequest &req, Plan &plan)
         if (ok) plan.vecD = 4;
     }
 
+    {
+        const int64_t v = 16 / esz;          // elements in 16 bytes (1 for complex128: always whole)
+        auto rows16 = [&](bool inD) {
+            auto S = [&](const Mode &md) { return inD ? md.sD : md.sA; };
+            if (v == 1) return true;
+            if (plan.m.empty() || S(plan.m[0]) != 1 || plan.m[0].extent % v != 0) return false;
+            for (size_t i = 1; i < plan.m.size(); ++i) if (S(plan.m[i]) % v) return false;
+            for (auto &md : plan.batch) if (S(md) % v) return false;
+            for (auto &md : (inD ? plan.n : plan.k)) if (S(md) % v) return false;
+            return true;
+        };
+        plan.rows16D = rows16(true);
+        plan.rows16A = rows16(false);
+    }
+
     // ---- kernel choice ----
     const int64_t entries = 2 * (plan.M + plan.N + plan.K) + 3 * plan.Bt;
     const bool tiled_ok = !plan.has_isolated && entries <= kMaxTableEntries;
     plan.kernel = BTC_KERNEL_GENERIC;
     if (req.force_kernel == BTC_KERNEL_TILED && !tiled_ok) return BTC_ERR_NOT_SUPPORTED;
+    // (with at most four contracted indices the streaming kernel serves every size)
     if (req.force_kernel == BTC_KERNEL_TILED ||
         (req.force_kernel == BTC_KERNEL_AUTO && tiled_ok &&
-         double(plan.M) * double(plan.N) * double(plan.K) * double(plan.Bt) >= 32768.0))
+         (double(plan.M) * double(plan.N) * double(plan.K) * double(plan.Bt) >= 32768.0 || plan.K <= 4)))
         plan.kernel = BTC_KERNEL_TILED;
 
     if (plan.kernel == BTC_KERNEL_TILED) {

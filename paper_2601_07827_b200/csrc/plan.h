@@ -55,6 +55,9 @@ struct Plan {
     int32_t vecA = 1, vecB = 1;          // elements per global load that the strides allow
     int32_t vecD = 1;                    // 4: groups of four consecutive m are 16 aligned bytes of D
     int64_t alignA = 1, alignB = 1;      // required base-pointer alignment (bytes) for vecA / vecB
+    // any element type: groups of 16 bytes along the first M mode are contiguous, 16-byte aligned (given an aligned
+    // base) and whole in D / in A (what the streaming kernel for K <= 4 needs for its vector accesses)
+    bool rows16D = false, rows16A = false;
 
     // element-offset tables (host copies; the API object uploads them)
     std::vector<int64_t> offA_m, offD_m, offB_n, offD_n, offA_k, offB_k, offA_h, offB_h, offD_h;

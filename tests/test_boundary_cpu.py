@@ -147,8 +147,11 @@ def test_planner_kernel_choice_and_split_k(api, handle):
     assert op.split_k == 1 and op.workspace_size() == 0
     op.set_attr(api.ATTR_KERNEL, api.KERNEL_GENERIC)
     assert op.kernel == api.KERNEL_GENERIC
-    tiny = _op(api, handle, (2, 3), "ik", (3, 2), "kj", (2, 2), "ij")
+    tiny = _op(api, handle, (2, 5), "ik", (5, 2), "kj", (2, 2), "ij")
     assert tiny.kernel == api.KERNEL_GENERIC
+    # at most four contracted indices: the streaming kernel, whatever the size
+    tiny = _op(api, handle, (2, 3), "ik", (3, 2), "kj", (2, 2), "ij")
+    assert tiny.kernel == api.KERNEL_TILED and tiny.variant == 100
     # Case 4, isolated label x: by default A is first summed over x into the workspace and the tiled
     # kernel contracts the result; with the pre-reduction off the generic kernel sums x itself
     case4 = _op(api, handle, (64, 64, 5), "ikx", (64, 64), "kj", (64, 64), "ij")

@@ -101,8 +101,11 @@ def test_paper_test_categories(api, handle, cat, dtype):
     cplx = dtype.is_complex
     alpha = complex(0.75, -1.25) if cplx else 0.75
     beta = complex(-0.5, 0.25) if cplx else -0.5
-    worst, _, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, beta, conjA=cplx, conjC=cplx)
+    worst, status, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, beta, conjA=cplx, conjC=cplx, want_status=True)
     assert worst <= 1.0, worst
+    if cat in ("hadamard", "outer_product", "zero_mode_A"):
+        # no contracted label: the bandwidth-bound streaming kernel (Appendix "Testing" items 1, 6, 8)
+        assert status["variant"] == 100 and status["launches"] == 1, status
 
 
 def test_strict_fp32_precision_runs_the_fma_kernels(api, handle):
@@ -512,3 +515,36 @@ def test_host_buffer_entry_point_reports_a_device_timeout(api, handle):
     scale = oracle.contract(A.numpy(), "ki", B.numpy(), "kj", None, "ij", want.numpy(), "ij", 1.0, 0.0)
     pos = D.offsets()
     assert helpers.compare(hD.buffer[pos].numpy(), want.buffer[pos].numpy(), scale, torch.float64) <= 1.0
+
+
+STREAM = {
+    # name: (labelsA, labelsB, labelsD, extents, strides of D or None)
+    "outer_product_vector_rows": ("ij", "kl", "ijkl", dict(i=64, j=9, k=7, l=5), None),
+    "outer_product_odd_rows": ("ij", "kl", "ijkl", dict(i=37, j=9, k=7, l=5), None),
+    "rank_two_update": ("ik", "kj", "ij", dict(i=260, j=130, k=2), None),
+    "four_contracted_batch": ("kiz", "jkz", "ijz", dict(i=72, j=50, k=4, z=6), None),
+    "three_contracted_rows_strided_in_A": ("ki", "kj", "ij", dict(i=128, j=33, k=3), None),
+    "scalar_times_tensor_permuted": ("", "ijk", "kji", dict(i=20, j=12, k=36), None),
+    "hadamard_three_labels": ("ijk", "ijk", "ijk", dict(i=32, j=11, k=9), None),
+    "padded_output": ("i", "j", "ij", dict(i=96, j=40), (1, 100)),
+}
+
+
+@pytest.mark.parametrize("dtype", REAL_AND_COMPLEX)
+@pytest.mark.parametrize("name", list(STREAM))
+def test_streaming_kernel_for_at_most_four_contracted_indices(api, handle, name, dtype):
+    """Outer products, rank-k updates with k <= 4, a scalar operand, Hadamard products: the streaming kernel
+    (one thread per 16 bytes of D) for every element type, with and without 16-byte rows in D and A, beta != 0,
+    conjugation, a batch label, padding in D."""
+    la, lb, ld, ext, sD = STREAM[name]
+    A = helpers.random_tensor(151, _ext(la, ext), None, dtype)
+    B = helpers.random_tensor(152, _ext(lb, ext), None, dtype)
+    C = helpers.random_tensor(153, _ext(ld, ext), sD, dtype)
+    D = inputs.place(None, _ext(ld, ext), sD, dtype)
+    cplx = dtype.is_complex
+    alpha = complex(0.75, -1.25) if cplx else 0.75
+    beta = complex(-0.5, 0.25) if cplx else -0.5
+    worst, status, _ = helpers.run_case(handle, A, la, B, lb, C, D, ld, alpha, beta, conjA=cplx, conjB=cplx, conjC=cplx,
+                                        want_status=True)
+    assert worst <= 1.0, worst
+    assert status["variant"] == 100 and status["launches"] == 1, status
