@@ -83,7 +83,13 @@ def roofline_for(w, kernel_ms, variant=-1, units=1):
     gbs = nbytes / (kernel_ms * 1e-3) / 1e9
     f32 = w.dtype in ("f32", "c32")
     umma = f32 and (10 <= variant <= 21 or variant == 23)
-    if not f32:
+    if variant == 100:
+        # at most four contracted indices: FMA pipe of the element type
+        kernel, bound, executed = "stream_kernel", "alu", flops
+        peak = FP32_PEAK_TFLOPS if f32 else FP64_PEAK_TFLOPS
+        peak_measured = PEAKS.get("fp32_fma_tflops" if f32 else "fp64_fma_tflops")
+        source = "FMA pipe of the element type (unit count); peak_measured = the register-resident FMA loop of this run"
+    elif not f32:
         kernel, bound, executed = "tiled_f64_kernel", "tensor", flops
         peak, peak_measured = FP64_PEAK_TFLOPS, PEAKS.get("fp64_mma_m16n8k16_tflops")
         source = ("FP64 tensor (DMMA) pipe: 148 SMs x 64 FMA/clk x 2 x 1.965 GHz (unit count); peak_measured = the "
@@ -489,7 +495,7 @@ def per_config(args, torch, api, inputs, handle):
             ("single", "cfg3_f32_batched_permuted", False), ("single", "cfg4_c64_conj", False), ("single", "cfg4c_c32_conj", False),
             ("single", "cfg5_f32_tensor_network", True), ("batched", "cfg5_f32_tensor_network", 64),
             ("single", "cfg5b_f32_tensor_network_rev", True), ("batched", "cfg5b_f32_tensor_network_rev", 64),
-            ("single", "cfg6_f64_case4_isolated", False)] + [("ew", name, None) for name in E]
+            ("single", "cfg6_f64_case4_isolated", False), ("single", "cfg7_f32_outer_product", False)] + [("ew", name, None) for name in E]
     for kind, name, arg in plan:
         try:
             if kind == "single":

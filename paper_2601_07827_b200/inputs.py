@@ -338,6 +338,9 @@ def workloads() -> Dict[str, Workload]:
     # 5b: same with D's fastest label being B's slowest (adversarial output order)
     w["cfg5b_f32_tensor_network_rev"] = dataclasses.replace(
         w["cfg5_f32_tensor_network"], name="cfg5b_f32_tensor_network_rev", labelsD="jeidhcgbfa")
+    # 7: outer product with interleaved output labels (no contracted label): 1 GiB of D from two 64 KiB inputs
+    w["cfg7_f32_outer_product"] = Workload(
+        "cfg7_f32_outer_product", "f32", "ab", "cd", "acbd", _all(128, "abcd"), alpha=1.0, beta=0.0, seed=7000)
     # 6: Case 4, the ladder term with an extra label x that only A carries (summed over first):
     #    D[a,b,i,j] = sum_cd (sum_x A[a,b,c,d,x]) T[c,d,i,j];  A is 1 GiB, the sum over x is HBM-bound
     e6 = {**_all(64, "abcd"), **_all(32, "ij"), "x": 8}
