@@ -343,6 +343,11 @@ int finish_plan(btc_contraction_s *op)
         op->grid[0] = int32_t(blocks); op->grid[1] = warp_per_elem ? 32 : 1; op->grid[2] = 1;
         pl.tile = TileConfig();
         pl.split_k = 1;
+        if (op->handle.device >= 0) {            // no tables, only the device error word
+            if (cudaMalloc(reinterpret_cast<void **>(&op->d_tables), 256) != cudaSuccess) { cudaGetLastError(); op->d_tables = nullptr; return BTC_ERR_OUT_OF_MEMORY; }
+            if (cudaMemset(op->d_tables, 0, 256) != cudaSuccess) { cudaGetLastError(); return BTC_ERR_CUDA; }
+            op->d_error = reinterpret_cast<int32_t *>(op->d_tables);
+        }
         return BTC_SUCCESS;
     }
 
@@ -908,6 +913,22 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream, const void *alp
 }
 
 namespace {
+// Spans of the tensors the kernels address, in planned roles (a Case 4 input that was summed first is
+// the dense result of that sum); a pointer-array batch reaches other buffers, so its spans are left open.
+void fill_spans(const btc_contraction_s *op, OffsetSpans &sp, bool open = false)
+{
+    const int64_t big = int64_t(1) << 62;
+    int64_t lo[2] = {op->spanA_lo, op->spanB_lo}, hi[2] = {op->spanA_hi, op->spanB_hi};
+    if (op->sumA.active) { lo[0] = 0; hi[0] = op->sumA.total_keep - 1; }
+    if (op->sumB.active) { lo[1] = 0; hi[1] = op->sumB.total_keep - 1; }
+    const int a = op->plan.swapped ? 1 : 0;
+    sp.lo[0] = lo[a]; sp.hi[0] = hi[a]; sp.lo[1] = lo[1 - a]; sp.hi[1] = hi[1 - a];
+    sp.lo[2] = op->spanD_lo; sp.hi[2] = op->spanD_hi;
+    if (open)
+        for (int i = 0; i < 3; ++i) { sp.lo[i] = -big; sp.hi[i] = big; }
+    sp.error_word = op->d_error;
+}
+
 btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A, const void *B,
                          const void *beta, const void *C, void *D, void *workspace, size_t workspace_bytes,
                          btc_status_t *status, const BatchView *bv)
@@ -972,6 +993,7 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
         gp.alpha[0] = al[0]; gp.alpha[1] = al[1]; gp.beta[0] = be[0]; gp.beta[1] = be[1];
         gp.conjA = pl.conjA; gp.conjB = pl.conjB; gp.conjC = pl.conjC;
         gp.use_ab = use_ab; gp.use_c = use_c;
+        fill_spans(op, gp.spans);
         bool wpe = pl.kernel == BTC_KERNEL_GENERIC && op->grid[1] == 32;
         int blocks = op->grid[0];
         if (pl.kernel != BTC_KERNEL_GENERIC) {   // alpha == 0 on a tiled plan: D = beta * op(C)
@@ -1006,6 +1028,7 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
         tp.partials = workspace ? static_cast<char *>(workspace) + op->partials_offset : nullptr;
         tp.error_word = op->d_error;
         tp.poll_limit = op->poll_limit;
+        fill_spans(op, tp.spans, bv != nullptr);
         tp.tmaA_coord_m = op->d_tma_coord_m; tp.tmaA_coord_k = op->d_tma_coord_k; tp.tmaA_coord_h = op->d_tma_coord_h;
         tp.skinny_orderA = op->d_skinny_order[0]; tp.skinny_orderB = op->d_skinny_order[3];
         tp.skinny_regular = op->skinny_regular ? 1 : 0;
@@ -1061,6 +1084,7 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
                         std::swap(sp.M, sp.N); std::swap(sp.tiles_m, sp.tiles_n);
                         std::swap(sp.dirA, sp.dirB); std::swap(sp.vecA, sp.vecB);
                         std::swap(sp.conjA, sp.conjB);
+                        std::swap(sp.spans.lo[0], sp.spans.lo[1]); std::swap(sp.spans.hi[0], sp.spans.hi[1]);
                         sp.skinny_orderA = op->d_skinny_order[2]; sp.skinny_orderB = op->d_skinny_order[1];
                         sp.skinny_vec_n = 4;
                     }

@@ -119,6 +119,7 @@ __device__ __forceinline__ void store_tile_image(const TiledParams &p, const Til
                 const int idx = base + u * NT;
                 const int row = (idx % (BM / V)) * V, col = idx / (BM / V);
                 ok[u] = idx < COUNT && row < tc.rows_valid && col < tc.cols_valid;   // rows_valid % V == 0 here
+                ok[u] = ok[u] && BTC_IN_SPAN(p.spans, 2, rowD[row] + colD[col], V);
                 if (ok[u] && p.use_c)
                     c[u].raw = *reinterpret_cast<const uint4 *>(static_cast<const Acc *>(p.C) + (rowD[row] + colD[col]) * W);
             }
@@ -142,6 +143,7 @@ __device__ __forceinline__ void store_tile_image(const TiledParams &p, const Til
                 const int idx = base + u * NT;
                 const int row = idx % BM, col = idx / BM;
                 ok[u] = idx < COUNT && row < tc.rows_valid && col < tc.cols_valid;
+                ok[u] = ok[u] && BTC_IN_SPAN(p.spans, 2, rowD[row] + colD[col], 1);
                 c_r[u] = c_i[u] = Acc(0);
                 if (ok[u] && p.use_c) {
                     const Acc *cp = static_cast<const Acc *>(p.C) + (rowD[row] + colD[col]) * W;
@@ -191,6 +193,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const TiledParams p)
         const int row = idx % bm, col = idx / bm;
         if (idx >= bm * bn || row >= rows_valid || col >= cols_valid) continue;
         const int64_t off = p.offD_m[m0 + row] + hD + p.offD_n[n0 + col];
+        if (!BTC_IN_SPAN(p.spans, 2, off, 1)) continue;
         Acc c_r = 0, c_i = 0;
         if (p.use_c) {
             const Acc *cp = static_cast<const Acc *>(p.C) + off * W;

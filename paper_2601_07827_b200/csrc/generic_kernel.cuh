@@ -47,6 +47,7 @@ __global__ void __launch_bounds__(256) generic_contract_kernel(const GenericPara
                     oa += i * p.sA_k[d];
                     ob += i * p.sB_k[d];
                 }
+                if (!BTC_IN_SPAN(p.spans, 0, oa, 1) || !BTC_IN_SPAN(p.spans, 1, ob, 1)) continue;
                 const double ar = double(A[NC * oa]), br = double(B[NC * ob]);
                 if (CPLX) {
                     const double ai = sa * double(A[NC * oa + (NC - 1)]);
@@ -65,7 +66,7 @@ __global__ void __launch_bounds__(256) generic_contract_kernel(const GenericPara
                 }
             }
         }
-        if (lane == 0) {
+        if (lane == 0 && BTC_IN_SPAN(p.spans, 2, offD, 1)) {
             double d_r = p.alpha[0] * acc_r - p.alpha[1] * acc_i;
             double d_i = p.alpha[0] * acc_i + p.alpha[1] * acc_r;
             if (p.use_c) {

@@ -5,6 +5,27 @@
 
 namespace btc {
 
+// Memory span of each tensor in elements relative to its pointer ([lo, hi] inclusive; 0: M-side input,
+// 1: N-side input, 2: D and C) and the device error word.  Debug builds (-DBTC_CHECK_OFFSETS) compare every
+// global offset the kernels compute with these and record kErrOffsetRange instead of making the access.
+struct OffsetSpans {
+    int64_t lo[3], hi[3];
+    int32_t *error_word;
+};
+constexpr int kErrOffsetRange = 20;
+
+#if defined(BTC_CHECK_OFFSETS) && defined(__CUDACC__)
+__device__ __forceinline__ bool offset_in_span(const OffsetSpans &s, int which, int64_t off, int count)
+{
+    const bool ok = off >= s.lo[which] && off + count - 1 <= s.hi[which];
+    if (!ok && s.error_word) atomicCAS(s.error_word, 0, kErrOffsetRange);
+    return ok;
+}
+#define BTC_IN_SPAN(spans, which, off, count) offset_in_span(spans, which, off, count)
+#else
+#define BTC_IN_SPAN(spans, which, off, count) true
+#endif
+
 constexpr int kGenericMaxD = 32;   // loop dimensions over D (batch + free), after merging
 constexpr int kGenericMaxK = 64;   // summed loop dimensions
 
@@ -19,6 +40,7 @@ struct GenericParams {
     double alpha[2], beta[2];
     int32_t conjA, conjB, conjC;
     int32_t use_ab, use_c;
+    OffsetSpans spans;
 };
 
 // Sum over the isolated labels of one input (Case 4): kept and isolated loop dimensions of the
@@ -71,6 +93,7 @@ struct TiledParams {
     void *partials;                   // split-K scratch (workspace), or nullptr
     int32_t *error_word;              // device word; set non-zero when a bounded wait gave up
     uint32_t poll_limit;              // polls after which a device-side wait gives up
+    OffsetSpans spans;                // what the offset checks of debug builds compare with
     // bulk-tensor-copy variants: box origin of the M-side operand = coord_m[tile of M] + coord_k[stage]
     // + coord_h[batch entry], five coordinates each
     const int32_t *tmaA_coord_m, *tmaA_coord_k, *tmaA_coord_h;

@@ -77,7 +77,7 @@ constexpr int kErrSkinnyLoad = 8, kErrSkinnyConvert = 9, kErrSkinnyMma = 10, kEr
 // in piece order: .x bits 0-10 destination in 16-byte units, bits 11-17 first row, bits 18-23 first k,
 // bit 24 k < K;  .y element offset of the piece relative to the tile's first row (regular operands).
 __device__ __forceinline__ void skinny_load_tile(unsigned tile, const float *g, const int64_t *row_off, const int64_t *koff,
-                                                 const uint2 *table, int pieces, int rows_valid, int pt)
+                                                 const uint2 *table, int pieces, int rows_valid, int pt, const OffsetSpans &spans, int which)
 {
 #pragma unroll 1
     for (int e0 = pt; e0 < pieces; e0 += 8 * SkinnyTile::GROUP_THREADS) {
@@ -92,6 +92,7 @@ __device__ __forceinline__ void skinny_load_tile(unsigned tile, const float *g, 
             dst[j] = (pk & 2047u) << 4;
             valid[j] = ((pk >> 24) & 1u) && row < rows_valid;
             off[j] = valid[j] ? row_off[row] + koff[k] : 0;
+            if (valid[j] && !BTC_IN_SPAN(spans, which, off[j], 4)) { valid[j] = false; off[j] = 0; }
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j)
@@ -99,8 +100,9 @@ __device__ __forceinline__ void skinny_load_tile(unsigned tile, const float *g, 
     }
 }
 // The same for a regular operand (every tile's rows lie relative to its first row as tile 0's do):
-// `g` points at the tile's first row, the table gives the rest; no offset arrays are needed.
-__device__ __forceinline__ void skinny_load_tile_regular(unsigned tile, const float *g, const uint2 *table, int pieces, int rows_valid, int pt)
+// `base` is the offset of the tile's first row, the table gives the rest; no offset arrays are needed.
+__device__ __forceinline__ void skinny_load_tile_regular(unsigned tile, const float *g, int64_t base, const uint2 *table, int pieces, int rows_valid,
+                                                         int pt, const OffsetSpans &spans, int which)
 {
 #pragma unroll 1
     for (int e0 = pt; e0 < pieces; e0 += 8 * SkinnyTile::GROUP_THREADS) {
@@ -112,9 +114,10 @@ __device__ __forceinline__ void skinny_load_tile_regular(unsigned tile, const fl
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const bool valid = ((q[j].x >> 24) & 1u) && int((q[j].x >> 11) & 127u) < rows_valid;
+            bool valid = ((q[j].x >> 24) & 1u) && int((q[j].x >> 11) & 127u) < rows_valid;
+            valid = valid && BTC_IN_SPAN(spans, which, base + int(q[j].y), 4);
             if (e0 + j * SkinnyTile::GROUP_THREADS < pieces)
-                cp_async_bytes<16>(tile + ((q[j].x & 2047u) << 4), g + (valid ? int(q[j].y) : 0), valid);
+                cp_async_bytes<16>(tile + ((q[j].x & 2047u) << 4), g + (valid ? base + int(q[j].y) : 0), valid);
         }
     }
 }
@@ -237,7 +240,8 @@ struct SkinnyStore {
                         float4 cv[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
-                            cv[q] = (row_ok && 4 * (q0 + q) < cols_here) ? *reinterpret_cast<const float4 *>(C + off[q0 + q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            cv[q] = (row_ok && 4 * (q0 + q) < cols_here && BTC_IN_SPAN(p.spans, 2, off[q0 + q], 4))
+                                        ? *reinterpret_cast<const float4 *>(C + off[q0 + q]) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             v[q0 + q].x += beta * cv[q].x; v[q0 + q].y += beta * cv[q].y;
@@ -247,13 +251,13 @@ struct SkinnyStore {
                 }
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
-                    if (row_ok && 4 * q < cols_here) *reinterpret_cast<float4 *>(D + off[q]) = v[q];
+                    if (row_ok && 4 * q < cols_here && BTC_IN_SPAN(p.spans, 2, off[q], 4)) *reinterpret_cast<float4 *>(D + off[q]) = v[q];
             } else {
                 const int64_t mine = c0 == 0 ? co[0] : c0 == 32 ? co[1] : c0 == 64 ? co[2] : co[3];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     const int64_t off = ro + (dreg ? co[0] + p.skinny_col_rel[c0 + j] : __shfl_sync(0xffffffffu, mine, j));
-                    if (row_ok && j < cols_here) {
+                    if (row_ok && j < cols_here && BTC_IN_SPAN(p.spans, 2, off, 1)) {
                         float v = alpha * __uint_as_float(r[j]);
                         if (p.use_c) v += beta * C[off];
                         D[off] = v;
@@ -512,16 +516,16 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             if (t + 1 < t1) fetch(wn);
             if (new_strip) {
                 if (sidx > 0 && !mbar_wait_bounded(a_empty, unsigned(sidx - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
-                if (regular) skinny_load_tile_regular(araw, A + row_base, pieceA, pieces, w.rows_valid, pt);
-                else skinny_load_tile(araw, A, rA, koffA, pieceA, pieces, w.rows_valid, pt);
+                if (regular) skinny_load_tile_regular(araw, A, row_base, pieceA, pieces, w.rows_valid, pt, p.spans, 0);
+                else skinny_load_tile(araw, A, rA, koffA, pieceA, pieces, w.rows_valid, pt, p.spans, 0);
                 mbar_arrive_on_copies(a_full);
             }
             BTC_PHASE_END(t_work);
             if (i >= 2 && !mbar_wait_bounded(b_empty0 + 8u * s, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
             BTC_PHASE_END(t_wait);
             BTC_EVENT(p, pt == 0, 0, i);
-            if (regular) skinny_load_tile_regular(braw0 + unsigned(s) * T::B_BYTES, B + col_base, pieceB, pieces, w.cols_valid, pt);
-            else skinny_load_tile(braw0 + unsigned(s) * T::B_BYTES, B, cB, koffB, pieceB, pieces, w.cols_valid, pt);
+            if (regular) skinny_load_tile_regular(braw0 + unsigned(s) * T::B_BYTES, B, col_base, pieceB, pieces, w.cols_valid, pt, p.spans, 1);
+            else skinny_load_tile(braw0 + unsigned(s) * T::B_BYTES, B, cB, koffB, pieceB, pieces, w.cols_valid, pt, p.spans, 1);
             mbar_arrive_on_copies(b_full0 + 8u * s);
             BTC_EVENT(p, pt == 0, 1, i);
             w = wn;

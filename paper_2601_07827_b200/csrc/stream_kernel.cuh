@@ -67,6 +67,10 @@ __global__ void __launch_bounds__(kStreamThreads) stream_kernel(const TiledParam
         if (k >= K) continue;
         koB[k] = p.offB_k[k] + hB;
         const int64_t ko = p.offA_k[k];
+#ifdef BTC_CHECK_OFFSETS
+        for (int v = 0; v < V; ++v)
+            if (!BTC_IN_SPAN(p.spans, 0, ((V > 1 && VEC_A) ? xA + v : p.offA_m[m + v] + p.offA_h[h]) + ko, 1)) return;
+#endif
         if (V > 1 && VEC_A) {
             a[k].raw = *reinterpret_cast<const uint4 *>(A + (xA + ko) * W);
         } else {
@@ -87,6 +91,11 @@ __global__ void __launch_bounds__(kStreamThreads) stream_kernel(const TiledParam
         if (y >= p.N) break;
         const int64_t oB = p.offB_n[y];
         const int64_t oD = xD + p.offD_n[y];
+#ifdef BTC_CHECK_OFFSETS
+        bool in_span = BTC_IN_SPAN(p.spans, 2, oD, V);
+        for (int k = 0; k < K; ++k) in_span = in_span && BTC_IN_SPAN(p.spans, 1, oB + koB[k], 1);
+        if (!in_span) continue;
+#endif
         R acc[V][W];
 #pragma unroll
         for (int v = 0; v < V; ++v)

@@ -106,7 +106,7 @@ template <int REGS> __device__ __forceinline__ void reg_dec() { asm volatile("se
 template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES, int DIR, int VEC>
 __device__ __forceinline__ void gather_tile(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
                                             const int64_t *koff, int rows_valid, int64_t k0,
-                                            int64_t k_end, int s_row, int s_k, int tid)
+                                            int64_t k_end, int s_row, int s_k, int tid, const OffsetSpans &spans, int which)
 {
     constexpr int NFAST = (DIR == 0 ? ROWS : BK) / VEC;
     constexpr int SLOTS = ROWS * BK / VEC;
@@ -126,6 +126,7 @@ __device__ __forceinline__ void gather_tile(unsigned smem, const char *__restric
             const int k = DIR == 0 ? o : f;
             valid[j] = s < SLOTS && (r < rows_valid) && (k0 + k < k_end);
             off[j] = valid[j] ? row_off[r] + koff[k0 + k] : 0;
+            if (valid[j] && !BTC_IN_SPAN(spans, which, off[j], VEC)) { valid[j] = false; off[j] = 0; }
         }
 #pragma unroll
         for (int j = 0; j < BATCH; ++j) {
@@ -143,26 +144,26 @@ __device__ __forceinline__ void gather_tile(unsigned smem, const char *__restric
 template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES, int DIR>
 __device__ __forceinline__ void gather_dispatch_vec(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
                                                     const int64_t *koff, int rows_valid, int64_t k0,
-                                                    int64_t k_end, int vec, int s_row, int s_k, int tid)
+                                                    int64_t k_end, int vec, int s_row, int s_k, int tid, const OffsetSpans &spans, int which)
 {
     constexpr int VMAX = 16 / ELEM_BYTES;   // 4 for fp32, 2 for fp64 and complex64, 1 for complex128
     if (VMAX >= 4 && vec == 4)
-        gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, DIR, (VMAX >= 4 ? 4 : 1)>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
+        gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, DIR, (VMAX >= 4 ? 4 : 1)>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid, spans, which);
     else if (VMAX >= 2 && vec == 2)
-        gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, DIR, (VMAX >= 2 ? 2 : 1)>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
+        gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, DIR, (VMAX >= 2 ? 2 : 1)>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid, spans, which);
     else
-        gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, DIR, 1>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid);
+        gather_tile<ROWS, BK, NTHREADS, ELEM_BYTES, DIR, 1>(smem, g, row_off, koff, rows_valid, k0, k_end, s_row, s_k, tid, spans, which);
 }
 
 template <int ROWS, int BK, int NTHREADS, int ELEM_BYTES>
 __device__ __forceinline__ void gather_dispatch(unsigned smem, const char *__restrict__ g, const int64_t *row_off,
                                                 const int64_t *koff, int rows_valid, int64_t k0,
-                                                int64_t k_end, int dir, int vec, int s_row, int s_k, int tid)
+                                                int64_t k_end, int dir, int vec, int s_row, int s_k, int tid, const OffsetSpans &spans, int which)
 {
     if (dir == 0)
-        gather_dispatch_vec<ROWS, BK, NTHREADS, ELEM_BYTES, 0>(smem, g, row_off, koff, rows_valid, k0, k_end, vec, s_row, s_k, tid);
+        gather_dispatch_vec<ROWS, BK, NTHREADS, ELEM_BYTES, 0>(smem, g, row_off, koff, rows_valid, k0, k_end, vec, s_row, s_k, tid, spans, which);
     else
-        gather_dispatch_vec<ROWS, BK, NTHREADS, ELEM_BYTES, 1>(smem, g, row_off, koff, rows_valid, k0, k_end, vec, s_row, s_k, tid);
+        gather_dispatch_vec<ROWS, BK, NTHREADS, ELEM_BYTES, 1>(smem, g, row_off, koff, rows_valid, k0, k_end, vec, s_row, s_k, tid, spans, which);
 }
 
 
@@ -258,9 +259,9 @@ __device__ __forceinline__ void producer_loop(const Params &p, const TileCoords 
         const unsigned sb = sa + A_BYTES;
         const int64_t k0 = c.k_begin + int64_t(kt) * BK;
         gather_dispatch<BM, BK, PRODUCERS, EB>(sa, static_cast<const char *>(p.A), rowA, ka, c.rows_valid, k0,
-                                               c.k_end, p.dirA, p.vecA, a_srow, a_sk, tid);
+                                               c.k_end, p.dirA, p.vecA, a_srow, a_sk, tid, p.spans, 0);
         gather_dispatch<BN, BK, PRODUCERS, EB>(sb, static_cast<const char *>(p.B), colB, kb, c.cols_valid, k0,
-                                               c.k_end, p.dirB, p.vecB, b_srow, b_sk, tid);
+                                               c.k_end, p.dirB, p.vecB, b_srow, b_sk, tid, p.spans, 1);
         mbar_arrive_on_copies(full0 + 8u * s);
     }
     cp_async_wait_all();

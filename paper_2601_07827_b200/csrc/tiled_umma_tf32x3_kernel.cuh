@@ -219,6 +219,8 @@ struct UmmaOperand {
     int64_t k_begin, k_end;
     int dir;                     // 1: k is the contiguous direction, 0: the rows are
     int vec;                     // 4: every 16-byte piece is contiguous, aligned and in range as a whole
+    const OffsetSpans *spans;    // debug builds: what the offsets are checked against
+    int which;
 };
 
 // The 16-byte pieces of an R x 32 operand tile that producer thread pt (0..127) copies: R / 16
@@ -294,8 +296,10 @@ __device__ __forceinline__ void umma_produce(unsigned tile, const UmmaProducerLa
         for (int i = 0; i < SLOTS; ++i) {
             const bool second = umma_slot_half<R>(o.dir, i) != 0;
             if (BK < 32 && second && l.kq + 16 >= BK) continue;
-            const bool valid = ((l.rows_in >> i) & 1u) && (second ? so.in1 : so.in0);
-            cp_async_bytes<16>(tile + l.pos0 + umma_slot_pos<R>(o.dir, i), o.g + l.rowoff[i] + (second ? so.kofs1 : so.kofs0), valid);
+            bool valid = ((l.rows_in >> i) & 1u) && (second ? so.in1 : so.in0);
+            int64_t off = l.rowoff[i] + (second ? so.kofs1 : so.kofs0);
+            if (valid && !BTC_IN_SPAN(*o.spans, o.which, off, 4)) { valid = false; off = 0; }
+            cp_async_bytes<16>(tile + l.pos0 + umma_slot_pos<R>(o.dir, i), o.g + off, valid);
         }
     } else {
 #pragma unroll 2
@@ -311,6 +315,7 @@ __device__ __forceinline__ void umma_produce(unsigned tile, const UmmaProducerLa
                 const int64_t ke = k + (o.dir == 1 ? e : 0);
                 in[e] = re < o.rows_valid && ke < o.k_end;
                 off[e] = in[e] ? o.row_off[re] + o.koff[ke] : 0;
+                if (in[e] && !BTC_IN_SPAN(*o.spans, o.which, off[e], 1)) { in[e] = false; off[e] = 0; }
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e)
@@ -445,10 +450,10 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 float cv[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    cv[j] = (p.use_c && row_ok && c0 + j < tc.cols_valid) ? C[ro + cD[c0 + j]] : 0.f;
+                    cv[j] = (p.use_c && row_ok && c0 + j < tc.cols_valid && BTC_IN_SPAN(p.spans, 2, ro + cD[c0 + j], 1)) ? C[ro + cD[c0 + j]] : 0.f;
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    if (row_ok && c0 + j < tc.cols_valid) {
+                    if (row_ok && c0 + j < tc.cols_valid && BTC_IN_SPAN(p.spans, 2, ro + cD[c0 + j], 1)) {
                         float v = alpha * __uint_as_float(r[j]);
                         if (p.use_c) v += beta * cv[j];
                         D[ro + cD[c0 + j]] = v;
@@ -600,8 +605,8 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 for (int i = pt; i < T::BN; i += T::PRODUCER_THREADS) cB[i] = i < tc.cols_valid ? p.offB_n[tc.n0 + i] + hB : 0;
             }
             if (!umma_group_sync(producer_sync0 + 8u * buf, unsigned(n >> 1) & 1u, abort_flag, p.error_word, p.poll_limit)) break;
-            const UmmaOperand opA = {static_cast<const float *>(p.A), rA, staged ? koffA : p.offA_k, tc.rows_valid, 0, p.K, p.dirA, p.vecA};
-            const UmmaOperand opB = {static_cast<const float *>(p.B), cB, staged ? koffB : p.offB_k, tc.cols_valid, 0, p.K, p.dirB, p.vecB};
+            const UmmaOperand opA = {static_cast<const float *>(p.A), rA, staged ? koffA : p.offA_k, tc.rows_valid, 0, p.K, p.dirA, p.vecA, &p.spans, 0};
+            const UmmaOperand opB = {static_cast<const float *>(p.B), cB, staged ? koffB : p.offB_k, tc.cols_valid, 0, p.K, p.dirB, p.vecB, &p.spans, 1};
             UmmaProducerLane<T::BM> la;
             UmmaProducerLane<T::BN> lb;
             if (!T::A_TMA) umma_producer_init<T::BM>(la, opA, pt);

@@ -67,10 +67,12 @@ def run_case(handle, A, la, B, lb, C, D, ld, alpha=1.0, beta=0.0, conjA=False, c
         op.execute_host(0, A.data_ptr(), B.data_ptr(), hC.data_ptr() if hC is not None else 0, hD.data_ptr())
         result = hD.buffer
     else:
-        _, status = _api.contract(handle, dA, la, dB, lb, dC, dD, ld, alpha, beta, conjA, conjB, conjC,
-                                  stream=torch.cuda.current_stream().cuda_stream, kernel=kernel,
-                                  split_k=split_k, want_status=want_status, variant=variant, pre_reduce=pre_reduce)
+        op, status = _api.contract(handle, dA, la, dB, lb, dC, dD, ld, alpha, beta, conjA, conjB, conjC,
+                                   stream=torch.cuda.current_stream().cuda_stream, kernel=kernel,
+                                   split_k=split_k, want_status=want_status, variant=variant, pre_reduce=pre_reduce)
         torch.cuda.synchronize()
+        # no bounded wait gave up; in builds with offset checks (BTC_CHECK_OFFSETS=1): no offset left its tensor
+        assert op.device_error == 0, op.device_error
         result = dD.buffer.cpu()
 
     # oracle on the same inputs
