@@ -182,7 +182,13 @@ btc_error_t btc_execute(btc_contraction_t op, void *cuda_stream,
                         btc_status_t *status);
 
 /* Convenience for callers whose buffers live in HOST memory: copies A, B (and C when beta != 0)
- * to device buffers it allocates, executes, copies D back, frees, and synchronises the stream.
+ * to device buffers it allocates, executes, copies D back, and synchronises the stream.  Large
+ * operations run in slabs: the larger input is cut along the label with its largest stride and slab
+ * i + 1 is copied (on a stream of the library's own) while slab i is contracted, so that the transfer
+ * hides the arithmetic; a contracted label's slabs accumulate into D, which changes the order of the
+ * sum, not its value beyond rounding.  The device buffers of this path stay with the operation object
+ * until it is destroyed or re-planned; calls on one operation object must not overlap in time.
+ * Pinned host memory is what lets the copies overlap.
  * Pointers address logical element (0,...,0) of host tensors laid out as the descriptors say;
  * each tensor's whole strided span is transferred.  Errors as btc_execute plus OUT_OF_MEMORY, and
  * DEVICE_TIMEOUT when a bounded device-side wait gave up (D is then incomplete). */

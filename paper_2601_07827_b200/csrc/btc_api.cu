@@ -78,6 +78,23 @@ struct btc_contraction_s {
     size_t sumB_offset = 0, partials_offset = 0;
     // memory spans of the caller's tensors in elements (the plan may describe A' and B' instead)
     int64_t spanA_lo = 0, spanA_hi = 0, spanB_lo = 0, spanB_hi = 0, spanD_lo = 0, spanD_hi = 0;
+    struct HostPipeline *host = nullptr;   // built by the first btc_execute_host
+};
+
+// Host-buffer execution in slabs (btc_execute_host): the larger input is cut along the label with its largest
+// stride, slab i + 1 is copied to the device while slab i is contracted.
+struct HostPipeline {
+    bool tried = false, usable = false;
+    bool slab_is_A = true;                 // which caller-side input is cut
+    int64_t extent = 0, slab = 0;          // extent of the cut label, slab length
+    int idxX = -1, idxY = -1, idxD = -1;   // position of the label in the cut input, the other input, D (-1: absent)
+    int64_t strideX = 0, strideY = 0, strideD = 0;
+    btc_contraction_s *sub[2] = {nullptr, nullptr};   // operation for a full slab / for the remainder
+    int64_t sub_lo[2] = {0, 0}, sub_hi[2] = {0, 0};   // span of a slab of the cut input (elements, relative to its first element)
+    char *bufX[2] = {nullptr, nullptr}, *bufY = nullptr, *bufD = nullptr, *bufC = nullptr, *ws = nullptr;
+    size_t bytesX = 0, bytesY = 0, bytesD = 0, bytesC = 0, bytesW = 0;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t loaded[2] = {nullptr, nullptr}, consumed[2] = {nullptr, nullptr};
 };
 
 struct btc_elementwise_s {
@@ -89,6 +106,8 @@ struct btc_elementwise_s {
 };
 
 namespace {
+
+void free_host_pipeline(btc_contraction_s *op);
 
 // ---- tiled kernel variants -------------------------------------------------------------------
 using F64Big = F64Tile<false, 128, 128, 2, 4, 4, 1>;
@@ -783,6 +802,7 @@ btc_error_t btc_destroy_contraction(btc_contraction_t *op)
 {
     if (!op) return BTC_ERR_INVALID_ARGUMENT;
     if (*op) {
+        free_host_pipeline(*op);
         free_tables(*op);
         delete *op;
     }
@@ -839,6 +859,7 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
     } else {
         return BTC_ERR_INVALID_ARGUMENT;
     }
+    free_host_pipeline(op);    // built for the previous plan
     int rc = replan(op);
     if (rc != BTC_SUCCESS) {   // keep the object usable with its previous plan
         op->req = saved;
@@ -1239,6 +1260,195 @@ btc_error_t btc_execute_batched(btc_contraction_t op, void *cuda_stream, const v
                         nullptr, &bv);
 }
 
+}  // extern "C"
+
+namespace {
+
+void free_host_pipeline(btc_contraction_s *op)
+{
+    HostPipeline *hp = op->host;
+    if (!hp) return;
+    for (int i = 0; i < 2; ++i) {
+        if (hp->sub[i]) { free_tables(hp->sub[i]); delete hp->sub[i]; }
+        if (hp->bufX[i]) cudaFree(hp->bufX[i]);
+        if (hp->loaded[i]) cudaEventDestroy(hp->loaded[i]);
+        if (hp->consumed[i]) cudaEventDestroy(hp->consumed[i]);
+    }
+    for (char *b : {hp->bufY, hp->bufD, hp->bufC, hp->ws}) if (b) cudaFree(b);
+    if (hp->copy_stream) cudaStreamDestroy(hp->copy_stream);
+    cudaGetLastError();
+    delete hp;
+    op->host = nullptr;
+}
+
+int position_of(const std::vector<int64_t> &labels, int64_t label)
+{
+    int at = -1;
+    for (size_t i = 0; i < labels.size(); ++i)
+        if (labels[i] == label) { if (at >= 0) return -2; at = int(i); }       // -2: repeated
+    return at;
+}
+
+void span_of_desc(const TensorDesc &t, int64_t &lo, int64_t &hi)
+{
+    lo = hi = 0;
+    for (size_t i = 0; i < t.extent.size(); ++i) {
+        const int64_t d = t.stride[i] * (t.extent[i] - 1);
+        if (d < 0) lo += d; else hi += d;
+    }
+}
+
+// Decide how to cut the operation for host-buffer execution and build what that needs.  Not usable (the
+// plain path runs) when no label qualifies or the slabs would overlap too much in memory.
+void build_host_pipeline(btc_contraction_s *op)
+{
+    HostPipeline *hp = new (std::nothrow) HostPipeline;
+    op->host = hp;
+    if (!hp) return;
+    hp->tried = true;
+    const PlanRequest &rq = op->req;
+    const size_t esz = dtype_size(rq.D.dtype);
+    const int64_t spanA = op->spanA_hi - op->spanA_lo + 1, spanB = op->spanB_hi - op->spanB_lo + 1;
+    hp->slab_is_A = spanA >= spanB;
+    const TensorDesc &X = hp->slab_is_A ? rq.A : rq.B, &Y = hp->slab_is_A ? rq.B : rq.A;
+    const std::vector<int64_t> &lX = hp->slab_is_A ? rq.labelsA : rq.labelsB, &lY = hp->slab_is_A ? rq.labelsB : rq.labelsA;
+    if (size_t(std::max(spanA, spanB)) * esz < (size_t(64) << 20)) return;       // small inputs: one copy is as good
+    // the label with the largest stride in the cut input that occurs once there and at most once elsewhere
+    int best = -1;
+    for (size_t i = 0; i < lX.size(); ++i) {
+        if (position_of(lX, lX[i]) != int(i) || X.extent[i] < 4 || X.stride[i] <= 0) continue;
+        const int inY = position_of(lY, lX[i]), inD = position_of(rq.labelsD, lX[i]);
+        if (inY == -2 || inD == -2) continue;
+        if (inY < 0 && inD < 0) continue;                      // a label only in this input (Case 4): leave it whole
+        if (best < 0 || X.stride[i] > X.stride[size_t(best)]) best = int(i);
+    }
+    if (best < 0) return;
+    hp->idxX = best;
+    hp->idxY = position_of(lY, lX[size_t(best)]);
+    hp->idxD = position_of(rq.labelsD, lX[size_t(best)]);
+    hp->extent = X.extent[size_t(best)];
+    hp->strideX = X.stride[size_t(best)];
+    hp->strideY = hp->idxY >= 0 ? Y.stride[size_t(hp->idxY)] : 0;
+    hp->strideD = hp->idxD >= 0 ? rq.D.stride[size_t(hp->idxD)] : 0;
+    // about eight slabs, none below 32 MiB
+    int64_t slabs = 8;
+    while (slabs > 2 && size_t(std::max(spanA, spanB)) * esz / size_t(slabs) < (size_t(32) << 20)) --slabs;
+    hp->slab = (hp->extent + slabs - 1) / slabs;
+    if (hp->slab < 1 || hp->slab >= hp->extent) return;
+    const int64_t lengths[2] = {hp->slab, hp->extent % hp->slab};
+    for (int i = 0; i < 2; ++i) {
+        if (lengths[i] == 0) continue;
+        btc_contraction_s *sub = new (std::nothrow) btc_contraction_s;
+        if (!sub) return;
+        hp->sub[i] = sub;
+        sub->handle = op->handle;
+        sub->req = rq;
+        sub->pre_reduce = op->pre_reduce;
+        sub->poll_limit = op->poll_limit;
+        TensorDesc &sX = hp->slab_is_A ? sub->req.A : sub->req.B, &sY = hp->slab_is_A ? sub->req.B : sub->req.A;
+        sX.extent[size_t(hp->idxX)] = lengths[i];
+        if (hp->idxY >= 0) sY.extent[size_t(hp->idxY)] = lengths[i];
+        if (hp->idxD >= 0) sub->req.D.extent[size_t(hp->idxD)] = lengths[i];
+        // a contracted label: later slabs accumulate into D, which needs C's description (= D's)
+        sub->req.has_c = true;
+        sub->req.C = sub->req.D;
+        sub->req.labelsC = sub->req.labelsD;
+        sub->req.conjC = rq.has_c ? rq.conjC : false;
+        sub->alpha[0] = op->alpha[0]; sub->alpha[1] = op->alpha[1];
+        sub->beta[0] = op->beta[0]; sub->beta[1] = op->beta[1];
+        if (replan(sub) != BTC_SUCCESS) return;
+        span_of_desc(sX, hp->sub_lo[i], hp->sub_hi[i]);
+        hp->bytesW = std::max(hp->bytesW, sub->workspace_bytes);
+    }
+    // slabs of the cut input must not overlap much in memory, or the copies would repeat most of it
+    const int64_t slab_span = hp->sub_hi[0] - hp->sub_lo[0] + 1;
+    if (double(slab_span) * double((hp->extent + hp->slab - 1) / hp->slab) > 1.25 * double(hp->slab_is_A ? spanA : spanB)) return;
+    hp->bytesX = size_t(slab_span) * esz;
+    hp->bytesY = size_t(hp->slab_is_A ? spanB : spanA) * esz;
+    hp->bytesD = size_t(op->spanD_hi - op->spanD_lo + 1) * esz;
+    hp->bytesC = hp->bytesD;
+    bool ok = cudaStreamCreateWithFlags(&hp->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i) {
+        ok = cudaEventCreateWithFlags(&hp->loaded[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&hp->consumed[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaMalloc(reinterpret_cast<void **>(&hp->bufX[i]), hp->bytesX) == cudaSuccess;
+    }
+    ok = ok && cudaMalloc(reinterpret_cast<void **>(&hp->bufY), hp->bytesY) == cudaSuccess &&
+         cudaMalloc(reinterpret_cast<void **>(&hp->bufD), hp->bytesD) == cudaSuccess &&
+         (hp->bytesW == 0 || cudaMalloc(reinterpret_cast<void **>(&hp->ws), hp->bytesW) == cudaSuccess);
+    if (!ok) { cudaGetLastError(); return; }
+    hp->usable = true;
+}
+
+// The slabbed run.  X = the cut input, Y = the other one.
+btc_error_t run_host_pipeline(btc_contraction_s *op, cudaStream_t st, const void *alpha, const void *A, const void *B,
+                              const void *beta, const void *C, void *D, bool use_c)
+{
+    HostPipeline *hp = op->host;
+    const size_t esz = dtype_size(op->plan.dtype);
+    const bool c_is_d = use_c && C == D;
+    if (use_c && !c_is_d && !hp->bufC && cudaMalloc(reinterpret_cast<void **>(&hp->bufC), hp->bytesC) != cudaSuccess) {
+        cudaGetLastError();
+        return BTC_ERR_OUT_OF_MEMORY;
+    }
+    const char *hX = static_cast<const char *>(hp->slab_is_A ? A : B), *hY = static_cast<const char *>(hp->slab_is_A ? B : A);
+    const int64_t loY = (hp->slab_is_A ? op->spanB_lo : op->spanA_lo) * int64_t(esz), loD = op->spanD_lo * int64_t(esz);
+    bool ok = true;
+    auto copy = [&](void *dst, const void *src, size_t n, cudaMemcpyKind kind, cudaStream_t on) {
+        ok = ok && cudaMemcpyAsync(dst, src, n, kind, on) == cudaSuccess;
+    };
+    // the whole of the smaller input, of D's span (padding between its elements must survive the round trip) and of C
+    copy(hp->bufY, hY + loY, hp->bytesY, cudaMemcpyHostToDevice, st);
+    copy(hp->bufD, static_cast<const char *>(D) + loD, hp->bytesD, cudaMemcpyHostToDevice, st);
+    if (use_c && !c_is_d) copy(hp->bufC, static_cast<const char *>(C) + loD, hp->bytesC, cudaMemcpyHostToDevice, st);
+    const char *dY = hp->bufY - loY;
+    char *dD = hp->bufD - loD;
+    const char *dC = use_c ? (c_is_d ? dD : hp->bufC - loD) : nullptr;
+    const bool accumulate = hp->idxD < 0;          // a contracted label: slabs add up in D
+    const double one[2] = {1.0, 0.0};
+    float one_f[2] = {1.f, 0.f};
+    const void *beta_one = (op->plan.dtype == BTC_F32 || op->plan.dtype == BTC_C32) ? static_cast<const void *>(one_f) : static_cast<const void *>(one);
+    const int64_t count = (hp->extent + hp->slab - 1) / hp->slab;
+    // copies run on a stream of their own, one slab ahead of the contraction
+    cudaEvent_t start = hp->consumed[0];           // reused below only after its first wait
+    ok = ok && cudaEventRecord(start, st) == cudaSuccess && cudaStreamWaitEvent(hp->copy_stream, start, 0) == cudaSuccess;
+    btc_error_t rc = BTC_SUCCESS;
+    for (int64_t i = 0; i < count && ok && rc == BTC_SUCCESS; ++i) {
+        const int b = int(i & 1), which = (i + 1 == count && hp->extent % hp->slab) ? 1 : 0;
+        const int64_t first = i * hp->slab;
+        const int64_t loX = hp->sub_lo[which] * int64_t(esz);
+        const size_t bytes = size_t(hp->sub_hi[which] - hp->sub_lo[which] + 1) * esz;
+        if (i >= 2) ok = ok && cudaStreamWaitEvent(hp->copy_stream, hp->consumed[b], 0) == cudaSuccess;
+        copy(hp->bufX[b], hX + first * hp->strideX * int64_t(esz) + loX, bytes, cudaMemcpyHostToDevice, hp->copy_stream);
+        ok = ok && cudaEventRecord(hp->loaded[b], hp->copy_stream) == cudaSuccess && cudaStreamWaitEvent(st, hp->loaded[b], 0) == cudaSuccess;
+        if (!ok) break;
+        const char *pX = hp->bufX[b] - loX;
+        const char *pY = dY + first * hp->strideY * int64_t(esz);
+        char *pD = dD + first * hp->strideD * int64_t(esz);
+        const char *pC = dC ? dC + first * hp->strideD * int64_t(esz) : nullptr;
+        const void *b_ptr = beta, *c_ptr = pC;
+        if (accumulate && i > 0) { b_ptr = beta_one; c_ptr = pD; }     // D += alpha * this slab
+        rc = btc_execute(hp->sub[which], st, alpha, hp->slab_is_A ? pX : pY, hp->slab_is_A ? pY : pX, b_ptr, c_ptr, pD,
+                         hp->ws, hp->bytesW, nullptr);
+        ok = ok && cudaEventRecord(hp->consumed[b], st) == cudaSuccess;
+    }
+    copy(static_cast<char *>(D) + loD, hp->bufD, hp->bytesD, cudaMemcpyDeviceToHost, st);
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaStreamSynchronize(hp->copy_stream) != cudaSuccess) ok = false;
+    if (!ok) { cudaGetLastError(); return rc != BTC_SUCCESS ? rc : BTC_ERR_CUDA; }
+    if (rc != BTC_SUCCESS) return rc;
+    for (int i = 0; i < 2; ++i)
+        if (hp->sub[i] && hp->sub[i]->d_error) {
+            int32_t word = 0;
+            if (cudaMemcpy(&word, hp->sub[i]->d_error, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return BTC_ERR_CUDA; }
+            if (word != 0) return BTC_ERR_DEVICE_TIMEOUT;
+        }
+    return BTC_SUCCESS;
+}
+
+}  // namespace
+
+extern "C" {
+
 btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void *alpha, const void *A,
                              const void *B, const void *beta, const void *C, void *D)
 {
@@ -1252,6 +1462,12 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
     const bool use_ab = !is_zero(al), use_c = !is_zero(be);
     if ((use_ab && (!A || !B)) || (use_c && !C)) return BTC_ERR_INVALID_ARGUMENT;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+    // large inputs: cut the larger one into slabs and copy slab i + 1 while slab i is contracted
+    if (use_ab && op->poll_limit == kWaitPollLimit) {
+        if (!op->host) build_host_pipeline(op);
+        if (op->host && op->host->usable) return run_host_pipeline(op, st, alpha, A, B, beta, C, D, use_c);
+    }
 
     struct Buf {
         char *dev = nullptr;

@@ -22,6 +22,8 @@ CASES = {
     "cfg4_c64_conj": (20000, 256 * 256),
     "cfg6_f64_case4_isolated": (6000, 64 * 64),       # Case 4: A summed over its isolated label first
     "cfg6b_f64_case4_isolated_fast": (6000, 32 * 32),
+    "cfg4c_c32_conj": (20000, 256 * 256),                 # complex64
+    "cfg7_f32_outer_product": (200000, 128 * 128),        # no contracted label: the streaming kernel
 }
 
 
@@ -78,6 +80,59 @@ def test_full_size_sampled(name):
         after = D.buffer.view(width).reshape(D.buffer.numel(), -1)[~touched]
         assert torch.equal(before, after)
         assert not torch.isnan(torch.view_as_real(D.buffer[touched]) if D.buffer.is_complex() else D.buffer[touched]).any()
+
+
+def _sampled_check(w, hA, hB, hC, D_layout, result_buffer, origin, n_random, slab, dtype):
+    """Oracle at sampled elements of D against `result_buffer` (a flat tensor holding D's span)."""
+    extents, strides = D_layout
+    total = int(np.prod(extents))
+    rng = np.random.default_rng(2025)
+    want = np.unique(np.concatenate([rng.integers(0, total, size=n_random), np.arange(min(slab, total))]))
+    d_stub = np.zeros(1, dtype=hA.numpy().dtype)
+    vals, scale = oracle.contract(hA.numpy(), w.labelsA, hB.numpy(), w.labelsB,
+                                  hC.numpy() if hC is not None else None, w.labelsD, d_stub, w.labelsD,
+                                  w.alpha, w.beta, conjA=w.conjA, conjB=w.conjB, conjC=w.conjC, want=want,
+                                  layouts={"D": (extents, strides)})
+    pos = np.full(want.shape, origin, dtype=np.int64)
+    rem = want.copy()
+    for e, st in zip(extents, strides):
+        pos += (rem % e) * st
+        rem //= e
+    got = result_buffer[torch.from_numpy(pos)].numpy()
+    return helpers.compare(got, vals, scale, dtype)
+
+
+@pytest.mark.parametrize("name", ["cfg2p_f64_ccsd_ladder_profile", "cfg3p_f32_batched_permuted_profile", "cfg4_c64_conj"])
+def test_full_size_host_buffers_in_slabs(name):
+    """btc_execute_host on inputs large enough to be cut into slabs (copies overlapped with the contraction):
+    a contracted label whose slabs accumulate into D in place (the ladder term), a batch label with a padded
+    output, and a free label.  Sampled elements against the oracle; bytes between D's elements keep their
+    canaries; a second call on the same operation object gives the same bits."""
+    api = helpers.api()
+    handle = api.Handle()
+    w = inputs.workloads()[name]
+    A, B, C, D = inputs.make_workload_tensors(w, device="cuda")
+    hA, hB, hD = A.to("cpu"), B.to("cpu"), D.to("cpu")
+    hC0 = C.to("cpu") if C is not None else None             # C before the in-place update
+    del A, B, C, D
+    dt = api.dtype_code(hD.dtype)
+    tA = api.TensorInfo(handle, dt, hA.extents, hA.strides)
+    tB = api.TensorInfo(handle, dt, hB.extents, hB.strides)
+    tD = api.TensorInfo(handle, dt, hD.extents, hD.strides)
+    op = api.Contraction(handle, tA, w.labelsA, tB, w.labelsB, tD if hC0 is not None else None, w.labelsD,
+                         tD, w.labelsD, w.alpha, w.beta, w.conjA, w.conjB, w.conjC)
+    results = []
+    for _ in range(2):
+        out = hD.clone()
+        c_ptr = 0 if hC0 is None else (out.data_ptr() if w.in_place else hC0.data_ptr())
+        op.execute_host(torch.cuda.current_stream().cuda_stream, hA.data_ptr(), hB.data_ptr(), c_ptr, out.data_ptr())
+        results.append(out)
+    assert torch.equal(results[0].buffer.view(torch.uint8), results[1].buffer.view(torch.uint8))
+    out = results[0]
+    worst = _sampled_check(w, hA, hB, hC0, (hD.extents, hD.strides), out.buffer, hD.origin, 4000, 4096, hD.dtype)
+    assert worst <= 1.0, worst
+    if not w.in_place:
+        assert helpers.canary_intact(hD.buffer, out.buffer, hD.offsets())
 
 
 @pytest.mark.parametrize("name", list(inputs.elementwise_workloads()))
