@@ -192,6 +192,55 @@ def contract(A: np.ndarray, labelsA, B: np.ndarray, labelsB,
     return scale
 
 
+def contract_mixed(A: np.ndarray, labelsA, B: np.ndarray, labelsB,
+                   C: Optional[np.ndarray], labelsC, D: np.ndarray, labelsD,
+                   alpha=1.0, beta=0.0, *, conjA=False, conjB=False, conjC=False,
+                   want: Optional[Sequence[int]] = None, layouts: Optional[dict] = None):
+    """The contraction with an element type per tensor (float32 / float64 / complex64 / complex128 in any
+    mix whose result type can hold the result: D must be complex when an input is).  Same calling
+    conventions and return values as ``contract`` (scale always returned)."""
+    lib = _load()
+    for t in (A, B, C, D):
+        if t is not None and np.dtype(t.dtype) not in _DTYPE_CODE:
+            raise OracleError(ERR_NOT_SUPPORTED)
+    layouts = layouts or {}
+    keep: list = []
+    tA = _describe(A, labelsA, conjA, keep, *layouts.get("A", (None, None)))
+    tB = _describe(B, labelsB, conjB, keep, *layouts.get("B", (None, None)))
+    tC = _describe(C, labelsC, conjC, keep, *layouts.get("C", (None, None)))
+    tD = _describe(D, labelsD, False, keep, *layouts.get("D", (None, None)))
+    al = np.array([complex(alpha).real, complex(alpha).imag], dtype=np.float64)
+    be = np.array([complex(beta).real, complex(beta).imag], dtype=np.float64)
+    n_eval = 1
+    for e in (layouts["D"][0] if "D" in layouts else D.shape):
+        n_eval *= int(e)
+    want_arr = out_val = None
+    if want is not None:
+        want_arr = np.ascontiguousarray(np.asarray(want, dtype=np.int64)).reshape(-1)
+        n_eval = want_arr.size
+        if n_eval == 0:
+            want_arr = np.zeros(1, dtype=np.int64)
+        out_val = np.empty(max(n_eval, 1), dtype=D.dtype)[:n_eval]
+    scale = np.empty(max(n_eval, 1), dtype=np.float64)[:n_eval]
+    code = lambda t: _DTYPE_CODE[np.dtype(t.dtype)] if t is not None else _DTYPE_CODE[np.dtype(D.dtype)]
+    lib.orc_contract_mixed.restype = ctypes.c_int
+    lib.orc_contract_mixed.argtypes = [ctypes.c_int] * 4 + [ctypes.POINTER(_Tensor)] * 4 + [
+        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    rc = lib.orc_contract_mixed(
+        code(A), code(B), code(C), code(D),
+        ctypes.byref(tA) if tA is not None else None, ctypes.byref(tB) if tB is not None else None,
+        ctypes.byref(tC) if tC is not None else None, ctypes.byref(tD),
+        al.ctypes.data, be.ctypes.data,
+        n_eval if want_arr is not None else 0,
+        want_arr.ctypes.data if want_arr is not None else None,
+        out_val.ctypes.data if out_val is not None else None, scale.ctypes.data)
+    if rc != OK:
+        raise OracleError(rc)
+    if want_arr is not None:
+        return out_val, scale
+    return scale
+
+
 _lib_ew = None
 
 

@@ -325,6 +325,117 @@ int orc_contract(int dtype, const orc_tensor *A, const orc_tensor *B, const orc_
     return ORC_OK;
 }
 
+/*
+ * Mixed element types (Sec. "Challenge: Datatypes": the reference implementation lets every tensor
+ * have its own type).  Same definition, same loop order; every operand is read through its own type
+ * (a real element is the complex number with zero imaginary part), products and sums are formed in
+ * long double, and the result is rounded once to D's type.  D must be complex when any of A, B, C is;
+ * alpha and beta are given as two doubles each (re, im; the imaginary part must be 0 when D is real).
+ * Written as one plain function with a reader per element instead of one loop nest per type
+ * combination: slower, easier to check.
+ */
+static void orc_read(int dtype, const void *base, int64_t off, long double *re, long double *im)
+{
+    switch (dtype) {
+    case ORC_F32: *re = ((const float *)base)[off]; *im = 0; break;
+    case ORC_F64: *re = ((const double *)base)[off]; *im = 0; break;
+    case ORC_C32: *re = ((const float *)base)[2 * off]; *im = ((const float *)base)[2 * off + 1]; break;
+    default: *re = ((const double *)base)[2 * off]; *im = ((const double *)base)[2 * off + 1]; break;
+    }
+}
+
+static void orc_write(int dtype, void *base, int64_t off, long double re, long double im)
+{
+    switch (dtype) {
+    case ORC_F32: ((float *)base)[off] = (float)re; break;
+    case ORC_F64: ((double *)base)[off] = (double)re; break;
+    case ORC_C32: ((float *)base)[2 * off] = (float)re; ((float *)base)[2 * off + 1] = (float)im; break;
+    default: ((double *)base)[2 * off] = (double)re; ((double *)base)[2 * off + 1] = (double)im; break;
+    }
+}
+
+static int orc_is_complex(int dtype) { return dtype == ORC_C32 || dtype == ORC_C64; }
+
+int orc_contract_mixed(int dtypeA, int dtypeB, int dtypeC, int dtypeD, const orc_tensor *A, const orc_tensor *B,
+                       const orc_tensor *C, const orc_tensor *D, const double *alpha, const double *beta,
+                       int64_t n_want, const int64_t *want, void *out_val, double *out_scale)
+{
+    orc_loops L;
+    if (!alpha || !beta || !D) return ORC_ERR_INVALID_ARGUMENT;
+    if (want && !out_val) return ORC_ERR_INVALID_ARGUMENT;
+    const int types[4] = {dtypeA, dtypeB, dtypeC, dtypeD};
+    for (int i = 0; i < 4; ++i)
+        if (types[i] < ORC_F32 || types[i] > ORC_C64) return ORC_ERR_NOT_SUPPORTED;
+    const int c_is_used = beta[0] != 0 || beta[1] != 0;
+    if (!orc_is_complex(dtypeD)) {
+        if (orc_is_complex(dtypeA) || orc_is_complex(dtypeB) || (c_is_used && orc_is_complex(dtypeC))) return ORC_ERR_NOT_SUPPORTED;
+        if (alpha[1] != 0 || beta[1] != 0) return ORC_ERR_NOT_SUPPORTED;
+    }
+    int rc = orc_prepare(A, B, C, D, c_is_used, &L);
+    if (rc != ORC_OK) return rc;
+    if (want)
+        for (int64_t e = 0; e < n_want; ++e)
+            if (want[e] < 0 || want[e] >= L.sizeD) return ORC_ERR_INVALID_ARGUMENT;
+    if (!c_is_used) C = NULL;
+    const long double al_r = alpha[0], al_i = alpha[1], be_r = beta[0], be_i = beta[1];
+    const int use_ab = (al_r != 0 || al_i != 0);
+    const long double abs_al = sqrtl(al_r * al_r + al_i * al_i), abs_be = sqrtl(be_r * be_r + be_i * be_i);
+    const long double sgnA = A->conj ? -1 : 1, sgnB = B->conj ? -1 : 1, sgnC = (C && C->conj) ? -1 : 1;
+    const int64_t total = want ? n_want : L.sizeD;
+    const int out_type = dtypeD;
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < total; ++e) {
+        int64_t lin = want ? want[e] : e;
+        int64_t offA = 0, offB = 0, offD = 0;
+        for (int k = 0; k < L.nD; ++k) { /* first label of D fastest */
+            int64_t i = lin % L.d[k].extent;
+            lin /= L.d[k].extent;
+            offA += i * L.d[k].sA;
+            offB += i * L.d[k].sB;
+            offD += i * L.d[k].sD;
+        }
+        long double acc_r = 0, acc_i = 0, absacc = 0;
+        if (use_ab) {
+            int64_t idx[ORC_MAX_LABELS];
+            int64_t oa = offA, ob = offB;
+            for (int k = 0; k < L.nS; ++k) idx[k] = 0;
+            for (int64_t s = 0; s < L.sizeS; ++s) {
+                long double ar, ai, br, bi;
+                orc_read(dtypeA, A->data, oa, &ar, &ai);
+                orc_read(dtypeB, B->data, ob, &br, &bi);
+                ai *= sgnA;
+                bi *= sgnB;
+                acc_r += ar * br - ai * bi;
+                acc_i += ar * bi + ai * br;
+                absacc += sqrtl(ar * ar + ai * ai) * sqrtl(br * br + bi * bi);
+                for (int k = 0; k < L.nS; ++k) { /* odometer over the summed labels, first fastest */
+                    oa += L.s[k].sA;
+                    ob += L.s[k].sB;
+                    if (++idx[k] < L.s[k].extent) break;
+                    oa -= idx[k] * L.s[k].sA;
+                    ob -= idx[k] * L.s[k].sB;
+                    idx[k] = 0;
+                }
+            }
+        }
+        long double d_r = al_r * acc_r - al_i * acc_i;
+        long double d_i = al_r * acc_i + al_i * acc_r;
+        long double sc = abs_al * absacc;
+        if (C) {
+            long double cr, ci;
+            orc_read(dtypeC, C->data, offD, &cr, &ci);
+            ci *= sgnC;
+            d_r += be_r * cr - be_i * ci;
+            d_i += be_r * ci + be_i * cr;
+            sc += abs_be * sqrtl(cr * cr + ci * ci);
+        }
+        if (want) orc_write(out_type, out_val, e, d_r, d_i);
+        else orc_write(out_type, D->data, offD, d_r, d_i);
+        if (out_scale) out_scale[e] = (double)sc;
+    }
+    return ORC_OK;
+}
+
 /* Width of the wide accumulator's significand, so a test can see what "wide" meant here. */
 int orc_long_double_mant_dig(void) { return __LDBL_MANT_DIG__; }
 

@@ -517,3 +517,104 @@ def test_workload_symmetry_and_sizes():
     assert np.array_equal(V, V.transpose(1, 0, 3, 2)) and C is D
     s3 = inputs.scaled_down(W["cfg3_f32_batched_permuted"], {"z": 2, "a": 5, "b": 6, "j": 7, "k": 3, "l": 2})
     assert s3.stridesD == (1, 15, 90, 180)
+
+
+# ---------------------------------------------------------------- mixed element types
+def run_mixed(A, la, B, lb, C, ld, dtypeD, alpha=1.0, beta=0.0, **kw):
+    ext = {}
+    for t, l in ((A, la), (B, lb)):
+        for e, ch in zip(t.shape, l):
+            ext[ch] = e
+    D = np.full([ext[ch] for ch in ld], np.nan, dtype=dtypeD, order="F")
+    scale = oracle.contract_mixed(A, la, B, lb, C, ld, D, ld, alpha, beta, **kw)
+    return D, scale
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_mixed_entry_point_with_one_type_equals_the_plain_oracle(dtype):
+    """The mixed-type loop nest must be the same function when every tensor has the same type: identical
+    bits for the 64-bit types (both accumulate in long double, in the same order), one rounding apart
+    for the 32-bit types (double against long double accumulators)."""
+    rng = np.random.default_rng(71)
+    A, B, C = rnd(rng, (5, 6, 3), dtype), rnd(rng, (3, 6, 4), dtype), rnd(rng, (4, 5), dtype)
+    cplx = np.issubdtype(dtype, np.complexfloating)
+    alpha, beta = (0.5 - 0.25j, 1.5 + 2j) if cplx else (0.5, 1.5)
+    want, scale = run(A, "ikl", B, "lkj", C, "ji", alpha, beta, conjA=cplx, conjC=cplx)
+    got, scale2 = run_mixed(A, "ikl", B, "lkj", C, "ji", dtype, alpha, beta, conjA=cplx, conjC=cplx)
+    if dtype in (np.float64, np.complex128):
+        assert np.array_equal(got, want)
+    else:
+        assert np.all(np.abs(got.astype(np.complex128) - want.astype(np.complex128)) <= 2.0 ** -22 * np.abs(want))
+    assert np.allclose(scale, scale2, rtol=1e-6)
+
+
+@pytest.mark.parametrize("real,cplx", [(np.float64, np.complex128), (np.float32, np.complex64)])
+@pytest.mark.parametrize("which", ["A", "B", "C", "AB"])
+def test_real_operand_among_complex_ones_equals_its_promoted_copy(real, cplx, which):
+    """A real tensor is the complex tensor with zero imaginary parts: mixing it in must give what the
+    plain oracle gives on the explicitly promoted copy (bit-identical in 64-bit; conj of a real operand
+    is a no-op)."""
+    rng = np.random.default_rng(72)
+    tA = real if "A" in which else cplx
+    tB = real if "B" in which else cplx
+    tC = real if "C" in which else cplx
+    A, B, C = rnd(rng, (4, 7), tA), rnd(rng, (7, 5), tB), rnd(rng, (4, 5), tC)
+    alpha, beta = 0.75 - 0.5j, -0.25 + 1.0j
+    got, scale = run_mixed(A, "ik", B, "kj", C, "ij", cplx, alpha, beta, conjA=True, conjB=True, conjC=True)
+    want, _ = run(A.astype(cplx), "ik", B.astype(cplx), "kj", C.astype(cplx), "ij", alpha, beta, conjA=True, conjB=True, conjC=True)
+    if cplx is np.complex128:
+        assert np.array_equal(got, want)
+    else:
+        assert close(got, want, scale, cplx, factor=0.1)
+
+
+def test_mixed_types_against_explicit_loops_and_einsum():
+    """Hand loops in Python complex arithmetic on a tiny case with three different element types, and numpy
+    einsum on promoted copies, pin products, conjugation and the alpha / beta step of the mixed loop nest."""
+    rng = np.random.default_rng(73)
+    A = rnd(rng, (3, 2, 4), np.float32)                  # A[i,k,l] real, 32-bit
+    B = rnd(rng, (4, 2, 3), np.complex64)                # B[l,k,j]
+    C = rnd(rng, (3, 3), np.float64)                     # C[j,i] real, 64-bit
+    alpha, beta = 1.25 + 0.5j, 0.5 - 1.5j
+    got, scale = run_mixed(A, "ikl", B, "lkj", C, "ji", np.complex128, alpha, beta, conjB=True)
+    want = np.zeros((3, 3), dtype=np.complex128)
+    for j in range(3):
+        for i in range(3):
+            acc = 0j
+            for k in range(2):
+                for l in range(4):
+                    acc += complex(A[i, k, l]) * complex(B[l, k, j]).conjugate()
+            want[j, i] = alpha * acc + beta * complex(C[j, i])
+    assert np.allclose(got, want, rtol=1e-13, atol=1e-13)
+    ein = alpha * np.einsum("ikl,lkj->ji", A.astype(np.complex128), np.conj(B).astype(np.complex128)) + beta * C
+    assert np.allclose(got, ein, rtol=1e-13, atol=1e-13)
+    # scale = |alpha| sum |a||b| + |beta||c|
+    s = abs(alpha) * np.einsum("ikl,lkj->ji", np.abs(A).astype(np.float64), np.abs(B).astype(np.float64)) + abs(beta) * np.abs(C)
+    assert np.allclose(scale.reshape(3, 3, order="F"), s, rtol=1e-6)
+
+
+def test_float32_storage_is_accumulated_wider_than_float32():
+    """fp32 tensors through the mixed entry point: the sum is formed wider than fp32 and rounded once, so on
+    a long ill-conditioned sum it is far closer to the exact value than fp32 accumulation is."""
+    n = 20000
+    a = np.asarray(np.full((1, n), 1.0), dtype=np.float32, order="F")
+    b = np.asarray(np.full((n, 1), 1e-4), dtype=np.float32, order="F")
+    b[0, 0] = 1e4                                         # large first term swallows small ones in fp32
+    got, _ = run_mixed(a, "ik", b, "kj", None, "ij", np.float32)
+    exact = float(np.sum(b.astype(np.float64)))
+    assert abs(float(got[0, 0]) - exact) <= 2.0 ** -23 * exact
+    naive = np.float32(0)
+    for x in b[:, 0]:
+        naive = np.float32(naive + x)
+    assert abs(float(naive) - exact) > 100 * abs(float(got[0, 0]) - exact)
+
+
+def test_mixed_types_reject_a_real_result_of_complex_inputs():
+    rng = np.random.default_rng(74)
+    A, B = rnd(rng, (3, 4), np.complex128), rnd(rng, (4, 2), np.float64)
+    D = np.zeros((3, 2), dtype=np.float64, order="F")
+    with pytest.raises(oracle.OracleError) as ei:
+        oracle.contract_mixed(A, "ik", B, "kj", None, "ij", D, "ij")
+    assert ei.value.code == oracle.ERR_NOT_SUPPORTED
+    with pytest.raises(oracle.OracleError):                # a complex alpha cannot scale a real result
+        oracle.contract_mixed(B, "ik", B.T.copy(order="F"), "kj", None, "ij", np.zeros((4, 4), order="F"), "ij", alpha=1j)
