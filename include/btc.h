@@ -92,6 +92,10 @@ btc_error_t btc_destroy_tensor_info(btc_tensor_info_t *info);
  *   conjX       non-zero: op(X) = element-wise complex conjugate; ignored for real types
  *   alpha,beta  host scalars of D's element type stored as the defaults of the operation;
  *               NULL means alpha = 1, beta = 0
+ * Element types (Sec. "Challenge: Datatypes"): normally all four tensors share one type.  Real and
+ * complex tensors of one part width may be mixed (a real operand counts as complex with zero
+ * imaginary parts) as long as D is complex whenever A, B or C is; such operations run on the
+ * per-element kernel (exact, not fast).  32- and 64-bit parts cannot be mixed (NOT_SUPPORTED).
  * All validation and planning (label classes, mode fusion, kernel and tile choice, device-side
  * offset tables) happens here; the call may allocate device memory and copy small tables with
  * the default stream.  Errors: INVALID_ARGUMENT, EXTENT_MISMATCH, C_D_MISMATCH, D_ALIASING,
@@ -140,8 +144,10 @@ enum {
                                  precision an operation may ask for (Sec. "Tensor Operation Descriptors").  DEFAULT:
                                  fp32 products are formed from three TF32 tensor-core products (error of a
                                  product <= 2^-22 |a||b|, fp32 accumulation); STRICT: fp32 operations run on
-                                 the FMA pipe in IEEE fp32 (about a third of the speed).  No effect on fp64
-                                 and complex128 (always IEEE fp64); STRICT is NOT_SUPPORTED for complex64 */
+                                 the FMA pipe in IEEE fp32 (about a third of the speed); FP64_SUMS: fp32 /
+                                 complex64 storage, products and sums kept in fp64 and rounded once to the
+                                 element type (runs the per-element kernel: exact but slow).  No effect on
+                                 fp64 and complex128 (always IEEE fp64); STRICT is NOT_SUPPORTED for complex64 */
     BTC_ATTR_BATCH_HINT = 11, /* int32 >= 1, read/write (write re-plans): how many pointer-array entries
                                  btc_execute_batched will usually be given.  Tile variant and split-K
                                  are then chosen for that many entries in flight (no split-K when the
@@ -153,7 +159,7 @@ enum {
                                  labels are summed inside the generic kernel.  Read: bit 0 / bit 1
                                  set when A / B is summed first in the current plan             */
 };
-enum { BTC_PRECISION_DEFAULT = 0, BTC_PRECISION_STRICT = 1 };
+enum { BTC_PRECISION_DEFAULT = 0, BTC_PRECISION_STRICT = 1, BTC_PRECISION_FP64_SUMS = 2 };
 enum {
     BTC_KERNEL_AUTO = 0,
     BTC_KERNEL_GENERIC = 1,   /* one thread per element of D, any legal input                  */

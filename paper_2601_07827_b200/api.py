@@ -44,7 +44,7 @@ ATTR_PRE_REDUCE = 10
 ATTR_BATCH_HINT = 11
 ATTR_COMPUTE_PRECISION = 12
 ATTR_POLL_LIMIT = 13
-PRECISION_DEFAULT, PRECISION_STRICT = 0, 1
+PRECISION_DEFAULT, PRECISION_STRICT, PRECISION_FP64_SUMS = 0, 1, 2
 KERNEL_AUTO, KERNEL_GENERIC, KERNEL_TILED = 0, 1, 2
 STATUS_KERNEL, STATUS_LAUNCHES, STATUS_GRID, STATUS_SPLIT_K, STATUS_VARIANT = 1, 2, 3, 4, 5
 

@@ -618,7 +618,7 @@ int replan(btc_contraction_s *op)
     op->spanD_lo = pl.spanD_lo; op->spanD_hi = pl.spanD_hi;
     op->sumA = op->sumB = IsolatedSum();
     op->sumB_offset = op->partials_offset = 0;
-    if (pl.has_isolated && op->pre_reduce) {
+    if (pl.has_isolated && op->pre_reduce && !pl.mixed) {
         // Case 4: plan the contraction of the summed inputs A', B' instead
         PlanRequest inner;
         IsolatedSum sa, sb;
@@ -850,9 +850,9 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
         if (v < 0) return BTC_ERR_INVALID_ARGUMENT;
         op->req.force_split_k = v;
     } else if (key == BTC_ATTR_COMPUTE_PRECISION) {
-        if (v != BTC_PRECISION_DEFAULT && v != BTC_PRECISION_STRICT) return BTC_ERR_INVALID_ARGUMENT;
+        if (v != BTC_PRECISION_DEFAULT && v != BTC_PRECISION_STRICT && v != BTC_PRECISION_FP64_SUMS) return BTC_ERR_INVALID_ARGUMENT;
         if (v == BTC_PRECISION_STRICT && op->plan.dtype == BTC_C32) return BTC_ERR_NOT_SUPPORTED;
-        op->req.strict_fp32 = v == BTC_PRECISION_STRICT ? 1 : 0;
+        op->req.strict_fp32 = v;
     } else if (key == BTC_ATTR_BATCH_HINT) {
         if (v < 1) return BTC_ERR_INVALID_ARGUMENT;
         op->req.batch_hint = v;
@@ -890,7 +890,7 @@ btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t 
     case BTC_ATTR_VARIANT: i32[0] = pl.tile.variant; n = 4; break;
     case BTC_ATTR_PRE_REDUCE: i32[0] = (op->sumA.active ? 1 : 0) | (op->sumB.active ? 2 : 0); n = 4; break;
     case BTC_ATTR_BATCH_HINT: i32[0] = op->req.batch_hint; n = 4; break;
-    case BTC_ATTR_COMPUTE_PRECISION: i32[0] = op->req.strict_fp32 ? BTC_PRECISION_STRICT : BTC_PRECISION_DEFAULT; n = 4; break;
+    case BTC_ATTR_COMPUTE_PRECISION: i32[0] = op->req.strict_fp32; n = 4; break;
     case BTC_ATTR_DEVICE_ERROR:
         i32[0] = 0;
         if (op->d_error) {
@@ -963,11 +963,12 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
     const bool use_ab = !is_zero(al), use_c = !is_zero(be);
     if (use_ab && (!A || !B)) return BTC_ERR_INVALID_ARGUMENT;
     if (use_c && (!C || !pl.has_c_desc)) return BTC_ERR_INVALID_ARGUMENT;
-    const size_t part = dtype_is_complex(pl.dtype) ? dtype_size(pl.dtype) / 2 : dtype_size(pl.dtype);
     auto misaligned = [&](const void *p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) != 0; };
     // complex128 accesses are 16-byte wide; everything else needs its element alignment
-    const size_t need = pl.dtype == BTC_C64 ? 16 : (pl.dtype == BTC_C32 ? 8 : part);
-    if (misaligned(A, need) || misaligned(B, need) || misaligned(C, need) || misaligned(D, need))
+    auto need_of = [](btc_dtype_t t) -> size_t { return t == BTC_C64 ? 16 : (t == BTC_C32 ? 8 : dtype_size(t)); };
+    const size_t need = need_of(pl.dtype);
+    if (misaligned(A, need_of(op->req.A.dtype)) || misaligned(B, need_of(op->req.B.dtype)) ||
+        misaligned(C, need_of(op->req.has_c ? op->req.C.dtype : pl.dtype)) || misaligned(D, need))
         return BTC_ERR_MISALIGNED;
     if (op->workspace_bytes > 0 && !bv) {        // a pointer-array batch has checked its own layout
         if (!workspace || workspace_bytes < op->workspace_bytes) return BTC_ERR_WORKSPACE_TOO_SMALL;
@@ -1013,6 +1014,7 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
         gp.total_k = pl.K;
         gp.alpha[0] = al[0]; gp.alpha[1] = al[1]; gp.beta[0] = be[0]; gp.beta[1] = be[1];
         gp.conjA = pl.conjA; gp.conjB = pl.conjB; gp.conjC = pl.conjC;
+        gp.cplxA = pl.cplxA; gp.cplxB = pl.cplxB; gp.cplxC = pl.cplxC;
         gp.use_ab = use_ab; gp.use_c = use_c;
         fill_spans(op, gp.spans);
         bool wpe = pl.kernel == BTC_KERNEL_GENERIC && op->grid[1] == 32;
@@ -1464,7 +1466,7 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
     // large inputs: cut the larger one into slabs and copy slab i + 1 while slab i is contracted
-    if (use_ab && op->poll_limit == kWaitPollLimit) {
+    if (use_ab && op->poll_limit == kWaitPollLimit && !pl.mixed) {
         if (!op->host) build_host_pipeline(op);
         if (op->host && op->host->usable) return run_host_pipeline(op, st, alpha, A, B, beta, C, D, use_c);
     }
@@ -1474,11 +1476,11 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
         int64_t lo = 0, hi = 0;
         size_t bytes() const { return size_t(hi - lo + 1); }
     } bA, bB, bC, bD;
-    auto span_bytes = [&](Buf &b, int64_t lo, int64_t hi) { b.lo = lo * int64_t(esz); b.hi = hi * int64_t(esz) + int64_t(esz) - 1; };
-    span_bytes(bA, op->spanA_lo, op->spanA_hi);
-    span_bytes(bB, op->spanB_lo, op->spanB_hi);
-    span_bytes(bD, op->spanD_lo, op->spanD_hi);
-    bC = bD;
+    auto span_bytes = [&](Buf &b, int64_t lo, int64_t hi, size_t es) { b.lo = lo * int64_t(es); b.hi = hi * int64_t(es) + int64_t(es) - 1; };
+    span_bytes(bA, op->spanA_lo, op->spanA_hi, dtype_size(op->req.A.dtype));
+    span_bytes(bB, op->spanB_lo, op->spanB_hi, dtype_size(op->req.B.dtype));
+    span_bytes(bD, op->spanD_lo, op->spanD_hi, esz);
+    span_bytes(bC, op->spanD_lo, op->spanD_hi, dtype_size(op->req.has_c ? op->req.C.dtype : pl.dtype));
     const bool c_is_d = use_c && C == D;
     void *ws = nullptr;
     btc_error_t rc = BTC_SUCCESS;

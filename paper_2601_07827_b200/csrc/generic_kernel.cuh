@@ -48,10 +48,12 @@ __global__ void __launch_bounds__(256) generic_contract_kernel(const GenericPara
                     ob += i * p.sB_k[d];
                 }
                 if (!BTC_IN_SPAN(p.spans, 0, oa, 1) || !BTC_IN_SPAN(p.spans, 1, ob, 1)) continue;
-                const double ar = double(A[NC * oa]), br = double(B[NC * ob]);
+                // a real operand among complex ones is read as (re, 0)
+                const int na = p.cplxA ? 2 : 1, nb = p.cplxB ? 2 : 1;
+                const double ar = double(A[na * oa]), br = double(B[nb * ob]);
                 if (CPLX) {
-                    const double ai = sa * double(A[NC * oa + (NC - 1)]);
-                    const double bi = sb * double(B[NC * ob + (NC - 1)]);
+                    const double ai = p.cplxA ? sa * double(A[na * oa + 1]) : 0.0;
+                    const double bi = p.cplxB ? sb * double(B[nb * ob + 1]) : 0.0;
                     acc_r += ar * br - ai * bi;
                     acc_i += ar * bi + ai * br;
                 } else {
@@ -70,8 +72,9 @@ __global__ void __launch_bounds__(256) generic_contract_kernel(const GenericPara
             double d_r = p.alpha[0] * acc_r - p.alpha[1] * acc_i;
             double d_i = p.alpha[0] * acc_i + p.alpha[1] * acc_r;
             if (p.use_c) {
-                const double cr = double(C[NC * offD]);
-                const double ci = CPLX ? sc * double(C[NC * offD + (NC - 1)]) : 0.0;
+                const int nc = p.cplxC ? 2 : 1;
+                const double cr = double(C[nc * offD]);
+                const double ci = p.cplxC ? sc * double(C[nc * offD + 1]) : 0.0;
                 d_r += p.beta[0] * cr - p.beta[1] * ci;
                 d_i += p.beta[0] * ci + p.beta[1] * cr;
             }

@@ -40,6 +40,7 @@ struct GenericParams {
     double alpha[2], beta[2];
     int32_t conjA, conjB, conjC;
     int32_t use_ab, use_c;
+    int32_t cplxA, cplxB, cplxC;      // 1: that operand's elements are (re, im) pairs; D's type is the kernel's
     OffsetSpans spans;
 };
 

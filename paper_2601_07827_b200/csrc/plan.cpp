@@ -142,9 +142,18 @@ int make_plan(const PlanRequest &req, Plan &plan)
         for (int64_t e : T[t]->extent)
             if (e < 1) return BTC_ERR_INVALID_EXTENT;
     }
-    if (req.A.dtype != req.D.dtype || req.B.dtype != req.D.dtype ||
-        (req.has_c && req.C.dtype != req.D.dtype))
-        return BTC_ERR_NOT_SUPPORTED;
+    // Element types (Sec. "Challenge: Datatypes"): the tensors may mix real and complex elements of one part
+    // width; D must be complex when an input is.  Other mixes (32- with 64-bit parts) are not supported.
+    const bool mixed = req.A.dtype != req.D.dtype || req.B.dtype != req.D.dtype || (req.has_c && req.C.dtype != req.D.dtype);
+    {
+        auto part = [](btc_dtype_t t) { return (t == BTC_F32 || t == BTC_C32) ? 4 : 8; };
+        const btc_dtype_t c_type = req.has_c ? req.C.dtype : req.D.dtype;
+        if (part(req.A.dtype) != part(req.D.dtype) || part(req.B.dtype) != part(req.D.dtype) || part(c_type) != part(req.D.dtype))
+            return BTC_ERR_NOT_SUPPORTED;
+        if (!dtype_is_complex(req.D.dtype) &&
+            (dtype_is_complex(req.A.dtype) || dtype_is_complex(req.B.dtype) || dtype_is_complex(c_type)))
+            return BTC_ERR_NOT_SUPPORTED;
+    }
     for (size_t i = 0; i < req.labelsD.size(); ++i)
         for (size_t j = 0; j < i; ++j)
             if (req.labelsD[i] == req.labelsD[j]) return BTC_ERR_NOT_SUPPORTED;
@@ -183,9 +192,13 @@ int make_plan(const PlanRequest &req, Plan &plan)
     // ---- classify (Sec. "Operations": H, F_A, F_B, P; I_A / I_B of Case 4) ----
     plan = Plan();
     plan.dtype = req.D.dtype;
-    plan.conjA = req.conjA && dtype_is_complex(plan.dtype);
-    plan.conjB = req.conjB && dtype_is_complex(plan.dtype);
-    plan.conjC = req.conjC && dtype_is_complex(plan.dtype);
+    plan.mixed = mixed;
+    plan.cplxA = dtype_is_complex(req.A.dtype);
+    plan.cplxB = dtype_is_complex(req.B.dtype);
+    plan.cplxC = dtype_is_complex(req.has_c ? req.C.dtype : req.D.dtype);
+    plan.conjA = req.conjA && plan.cplxA;
+    plan.conjB = req.conjB && plan.cplxB;
+    plan.conjC = req.conjC && plan.cplxC;
     plan.has_c_desc = req.has_c;
     for (auto &r : rows) {
         if (r.extent == 1) continue;  // contributes no loop and no offset
@@ -220,6 +233,7 @@ int make_plan(const PlanRequest &req, Plan &plan)
             for (auto *g : {&plan.batch, &plan.m, &plan.n, &plan.k})
                 for (auto &md : *g) std::swap(md.sA, md.sB);
             std::swap(plan.conjA, plan.conjB);
+            std::swap(plan.cplxA, plan.cplxB);
             plan.swapped = true;
         }
     }
@@ -378,7 +392,9 @@ int make_plan(const PlanRequest &req, Plan &plan)
 
     // ---- kernel choice ----
     const int64_t entries = 2 * (plan.M + plan.N + plan.K) + 3 * plan.Bt;
-    const bool tiled_ok = !plan.has_isolated && entries <= kMaxTableEntries;
+    // mixed element types and 32-bit storage with sums kept in fp64 run on the per-element kernel
+    const bool wide_sums = req.strict_fp32 == 2 && esz0 == (dtype_is_complex(plan.dtype) ? 8 : 4);
+    const bool tiled_ok = !plan.has_isolated && entries <= kMaxTableEntries && !plan.mixed && !wide_sums;
     plan.kernel = BTC_KERNEL_GENERIC;
     if (req.force_kernel == BTC_KERNEL_TILED && !tiled_ok) return BTC_ERR_NOT_SUPPORTED;
     // (with at most four contracted indices the streaming kernel serves every size)

@@ -42,6 +42,9 @@ struct Plan {
     bool swapped = false;        // true: the caller's B is the plan's A
     bool has_c_desc = false;
     bool has_isolated = false;   // Case 4 labels present; if planned as they are, the generic kernel sums them
+    // element types differ between the tensors (same part width; D complex when an input is): which of the
+    // planned A, B and C are complex.  Such operations run on the per-element kernel.
+    bool mixed = false, cplxA = false, cplxB = false, cplxC = false;
 
     // loop dimensions in planned order, first entry fastest in the linearised index
     std::vector<Mode> batch, m, n, k;
@@ -76,7 +79,7 @@ struct PlanRequest {
     int32_t force_kernel = BTC_KERNEL_AUTO;
     int32_t force_split_k = 0;   // 0 = choose
     int32_t force_variant = -1;  // -1 = choose; otherwise index of the tile variant for the dtype
-    int32_t strict_fp32 = 0;     // 1: fp32 / complex64 products and sums in IEEE fp32 (no TF32 split)
+    int32_t strict_fp32 = 0;     // 1: fp32 / complex64 products and sums in IEEE fp32 (no TF32 split); 2: sums kept in fp64
     int32_t batch_hint = 1;      // pointer-array entries the operation is expected to run with at a time
     int32_t sm_count = 148;
 };

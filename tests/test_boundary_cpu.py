@@ -196,3 +196,16 @@ def test_elementwise_planning_without_a_device(api, handle):
         buf = (ctypes.c_float * 64 * 32 * 16)()
         p = ctypes.addressof(buf)
         assert _code(api, lambda: same.execute(0, p, p, p)) == api.ERR_CUDA
+
+
+def test_element_type_mixes(api, handle):
+    """Real among complex operands of one part width plan (on the per-element kernel); 32- with 64-bit parts and
+    a real result of a complex input are refused (Sec. "Challenge: Datatypes": an implementation may support
+    fewer mixes than the reference one)."""
+    t = lambda dt, ext: api.TensorInfo(handle, dt, ext)
+    op = api.Contraction(handle, t(api.F64, (4, 5)), "ik", t(api.C64, (5, 3)), "kj", None, "ij", t(api.C64, (4, 3)), "ij")
+    assert op.kernel == api.KERNEL_GENERIC
+    for a, b, d in ((api.F32, api.F64, api.F64), (api.C64, api.F64, api.F64), (api.C32, api.C64, api.C64)):
+        with pytest.raises(api.BtcError) as ei:
+            api.Contraction(handle, t(a, (4, 5)), "ik", t(b, (5, 3)), "kj", None, "ij", t(d, (4, 3)), "ij")
+        assert ei.value.code == api.ERR_NOT_SUPPORTED
