@@ -539,7 +539,8 @@ int finish_plan(btc_contraction_s *op)
             }
             int64_t klo = 0, khi = 0;
             for (int64_t k = 0; k < int64_t(k_off.size()); ++k) { klo = std::min(klo, k_off[size_t(k)]); khi = std::max(khi, k_off[size_t(k)]); }
-            return hi + khi < (int64_t(1) << 30) && lo + klo > -(int64_t(1) << 30);
+            // (offsets inside a tile are kept in 20 bits, in units of four elements)
+            return hi + khi < (int64_t(1) << 20) && lo + klo > -(int64_t(1) << 20);
         };
         op->skinny_regular = regular(pl.offA_m, pl.offA_k) && regular(pl.offB_n, pl.offB_k);
         const std::vector<int64_t> none(1, 0);

@@ -38,7 +38,9 @@ namespace btc {
 
 struct SkinnyTile {
     static constexpr int BM = 128, BN = 128, KMAX = 64;
-    static constexpr int B_STAGES = 2;
+    // the N-side tiles wait in a ring of raw stages (filled up to three tiles ahead of the tensor core, to ride out
+    // the memory latency); their tails are made just in time into a shorter ring
+    static constexpr int RAW_STAGES = 3, LO_STAGES = 2;
     static constexpr int EPILOGUE_WARPS = 4, CONVERTER_WARPS = 4, LOADER_WARPS = 4;
     static constexpr int GROUP_THREADS = 128;
     static constexpr int MMA_WARP = EPILOGUE_WARPS + CONVERTER_WARPS + LOADER_WARPS;
@@ -50,11 +52,11 @@ struct SkinnyTile {
     static constexpr int PER_THREAD = PIECES / GROUP_THREADS;
     static constexpr int ACC_COLS = 128, A_COLS = 2 * KMAX;  // tensor-memory columns: accumulator; head + tail of the M side
     static constexpr int TMEM_COLS = 512;                    // 2 accumulators + 2 M-side operand buffers
-    static constexpr int NUM_BARS = 20;
+    static constexpr int NUM_BARS = 24;
     static constexpr int SPLIT_COL = 64;                     // columns below: epilogue warps; from here on: the converter warps, between conversions
-    // N-side raw[2] | N-side tail[2] | M-side raw | row / column offsets | k offsets | piece tables | barriers | slot, abort
-    static constexpr size_t SMEM_BYTES = size_t(2 * B_STAGES) * B_BYTES + A_BYTES +
-                                         size_t(2 * BM + B_STAGES * BN + 2 * KMAX) * 8 + size_t(2 * PIECES) * 8 +
+    // N-side raw[3] | N-side tail[2] | M-side raw | row / column offsets | k offsets | piece tables | barriers | slot, abort
+    static constexpr size_t SMEM_BYTES = size_t(RAW_STAGES + LO_STAGES) * B_BYTES + A_BYTES +
+                                         size_t(2 * BM + RAW_STAGES * BN + 2 * KMAX) * 8 + size_t(2 * PIECES) * 4 +
                                          size_t(NUM_BARS) * 8 + 16 + 1024;
 };
 
@@ -73,11 +75,13 @@ struct SkinnyTile {
 constexpr int kErrSkinnyLoad = 8, kErrSkinnyConvert = 9, kErrSkinnyMma = 10, kErrSkinnyEpilogue = 11;
 
 // One operand tile: every loader thread copies its pieces (entries pt, pt + 128, ... of the piece
-// order), eight look-ups first, then their eight copies.  `table` (shared memory) holds per piece,
-// in piece order: .x bits 0-10 destination in 16-byte units, bits 11-17 first row, bits 18-23 first k,
-// bit 24 k < K;  .y element offset of the piece relative to the tile's first row (regular operands).
+// order), eight look-ups first, then their eight copies.  `table` (shared memory) holds per piece, in
+// piece order: bits 0-10 the piece (see skinny_a_pos / skinny_b_pos), bit 11 its k < K, bits 12-31 (signed)
+// its offset relative to the tile's first row in units of four elements (regular operands only).
+template <bool IS_A>
 __device__ __forceinline__ void skinny_load_tile(unsigned tile, const float *g, const int64_t *row_off, const int64_t *koff,
-                                                 const uint2 *table, int pieces, int rows_valid, int pt, const OffsetSpans &spans, int which)
+                                                 const unsigned *table, int pieces, int dir, int rows_valid, int pt,
+                                                 const OffsetSpans &spans, int which)
 {
 #pragma unroll 1
     for (int e0 = pt; e0 < pieces; e0 += 8 * SkinnyTile::GROUP_THREADS) {
@@ -87,10 +91,10 @@ __device__ __forceinline__ void skinny_load_tile(unsigned tile, const float *g, 
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int e = e0 + j * SkinnyTile::GROUP_THREADS;
-            const unsigned pk = e < pieces ? table[e].x : 0u;
-            const int row = int(pk >> 11) & 127, k = int(pk >> 18) & 63;
-            dst[j] = (pk & 2047u) << 4;
-            valid[j] = ((pk >> 24) & 1u) && row < rows_valid;
+            const unsigned pk = e < pieces ? table[e] : 0u;
+            int row, k;
+            dst[j] = IS_A ? skinny_a_pos(dir, pk & 2047u, row, k) : skinny_b_pos(dir, pk & 2047u, row, k);
+            valid[j] = ((pk >> 11) & 1u) && row < rows_valid;
             off[j] = valid[j] ? row_off[row] + koff[k] : 0;
             if (valid[j] && !BTC_IN_SPAN(spans, which, off[j], 4)) { valid[j] = false; off[j] = 0; }
         }
@@ -101,23 +105,26 @@ __device__ __forceinline__ void skinny_load_tile(unsigned tile, const float *g, 
 }
 // The same for a regular operand (every tile's rows lie relative to its first row as tile 0's do):
 // `base` is the offset of the tile's first row, the table gives the rest; no offset arrays are needed.
-__device__ __forceinline__ void skinny_load_tile_regular(unsigned tile, const float *g, int64_t base, const uint2 *table, int pieces, int rows_valid,
-                                                         int pt, const OffsetSpans &spans, int which)
+template <bool IS_A>
+__device__ __forceinline__ void skinny_load_tile_regular(unsigned tile, const float *g, int64_t base, const unsigned *table, int pieces,
+                                                         int dir, int rows_valid, int pt, const OffsetSpans &spans, int which)
 {
 #pragma unroll 1
     for (int e0 = pt; e0 < pieces; e0 += 8 * SkinnyTile::GROUP_THREADS) {
-        uint2 q[8];
+        unsigned q[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int e = e0 + j * SkinnyTile::GROUP_THREADS;
-            q[j] = e < pieces ? table[e] : make_uint2(0u, 0u);
+            q[j] = e < pieces ? table[e] : 0u;
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            bool valid = ((q[j].x >> 24) & 1u) && int((q[j].x >> 11) & 127u) < rows_valid;
-            valid = valid && BTC_IN_SPAN(spans, which, base + int(q[j].y), 4);
-            if (e0 + j * SkinnyTile::GROUP_THREADS < pieces)
-                cp_async_bytes<16>(tile + ((q[j].x & 2047u) << 4), g + (valid ? base + int(q[j].y) : 0), valid);
+            int row, k;
+            const unsigned dst = IS_A ? skinny_a_pos(dir, q[j] & 2047u, row, k) : skinny_b_pos(dir, q[j] & 2047u, row, k);
+            const int64_t off = base + 4 * int64_t(int(q[j]) >> 12);
+            bool valid = ((q[j] >> 11) & 1u) && row < rows_valid;
+            valid = valid && BTC_IN_SPAN(spans, which, off, 4);
+            if (e0 + j * SkinnyTile::GROUP_THREADS < pieces) cp_async_bytes<16>(tile + dst, g + (valid ? off : 0), valid);
         }
     }
 }
@@ -274,23 +281,24 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
     extern __shared__ __align__(16) unsigned char smem_unaligned[];
     unsigned char *smem_raw = smem_unaligned +
         ((1024u - (static_cast<unsigned>(__cvta_generic_to_shared(smem_unaligned)) & 1023u)) & 1023u);
-    unsigned char *cursor = smem_raw + size_t(2 * T::B_STAGES) * T::B_BYTES + T::A_BYTES;
+    unsigned char *cursor = smem_raw + size_t(T::RAW_STAGES + T::LO_STAGES) * T::B_BYTES + T::A_BYTES;
     int64_t *rowA = reinterpret_cast<int64_t *>(cursor);                 // [2][BM]
-    int64_t *colB = rowA + 2 * T::BM;                                    // [B_STAGES][BN]
-    int64_t *koffA = colB + T::B_STAGES * T::BN;                         // [KMAX]
+    int64_t *colB = rowA + 2 * T::BM;                                    // [RAW_STAGES][BN]
+    int64_t *koffA = colB + T::RAW_STAGES * T::BN;                       // [KMAX]
     int64_t *koffB = koffA + T::KMAX;                                    // [KMAX]
-    uint2 *pieceA = reinterpret_cast<uint2 *>(koffB + T::KMAX);          // [PIECES] piece tables
-    uint2 *pieceB = pieceA + T::PIECES;                                  // [PIECES]
+    unsigned *pieceA = reinterpret_cast<unsigned *>(koffB + T::KMAX);    // [PIECES] piece tables
+    unsigned *pieceB = pieceA + T::PIECES;                               // [PIECES]
     uint64_t *bars = reinterpret_cast<uint64_t *>(pieceB + T::PIECES);
     unsigned *tmem_slot = reinterpret_cast<unsigned *>(bars + T::NUM_BARS);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     const unsigned braw0 = static_cast<unsigned>(__cvta_generic_to_shared(smem_raw));
-    const unsigned blo0 = braw0 + unsigned(T::B_STAGES) * T::B_BYTES;
-    const unsigned araw = blo0 + unsigned(T::B_STAGES) * T::B_BYTES;
+    const unsigned blo0 = braw0 + unsigned(T::RAW_STAGES) * T::B_BYTES;
+    const unsigned araw = blo0 + unsigned(T::LO_STAGES) * T::B_BYTES;
     const unsigned bar0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
     const unsigned a_full = bar0, a_empty = bar0 + 8u;
-    const unsigned b_full0 = bar0 + 16u, b_conv0 = b_full0 + 16u, b_empty0 = b_conv0 + 16u;   // [2] each
-    const unsigned ta_full0 = b_empty0 + 16u, ta_empty0 = ta_full0 + 16u;                     // [2] each
+    const unsigned raw_full0 = bar0 + 16u, raw_empty0 = raw_full0 + 24u;                      // [3] each
+    const unsigned lo_conv0 = raw_empty0 + 24u, lo_empty0 = lo_conv0 + 16u;                   // [2] each
+    const unsigned ta_full0 = lo_empty0 + 16u, ta_empty0 = ta_full0 + 16u;                    // [2] each
     const unsigned acc_full0 = ta_empty0 + 16u, acc_empty0 = acc_full0 + 16u;                 // [2] each
     const unsigned loader_sync = acc_empty0 + 16u, drain = loader_sync + 8u;
 
@@ -308,26 +316,29 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
     }
     for (int e = tid; e < pieces; e += T::THREADS) {
         int row, k;
-        unsigned dst = skinny_a_pos(p.dirA, p.skinny_orderA[e], row, k);
-        bool in = row < p.M && k < K;
-        pieceA[e] = make_uint2((dst >> 4) | (unsigned(row) << 11) | (unsigned(k) << 18) | (unsigned(k < K) << 24),
-                               unsigned(int(in ? p.offA_m[row] - p.offA_m[0] + p.offA_k[k] : 0)));
-        dst = skinny_b_pos(p.dirB, p.skinny_orderB[e], row, k);
-        in = row < p.N && k < K;
-        pieceB[e] = make_uint2((dst >> 4) | (unsigned(row) << 11) | (unsigned(k) << 18) | (unsigned(k < K) << 24),
-                               unsigned(int(in ? p.offB_n[row] - p.offB_n[0] + p.offB_k[k] : 0)));
+        unsigned code = p.skinny_orderA[e];
+        skinny_a_pos(p.dirA, code, row, k);
+        int64_t rel = (row < p.M && k < K) ? p.offA_m[row] - p.offA_m[0] + p.offA_k[k] : 0;
+        pieceA[e] = code | (unsigned(k < K) << 11) | (unsigned(int(rel / 4)) << 12);
+        code = p.skinny_orderB[e];
+        skinny_b_pos(p.dirB, code, row, k);
+        rel = (row < p.N && k < K) ? p.offB_n[row] - p.offB_n[0] + p.offB_k[k] : 0;
+        pieceB[e] = code | (unsigned(k < K) << 11) | (unsigned(int(rel / 4)) << 12);
     }
     if (tid == 0) {
         mbar_init(a_full, T::GROUP_THREADS);
         mbar_init(a_empty, T::GROUP_THREADS);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(b_full0 + 8u * s, T::GROUP_THREADS);
-            mbar_init(b_conv0 + 8u * s, T::GROUP_THREADS);
-            mbar_init(b_empty0 + 8u * s, 1);
+            mbar_init(lo_conv0 + 8u * s, T::GROUP_THREADS);
+            mbar_init(lo_empty0 + 8u * s, 1);
             mbar_init(ta_full0 + 8u * s, T::GROUP_THREADS);
             mbar_init(ta_empty0 + 8u * s, 1);
             mbar_init(acc_full0 + 8u * s, 1);
             mbar_init(acc_empty0 + 8u * s, 2 * T::GROUP_THREADS);
+        }
+        for (int s = 0; s < T::RAW_STAGES; ++s) {
+            mbar_init(raw_full0 + 8u * s, T::GROUP_THREADS);
+            mbar_init(raw_empty0 + 8u * s, 1);
         }
         mbar_init(loader_sync, T::GROUP_THREADS);
         mbar_init(drain, 1);
@@ -427,13 +438,15 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
                 mbar_arrive(a_empty);                 // the raw M-side buffer may be refilled
             }
             BTC_PHASE_END(t_work);
-            if (!mbar_wait_bounded(b_full0 + 8u * s, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)) break;
+            const int r = i % T::RAW_STAGES;
+            if (!mbar_wait_bounded(raw_full0 + 8u * r, unsigned(i / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)) break;
+            // the tail stage is free once the tensor core has finished the tile two before this one
+            if (i >= 2 && !mbar_wait_bounded(lo_empty0 + 8u * s, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)) break;
             BTC_PHASE_END(t_wait);
             BTC_EVENT(p, ct == 0, 2, i);
             // N side: position-independent pass; the raw stage is the head, the tail goes to the same
-            // position of the tail stage.  (The tail stage is free: this stage's copies were issued only
-            // after the MMAs that read both had completed.)
-            const unsigned src = braw0 + unsigned(s) * T::B_BYTES + unsigned(ct) * 16u;
+            // position of the tail stage
+            const unsigned src = braw0 + unsigned(r) * T::B_BYTES + unsigned(ct) * 16u;
             const unsigned dst = blo0 + unsigned(s) * T::B_BYTES + unsigned(ct) * 16u;
             const int per = (kp <= 32 ? T::B_BLOCK_BYTES : T::B_BYTES) / 16 / T::GROUP_THREADS;   // 8 or 16 pieces per thread
 #pragma unroll
@@ -453,7 +466,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
                 }
             }
             proxy_fence_async();                      // the tensor core reads both stages through the async proxy
-            mbar_arrive(b_conv0 + 8u * s);
+            mbar_arrive(lo_conv0 + 8u * s);
             BTC_EVENT(p, ct == 0, 3, i);
             if (i > 0) {
                 const int ip = i - 1, buf = ip & 1;
@@ -505,7 +518,8 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             const int i = int(t - t0), s = i & 1;
             const bool new_strip = t == t0 || w.nt == 0;
             if (new_strip) ++sidx;
-            int64_t *rA = rowA + (sidx & 1) * T::BM, *cB = colB + s * T::BN;
+            const int r = i % T::RAW_STAGES;
+            int64_t *rA = rowA + (sidx & 1) * T::BM, *cB = colB + r * T::BN;
             const int64_t row_base = next_row, col_base = next_col;
             if (!regular) {
                 if (new_strip) rA[pt] = next_row;
@@ -516,17 +530,18 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             if (t + 1 < t1) fetch(wn);
             if (new_strip) {
                 if (sidx > 0 && !mbar_wait_bounded(a_empty, unsigned(sidx - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
-                if (regular) skinny_load_tile_regular(araw, A, row_base, pieceA, pieces, w.rows_valid, pt, p.spans, 0);
-                else skinny_load_tile(araw, A, rA, koffA, pieceA, pieces, w.rows_valid, pt, p.spans, 0);
+                if (regular) skinny_load_tile_regular<true>(araw, A, row_base, pieceA, pieces, p.dirA, w.rows_valid, pt, p.spans, 0);
+                else skinny_load_tile<true>(araw, A, rA, koffA, pieceA, pieces, p.dirA, w.rows_valid, pt, p.spans, 0);
                 mbar_arrive_on_copies(a_full);
             }
             BTC_PHASE_END(t_work);
-            if (i >= 2 && !mbar_wait_bounded(b_empty0 + 8u * s, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
+            if (i >= T::RAW_STAGES &&
+                !mbar_wait_bounded(raw_empty0 + 8u * r, unsigned(i / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
             BTC_PHASE_END(t_wait);
             BTC_EVENT(p, pt == 0, 0, i);
-            if (regular) skinny_load_tile_regular(braw0 + unsigned(s) * T::B_BYTES, B, col_base, pieceB, pieces, w.cols_valid, pt, p.spans, 1);
-            else skinny_load_tile(braw0 + unsigned(s) * T::B_BYTES, B, cB, koffB, pieceB, pieces, w.cols_valid, pt, p.spans, 1);
-            mbar_arrive_on_copies(b_full0 + 8u * s);
+            if (regular) skinny_load_tile_regular<false>(braw0 + unsigned(r) * T::B_BYTES, B, col_base, pieceB, pieces, p.dirB, w.cols_valid, pt, p.spans, 1);
+            else skinny_load_tile<false>(braw0 + unsigned(r) * T::B_BYTES, B, cB, koffB, pieceB, pieces, p.dirB, w.cols_valid, pt, p.spans, 1);
+            mbar_arrive_on_copies(raw_full0 + 8u * r);
             BTC_EVENT(p, pt == 0, 1, i);
             w = wn;
         }
@@ -560,14 +575,14 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             BTC_PHASE_END(t_issue);
             if (i >= 2 && !mbar_wait_bounded(acc_empty0 + 8u * buf, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
             BTC_PHASE_END(t_acc);
-            if (!mbar_wait_bounded(b_conv0 + 8u * s, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
+            if (!mbar_wait_bounded(lo_conv0 + 8u * s, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
             BTC_PHASE_END(t_conv);
             BTC_EVENT(p, lane == 0, 4, i);
             tc_fence_after();
             if (leader) {
                 const unsigned tacc = tmem_base + unsigned(buf * T::ACC_COLS);
                 const unsigned ta = tmem_a0 + unsigned((sidx & 1) * T::A_COLS);      // head columns; tail KMAX further
-                const unsigned b_hi = braw0 + unsigned(s) * T::B_BYTES, b_lo = blo0 + unsigned(s) * T::B_BYTES;
+                const unsigned b_hi = braw0 + unsigned(i % T::RAW_STAGES) * T::B_BYTES, b_lo = blo0 + unsigned(s) * T::B_BYTES;
 #pragma unroll 1
                 for (int j = 0; j < ksteps; ++j) {
                     const unsigned at = unsigned(j >> 2) * T::B_BLOCK_BYTES + unsigned(j & 3) * b_step;
@@ -577,7 +592,8 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
                     umma_tf32_ts(tacc, ta + unsigned(8 * j), dbl, idesc, 1u);
                     umma_tf32_ts(tacc, ta + unsigned(8 * j), dbh, idesc, 1u);
                 }
-                umma_commit(b_empty0 + 8u * s);               // fires when these MMAs have read both stages
+                umma_commit(raw_empty0 + 8u * unsigned(i % T::RAW_STAGES));       // fire when these MMAs have read the stages
+                umma_commit(lo_empty0 + 8u * s);
                 umma_commit(acc_full0 + 8u * buf);
                 if (t + 1 == t1 || nt == 0) umma_commit(ta_empty0 + 8u * (sidx & 1));
             }
