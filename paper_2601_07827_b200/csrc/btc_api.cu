@@ -63,8 +63,8 @@ struct btc_contraction_s {
     const int32_t *d_tma_coord_m = nullptr, *d_tma_coord_k = nullptr, *d_tma_coord_h = nullptr;
     // short-K streaming kernel: piece orders of the operand tiles; how many consecutive m are contiguous in D
     // ([0], [1]: the plan's A as the kernel's M side / N side; [2], [3]: the plan's B likewise)
-    std::vector<uint16_t> skinny_order[4];
-    const uint16_t *d_skinny_order[4] = {nullptr, nullptr, nullptr, nullptr};
+    std::vector<uint32_t> skinny_order[4];
+    const uint32_t *d_skinny_order[4] = {nullptr, nullptr, nullptr, nullptr};
     int64_t skinny_run_m = 1;
     bool skinny_regular = false;
     bool skinny_d_regular[2] = {false, false};     // D's rows (m) / columns (n) regular
@@ -520,8 +520,15 @@ int finish_plan(btc_contraction_s *op)
                 if (la == lb) return a.dst < b.dst;
                 return first[la] != first[lb] ? first[la] < first[lb] : la < lb;
             });
-            std::vector<uint16_t> out;
-            for (auto &x : v) out.push_back(x.e);
+            // per piece, in that order: bits 0-10 the piece, bit 11 its k < K, bits 12-31 (signed) its offset
+            // relative to the tile's first row in units of four elements (used for regular operands only)
+            std::vector<uint32_t> out;
+            for (auto &x : v) {
+                int row, k;
+                if (n_side) skinny_b_pos(d, unsigned(x.e), row, k); else skinny_a_pos(d, unsigned(x.e), row, k);
+                const int64_t rel = (row < rows && k < pl.K) ? row_off[size_t(row)] - row_off[0] + k_off[size_t(k)] : 0;
+                out.push_back(uint32_t(x.e) | (uint32_t(k < pl.K) << 11) | (uint32_t(int32_t(rel / 4)) << 12));
+            }
             return out;
         };
         op->skinny_order[0] = operand_order(pl.offA_m, pl.offA_k, pl.M, pl.dirA, false);
@@ -575,7 +582,7 @@ int finish_plan(btc_contraction_s *op)
         size_t blob_bytes[4], bstart[4];
         for (int i = 0; i < 4; ++i) {
             blob[i] = op->skinny_order[i].data();
-            blob_bytes[i] = op->skinny_order[i].size() * 2;
+            blob_bytes[i] = op->skinny_order[i].size() * 4;
             bstart[i] = total;
             total += (blob_bytes[i] + 255) / 256 * 32;
         }
@@ -604,7 +611,7 @@ int finish_plan(btc_contraction_s *op)
         op->d_tma_coord_m = reinterpret_cast<const int32_t *>(op->d_tables + cstart[0]);
         op->d_tma_coord_k = reinterpret_cast<const int32_t *>(op->d_tables + cstart[1]);
         op->d_tma_coord_h = reinterpret_cast<const int32_t *>(op->d_tables + cstart[2]);
-        for (int i = 0; i < 4; ++i) op->d_skinny_order[i] = reinterpret_cast<const uint16_t *>(op->d_tables + bstart[i]);
+        for (int i = 0; i < 4; ++i) op->d_skinny_order[i] = reinterpret_cast<const uint32_t *>(op->d_tables + bstart[i]);
     }
     return BTC_SUCCESS;
 }

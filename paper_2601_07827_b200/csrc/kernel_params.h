@@ -101,7 +101,7 @@ struct TiledParams {
     // short-K streaming kernel: the 16-byte pieces of an operand tile (128 rows x up to 64 k), each
     // list sorted by address in its tensor (see skinny_umma_kernel.cuh); skinny_vec_n = 4: groups of
     // four consecutive n are four consecutive, 16-byte aligned elements of D (and C)
-    const uint16_t *skinny_orderA, *skinny_orderB;
+    const uint32_t *skinny_orderA, *skinny_orderB;
     int32_t skinny_vec_n;
     // 1: in both operands every tile's rows lie relative to the tile's first row as those of tile 0 do, and
     // the offsets inside a tile fit 32 bits: tiles are addressed by their first row's offset alone

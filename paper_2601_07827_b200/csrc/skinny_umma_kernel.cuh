@@ -5,8 +5,10 @@
 //
 // All of K fits one shared-memory tile, so there is no k loop and no stage ring along k.
 // Persistent CTAs (one per SM) each take a contiguous range of the 128 x 128 output tiles, ordered
-// (batch entry, tile row, tile column) with the column fastest, so that consecutive tiles of a CTA
-// share their M-side operand tile ("strip"), which is fetched and converted once per strip.
+// (batch entry, pair of tile rows, tile column, half of the pair): the tiles of one tile row share their
+// M-side operand tile ("strip"), which is fetched and converted once per strip and stays in tensor
+// memory, and the two tiles of a pair share their N-side tile, so every operand tile fetched feeds two
+// output tiles (a 256 x 128 block of D per 128 x K tile of B).
 //   loaders     fetch the operand tiles with 16-byte asynchronous copies enumerated IN MEMORY
 //               ORDER: the host sorts the tile's 16-byte pieces by address once per operation
 //               ("piece order" tables), so a warp's 32 copies cover whole 128-byte lines even when
@@ -59,18 +61,6 @@ struct SkinnyTile {
                                          size_t(2 * BM + RAW_STAGES * BN + 2 * KMAX) * 8 + size_t(2 * PIECES) * 4 +
                                          size_t(NUM_BARS) * 8 + 16 + 1024;
 };
-
-// debug builds (-DBTC_STAMPS -DBTC_EVENTS): CTA 0 records the SM clock at eight events of its first 64 tiles
-#if defined(BTC_STAMPS) && defined(BTC_EVENTS)
-#define BTC_EVENT(p, who, ev, i) do { if ((who) && (p).stamps && blockIdx.x == 0 && (i) < 64) (p).stamps[2048 + (ev) * 64 + (i)] = clock64(); } while (0)
-#else
-#define BTC_EVENT(p, who, ev, i) do { } while (0)
-#endif
-#if defined(BTC_STAMPS) && defined(BTC_EVENTS_EPI)
-#define BTC_EPI_EVENT(p, who, ev, i) do { if ((who) && (p).stamps && blockIdx.x == 0 && (i) < 64) (p).stamps[2048 + (ev) * 64 + (i)] = clock64(); } while (0)
-#else
-#define BTC_EPI_EVENT(p, who, ev, i) do { } while (0)
-#endif
 
 constexpr int kErrSkinnyLoad = 8, kErrSkinnyConvert = 9, kErrSkinnyMma = 10, kErrSkinnyEpilogue = 11;
 
@@ -135,38 +125,76 @@ struct SkinnyWork {
     int64_t m0, n0;
     int rows_valid, cols_valid;
 };
-__device__ __forceinline__ void skinny_work_fill(const TiledParams &p, SkinnyWork &w)
-{
-    w.m0 = int64_t(w.mt) * SkinnyTile::BM;
-    w.n0 = int64_t(w.nt) * SkinnyTile::BN;
-    w.rows_valid = int(imin64(SkinnyTile::BM, p.M - w.m0));
-    w.cols_valid = int(imin64(SkinnyTile::BN, p.N - w.n0));
-}
-// tile t of the list (batch entry, tile row, tile column), column fastest
-__device__ __forceinline__ SkinnyWork skinny_work_at(const TiledParams &p, int64_t t)
-{
-    SkinnyWork w;
-    w.nt = int(t % p.tiles_n);
-    const int64_t q = t / p.tiles_n;
-    w.mt = int(q % p.tiles_m);
-    w.h = q / p.tiles_m;
-    skinny_work_fill(p, w);
-    return w;
-}
-// the tile after w (no divisions: every role steps through its tiles with this)
-__device__ __forceinline__ SkinnyWork skinny_work_next(const TiledParams &p, const SkinnyWork &w)
-{
-    SkinnyWork n = w;
-    if (++n.nt == p.tiles_n) {
-        n.nt = 0;
-        if (++n.mt == p.tiles_m) {
-            n.mt = 0;
-            ++n.h;
-        }
+
+// A CTA's walk through its output tiles.  The tile list is ordered (batch entry, pair of tile rows, tile
+// column, half of the pair) with the half fastest: the two tiles of a pair use the same N-side tile, which
+// is therefore fetched and converted once for both (each half has its own M-side operand in tensor
+// memory, kept for the whole strip).  With one tile row, or too few pairs to occupy the grid, halves = 1
+// and every tile is its own pair.  A pair's second half may not exist (odd number of tile rows): the walk
+// skips it.  Every role steps through the same walk, so the counters below agree between them.
+struct SkinnyIter {
+    int64_t h, left;         // batch entry; slots from this one to the end of the CTA's range
+    int halves, half, nt, mt, since;
+    int i, bi, an0, an1;     // tiles before this one; N-side tiles before this one's; M-side tiles loaded before, per half
+    int abuf;                // tensor-memory buffer of this tile's M-side operand: its half, or (halves = 1) alternating by strip
+    bool valid, new_a;       // new_a: the first tile of its half's strip for this CTA (its M-side tile must be loaded)
+
+    __device__ __forceinline__ void start(const TiledParams &p, int halves_, int64_t pair0, int64_t pair1)
+    {
+        halves = halves_;
+        const int tiles_mp = (p.tiles_m + halves - 1) / halves;
+        nt = int(pair0 % p.tiles_n);
+        const int64_t q = pair0 / p.tiles_n;
+        mt = int(q % tiles_mp) * halves;
+        h = q / tiles_mp;
+        half = 0; since = 0;
+        left = (pair1 - pair0) * halves;
+        valid = left > 0;
+        i = bi = an0 = an1 = abuf = 0;
+        new_a = true;
     }
-    skinny_work_fill(p, n);
-    return n;
-}
+    __device__ __forceinline__ void advance(const TiledParams &p)
+    {
+        if (new_a) { if (half) ++an1; else ++an0; }
+        for (;;) {
+            --left; ++since;
+            if (left <= 0) { valid = false; return; }
+            if (++half == halves) {
+                half = 0;
+                mt -= halves - 1;
+                if (++nt == p.tiles_n) {
+                    nt = 0;
+                    mt += halves;
+                    if (mt >= p.tiles_m) { mt = 0; ++h; }
+                }
+            } else {
+                ++mt;
+            }
+            if (mt < p.tiles_m) break;
+        }
+        ++i;
+        if (half == 0) ++bi;
+        new_a = nt == 0 || since < halves;
+        if (halves == 2) abuf = half;
+        else if (new_a) abuf = an0 & 1;
+    }
+    __device__ __forceinline__ bool first_of_b() const { return half == 0; }
+    __device__ __forceinline__ bool last_of_b(const TiledParams &p) const { return half == halves - 1 || mt + 1 >= p.tiles_m; }
+    // no later tile of this CTA uses this half's M-side operand
+    __device__ __forceinline__ bool last_for_a(const TiledParams &p) const { return nt + 1 == p.tiles_n || left <= halves; }
+    // at a tile with new_a: how often this tile's operand buffer has been filled before
+    __device__ __forceinline__ int a_before() const { return halves == 1 ? (an0 >> 1) : (half ? an1 : an0); }
+    __device__ __forceinline__ SkinnyWork work(const TiledParams &p) const
+    {
+        SkinnyWork w;
+        w.h = h; w.mt = mt; w.nt = nt;
+        w.m0 = int64_t(mt) * SkinnyTile::BM;
+        w.n0 = int64_t(nt) * SkinnyTile::BN;
+        w.rows_valid = int(imin64(SkinnyTile::BM, p.M - w.m0));
+        w.cols_valid = int(imin64(SkinnyTile::BN, p.N - w.n0));
+        return w;
+    }
+};
 
 // What one thread keeps to write its row of the accumulators to D.  Thread `row` owns row `row` of every
 // tile (tensor-memory lane `row`).  Two ways to write:
@@ -185,8 +213,8 @@ struct SkinnyStore {
     float alpha, beta;
     bool vecn, dreg;
     int row, lane;
-    int64_t ro, ro_next, co_next[4];
-    bool row_ok, row_ok_next;
+    int64_t ro0, ro1, ro_next, co_next[4];           // row offsets of the two halves' strips
+    bool ok0, ok1, row_ok_next;
 
     __device__ __forceinline__ void init(const TiledParams &p, int row_, int lane_)
     {
@@ -195,10 +223,10 @@ struct SkinnyStore {
         alpha = float(p.alpha[0]); beta = float(p.beta[0]);
         vecn = p.skinny_vec_n == 4; dreg = p.skinny_d_regular != 0;
         row = row_; lane = lane_;
-        ro = ro_next = 0; row_ok = row_ok_next = false;
+        ro0 = ro1 = ro_next = 0; ok0 = ok1 = row_ok_next = false;
         co_next[0] = co_next[1] = co_next[2] = co_next[3] = 0;
     }
-    // start fetching what tile wk needs; `strip_start`: wk is the first tile of a strip for this CTA
+    // start fetching what tile wk needs; `strip_start`: wk is the first tile of its half's strip for this CTA
     __device__ __forceinline__ void fetch(const TiledParams &p, const SkinnyWork &wk, bool strip_start)
     {
         if (strip_start) {
@@ -214,12 +242,21 @@ struct SkinnyStore {
             for (int c = 0; c < 4; ++c) co_next[c] = (c * 32 + lane < wk.cols_valid) ? p.offD_n[wk.n0 + c * 32 + lane] : 0;
         }
     }
+    // the strip of half `half` starts: what fetch() brought is its row offset
+    __device__ __forceinline__ void take_rows(int half)
+    {
+        if (half) { ro1 = ro_next; ok1 = row_ok_next; } else { ro0 = ro_next; ok0 = row_ok_next; }
+    }
     // Columns [c_begin, c_end) (multiples of 32) of the accumulator at `tacc` (this warp's lane quarter)
     // -> D.  `co` = the column offsets fetched for this tile.  Arrives on `done_bar` as soon as the
     // columns are in registers.
-    __device__ __forceinline__ void tile(const TiledParams &p, const SkinnyWork &w, unsigned tacc, int c_begin, int c_end,
+    __device__ __forceinline__ void tile(const TiledParams &p, const SkinnyWork &w, int half, unsigned tacc, int c_begin, int c_end,
                                          unsigned done_bar, const int64_t (&co)[4])
     {
+        const int64_t ro = half ? ro1 : ro0;
+        const bool row_ok = half ? ok1 : ok0;
+        const bool lean = vecn && dreg && !p.use_c && w.rows_valid == SkinnyTile::BM && w.cols_valid == SkinnyTile::BN;
+        (void)lean;
 #pragma unroll 1
         for (int c0 = c_begin; c0 < c_end; c0 += 32) {       // rolled: keeps the code small
             unsigned r[32];
@@ -231,6 +268,18 @@ struct SkinnyStore {
                 mbar_arrive(done_bar);
             }
             const int cols_here = w.cols_valid - c0;         // valid columns from c0 on (may be <= 0)
+#ifndef BTC_CHECK_OFFSETS
+            if (lean) {
+                // whole tile, regular columns, no C: nothing to decide per store
+                float *base = D + (ro + co[0]);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<float4 *>(base + p.skinny_col_rel[c0 + 4 * q]) =
+                        make_float4(alpha * __uint_as_float(r[4 * q]), alpha * __uint_as_float(r[4 * q + 1]),
+                                    alpha * __uint_as_float(r[4 * q + 2]), alpha * __uint_as_float(r[4 * q + 3]));
+                continue;
+            }
+#endif
             if (vecn) {
                 int64_t off[8];
 #pragma unroll
@@ -306,7 +355,9 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
     const int K = int(p.K);
     const int ksteps = (K + 7) / 8, kp = 8 * ksteps;                     // tensor-core steps of 8 k; k padded with zeros
     const int pieces = 32 * kp;                                         // 16-byte pieces of an operand tile in use
-    const int64_t total = int64_t(p.tiles_m) * p.tiles_n * p.Bt;
+    // pairs of tile rows share their N-side tiles when that leaves a pair or more for every CTA
+    const int halves = (p.tiles_m >= 2 && int64_t((p.tiles_m + 1) / 2) * p.tiles_n * p.Bt >= int64_t(gridDim.x)) ? 2 : 1;
+    const int64_t total = int64_t((p.tiles_m + halves - 1) / halves) * p.tiles_n * p.Bt;      // pairs
     const int64_t t0 = total * blockIdx.x / gridDim.x, t1 = total * (blockIdx.x + 1) / gridDim.x;
 
     // ---- set-up: k offsets, barriers, tensor memory ----
@@ -314,16 +365,9 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         koffA[i] = i < K ? p.offA_k[i] : 0;
         koffB[i] = i < K ? p.offB_k[i] : 0;
     }
-    for (int e = tid; e < pieces; e += T::THREADS) {
-        int row, k;
-        unsigned code = p.skinny_orderA[e];
-        skinny_a_pos(p.dirA, code, row, k);
-        int64_t rel = (row < p.M && k < K) ? p.offA_m[row] - p.offA_m[0] + p.offA_k[k] : 0;
-        pieceA[e] = code | (unsigned(k < K) << 11) | (unsigned(int(rel / 4)) << 12);
-        code = p.skinny_orderB[e];
-        skinny_b_pos(p.dirB, code, row, k);
-        rel = (row < p.N && k < K) ? p.offB_n[row] - p.offB_n[0] + p.offB_k[k] : 0;
-        pieceB[e] = code | (unsigned(k < K) << 11) | (unsigned(int(rel / 4)) << 12);
+    for (int e = tid; e < pieces; e += T::THREADS) {      // the piece tables, as the host prepared them
+        pieceA[e] = p.skinny_orderA[e];
+        pieceB[e] = p.skinny_orderB[e];
     }
     if (tid == 0) {
         mbar_init(a_full, T::GROUP_THREADS);
@@ -359,195 +403,173 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         // ------------------------------------------------------------- epilogue (first half of the columns)
         SkinnyStore st;
         st.init(p, tid, lane);
-        SkinnyWork w = skinny_work_at(p, t0);
-        if (t0 < t1) st.fetch(p, w, true);
-        long long t_wait = 0, t_work = 0;
-        (void)t_wait; (void)t_work;
-        BTC_PHASE_BEGIN();
+        SkinnyIter it;
+        it.start(p, halves, t0, t1);
+        if (it.valid) st.fetch(p, it.work(p), true);
 #pragma unroll 1
-        for (int64_t t = t0; t < t1; ++t) {
-            const int i = int(t - t0), buf = i & 1;
-            const SkinnyWork wn = skinny_work_next(p, w);
-            if (t == t0 || w.nt == 0) { st.ro = st.ro_next; st.row_ok = st.row_ok_next; }
+        while (it.valid) {
+            const int i = it.i, buf = i & 1, half = it.half;
+            const SkinnyWork w = it.work(p);
+            if (it.new_a) st.take_rows(half);
             int64_t co[4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) co[c] = st.co_next[c];
-            if (t + 1 < t1) st.fetch(p, wn, wn.nt == 0);
-            BTC_PHASE_END(t_work);
+            it.advance(p);
+            if (it.valid) st.fetch(p, it.work(p), it.new_a);
             if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit)) break;
-            BTC_PHASE_END(t_wait);
-            BTC_EVENT(p, tid == 0, 6, i);
             tc_fence_after();
-            st.tile(p, w, tmem_base + (unsigned(warp * 32) << 16) + unsigned(buf * T::ACC_COLS), 0, T::SPLIT_COL, acc_empty0 + 8u * buf, co);
-            BTC_EVENT(p, tid == 0, 7, i);
-            w = wn;
+            st.tile(p, w, half, tmem_base + (unsigned(warp * 32) << 16) + unsigned(buf * T::ACC_COLS), 0, T::SPLIT_COL, acc_empty0 + 8u * buf, co);
         }
-        BTC_PHASE_END(t_work);
-        BTC_PHASE_STORE(p, tid == 0, 0, t_wait);
-        BTC_PHASE_STORE(p, tid == 0, 1, t_work);
     } else if (warp < T::EPILOGUE_WARPS + T::CONVERTER_WARPS) {
         // ------------------------------------------------------------- converters
         const int ct = tid - 32 * T::EPILOGUE_WARPS;             // row of the M-side tile = tensor-memory lane
-        int sidx = -1;
-        long long t_wait = 0, t_work = 0;
-        (void)t_wait; (void)t_work;
         // Between conversions these warps also write the second half of the columns of the tile before
         // (its accumulator is complete by then), which doubles the warps that keep stores in flight.
         SkinnyStore st;
         st.init(p, ct, lane);
-        SkinnyWork w = skinny_work_at(p, t0), wprev = w;
+        SkinnyIter it;
+        it.start(p, halves, t0, t1);
+        SkinnyWork wprev = it.work(p);
+        int half_prev = 0, i_last = -1;
         int64_t co_prev[4] = {0, 0, 0, 0};
-        BTC_PHASE_BEGIN();
+        bool ok = true;
 #pragma unroll 1
-        for (int64_t t = t0; t < t1; ++t) {
-            const int i = int(t - t0), s = i & 1;
-            const bool new_strip = t == t0 || w.nt == 0;
-            st.fetch(p, w, new_strip);                // for this tile's store, one iteration from now
-            if (new_strip) {
-                ++sidx;
-                const int ab = sidx & 1;
-                if (!mbar_wait_bounded(a_full, unsigned(sidx) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)) break;
-                if (sidx >= 2 &&
-                    !mbar_wait_bounded(ta_empty0 + 8u * ab, unsigned((sidx >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit))
+        while (it.valid) {
+            const int i = it.i, half_now = it.half;
+            const SkinnyWork w = it.work(p);
+            const bool new_a = it.new_a;
+            st.fetch(p, w, new_a);                    // for this tile's store, one iteration from now
+            if (new_a) {
+                const int loads = it.an0 + it.an1, mine = it.a_before(), ab = it.abuf;
+                if (!(ok = mbar_wait_bounded(a_full, unsigned(loads) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit))) break;
+                // the operand buffer is free once the tensor core has finished the strip that used it before
+                if (mine >= 1 &&
+                    !(ok = mbar_wait_bounded(ta_empty0 + 8u * ab, unsigned(mine - 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)))
                     break;
                 tc_fence_after();
                 const unsigned ta = tmem_a0 + unsigned(ab * T::A_COLS) + (unsigned(ct & ~31) << 16);
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    if (half * 32 >= kp) break;
+                for (int kh = 0; kh < 2; ++kh) {
+                    if (kh * 32 >= kp) break;
                     float x[32];
                     if (p.dirA == 0) {
 #pragma unroll
                         for (int k = 0; k < 32; ++k)
-                            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x[k]) : "r"(araw + unsigned((half * 32 + k) * T::BM + ct) * 4u) : "memory");
+                            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x[k]) : "r"(araw + unsigned((kh * 32 + k) * T::BM + ct) * 4u) : "memory");
                     } else {
 #pragma unroll
                         for (int c = 0; c < 8; ++c)
                             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
                                          : "=f"(x[4 * c]), "=f"(x[4 * c + 1]), "=f"(x[4 * c + 2]), "=f"(x[4 * c + 3])
-                                         : "r"(araw + unsigned(ct) * 256u + (unsigned(((half * 8 + c) ^ ct) & 15) << 4)) : "memory");
+                                         : "r"(araw + unsigned(ct) * 256u + (unsigned(((kh * 8 + c) ^ ct) & 15) << 4)) : "memory");
                     }
-                    tmem_store32(ta + unsigned(half * 32), x);
+                    tmem_store32(ta + unsigned(kh * 32), x);
 #pragma unroll
                     for (int k = 0; k < 32; ++k) x[k] -= __uint_as_float(__float_as_uint(x[k]) & 0xffffe000u);
-                    tmem_store32(ta + unsigned(T::KMAX + half * 32), x);
+                    tmem_store32(ta + unsigned(T::KMAX + kh * 32), x);
                 }
                 tmem_store_wait();
                 tc_fence_before();
                 mbar_arrive(ta_full0 + 8u * ab);
                 mbar_arrive(a_empty);                 // the raw M-side buffer may be refilled
             }
-            BTC_PHASE_END(t_work);
-            const int r = i % T::RAW_STAGES;
-            if (!mbar_wait_bounded(raw_full0 + 8u * r, unsigned(i / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)) break;
-            // the tail stage is free once the tensor core has finished the tile two before this one
-            if (i >= 2 && !mbar_wait_bounded(lo_empty0 + 8u * s, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)) break;
-            BTC_PHASE_END(t_wait);
-            BTC_EVENT(p, ct == 0, 2, i);
-            // N side: position-independent pass; the raw stage is the head, the tail goes to the same
-            // position of the tail stage
-            const unsigned src = braw0 + unsigned(r) * T::B_BYTES + unsigned(ct) * 16u;
-            const unsigned dst = blo0 + unsigned(s) * T::B_BYTES + unsigned(ct) * 16u;
-            const int per = (kp <= 32 ? T::B_BLOCK_BYTES : T::B_BYTES) / 16 / T::GROUP_THREADS;   // 8 or 16 pieces per thread
-#pragma unroll
-            for (int i0 = 0; i0 < 16; i0 += 8) {
-                if (i0 >= per) break;
-                float x[8][4];
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                                 : "=f"(x[q][0]), "=f"(x[q][1]), "=f"(x[q][2]), "=f"(x[q][3]) : "r"(src + unsigned(i0 + q) * 2048u) : "memory");
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    float lo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) lo[e] = x[q][e] - __uint_as_float(__float_as_uint(x[q][e]) & 0xffffe000u);
-                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + unsigned(i0 + q) * 2048u), "f"(lo[0]), "f"(lo[1]), "f"(lo[2]), "f"(lo[3]) : "memory");
+            if (it.first_of_b()) {
+                const int bi = it.bi, r = bi % T::RAW_STAGES, s = bi & 1;
+                if (!(ok = mbar_wait_bounded(raw_full0 + 8u * r, unsigned(bi / T::RAW_STAGES) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit))) break;
+                // the tail stage is free once the tensor core has finished the tiles of the N-side tile two before
+                if (bi >= 2 && !(ok = mbar_wait_bounded(lo_empty0 + 8u * s, unsigned((bi >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit))) break;
+                // N side: position-independent pass; the raw stage is the head, the tail goes to the same
+                // position of the tail stage
+                const unsigned src = braw0 + unsigned(r) * T::B_BYTES + unsigned(ct) * 16u;
+                const unsigned dst = blo0 + unsigned(s) * T::B_BYTES + unsigned(ct) * 16u;
+                const int per = (kp <= 32 ? T::B_BLOCK_BYTES : T::B_BYTES) / 16 / T::GROUP_THREADS;   // 8 or 16 pieces per thread
+    #pragma unroll
+                for (int i0 = 0; i0 < 16; i0 += 8) {
+                    if (i0 >= per) break;
+                    float x[8][4];
+    #pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(x[q][0]), "=f"(x[q][1]), "=f"(x[q][2]), "=f"(x[q][3]) : "r"(src + unsigned(i0 + q) * 2048u) : "memory");
+    #pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        float lo[4];
+    #pragma unroll
+                        for (int e = 0; e < 4; ++e) lo[e] = x[q][e] - __uint_as_float(__float_as_uint(x[q][e]) & 0xffffe000u);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst + unsigned(i0 + q) * 2048u), "f"(lo[0]), "f"(lo[1]), "f"(lo[2]), "f"(lo[3]) : "memory");
+                    }
                 }
+                proxy_fence_async();                  // the tensor core reads both stages through the async proxy
+                mbar_arrive(lo_conv0 + 8u * s);
             }
-            proxy_fence_async();                      // the tensor core reads both stages through the async proxy
-            mbar_arrive(lo_conv0 + 8u * s);
-            BTC_EVENT(p, ct == 0, 3, i);
             if (i > 0) {
                 const int ip = i - 1, buf = ip & 1;
-                if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit)) break;
+                if (!(ok = mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit))) break;
                 tc_fence_after();
-                st.tile(p, wprev, tmem_base + (unsigned(ct & ~31) << 16) + unsigned(buf * T::ACC_COLS), T::SPLIT_COL, T::BN,
+                st.tile(p, wprev, half_prev, tmem_base + (unsigned(ct & ~31) << 16) + unsigned(buf * T::ACC_COLS), T::SPLIT_COL, T::BN,
                         acc_empty0 + 8u * buf, co_prev);
             }
             // what was fetched at the top of this iteration belongs to this tile: keep it for the next iteration
 #pragma unroll
             for (int c = 0; c < 4; ++c) co_prev[c] = st.co_next[c];
-            if (new_strip) { st.ro = st.ro_next; st.row_ok = st.row_ok_next; }
-            wprev = w;
-            w = skinny_work_next(p, w);
+            if (new_a) st.take_rows(half_now);
+            wprev = w; half_prev = half_now; i_last = i;
+            it.advance(p);
         }
-        if (t1 > t0 && !*abort_flag) {                // the last tile's second half
-            const int ip = int(t1 - t0) - 1, buf = ip & 1;
-            if (mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(ip >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit)) {
+        if (ok && i_last >= 0 && !*abort_flag) {      // the last tile's second half of the columns
+            const int buf = i_last & 1;
+            if (mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(i_last >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit)) {
                 tc_fence_after();
-                st.tile(p, wprev, tmem_base + (unsigned(ct & ~31) << 16) + unsigned(buf * T::ACC_COLS), T::SPLIT_COL, T::BN,
+                st.tile(p, wprev, half_prev, tmem_base + (unsigned(ct & ~31) << 16) + unsigned(buf * T::ACC_COLS), T::SPLIT_COL, T::BN,
                         acc_empty0 + 8u * buf, co_prev);
             }
         }
-        BTC_PHASE_END(t_work);
-        BTC_PHASE_STORE(p, ct == 0, 2, t_wait);
-        BTC_PHASE_STORE(p, ct == 0, 3, t_work);
     } else if (warp < T::MMA_WARP) {
         // ------------------------------------------------------------- loaders
         const int pt = tid - 32 * (T::EPILOGUE_WARPS + T::CONVERTER_WARPS);
         const float *A = static_cast<const float *>(p.A), *B = static_cast<const float *>(p.B);
-        int sidx = -1;
-        long long t_wait = 0, t_work = 0;
-        (void)t_wait; (void)t_work;
         // Regular operands: a tile is addressed by its first row's offset alone, fetched one tile ahead
         // (every thread reads the same table entry).  Otherwise the threads build the tile's row and
         // column offset arrays in shared memory, one entry each, also fetched one tile ahead.
         const bool regular = p.skinny_regular != 0;
-        SkinnyWork w = skinny_work_at(p, t0);
+        SkinnyIter it;
+        it.start(p, halves, t0, t1);
         int64_t next_row = 0, next_col = 0;
-        auto fetch = [&](const SkinnyWork &wk) {
+        auto fetch = [&](const SkinnyIter &at) {
+            const SkinnyWork wk = at.work(p);
             const int r = regular ? 0 : pt;
-            next_row = r < wk.rows_valid ? p.offA_m[wk.m0 + r] + p.offA_h[wk.h] : 0;
-            next_col = r < wk.cols_valid ? p.offB_n[wk.n0 + r] + p.offB_h[wk.h] : 0;
+            if (at.new_a) next_row = r < wk.rows_valid ? p.offA_m[wk.m0 + r] + p.offA_h[wk.h] : 0;
+            if (at.first_of_b()) next_col = r < wk.cols_valid ? p.offB_n[wk.n0 + r] + p.offB_h[wk.h] : 0;
         };
-        if (t0 < t1) fetch(w);
-        BTC_PHASE_BEGIN();
+        if (it.valid) fetch(it);
 #pragma unroll 1
-        for (int64_t t = t0; t < t1; ++t) {
-            const int i = int(t - t0), s = i & 1;
-            const bool new_strip = t == t0 || w.nt == 0;
-            if (new_strip) ++sidx;
-            const int r = i % T::RAW_STAGES;
-            int64_t *rA = rowA + (sidx & 1) * T::BM, *cB = colB + r * T::BN;
+        while (it.valid) {
+            const int i = it.i, bi = it.bi, r = bi % T::RAW_STAGES, loads = it.an0 + it.an1;
+            const bool new_a = it.new_a, new_b = it.first_of_b();
+            const SkinnyWork w = it.work(p);
+            int64_t *rA = rowA + (loads & 1) * T::BM, *cB = colB + r * T::BN;
             const int64_t row_base = next_row, col_base = next_col;
             if (!regular) {
-                if (new_strip) rA[pt] = next_row;
-                cB[pt] = next_col;
+                if (new_a) rA[pt] = next_row;
+                if (new_b) cB[pt] = next_col;
                 if (!umma_group_sync(loader_sync, unsigned(i) & 1u, abort_flag, p.error_word, p.poll_limit)) break;
             }
-            const SkinnyWork wn = skinny_work_next(p, w);
-            if (t + 1 < t1) fetch(wn);
-            if (new_strip) {
-                if (sidx > 0 && !mbar_wait_bounded(a_empty, unsigned(sidx - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
+            it.advance(p);
+            if (it.valid) fetch(it);
+            if (new_a) {
+                if (loads > 0 && !mbar_wait_bounded(a_empty, unsigned(loads - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
                 if (regular) skinny_load_tile_regular<true>(araw, A, row_base, pieceA, pieces, p.dirA, w.rows_valid, pt, p.spans, 0);
                 else skinny_load_tile<true>(araw, A, rA, koffA, pieceA, pieces, p.dirA, w.rows_valid, pt, p.spans, 0);
                 mbar_arrive_on_copies(a_full);
             }
-            BTC_PHASE_END(t_work);
-            if (i >= T::RAW_STAGES &&
-                !mbar_wait_bounded(raw_empty0 + 8u * r, unsigned(i / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
-            BTC_PHASE_END(t_wait);
-            BTC_EVENT(p, pt == 0, 0, i);
-            if (regular) skinny_load_tile_regular<false>(braw0 + unsigned(r) * T::B_BYTES, B, col_base, pieceB, pieces, p.dirB, w.cols_valid, pt, p.spans, 1);
-            else skinny_load_tile<false>(braw0 + unsigned(r) * T::B_BYTES, B, cB, koffB, pieceB, pieces, p.dirB, w.cols_valid, pt, p.spans, 1);
-            mbar_arrive_on_copies(raw_full0 + 8u * r);
-            BTC_EVENT(p, pt == 0, 1, i);
-            w = wn;
+            if (new_b) {
+                if (bi >= T::RAW_STAGES &&
+                    !mbar_wait_bounded(raw_empty0 + 8u * r, unsigned(bi / T::RAW_STAGES - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
+                if (regular) skinny_load_tile_regular<false>(braw0 + unsigned(r) * T::B_BYTES, B, col_base, pieceB, pieces, p.dirB, w.cols_valid, pt, p.spans, 1);
+                else skinny_load_tile<false>(braw0 + unsigned(r) * T::B_BYTES, B, cB, koffB, pieceB, pieces, p.dirB, w.cols_valid, pt, p.spans, 1);
+                mbar_arrive_on_copies(raw_full0 + 8u * r);
+            }
         }
-        BTC_PHASE_END(t_work);
-        BTC_PHASE_STORE(p, pt == 0, 4, t_wait);
-        BTC_PHASE_STORE(p, pt == 0, 5, t_work);
         cp_async_wait_all();
     } else {
         // ------------------------------------------------------------- MMA warp
@@ -558,31 +580,21 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         const unsigned b_lay = b_mn ? 1u : 2u, b_lbo = b_mn ? 512u : 16u, b_sbo = b_mn ? 16u * T::BN : 1024u;
         const unsigned b_step = b_mn ? 32u * T::BN : 32u;        // 8 k: two k-atoms, or 32 bytes of a row
         const bool leader = elect_one();
-        int sidx = -1;
-        long long t_acc = 0, t_conv = 0, t_issue = 0;
-        (void)t_acc; (void)t_conv; (void)t_issue;
-        int nt = skinny_work_at(p, t0).nt;
-        BTC_PHASE_BEGIN();
+        SkinnyIter it;
+        it.start(p, halves, t0, t1);
 #pragma unroll 1
-        for (int64_t t = t0; t < t1; ++t) {
-            const int i = int(t - t0), s = i & 1, buf = i & 1;
-            const bool new_strip = t == t0 || nt == 0;
-            if (++nt == p.tiles_n) nt = 0;           // now the column of the next tile
-            if (new_strip) {
-                ++sidx;
-                if (!mbar_wait_bounded(ta_full0 + 8u * (sidx & 1), unsigned(sidx >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
-            }
-            BTC_PHASE_END(t_issue);
+        for (; it.valid; it.advance(p)) {
+            const int i = it.i, buf = i & 1, bi = it.bi, r = bi % T::RAW_STAGES, s = bi & 1;
+            if (it.new_a &&
+                !mbar_wait_bounded(ta_full0 + 8u * unsigned(it.abuf), unsigned(it.a_before()) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
             if (i >= 2 && !mbar_wait_bounded(acc_empty0 + 8u * buf, unsigned((i >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
-            BTC_PHASE_END(t_acc);
-            if (!mbar_wait_bounded(lo_conv0 + 8u * s, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
-            BTC_PHASE_END(t_conv);
-            BTC_EVENT(p, lane == 0, 4, i);
+            if (it.first_of_b() &&
+                !mbar_wait_bounded(lo_conv0 + 8u * s, unsigned(bi >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyMma, p.poll_limit)) break;
             tc_fence_after();
             if (leader) {
                 const unsigned tacc = tmem_base + unsigned(buf * T::ACC_COLS);
-                const unsigned ta = tmem_a0 + unsigned((sidx & 1) * T::A_COLS);      // head columns; tail KMAX further
-                const unsigned b_hi = braw0 + unsigned(i % T::RAW_STAGES) * T::B_BYTES, b_lo = blo0 + unsigned(s) * T::B_BYTES;
+                const unsigned ta = tmem_a0 + unsigned(it.abuf * T::A_COLS);            // head columns; tail KMAX further
+                const unsigned b_hi = braw0 + unsigned(r) * T::B_BYTES, b_lo = blo0 + unsigned(s) * T::B_BYTES;
 #pragma unroll 1
                 for (int j = 0; j < ksteps; ++j) {
                     const unsigned at = unsigned(j >> 2) * T::B_BLOCK_BYTES + unsigned(j & 3) * b_step;
@@ -592,16 +604,15 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
                     umma_tf32_ts(tacc, ta + unsigned(8 * j), dbl, idesc, 1u);
                     umma_tf32_ts(tacc, ta + unsigned(8 * j), dbh, idesc, 1u);
                 }
-                umma_commit(raw_empty0 + 8u * unsigned(i % T::RAW_STAGES));       // fire when these MMAs have read the stages
-                umma_commit(lo_empty0 + 8u * s);
+                if (it.last_of_b(p)) {                // fire when the MMAs so far have read the stages
+                    umma_commit(raw_empty0 + 8u * unsigned(r));
+                    umma_commit(lo_empty0 + 8u * s);
+                }
                 umma_commit(acc_full0 + 8u * buf);
-                if (t + 1 == t1 || nt == 0) umma_commit(ta_empty0 + 8u * (sidx & 1));
+                if (it.last_for_a(p)) umma_commit(ta_empty0 + 8u * unsigned(it.abuf));
             }
             __syncwarp();
-            BTC_EVENT(p, lane == 0, 5, i);
         }
-        BTC_PHASE_STORE(p, lane == 0, 6, t_acc);
-        BTC_PHASE_STORE(p, lane == 0, 7, t_conv);
         tc_fence_before();
     }
 
