@@ -662,6 +662,33 @@ cudaError_t launch_isolated_sum(const IsolatedSum &s, const void *src, void *dst
     p.total_keep = s.total_keep; p.total_iso = s.total_iso;
     for (int i = 0; i < p.nk; ++i) { p.ext_k[i] = s.keep_ext[size_t(i)]; p.str_k[i] = s.keep_str[size_t(i)]; }
     for (int i = 0; i < p.ni; ++i) { p.ext_i[i] = s.iso_ext[size_t(i)]; p.str_i[i] = s.iso_str[size_t(i)]; }
+    // contiguous isolated index of whole 16-byte vectors, kept strides and base aligned alike: lanes share
+    // result elements and read vectors
+    constexpr int64_t V = 16 / int64_t(sizeof(R) * (CPLX ? 2 : 1));
+    bool vec = s.iso_ext.size() == 1 && s.iso_str[0] == 1 && s.iso_ext[0] % V == 0 && reinterpret_cast<uintptr_t>(src) % 16 == 0;
+    for (size_t i = 0; vec && i < s.keep_str.size(); ++i) vec = s.keep_str[i] % V == 0;
+    if (vec) {
+        const int64_t nvec = s.iso_ext[0] / V;
+        const int log_l = nvec >= 8 ? 3 : nvec >= 4 ? 2 : nvec >= 2 ? 1 : 0;
+        int64_t blocks = ((s.total_keep << log_l) + 255) / 256;
+        const int64_t cap = int64_t(sm_count) * 32;
+        if (blocks > cap) blocks = cap;
+        if (blocks < 1) blocks = 1;
+        const bool narrow = s.total_keep < (int64_t(1) << 31);
+#define BTC_ISO_VEC(LOG_L)                                                                                     \
+        do {                                                                                                   \
+            if (narrow) isolated_sum_vector_kernel<R, CPLX, LOG_L, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);   \
+            else isolated_sum_vector_kernel<R, CPLX, LOG_L, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);           \
+        } while (0)
+        switch (log_l) {
+        case 3: BTC_ISO_VEC(3); break;
+        case 2: BTC_ISO_VEC(2); break;
+        case 1: BTC_ISO_VEC(1); break;
+        default: BTC_ISO_VEC(0); break;
+        }
+#undef BTC_ISO_VEC
+        return cudaGetLastError();
+    }
     const int lanes = s.lanes_over_iso ? 32 : 1;
     int64_t blocks = (s.total_keep * lanes + 255) / 256;
     const int64_t cap = int64_t(sm_count) * 32;

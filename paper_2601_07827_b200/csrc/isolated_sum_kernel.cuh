@@ -3,7 +3,8 @@
 // A bandwidth-bound pass: X is read once through its strides, X' is written densely (kept labels
 // in order of increasing |stride| in X, so consecutive threads read and write neighbouring
 // elements).  LANES = 1: one thread per element of X'.  LANES = 32: one warp per element, lanes
-// striding over the isolated index, for tensors whose isolated label is the contiguous one.
+// striding over the isolated index, for tensors whose isolated label is the contiguous one; where that
+// label's runs are whole 16-byte vectors, the vector kernel at the end of this file runs instead.
 // Sums are kept in double (pairs for complex) for every element type; conjugation commutes with
 // the sum and stays with the contraction.
 #pragma once
@@ -86,6 +87,75 @@ __global__ void __launch_bounds__(256) isolated_sum_kernel(const IsolatedSumPara
             }
             const int64_t e = e0 + j * ngroups;
             if (lane == 0 && e < p.total_keep) {
+                dst[NC * e] = R(acc_r[j]);
+                if (CPLX) dst[NC * e + (NC - 1)] = R(acc_i[j]);
+            }
+        }
+    }
+}
+
+// The isolated index is the contiguous one (stride 1, a multiple of 16 bytes long, every kept stride a
+// multiple of 16 bytes too): L = 2^LOG_L neighbouring lanes share a result element, each lane reads
+// 16-byte vectors L vectors apart (the L lanes together one run of 16 L bytes), sums its own vectors
+// in registers and the lanes finish with LOG_L shuffle steps.  E = 2 result elements per lane group are in
+// flight at a time (measured: 4 or 8 are slower, the reads then come from more places at once).
+template <typename R, bool CPLX, int LOG_L, typename I>
+__global__ void __launch_bounds__(256) isolated_sum_vector_kernel(const IsolatedSumParams p)
+{
+    constexpr int NC = CPLX ? 2 : 1, L = 1 << LOG_L;
+    constexpr int W = 16 / int(sizeof(R));             // words of type R per vector
+    constexpr int V = W / NC;                          // elements per vector
+    constexpr int E = 2, U = 2;
+    union Pack { uint4 raw; R w[W]; };
+    const R *src = static_cast<const R *>(p.src);
+    R *dst = static_cast<R *>(p.dst);
+    const int sub = int(threadIdx.x) & (L - 1);
+    const int64_t group = (int64_t(blockIdx.x) * blockDim.x + threadIdx.x) >> LOG_L;
+    const int64_t ngroups = (int64_t(gridDim.x) * blockDim.x) >> LOG_L;
+    const int64_t nvec = p.total_iso / V;
+    // every lane of a warp runs the same number of passes (the shuffles below need all of them)
+    const int64_t group_w = (int64_t(blockIdx.x) * blockDim.x + (threadIdx.x & ~31u)) >> LOG_L;      // the warp's first group
+    for (int64_t pass = 0; group_w + pass < p.total_keep; pass += ngroups * E) {
+        const int64_t e0 = group + pass;
+        int64_t base[E];
+        bool live[E];
+        double acc_r[E], acc_i[E];
+#pragma unroll
+        for (int j = 0; j < E; ++j) {
+            const int64_t e = e0 + j * ngroups;
+            live[j] = e < p.total_keep;
+            base[j] = live[j] ? decode_offset<I>(I(e), p.nk, p.ext_k, p.str_k) : 0;
+            acc_r[j] = acc_i[j] = 0.0;
+        }
+        for (int64_t v0 = sub; v0 < nvec; v0 += int64_t(U) * L) {
+            Pack x[E][U];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int j = 0; j < E; ++j) {
+                    const int64_t v = v0 + int64_t(u) * L;
+                    x[j][u].raw = make_uint4(0, 0, 0, 0);
+                    if (live[j] && v < nvec) x[j][u].raw = *reinterpret_cast<const uint4 *>(src + NC * (base[j] + v * V));
+                }
+#pragma unroll
+            for (int j = 0; j < E; ++j)
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int w = 0; w < W; ++w) {
+                        if (CPLX && (w & 1)) acc_i[j] += double(x[j][u].w[w]);
+                        else acc_r[j] += double(x[j][u].w[w]);
+                    }
+        }
+#pragma unroll
+        for (int j = 0; j < E; ++j) {
+#pragma unroll
+            for (int o = L / 2; o > 0; o >>= 1) {
+                acc_r[j] += __shfl_xor_sync(0xffffffffu, acc_r[j], o);
+                if (CPLX) acc_i[j] += __shfl_xor_sync(0xffffffffu, acc_i[j], o);
+            }
+            const int64_t e = e0 + j * ngroups;
+            if (sub == 0 && e < p.total_keep) {
                 dst[NC * e] = R(acc_r[j]);
                 if (CPLX) dst[NC * e + (NC - 1)] = R(acc_i[j]);
             }
