@@ -164,6 +164,57 @@ __device__ __forceinline__ void store_tile_image(const TiledParams &p, const Til
     }
 }
 
+// Split-K inside a cluster: every CTA of the cluster has parked the image of its partial tile at the
+// same place of its shared memory.  CTA `rank` finishes the rank-th share of the tile's elements: it
+// adds the partial values of all CTAs in rank order (so the result does not depend on scheduling; the
+// same order as splitk_reduce_kernel) and writes D.  The caller puts a cluster barrier before and after.
+template <typename Acc, int W, int BM, int BN, int NT>
+__device__ __forceinline__ void splitk_finish_cluster(const TiledParams &p, const TileCoords &tc, const Acc *image,
+                                                      const int64_t *rowD, const int64_t *colD, int t)
+{
+    static_assert(sizeof(Acc) == 8, "distributed shared memory is read in 8-byte words");
+    constexpr int P = ImagePitch<BM>::value;
+    const int split = p.split_k;
+    const int share = (BM * BN + split - 1) / split;
+    const int begin = tc.ks * share, end = begin + share < BM * BN ? begin + share : BM * BN;
+    const unsigned image0 = static_cast<unsigned>(__cvta_generic_to_shared(image));
+    constexpr int UE = 4;
+#pragma unroll 1
+    for (int base = begin + t; base < end; base += UE * NT) {
+        Acc s_r[UE], s_i[UE];
+#pragma unroll
+        for (int u = 0; u < UE; ++u) s_r[u] = s_i[u] = Acc(0);
+        for (int r = 0; r < split; ++r) {
+            Acc v_r[UE], v_i[UE];
+#pragma unroll
+            for (int u = 0; u < UE; ++u) {
+                const int idx = base + u * NT;
+                const int row = idx % BM, col = idx / BM;
+                const unsigned a = cluster_map(image0 + unsigned(col * P + row) * unsigned(W * 8), unsigned(r));
+                v_r[u] = idx < end ? cluster_load_f64(a) : Acc(0);
+                v_i[u] = (W == 2 && idx < end) ? cluster_load_f64(a + 8u) : Acc(0);
+            }
+#pragma unroll
+            for (int u = 0; u < UE; ++u) { s_r[u] += v_r[u]; s_i[u] += v_i[u]; }
+        }
+#pragma unroll
+        for (int u = 0; u < UE; ++u) {
+            const int idx = base + u * NT;
+            const int row = idx % BM, col = idx / BM;
+            if (idx >= end || row >= tc.rows_valid || col >= tc.cols_valid) continue;
+            const int64_t off = rowD[row] + colD[col];
+            if (!BTC_IN_SPAN(p.spans, 2, off, 1)) continue;
+            Acc c_r = 0, c_i = 0;
+            if (p.use_c) {
+                const Acc *cp = static_cast<const Acc *>(p.C) + off * W;
+                c_r = cp[0];
+                if (W == 2) c_i = cp[W - 1];
+            }
+            finish_element<Acc, W>(p, off, s_r[u], s_i[u], c_r, c_i);
+        }
+    }
+}
+
 // Second pass of split-K for every tiled kernel of one element type: scratch holds, per (batch,
 // slice, tile), the dense image [column][row][word] of raw partial sums.  One CTA per (tile,
 // batch); slices are added in increasing order, so the result does not depend on scheduling.

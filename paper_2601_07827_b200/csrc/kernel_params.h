@@ -92,6 +92,10 @@ struct TiledParams {
     int32_t use_c;
     double alpha[2], beta[2];
     void *partials;                   // split-K scratch (workspace), or nullptr
+    // 1 (fp64 kernels, split_k = 2, 4 or 8): the CTAs of one tile's k slices form a thread-block cluster
+    // (slice = rank in the cluster, so the work list runs slice-fastest) and add their partial tiles through
+    // distributed shared memory: one launch, no scratch
+    int32_t cluster_split;
     int32_t *error_word;              // device word; set non-zero when a bounded wait gave up
     uint32_t poll_limit;              // polls after which a device-side wait gives up
     OffsetSpans spans;                // what the offset checks of debug builds compare with

@@ -74,6 +74,26 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity,
     return false;
 }
 
+// Cluster-wide barrier of all threads that have not exited (release / acquire: shared-memory writes
+// made before it are visible to the other CTAs of the cluster after it).
+__device__ __forceinline__ void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// the address of this CTA's shared-memory location `addr` in the CTA of rank `rank` of the cluster
+__device__ __forceinline__ unsigned cluster_map(unsigned addr, unsigned rank)
+{
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ double cluster_load_f64(unsigned addr)
+{
+    double v;
+    asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(v) : "r"(addr) : "memory");
+    return v;
+}
+
 // Self-test of the bounded wait: every thread waits on an mbarrier that nobody arrives on, with a
 // small poll limit.  The wait must give up, raise the abort flag and write the error word; the
 // kernel then returns normally, so the context stays usable.  (A template only so that the
@@ -174,14 +194,15 @@ struct TileCoords {
     int rows_valid, cols_valid, num_kt;
 };
 
-// `work` enumerates (tile, k slice, batch), tile fastest
+// `work` enumerates (tile, k slice, batch), tile fastest -- or, where the slices of a tile form a
+// cluster, (k slice, tile, batch), slice fastest
 template <int BM, int BN, int BK, typename Params>
 __device__ __forceinline__ TileCoords tile_coords_at(const Params &p, int64_t work)
 {
     TileCoords c;
     const int tiles = p.tiles_m * p.tiles_n;
-    c.tile = int(work % tiles);
-    c.ks = int((work / tiles) % p.split_k);
+    c.tile = p.cluster_split ? int((work / p.split_k) % tiles) : int(work % tiles);
+    c.ks = p.cluster_split ? int(work % p.split_k) : int((work / tiles) % p.split_k);
     c.h = work / (int64_t(tiles) * p.split_k);
     const int tile_m = p.raster_n_fast ? c.tile / p.tiles_n : c.tile % p.tiles_m;
     const int tile_n = p.raster_n_fast ? c.tile % p.tiles_n : c.tile / p.tiles_m;

@@ -263,6 +263,16 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     }
     consumer_barrier<T::CONSUMER_THREADS>();
     if (ctid == 0) BTC_STAMP(p, 6);                     // image parked
+    if (p.cluster_split) {
+        // the k slices of this tile are the CTAs of this cluster: add them up through distributed shared
+        // memory, every CTA a share of the tile.  (Producer warps have returned; a CTA that gave up has
+        // returned too and left the error word, which keeps D untouched as the two-kernel path does.)
+        cluster_barrier();
+        if (!(p.error_word && *static_cast<volatile int32_t *>(p.error_word) != 0))
+            splitk_finish_cluster<double, W, T::BM, T::BN, T::CONSUMER_THREADS>(p, tc, image, rowD, colD, ctid);
+        cluster_barrier();                              // nobody leaves while its image is being read
+        return;
+    }
     store_tile_image<double, W, T::BM, T::BN, T::CONSUMER_THREADS>(p, tc, image, rowD, colD, ctid);
     if (ctid == 0) BTC_STAMP(p, 7);                     // stores issued
 }
