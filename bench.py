@@ -141,6 +141,8 @@ def parse():
     ap.add_argument("--workload", default="all", help="one workload name, or 'all': the headline workload plus per_config")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--results-from", default="", help="write RESULTS.md from a file holding a JSON line of the default run (no GPU needed)")
+    ap.add_argument("--results-out", default=os.path.join(os.path.dirname(os.path.abspath(__file__)), "RESULTS.md"))
     ap.add_argument("--variant", type=int, default=-1, help="force a tile variant (tuning runs)")
     ap.add_argument("--batched", type=int, default=0,
                     help="one step = one btc_execute_batched call over this many distinct (A, B, D) buffer sets")
@@ -495,7 +497,7 @@ def per_config(args, torch, api, inputs, handle):
             ("single", "cfg3_f32_batched_permuted", False), ("single", "cfg4_c64_conj", False), ("single", "cfg4c_c32_conj", False),
             ("single", "cfg5_f32_tensor_network", True), ("batched", "cfg5_f32_tensor_network", 64),
             ("single", "cfg5b_f32_tensor_network_rev", True), ("batched", "cfg5b_f32_tensor_network_rev", 64),
-            ("single", "cfg6_f64_case4_isolated", False), ("single", "cfg7_f32_outer_product", False)] + [("ew", name, None) for name in E]
+            ("single", "cfg6_f64_case4_isolated", False), ("single", "cfg6b_f64_case4_isolated_fast", False), ("single", "cfg7_f32_outer_product", False)] + [("ew", name, None) for name in E]
     for kind, name, arg in plan:
         try:
             if kind == "single":
@@ -511,8 +513,62 @@ def per_config(args, torch, api, inputs, handle):
     return out
 
 
+def write_results(src, dst):
+    """RESULTS.md from the JSON line of a default run: every figure in the table is a field of that line."""
+    with open(src) as f:
+        lines = [l for l in f.read().splitlines() if l.startswith("{")]
+    d = json.loads(lines[-1])
+    pk, roof, e2e, cpu = d.get("peaks", {}), d["roofline"], d["e2e"], d.get("cpu_baseline") or {}
+
+    def frac(r):
+        if not r or r.get("frac") is None:
+            return "-"
+        names = {"hbm": "HBM copy bandwidth", "tensor": "tensor-pipe peak", "alu": "FMA-pipe peak"}
+        return f"{r['frac']:.2f} of {names.get(r['bound'], r['bound'])} ({r['peak']:.4g} {r['unit']})"
+
+    out = []
+    out.append("# RESULTS - one B200, CUDA events, operands resident in HBM")
+    out.append("")
+    out.append(f"Written by `python bench.py --results-from <file>` from the JSON line of one default run (`python bench.py`,")
+    out.append(f"{d['steps']} timed steps after {d['warmup']} warm-up steps for the headline workload); nothing here is typed by hand.")
+    out.append(f"SM clock while timing: {d['clocks'].get('sm_mhz')} MHz of {d['clocks'].get('sm_max_mhz')}, throttle reasons {d['clocks'].get('reasons')}"
+               + (f"; other workloads {d['per_config_clocks'].get('sm_mhz')} MHz, reasons {d['per_config_clocks'].get('reasons')}." if d.get("per_config_clocks") else "."))
+    out.append("")
+    if pk:
+        out.append("Peaks measured in the same run by the library's own micro-kernels (`btc_measure_peak`): "
+                   f"FP64 FMA {pk['fp64_fma_tflops']:.1f}, FP64 MMA m16n8k16 {pk['fp64_mma_m16n8k16_tflops']:.1f}, m8n8k4 {pk['fp64_mma_m8n8k4_tflops']:.1f}, "
+                   f"FP32 FMA {pk['fp32_fma_tflops']:.1f}, TF32 mma.sync {pk['tf32_mma_sync_tflops']:.0f} TFLOP/s; HBM read {pk['hbm_read_gbs']:.0f}, "
+                   f"write {pk['hbm_write_gbs']:.0f}, copy {pk['hbm_copy_gbs']:.0f} GB/s.  The roofline fractions below use the driver-measured copy bandwidth "
+                   "and the unit-count pipe peaks named in each row's `roofline.peak_source`.")
+        out.append("")
+    out.append("| workload | mode | time per call | rate | fraction of the bounding roofline | kernel | launches |")
+    out.append("|---|---|---|---|---|---|---|")
+    out.append(f"| {d['config']['workload']} (headline) | single execute, back to back | {d['ms_per_step']:.3f} ms | {d['value'] / 1e3:.2f} TFLOP/s | "
+               f"{frac(roof)} | {roof.get('kernel')} | {d['gpu_launches'] // d['steps']} |")
+    for v in d.get("per_config", []):
+        r = v.get("roofline", {})
+        ms = v["ms"]
+        t = f"{ms:.3f} ms" if ms >= 0.1 else f"{ms * 1e3:.1f} us"
+        rate = ", ".join(x for x in (f"{v['gflops'] / 1e3:.2f} TFLOP/s" if v.get("gflops") else "",
+                                     f"{v['gbs']:.0f} GB/s" if v.get("gbs") else "") if x)
+        out.append(f"| {v['workload']} | {v.get('mode', '')} | {t} | {rate} | {frac(r)} | {r.get('kernel')} | {v.get('launches', '')} |")
+    out.append("")
+    out.append(f"End to end through `btc_execute_host` (pinned host buffers, copies inside the timed region), headline workload: "
+               f"{e2e['value'] / 1e3:.2f} TFLOP/s ({e2e['h2d_bytes_per_step'] / 1e9:.2f} GB in, {e2e['d2h_bytes_per_step'] / 1e9:.2f} GB out per step).")
+    if cpu:
+        out.append(f"CPU oracle on the same box ({cpu.get('cores')} threads; {cpu.get('sample')}): {cpu.get('value'):.2f} {cpu.get('unit')} - a baseline for context, not a target.")
+    out.append("")
+    out.append("Every workload passes element-wise parity against the CPU oracle at these sizes (`tests/test_gpu_fullsize.py`, sampled")
+    out.append("elements for the large ones) within 1e-12 (64-bit parts) / 1e-5 (32-bit parts) of sum |a||b|.  What bounds each row: DESIGN.md section 7.")
+    with open(dst, "w") as f:
+        f.write("\n".join(out) + "\n")
+
+
 def main():
     args = parse()
+    if args.results_from:
+        write_results(args.results_from, args.results_out)
+        return
     from paper_2601_07827_b200 import inputs
     with_per_config = args.workload == "all"
     if with_per_config:
