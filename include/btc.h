@@ -20,6 +20,9 @@
  *
  * Threads: objects are immutable after creation except through btc_set_attr; executing one
  * contraction object from several host threads is allowed when each call has its own workspace.
+ *
+ * Environment: BTC_LOG (any value) prints every contraction's plan to stderr when it is created,
+ * and a note when a problem of more than 1 GFLOP lands on the per-element kernel.
  */
 #ifndef BTC_H_
 #define BTC_H_

@@ -839,7 +839,15 @@ btc_error_t btc_create_contraction(btc_handle_t handle, btc_tensor_info_t A, con
         delete op;
         return rc;
     }
-    if (std::getenv("BTC_LOG")) std::fprintf(stderr, "[btc] %s\n", op->plan.describe().c_str());
+    if (std::getenv("BTC_LOG")) {
+        std::fprintf(stderr, "[btc] %s\n", op->plan.describe().c_str());
+        // a large problem on the per-element kernel is almost always an unintended fall-back: say so
+        const Plan &pl = op->plan;
+        const double flops = 2.0 * double(pl.Bt) * double(pl.M) * double(pl.N) * double(pl.K);
+        if (pl.kernel == BTC_KERNEL_GENERIC && flops > 1e9)
+            std::fprintf(stderr, "[btc] note: %.3g flop on the per-element kernel (no tiled plan fits: offset tables too large, "
+                                 "mixed element types, or forced by attribute)\n", flops);
+    }
     *out = op;
     return BTC_SUCCESS;
 }
