@@ -27,9 +27,6 @@
 
 using namespace btc;
 
-#ifdef BTC_STAMPS
-static __device__ long long btc_stamp_buffer[512 * 8];   // debug builds only
-#endif
 
 struct btc_handle_s {
     int device = -1;       // -1: no CUDA device (objects can be validated and planned, not run)
@@ -1109,9 +1106,6 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
         tp.tmaA_coord_m = op->d_tma_coord_m; tp.tmaA_coord_k = op->d_tma_coord_k; tp.tmaA_coord_h = op->d_tma_coord_h;
         tp.skinny_orderA = op->d_skinny_order[0]; tp.skinny_orderB = op->d_skinny_order[3];
         tp.skinny_regular = op->skinny_regular ? 1 : 0;
-#ifdef BTC_STAMPS
-        { void *sp = nullptr; cudaGetSymbolAddress(&sp, btc_stamp_buffer); tp.stamps = static_cast<long long *>(sp); }
-#endif
         int64_t ctas = op->grid[0];
         int64_t reduce_ctas = (ctas / pl.split_k) * ((int64_t(pl.tile.bm) * pl.tile.bn + 1023) / 1024);
         // 16-byte stores of D (and loads of C) need those base pointers aligned too
@@ -1577,12 +1571,6 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
     return rc;
 }
 
-#ifdef BTC_STAMPS
-btc_error_t btc_debug_read_stamps(long long *dst)
-{
-    return cudaMemcpyFromSymbol(dst, btc_stamp_buffer, sizeof(long long) * 512 * 8) == cudaSuccess ? BTC_SUCCESS : BTC_ERR_CUDA;
-}
-#endif
 
 // ---- execute without any allocation -------------------------------------------------------------
 // Scratch for split-K partial sums that belongs to the library image itself: every GPU that loads

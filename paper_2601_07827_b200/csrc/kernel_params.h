@@ -114,9 +114,6 @@ struct TiledParams {
     // after the tile's first column (read through the constant bank instead of per-lane tables)
     int32_t skinny_d_regular;
     int32_t skinny_col_rel[128];
-#ifdef BTC_STAMPS
-    long long *stamps;                // debug build only: per-CTA phase time stamps (8 per CTA)
-#endif
 };
 
 }  // namespace btc

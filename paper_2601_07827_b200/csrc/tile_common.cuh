@@ -11,12 +11,6 @@ namespace btc {
 
 constexpr int kProducerWarps = 4;   // one warpgroup
 
-// Debug builds (-DBTC_STAMPS) record the SM clock at a few points of each CTA's life.
-#ifdef BTC_STAMPS
-#define BTC_STAMP(p, slot) do { if ((p).stamps && blockIdx.x < 512) (p).stamps[blockIdx.x * 8 + (slot)] = clock64(); } while (0)
-#else
-#define BTC_STAMP(p, slot) do { } while (0)
-#endif
 // k-offset entries per operand that a CTA keeps in shared memory (its whole k slice when it fits)
 constexpr int kKoffCap = 1024;
 

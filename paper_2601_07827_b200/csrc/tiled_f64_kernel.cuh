@@ -107,7 +107,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     const unsigned empty0 = full0 + 8u * T::STAGES;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) BTC_STAMP(p, 0);
     const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
     const int rows_valid = tc.rows_valid, cols_valid = tc.cols_valid, num_kt = tc.num_kt;
     (void)rows_valid; (void)cols_valid;
@@ -118,14 +117,12 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
     const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
     const int b_srow = p.dirB == 0 ? 1 : T::PITCH_K, b_sk = p.dirB == 0 ? T::PITCH_FREE_B : 1;
 
-    if (tid == 0) BTC_STAMP(p, 1);                      // set-up done
     if (warp < kProducerWarps) {
         // ------------------------------------------------------------------ producers
         if (T::REBALANCE_REGS) reg_dec<40>();
         const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
         producer_loop<T::BM, T::BN, T::BK, EB, T::STAGES, T::STAGE_WORDS * 8, T::A_ELEMS * EB, T::PRODUCER_THREADS>(
             p, tc, stage0, rowA, colB, koffA, koffB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
-        if (tid == 0) BTC_STAMP(p, 2);                  // producers done issuing
         return;
     }
 
@@ -172,7 +169,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
 #pragma unroll
         for (int j = 0; j < T::FN; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
 
-    if (ctid == 0) BTC_STAMP(p, 3);                     // consumers ready
     bool ok = true;
     for (int kt = 0; kt < num_kt; ++kt) {
         const int s = kt % T::STAGES, round = kt / T::STAGES;
@@ -180,7 +176,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
             ok = false;
             break;
         }
-        if (kt == 0 && ctid == 0) BTC_STAMP(p, 4);      // first stage has landed
         const double *sa = stage_base + size_t(s) * T::STAGE_WORDS;
         const double *sb = sa + T::A_ELEMS * W;
         if (T::MMA16) {
@@ -238,7 +233,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
         if (lane == 0) mbar_arrive(empty0 + 8u * s);
     }
     (void)ok;   // a wait that gave up has raised the CTA's abort flag
-    if (ctid == 0) BTC_STAMP(p, 5);                     // main loop done
 
     // Epilogue: park the fragments as an image of the tile (rows contiguous) in the now idle
     // stage buffers, then all consumer threads walk it (see epilogue_common.cuh).
@@ -262,7 +256,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
         }
     }
     consumer_barrier<T::CONSUMER_THREADS>();
-    if (ctid == 0) BTC_STAMP(p, 6);                     // image parked
     if (p.cluster_split) {
         // the k slices of this tile are the CTAs of this cluster: add them up through distributed shared
         // memory, every CTA a share of the tile.  (Producer warps have returned; a CTA that gave up has
@@ -274,7 +267,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_f64_kernel(cons
         return;
     }
     store_tile_image<double, W, T::BM, T::BN, T::CONSUMER_THREADS>(p, tc, image, rowD, colD, ctid);
-    if (ctid == 0) BTC_STAMP(p, 7);                     // stores issued
 }
 
 }  // namespace btc

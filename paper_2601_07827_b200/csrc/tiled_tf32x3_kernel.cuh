@@ -87,7 +87,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
     const unsigned empty0 = full0 + 8u * T::STAGES;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) BTC_STAMP(p, 0);
     const TileCoords tc = tile_coords<T::BM, T::BN, T::BK>(p);
     tile_setup<T::BM, T::BN, T::STAGES, T::THREADS, T::PRODUCER_THREADS, T::CONSUMER_WARPS>(
         p, tc, rowA, rowD, colB, colD, koffA, koffB, full0, empty0, abort_flag, tid);
@@ -95,13 +94,11 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
     const int a_srow = p.dirA == 0 ? 1 : T::PITCH_K, a_sk = p.dirA == 0 ? T::PITCH_FREE_A : 1;
     const int b_srow = p.dirB == 0 ? 1 : T::PITCH_K, b_sk = p.dirB == 0 ? T::PITCH_FREE_B : 1;
 
-    if (tid == 0) BTC_STAMP(p, 1);                      // set-up done
     if (warp < kProducerWarps) {
         if (T::REBALANCE_REGS) reg_dec<40>();
         const unsigned stage0 = static_cast<unsigned>(__cvta_generic_to_shared(stage_base));
         producer_loop<T::BM, T::BN, T::BK, EB, T::STAGES, T::STAGE_WORDS * 4, T::A_ELEMS * EB, T::PRODUCER_THREADS>(
             p, tc, stage0, rowA, colB, koffA, koffB, full0, empty0, abort_flag, a_srow, a_sk, b_srow, b_sk, tid);
-        if (tid == 0) BTC_STAMP(p, 2);                  // producers done issuing
         return;
     }
 
@@ -146,7 +143,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[i][j][c] = 0.f;
 
-    if (ctid == 0) BTC_STAMP(p, 3);                     // consumers ready
     bool ok = true;
     for (int kt = 0; kt < tc.num_kt; ++kt) {
         const int s = kt % T::STAGES, round = kt / T::STAGES;
@@ -154,7 +150,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
             ok = false;
             break;
         }
-        if (kt == 0 && ctid == 0) BTC_STAMP(p, 4);      // first stage has landed
         const float *sa = stage_base + size_t(s) * T::STAGE_WORDS;
         const float *sb = sa + T::A_ELEMS * W;
 #pragma unroll
@@ -192,7 +187,6 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
         if (lane == 0) mbar_arrive(empty0 + 8u * s);
     }
     (void)ok;   // a wait that gave up has raised the CTA's abort flag
-    if (ctid == 0) BTC_STAMP(p, 5);                     // main loop done
 
     // Epilogue: fragments -> image of the tile in the idle stage buffers -> rolled walk.
     // Fragment (fi, fj): c0, c1 -> row g, columns 2t, 2t+1; c2, c3 -> row g+8, same columns.
@@ -219,9 +213,7 @@ __global__ void __launch_bounds__(T::THREADS, T::MIN_CTAS) tiled_tf32x3_kernel(c
             }
         }
     consumer_barrier<T::CONSUMER_THREADS>();
-    if (ctid == 0) BTC_STAMP(p, 6);                     // image parked
     store_tile_image<float, W, T::BM, T::BN, T::CONSUMER_THREADS>(p, tc, image, rowD, colD, ctid);
-    if (ctid == 0) BTC_STAMP(p, 7);                     // stores issued
 }
 
 }  // namespace btc

@@ -326,16 +326,6 @@ __device__ __forceinline__ void umma_produce(unsigned tile, const UmmaProducerLa
 
 constexpr int kErrAccumWait = 3, kErrTailFullWait = 4, kErrTailEmptyWait = 5, kErrGroupSync = 6;
 
-// Debug builds (-DBTC_STAMPS) add up the SM clock cycles one thread spends in each phase.
-#ifdef BTC_STAMPS
-#define BTC_PHASE_BEGIN() long long phase_t0 = clock64()
-#define BTC_PHASE_END(acc) do { const long long phase_t1 = clock64(); (acc) += phase_t1 - phase_t0; phase_t0 = phase_t1; } while (0)
-#define BTC_PHASE_STORE(p, who, slot, acc) do { if ((who) && (p).stamps && blockIdx.x < 512) (p).stamps[blockIdx.x * 8 + (slot)] = (acc); } while (0)
-#else
-#define BTC_PHASE_BEGIN() do { } while (0)
-#define BTC_PHASE_END(acc) do { } while (0)
-#define BTC_PHASE_STORE(p, who, slot, acc) do { } while (0)
-#endif
 
 // Group-wide rendezvous on an mbarrier (every member arrives, then waits with a bound): unlike a
 // named barrier it cannot hang when a member has left after an abort.
@@ -468,9 +458,6 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         const int group = (tid - T::EPILOGUE_THREADS) / T::CONVERTER_THREADS;
         bool ok = true;
         int g = 0;                                   // stage counter across tiles
-        long long t_raw = 0, t_tail = 0, t_work = 0;
-        (void)t_raw; (void)t_tail; (void)t_work;
-        BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x) {
 #pragma unroll 1
@@ -481,13 +468,11 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     ok = false;
                     break;
                 }
-                BTC_PHASE_END(t_raw);
                 if (g >= T::TAIL_STAGES &&
                     !mbar_wait_bounded(tail_empty0 + 8u * t, unsigned(g / T::TAIL_STAGES - 1) & 1u, abort_flag, p.error_word, kErrTailEmptyWait, p.poll_limit)) {
                     ok = false;
                     break;
                 }
-                BTC_PHASE_END(t_tail);
 #pragma unroll
                 for (int sub = 0; sub < T::SUBS; ++sub) {
                 if (st * T::SUBS + sub >= num_kt) break;     // a tile's last stage may hold fewer sub-stages
@@ -579,20 +564,13 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                 }
                 proxy_fence_async();             // the tensor core reads both stages through the async proxy
                 mbar_arrive(tail_full0 + 8u * t);
-                BTC_PHASE_END(t_work);
             }
         }
-        BTC_PHASE_STORE(p, ct == 0 && group == 0, 0, t_raw);
-        BTC_PHASE_STORE(p, ct == 0 && group == 0, 1, t_tail);
-        BTC_PHASE_STORE(p, ct == 0 && group == 0, 2, t_work);
     } else if (warp < T::MMA_WARP) {
         // ------------------------------------------------------------- producers
         const int pt = tid - T::EPILOGUE_THREADS - 32 * T::CONVERTER_WARPS;
         bool ok = true;
         int g = 0, n = 0;
-        long long t_setup = 0, t_empty = 0, t_copy = 0;
-        (void)t_setup; (void)t_empty; (void)t_copy;
-        BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x, ++n) {
             const TileCoords tc = tile_coords_at<T::BM, T::BN, T::BK>(p, work);
@@ -622,7 +600,6 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
             UmmaStageOffsets sa = {0, 0, false, false}, sb = sa, sa_next = sa, sb_next = sa;
             if (!T::A_TMA && opA.vec == 4) sa_next = umma_lookup<T::BM>(la, opA, 0);
             if (opB.vec == 4) sb_next = umma_lookup<T::BN, T::BK>(lb, opB, 0);
-            BTC_PHASE_END(t_setup);
 #pragma unroll 1
             for (int st_i = 0; st_i < num_st; ++st_i, ++g) {
                 const int s = g % T::RAW_STAGES;
@@ -638,7 +615,6 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     ok = false;
                     break;
                 }
-                BTC_PHASE_END(t_empty);
                 const int subs_here = num_kt - st_i * T::SUBS < T::SUBS ? num_kt - st_i * T::SUBS : T::SUBS;
                 if (T::A_TMA && pt == 0) mbar_arrive_expect_tx(raw_full0 + 8u * s, unsigned(T::A_BYTES) * unsigned(subs_here));
 #pragma unroll
@@ -663,11 +639,8 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     umma_produce<T::BN, T::BK>(st + T::A_BYTES, lb, opB, k0, sb);
                 }
                 mbar_arrive_on_copies(raw_full0 + 8u * s);
-                BTC_PHASE_END(t_copy);
             }
         }
-        BTC_PHASE_STORE(p, pt == 0, 3, t_empty);
-        BTC_PHASE_STORE(p, pt == 0, 7, t_setup);
         cp_async_wait_all();
     } else {
         // ------------------------------------------------------------- MMA warp
@@ -684,20 +657,12 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
         const bool leader = elect_one();
         bool ok = true;
         int g = 0, n = 0;
-        long long t_acc = 0, t_full = 0, t_issue = 0;
-        (void)t_acc; (void)t_full; (void)t_issue;
-#ifdef BTC_STAMPS
-        long long wall_ns;                       // the main loop in wall-clock time: gives the SM clock it ran at
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(wall_ns));
-#endif
-        BTC_PHASE_BEGIN();
 #pragma unroll 1
         for (int64_t work = blockIdx.x; ok && work < total; work += gridDim.x, ++n) {
             const int buf = n & 1;
             if (n >= 2 &&
                 !mbar_wait_bounded(accum_empty0 + 8u * buf, unsigned((n >> 1) - 1) & 1u, abort_flag, p.error_word, kErrAccumWait, p.poll_limit))
                 break;
-            BTC_PHASE_END(t_acc);
             tc_fence_after();
             const unsigned tacc = tmem_base + unsigned(buf * T::ACC_COLS);
 #pragma unroll 1
@@ -707,7 +672,6 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     ok = false;
                     break;
                 }
-                BTC_PHASE_END(t_full);
                 tc_fence_after();
                 if (leader) {
 #pragma unroll
@@ -739,20 +703,8 @@ __global__ void __launch_bounds__(T::THREADS, 1) tiled_umma_tf32x3_kernel(const 
                     if (st + 1 == num_st) umma_commit(accum_full0 + 8u * buf);
                 }
                 __syncwarp();
-                BTC_PHASE_END(t_issue);
             }
         }
-#ifdef BTC_STAMPS
-        {
-            long long now;
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-            t_full += t_acc;                     // slot 4: all waiting; slot 6: nanoseconds
-            t_acc = now - wall_ns;
-        }
-#endif
-        BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 6, t_acc);
-        BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 4, t_full);
-        BTC_PHASE_STORE(p, threadIdx.x % 32 == 0, 5, t_issue);
         tc_fence_before();
     }
 
