@@ -967,6 +967,7 @@ namespace {
 struct BatchView {
     int64_t count;
     const int64_t *offA_h, *offB_h, *offD_h;   // [count * Bt], planned roles
+    const int64_t *host_tab = nullptr;         // the same three tables on the host, when they ride in the kernel's parameters instead
     void *partials;
     bool aligned16_D, aligned_A, aligned_B;     // every entry's pointer keeps the vector alignment
     bool aligned16_A;                           // every entry's M-side input pointer is 16-byte aligned
@@ -1153,7 +1154,16 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
                     // thread writes 16-byte pieces and neighbouring threads neighbouring pieces.  With long
                     // runs a warp's 32 consecutive rows of one column are a whole line as they are.
                     TiledParams sp = tp;
+                    SkinnyBatch sb;
+                    sb.count = 0; sb.pad = 0;
+                    const int64_t *tabA = nullptr, *tabB = nullptr;
+                    if (bv && bv->host_tab) {
+                        sb.count = int32_t(tp.Bt);
+                        tabA = bv->host_tab; tabB = bv->host_tab + tp.Bt;
+                        std::memcpy(sb.offD_h, bv->host_tab + 2 * tp.Bt, size_t(tp.Bt) * sizeof(int64_t));
+                    }
                     if (tp.vecD == 4 && op->skinny_run_m < 32) {
+                        std::swap(tabA, tabB);
                         std::swap(sp.A, sp.B);
                         std::swap(sp.offA_m, sp.offB_n); std::swap(sp.offD_m, sp.offD_n);
                         std::swap(sp.offA_k, sp.offB_k); std::swap(sp.offA_h, sp.offB_h);
@@ -1169,7 +1179,11 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
                     const std::vector<int64_t> &col_off = exchanged ? pl.offD_m : pl.offD_n;
                     sp.skinny_d_regular = op->skinny_d_regular[exchanged ? 0 : 1] ? 1 : 0;
                     for (size_t c = 0; c < 128; ++c) sp.skinny_col_rel[c] = c < col_off.size() ? int32_t(col_off[c] - col_off[0]) : 0;
-                    ce = launch_skinny_umma(sp, int(ctas), st);
+                    if (sb.count) {
+                        std::memcpy(sb.offA_h, tabA, size_t(tp.Bt) * sizeof(int64_t));
+                        std::memcpy(sb.offB_h, tabB, size_t(tp.Bt) * sizeof(int64_t));
+                    }
+                    ce = launch_skinny_umma(sp, sb, int(ctas), st);
                 }
                 break;
             case 8: ce = launch_tiled_tf32<F32TcWide>(tp, ctas, reduce_ctas, st); break;
@@ -1304,7 +1318,13 @@ btc_error_t btc_execute_batched(btc_contraction_t op, void *cuda_stream, const v
         }
     }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    if (cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int64_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    // The short-K streaming kernel takes the offsets of up to 64 entries in its parameters: no copy before
+    // the launch (which would also keep consecutive launches from overlapping their set-up).
+    const bool in_params = pl.kernel == BTC_KERNEL_TILED && pl.dtype == BTC_F32 && pl.tile.variant == kSkinnyVariant &&
+                           count * Bt <= kSkinnyInlineEntries && pl.vecA == 4 && pl.vecB == 4 && bv.aligned_A && bv.aligned_B;
+    if (in_params) {
+        bv.host_tab = tab.data();
+    } else if (cudaMemcpyAsync(workspace, tab.data(), tab.size() * sizeof(int64_t), cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return BTC_ERR_CUDA;
     }

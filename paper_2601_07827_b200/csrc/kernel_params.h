@@ -116,4 +116,12 @@ struct TiledParams {
     int32_t skinny_col_rel[128];
 };
 
+// Short-K streaming kernel, pointer-array calls of few entries: the per-entry offsets ride in the kernel's
+// parameters instead of a table uploaded before the launch (count = 0: the tables of TiledParams count).
+constexpr int kSkinnyInlineEntries = 64;
+struct SkinnyBatch {
+    int32_t count, pad;
+    int64_t offA_h[kSkinnyInlineEntries], offB_h[kSkinnyInlineEntries], offD_h[kSkinnyInlineEntries];
+};
+
 }  // namespace btc

@@ -9,7 +9,7 @@ namespace btc {
 
 // fp32, K <= 64: persistent tcgen05 kernel that streams D (skinny_umma_kernel.cuh)
 constexpr int kSkinnyMaxK = 64;
-cudaError_t launch_skinny_umma(const TiledParams &p, int ctas, cudaStream_t stream);
+cudaError_t launch_skinny_umma(const TiledParams &p, const SkinnyBatch &batch, int ctas, cudaStream_t stream);
 
 // any element type (0 fp32, 1 fp64, 2 complex64, 3 complex128), K <= 4: one thread per 16 bytes of D
 // (stream_kernel.cuh).  vec_d: groups of 16 bytes along the first M mode are contiguous and aligned in D

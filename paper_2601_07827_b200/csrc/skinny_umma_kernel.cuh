@@ -227,11 +227,11 @@ struct SkinnyStore {
         co_next[0] = co_next[1] = co_next[2] = co_next[3] = 0;
     }
     // start fetching what tile wk needs; `strip_start`: wk is the first tile of its half's strip for this CTA
-    __device__ __forceinline__ void fetch(const TiledParams &p, const SkinnyWork &wk, bool strip_start)
+    __device__ __forceinline__ void fetch(const TiledParams &p, const SkinnyBatch &sb, const SkinnyWork &wk, bool strip_start)
     {
         if (strip_start) {
             row_ok_next = row < wk.rows_valid;
-            ro_next = row_ok_next ? p.offD_m[wk.m0 + row] + p.offD_h[wk.h] : 0;
+            ro_next = row_ok_next ? p.offD_m[wk.m0 + row] + (sb.count ? sb.offD_h[wk.h] : p.offD_h[wk.h]) : 0;
         }
         if (dreg) {
             co_next[0] = p.offD_n[wk.n0];
@@ -324,7 +324,7 @@ struct SkinnyStore {
     }
 };
 
-__global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(const TiledParams p)
+__global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(const __grid_constant__ TiledParams p, const __grid_constant__ SkinnyBatch sb)
 {
     using T = SkinnyTile;
     extern __shared__ __align__(16) unsigned char smem_unaligned[];
@@ -360,6 +360,8 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
     const int64_t total = int64_t((p.tiles_m + halves - 1) / halves) * p.tiles_n * p.Bt;      // pairs
     const int64_t t0 = total * blockIdx.x / gridDim.x, t1 = total * (blockIdx.x + 1) / gridDim.x;
 
+    // the next grid in the stream may begin its own set-up as soon as SMs become free
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // ---- set-up: k offsets, barriers, tensor memory ----
     for (int i = tid; i < T::KMAX; i += T::THREADS) {
         koffA[i] = i < K ? p.offA_k[i] : 0;
@@ -397,6 +399,9 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
     __syncthreads();
     tc_fence_after();
     const unsigned tmem_base = *tmem_slot;
+    // Up to here only the operation's own tables were read.  From here on operand data is read and D is
+    // written: the grid launched before this one in the stream must be complete and its writes visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const unsigned tmem_a0 = tmem_base + 2u * T::ACC_COLS;
 
     if (warp < T::EPILOGUE_WARPS) {
@@ -405,7 +410,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         st.init(p, tid, lane);
         SkinnyIter it;
         it.start(p, halves, t0, t1);
-        if (it.valid) st.fetch(p, it.work(p), true);
+        if (it.valid) st.fetch(p, sb, it.work(p), true);
 #pragma unroll 1
         while (it.valid) {
             const int i = it.i, buf = i & 1, half = it.half;
@@ -415,7 +420,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
 #pragma unroll
             for (int c = 0; c < 4; ++c) co[c] = st.co_next[c];
             it.advance(p);
-            if (it.valid) st.fetch(p, it.work(p), it.new_a);
+            if (it.valid) st.fetch(p, sb, it.work(p), it.new_a);
             if (!mbar_wait_bounded(acc_full0 + 8u * buf, unsigned(i >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyEpilogue, p.poll_limit)) break;
             tc_fence_after();
             st.tile(p, w, half, tmem_base + (unsigned(warp * 32) << 16) + unsigned(buf * T::ACC_COLS), 0, T::SPLIT_COL, acc_empty0 + 8u * buf, co);
@@ -438,7 +443,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             const int i = it.i, half_now = it.half;
             const SkinnyWork w = it.work(p);
             const bool new_a = it.new_a;
-            st.fetch(p, w, new_a);                    // for this tile's store, one iteration from now
+            st.fetch(p, sb, w, new_a);                    // for this tile's store, one iteration from now
             if (new_a) {
                 const int loads = it.an0 + it.an1, mine = it.a_before(), ab = it.abuf;
                 if (!(ok = mbar_wait_bounded(a_full, unsigned(loads) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit))) break;
@@ -538,8 +543,8 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         auto fetch = [&](const SkinnyIter &at) {
             const SkinnyWork wk = at.work(p);
             const int r = regular ? 0 : pt;
-            if (at.new_a) next_row = r < wk.rows_valid ? p.offA_m[wk.m0 + r] + p.offA_h[wk.h] : 0;
-            if (at.first_of_b()) next_col = r < wk.cols_valid ? p.offB_n[wk.n0 + r] + p.offB_h[wk.h] : 0;
+            if (at.new_a) next_row = r < wk.rows_valid ? p.offA_m[wk.m0 + r] + (sb.count ? sb.offA_h[wk.h] : p.offA_h[wk.h]) : 0;
+            if (at.first_of_b()) next_col = r < wk.cols_valid ? p.offB_n[wk.n0 + r] + (sb.count ? sb.offB_h[wk.h] : p.offB_h[wk.h]) : 0;
         };
         if (it.valid) fetch(it);
 #pragma unroll 1
