@@ -40,9 +40,11 @@ namespace btc {
 
 struct SkinnyTile {
     static constexpr int BM = 128, BN = 128, KMAX = 64;
-    // the N-side tiles wait in a ring of raw stages (filled up to three tiles ahead of the tensor core, to ride out
-    // the memory latency); their tails are made just in time into a shorter ring
-    static constexpr int RAW_STAGES = 3, LO_STAGES = 2;
+    // the N-side tiles wait in a ring of raw stages (each serves the two tiles of a pair, so two stages are
+    // four tiles of lead over the tensor core); their tails are made just in time into a ring of the same
+    // length; the M-side tile has two raw buffers, so that both halves' tiles of the next strip are
+    // fetched while the tensor core still works on this one
+    static constexpr int RAW_STAGES = 2, LO_STAGES = 2, A_STAGES = 2;
     static constexpr int EPILOGUE_WARPS = 4, CONVERTER_WARPS = 4, LOADER_WARPS = 4;
     static constexpr int GROUP_THREADS = 128;
     static constexpr int MMA_WARP = EPILOGUE_WARPS + CONVERTER_WARPS + LOADER_WARPS;
@@ -57,7 +59,7 @@ struct SkinnyTile {
     static constexpr int NUM_BARS = 24;
     static constexpr int SPLIT_COL = 64;                     // columns below: epilogue warps; from here on: the converter warps, between conversions
     // N-side raw[3] | N-side tail[2] | M-side raw | row / column offsets | k offsets | piece tables | barriers | slot, abort
-    static constexpr size_t SMEM_BYTES = size_t(RAW_STAGES + LO_STAGES) * B_BYTES + A_BYTES +
+    static constexpr size_t SMEM_BYTES = size_t(RAW_STAGES + LO_STAGES) * B_BYTES + size_t(A_STAGES) * A_BYTES +
                                          size_t(2 * BM + RAW_STAGES * BN + 2 * KMAX) * 8 + size_t(2 * PIECES) * 4 +
                                          size_t(NUM_BARS) * 8 + 16 + 1024;
 };
@@ -330,7 +332,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
     extern __shared__ __align__(16) unsigned char smem_unaligned[];
     unsigned char *smem_raw = smem_unaligned +
         ((1024u - (static_cast<unsigned>(__cvta_generic_to_shared(smem_unaligned)) & 1023u)) & 1023u);
-    unsigned char *cursor = smem_raw + size_t(T::RAW_STAGES + T::LO_STAGES) * T::B_BYTES + T::A_BYTES;
+    unsigned char *cursor = smem_raw + size_t(T::RAW_STAGES + T::LO_STAGES) * T::B_BYTES + size_t(T::A_STAGES) * T::A_BYTES;
     int64_t *rowA = reinterpret_cast<int64_t *>(cursor);                 // [2][BM]
     int64_t *colB = rowA + 2 * T::BM;                                    // [RAW_STAGES][BN]
     int64_t *koffA = colB + T::RAW_STAGES * T::BN;                       // [KMAX]
@@ -342,11 +344,11 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     const unsigned braw0 = static_cast<unsigned>(__cvta_generic_to_shared(smem_raw));
     const unsigned blo0 = braw0 + unsigned(T::RAW_STAGES) * T::B_BYTES;
-    const unsigned araw = blo0 + unsigned(T::LO_STAGES) * T::B_BYTES;
+    const unsigned araw0 = blo0 + unsigned(T::LO_STAGES) * T::B_BYTES;      // two raw M-side buffers
     const unsigned bar0 = static_cast<unsigned>(__cvta_generic_to_shared(bars));
-    const unsigned a_full = bar0, a_empty = bar0 + 8u;
-    const unsigned raw_full0 = bar0 + 16u, raw_empty0 = raw_full0 + 24u;                      // [3] each
-    const unsigned lo_conv0 = raw_empty0 + 24u, lo_empty0 = lo_conv0 + 16u;                   // [2] each
+    const unsigned a_full0 = bar0, a_empty0 = bar0 + 16u;                                     // [2] each
+    const unsigned raw_full0 = bar0 + 32u, raw_empty0 = raw_full0 + 8u * T::RAW_STAGES;       // [RAW_STAGES] each
+    const unsigned lo_conv0 = raw_empty0 + 8u * T::RAW_STAGES, lo_empty0 = lo_conv0 + 16u;    // [2] each
     const unsigned ta_full0 = lo_empty0 + 16u, ta_empty0 = ta_full0 + 16u;                    // [2] each
     const unsigned acc_full0 = ta_empty0 + 16u, acc_empty0 = acc_full0 + 16u;                 // [2] each
     const unsigned loader_sync = acc_empty0 + 16u, drain = loader_sync + 8u;
@@ -372,9 +374,9 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
         pieceB[e] = p.skinny_orderB[e];
     }
     if (tid == 0) {
-        mbar_init(a_full, T::GROUP_THREADS);
-        mbar_init(a_empty, T::GROUP_THREADS);
         for (int s = 0; s < 2; ++s) {
+            mbar_init(a_full0 + 8u * s, T::GROUP_THREADS);
+            mbar_init(a_empty0 + 8u * s, T::GROUP_THREADS);
             mbar_init(lo_conv0 + 8u * s, T::GROUP_THREADS);
             mbar_init(lo_empty0 + 8u * s, 1);
             mbar_init(ta_full0 + 8u * s, T::GROUP_THREADS);
@@ -446,7 +448,8 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             st.fetch(p, sb, w, new_a);                    // for this tile's store, one iteration from now
             if (new_a) {
                 const int loads = it.an0 + it.an1, mine = it.a_before(), ab = it.abuf;
-                if (!(ok = mbar_wait_bounded(a_full, unsigned(loads) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit))) break;
+                const unsigned araw = araw0 + unsigned(loads & 1) * T::A_BYTES;
+                if (!(ok = mbar_wait_bounded(a_full0 + 8u * unsigned(loads & 1), unsigned(loads >> 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit))) break;
                 // the operand buffer is free once the tensor core has finished the strip that used it before
                 if (mine >= 1 &&
                     !(ok = mbar_wait_bounded(ta_empty0 + 8u * ab, unsigned(mine - 1) & 1u, abort_flag, p.error_word, kErrSkinnyConvert, p.poll_limit)))
@@ -476,7 +479,7 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
                 tmem_store_wait();
                 tc_fence_before();
                 mbar_arrive(ta_full0 + 8u * ab);
-                mbar_arrive(a_empty);                 // the raw M-side buffer may be refilled
+                mbar_arrive(a_empty0 + 8u * unsigned(loads & 1));     // this raw M-side buffer may be refilled
             }
             if (it.first_of_b()) {
                 const int bi = it.bi, r = bi % T::RAW_STAGES, s = bi & 1;
@@ -562,10 +565,12 @@ __global__ void __launch_bounds__(SkinnyTile::THREADS, 1) skinny_umma_kernel(con
             it.advance(p);
             if (it.valid) fetch(it);
             if (new_a) {
-                if (loads > 0 && !mbar_wait_bounded(a_empty, unsigned(loads - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
+                const unsigned araw = araw0 + unsigned(loads & 1) * T::A_BYTES;
+                if (loads >= 2 &&
+                    !mbar_wait_bounded(a_empty0 + 8u * unsigned(loads & 1), unsigned((loads >> 1) - 1) & 1u, abort_flag, p.error_word, kErrSkinnyLoad, p.poll_limit)) break;
                 if (regular) skinny_load_tile_regular<true>(araw, A, row_base, pieceA, pieces, p.dirA, w.rows_valid, pt, p.spans, 0);
                 else skinny_load_tile<true>(araw, A, rA, koffA, pieceA, pieces, p.dirA, w.rows_valid, pt, p.spans, 0);
-                mbar_arrive_on_copies(a_full);
+                mbar_arrive_on_copies(a_full0 + 8u * unsigned(loads & 1));
             }
             if (new_b) {
                 if (bi >= T::RAW_STAGES &&
