@@ -1704,6 +1704,19 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
         const Mode &m = pl.keep[size_t(i)];
         p.ext_k[i] = m.extent; p.sA_k[i] = m.sA; p.sB_k[i] = m.sB; p.sC_k[i] = m.sD;
     }
+    {
+        auto reciprocal = [](int64_t ext, uint32_t &mul, uint32_t &shift) {
+            int s = 0;
+            while ((int64_t(1) << s) < ext) ++s;
+            shift = uint32_t(31 + s);
+            mul = uint32_t(((uint64_t(1) << shift) + uint64_t(ext) - 1) / uint64_t(ext));
+        };
+        const int64_t vlen = int64_t(16 / dtype_size(pl.dtype));
+        for (int i = 0; i < p.nk; ++i)
+            if (p.ext_k[i] < (int64_t(1) << 31)) reciprocal(p.ext_k[i], p.div_mul[i], p.div_shift[i]);
+        if (p.nk > 0 && vlen > 0 && p.ext_k[0] % vlen == 0 && p.ext_k[0] < (int64_t(1) << 31))
+            reciprocal(p.ext_k[0] / vlen, p.div_mul[kGenericMaxD], p.div_shift[kGenericMaxD]);
+    }
     int64_t min_sum = INT64_MAX, min_keep = INT64_MAX;
     for (int i = 0; i < p.ns; ++i) {
         p.ext_s[i] = pl.sum[size_t(i)].extent; p.sA_s[i] = pl.sum[size_t(i)].sA;

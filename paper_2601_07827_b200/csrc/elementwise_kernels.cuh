@@ -20,6 +20,15 @@
 
 namespace btc {
 
+// lin / ext for the loop dimension `d` of p (kGenericMaxD: dimension 0 counted in vectors): 32-bit indices
+// multiply by the reciprocal prepared on the host, 64-bit indices divide
+template <typename I>
+__device__ __forceinline__ I elementwise_div(const ElementwiseParams &p, I lin, I ext, int d)
+{
+    if (sizeof(I) == 4) return I((uint64_t(uint32_t(lin)) * p.div_mul[d]) >> p.div_shift[d]);
+    return lin / ext;
+}
+
 // arithmetic type of alpha * a + beta * b where nothing is summed: the part type itself
 template <typename R> struct ElementwiseScalar { typedef R type; };
 
@@ -104,7 +113,7 @@ __global__ void __launch_bounds__(256) elementwise_direct_kernel(const Elementwi
                 I lin = I(in[u] ? e : 0);
                 for (int d = 0; d < p.nk; ++d) {
                     const I ext = I(p.ext_k[d]);
-                    const I q = lin / ext;
+                    const I q = elementwise_div<I>(p, lin, ext, d);
                     const int64_t i = int64_t(lin - q * ext);
                     lin = q;
                     offA[u] += i * p.sA_k[d];
@@ -142,7 +151,7 @@ __global__ void __launch_bounds__(256) elementwise_direct_kernel(const Elementwi
         I lin = I(e);
         for (int d = 0; d < p.nk; ++d) {
             const I ext = I(p.ext_k[d]);
-            const I q = lin / ext;
+            const I q = elementwise_div<I>(p, lin, ext, d);
             const int64_t i = int64_t(lin - q * ext);
             lin = q;
             offA += i * p.sA_k[d];
@@ -189,13 +198,13 @@ __global__ void __launch_bounds__(256) elementwise_vector_kernel(const Elementwi
             in[u] = v < nvec;
             I lin = I(in[u] ? v : 0);
             const I ext0 = I(p.ext_k[0] / V);
-            const I q0 = lin / ext0;
+            const I q0 = elementwise_div<I>(p, lin, ext0, kGenericMaxD);
             const int64_t i0 = int64_t(lin - q0 * ext0) * V;
             lin = q0;
             offA[u] = i0 * p.sA_k[0]; offB[u] = i0 * p.sB_k[0]; offC[u] = i0;
             for (int d = 1; d < p.nk; ++d) {
                 const I ext = I(p.ext_k[d]);
-                const I q = lin / ext;
+                const I q = elementwise_div<I>(p, lin, ext, d);
                 const int64_t i = int64_t(lin - q * ext);
                 lin = q;
                 offA[u] += i * p.sA_k[d];

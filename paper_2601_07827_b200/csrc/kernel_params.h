@@ -63,6 +63,10 @@ struct ElementwiseParams {
     int64_t total_keep, total_sum;
     int64_t ext_k[kGenericMaxD], sA_k[kGenericMaxD], sB_k[kGenericMaxD], sC_k[kGenericMaxD];
     int64_t ext_s[kGenericMaxD], sA_s[kGenericMaxD];
+    // division by ext_k[d] (and by ext_k[0] / vector length, last entry) without a divide, for 32-bit
+    // indices below 2^31: q = (n * div_mul) >> div_shift in 64 bits, div_shift = 31 + ceil(log2 ext),
+    // div_mul = ceil(2^div_shift / ext) (exact for n < 2^31 since div_mul * ext - 2^div_shift < ext)
+    uint32_t div_mul[kGenericMaxD + 1], div_shift[kGenericMaxD + 1];
     int32_t tile_mode_a;              // transposing kernel: the dimension A is read along (C: dimension 0)
     int32_t tiles_c, tiles_a;         // transposing kernel: tiles along those two dimensions
     int64_t rest;                     // transposing kernel: product of the other dimensions' extents
