@@ -267,14 +267,18 @@ __global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise
     extern __shared__ __align__(16) unsigned char tile_bytes[];
     R (*tile)[TC][TA + 1] = reinterpret_cast<R (*)[TC][TA + 1]>(tile_bytes);
     const int ma = p.tile_mode_a;
-    const int64_t tile_c = blockIdx.x % p.tiles_c;
-    const int64_t tile_a = (blockIdx.x / p.tiles_c) % p.tiles_a;
-    int64_t lin = blockIdx.x / (int64_t(p.tiles_c) * p.tiles_a);
+    // (32-bit arithmetic: the grid has fewer than 2^31 CTAs; an extent of 2^31 or more has no
+    // reciprocal -- its multiplier is 0 -- and the quotient 0 that comes out is the right one)
+    const uint32_t q_c = blockIdx.x / uint32_t(p.tiles_c), q_a = q_c / uint32_t(p.tiles_a);
+    const int64_t tile_c = blockIdx.x - q_c * uint32_t(p.tiles_c);
+    const int64_t tile_a = q_c - q_a * uint32_t(p.tiles_a);
+    uint32_t lin = q_a;
     int64_t restA = 0, restB = 0, restC = 0;
     for (int d = 1; d < p.nk; ++d) {
         if (d == ma) continue;
-        const int64_t i = lin % p.ext_k[d];
-        lin /= p.ext_k[d];
+        const uint32_t q = elementwise_div<uint32_t>(p, lin, uint32_t(p.ext_k[d]), d);
+        const int64_t i = int64_t(lin - q * uint32_t(p.ext_k[d]));
+        lin = q;
         restA += i * p.sA_k[d];
         restB += i * p.sB_k[d];
         restC += i * p.sC_k[d];
