@@ -159,3 +159,41 @@ def test_elementwise_full_size_sampled(name):
     got = C.buffer[pos].cpu().numpy()
     assert helpers.compare(got, vals, scale, C.dtype) <= 1.0
     assert op.kernel in (api.EW_KERNEL_DIRECT, api.EW_KERNEL_TRANSPOSING)
+
+
+@pytest.mark.parametrize("name,count", [("cfg5_f32_tensor_network", 64), ("cfg5b_f32_tensor_network_rev", 64),
+                                        ("cfg1_f64_small", 148)])
+def test_batched_launch_configuration_of_the_benchmark(name, count):
+    """The pointer-array call bench.py times for the small workloads (batch hint = count, `count` buffer
+    sets in one launch): every entry gets the same inputs, so every entry's D must equal entry 0's bit for
+    bit, and entry 0 is compared with the oracle at sampled elements."""
+    api = helpers.api()
+    handle = api.Handle()
+    w = inputs.workloads()[name]
+    A, B, C, D = inputs.make_workload_tensors(w, device="cuda")
+    hA, hB = A.to("cpu"), B.to("cpu")
+    hC = C.to("cpu") if C is not None else None
+    rep = lambda t: torch.stack([t.buffer] * count).contiguous()
+    pA, pB, pD = rep(A), rep(B), rep(D)
+    pC = rep(C) if (C is not None and not w.in_place) else None
+    dt = api.dtype_code(D.dtype)
+    tA = api.TensorInfo(handle, dt, A.extents, A.strides)
+    tB = api.TensorInfo(handle, dt, B.extents, B.strides)
+    tD = api.TensorInfo(handle, dt, D.extents, D.strides)
+    op = api.Contraction(handle, tA, w.labelsA, tB, w.labelsB, tD if C is not None else None, w.labelsD, tD, w.labelsD,
+                         w.alpha, w.beta, w.conjA, w.conjB, w.conjC)
+    op.set_attr(api.ATTR_BATCH_HINT, count)
+    item = D.buffer.element_size()
+    ptrs = lambda pool, t: [pool.data_ptr() + (i * t.buffer.numel() + t.origin) * item for i in range(count)]
+    lA, lB, lD = ptrs(pA, A), ptrs(pB, B), ptrs(pD, D)
+    lC = None if C is None else (lD if w.in_place else ptrs(pC, C))
+    ws_bytes = op.batched_workspace_size(count)
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
+    op.execute_batched(torch.cuda.current_stream().cuda_stream, lA, lB, lC, lD, workspace=ws.data_ptr(), workspace_bytes=ws_bytes)
+    torch.cuda.synchronize()
+    assert op.device_error == 0
+    width = {4: torch.int32, 8: torch.int64}[item]
+    bits = pD.view(width)
+    assert torch.equal(bits, bits[0:1].expand_as(bits)), "entries with equal inputs differ"
+    worst = _sampled_check(w, hA, hB, hC, (D.extents, D.strides), pD[0].cpu(), D.origin, 20000, 4096, D.dtype)
+    assert worst <= 1.0, worst
