@@ -23,6 +23,7 @@
 #include "tiled_tf32x3_kernel.cuh"
 #include "tiled_umma_tf32x3_kernel.cuh"
 #include "isolated_sum_kernel.cuh"
+#include "complex_expand_kernel.cuh"
 #include "elementwise_kernels.cuh"
 
 using namespace btc;
@@ -76,6 +77,13 @@ struct btc_contraction_s {
     // memory spans of the caller's tensors in elements (the plan may describe A' and B' instead)
     int64_t spanA_lo = 0, spanA_hi = 0, spanB_lo = 0, spanB_hi = 0, spanD_lo = 0, spanD_hi = 0;
     struct HostPipeline *host = nullptr;   // built by the first btc_execute_host
+    // complex64 on the fp32 tensor-core path (complex_expand_kernel.cuh): the smaller input X is expanded
+    // into the front of the workspace, then `real_inner`, an fp32 contraction over the real views, runs.
+    // Used when that operation lands on a tcgen05 kernel; beta must be real and C not conjugated at execute.
+    btc_contraction_s *real_inner = nullptr;
+    bool real_expand_A = true;              // X is the caller's A (else B)
+    ComplexExpandParams real_expand;        // loop dimensions of X in X'' order (pointers and scalars filled at execute)
+    size_t real_x_bytes = 0;                // bytes of X'' (rounded up to 256)
 };
 
 // Host-buffer execution in slabs (btc_execute_host): the larger input is cut along the label with its largest
@@ -624,8 +632,114 @@ int finish_plan(btc_contraction_s *op)
     return BTC_SUCCESS;
 }
 
+int replan(btc_contraction_s *op);
+
+void free_real_form(btc_contraction_s *op)
+{
+    if (op->real_inner) {
+        free_tables(op->real_inner);
+        delete op->real_inner;
+        op->real_inner = nullptr;
+    }
+    op->real_x_bytes = 0;
+}
+
+// complex64 -> fp32: set up the real form of the operation (complex_expand_kernel.cuh) when it is worth
+// it, i.e. when the real contraction is planned onto a tcgen05 kernel.  Leaves op->real_inner null otherwise.
+void build_real_form(btc_contraction_s *op)
+{
+    free_real_form(op);
+    const PlanRequest &rq = op->req;
+    const Plan &pl = op->plan;
+    if (op->handle.device < 0 || pl.dtype != BTC_C32 || pl.mixed || pl.has_isolated || pl.kernel != BTC_KERNEL_TILED ||
+        rq.strict_fp32 != 0 || rq.force_variant >= 0 || rq.force_split_k != 0)
+        return;
+    auto count = [](const TensorDesc &t) { int64_t n = 1; for (int64_t e : t.extent) n *= e; return n; };
+    auto distinct = [](const std::vector<int64_t> &l) {
+        for (size_t i = 0; i < l.size(); ++i)
+            for (size_t j = i + 1; j < l.size(); ++j) if (l[i] == l[j]) return false;
+        return true;
+    };
+    const bool expand_A = count(rq.A) <= count(rq.B);
+    const TensorDesc &X = expand_A ? rq.A : rq.B, &Y = expand_A ? rq.B : rq.A;
+    const std::vector<int64_t> &lX = expand_A ? rq.labelsA : rq.labelsB, &lY = expand_A ? rq.labelsB : rq.labelsA;
+    if (!distinct(lX) || X.extent.size() + 2 > size_t(kExpandMaxD)) return;
+    auto find = [](const std::vector<int64_t> &l, int64_t x) { for (size_t i = 0; i < l.size(); ++i) if (l[i] == x) return int(i); return -1; };
+    // two labels of our own: u (parts of Y, contracted) and v (parts of D)
+    int64_t top = 0;
+    for (auto *l : {&rq.labelsA, &rq.labelsB, &rq.labelsC, &rq.labelsD}) for (int64_t x : *l) top = std::max(top, x);
+    if (top > INT64_MAX - 2) return;
+    const int64_t U = top + 1, V = top + 2;
+    // X's loop dimensions in the order of X'': contracted ones by |stride in Y|, then the others by |stride in D|
+    struct Dim { int64_t label, ext, sx, key; };
+    std::vector<Dim> kc, rest;
+    for (size_t i = 0; i < lX.size(); ++i) {
+        const int iy = find(lY, lX[i]), id = find(rq.labelsD, lX[i]);
+        if (id < 0 && iy >= 0) kc.push_back({lX[i], X.extent[i], X.stride[i], std::llabs(Y.stride[size_t(iy)])});
+        else if (id >= 0) rest.push_back({lX[i], X.extent[i], X.stride[i], std::llabs(rq.D.stride[size_t(id)])});
+        else return;                        // a label of X alone (Case 4): not here
+    }
+    auto by_key = [](const Dim &a, const Dim &b) { return a.key < b.key; };
+    std::stable_sort(kc.begin(), kc.end(), by_key);
+    std::stable_sort(rest.begin(), rest.end(), by_key);
+    ComplexExpandParams ep;
+    std::memset(&ep, 0, sizeof ep);
+    ep.total = ep.total_k = 1;
+    TensorDesc Xr, Yr, Dr, Cr;
+    std::vector<int64_t> lXr, lYr, lDr, lCr;
+    Xr.dtype = Yr.dtype = Dr.dtype = Cr.dtype = BTC_F32;
+    Xr.extent.push_back(2); Xr.stride.push_back(1); lXr.push_back(U);
+    int64_t run = 2;
+    for (auto &d : kc) {
+        ep.ext[ep.nd] = d.ext; ep.stride[ep.nd] = d.sx; ++ep.nd;
+        Xr.extent.push_back(d.ext); Xr.stride.push_back(run); lXr.push_back(d.label);
+        run *= d.ext; ep.total_k *= d.ext;
+    }
+    Xr.extent.push_back(2); Xr.stride.push_back(run); lXr.push_back(V);
+    run *= 2;
+    for (auto &d : rest) {
+        ep.ext[ep.nd] = d.ext; ep.stride[ep.nd] = d.sx; ++ep.nd;
+        Xr.extent.push_back(d.ext); Xr.stride.push_back(run); lXr.push_back(d.label);
+        run *= d.ext;
+    }
+    ep.total = run / 4;
+    auto real_view = [](const TensorDesc &t, const std::vector<int64_t> &labels, int64_t part, TensorDesc &out, std::vector<int64_t> &lout) {
+        out.extent.assign(1, 2); out.stride.assign(1, 1); lout.assign(1, part);
+        for (size_t i = 0; i < t.extent.size(); ++i) {
+            out.extent.push_back(t.extent[i]); out.stride.push_back(2 * t.stride[i]); lout.push_back(labels[i]);
+        }
+    };
+    real_view(Y, lY, U, Yr, lYr);
+    real_view(rq.D, rq.labelsD, V, Dr, lDr);
+    if (rq.has_c) real_view(rq.C, rq.labelsC, V, Cr, lCr);
+    btc_contraction_s *in = new (std::nothrow) btc_contraction_s;
+    if (!in) return;
+    in->handle = op->handle;
+    in->req.A = expand_A ? Xr : Yr; in->req.labelsA = expand_A ? lXr : lYr;
+    in->req.B = expand_A ? Yr : Xr; in->req.labelsB = expand_A ? lYr : lXr;
+    in->req.D = Dr; in->req.labelsD = lDr;
+    in->req.has_c = rq.has_c;
+    if (rq.has_c) { in->req.C = Cr; in->req.labelsC = lCr; }
+    in->req.batch_hint = rq.batch_hint;
+    in->poll_limit = op->poll_limit;
+    in->alpha[0] = 1.0; in->alpha[1] = 0.0; in->beta[0] = op->beta[0]; in->beta[1] = 0.0;
+    const bool planned = replan(in) == BTC_SUCCESS && in->plan.kernel == BTC_KERNEL_TILED && in->plan.dtype == BTC_F32 &&
+                         f32_persistent(in->plan.tile.variant);
+    if (!planned) {
+        free_tables(in);
+        delete in;
+        return;
+    }
+    op->real_inner = in;
+    op->real_expand_A = expand_A;
+    op->real_expand = ep;
+    op->real_x_bytes = (size_t(ep.total) * 16 + 255) / 256 * 256;
+    op->workspace_bytes = std::max(op->workspace_bytes, op->real_x_bytes + in->workspace_bytes);
+}
+
 int replan(btc_contraction_s *op)
 {
+    free_real_form(op);
     op->req.sm_count = op->handle.sm_count;
     int rc = make_plan(op->req, op->plan);
     if (rc != BTC_SUCCESS) return rc;
@@ -657,6 +771,7 @@ int replan(btc_contraction_s *op)
     op->sumB_offset = bytesA;
     op->partials_offset = bytesA + bytesB;
     op->workspace_bytes += op->partials_offset;
+    build_real_form(op);
     return BTC_SUCCESS;
 }
 
@@ -854,6 +969,7 @@ btc_error_t btc_destroy_contraction(btc_contraction_t *op)
     if (!op) return BTC_ERR_INVALID_ARGUMENT;
     if (*op) {
         free_host_pipeline(*op);
+        free_real_form(*op);
         free_tables(*op);
         delete *op;
     }
@@ -881,7 +997,8 @@ btc_error_t btc_set_attr(btc_contraction_t op, int32_t key, const void *value, s
     }
     if (key == BTC_ATTR_DEVICE_ERROR) {          // writing 0 clears the device error word
         if (v != 0) return BTC_ERR_INVALID_ARGUMENT;
-        if (op->d_error && cudaMemset(op->d_error, 0, sizeof(int32_t)) != cudaSuccess) {
+        if ((op->d_error && cudaMemset(op->d_error, 0, sizeof(int32_t)) != cudaSuccess) ||
+            (op->real_inner && op->real_inner->d_error && cudaMemset(op->real_inner->d_error, 0, sizeof(int32_t)) != cudaSuccess)) {
             cudaGetLastError();
             return BTC_ERR_CUDA;
         }
@@ -928,24 +1045,28 @@ btc_error_t btc_get_attr(btc_contraction_t op, int32_t key, void *value, size_t 
     const void *src = i32;
     size_t n = 0;
     const Plan &pl = op->plan;
+    // what runs: for complex64 operations in their real form, the fp32 operation's kernel, tile, grid
+    const btc_contraction_s *run = op->real_inner ? op->real_inner : op;
+    const Plan &rp = run->plan;
     switch (key) {
-    case BTC_ATTR_KERNEL: i32[0] = pl.kernel; n = 4; break;
-    case BTC_ATTR_SPLIT_K: i32[0] = pl.split_k; n = 4; break;
-    case BTC_ATTR_TILE: i32[0] = pl.tile.bm; i32[1] = pl.tile.bn; i32[2] = pl.tile.bk; n = 12; break;
+    case BTC_ATTR_KERNEL: i32[0] = rp.kernel; n = 4; break;
+    case BTC_ATTR_SPLIT_K: i32[0] = rp.split_k; n = 4; break;
+    case BTC_ATTR_TILE: i32[0] = rp.tile.bm; i32[1] = rp.tile.bn; i32[2] = rp.tile.bk; n = 12; break;
     case BTC_ATTR_GROUPS: i64[0] = pl.Bt; i64[1] = pl.M; i64[2] = pl.N; i64[3] = pl.K; src = i64; n = 32; break;
-    case BTC_ATTR_GRID: i32[0] = op->grid[0]; i32[1] = op->grid[1]; i32[2] = op->grid[2]; n = 12; break;
+    case BTC_ATTR_GRID: i32[0] = run->grid[0]; i32[1] = run->grid[1]; i32[2] = run->grid[2]; n = 12; break;
     case BTC_ATTR_NUM_MODES:
         i32[0] = int32_t(pl.batch.size()); i32[1] = int32_t(pl.m.size());
         i32[2] = int32_t(pl.n.size()); i32[3] = int32_t(pl.k.size()); n = 16; break;
     case BTC_ATTR_SWAPPED: i32[0] = pl.swapped ? 1 : 0; n = 4; break;
-    case BTC_ATTR_VARIANT: i32[0] = pl.tile.variant; n = 4; break;
+    case BTC_ATTR_VARIANT: i32[0] = rp.tile.variant; n = 4; break;
     case BTC_ATTR_PRE_REDUCE: i32[0] = (op->sumA.active ? 1 : 0) | (op->sumB.active ? 2 : 0); n = 4; break;
     case BTC_ATTR_BATCH_HINT: i32[0] = op->req.batch_hint; n = 4; break;
     case BTC_ATTR_COMPUTE_PRECISION: i32[0] = op->req.strict_fp32; n = 4; break;
     case BTC_ATTR_DEVICE_ERROR:
         i32[0] = 0;
-        if (op->d_error) {
-            if (cudaMemcpy(&i32[0], op->d_error, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        for (const btc_contraction_s *o : {static_cast<const btc_contraction_s *>(op), static_cast<const btc_contraction_s *>(op->real_inner)}) {
+            if (!o || !o->d_error || i32[0] != 0) continue;
+            if (cudaMemcpy(&i32[0], o->d_error, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) {
                 cudaGetLastError();
                 return BTC_ERR_CUDA;
             }
@@ -1027,6 +1148,31 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
         if (misaligned(workspace, 256)) return BTC_ERR_MISALIGNED;
     }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // complex64 through its real form on the fp32 tensor-core kernels: expand the smaller input (alpha and
+    // both conjugations go into it), then run the real contraction over the float views of the other
+    // tensors.  Needs a real beta and C as it is; pointer-array calls keep the complex kernels.
+    if (op->real_inner && !bv && use_ab && be[1] == 0.0 && !(use_c && pl.conjC)) {
+        ComplexExpandParams ep = op->real_expand;
+        ep.src = static_cast<const float2 *>(op->real_expand_A ? A : B);
+        ep.dst = static_cast<float *>(workspace);
+        ep.alpha_r = float(al[0]); ep.alpha_i = float(al[1]);
+        ep.conj_x = (op->real_expand_A ? op->req.conjA : op->req.conjB) ? 1 : 0;
+        ep.conj_y = (op->real_expand_A ? op->req.conjB : op->req.conjA) ? 1 : 0;
+        int64_t blocks = (ep.total + 255) / 256;
+        const int64_t cap = int64_t(op->handle.sm_count) * 16;
+        if (blocks > cap) blocks = cap;
+        complex_expand_kernel<<<unsigned(blocks), 256, 0, st>>>(ep);
+        if (cudaGetLastError() != cudaSuccess) return BTC_ERR_CUDA;
+        const float one = 1.f, beta_r = float(be[0]);
+        const void *pa = op->real_expand_A ? workspace : A, *pb = op->real_expand_A ? B : workspace;
+        btc_contraction_s *in = op->real_inner;
+        in->poll_limit = op->poll_limit;
+        const btc_error_t rc = execute_impl(in, cuda_stream, &one, pa, pb, &beta_r, use_c ? C : nullptr, D,
+                                            static_cast<char *>(workspace) + op->real_x_bytes, workspace_bytes - op->real_x_bytes,
+                                            status, nullptr);
+        if (rc == BTC_SUCCESS && status && *status) (*status)->launches += 1;
+        return rc;
+    }
     int launches = 0;
     int ran_variant = op->plan.kernel == BTC_KERNEL_TILED ? op->plan.tile.variant : -1;
     cudaError_t ce = cudaSuccess;
@@ -1512,9 +1658,11 @@ btc_error_t run_host_pipeline(btc_contraction_s *op, cudaStream_t st, const void
     if (!ok) { cudaGetLastError(); return rc != BTC_SUCCESS ? rc : BTC_ERR_CUDA; }
     if (rc != BTC_SUCCESS) return rc;
     for (int i = 0; i < 2; ++i)
-        if (hp->sub[i] && hp->sub[i]->d_error) {
+        for (const btc_contraction_s *o : {static_cast<const btc_contraction_s *>(hp->sub[i]),
+                                           static_cast<const btc_contraction_s *>(hp->sub[i] ? hp->sub[i]->real_inner : nullptr)}) {
+            if (!o || !o->d_error) continue;
             int32_t word = 0;
-            if (cudaMemcpy(&word, hp->sub[i]->d_error, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return BTC_ERR_CUDA; }
+            if (cudaMemcpy(&word, o->d_error, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return BTC_ERR_CUDA; }
             if (word != 0) return BTC_ERR_DEVICE_TIMEOUT;
         }
     return BTC_SUCCESS;
@@ -1580,9 +1728,10 @@ btc_error_t btc_execute_host(btc_contraction_t op, void *cuda_stream, const void
         cudaMemcpyAsync(static_cast<char *>(D) + bD.lo, bD.dev, bD.bytes(), cudaMemcpyDeviceToHost, st) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
     if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
     // a bounded device-side wait that gave up left D incomplete: say so
-    if (rc == BTC_SUCCESS && op->d_error) {
+    for (const btc_contraction_s *o : {static_cast<const btc_contraction_s *>(op), static_cast<const btc_contraction_s *>(op->real_inner)}) {
+        if (rc != BTC_SUCCESS || !o || !o->d_error) continue;
         int32_t word = 0;
-        if (cudaMemcpy(&word, op->d_error, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
+        if (cudaMemcpy(&word, o->d_error, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); fail(BTC_ERR_CUDA); }
         else if (word != 0) fail(BTC_ERR_DEVICE_TIMEOUT);
     }
     for (Buf *b : {&bA, &bB, &bD}) if (b->dev) cudaFree(b->dev);
