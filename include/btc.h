@@ -23,8 +23,9 @@
  *
  * complex64 operations of at least about 2 GFLOP run as a real fp32 contraction on the tensor cores: the
  * smaller input is first expanded into the workspace (16 bytes per element; counted in
- * btc_contraction_workspace_size), so such an operation needs a workspace even without split-K, and its
- * kernel, variant, tile and grid attributes describe the fp32 contraction that runs.
+ * btc_contraction_workspace_size).  A call whose workspace has no room for that (or none at all, or the
+ * library's static scratch when it is too small) runs the complex kernels instead, with the same result
+ * within the tolerance.  The kernel, variant, tile and grid attributes describe the fp32 contraction.
  *
  * Environment: BTC_LOG (any value) prints every contraction's plan to stderr when it is created,
  * and a note when a problem of more than 1 GFLOP lands on the per-element kernel.

@@ -67,6 +67,7 @@ struct btc_contraction_s {
     bool skinny_regular = false;
     bool skinny_d_regular[2] = {false, false};     // D's rows (m) / columns (n) regular
     size_t workspace_bytes = 0;
+    size_t workspace_floor = 0;   // what the operation needs at least (without the real form of complex64, which is then not used)
     int32_t grid[3] = {0, 0, 0};
     // Case 4: inputs with isolated labels are first summed into the front of the workspace
     // (A' at offset 0, B' behind it), split-K partial sums follow at `partials_offset`
@@ -734,7 +735,7 @@ void build_real_form(btc_contraction_s *op)
     op->real_expand_A = expand_A;
     op->real_expand = ep;
     op->real_x_bytes = (size_t(ep.total) * 16 + 255) / 256 * 256;
-    op->workspace_bytes = std::max(op->workspace_bytes, op->real_x_bytes + in->workspace_bytes);
+    op->workspace_bytes = std::max(op->workspace_floor, op->real_x_bytes + in->workspace_bytes);
 }
 
 int replan(btc_contraction_s *op)
@@ -771,6 +772,7 @@ int replan(btc_contraction_s *op)
     op->sumB_offset = bytesA;
     op->partials_offset = bytesA + bytesB;
     op->workspace_bytes += op->partials_offset;
+    op->workspace_floor = op->workspace_bytes;
     build_real_form(op);
     return BTC_SUCCESS;
 }
@@ -1143,15 +1145,16 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
     if (misaligned(A, need_of(op->req.A.dtype)) || misaligned(B, need_of(op->req.B.dtype)) ||
         misaligned(C, need_of(op->req.has_c ? op->req.C.dtype : pl.dtype)) || misaligned(D, need))
         return BTC_ERR_MISALIGNED;
-    if (op->workspace_bytes > 0 && !bv) {        // a pointer-array batch has checked its own layout
-        if (!workspace || workspace_bytes < op->workspace_bytes) return BTC_ERR_WORKSPACE_TOO_SMALL;
+    if (op->workspace_floor > 0 && !bv) {        // a pointer-array batch has checked its own layout
+        if (!workspace || workspace_bytes < op->workspace_floor) return BTC_ERR_WORKSPACE_TOO_SMALL;
         if (misaligned(workspace, 256)) return BTC_ERR_MISALIGNED;
     }
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     // complex64 through its real form on the fp32 tensor-core kernels: expand the smaller input (alpha and
     // both conjugations go into it), then run the real contraction over the float views of the other
     // tensors.  Needs a real beta and C as it is; pointer-array calls keep the complex kernels.
-    if (op->real_inner && !bv && use_ab && be[1] == 0.0 && !(use_c && pl.conjC)) {
+    if (op->real_inner && !bv && use_ab && be[1] == 0.0 && !(use_c && pl.conjC) && workspace && !misaligned(workspace, 256) &&
+        workspace_bytes >= op->real_x_bytes + op->real_inner->workspace_bytes) {
         ComplexExpandParams ep = op->real_expand;
         ep.src = static_cast<const float2 *>(op->real_expand_A ? A : B);
         ep.dst = static_cast<float *>(workspace);
@@ -1403,7 +1406,7 @@ btc_error_t btc_contraction_batched_workspace_size(btc_contraction_t op, int64_t
 {
     if (!op || !bytes || count < 1) return BTC_ERR_INVALID_ARGUMENT;
     if (!batch_in_one_launch(op)) { *bytes = op->workspace_bytes; return BTC_SUCCESS; }
-    *bytes = batch_tables_bytes(op, count) + (op->workspace_bytes - op->partials_offset) * size_t(count);
+    *bytes = batch_tables_bytes(op, count) + (op->workspace_floor - op->partials_offset) * size_t(count);
     return BTC_SUCCESS;
 }
 
@@ -1755,7 +1758,7 @@ btc_error_t btc_execute_static_scratch(btc_contraction_t op, void *cuda_stream, 
     static std::atomic<void *> scratch_of_device[64] = {};
     if (!op || !D) return BTC_ERR_INVALID_ARGUMENT;
     if (op->handle.device < 0) return BTC_ERR_CUDA;
-    if (op->workspace_bytes > size_t(BTC_STATIC_SCRATCH_BYTES)) return BTC_ERR_SCRATCH_LIMIT;
+    if (op->workspace_floor > size_t(BTC_STATIC_SCRATCH_BYTES)) return BTC_ERR_SCRATCH_LIMIT;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return BTC_ERR_CUDA; }
     // the symbol's address differs per device: the operation's device must be the current one
