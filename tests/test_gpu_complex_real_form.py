@@ -65,3 +65,28 @@ def test_complex64_real_form(api, handle, name):
         rem //= e
     got = dD.buffer.cpu()[torch.from_numpy(pos)].numpy()
     assert helpers.compare(got, vals, scale, dtype) <= 1.0
+
+
+def test_without_room_in_the_workspace_the_complex_kernels_run(api, handle):
+    la, lb, ld, ext = "ki", "kj", "ij", dict(i=2048, j=4096, k=192)     # many tiles: the complex plan itself needs no scratch
+    dtype = torch.complex64
+    A = helpers.random_tensor(21, _ext(la, ext), None, dtype).to("cuda")
+    B = helpers.random_tensor(22, _ext(lb, ext), None, dtype).to("cuda")
+    D1 = helpers.random_tensor(23, _ext(ld, ext), None, dtype).to("cuda")
+    D2 = helpers.random_tensor(23, _ext(ld, ext), None, dtype).to("cuda")
+    dt = api.dtype_code(dtype)
+    info = lambda t: api.TensorInfo(handle, dt, t.extents, t.strides)
+    op = api.Contraction(handle, info(A), la, info(B), lb, None, ld, info(D1), ld, 1.0, 0.0)
+    need = op.workspace_size()
+    assert need > 0 and 10 <= op.variant <= 21          # planned in its real form
+    stream = torch.cuda.current_stream().cuda_stream
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    st1 = op.execute(stream, A.data_ptr(), B.data_ptr(), 0, D1.data_ptr(), workspace=ws.data_ptr(), workspace_bytes=need, want_status=True)
+    st2 = op.execute(stream, A.data_ptr(), B.data_ptr(), 0, D2.data_ptr(), want_status=True)       # no workspace at all
+    torch.cuda.synchronize()
+    assert op.device_error == 0
+    assert 10 <= st1["variant"] <= 21 and not (10 <= st2["variant"] <= 21), (st1, st2)
+    # two different summation schemes of the same contraction: equal within the tolerance's scale
+    a, b = D1.buffer[D1.offsets()], D2.buffer[D2.offsets()]
+    scale = float(ext["k"]) * 1.0
+    assert float((a - b).abs().max()) <= 2e-5 * scale
