@@ -103,8 +103,10 @@ btc_error_t btc_destroy_tensor_info(btc_tensor_info_t *info);
  *               NULL means alpha = 1, beta = 0
  * Element types (Sec. "Challenge: Datatypes"): normally all four tensors share one type.  Real and
  * complex tensors of one part width may be mixed (a real operand counts as complex with zero
- * imaginary parts) as long as D is complex whenever A, B or C is; such operations run on the
- * per-element kernel (exact, not fast).  32- and 64-bit parts cannot be mixed (NOT_SUPPORTED).
+ * imaginary parts) as long as D is complex whenever A, B or C is.  One real and one complex input
+ * with a complex C (or none), real alpha and beta and no conjugation of the complex tensors run on
+ * the tiled kernels (the complex tensors are read as real ones with one more mode); other mixes run
+ * on the per-element kernel (exact, not fast).  32- and 64-bit parts cannot be mixed (NOT_SUPPORTED).
  * All validation and planning (label classes, mode fusion, kernel and tile choice, device-side
  * offset tables) happens here; the call may allocate device memory and copy small tables with
  * the default stream.  Errors: INVALID_ARGUMENT, EXTENT_MISMATCH, C_D_MISMATCH, D_ALIASING,

@@ -85,6 +85,10 @@ struct btc_contraction_s {
     bool real_expand_A = true;              // X is the caller's A (else B)
     ComplexExpandParams real_expand;        // loop dimensions of X in X'' order (pointers and scalars filled at execute)
     size_t real_x_bytes = 0;                // bytes of X'' (rounded up to 256)
+    // One real and one complex input (mixed element types): with the complex tensors read as real tensors
+    // with one more mode (the part, a free label of the complex input and of D) the operation is an
+    // ordinary real contraction, `real_inner` with real_view_only set: nothing is expanded.
+    bool real_view_only = false;
 };
 
 // Host-buffer execution in slabs (btc_execute_host): the larger input is cut along the label with its largest
@@ -643,6 +647,54 @@ void free_real_form(btc_contraction_s *op)
         op->real_inner = nullptr;
     }
     op->real_x_bytes = 0;
+    op->real_view_only = false;
+}
+
+// Mixed element types, one real and one complex input: D = alpha A B with A real is, part by part, the real
+// contraction of A with B read as a real tensor (Eq. (case2) holds for each part).  Needs real scalars and no
+// conjugation of the complex tensors at execute; then the tiled kernels of the part type run instead of
+// the per-element kernel.
+void build_mixed_real_view(btc_contraction_s *op)
+{
+    const PlanRequest &rq = op->req;
+    const Plan &pl = op->plan;
+    if (op->handle.device < 0 || !pl.mixed || rq.force_kernel == BTC_KERNEL_GENERIC) return;
+    const bool ca = dtype_is_complex(rq.A.dtype), cb = dtype_is_complex(rq.B.dtype);
+    if (ca == cb || !dtype_is_complex(rq.D.dtype) || (rq.has_c && rq.C.dtype != rq.D.dtype)) return;
+    if ((ca && rq.conjA) || (cb && rq.conjB)) return;
+    const btc_dtype_t part = rq.D.dtype == BTC_C32 ? BTC_F32 : BTC_F64;
+    int64_t top = 0;
+    for (auto *l : {&rq.labelsA, &rq.labelsB, &rq.labelsC, &rq.labelsD}) for (int64_t x : *l) top = std::max(top, x);
+    if (top > INT64_MAX - 1) return;
+    const int64_t V = top + 1;
+    auto real_view = [&](const TensorDesc &t, const std::vector<int64_t> &labels, TensorDesc &out, std::vector<int64_t> &lout) {
+        out.dtype = part;
+        out.extent.assign(1, 2); out.stride.assign(1, 1); lout.assign(1, V);
+        for (size_t i = 0; i < t.extent.size(); ++i) {
+            out.extent.push_back(t.extent[i]); out.stride.push_back(2 * t.stride[i]); lout.push_back(labels[i]);
+        }
+    };
+    btc_contraction_s *in = new (std::nothrow) btc_contraction_s;
+    if (!in) return;
+    in->handle = op->handle;
+    in->req = rq;                                    // attributes (precision, hints, forced variants) carry over
+    in->req.conjA = in->req.conjB = in->req.conjC = false;
+    if (ca) real_view(rq.A, rq.labelsA, in->req.A, in->req.labelsA); else in->req.A.dtype = part;
+    if (cb) real_view(rq.B, rq.labelsB, in->req.B, in->req.labelsB); else in->req.B.dtype = part;
+    real_view(rq.D, rq.labelsD, in->req.D, in->req.labelsD);
+    if (rq.has_c) real_view(rq.C, rq.labelsC, in->req.C, in->req.labelsC);
+    in->poll_limit = op->poll_limit;
+    in->pre_reduce = op->pre_reduce;
+    in->alpha[0] = op->alpha[0]; in->alpha[1] = 0.0; in->beta[0] = op->beta[0]; in->beta[1] = 0.0;
+    if (replan(in) != BTC_SUCCESS || in->plan.kernel != BTC_KERNEL_TILED) {
+        free_tables(in);
+        delete in;
+        return;
+    }
+    op->real_inner = in;
+    op->real_view_only = true;
+    op->real_x_bytes = 0;
+    op->workspace_bytes = std::max(op->workspace_floor, in->workspace_bytes);
 }
 
 // complex64 -> fp32: set up the real form of the operation (complex_expand_kernel.cuh) when it is worth
@@ -774,6 +826,7 @@ int replan(btc_contraction_s *op)
     op->workspace_bytes += op->partials_offset;
     op->workspace_floor = op->workspace_bytes;
     build_real_form(op);
+    if (!op->real_inner) build_mixed_real_view(op);
     return BTC_SUCCESS;
 }
 
@@ -1153,7 +1206,20 @@ btc_error_t execute_impl(btc_contraction_t op, void *cuda_stream, const void *al
     // complex64 through its real form on the fp32 tensor-core kernels: expand the smaller input (alpha and
     // both conjugations go into it), then run the real contraction over the float views of the other
     // tensors.  Needs a real beta and C as it is; pointer-array calls keep the complex kernels.
-    if (op->real_inner && !bv && use_ab && be[1] == 0.0 && !(use_c && pl.conjC) && workspace && !misaligned(workspace, 256) &&
+    if (op->real_inner && op->real_view_only) {
+        // mixed element types through the real views (build_mixed_real_view): real scalars, C as it is,
+        // and room for the real operation's own scratch; otherwise the per-element kernel below
+        btc_contraction_s *in = op->real_inner;
+        const bool room = in->workspace_floor == 0 || (workspace && !misaligned(workspace, 256) && workspace_bytes >= in->workspace_floor);
+        if (!bv && al[1] == 0.0 && be[1] == 0.0 && !(use_c && op->req.conjC) && room) {
+            in->poll_limit = op->poll_limit;
+            const float af = float(al[0]), bf = float(be[0]);
+            const bool f32 = in->plan.dtype == BTC_F32;
+            return execute_impl(in, cuda_stream, f32 ? static_cast<const void *>(&af) : static_cast<const void *>(&al[0]), A, B,
+                                f32 ? static_cast<const void *>(&bf) : static_cast<const void *>(&be[0]), use_c ? C : nullptr, D,
+                                workspace, workspace_bytes, status, nullptr);
+        }
+    } else if (op->real_inner && !bv && use_ab && be[1] == 0.0 && !(use_c && pl.conjC) && workspace && !misaligned(workspace, 256) &&
         workspace_bytes >= op->real_x_bytes + op->real_inner->workspace_bytes) {
         ComplexExpandParams ep = op->real_expand;
         ep.src = static_cast<const float2 *>(op->real_expand_A ? A : B);

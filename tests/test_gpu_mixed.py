@@ -104,3 +104,35 @@ def test_unsupported_mixes_are_refused():
     with pytest.raises(api.BtcError) as ei:      # a real result of a complex input
         api.Contraction(handle, t(api.C64, (4, 5)), "ik", t(api.F64, (5, 3)), "kj", None, "ij", t(api.F64, (4, 3)), "ij")
     assert ei.value.code == api.ERR_NOT_SUPPORTED
+
+
+REAL_VIEW_SHAPES = {
+    # large enough for a tiled plan of the real contraction
+    "matrix_product": ("ki", "kj", "ij", dict(i=192, j=160, k=96)),
+    "batch_and_permuted_output": ("hik", "kjh", "jih", dict(h=3, i=96, j=80, k=64)),
+    "isolated_label": ("ikx", "kj", "ij", dict(i=128, j=96, k=48, x=3)),
+}
+
+
+@pytest.mark.parametrize("real,cplx", PAIRS)
+@pytest.mark.parametrize("which", ["A", "B"])
+@pytest.mark.parametrize("shape", list(REAL_VIEW_SHAPES))
+def test_one_real_input_runs_the_tiled_kernels_through_real_views(real, cplx, which, shape):
+    """One real and one complex input, real scalars, nothing conjugated: the complex tensors are read as real
+    tensors with one more mode and the tiled kernels of the part type run; with a complex alpha the same
+    operation object falls back to the per-element kernel.  Both against the mixed-type oracle."""
+    api = helpers.api()
+    handle = api.Handle()
+    la, lb, ld, ext = REAL_VIEW_SHAPES[shape]
+    tA, tB = (real if x in which else cplx for x in "AB")
+    A = helpers.random_tensor(221, _ext(la, ext), None, tA)
+    B = helpers.random_tensor(222, _ext(lb, ext), None, tB)
+    C = helpers.random_tensor(223, _ext(ld, ext), None, cplx)
+    D = inputs.place(None, _ext(ld, ext), None, cplx)
+    pos = D.offsets()
+    for alpha, beta, tiled in ((0.75, -0.5, True), (complex(0.75, -1.25), -0.5, False)):
+        got, status, op = _run(api, handle, A, la, B, lb, C, D, ld, alpha, beta)
+        assert (status["kernel"] == api.KERNEL_TILED) == tiled, status
+        want = D.clone()
+        scale = oracle.contract_mixed(A.numpy(), la, B.numpy(), lb, C.numpy(), ld, want.numpy(), ld, alpha, beta)
+        assert helpers.compare(got[pos].numpy(), want.buffer[pos].numpy(), scale, cplx) <= 1.0
