@@ -416,8 +416,10 @@ int finish_plan(btc_contraction_s *op)
         const bool box24 = umma_ok && make_tma_operand(pl, 128, 24, probe), box32 = umma_ok && make_tma_operand(pl, 128, 32, probe);
         // (weights from the batched permuted workload: 21, two sub-stages of 24 k per hand-off, is 2 % ahead of
         // the gathering variant 13, the single-sub-stage ones 17-20 a little behind their twins 13 / 14)
-        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 2.6}, {14, 2.3}, {13, 2.0},
-                             {box24 ? 17 : 13, 1.85}, {box32 ? 18 : 13, 1.95}, {box32 ? 19 : 14, 2.25}, {box24 ? 20 : 14, 2.1},
+        // (measured on 4096 x 4096 x 2048 fp32 in three operand layouts: 19: 222-224 TFLOP/s, 14: 206-214, 16: 188-196,
+        // 11: 182-185, 12: 152-154; the 128 x 256 tile with both operands in shared memory stays behind)
+        const Cand f32c[] = {{6, 1.0}, {8, 1.0}, {9, 0.93}, {7, 0.75}, {12, 1.7}, {14, 2.3}, {13, 2.0},
+                             {box24 ? 17 : 13, 1.85}, {box32 ? 18 : 13, 1.95}, {box32 ? 19 : 14, box32 ? 2.45 : 2.3}, {box24 ? 20 : 14, 2.1},
                              {box24 ? 21 : 13, 2.04}};
         const Cand f32strict[] = {{0, 1.0}, {2, 1.0}, {1, 0.75}};   // FFMA kernels: 128x128, 256x96, 64x64
         const Cand f64c[] = {{2, 1.0}, {1, 0.75}};       // big tile: the m16n8k16 variant
