@@ -410,7 +410,12 @@ int finish_plan(btc_contraction_s *op)
         // enter only when there is enough work to fill the SMs without split-K; their weights
         // reflect measured throughput relative to the mma.sync variants.
         const double flops = 2.0 * double(pl.M) * double(pl.N) * double(pl.K) * double(pl.Bt);
-        const bool umma_ok = pl.dtype == BTC_F32 && flops * double(hint) >= 2e9 && pl.K >= 64;
+        // (measured against the mma.sync variants with their split-K: ahead from about 0.6 GFLOP on when 128 x 128
+        // tiles fill at least 64 SMs -- 1024 x 1024 x 512: 25 against 31 us, 4096 x 512 x 256: 19 against 47 us --
+        // and on a par at 512^3)
+        const double tiles128 = double((pl.M + 127) / 128) * double((pl.N + 127) / 128) * double(pl.Bt) * double(hint);
+        const bool umma_ok = pl.dtype == BTC_F32 && pl.K >= 64 &&
+                             (flops * double(hint) >= 2e9 || (flops * double(hint) >= 0.6e9 && tiles128 >= 64.0));
         // 17-20 fetch the M side with bulk tensor copies; they enter when that operand is a tensor of boxes
         TmaOperand probe;
         const bool box24 = umma_ok && make_tma_operand(pl, 128, 24, probe), box32 = umma_ok && make_tma_operand(pl, 128, 32, probe);
