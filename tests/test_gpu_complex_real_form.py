@@ -36,13 +36,21 @@ CASES = {
 }
 
 
+# strides (elements) per tensor for the cases that are not dense column-major: padding, a reversed mode
+STRIDES = {
+    "padded_and_reversed": ((-1, 330), (1, 336), (264, -1)),
+}
+CASES["padded_and_reversed"] = ("ki", "kj", "ji", dict(i=256, j=2048, k=320), True, False, 0.5 + 0.5j, -0.25, True)
+
+
 @pytest.mark.parametrize("name", list(CASES))
 def test_complex64_real_form(api, handle, name):
     la, lb, ld, ext, conjA, conjB, alpha, beta, real_form = CASES[name]
     dtype = torch.complex64
-    A = helpers.random_tensor(11, _ext(la, ext), None, dtype)
-    B = helpers.random_tensor(12, _ext(lb, ext), None, dtype)
-    D = helpers.random_tensor(13, _ext(ld, ext), None, dtype)
+    sA, sB, sD = STRIDES.get(name, (None, None, None))
+    A = helpers.random_tensor(11, _ext(la, ext), sA, dtype)
+    B = helpers.random_tensor(12, _ext(lb, ext), sB, dtype)
+    D = helpers.random_tensor(13, _ext(ld, ext), sD, dtype)
     use_c = beta != 0.0
     dA, dB, dD = A.to("cuda"), B.to("cuda"), D.to("cuda")
     op, status = api.contract(handle, dA, la, dB, lb, dD if use_c else None, dD, ld, alpha, beta, conjA, conjB, False,
@@ -65,6 +73,7 @@ def test_complex64_real_form(api, handle, name):
         rem //= e
     got = dD.buffer.cpu()[torch.from_numpy(pos)].numpy()
     assert helpers.compare(got, vals, scale, dtype) <= 1.0
+    assert helpers.canary_intact(D.buffer, dD.buffer.cpu(), D.offsets()), "bytes outside D's elements were modified"
 
 
 def test_without_room_in_the_workspace_the_complex_kernels_run(api, handle):
