@@ -309,6 +309,45 @@ __global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise
             tile[0][ty + ROWS1 * r][tx] = v_r[r];
             if (CPLX) tile[NC - 1][ty + ROWS1 * r][tx] = p.conjA ? -v_i[r] : v_i[r];
         }
+    } else if (p.ns == 1 && p.use_a) {
+        // One summed dimension (the usual case after chained dimensions are merged): a running pointer per
+        // row instead of an index decode per element, eight loads in flight, whole groups of eight without
+        // bounds tests (an element costs a load, a conversion and an add: the loop is issue-bound otherwise).
+        const R *A = static_cast<const R *>(p.A);
+        const int64_t step = NC * p.sA_s[0];
+        const bool a_in = a0 + tx < ext_a;
+        const R *row0 = A + NC * (restA + (a0 + tx) * p.sA_k[ma] + (c0 + ty) * p.sA_k[0]);
+        const int64_t rstep = NC * ROWS1 * p.sA_k[0];
+        const int rows_in = int(ext_c - c0 - ty < int64_t(TC) ? ext_c - c0 - ty : int64_t(TC));   // rows ty + ROWS1 r < rows_in exist
+#pragma unroll 1
+        for (int r = 0; r < PER1; ++r) {
+            double acc_r = 0.0, acc_i = 0.0;
+            if (a_in && ROWS1 * r < rows_in) {
+                const R *q = row0 + r * rstep;
+                int64_t left = p.total_sum;
+                for (; left >= 8; left -= 8) {
+                    R v_r[8], v_i[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        v_r[u] = q[u * step];
+                        v_i[u] = CPLX ? q[u * step + (NC - 1)] : R(0);
+                    }
+                    q += 8 * step;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        acc_r += double(v_r[u]);
+                        if (CPLX) acc_i += double(v_i[u]);
+                    }
+                }
+                for (; left > 0; --left) {
+                    acc_r += double(q[0]);
+                    if (CPLX) acc_i += double(q[NC - 1]);
+                    q += step;
+                }
+            }
+            tile[0][ty + ROWS1 * r][tx] = R(acc_r);
+            if (CPLX) tile[NC - 1][ty + ROWS1 * r][tx] = R(p.conjA ? -acc_i : acc_i);   // conjugation commutes with the sum
+        }
     } else {
 #pragma unroll
         for (int r = 0; r < PER1; ++r) {
