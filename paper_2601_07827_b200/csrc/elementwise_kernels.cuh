@@ -66,6 +66,31 @@ __device__ __forceinline__ void elementwise_sum(const ElementwiseParams &p, int6
             acc_r = double(A[NC * base]);
             if (CPLX) acc_i = double(A[NC * base + (NC - 1)]);
         }
+    } else if (p.ns == 1) {
+        // one summed dimension: a running pointer, whole groups of U loads without bounds tests
+        const int64_t step = NC * LANES * p.sA_s[0];
+        const R *q = A + NC * (base + lane * p.sA_s[0]);
+        int64_t left = (p.total_sum - lane + LANES - 1) / LANES;      // this lane's share of the summed index
+        if (left < 0) left = 0;
+        for (; left >= U; left -= U) {
+            R v_r[U], v_i[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                v_r[u] = q[u * step];
+                v_i[u] = CPLX ? q[u * step + (NC - 1)] : R(0);
+            }
+            q += U * step;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                acc_r += double(v_r[u]);
+                if (CPLX) acc_i += double(v_i[u]);
+            }
+        }
+        for (; left > 0; --left) {
+            acc_r += double(q[0]);
+            if (CPLX) acc_i += double(q[NC - 1]);
+            q += step;
+        }
     } else {
         for (int64_t s0 = lane; s0 < p.total_sum; s0 += int64_t(U) * LANES) {
             R v_r[U], v_i[U];
@@ -73,8 +98,7 @@ __device__ __forceinline__ void elementwise_sum(const ElementwiseParams &p, int6
             for (int u = 0; u < U; ++u) {
                 const int64_t s = s0 + int64_t(u) * LANES;
                 const bool in = s < p.total_sum;
-                // one summed dimension: its index times its stride, no decoding
-                const int64_t off = base + (in ? (p.ns == 1 ? s * p.sA_s[0] : decode_offset<I>(I(s), p.ns, p.ext_s, p.sA_s)) : 0);
+                const int64_t off = base + (in ? decode_offset<I>(I(s), p.ns, p.ext_s, p.sA_s) : 0);
                 v_r[u] = in ? A[NC * off] : R(0);
                 v_i[u] = (CPLX && in) ? A[NC * off + (NC - 1)] : R(0);
             }
