@@ -54,6 +54,35 @@ __global__ void __launch_bounds__(256) isolated_sum_kernel(const IsolatedSumPara
             base[j] = live[j] ? decode_offset<I>(I(e), p.nk, p.ext_k, p.str_k) : 0;
             acc_r[j] = acc_i[j] = 0.0;
         }
+        if (LANES == 1 && p.ni == 1) {
+            // one isolated dimension, one result element per thread: a running pointer and whole groups of
+            // eight loads without bounds tests (the general loop below is bound by instruction issue for
+            // 4-byte elements: an index decode and a test per load)
+            if (live[0]) {
+                const int64_t step = NC * p.str_i[0];
+                const R *q = src + NC * base[0];
+                int64_t left = p.total_iso;
+                for (; left >= 8; left -= 8) {
+                    R w_r[8], w_i[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        w_r[u] = q[u * step];
+                        w_i[u] = CPLX ? q[u * step + (NC - 1)] : R(0);
+                    }
+                    q += 8 * step;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        acc_r[0] += double(w_r[u]);
+                        if (CPLX) acc_i[0] += double(w_i[u]);
+                    }
+                }
+                for (; left > 0; --left) {
+                    acc_r[0] += double(q[0]);
+                    if (CPLX) acc_i[0] += double(q[NC - 1]);
+                    q += step;
+                }
+            }
+        } else
         for (int64_t s0 = lane; s0 < p.total_iso; s0 += int64_t(U) * LANES) {
             R v_r[E][U], v_i[E][U];
 #pragma unroll
