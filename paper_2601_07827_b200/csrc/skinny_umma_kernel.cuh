@@ -274,6 +274,12 @@ struct SkinnyStore {
             if (lean) {
                 // whole tile, regular columns, no C: nothing to decide per store
                 float *base = D + (ro + co[0]);
+                if (alpha == 1.f) {                  // the accumulator registers go out as they are
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        *reinterpret_cast<uint4 *>(base + p.skinny_col_rel[c0 + 4 * q]) = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+                    continue;
+                }
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
                     *reinterpret_cast<float4 *>(base + p.skinny_col_rel[c0 + 4 * q]) =
