@@ -1955,18 +1955,20 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const bool narrow = pl.total_keep < (int64_t(1) << 31) && pl.total_sum < (int64_t(1) << 31);
     const bool transposing = pl.kernel == ElementwiseKernel::TRANSPOSING && use_a;
+#define BTC_EW_TRANSPOSE(R, CPLX, I, SUMS, WHEN, FLAGS)                                                            \
+    if (WHEN) {                                                                                                    \
+        if (set_smem_once(elementwise_transposing_kernel<R, CPLX, I, SUMS>, TT::SMEM_BYTES, FLAGS) != cudaSuccess) return BTC_ERR_CUDA; \
+        elementwise_transposing_kernel<R, CPLX, I, SUMS><<<unsigned(blocks), TT::THREADS, TT::SMEM_BYTES, st>>>(p); \
+    }
 #define BTC_EW_LAUNCH(R, CPLX)                                                                                     \
     do {                                                                                                           \
         if (transposing) {                                                                                         \
             typedef TransposeTile<R, CPLX> TT;                                                                     \
-            static std::atomic<bool> configured[64] = {}, configured_wide[64] = {};                                             \
-            if (narrow) {                                                                                          \
-                if (set_smem_once(elementwise_transposing_kernel<R, CPLX, uint32_t>, TT::SMEM_BYTES, configured) != cudaSuccess) return BTC_ERR_CUDA; \
-                elementwise_transposing_kernel<R, CPLX, uint32_t><<<unsigned(blocks), TT::THREADS, TT::SMEM_BYTES, st>>>(p); \
-            } else {                                                                                               \
-                if (set_smem_once(elementwise_transposing_kernel<R, CPLX, int64_t>, TT::SMEM_BYTES, configured_wide) != cudaSuccess) return BTC_ERR_CUDA; \
-                elementwise_transposing_kernel<R, CPLX, int64_t><<<unsigned(blocks), TT::THREADS, TT::SMEM_BYTES, st>>>(p); \
-            }                                                                                                      \
+            static std::atomic<bool> configured[4][64] = {};                                                       \
+            BTC_EW_TRANSPOSE(R, CPLX, uint32_t, false, narrow && p.ns == 0, configured[0]);                        \
+            BTC_EW_TRANSPOSE(R, CPLX, uint32_t, true, narrow && p.ns != 0, configured[1]);                         \
+            BTC_EW_TRANSPOSE(R, CPLX, int64_t, false, !narrow && p.ns == 0, configured[2]);                        \
+            BTC_EW_TRANSPOSE(R, CPLX, int64_t, true, !narrow && p.ns != 0, configured[3]);                         \
         } else if (lanes == 32) {                                                                                  \
             if (narrow) elementwise_direct_kernel<R, CPLX, 32, uint32_t><<<unsigned(blocks), 256, 0, st>>>(p);      \
             else elementwise_direct_kernel<R, CPLX, 32, int64_t><<<unsigned(blocks), 256, 0, st>>>(p);              \
@@ -2032,6 +2034,7 @@ btc_error_t btc_elementwise_execute(btc_elementwise_t op, void *cuda_stream, con
     default: BTC_EW_LAUNCH(double, true); break;
     }
 #undef BTC_EW_LAUNCH
+#undef BTC_EW_TRANSPOSE
     return cudaGetLastError() == cudaSuccess ? BTC_SUCCESS : BTC_ERR_CUDA;
 }
 

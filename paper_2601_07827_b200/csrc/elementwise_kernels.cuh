@@ -281,7 +281,9 @@ template <typename R, bool CPLX> struct TransposeTile {
 // blockIdx.x enumerates (tile along C's dimension 0, tile along A's dimension, rest), first fastest.
 // Each thread handles TC * TA / THREADS elements in either phase; the tile holds values already
 // summed and rounded to the element type.
-template <typename R, bool CPLX, typename I>
+// SUMS: compiled with the branches for summed dimensions (and for alpha = 0); the pure permutation
+// is a kernel of its own, so that it keeps its register count and occupancy.
+template <typename R, bool CPLX, typename I, bool SUMS>
 __global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise_transposing_kernel(const ElementwiseParams p)
 {
     constexpr int NC = CPLX ? 2 : 1;
@@ -314,7 +316,7 @@ __global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise
     // inside the bounds test of its own iteration would leave one load in flight per thread.
     {
     const int tx = threadIdx.x % TA, ty = threadIdx.x / TA;
-    if (p.ns == 0 && p.use_a) {
+    if (!SUMS) {
         const R *A = static_cast<const R *>(p.A);
         R v_r[PER1], v_i[PER1];
         const bool a_in = a0 + tx < ext_a;
@@ -333,7 +335,7 @@ __global__ void __launch_bounds__((TransposeTile<R, CPLX>::THREADS)) elementwise
             tile[0][ty + ROWS1 * r][tx] = v_r[r];
             if (CPLX) tile[NC - 1][ty + ROWS1 * r][tx] = p.conjA ? -v_i[r] : v_i[r];
         }
-    } else if (p.ns == 1 && p.use_a) {
+    } else if (SUMS && p.ns == 1 && p.use_a) {
         // One summed dimension (the usual case after chained dimensions are merged): a running pointer per
         // row instead of an index decode per element, eight loads in flight, whole groups of eight without
         // bounds tests (an element costs a load, a conversion and an add: the loop is issue-bound otherwise).
